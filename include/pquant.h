@@ -1,0 +1,157 @@
+/*
+ * pquant.h -- C ABI of the B200 (sm_100a) pQuant decoupled linear layer.
+ *
+ * The layer (paper Sec. 3.1-3.3) replaces a projection Y = W X by
+ *
+ *     Y[t,n] = alpha_n * g_t * (B_e A_e x_t)[n]  +  beta_n * (lam / gamma_t) * sum_k S[n,k] q[t,k]
+ *
+ * with S = Sign(W - mu) (Eq. 3-4), mu = mean W, lam = mean |W| (Eq. 6),
+ * q = RoundClip(x * gamma_t) in int8 with gamma_t = 2^7 / max_k |x_tk| (Eq. 7-9),
+ * the 1-bit product de-quantised by lam / gamma_t (Eq. 10), the two branches
+ * summed under the feature scales alpha, beta (Eq. 11), and the high-precision
+ * (HP) branch A_e (r x K), B_e (N x r) chosen per token by a top-1 softmax
+ * router, e = argmax_j (Wr x_t)_j, g_t = softmax(Wr x_t)_e (Sec. 3.3).
+ * The backward pass is the straight-through estimator of App. B.1.
+ *
+ * Conventions common to every entry point
+ *   - every data pointer is a DEVICE pointer owned by the caller; the library
+ *     never allocates, frees or keeps device memory between calls;
+ *   - work is only enqueued on `stream` (a cudaStream_t passed as void*); no
+ *     call synchronises the device;
+ *   - the return value is a status: PQ_OK (0) or a negative PQ_ERR_* code.
+ *     Nothing is thrown.  After an error the outputs are undefined;
+ *   - matrices are dense row-major: X[T,K] bf16, latent W[N,K] fp32,
+ *     A[E,r,K] bf16, B[E,N,r] bf16, Wr[E,K] bf16, Y[T,N] bf16.  bf16 is passed
+ *     as uint16_t bit patterns.  All base pointers must be 16-byte aligned;
+ *   - alpha / beta hold one float (the paper's scalars) or N floats when
+ *     PQ_SCALE_VECTOR is set in pq_desc.flags;
+ *   - kernels wait on hardware barriers with a bounded spin; if a wait runs
+ *     out the kernel records a code in a device status word that
+ *     pq_device_status() reads back (PQ_ERR_TIMEOUT).
+ */
+#ifndef PQUANT_H_
+#define PQUANT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  PQ_OK = 0,
+  PQ_ERR_NULL = -1,        /* a required pointer is NULL                        */
+  PQ_ERR_SHAPE = -2,       /* a size violates the documented constraints        */
+  PQ_ERR_ALIGN = -3,       /* a pointer is not 16-byte aligned                  */
+  PQ_ERR_WORKSPACE = -4,   /* workspace / saved buffer too small                */
+  PQ_ERR_UNSUPPORTED = -5, /* valid request this build does not implement       */
+  PQ_ERR_CUDA = -6,        /* a CUDA runtime / driver call failed               */
+  PQ_ERR_TIMEOUT = -7      /* a device-side bounded wait ran out                */
+};
+
+enum { PQ_SCALE_VECTOR = 1u }; /* pq_desc.flags: alpha, beta have N entries instead of 1 */
+
+enum { PQ_PHASE_PACK = 0, PQ_PHASE_FWD = 1, PQ_PHASE_BWD = 2, PQ_PHASE_DECODE = 3 };
+
+/* Shape of one layer.  Constraints: T >= 1; K, N multiples of 32 (bit words,
+ * 16-byte rows); r == 0 (pure 1-bit layer, the paper's attention projections,
+ * E ignored) or r a multiple of 8 with 8 <= r <= 256 and 1 <= E <= 16;
+ * top_k must be 1 (the paper's gating).  The training path additionally needs
+ * r <= 128. */
+typedef struct pq_desc {
+  uint32_t size;  /* sizeof(pq_desc), checked */
+  uint32_t flags;
+  int32_t T, K, N;
+  int32_t r, E, top_k;
+} pq_desc;
+
+/* Host-side view into the caller-allocated `saved` buffer that the training
+ * forward fills and the backward reads (filled by pq_saved_view; all device
+ * pointers into that buffer).  "sorted order": row p holds token perm[p];
+ * tokens are sorted by expert, stably (the permutation implied by Sec. 3.3's
+ * sparse activation).  With E <= 1 the permutation is the identity. */
+typedef struct pq_saved_view {
+  int8_t* q;          /* [T,K]  int8 activations, sorted order (Eq. 7)                 */
+  uint16_t* xt;       /* [T,K]  bf16 q/gamma, sorted order (backward operand)          */
+  uint16_t* xs;       /* [T,K]  bf16 copy of X in sorted order; NULL when E <= 1       */
+  float* gamma;       /* [T]    gamma_t, sorted order (Eq. 9)                          */
+  float* gate;        /* [T]    g_t, sorted order                                      */
+  float* probs;       /* [T,E]  router softmax, sorted order; NULL when E <= 1         */
+  int32_t* expert;    /* [T]    e_t, TOKEN order                                       */
+  int32_t* perm;      /* [T]    perm[p] = token at sorted position p                   */
+  int32_t* pos;       /* [T]    inverse: pos[token] = p                                */
+  int32_t* offsets;   /* [E+1]  sorted positions of expert e: offsets[e]..offsets[e+1] */
+  uint16_t* h;        /* [max_items*128, r] bf16 HP hidden activations, one 128-row block per item */
+  /* Item table.  An item is the intersection of one 128-row tile of the sorted
+   * order with one expert's range; rows of an item's block outside that range
+   * are zero.  items[i] = {tile, expert, first row, end row} (rows relative to
+   * the tile).  Items are ordered by tile, hence by expert. */
+  int32_t* n_items;            /* [1]                                          */
+  int32_t* items;              /* [max_items][4]                               */
+  int32_t* tile_item_begin;    /* [ceil(T/128)+1] first item of each tile      */
+  int32_t* expert_item_begin;  /* [E+1] first item of each expert              */
+  int32_t max_items;           /* ceil(T/128) + max(E,1) - 1                   */
+} pq_saved_view;
+
+/* Bytes the caller must provide. */
+size_t pq_workspace_bytes(const pq_desc* d, int phase);
+size_t pq_saved_bytes(const pq_desc* d);
+int pq_saved_view_init(const pq_desc* d, void* saved, pq_saved_view* out);
+
+/* Offline / per-step weight quantisation (Eq. 3, 4, 6; storage App. A).
+ *   W        [N,K] fp32 latent weights (in)
+ *   w_bits   [N,K/32] uint32 (out): bit j of word i of a row <-> k = 32 i + j, 1 <-> +1
+ *            (as bytes: the paper's 8 weights per uint8, LSB first)
+ *   w_s8     [N,K] int8 +-1 (out), may be NULL for an inference-only pack
+ *   w_scales [2] float (out) = { lam, mu }, fp64-accumulated, rounded once
+ *   ws       workspace of pq_workspace_bytes(d, PQ_PHASE_PACK) bytes
+ * Only d->N and d->K are read. */
+int pq_pack_weights(const pq_desc* d, const float* W, uint32_t* w_bits, int8_t* w_s8,
+                    float* w_scales, void* ws, size_t ws_bytes, void* stream);
+
+/* Forward of the layer (Eq. 10-11, Sec. 3.3).
+ *   training (w_s8 != NULL): tensor-core path; fills `saved` (may be NULL when
+ *     no backward follows).  A, B may be NULL iff r == 0; Wr NULL iff E <= 1.
+ *   decode (w_s8 == NULL): small-T path straight from the packed bits
+ *     (T <= 16), nothing is saved. */
+int pq_linear_forward(const pq_desc* d, const uint16_t* X, const uint32_t* w_bits,
+                      const int8_t* w_s8, const float* w_scales, const uint16_t* A,
+                      const uint16_t* B, const uint16_t* Wr, const float* alpha,
+                      const float* beta, uint16_t* Y, void* saved, size_t saved_bytes, void* ws,
+                      size_t ws_bytes, void* stream);
+
+/* Straight-through backward (App. B.1): Sign, Round and Clip pass the gradient
+ * unchanged; mu, lam, gamma are constants.  Every gradient is OVERWRITTEN.
+ *   dY [T,N] bf16 (in);  dX [T,K] bf16;  dW [N,K] fp32 (w.r.t. the latent W);
+ *   dA [E,r,K], dB [E,N,r], dWr [E,K] fp32;  dalpha, dbeta fp32 with the same
+ *   length as alpha, beta.  dA/dB/dalpha may be NULL iff r == 0; dWr iff E <= 1. */
+int pq_linear_backward(const pq_desc* d, const uint16_t* dY, const uint16_t* X,
+                       const int8_t* w_s8, const float* w_scales, const uint16_t* A,
+                       const uint16_t* B, const uint16_t* Wr, const float* alpha,
+                       const float* beta, const void* saved, size_t saved_bytes, uint16_t* dX,
+                       float* dW, float* dA, float* dB, float* dWr, float* dalpha, float* dbeta,
+                       void* ws, size_t ws_bytes, void* stream);
+
+/* Test hook for the tensor-core engine: D[M,N] = A . B^T-style contraction with
+ * raw accumulators written out (int32 for mode 0, fp32 otherwise), so that the
+ * integer 1-bit product (Eq. 10) can be checked bit for bit.
+ *   mode 0: int8,  A[M,K] and B[N,K] both K-contiguous
+ *   mode 1: bf16,  A[M,K], B[N,K] both K-contiguous
+ *   mode 2: bf16,  A[M,K] K-contiguous, B[K,N] N-contiguous
+ *   mode 3: bf16,  A[K,M] M-contiguous, B[K,N] N-contiguous
+ * M, N, K multiples of 8 (bf16) / 16 (int8). */
+int pq_debug_gemm(int mode, int M, int N, int K, const void* A, const void* B, void* D,
+                  void* stream);
+
+/* Reads the device status word written by a kernel whose bounded wait ran out.
+ * Synchronises `stream`.  code = 0 when no wait failed; `where` identifies the
+ * waiting role.  The word is cleared by the call. */
+int pq_device_status(void* stream, int* code, int* where);
+
+const char* pq_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PQUANT_H_ */

@@ -1,0 +1,169 @@
+"""ctypes binding of libpquant.so: the C entry points under their own names.
+
+Argument marshalling only -- torch tensors are turned into device pointers and
+the current CUDA stream is passed along; every step of the layer runs in the
+library's kernels.  A missing library is an error (there is no fallback).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libpquant.so")
+
+PQ_OK = 0
+PQ_ERR_NULL, PQ_ERR_SHAPE, PQ_ERR_ALIGN, PQ_ERR_WORKSPACE = -1, -2, -3, -4
+PQ_ERR_UNSUPPORTED, PQ_ERR_CUDA, PQ_ERR_TIMEOUT = -5, -6, -7
+PQ_SCALE_VECTOR = 1
+PQ_PHASE_PACK, PQ_PHASE_FWD, PQ_PHASE_BWD, PQ_PHASE_DECODE = 0, 1, 2, 3
+
+EXPORTS = ("pq_status_string", "pq_workspace_bytes", "pq_saved_bytes", "pq_saved_view_init",
+           "pq_pack_weights", "pq_linear_forward", "pq_linear_backward", "pq_debug_gemm",
+           "pq_device_status")
+
+
+class PqError(RuntimeError):
+    def __init__(self, fn: str, status: int):
+        self.status = status
+        super().__init__(f"{fn} failed: {status} ({pq_status_string(status)})")
+
+
+class pq_desc(ctypes.Structure):
+    _fields_ = [("size", ctypes.c_uint32), ("flags", ctypes.c_uint32),
+                ("T", ctypes.c_int32), ("K", ctypes.c_int32), ("N", ctypes.c_int32),
+                ("r", ctypes.c_int32), ("E", ctypes.c_int32), ("top_k", ctypes.c_int32)]
+
+
+class pq_saved_view(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in
+                ("q", "xt", "xs", "gamma", "gate", "probs", "expert", "perm", "pos", "offsets", "h",
+                 "n_items", "items", "tile_item_begin", "expert_item_begin")] + [("max_items", ctypes.c_int32)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Open libpquant.so (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run __graft_entry__.build() (nvcc, sm_100a) first")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, sz, ci = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int
+        dp = ctypes.POINTER(pq_desc)
+        L.pq_status_string.restype = ctypes.c_char_p
+        L.pq_status_string.argtypes = [ci]
+        L.pq_workspace_bytes.restype = sz
+        L.pq_workspace_bytes.argtypes = [dp, ci]
+        L.pq_saved_bytes.restype = sz
+        L.pq_saved_bytes.argtypes = [dp]
+        L.pq_saved_view_init.restype = ci
+        L.pq_saved_view_init.argtypes = [dp, vp, ctypes.POINTER(pq_saved_view)]
+        L.pq_pack_weights.restype = ci
+        L.pq_pack_weights.argtypes = [dp, vp, vp, vp, vp, vp, sz, vp]
+        L.pq_linear_forward.restype = ci
+        L.pq_linear_forward.argtypes = [dp] + [vp] * 10 + [vp, sz, vp, sz, vp]
+        L.pq_linear_backward.restype = ci
+        L.pq_linear_backward.argtypes = [dp] + [vp] * 9 + [vp, sz] + [vp] * 7 + [vp, sz, vp]
+        L.pq_debug_gemm.restype = ci
+        L.pq_debug_gemm.argtypes = [ci, ci, ci, ci, vp, vp, vp, vp]
+        L.pq_device_status.restype = ci
+        L.pq_device_status.argtypes = [vp, ctypes.POINTER(ci), ctypes.POINTER(ci)]
+        _lib = L
+    return _lib
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _nbytes(t):
+    return 0 if t is None else t.numel() * t.element_size()
+
+
+def _stream(stream):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _check(fn, status):
+    if status != PQ_OK:
+        raise PqError(fn, status)
+
+
+def make_desc(T, K, N, r=0, E=0, top_k=1, scale_vector=False) -> pq_desc:
+    return pq_desc(ctypes.sizeof(pq_desc), PQ_SCALE_VECTOR if scale_vector else 0, T, K, N, r, E, top_k)
+
+
+def pq_status_string(status: int) -> str:
+    return lib().pq_status_string(status).decode()
+
+
+def pq_workspace_bytes(d: pq_desc, phase: int) -> int:
+    return lib().pq_workspace_bytes(ctypes.byref(d), phase)
+
+
+def pq_saved_bytes(d: pq_desc) -> int:
+    return lib().pq_saved_bytes(ctypes.byref(d))
+
+
+def pq_saved_view_init(d: pq_desc, saved: torch.Tensor) -> dict:
+    """Typed torch views into the `saved` byte buffer, keyed like the C struct."""
+    v = pq_saved_view()
+    _check("pq_saved_view_init", lib().pq_saved_view_init(ctypes.byref(d), _ptr(saved), ctypes.byref(v)))
+    base = saved.data_ptr()
+    E = max(d.E, 1) if d.r > 0 else 1
+    mt = (d.T + 127) // 128
+
+    def view(ptr, dtype, *shape):
+        if not ptr:
+            return None
+        n = 1
+        for s in shape:
+            n *= s
+        nbytes = n * torch.empty(0, dtype=dtype).element_size()
+        return saved[ptr - base: ptr - base + nbytes].view(dtype).view(*shape)
+
+    return dict(
+        q=view(v.q, torch.int8, d.T, d.K), xt=view(v.xt, torch.bfloat16, d.T, d.K),
+        xs=view(v.xs, torch.bfloat16, d.T, d.K), gamma=view(v.gamma, torch.float32, d.T),
+        gate=view(v.gate, torch.float32, d.T), probs=view(v.probs, torch.float32, d.T, E),
+        expert=view(v.expert, torch.int32, d.T), perm=view(v.perm, torch.int32, d.T),
+        pos=view(v.pos, torch.int32, d.T), offsets=view(v.offsets, torch.int32, E + 1),
+        h=view(v.h, torch.bfloat16, v.max_items * 128, d.r) if d.r > 0 else None,
+        n_items=view(v.n_items, torch.int32, 1), items=view(v.items, torch.int32, v.max_items, 4),
+        tile_item_begin=view(v.tile_item_begin, torch.int32, mt + 1),
+        expert_item_begin=view(v.expert_item_begin, torch.int32, E + 1), max_items=v.max_items)
+
+
+def pq_pack_weights(d, W, w_bits, w_s8, w_scales, ws, stream=None):
+    _check("pq_pack_weights", lib().pq_pack_weights(ctypes.byref(d), _ptr(W), _ptr(w_bits), _ptr(w_s8), _ptr(w_scales),
+                                                     _ptr(ws), _nbytes(ws), _stream(stream)))
+
+
+def pq_linear_forward(d, X, w_bits, w_s8, w_scales, A, B, Wr, alpha, beta, Y, saved, ws, stream=None):
+    _check("pq_linear_forward", lib().pq_linear_forward(
+        ctypes.byref(d), _ptr(X), _ptr(w_bits), _ptr(w_s8), _ptr(w_scales), _ptr(A), _ptr(B), _ptr(Wr), _ptr(alpha),
+        _ptr(beta), _ptr(Y), _ptr(saved), _nbytes(saved), _ptr(ws), _nbytes(ws), _stream(stream)))
+
+
+def pq_linear_backward(d, dY, X, w_s8, w_scales, A, B, Wr, alpha, beta, saved, dX, dW, dA, dB, dWr, dalpha, dbeta, ws,
+                       stream=None):
+    _check("pq_linear_backward", lib().pq_linear_backward(
+        ctypes.byref(d), _ptr(dY), _ptr(X), _ptr(w_s8), _ptr(w_scales), _ptr(A), _ptr(B), _ptr(Wr), _ptr(alpha), _ptr(beta),
+        _ptr(saved), _nbytes(saved), _ptr(dX), _ptr(dW), _ptr(dA), _ptr(dB), _ptr(dWr), _ptr(dalpha), _ptr(dbeta),
+        _ptr(ws), _nbytes(ws), _stream(stream)))
+
+
+def pq_debug_gemm(mode, M, N, K, A, B, D, stream=None):
+    _check("pq_debug_gemm", lib().pq_debug_gemm(mode, M, N, K, _ptr(A), _ptr(B), _ptr(D), _stream(stream)))
+
+
+def pq_device_status(stream=None) -> tuple[int, int]:
+    code, where = ctypes.c_int(0), ctypes.c_int(0)
+    _check("pq_device_status", lib().pq_device_status(_stream(stream), ctypes.byref(code), ctypes.byref(where)))
+    return code.value, where.value

@@ -1,0 +1,245 @@
+// C ABI of the pQuant layer: argument checks, carving of the caller's saved /
+// workspace buffers, launch sequencing.  No device allocation, no device
+// synchronisation (except pq_device_status, which says so).
+#include <cstring>
+
+#include "pq_kernels.cuh"
+
+namespace pq {
+
+static inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+
+struct Carver {
+  uint8_t* base;
+  size_t off = 0;
+  explicit Carver(void* b) : base(static_cast<uint8_t*>(b)) {}
+  template <class T>
+  T* take(size_t count) {
+    T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+    off += align_up(count * sizeof(T));
+    return p;
+  }
+};
+
+static inline int mtiles_of(const pq_desc* d) { return (d->T + kTileRows - 1) / kTileRows; }
+static inline int experts_of(const pq_desc* d) { return d->r > 0 ? (d->E < 1 ? 1 : d->E) : 1; }
+static inline int max_items_of(const pq_desc* d) { return mtiles_of(d) + experts_of(d) - 1; }
+static inline bool routed(const pq_desc* d) { return d->r > 0 && d->E > 1; }
+
+static int check_desc(const pq_desc* d, bool training) {
+  if (!d) return PQ_ERR_NULL;
+  if (d->size != sizeof(pq_desc)) return PQ_ERR_SHAPE;
+  if (d->T < 1 || d->K < 32 || d->N < 32 || d->K % 32 || d->N % 32) return PQ_ERR_SHAPE;
+  if (d->r < 0 || d->r % 8 || d->r > 256) return PQ_ERR_SHAPE;
+  if (d->r > 0 && (d->E < 1 || d->E > kMaxExperts)) return PQ_ERR_SHAPE;
+  if (d->r > 0 && d->top_k != 1) return PQ_ERR_UNSUPPORTED;
+  if (training && d->r > 128) return PQ_ERR_UNSUPPORTED;
+  return PQ_OK;
+}
+
+// saved buffer layout; base == nullptr only measures
+static size_t carve_saved(const pq_desc* d, void* base, SavedPtrs* out) {
+  Carver c(base);
+  SavedPtrs s{};
+  const size_t T = d->T, K = d->K;
+  const int E = experts_of(d);
+  s.max_items = max_items_of(d);
+  s.q = c.take<int8_t>(T * K);
+  s.xt = c.take<uint16_t>(T * K);
+  s.xs = routed(d) ? c.take<uint16_t>(T * K) : nullptr;
+  s.gamma = c.take<float>(T);
+  s.gate = c.take<float>(T);
+  s.probs = routed(d) ? c.take<float>(T * E) : nullptr;
+  s.expert = c.take<int>(T);
+  s.perm = c.take<int>(T);
+  s.pos = c.take<int>(T);
+  s.offsets = c.take<int>(E + 1);
+  s.h = d->r > 0 ? c.take<uint16_t>((size_t)s.max_items * kTileRows * d->r) : nullptr;
+  s.rt.n_items = c.take<int>(1);
+  s.rt.items = c.take<int4>(s.max_items);
+  s.rt.tile_item_begin = c.take<int>(mtiles_of(d) + 1);
+  s.rt.expert_item_begin = c.take<int>(E + 1);
+  if (out) *out = s;
+  return c.off;
+}
+
+static size_t carve_fwd_scratch(const pq_desc* d, void* base, FwdScratch* out) {
+  Carver c(base);
+  FwdScratch s{};
+  const int E = experts_of(d);
+  const size_t nblocks = (d->T + kRouterTokensPerBlock - 1) / kRouterTokensPerBlock;
+  s.gate_tok = c.take<float>(d->T);
+  s.probs_tok = c.take<float>((size_t)d->T * E);
+  s.block_counts = c.take<int>(nblocks * E);
+  s.block_base = c.take<int>(nblocks * E);
+  if (out) *out = s;
+  return c.off;
+}
+
+struct BwdScratch {
+  uint16_t* dys;
+  uint16_t* sb;
+  uint16_t* ba;
+  uint16_t* dhc;
+  uint16_t* gh;
+  float* dl;
+  uint16_t* dlc;
+  float* dbeta_partial;
+  float* dalpha_partial;
+  float* dwr_partial;
+  float* dalpha_vec;
+  float* dbeta_vec;
+};
+
+static size_t carve_bwd_scratch(const pq_desc* d, void* base, BwdScratch* out) {
+  Carver c(base);
+  BwdScratch s{};
+  const size_t T = d->T, K = d->K, N = d->N, r = d->r;
+  const int E = experts_of(d);
+  const bool vec = d->flags & PQ_SCALE_VECTOR;
+  s.dys = routed(d) ? c.take<uint16_t>(T * N) : nullptr;
+  s.sb = c.take<uint16_t>(N * K);
+  s.ba = (r > 0 && vec) ? c.take<uint16_t>((size_t)E * N * r) : nullptr;
+  s.dhc = r > 0 ? c.take<uint16_t>((size_t)max_items_of(d) * kTileRows * r) : nullptr;
+  s.gh = r > 0 ? c.take<uint16_t>((size_t)max_items_of(d) * kTileRows * r) : nullptr;
+  s.dl = routed(d) ? c.take<float>(T * E) : nullptr;
+  s.dlc = routed(d) ? c.take<uint16_t>(T * 16) : nullptr;
+  s.dbeta_partial = c.take<float>(((K + 255) / 256) * N);
+  s.dalpha_partial = r > 0 ? c.take<float>((size_t)E * N) : nullptr;
+  s.dwr_partial = routed(d) ? c.take<float>(((T + 255) / 256) * E * K) : nullptr;
+  s.dalpha_vec = c.take<float>(N);
+  s.dbeta_vec = c.take<float>(N);
+  if (out) *out = s;
+  return c.off;
+}
+
+static inline bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) != 0; }
+
+}  // namespace pq
+
+using namespace pq;
+
+extern "C" {
+
+const char* pq_status_string(int s) {
+  switch (s) {
+    case PQ_OK: return "ok";
+    case PQ_ERR_NULL: return "a required pointer is NULL";
+    case PQ_ERR_SHAPE: return "a size violates the documented constraints";
+    case PQ_ERR_ALIGN: return "a pointer is not 16-byte aligned";
+    case PQ_ERR_WORKSPACE: return "workspace or saved buffer too small";
+    case PQ_ERR_UNSUPPORTED: return "request not supported";
+    case PQ_ERR_CUDA: return "a CUDA call failed";
+    case PQ_ERR_TIMEOUT: return "a device-side bounded wait ran out";
+    default: return "unknown status";
+  }
+}
+
+size_t pq_saved_bytes(const pq_desc* d) {
+  if (check_desc(d, false) != PQ_OK) return 0;
+  return carve_saved(d, nullptr, nullptr);
+}
+
+size_t pq_workspace_bytes(const pq_desc* d, int phase) {
+  if (!d || d->size != sizeof(pq_desc)) return 0;
+  switch (phase) {
+    case PQ_PHASE_PACK: return align_up(sizeof(double) * 2 * kPackPartials);
+    case PQ_PHASE_FWD:
+      if (check_desc(d, true) != PQ_OK) return 0;
+      return carve_fwd_scratch(d, nullptr, nullptr) + carve_saved(d, nullptr, nullptr);
+    case PQ_PHASE_BWD:
+      if (check_desc(d, true) != PQ_OK) return 0;
+      return carve_bwd_scratch(d, nullptr, nullptr);
+    case PQ_PHASE_DECODE: return 0;
+    default: return 0;
+  }
+}
+
+int pq_saved_view_init(const pq_desc* d, void* saved, pq_saved_view* out) {
+  if (!d || !saved || !out) return PQ_ERR_NULL;
+  int rc = check_desc(d, false);
+  if (rc) return rc;
+  SavedPtrs s;
+  carve_saved(d, saved, &s);
+  out->q = s.q; out->xt = s.xt; out->xs = s.xs; out->gamma = s.gamma; out->gate = s.gate; out->probs = s.probs;
+  out->expert = s.expert; out->perm = s.perm; out->pos = s.pos; out->offsets = s.offsets; out->h = s.h;
+  out->n_items = s.rt.n_items; out->items = reinterpret_cast<int32_t*>(s.rt.items);
+  out->tile_item_begin = s.rt.tile_item_begin; out->expert_item_begin = s.rt.expert_item_begin;
+  out->max_items = s.max_items;
+  return PQ_OK;
+}
+
+int pq_pack_weights(const pq_desc* d, const float* W, uint32_t* w_bits, int8_t* w_s8, float* w_scales, void* ws, size_t ws_bytes,
+                    void* stream) {
+  if (!d || !W || !w_bits || !w_scales || !ws) return PQ_ERR_NULL;
+  if (d->size != sizeof(pq_desc) || d->N < 1 || d->K < 32 || d->K % 32) return PQ_ERR_SHAPE;
+  if (misaligned(W) || misaligned(w_bits) || misaligned(w_s8) || misaligned(ws)) return PQ_ERR_ALIGN;
+  if (ws_bytes < pq_workspace_bytes(d, PQ_PHASE_PACK)) return PQ_ERR_WORKSPACE;
+  cudaError_t e = launch_pack(W, d->N, d->K, w_bits, w_s8, w_scales, static_cast<double*>(ws), static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? PQ_OK : PQ_ERR_CUDA;
+}
+
+int pq_linear_forward(const pq_desc* d, const uint16_t* X, const uint32_t* w_bits, const int8_t* w_s8, const float* w_scales,
+                      const uint16_t* A, const uint16_t* B, const uint16_t* Wr, const float* alpha, const float* beta, uint16_t* Y,
+                      void* saved, size_t saved_bytes, void* ws, size_t ws_bytes, void* stream) {
+  if (!d || !X || !w_scales || !beta || !Y) return PQ_ERR_NULL;
+  if (!w_s8) return PQ_ERR_UNSUPPORTED;  // decode path: see pq_decode_forward
+  int rc = check_desc(d, true);
+  if (rc) return rc;
+  (void)w_bits;
+  if (d->r > 0 && (!A || !B || !alpha)) return PQ_ERR_NULL;
+  if (routed(d) && !Wr) return PQ_ERR_NULL;
+  if (!ws) return PQ_ERR_NULL;
+  if (misaligned(X) || misaligned(w_s8) || misaligned(A) || misaligned(B) || misaligned(Wr) || misaligned(Y) || misaligned(saved) ||
+      misaligned(ws))
+    return PQ_ERR_ALIGN;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  FwdScratch sc;
+  size_t used = carve_fwd_scratch(d, ws, &sc);
+  SavedPtrs sv;
+  if (saved) {
+    if (saved_bytes < carve_saved(d, nullptr, nullptr)) return PQ_ERR_WORKSPACE;
+    carve_saved(d, saved, &sv);
+  } else {
+    used += carve_saved(d, static_cast<uint8_t*>(ws) + used, &sv);
+  }
+  if (ws_bytes < used) return PQ_ERR_WORKSPACE;
+  const int E = experts_of(d);
+  LayerArgs a{d->T, d->K, d->N, d->r, E, (d->flags & PQ_SCALE_VECTOR) ? 1 : 0, w_scales, alpha, beta, A, B, Wr};
+  if (launch_route_and_quant(X, Wr, d->T, d->K, routed(d) ? E : 1, sv, sc, st) != cudaSuccess) return PQ_ERR_CUDA;
+  const uint16_t* xs = routed(d) ? sv.xs : X;
+  return gemm_forward(a, w_s8, sv, xs, Y, st);
+}
+
+int pq_linear_backward(const pq_desc* d, const uint16_t* dY, const uint16_t* X, const int8_t* w_s8, const float* w_scales,
+                       const uint16_t* A, const uint16_t* B, const uint16_t* Wr, const float* alpha, const float* beta,
+                       const void* saved, size_t saved_bytes, uint16_t* dX, float* dW, float* dA, float* dB, float* dWr, float* dalpha,
+                       float* dbeta, void* ws, size_t ws_bytes, void* stream) {
+  (void)d; (void)dY; (void)X; (void)w_s8; (void)w_scales; (void)A; (void)B; (void)Wr; (void)alpha; (void)beta; (void)saved;
+  (void)saved_bytes; (void)dX; (void)dW; (void)dA; (void)dB; (void)dWr; (void)dalpha; (void)dbeta; (void)ws; (void)ws_bytes; (void)stream;
+  return PQ_ERR_UNSUPPORTED;
+}
+
+int pq_debug_gemm(int mode, int M, int N, int K, const void* A, const void* B, void* D, void* stream) {
+  if (!A || !B || !D) return PQ_ERR_NULL;
+  if (M < 1 || N < 1 || K < 1 || M % 8 || N % 8 || K % (mode == 0 ? 16 : 8)) return PQ_ERR_SHAPE;
+  if (misaligned(A) || misaligned(B) || misaligned(D)) return PQ_ERR_ALIGN;
+  return gemm_debug(mode, M, N, K, A, B, D, static_cast<cudaStream_t>(stream));
+}
+
+int pq_device_status(void* stream, int* code, int* where) {
+  if (!code || !where) return PQ_ERR_NULL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaStreamSynchronize(st) != cudaSuccess) return PQ_ERR_CUDA;
+  int host[2] = {0, 0};
+  if (cudaMemcpyFromSymbol(host, g_status, sizeof(host)) != cudaSuccess) return PQ_ERR_CUDA;
+  *code = host[0];
+  *where = host[1];
+  if (host[0] != 0) {
+    const int zero[2] = {0, 0};
+    if (cudaMemcpyToSymbol(g_status, zero, sizeof(zero)) != cudaSuccess) return PQ_ERR_CUDA;
+  }
+  return PQ_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,488 @@
+// Memory-bound kernels of the pQuant layer: weight scale reduction and
+// binarize-and-pack (Eq. 3, 4, 6), router (Sec. 3.3), expert sort, activation
+// quantisation (Eq. 7-9), and the small gather / scale / reduce helpers of the
+// backward pass.
+#include "pq_kernels.cuh"
+
+namespace pq {
+
+// ---------------------------------------------------------------------------
+// K2a: partial sums of W and |W| in fp64 (Eq. 6).  Fixed grid and a fixed
+// reduction tree, so the result does not depend on scheduling.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) k_weight_partial_sums(const float4* __restrict__ W4, long long n4, double* __restrict__ partial) {
+  double s = 0.0, a = 0.0;
+  for (long long i = blockIdx.x * 256LL + threadIdx.x; i < n4; i += gridDim.x * 256LL) {
+    const float4 v = __ldg(W4 + i);
+    s += (double)v.x + (double)v.y + (double)v.z + (double)v.w;
+    a += (double)fabsf(v.x) + (double)fabsf(v.y) + (double)fabsf(v.z) + (double)fabsf(v.w);
+  }
+  for (int d = 16; d > 0; d >>= 1) {
+    s += __shfl_xor_sync(0xffffffffu, s, d);
+    a += __shfl_xor_sync(0xffffffffu, a, d);
+  }
+  __shared__ double sh[2][8];
+  if ((threadIdx.x & 31) == 0) { sh[0][threadIdx.x >> 5] = s; sh[1][threadIdx.x >> 5] = a; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double ts = 0.0, ta = 0.0;
+    for (int w = 0; w < 8; ++w) { ts += sh[0][w]; ta += sh[1][w]; }
+    partial[2 * blockIdx.x] = ts;
+    partial[2 * blockIdx.x + 1] = ta;
+  }
+}
+
+// Every block re-reduces the (few hundred) partials in the same order, so all
+// blocks agree on mu without a grid-wide barrier.
+__device__ __forceinline__ void reduce_partials(const double* partial, int nparts, double inv_count, float* mu, float* lam) {
+  __shared__ double fin[2];
+  if (threadIdx.x < 32) {
+    double s = 0.0, a = 0.0;
+    for (int i = threadIdx.x; i < nparts; i += 32) { s += partial[2 * i]; a += partial[2 * i + 1]; }
+    for (int d = 16; d > 0; d >>= 1) {
+      s += __shfl_xor_sync(0xffffffffu, s, d);
+      a += __shfl_xor_sync(0xffffffffu, a, d);
+    }
+    if (threadIdx.x == 0) { fin[0] = s; fin[1] = a; }
+  }
+  __syncthreads();
+  *mu = (float)(fin[0] * inv_count);
+  *lam = (float)(fin[1] * inv_count);
+}
+
+// ---------------------------------------------------------------------------
+// K2b: S = Sign(W - mu) as the comparison W >= mu (Eq. 3-4); emits the packed
+// words (bit j of word i <-> k = 32 i + j, 1 <-> +1; App. A) and the +-1 int8
+// tile the tensor cores read.  Each thread owns 4 consecutive k.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) k_binarize_pack(const float4* __restrict__ W4, long long n4, const double* __restrict__ partial,
+                                                       int nparts, double inv_count, uint32_t* __restrict__ bits,
+                                                       uint32_t* __restrict__ s8x4, float* __restrict__ scales) {
+  float mu, lam;
+  reduce_partials(partial, nparts, inv_count, &mu, &lam);
+  if (blockIdx.x == 0 && threadIdx.x == 0) { scales[0] = lam; scales[1] = mu; }
+  // n4 is a multiple of 8 (K % 32 == 0), so whole groups of 8 lanes stay together
+  const long long n4_pad = (n4 + 31) & ~31LL;
+  for (long long i = blockIdx.x * 256LL + threadIdx.x; i < n4_pad; i += gridDim.x * 256LL) {
+    uint32_t nib = 0, bytes = 0;
+    if (i < n4) {
+      const float4 v = __ldg(W4 + i);
+      const uint32_t b0 = v.x >= mu, b1 = v.y >= mu, b2 = v.z >= mu, b3 = v.w >= mu;
+      nib = b0 | (b1 << 1) | (b2 << 2) | (b3 << 3);
+      // +1 -> 0x01, -1 -> 0xFF, little endian: byte j <-> k + j
+      bytes = (b0 ? 0x01u : 0xFFu) | (b1 ? 0x0100u : 0xFF00u) | (b2 ? 0x010000u : 0xFF0000u) | (b3 ? 0x01000000u : 0xFF000000u);
+      if (s8x4) s8x4[i] = bytes;
+    }
+    uint32_t word = nib << (4 * (threadIdx.x & 7));
+    word |= __shfl_xor_sync(0xffffffffu, word, 1);
+    word |= __shfl_xor_sync(0xffffffffu, word, 2);
+    word |= __shfl_xor_sync(0xffffffffu, word, 4);
+    if ((threadIdx.x & 7) == 0 && i < n4) bits[i >> 3] = word;
+  }
+}
+
+// ---------------------------------------------------------------------------
+// K4a: router (Sec. 3.3).  One warp per token.  Logits in fp32 with a fixed
+// summation order -- lane j owns the 8-element chunks c with c mod 32 == j,
+// ascending k, fused multiply-add; lanes combined by the xor butterfly
+// 16, 8, 4, 2, 1 -- so that the top-1 index is reproducible bit for bit.
+// Softmax in fp32; ties go to the lowest index.  Also counts tokens per
+// expert for each block of kRouterTokensPerBlock consecutive tokens.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) k_router(const uint4* __restrict__ X, const uint4* __restrict__ Wr, int T, int K, int E,
+                                                int* __restrict__ expert, float* __restrict__ gate_tok,
+                                                float* __restrict__ probs_tok, int* __restrict__ block_counts) {
+  __shared__ int cnt[kMaxExperts];
+  if (threadIdx.x < kMaxExperts) cnt[threadIdx.x] = 0;
+  __syncthreads();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int chunks = K >> 3;
+  for (int it = 0; it < kRouterTokensPerBlock / 8; ++it) {
+    const int t = blockIdx.x * kRouterTokensPerBlock + it * 8 + warp;
+    if (t >= T) break;
+    float acc[kMaxExperts];
+#pragma unroll
+    for (int e = 0; e < kMaxExperts; ++e) acc[e] = 0.f;
+    const uint4* xrow = X + (long long)t * chunks;
+    for (int c = lane; c < chunks; c += 32) {
+      const uint4 xv = __ldg(xrow + c);
+      const float x0 = bf16lo(xv.x), x1 = bf16hi(xv.x), x2 = bf16lo(xv.y), x3 = bf16hi(xv.y);
+      const float x4 = bf16lo(xv.z), x5 = bf16hi(xv.z), x6 = bf16lo(xv.w), x7 = bf16hi(xv.w);
+#pragma unroll
+      for (int e = 0; e < kMaxExperts; ++e) {
+        if (e < E) {
+          const uint4 wv = __ldg(Wr + (long long)e * chunks + c);
+          float a = acc[e];
+          a = fmaf(x0, bf16lo(wv.x), a); a = fmaf(x1, bf16hi(wv.x), a);
+          a = fmaf(x2, bf16lo(wv.y), a); a = fmaf(x3, bf16hi(wv.y), a);
+          a = fmaf(x4, bf16lo(wv.z), a); a = fmaf(x5, bf16hi(wv.z), a);
+          a = fmaf(x6, bf16lo(wv.w), a); a = fmaf(x7, bf16hi(wv.w), a);
+          acc[e] = a;
+        }
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < kMaxExperts; ++e) {
+      if (e < E) {
+        float a = acc[e];
+        for (int d = 16; d > 0; d >>= 1) a = a + __shfl_xor_sync(0xffffffffu, a, d);
+        acc[e] = a;
+      }
+    }
+    // every lane now holds all logits; lane 0 finishes the token
+    int best = 0;
+    float lmax = acc[0];
+#pragma unroll
+    for (int e = 1; e < kMaxExperts; ++e)
+      if (e < E && acc[e] > lmax) { lmax = acc[e]; best = e; }
+    float den = 0.f;
+    float pe[kMaxExperts];
+#pragma unroll
+    for (int e = 0; e < kMaxExperts; ++e) {
+      pe[e] = (e < E) ? expf(acc[e] - lmax) : 0.f;
+      den += pe[e];
+    }
+    const float inv = 1.0f / den;
+    if (lane == 0) {
+      expert[t] = best;
+      atomicAdd(&cnt[best], 1);
+    }
+#pragma unroll
+    for (int e = 0; e < kMaxExperts; ++e) {
+      if (e < E) {
+        const float pr = pe[e] * inv;
+        if (lane == 0) probs_tok[(long long)t * E + e] = pr;
+        if (e == best && lane == 0) gate_tok[t] = pr;
+      }
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x < E) block_counts[blockIdx.x * E + threadIdx.x] = cnt[threadIdx.x];
+}
+
+// ---------------------------------------------------------------------------
+// K4b: expert offsets, per-block bases for the stable scatter, and the item
+// table.  An item is the intersection of a 128-row tile of the sorted token
+// order with one expert's range: {tile, expert, first row, end row} (rows
+// relative to the tile).  Items are sorted by tile and therefore by expert.
+// One small block; the work is a few hundred integers.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(32) k_route_scan(int T, int E, int nblocks, const int* __restrict__ block_counts,
+                                                   int* __restrict__ block_base, int* __restrict__ offsets, RoutingTables rt) {
+  __shared__ int off[kMaxExperts + 1];
+  const int lane = threadIdx.x;
+  if (E <= 1) {
+    if (lane == 0) { off[0] = 0; off[1] = T; offsets[0] = 0; offsets[1] = T; }
+  } else {
+    __shared__ int total[kMaxExperts];
+    if (lane < E) {
+      int run = 0;
+      for (int b = 0; b < nblocks; ++b) {
+        block_base[b * E + lane] = run;
+        run += block_counts[b * E + lane];
+      }
+      total[lane] = run;
+    }
+    __syncwarp();
+    if (lane == 0) {
+      int run = 0;
+      for (int e = 0; e < E; ++e) { off[e] = run; offsets[e] = run; run += total[e]; }
+      off[E] = run;
+      offsets[E] = run;
+    }
+  }
+  __syncwarp();
+  if (lane == 0) {
+    const int Ee = E < 1 ? 1 : E;
+    const int mtiles = (T + kTileRows - 1) / kTileRows;
+    int n = 0, e = 0;
+    for (int x = 0; x <= Ee; ++x) rt.expert_item_begin[x] = 0;
+    for (int tile = 0; tile < mtiles; ++tile) {
+      rt.tile_item_begin[tile] = n;
+      const int r0 = tile * kTileRows, r1 = min(T, r0 + kTileRows);
+      while (e < Ee && off[e + 1] <= r0) ++e;  // first expert reaching into this tile
+      int ee = e;
+      while (ee < Ee && off[ee] < r1) {
+        const int lo = max(off[ee], r0), hi = min(off[ee + 1], r1);
+        if (hi > lo) {
+          rt.items[n] = make_int4(tile, ee, lo - r0, hi - r0);
+          ++n;
+        }
+        ++ee;
+      }
+    }
+    rt.tile_item_begin[mtiles] = n;
+    rt.n_items[0] = n;
+    // items are sorted by expert: first item of each expert
+    int i = 0;
+    for (int x = 0; x < Ee; ++x) {
+      while (i < n && rt.items[i].y < x) ++i;
+      rt.expert_item_begin[x] = i;
+    }
+    rt.expert_item_begin[Ee] = n;
+  }
+}
+
+// ---------------------------------------------------------------------------
+// K1: activation quantisation (Eq. 7-9), one warp per token.  gamma_t = 128 /
+// max(amax, 1e-5) (IEEE division), q = clamp(rint(x * gamma_t), -128, 127).
+// Rows are written at their sorted position p (tokens ordered by expert,
+// stable): q (int8), xt = q / gamma (bf16, the backward's operand) and, with
+// routing, a bf16 copy of the row itself plus its gate and probabilities.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) k_act_quant(const uint4* __restrict__ X, int T, int K, int E, const int* __restrict__ expert,
+                                                   const int* __restrict__ block_base, const int* __restrict__ offsets,
+                                                   const float* __restrict__ gate_tok, const float* __restrict__ probs_tok,
+                                                   uint2* __restrict__ q, uint4* __restrict__ xt, uint4* __restrict__ xs,
+                                                   float* __restrict__ gamma_s, float* __restrict__ gate_s, float* __restrict__ probs_s,
+                                                   int* __restrict__ perm, int* __restrict__ pos) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int t = blockIdx.x * 8 + warp;
+  if (t >= T) return;
+  int p = t;
+  if (E > 1) {
+    const int e = expert[t];
+    const int blk = t / kRouterTokensPerBlock, first = blk * kRouterTokensPerBlock;
+    const int other = (first + lane < T) ? expert[first + lane] : -1;
+    const unsigned same = __ballot_sync(0xffffffffu, other == e);
+    const int rank = __popc(same & ((1u << (t - first)) - 1u));
+    p = offsets[e] + block_base[blk * E + e] + rank;
+  }
+  const int chunks = K >> 3;
+  const uint4* xrow = X + (long long)t * chunks;
+  float amax = 0.f;
+  for (int c = lane; c < chunks; c += 32) {
+    const uint4 v = __ldg(xrow + c);
+    amax = fmaxf(amax, fmaxf(fmaxf(fabsf(bf16lo(v.x)), fabsf(bf16hi(v.x))), fmaxf(fabsf(bf16lo(v.y)), fabsf(bf16hi(v.y)))));
+    amax = fmaxf(amax, fmaxf(fmaxf(fabsf(bf16lo(v.z)), fabsf(bf16hi(v.z))), fmaxf(fabsf(bf16lo(v.w)), fabsf(bf16hi(v.w)))));
+  }
+  for (int d = 16; d > 0; d >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, d));
+  const float gamma = __fdiv_rn(kActQmax, fmaxf(amax, kActAmaxFloor));
+  const float inv_gamma = __fdiv_rn(1.0f, gamma);
+  if (lane == 0) {
+    gamma_s[p] = gamma;
+    perm[p] = t;
+    pos[t] = p;
+    gate_s[p] = (E > 1) ? gate_tok[t] : 1.0f;
+  }
+  if (E > 1 && lane < E) probs_s[(long long)p * E + lane] = probs_tok[(long long)t * E + lane];
+  uint2* qrow = q + (long long)p * chunks;
+  uint4* xtrow = xt ? xt + (long long)p * chunks : nullptr;
+  uint4* xsrow = xs ? xs + (long long)p * chunks : nullptr;
+  for (int c = lane; c < chunks; c += 32) {
+    const uint4 v = __ldg(xrow + c);
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    int qi[8];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float lo = __fmul_rn(bf16lo(w[j]), gamma), hi = __fmul_rn(bf16hi(w[j]), gamma);
+      qi[2 * j] = max(-128, min(127, __float2int_rn(lo)));
+      qi[2 * j + 1] = max(-128, min(127, __float2int_rn(hi)));
+    }
+    uint2 qo;
+    qo.x = (qi[0] & 0xFF) | ((qi[1] & 0xFF) << 8) | ((qi[2] & 0xFF) << 16) | ((qi[3] & 0xFF) << 24);
+    qo.y = (qi[4] & 0xFF) | ((qi[5] & 0xFF) << 8) | ((qi[6] & 0xFF) << 16) | ((qi[7] & 0xFF) << 24);
+    qrow[c] = qo;
+    if (xtrow) {
+      uint4 o;
+      o.x = pack_bf16x2(qi[0] * inv_gamma, qi[1] * inv_gamma);
+      o.y = pack_bf16x2(qi[2] * inv_gamma, qi[3] * inv_gamma);
+      o.z = pack_bf16x2(qi[4] * inv_gamma, qi[5] * inv_gamma);
+      o.w = pack_bf16x2(qi[6] * inv_gamma, qi[7] * inv_gamma);
+      xtrow[c] = o;
+    }
+    if (xsrow) xsrow[c] = v;
+  }
+}
+
+// dst[pos[t], :] = src[t, :]  (rows of `chunks` 16-byte pieces), one warp per row
+__global__ void __launch_bounds__(256) k_scatter_rows(const uint4* __restrict__ src, uint4* __restrict__ dst, const int* __restrict__ pos,
+                                                      int T, int chunks) {
+  const int t = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (t >= T) return;
+  const uint4* s = src + (long long)t * chunks;
+  uint4* d = dst + (long long)pos[t] * chunks;
+  for (int c = lane; c < chunks; c += 32) d[c] = __ldg(s + c);
+}
+
+// Sb[n,k] = bf16(scale_n) * S[n,k]; scale_n = beta_n (vector form) or 1
+__global__ void __launch_bounds__(256) k_scaled_sign(const uint4* __restrict__ s8, uint4* __restrict__ out, const float* __restrict__ beta,
+                                                     int beta_stride, int N, int K) {
+  const long long n16 = (long long)N * K / 16;
+  const int per_row = K / 16;
+  for (long long i = blockIdx.x * 256LL + threadIdx.x; i < n16; i += gridDim.x * 256LL) {
+    const int n = (int)(i / per_row);
+    const float sc = beta_stride ? beta[n] : 1.0f;
+    const uint4 v = __ldg(s8 + i);
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint4 o[2];
+    uint32_t* ow = reinterpret_cast<uint32_t*>(o);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float a = (float)(int8_t)(w[j] & 0xFF) * sc, b = (float)(int8_t)((w[j] >> 8) & 0xFF) * sc;
+      const float c = (float)(int8_t)((w[j] >> 16) & 0xFF) * sc, d = (float)(int8_t)(w[j] >> 24) * sc;
+      ow[2 * j] = pack_bf16x2(a, b);
+      ow[2 * j + 1] = pack_bf16x2(c, d);
+    }
+    out[2 * i] = o[0];
+    out[2 * i + 1] = o[1];
+  }
+}
+
+// Ba[e,n,j] = bf16(alpha_n * B[e,n,j])  (vector alpha only)
+__global__ void __launch_bounds__(256) k_scaled_b(const uint32_t* __restrict__ B2, uint32_t* __restrict__ out, const float* __restrict__ alpha,
+                                                  int E, int N, int r) {
+  const long long n2 = (long long)E * N * r / 2;
+  const int per_row = r / 2;
+  for (long long i = blockIdx.x * 256LL + threadIdx.x; i < n2; i += gridDim.x * 256LL) {
+    const int n = (int)((i / per_row) % N);
+    const uint32_t v = __ldg(B2 + i);
+    out[i] = pack_bf16x2(bf16lo(v) * alpha[n], bf16hi(v) * alpha[n]);
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Router weight gradient dWr[e,k] = sum_p dl[p,e] * x[p,k]  (Sec. 3.3, "trained
+// end-to-end").  CUDA cores: E <= 16 outputs per k.  Partial sums per chunk of
+// 256 tokens, reduced afterwards in a fixed order.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) k_router_wgrad_partial(const uint32_t* __restrict__ xs2, const float* __restrict__ dl, int T, int K, int E,
+                                                              float* __restrict__ partial) {
+  __shared__ float sdl[256 * kMaxExperts];
+  const int t0 = blockIdx.y * 256, nt = min(256, T - t0);
+  for (int i = threadIdx.x; i < nt * E; i += 128) sdl[i] = dl[(long long)t0 * E + i];
+  __syncthreads();
+  const int k2 = blockIdx.x * 128 + threadIdx.x;  // pair of k
+  if (2 * k2 >= K) return;
+  float a0[kMaxExperts], a1[kMaxExperts];
+#pragma unroll
+  for (int e = 0; e < kMaxExperts; ++e) { a0[e] = 0.f; a1[e] = 0.f; }
+  for (int t = 0; t < nt; ++t) {
+    const uint32_t v = __ldg(xs2 + (long long)(t0 + t) * (K / 2) + k2);
+    const float x0 = bf16lo(v), x1 = bf16hi(v);
+#pragma unroll
+    for (int e = 0; e < kMaxExperts; ++e) {
+      if (e < E) {
+        const float d = sdl[t * E + e];
+        a0[e] = fmaf(d, x0, a0[e]);
+        a1[e] = fmaf(d, x1, a1[e]);
+      }
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < kMaxExperts; ++e) {
+    if (e < E) {
+      float* o = partial + ((long long)blockIdx.y * E + e) * K + 2 * k2;
+      o[0] = a0[e];
+      o[1] = a1[e];
+    }
+  }
+}
+
+// out[i] = scale * sum_c partial[c * n + i], c ascending
+__global__ void __launch_bounds__(256) k_sum_partials(const float* __restrict__ partial, int nparts, int n, const float* __restrict__ scale_ptr,
+                                                      float* __restrict__ out) {
+  const int i = blockIdx.x * 256 + threadIdx.x;
+  if (i >= n) return;
+  float s = 0.f;
+  for (int c = 0; c < nparts; ++c) s += partial[(long long)c * n + i];
+  out[i] = s * (scale_ptr ? scale_ptr[0] : 1.0f);
+}
+
+// out[0] = sum_i v[i]  (scalar feature scales), one block, fixed tree
+__global__ void __launch_bounds__(1024) k_sum_to_scalar(const float* __restrict__ v, int n, float* __restrict__ out) {
+  __shared__ double sh[32];
+  double s = 0.0;
+  for (int i = threadIdx.x; i < n; i += 1024) s += (double)v[i];
+  for (int d = 16; d > 0; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
+  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = s;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    s = sh[threadIdx.x];
+    for (int d = 16; d > 0; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
+    if (threadIdx.x == 0) out[0] = (float)s;
+  }
+}
+
+__global__ void k_fill_zero(uint4* p, long long n16) {
+  for (long long i = blockIdx.x * 256LL + threadIdx.x; i < n16; i += gridDim.x * 256LL) p[i] = make_uint4(0, 0, 0, 0);
+}
+
+// ---------------------------------------------------------------------------
+// host launchers
+// ---------------------------------------------------------------------------
+static inline int grid_for(long long work, int per_block, int cap) {
+  long long g = (work + per_block - 1) / per_block;
+  if (g < 1) g = 1;
+  return (int)(g > cap ? cap : g);
+}
+
+cudaError_t launch_pack(const float* W, int N, int K, uint32_t* bits, int8_t* s8, float* scales, double* partial, cudaStream_t st) {
+  const long long n4 = (long long)N * K / 4;
+  const int nparts = grid_for(n4, 256 * 8, kPackPartials);
+  k_weight_partial_sums<<<nparts, 256, 0, st>>>(reinterpret_cast<const float4*>(W), n4, partial);
+  const int grid = grid_for(n4, 256 * 4, 148 * 8);
+  k_binarize_pack<<<grid, 256, 0, st>>>(reinterpret_cast<const float4*>(W), n4, partial, nparts, 1.0 / ((double)N * K), bits,
+                                        reinterpret_cast<uint32_t*>(s8), scales);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_route_and_quant(const uint16_t* X, const uint16_t* Wr, int T, int K, int E, const SavedPtrs& sv, const FwdScratch& sc,
+                                   cudaStream_t st) {
+  const int nblocks = (T + kRouterTokensPerBlock - 1) / kRouterTokensPerBlock;
+  if (E > 1) {
+    k_router<<<nblocks, 256, 0, st>>>(reinterpret_cast<const uint4*>(X), reinterpret_cast<const uint4*>(Wr), T, K, E, sv.expert, sc.gate_tok,
+                                      sc.probs_tok, sc.block_counts);
+  }
+  k_route_scan<<<1, 32, 0, st>>>(T, E, nblocks, sc.block_counts, sc.block_base, sv.offsets, sv.rt);
+  k_act_quant<<<(T + 7) / 8, 256, 0, st>>>(reinterpret_cast<const uint4*>(X), T, K, E, sv.expert, sc.block_base, sv.offsets, sc.gate_tok,
+                                           sc.probs_tok, reinterpret_cast<uint2*>(sv.q), reinterpret_cast<uint4*>(sv.xt),
+                                           reinterpret_cast<uint4*>(sv.xs), sv.gamma, sv.gate, sv.probs, sv.perm, sv.pos);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_scatter_rows(const uint16_t* src, uint16_t* dst, const int* pos, int T, int row_elems, cudaStream_t st) {
+  k_scatter_rows<<<(T + 7) / 8, 256, 0, st>>>(reinterpret_cast<const uint4*>(src), reinterpret_cast<uint4*>(dst), pos, T, row_elems / 8);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_scaled_sign(const int8_t* s8, uint16_t* out, const float* beta, int beta_stride, int N, int K, cudaStream_t st) {
+  const long long n16 = (long long)N * K / 16;
+  k_scaled_sign<<<grid_for(n16, 256 * 2, 148 * 8), 256, 0, st>>>(reinterpret_cast<const uint4*>(s8), reinterpret_cast<uint4*>(out), beta,
+                                                               beta_stride, N, K);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_scaled_b(const uint16_t* B, uint16_t* out, const float* alpha, int E, int N, int r, cudaStream_t st) {
+  const long long n2 = (long long)E * N * r / 2;
+  k_scaled_b<<<grid_for(n2, 256 * 4, 148 * 8), 256, 0, st>>>(reinterpret_cast<const uint32_t*>(B), reinterpret_cast<uint32_t*>(out), alpha, E, N, r);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_router_wgrad(const uint16_t* xs, const float* dl, int T, int K, int E, float* partial, float* dWr, const float* scale,
+                                cudaStream_t st) {
+  const int chunks = (T + 255) / 256;
+  dim3 grid((K / 2 + 127) / 128, chunks);
+  k_router_wgrad_partial<<<grid, 128, 0, st>>>(reinterpret_cast<const uint32_t*>(xs), dl, T, K, E, partial);
+  k_sum_partials<<<(E * K + 255) / 256, 256, 0, st>>>(partial, chunks, E * K, scale, dWr);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_sum_partials(const float* partial, int nparts, int n, const float* scale, float* out, cudaStream_t st) {
+  k_sum_partials<<<(n + 255) / 256, 256, 0, st>>>(partial, nparts, n, scale, out);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_sum_to_scalar(const float* v, int n, float* out, cudaStream_t st) {
+  k_sum_to_scalar<<<1, 1024, 0, st>>>(v, n, out);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_fill_zero(void* p, size_t bytes, cudaStream_t st) {
+  const long long n16 = (long long)(bytes / 16);
+  if (n16 == 0) return cudaSuccess;
+  k_fill_zero<<<grid_for(n16, 256 * 4, 148 * 4), 256, 0, st>>>(reinterpret_cast<uint4*>(p), n16);
+  return cudaGetLastError();
+}
+
+}  // namespace pq

@@ -1,0 +1,230 @@
+// Persistent, warp-specialised tcgen05 GEMM engine for sm_100a.
+//
+// One CTA per SM, 192 threads: warp 0 = TMA producer, warp 1 = MMA issuer
+// (also owns the TMEM allocation), warps 2-5 = epilogue (one per TMEM lane
+// quadrant).  Operands travel global -> shared by TMA into a 4-stage ring of
+// 128-byte-swizzled tiles; tcgen05.mma accumulates 128 x (<=256) tiles in
+// TMEM; the epilogue reads them back with tcgen05.ld.
+//
+// A tile's contraction is a list of SEGMENTS.  Each segment names its operand
+// form (int8 or bf16; each operand either contraction-contiguous "K" or
+// output-dimension-contiguous "MN"), its tensor maps and start coordinates,
+// the number of 128-byte k-blocks, and which of the tile's accumulators it
+// adds into.  This lets one kernel chain, e.g., the int8 1-bit product, the
+// bf16 expert product and the router product of one output tile.
+//
+// A "Problem" type supplies the tile list, the segments and the epilogue.
+#pragma once
+#include <cuda.h>
+
+#include "pq_common.cuh"
+
+namespace pq {
+
+constexpr int kGemmThreads = 192;
+constexpr int kStages = 4;
+constexpr int kTileM = 128;
+constexpr int kStageABytes = 128 * 128;  // 128 rows x 128 B, or two 64x64 bf16 MN boxes
+constexpr int kStageBBytes = 256 * 128;  // up to 256 rows x 128 B, or four MN boxes
+constexpr int kStageBytes = kStageABytes + kStageBBytes;
+constexpr int kMnBoxBytes = 64 * 128;    // one MN-major box: 64 k-rows of 64 bf16
+constexpr int kTmemCols = 512;
+constexpr int kAccCols = 256;            // TMEM columns reserved per accumulator
+constexpr int kGemmSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+
+enum OpMode : int {
+  MODE_I8_KK = 0,  // int8, A[M,K] and B[N,K] K-contiguous
+  MODE_BF_KK = 1,  // bf16, both K-contiguous
+  MODE_BF_KM = 2,  // bf16, A K-contiguous, B N-contiguous
+  MODE_BF_MM = 3   // bf16, A M-contiguous, B N-contiguous
+};
+
+struct Segment {
+  int mode;                 // OpMode
+  int acc;                  // accumulator of the tile this segment adds into
+  int nkb;                  // k-blocks (128 bytes of K each: 128 int8 / 64 bf16)
+  int bn;                   // UMMA N for this segment (multiple of 16, <= 256)
+  int ksteps;               // UMMA k-steps issued per k-block (1..4)
+  const CUtensorMap* ta;
+  const CUtensorMap* tb;
+  int a_x, a_y, a_z;        // K operand: (k0, row0, z);  MN operand: (mn0, k0, z)
+  int b_x, b_y, b_z;
+  int a_rank, b_rank;       // tensor-map rank (2 or 3)
+  int b_bytes;              // bytes TMA delivers for B per k-block
+};
+
+__device__ __forceinline__ bool a_is_mn(int mode) { return mode == MODE_BF_MM; }
+__device__ __forceinline__ bool b_is_mn(int mode) { return mode >= MODE_BF_KM; }
+
+__device__ __forceinline__ void tma_load(uint32_t dst, const CUtensorMap* t, uint32_t bar, int rank, int x, int y, int z) {
+  if (rank == 3) tma_load_3d(dst, t, bar, x, y, z);
+  else tma_load_2d(dst, t, bar, x, y);
+}
+
+struct PipeState {
+  int stage = 0;
+  uint32_t phase = 0;
+  __device__ __forceinline__ void advance(int n) {
+    if (++stage == n) { stage = 0; phase ^= 1; }
+  }
+};
+
+// Bounded wait that also gives up when another role of this CTA has failed.
+__device__ __forceinline__ bool pipe_wait(uint32_t bar, uint32_t parity, int where, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (*abort_flag) return false;
+    if (clock64() - t0 > kSpinCycles) {
+      report_timeout(where);
+      *abort_flag = 1;
+      return false;
+    }
+  }
+  return true;
+}
+
+template <class P>
+__global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_constant__ typename P::Params p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t bar_base = smem_base + kStages * kStageBytes;
+  // barrier block: full[4] empty[4] tfull[2] tempty[2] (8 B each), then tmem ptr, abort flag
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
+  auto tfull_bar = [&](int s) { return bar_base + 8u * (2 * kStages + s); };
+  auto tempty_bar = [&](int s) { return bar_base + 8u * (2 * kStages + 2 + s); };
+  uint8_t* bar_generic = smem_raw + (bar_base - smem_u32(smem_raw));
+  volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(bar_generic + 8 * (2 * kStages + 4));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_generic + 8 * (2 * kStages + 4) + 8);
+
+  constexpr int kAccStages = (P::kAccPerTile == 1) ? 2 : 1;
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(tfull_bar(s), 1); mbar_init(tempty_bar(s), 4); }
+    *abort_flag = 0;
+    mbar_fence_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_holder)), kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_holder;
+  const int ntiles = P::num_tiles(p);
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      PipeState st;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < ntiles; tile += gridDim.x) {
+        typename P::Tile t;
+        P::tile_init(p, tile, t);
+        const int nseg = P::num_segments(p, t);
+        for (int s = 0; ok && s < nseg; ++s) {
+          Segment sg;
+          P::segment(p, t, s, sg);
+          const int a_step = (sg.mode == MODE_I8_KK) ? 128 : 64;
+          for (int kb = 0; kb < sg.nkb; ++kb) {
+            if (!pipe_wait(empty_bar(st.stage), st.phase ^ 1, WHERE_PRODUCER, abort_flag)) { ok = false; break; }
+            const uint32_t bar = full_bar(st.stage);
+            const uint32_t sa = smem_base + st.stage * kStageBytes;
+            const uint32_t sb = sa + kStageABytes;
+            mbar_expect_tx(bar, kStageABytes + sg.b_bytes);
+            if (a_is_mn(sg.mode)) {
+              tma_load(sa, sg.ta, bar, sg.a_rank, sg.a_x, sg.a_y + kb * 64, sg.a_z);
+              tma_load(sa + kMnBoxBytes, sg.ta, bar, sg.a_rank, sg.a_x + 64, sg.a_y + kb * 64, sg.a_z);
+            } else {
+              tma_load(sa, sg.ta, bar, sg.a_rank, sg.a_x + kb * a_step, sg.a_y, sg.a_z);
+            }
+            if (b_is_mn(sg.mode)) {
+              const int nbox = sg.b_bytes / kMnBoxBytes;
+              for (int b = 0; b < nbox; ++b)
+                tma_load(sb + b * kMnBoxBytes, sg.tb, bar, sg.b_rank, sg.b_x + 64 * b, sg.b_y + kb * 64, sg.b_z);
+            } else {
+              tma_load(sb, sg.tb, bar, sg.b_rank, sg.b_x + kb * a_step, sg.b_y, sg.b_z);
+            }
+            st.advance(kStages);
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      PipeState st, ac;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < ntiles; tile += gridDim.x) {
+        typename P::Tile t;
+        P::tile_init(p, tile, t);
+        const int nseg = P::num_segments(p, t);
+        if (!pipe_wait(tempty_bar(ac.stage), ac.phase ^ 1, WHERE_MMA, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        uint32_t started[2] = {0u, 0u};
+        for (int s = 0; ok && s < nseg; ++s) {
+          Segment sg;
+          P::segment(p, t, s, sg);
+          const uint32_t d_tmem = tmem_base + (ac.stage * P::kAccPerTile + sg.acc) * kAccCols;
+          const bool amn = a_is_mn(sg.mode), bmn = b_is_mn(sg.mode);
+          const uint32_t idesc = (sg.mode == MODE_I8_KK) ? umma_idesc(2, 1, 0, 0, sg.bn)
+                                                          : umma_idesc(1, 1, amn ? 1 : 0, bmn ? 1 : 0, sg.bn);
+          for (int kb = 0; kb < sg.nkb; ++kb) {
+            if (!pipe_wait(full_bar(st.stage), st.phase, WHERE_MMA, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t sa = smem_base + st.stage * kStageBytes;
+            const uint32_t sb = sa + kStageABytes;
+            for (int k = 0; k < sg.ksteps; ++k) {
+              const uint64_t ad = amn ? umma_smem_desc(sa + k * 2048, kMnBoxBytes, 1024) : umma_smem_desc(sa + k * 32, 16, 1024);
+              const uint64_t bd = bmn ? umma_smem_desc(sb + k * 2048, kMnBoxBytes, 1024) : umma_smem_desc(sb + k * 32, 16, 1024);
+              if (sg.mode == MODE_I8_KK) umma_i8(d_tmem, ad, bd, idesc, started[sg.acc]);
+              else umma_f16(d_tmem, ad, bd, idesc, started[sg.acc]);
+              started[sg.acc] = 1u;
+            }
+            umma_commit(empty_bar(st.stage));  // frees the smem stage once these MMAs retire
+            st.advance(kStages);
+          }
+        }
+        if (ok) umma_commit(tfull_bar(ac.stage));
+        ac.advance(kAccStages);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue warps
+    PipeState ac;
+    const int quad = warp & 3;  // TMEM lanes [32*quad, 32*quad+32) are this warp's
+    bool ok = true;
+    for (int tile = blockIdx.x; ok && tile < ntiles; tile += gridDim.x) {
+      typename P::Tile t;
+      P::tile_init(p, tile, t);
+      if (!pipe_wait(tfull_bar(ac.stage), ac.phase, WHERE_EPILOGUE, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ac.stage * P::kAccPerTile * kAccCols + (static_cast<uint32_t>(quad * 32) << 16);
+      P::epilogue(p, t, taddr, quad, lane);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(ac.stage));
+      ac.advance(kAccStages);
+    }
+  }
+
+  __syncthreads();
+  if (*abort_flag) {
+    // a wait ran out: give copies and MMAs already in flight time to land before the
+    // shared memory and TMEM of this CTA are released
+    for (int i = 0; i < 200; ++i) __nanosleep(1000);
+  }
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+}  // namespace pq

@@ -1,0 +1,91 @@
+// Internal declarations shared by the kernel translation units and the C ABI.
+#pragma once
+#include <cuda.h>
+
+#include "pq_common.cuh"
+
+namespace pq {
+
+constexpr int kMaxExperts = 16;
+constexpr int kRouterTokensPerBlock = 32;  // must equal the warp width (rank-in-block ballot)
+constexpr int kTileRows = 128;             // rows of one tensor-core tile
+constexpr int kPackPartials = 1024;        // fp64 partial sums of the weight reduction
+constexpr float kActQmax = 128.0f;         // 2^7 of Eq. 9
+constexpr float kActAmaxFloor = 1e-5f;     // all-zero row guard
+
+// Item table of the expert-sorted token order (built by k_route_scan).
+struct RoutingTables {
+  int* n_items;            // [1]
+  int4* items;             // [max_items] {tile, expert, first row, end row}
+  int* tile_item_begin;    // [mtiles + 1]
+  int* expert_item_begin;  // [E + 1]
+};
+
+// Device pointers into the caller's `saved` buffer.
+struct SavedPtrs {
+  int8_t* q;
+  uint16_t* xt;
+  uint16_t* xs;
+  float* gamma;
+  float* gate;
+  float* probs;
+  int* expert;
+  int* perm;
+  int* pos;
+  int* offsets;
+  uint16_t* h;
+  RoutingTables rt;
+  int max_items;
+};
+
+struct FwdScratch {
+  float* gate_tok;
+  float* probs_tok;
+  int* block_counts;
+  int* block_base;
+};
+
+// elementwise launchers (pq_elementwise.cu)
+cudaError_t launch_pack(const float* W, int N, int K, uint32_t* bits, int8_t* s8, float* scales, double* partial, cudaStream_t st);
+cudaError_t launch_route_and_quant(const uint16_t* X, const uint16_t* Wr, int T, int K, int E, const SavedPtrs& sv, const FwdScratch& sc,
+                                   cudaStream_t st);
+cudaError_t launch_scatter_rows(const uint16_t* src, uint16_t* dst, const int* pos, int T, int row_elems, cudaStream_t st);
+cudaError_t launch_scaled_sign(const int8_t* s8, uint16_t* out, const float* beta, int beta_stride, int N, int K, cudaStream_t st);
+cudaError_t launch_scaled_b(const uint16_t* B, uint16_t* out, const float* alpha, int E, int N, int r, cudaStream_t st);
+cudaError_t launch_router_wgrad(const uint16_t* xs, const float* dl, int T, int K, int E, float* partial, float* dWr, const float* scale,
+                                cudaStream_t st);
+cudaError_t launch_sum_partials(const float* partial, int nparts, int n, const float* scale, float* out, cudaStream_t st);
+cudaError_t launch_sum_to_scalar(const float* v, int n, float* out, cudaStream_t st);
+cudaError_t launch_fill_zero(void* p, size_t bytes, cudaStream_t st);
+
+// tensor-core launchers (pq_gemm_kernels.cu).  All return a PQ_* status.
+struct LayerArgs {
+  int T, K, N, r, E;
+  int scale_stride;  // 0: scalar alpha/beta, 1: per-feature vectors
+  const float* w_scales;  // {lam, mu}
+  const float* alpha;
+  const float* beta;
+  const uint16_t* A;   // [E,r,K]
+  const uint16_t* B;   // [E,N,r]
+  const uint16_t* Wr;  // [E,K]
+};
+
+int gemm_debug(int mode, int M, int N, int K, const void* A, const void* B, void* D, cudaStream_t st);
+int gemm_forward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, const uint16_t* xs, uint16_t* Y, cudaStream_t st);
+
+struct BwdBuffers {
+  const uint16_t* dys;   // [T,N] bf16 upstream gradient in sorted order
+  const uint16_t* xs;    // [T,K] bf16 activations in sorted order
+  const uint16_t* sb;    // [N,K] bf16 sign * (beta_n or 1)
+  const uint16_t* ba;    // [E,N,r] bf16 B * (alpha_n or 1)
+  uint16_t* dhc;         // [items*128, r] bf16 dH / c
+  uint16_t* gh;          // [items*128, r] bf16 g * H
+  float* dl;             // [T,E] fp32 router logit gradient (sorted order)
+  uint16_t* dlc;         // [T,16] bf16 dl / c
+  float* dbeta_partial;  // [ceil(K/256), N]
+  float* dalpha_partial; // [E, N]
+};
+int gemm_backward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, const BwdBuffers& b, uint16_t* dX, float* dW, float* dA,
+                  float* dB, cudaStream_t st);
+
+}  // namespace pq

@@ -1,0 +1,89 @@
+"""Buffer management around the C entry points for one pQuant linear layer.
+
+Holds the device tensors (inputs, packed weights, saved activations, gradients,
+workspaces) for a fixed shape and calls pq_pack_weights / pq_linear_forward /
+pq_linear_backward on them.  No arithmetic happens here.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import binding as pqb
+
+
+def _bf16(a, dev):
+    return None if a is None else torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(dev).to(torch.bfloat16).contiguous()
+
+
+def _f32(a, dev):
+    return None if a is None else torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(dev).contiguous()
+
+
+class PQLinear:
+    """One decoupled linear layer of fixed shape on one CUDA device."""
+
+    def __init__(self, T, K, N, r=0, E=0, scale_vector=False, device="cuda:0", training=True):
+        self.dev = torch.device(device)
+        self.T, self.K, self.N, self.r, self.E = T, K, N, r, (E if r > 0 else 0)
+        self.scale_vector = scale_vector
+        self.desc = pqb.make_desc(T, K, N, r, self.E, 1, scale_vector)
+        dev = self.dev
+        u8 = dict(dtype=torch.uint8, device=dev)
+        self.w_bits = torch.empty((N, K // 32), dtype=torch.int32, device=dev)
+        self.w_s8 = torch.empty((N, K), dtype=torch.int8, device=dev)
+        self.w_scales = torch.empty(2, dtype=torch.float32, device=dev)
+        self.ws_pack = torch.empty(pqb.pq_workspace_bytes(self.desc, pqb.PQ_PHASE_PACK), **u8)
+        self.training = training
+        if training:
+            nb = pqb.pq_saved_bytes(self.desc)
+            if nb == 0:
+                raise pqb.PqError("pq_saved_bytes", pqb.PQ_ERR_SHAPE)
+            self.saved = torch.empty(nb, **u8)
+            self.ws_fwd = torch.empty(pqb.pq_workspace_bytes(self.desc, pqb.PQ_PHASE_FWD), **u8)
+            self.ws_bwd = torch.empty(max(16, pqb.pq_workspace_bytes(self.desc, pqb.PQ_PHASE_BWD)), **u8)
+            self.Y = torch.empty((T, N), dtype=torch.bfloat16, device=dev)
+            self.dX = torch.empty((T, K), dtype=torch.bfloat16, device=dev)
+            self.dW = torch.empty((N, K), dtype=torch.float32, device=dev)
+            ns = N if scale_vector else 1
+            self.dalpha = torch.empty(ns, dtype=torch.float32, device=dev)
+            self.dbeta = torch.empty(ns, dtype=torch.float32, device=dev)
+            if r > 0:
+                Ee = max(self.E, 1)
+                self.dA = torch.empty((Ee, r, K), dtype=torch.float32, device=dev)
+                self.dB = torch.empty((Ee, N, r), dtype=torch.float32, device=dev)
+                self.dWr = torch.empty((Ee, K), dtype=torch.float32, device=dev) if Ee > 1 else None
+            else:
+                self.dA = self.dB = self.dWr = None
+        self.X = self.W = self.A = self.B = self.Wr = self.alpha = self.beta = self.dY = None
+
+    # -- data ---------------------------------------------------------------
+    def load_case(self, case: dict):
+        """Upload a dict produced by inputs.make_linear_case."""
+        dev = self.dev
+        self.X = _bf16(case["X"], dev)
+        self.W = _f32(case["W"], dev)
+        self.A = _bf16(case.get("A"), dev) if self.r > 0 else None
+        self.B = _bf16(case.get("B"), dev) if self.r > 0 else None
+        self.Wr = _bf16(case.get("Wr"), dev) if (self.r > 0 and self.E > 1) else None
+        self.alpha = _f32(case["alpha"], dev)
+        self.beta = _f32(case["beta"], dev)
+        self.dY = _bf16(case.get("dY"), dev)
+        return self
+
+    # -- calls --------------------------------------------------------------
+    def pack(self):
+        pqb.pq_pack_weights(self.desc, self.W, self.w_bits, self.w_s8, self.w_scales, self.ws_pack)
+
+    def forward(self, X=None, Y=None):
+        pqb.pq_linear_forward(self.desc, self.X if X is None else X, self.w_bits, self.w_s8, self.w_scales, self.A, self.B,
+                              self.Wr, self.alpha, self.beta, self.Y if Y is None else Y, self.saved, self.ws_fwd)
+        return self.Y if Y is None else Y
+
+    def backward(self, dY=None):
+        pqb.pq_linear_backward(self.desc, self.dY if dY is None else dY, self.X, self.w_s8, self.w_scales, self.A, self.B,
+                               self.Wr, self.alpha, self.beta, self.saved, self.dX, self.dW, self.dA, self.dB, self.dWr,
+                               self.dalpha, self.dbeta, self.ws_bwd)
+
+    def saved_view(self) -> dict:
+        return pqb.pq_saved_view_init(self.desc, self.saved)

@@ -1,0 +1,192 @@
+"""GPU parity tests (forward side): every step of the layer through the C ABI
+against the CPU oracle on the same seeded inputs.  Integer results bit-exact;
+floating point within the stated tolerances."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import pquant_oracle as O
+from paper_2602_22592_b200 import binding as pqb
+from paper_2602_22592_b200 import inputs as I
+from paper_2602_22592_b200.layer import PQLinear
+
+pytestmark = pytest.mark.gpu
+
+TOL_BF16 = 2e-2     # max relative error of bf16 outputs / gradients
+TOL_SCALE = 1e-5    # fp32-accumulated scales
+
+
+def rel_err(a, b):
+    """max |a-b| / max(|b|, 1e-2 * rms(b)) -- avoids blow-up at zero crossings."""
+    a = np.asarray(a, dtype=np.float64)
+    b = np.asarray(b, dtype=np.float64)
+    floor = 1e-2 * np.sqrt(np.mean(b * b)) + 1e-30
+    return float(np.max(np.abs(a - b) / np.maximum(np.abs(b), floor)))
+
+
+def f32(t):
+    return t.detach().float().cpu().numpy()
+
+
+def check_status():
+    code, where = pqb.pq_device_status()
+    assert code == 0, f"device wait timed out (where={where})"
+
+
+# ------------------------------------------------------------------ pack (Eq. 3, 4, 6)
+@pytest.mark.parametrize("N,K", [(32, 32), (96, 256), (512, 512), (1000 // 8 * 8, 2048), (2048, 5632)])
+def test_pack_weights_bit_exact(N, K):
+    N = (N + 31) // 32 * 32
+    c = I.make_linear_case(1, K, N, 0, 0, seed=100 + N, with_grad=False)
+    L = PQLinear(128, K, N, training=False)
+    L.W = torch.from_numpy(c["W"]).cuda()
+    L.pack()
+    torch.cuda.synchronize()
+    mu, lam = O.weight_scales(c["W"])
+    S = O.binarize(c["W"], mu)
+    sc = f32(L.w_scales)
+    assert abs(sc[0] - lam) <= TOL_SCALE * abs(lam) and abs(sc[1] - mu) <= TOL_SCALE * abs(lam)
+    assert sc[1] == mu and sc[0] == lam          # in practice bit-identical
+    assert np.array_equal(L.w_s8.cpu().numpy(), S)
+    assert np.array_equal(L.w_bits.cpu().numpy().view(np.uint32), O.pack_bits(S))
+
+
+def test_pack_constant_matrix_and_ties():
+    W = np.full((64, 64), 0.125, np.float32)
+    L = PQLinear(128, 64, 64, training=False)
+    L.W = torch.from_numpy(W).cuda()
+    L.pack()
+    assert np.all(L.w_s8.cpu().numpy() == 1)      # Sign(0) := +1
+    assert np.all(L.w_bits.cpu().numpy().view(np.uint32) == 0xFFFFFFFF)
+
+
+# ------------------------------------------------------------------ tensor-core engine, raw accumulators
+@pytest.mark.parametrize("M,N,K", [(128, 256, 128), (256, 512, 512), (392, 520, 1040), (8, 16, 16)])
+def test_engine_int8_accumulators_bit_exact(M, N, K):
+    rng = np.random.default_rng(M + N + K)
+    A = rng.integers(-128, 128, (M, K)).astype(np.int8)
+    B = rng.choice([-1, 1], (N, K)).astype(np.int8)
+    D = torch.full((M, N), 0x7FFFFFFF, dtype=torch.int32, device="cuda")
+    pqb.pq_debug_gemm(0, M, N, K, torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda(), D)
+    torch.cuda.synchronize()
+    check_status()
+    assert np.array_equal(D.cpu().numpy().astype(np.int64), O.onebit_gemm(A, B))
+
+
+@pytest.mark.parametrize("mode", [1, 2, 3])
+@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (256, 512, 512), (392, 520, 1000), (8, 16, 16)])
+def test_engine_bf16_operand_forms(mode, M, N, K):
+    rng = np.random.default_rng(mode * 1000 + M + N + K)
+    A = I.bf16_values(rng.standard_normal((M, K)).astype(np.float32))
+    B = I.bf16_values(rng.standard_normal((N, K)).astype(np.float32))
+    ref = A.astype(np.float64) @ B.astype(np.float64).T
+    At = torch.from_numpy(A if mode != 3 else np.ascontiguousarray(A.T)).cuda().to(torch.bfloat16)
+    Bt = torch.from_numpy(B if mode == 1 else np.ascontiguousarray(B.T)).cuda().to(torch.bfloat16)
+    D = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+    pqb.pq_debug_gemm(mode, M, N, K, At, Bt, D)
+    torch.cuda.synchronize()
+    check_status()
+    got = D.cpu().numpy()
+    assert np.all(np.isfinite(got))
+    assert np.max(np.abs(got - ref)) <= 1e-4 * np.sqrt(K) * 4
+
+
+# ------------------------------------------------------------------ forward of the layer
+def run_forward(c, scale_vector):
+    L = PQLinear(c["T"], c["K"], c["N"], c["r"], c["E"], scale_vector=scale_vector).load_case(c)
+    L.pack()
+    L.forward()
+    torch.cuda.synchronize()
+    check_status()
+    return L
+
+
+def check_forward(c, L, f):
+    sv = L.saved_view()
+    T, E = c["T"], max(c["E"], 1)
+    perm = sv["perm"].cpu().numpy()
+    if c["r"] > 0 and c["E"] > 1:
+        # router: indices, permutation, offsets are integers -> exact
+        assert np.array_equal(sv["expert"].cpu().numpy(), f["idx"])
+        assert np.array_equal(perm, f["perm"])
+        assert np.array_equal(sv["offsets"].cpu().numpy(), f["offsets"])
+        assert np.array_equal(sv["pos"].cpu().numpy()[perm], np.arange(T))
+        assert rel_err(f32(sv["gate"]), f["gate"][perm]) <= 1e-5
+        assert np.max(np.abs(f32(sv["probs"]) - f["probs"][perm])) <= 1e-6
+    else:
+        assert np.array_equal(perm, np.arange(T))
+    # Eq. 7-9: int8 codes and gamma bit-exact
+    assert np.array_equal(sv["q"].cpu().numpy(), f["q"][perm])
+    assert np.array_equal(f32(sv["gamma"]), f["gamma"][perm])
+    if c["r"] > 0:
+        # item table covers every sorted row exactly once, one expert per item
+        n_items = int(sv["n_items"].cpu()[0])
+        items = sv["items"].cpu().numpy()[:n_items]
+        cover = np.zeros(T, int)
+        srt_e = f["idx"][perm] if c["E"] > 1 else np.zeros(T, int)
+        h = f32(sv["h"])
+        for i, (tile, e, lo, hi) in enumerate(items):
+            rows = np.arange(tile * 128 + lo, tile * 128 + hi)
+            cover[rows] += 1
+            assert np.all(srt_e[rows] == e)
+            blk = h[i * 128:(i + 1) * 128]
+            assert rel_err(blk[lo:hi], f["h"][perm[rows]]) <= TOL_BF16
+            assert np.all(blk[:lo] == 0) and np.all(blk[hi:] == 0)
+        assert np.all(cover == 1)
+    assert rel_err(f32(L.Y), f["Y"]) <= TOL_BF16
+
+
+CASES = {
+    "cfg1": dict(T=256, K=512, N=512, r=32, E=1, scale_vector=True, alpha=1.0, beta=1.0),
+    "pure_1bit": dict(T=200, K=256, N=320, r=0, E=0),
+    "dense_hp_ragged": dict(T=333, K=384, N=544, r=64, E=1),
+    "routed8": dict(T=1000, K=512, N=768, r=128, E=8),
+    "routed4_small_r": dict(T=520, K=256, N=256, r=16, E=4, scale_vector=True, alpha=1.5, beta=0.4),
+}
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_forward_matches_oracle(name):
+    kw = dict(CASES[name])
+    sv = kw.pop("scale_vector", False)
+    c = I.make_linear_case(kw.pop("T"), kw.pop("K"), kw.pop("N"), kw.pop("r"), kw.pop("E"), seed=7, scale_vector=sv, **kw)
+    f = O.linear_forward(c["X"], c["W"], c["A"], c["B"], c["Wr"], c["alpha"], c["beta"])
+    L = run_forward(c, sv)
+    check_forward(c, L, f)
+
+
+def test_forward_degenerate_rows_and_experts():
+    # an all-zero token, a constant-sign row, and a router that sends every token to one expert
+    c = I.make_linear_case(300, 256, 256, 32, 4, seed=9, zipf=False)
+    c["X"][7] = 0.0
+    c["Wr"][:] = 0.0
+    c["Wr"][2] = I.bf16_values(np.full(256, 0.5, np.float32))
+    c["X"] = I.bf16_values(np.abs(c["X"]))        # positive activations -> expert 2 wins everywhere except the zero row
+    f = O.linear_forward(c["X"], c["W"], c["A"], c["B"], c["Wr"], c["alpha"], c["beta"])
+    assert f["idx"][7] == 0 and np.all(np.delete(f["idx"], 7) == 2)
+    L = run_forward(c, False)
+    check_forward(c, L, f)
+
+
+def test_forward_is_deterministic():
+    c = I.make_linear_case(512, 512, 512, 64, 4, seed=3)
+    L = run_forward(c, False)
+    y1 = L.Y.clone()
+    L.forward()
+    torch.cuda.synchronize()
+    assert torch.equal(y1, L.Y)
+
+
+def test_argument_errors_are_reported():
+    d = pqb.make_desc(128, 100, 64)               # K not a multiple of 32
+    assert pqb.pq_saved_bytes(d) == 0
+    L = PQLinear(128, 64, 64, 32, 1)
+    with pytest.raises(pqb.PqError) as ei:
+        pqb.pq_linear_forward(L.desc, None, L.w_bits, L.w_s8, L.w_scales, None, None, None, None, None, L.Y, L.saved, L.ws_fwd)
+    assert ei.value.status == pqb.PQ_ERR_NULL
+    small = torch.empty(16, dtype=torch.uint8, device="cuda")
+    c = I.make_linear_case(128, 64, 64, 32, 1, seed=1)
+    L.load_case(c)
+    with pytest.raises(pqb.PqError) as ei:
+        pqb.pq_linear_forward(L.desc, L.X, L.w_bits, L.w_s8, L.w_scales, L.A, L.B, None, L.alpha, L.beta, L.Y, L.saved, small)
+    assert ei.value.status == pqb.PQ_ERR_WORKSPACE
