@@ -215,9 +215,62 @@ int pq_linear_backward(const pq_desc* d, const uint16_t* dY, const uint16_t* X, 
                        const uint16_t* A, const uint16_t* B, const uint16_t* Wr, const float* alpha, const float* beta,
                        const void* saved, size_t saved_bytes, uint16_t* dX, float* dW, float* dA, float* dB, float* dWr, float* dalpha,
                        float* dbeta, void* ws, size_t ws_bytes, void* stream) {
-  (void)d; (void)dY; (void)X; (void)w_s8; (void)w_scales; (void)A; (void)B; (void)Wr; (void)alpha; (void)beta; (void)saved;
-  (void)saved_bytes; (void)dX; (void)dW; (void)dA; (void)dB; (void)dWr; (void)dalpha; (void)dbeta; (void)ws; (void)ws_bytes; (void)stream;
-  return PQ_ERR_UNSUPPORTED;
+  if (!d || !dY || !X || !w_s8 || !w_scales || !beta || !saved || !dX || !dW || !dbeta || !ws) return PQ_ERR_NULL;
+  int rc = check_desc(d, true);
+  if (rc) return rc;
+  const bool hp = d->r > 0;
+  if (hp && (!A || !B || !alpha || !dA || !dB || !dalpha)) return PQ_ERR_NULL;
+  if (routed(d) && (!Wr || !dWr)) return PQ_ERR_NULL;
+  if (misaligned(dY) || misaligned(X) || misaligned(w_s8) || misaligned(A) || misaligned(B) || misaligned(Wr) || misaligned(saved) ||
+      misaligned(dX) || misaligned(dW) || misaligned(dA) || misaligned(dB) || misaligned(dWr) || misaligned(ws))
+    return PQ_ERR_ALIGN;
+  if (saved_bytes < carve_saved(d, nullptr, nullptr)) return PQ_ERR_WORKSPACE;
+  if (ws_bytes < carve_bwd_scratch(d, nullptr, nullptr)) return PQ_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  SavedPtrs sv;
+  carve_saved(d, const_cast<void*>(saved), &sv);
+  BwdScratch sc;
+  carve_bwd_scratch(d, ws, &sc);
+  const int E = experts_of(d);
+  const int vec = (d->flags & PQ_SCALE_VECTOR) ? 1 : 0;
+  LayerArgs a{d->T, d->K, d->N, d->r, E, vec, w_scales, alpha, beta, A, B, Wr};
+
+  BwdBuffers b{};
+  if (routed(d)) {
+    if (launch_scatter_rows(dY, sc.dys, sv.pos, d->T, d->N, st) != cudaSuccess) return PQ_ERR_CUDA;
+    b.dys = sc.dys;
+    b.xs = sv.xs;
+  } else {
+    b.dys = dY;
+    b.xs = X;
+  }
+  if (launch_scaled_sign(w_s8, sc.sb, beta, vec, d->N, d->K, st) != cudaSuccess) return PQ_ERR_CUDA;
+  b.sb = sc.sb;
+  if (hp && vec) {
+    if (launch_scaled_b(B, sc.ba, alpha, E, d->N, d->r, st) != cudaSuccess) return PQ_ERR_CUDA;
+    b.ba = sc.ba;
+  } else {
+    b.ba = B;
+  }
+  b.dhc = sc.dhc; b.gh = sc.gh; b.dl = sc.dl; b.dlc = sc.dlc;
+  b.dbeta_partial = sc.dbeta_partial; b.dalpha_partial = sc.dalpha_partial;
+  rc = gemm_backward(a, w_s8, sv, b, dX, dW, dA, dB, st);
+  if (rc) return rc;
+
+  if (routed(d)) {
+    if (launch_router_wgrad(sv.xs, sc.dl, d->T, d->K, E, sc.dwr_partial, dWr, nullptr, st) != cudaSuccess) return PQ_ERR_CUDA;
+  }
+  // dbeta_n = lam * sum over k-tiles of the partial sign-weighted row sums; scalar form sums over n
+  const int ntk = (d->K + 255) / 256;
+  if (launch_sum_partials(sc.dbeta_partial, ntk, d->N, w_scales, vec ? dbeta : sc.dbeta_vec, st) != cudaSuccess) return PQ_ERR_CUDA;
+  if (!vec && launch_sum_to_scalar(sc.dbeta_vec, d->N, dbeta, st) != cudaSuccess) return PQ_ERR_CUDA;
+  if (hp) {
+    if (launch_sum_partials(sc.dalpha_partial, E, d->N, nullptr, vec ? dalpha : sc.dalpha_vec, st) != cudaSuccess) return PQ_ERR_CUDA;
+    if (!vec && launch_sum_to_scalar(sc.dalpha_vec, d->N, dalpha, st) != cudaSuccess) return PQ_ERR_CUDA;
+  } else if (dalpha) {
+    if (cudaMemsetAsync(dalpha, 0, sizeof(float) * (vec ? d->N : 1), st) != cudaSuccess) return PQ_ERR_CUDA;
+  }
+  return PQ_OK;
 }
 
 int pq_debug_gemm(int mode, int M, int N, int K, const void* A, const void* B, void* D, void* stream) {

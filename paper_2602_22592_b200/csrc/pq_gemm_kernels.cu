@@ -309,4 +309,428 @@ int gemm_forward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, co
   return launch_gemm<FwdProblem<false>>(f, mtiles * f.ntn, st);
 }
 
+
+// ===========================================================================
+// backward (straight-through estimator, App. B.1)
+// ===========================================================================
+// The scale of the 1-bit input gradient: dX1 = c * (dYs . Sb) with
+//   scalar beta:  Sb = S,            c = lam * beta
+//   vector beta:  Sb = bf16(beta_n) S, c = lam
+// The HP and router contributions are accumulated in the same tile, so they
+// are pre-divided by c (and the whole tile multiplied by c in the epilogue).
+// c == 0 switches the 1-bit term off instead.
+__device__ __forceinline__ float dx_scale(const float* w_scales, const float* beta, int sstride) {
+  return sstride ? w_scales[0] : w_scales[0] * beta[0];
+}
+
+// ---------------------------------------------------------------------------
+// B1: dHraw = dYs . (alpha B_e) per item; epilogue forms
+//   dg_t = alpha * sum_j H dHraw,  dH = g dHraw  ->  dhc = dH / c  (bf16, masked)
+//   gh = g H (bf16, masked),  dl[t,j] = dg g (delta_je - p_tj),  dlc = dl / c
+// ---------------------------------------------------------------------------
+struct HpDhProblem {
+  static constexpr int kAccPerTile = 1;
+  struct Params {
+    CUtensorMap tdy, tba;  // dYs [T,N]; (alpha) B [E,N,r]
+    RoutingTables rt;
+    const uint16_t* H;
+    const float* gate;
+    const float* probs;
+    const float* w_scales;
+    const float* alpha;
+    const float* beta;
+    uint16_t* dhc;
+    uint16_t* gh;
+    float* dl;
+    uint16_t* dlc;
+    int T, N, r, E, bn, sstride;
+  };
+  struct Tile { int item; int4 it; };
+  __device__ static int num_tiles(const Params& p) { return p.rt.n_items[0]; }
+  __device__ static void tile_init(const Params& p, int i, Tile& t) { t.item = i; t.it = p.rt.items[i]; }
+  __device__ static int num_segments(const Params&, const Tile&) { return 1; }
+  __device__ static void segment(const Params& p, const Tile& t, int, Segment& s) {
+    s.mode = MODE_BF_KM; s.acc = 0; s.bn = p.bn; s.ksteps = 4; s.nkb = (p.N + 63) / 64;
+    s.ta = &p.tdy; s.a_rank = 2; s.a_x = 0; s.a_y = t.it.x * 128; s.a_z = 0;
+    s.tb = &p.tba; s.b_rank = 3; s.b_x = 0; s.b_y = 0; s.b_z = t.it.y;
+    s.b_bytes = (p.bn / 64) * kMnBoxBytes;
+  }
+  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane) {
+    const int row = quad * 32 + lane;
+    const bool live = row >= t.it.z && row < t.it.w;
+    const int pos = t.it.x * 128 + row;
+    const float c = dx_scale(p.w_scales, p.beta, p.sstride);
+    const float inv_cc = c != 0.f ? 1.0f / c : 1.0f;
+    const float ca = p.sstride ? 1.0f : p.alpha[0];
+    const float g = live ? p.gate[pos] : 0.f;
+    const long long hrow = ((long long)t.item * 128 + row) * p.r;
+    const uint4* hin = reinterpret_cast<const uint4*>(p.H + hrow);
+    uint4* dhc = reinterpret_cast<uint4*>(p.dhc + hrow);
+    uint4* gh = reinterpret_cast<uint4*>(p.gh + hrow);
+    float dg = 0.f;
+    for (int c32 = 0; c32 * 32 < p.r; ++c32) {
+      uint32_t v[32];
+      tmem_ld32(taddr + c32 * 32, v);
+      tmem_ld_wait();
+#pragma unroll
+      for (int q8 = 0; q8 < 4; ++q8) {
+        if (c32 * 32 + q8 * 8 < p.r) {
+          uint4 o1 = make_uint4(0, 0, 0, 0), o2 = make_uint4(0, 0, 0, 0);
+          if (live) {
+            const uint4 hv = hin[c32 * 4 + q8];
+            const uint32_t hw[4] = {hv.x, hv.y, hv.z, hv.w};
+            uint32_t w1[4], w2[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const float h0 = bf16lo(hw[j]), h1 = bf16hi(hw[j]);
+              const float d0 = __uint_as_float(v[q8 * 8 + 2 * j]), d1 = __uint_as_float(v[q8 * 8 + 2 * j + 1]);
+              dg = fmaf(h0, d0, dg);
+              dg = fmaf(h1, d1, dg);
+              const float sc = ca * g * inv_cc;
+              w1[j] = pack_bf16x2(sc * d0, sc * d1);
+              w2[j] = pack_bf16x2(g * h0, g * h1);
+            }
+            o1 = make_uint4(w1[0], w1[1], w1[2], w1[3]);
+            o2 = make_uint4(w2[0], w2[1], w2[2], w2[3]);
+          }
+          dhc[c32 * 4 + q8] = o1;
+          gh[c32 * 4 + q8] = o2;
+        }
+      }
+    }
+    if (p.E > 1 && live) {
+      dg *= ca;
+      uint32_t packed[8];
+      float prev = 0.f;
+#pragma unroll
+      for (int e = 0; e < 16; ++e) {
+        float d = 0.f;
+        if (e < p.E) {
+          d = dg * g * ((e == t.it.y ? 1.0f : 0.0f) - p.probs[(long long)pos * p.E + e]);
+          p.dl[(long long)pos * p.E + e] = d;
+        }
+        if (e & 1) packed[e >> 1] = pack_bf16x2(prev * inv_cc, d * inv_cc);
+        prev = d;
+      }
+      uint4* o = reinterpret_cast<uint4*>(p.dlc + (long long)pos * 16);
+      o[0] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+      o[1] = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+    }
+  }
+};
+
+// ---------------------------------------------------------------------------
+// B2: dX tile = c * ( dYs . Sb  +  sum_items dhc . A_e  +  dlc . Wr ), rows
+// scattered back to token order.
+// ---------------------------------------------------------------------------
+struct BwdDxProblem {
+  static constexpr int kAccPerTile = 1;
+  struct Params {
+    CUtensorMap tdy, tsb, tdh, ta3, tdl, twr;
+    RoutingTables rt;
+    const int* perm;
+    const float* w_scales;
+    const float* beta;
+    uint16_t* dX;
+    int T, N, K, r, E, sstride, ntk;
+  };
+  struct Tile { int m, kt, ib, ie, skip1; };
+  __device__ static int num_tiles(const Params& p) { return ((p.T + 127) / 128) * p.ntk; }
+  __device__ static void tile_init(const Params& p, int i, Tile& t) {
+    t.m = i / p.ntk; t.kt = i % p.ntk;
+    if (p.r > 0) { t.ib = p.rt.tile_item_begin[t.m]; t.ie = p.rt.tile_item_begin[t.m + 1]; } else { t.ib = t.ie = 0; }
+    t.skip1 = dx_scale(p.w_scales, p.beta, p.sstride) == 0.f;
+  }
+  __device__ static int num_segments(const Params& p, const Tile& t) { return (t.skip1 ? 0 : 1) + (t.ie - t.ib) + (p.E > 1 ? 1 : 0); }
+  __device__ static void segment(const Params& p, const Tile& t, int i, Segment& s) {
+    s.mode = MODE_BF_KM; s.acc = 0; s.bn = 256; s.ksteps = 4; s.a_rank = 2; s.a_x = 0; s.a_z = 0;
+    s.b_x = t.kt * 256; s.b_y = 0; s.b_z = 0; s.b_bytes = kStageBBytes;
+    if (!t.skip1) {
+      if (i == 0) {
+        s.nkb = (p.N + 63) / 64;
+        s.ta = &p.tdy; s.a_y = t.m * 128;
+        s.tb = &p.tsb; s.b_rank = 2;
+        return;
+      }
+      --i;
+    }
+    if (i < t.ie - t.ib) {
+      const int item = t.ib + i;
+      s.nkb = (p.r + 63) / 64;
+      s.ta = &p.tdh; s.a_y = item * 128;
+      s.tb = &p.ta3; s.b_rank = 3; s.b_z = p.rt.items[item].y;
+      return;
+    }
+    s.nkb = 1; s.ksteps = 1;
+    s.ta = &p.tdl; s.a_y = t.m * 128;
+    s.tb = &p.twr; s.b_rank = 2;
+  }
+  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane) {
+    const int pos = t.m * 128 + quad * 32 + lane;
+    const bool live = pos < p.T;
+    const int token = live ? (p.perm ? p.perm[pos] : pos) : 0;
+    const float c = dx_scale(p.w_scales, p.beta, p.sstride);
+    const float cc = c != 0.f ? c : 1.0f;
+    const bool has = num_segments(p, t) > 0;
+    uint4* xrow = reinterpret_cast<uint4*>(p.dX + (long long)token * p.K);
+    for (int c32 = 0; c32 < 8; ++c32) {
+      const int k0 = t.kt * 256 + c32 * 32;
+      if (k0 >= p.K) break;
+      uint32_t v[32];
+      tmem_ld32(taddr + c32 * 32, v);
+      tmem_ld_wait();
+      if (live) {
+#pragma unroll
+        for (int q8 = 0; q8 < 4; ++q8) {
+          uint32_t w[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            w[j] = has ? pack_bf16x2(cc * __uint_as_float(v[q8 * 8 + 2 * j]), cc * __uint_as_float(v[q8 * 8 + 2 * j + 1])) : 0u;
+          xrow[(k0 >> 3) + q8] = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      }
+    }
+  }
+};
+
+// ---------------------------------------------------------------------------
+// B3: G = dYs^T . xt (contraction over tokens); dW = beta_n G; per-tile partial
+// of dbeta_n = lam * sum_k S[n,k] G[n,k].
+// ---------------------------------------------------------------------------
+struct BwdDwProblem {
+  static constexpr int kAccPerTile = 1;
+  struct Params {
+    CUtensorMap tdyT, txt;
+    const int8_t* s8;
+    const float* beta;
+    float* dW;
+    float* dbeta_partial;
+    int T, N, K, sstride, ntk;
+  };
+  struct Tile { int nt, kt; };
+  __device__ static int num_tiles(const Params& p) { return ((p.N + 127) / 128) * p.ntk; }
+  __device__ static void tile_init(const Params& p, int i, Tile& t) { t.nt = i / p.ntk; t.kt = i % p.ntk; }
+  __device__ static int num_segments(const Params&, const Tile&) { return 1; }
+  __device__ static void segment(const Params& p, const Tile& t, int, Segment& s) {
+    s.mode = MODE_BF_MM; s.acc = 0; s.bn = 256; s.ksteps = 4; s.nkb = (p.T + 63) / 64;
+    s.ta = &p.tdyT; s.a_rank = 2; s.a_x = t.nt * 128; s.a_y = 0; s.a_z = 0;
+    s.tb = &p.txt; s.b_rank = 2; s.b_x = t.kt * 256; s.b_y = 0; s.b_z = 0;
+    s.b_bytes = kStageBBytes;
+  }
+  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane) {
+    const int n = t.nt * 128 + quad * 32 + lane;
+    const bool live = n < p.N;
+    const float be = live ? p.beta[n * p.sstride] : 0.f;
+    float4* wrow = reinterpret_cast<float4*>(p.dW + (long long)(live ? n : 0) * p.K);
+    const uint4* srow = reinterpret_cast<const uint4*>(p.s8 + (long long)(live ? n : 0) * p.K);
+    float part = 0.f;
+    for (int c32 = 0; c32 < 8; ++c32) {
+      const int k0 = t.kt * 256 + c32 * 32;
+      if (k0 >= p.K) break;
+      uint32_t v[32];
+      tmem_ld32(taddr + c32 * 32, v);
+      tmem_ld_wait();
+      if (live) {
+        const uint4 s0 = __ldg(srow + (k0 >> 4)), s1 = __ldg(srow + (k0 >> 4) + 1);
+        const uint32_t sw[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+#pragma unroll
+        for (int q4 = 0; q4 < 8; ++q4) {
+          const float g0 = __uint_as_float(v[q4 * 4]), g1 = __uint_as_float(v[q4 * 4 + 1]);
+          const float g2 = __uint_as_float(v[q4 * 4 + 2]), g3 = __uint_as_float(v[q4 * 4 + 3]);
+          const uint32_t sb = sw[q4];  // four +-1 bytes: bit 7 set <-> -1
+          part += (sb & 0x80u) ? -g0 : g0;
+          part += (sb & 0x8000u) ? -g1 : g1;
+          part += (sb & 0x800000u) ? -g2 : g2;
+          part += (sb & 0x80000000u) ? -g3 : g3;
+          wrow[(k0 >> 2) + q4] = make_float4(be * g0, be * g1, be * g2, be * g3);
+        }
+      }
+    }
+    if (live) p.dbeta_partial[(long long)t.kt * p.N + n] = part;
+  }
+};
+
+// ---------------------------------------------------------------------------
+// B4: dBraw_e = dYs^T . (g H) over the items of expert e; dB = alpha_n dBraw;
+// partial of dalpha_n = sum_j B_e[n,j] dBraw_e[n,j].
+// ---------------------------------------------------------------------------
+struct HpDbProblem {
+  static constexpr int kAccPerTile = 1;
+  struct Params {
+    CUtensorMap tdyT, tgh;
+    RoutingTables rt;
+    const uint16_t* B;
+    const float* alpha;
+    float* dB;
+    float* dalpha_partial;
+    int N, r, E, bn, sstride, ntn;
+  };
+  struct Tile { int nt, e, ib, ie; };
+  __device__ static int num_tiles(const Params& p) { return p.ntn * p.E; }
+  __device__ static void tile_init(const Params& p, int i, Tile& t) {
+    t.e = i / p.ntn; t.nt = i % p.ntn;
+    t.ib = p.rt.expert_item_begin[t.e]; t.ie = p.rt.expert_item_begin[t.e + 1];
+  }
+  __device__ static int num_segments(const Params&, const Tile& t) { return t.ie - t.ib; }
+  __device__ static void segment(const Params& p, const Tile& t, int i, Segment& s) {
+    const int item = t.ib + i;
+    s.mode = MODE_BF_MM; s.acc = 0; s.bn = p.bn; s.ksteps = 4; s.nkb = 2;
+    s.ta = &p.tdyT; s.a_rank = 2; s.a_x = t.nt * 128; s.a_y = p.rt.items[item].x * 128; s.a_z = 0;
+    s.tb = &p.tgh; s.b_rank = 2; s.b_x = 0; s.b_y = item * 128; s.b_z = 0;
+    s.b_bytes = (p.bn / 64) * kMnBoxBytes;
+  }
+  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane) {
+    const int n = t.nt * 128 + quad * 32 + lane;
+    const bool live = n < p.N;
+    const bool has = t.ie > t.ib;
+    const float al = live ? p.alpha[n * p.sstride] : 0.f;
+    const long long rowoff = ((long long)t.e * p.N + (live ? n : 0)) * p.r;
+    float4* out = reinterpret_cast<float4*>(p.dB + rowoff);
+    const uint4* bin = reinterpret_cast<const uint4*>(p.B + rowoff);
+    float part = 0.f;
+    for (int c32 = 0; c32 * 32 < p.r; ++c32) {
+      uint32_t v[32];
+      tmem_ld32(taddr + c32 * 32, v);
+      tmem_ld_wait();
+      if (live) {
+#pragma unroll
+        for (int q8 = 0; q8 < 4; ++q8) {
+          if (c32 * 32 + q8 * 8 < p.r) {
+            const uint4 bv = __ldg(bin + c32 * 4 + q8);
+            const uint32_t bw[4] = {bv.x, bv.y, bv.z, bv.w};
+            float a[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) a[j] = has ? __uint_as_float(v[q8 * 8 + j]) : 0.f;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              part = fmaf(bf16lo(bw[j]), a[2 * j], part);
+              part = fmaf(bf16hi(bw[j]), a[2 * j + 1], part);
+            }
+            out[c32 * 8 + q8 * 2] = make_float4(al * a[0], al * a[1], al * a[2], al * a[3]);
+            out[c32 * 8 + q8 * 2 + 1] = make_float4(al * a[4], al * a[5], al * a[6], al * a[7]);
+          }
+        }
+      }
+    }
+    if (live) p.dalpha_partial[(long long)t.e * p.N + n] = part;
+  }
+};
+
+// ---------------------------------------------------------------------------
+// B5: dA_e = c * dhc^T . Xs over the items of expert e.
+// ---------------------------------------------------------------------------
+struct HpDaProblem {
+  static constexpr int kAccPerTile = 1;
+  struct Params {
+    CUtensorMap tdhT, txs;
+    RoutingTables rt;
+    const float* w_scales;
+    const float* beta;
+    float* dA;
+    int K, r, E, sstride, ntk;
+  };
+  struct Tile { int e, kt, ib, ie; };
+  __device__ static int num_tiles(const Params& p) { return p.ntk * p.E; }
+  __device__ static void tile_init(const Params& p, int i, Tile& t) {
+    t.e = i / p.ntk; t.kt = i % p.ntk;
+    t.ib = p.rt.expert_item_begin[t.e]; t.ie = p.rt.expert_item_begin[t.e + 1];
+  }
+  __device__ static int num_segments(const Params&, const Tile& t) { return t.ie - t.ib; }
+  __device__ static void segment(const Params& p, const Tile& t, int i, Segment& s) {
+    const int item = t.ib + i;
+    s.mode = MODE_BF_MM; s.acc = 0; s.bn = 256; s.ksteps = 4; s.nkb = 2;
+    s.ta = &p.tdhT; s.a_rank = 2; s.a_x = 0; s.a_y = item * 128; s.a_z = 0;
+    s.tb = &p.txs; s.b_rank = 2; s.b_x = t.kt * 256; s.b_y = p.rt.items[item].x * 128; s.b_z = 0;
+    s.b_bytes = kStageBBytes;
+  }
+  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane) {
+    const int j = quad * 32 + lane;
+    const bool live = j < p.r;
+    const bool has = t.ie > t.ib;
+    const float c = dx_scale(p.w_scales, p.beta, p.sstride);
+    const float cc = c != 0.f ? c : 1.0f;
+    float4* out = reinterpret_cast<float4*>(p.dA + ((long long)t.e * p.r + (live ? j : 0)) * p.K);
+    for (int c32 = 0; c32 < 8; ++c32) {
+      const int k0 = t.kt * 256 + c32 * 32;
+      if (k0 >= p.K) break;
+      uint32_t v[32];
+      tmem_ld32(taddr + c32 * 32, v);
+      tmem_ld_wait();
+      if (live) {
+#pragma unroll
+        for (int q4 = 0; q4 < 8; ++q4) {
+          float a[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) a[i] = has ? cc * __uint_as_float(v[q4 * 4 + i]) : 0.f;
+          out[(k0 >> 2) + q4] = make_float4(a[0], a[1], a[2], a[3]);
+        }
+      }
+    }
+  }
+};
+
+int gemm_backward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, const BwdBuffers& b, uint16_t* dX, float* dW, float* dA,
+                  float* dB, cudaStream_t st) {
+  const int mtiles = (a.T + 127) / 128;
+  const int ntk = (a.K + 255) / 256, ntn128 = (a.N + 127) / 128;
+  const bool hp = a.r > 0;
+  const int r64 = h_round_up(a.r, 64);
+  const uint64_t item_rows = (uint64_t)sv.max_items * 128;
+  int rc;
+  if (hp) {
+    HpDhProblem::Params p;
+    if (!map2d(&p.tdy, false, b.dys, a.N, a.T, 64, 128)) return PQ_ERR_CUDA;
+    if (!map3d(&p.tba, b.ba, a.r, a.N, a.E, 64, 64)) return PQ_ERR_CUDA;
+    p.rt = sv.rt; p.H = sv.h; p.gate = sv.gate; p.probs = sv.probs; p.w_scales = a.w_scales; p.alpha = a.alpha; p.beta = a.beta;
+    p.dhc = b.dhc; p.gh = b.gh; p.dl = b.dl; p.dlc = b.dlc;
+    p.T = a.T; p.N = a.N; p.r = a.r; p.E = a.E; p.bn = r64; p.sstride = a.scale_stride;
+    rc = launch_gemm<HpDhProblem>(p, sv.max_items, st);
+    if (rc) return rc;
+  }
+  {
+    BwdDxProblem::Params p;
+    if (!map2d(&p.tdy, false, b.dys, a.N, a.T, 64, 128)) return PQ_ERR_CUDA;
+    if (!map2d(&p.tsb, false, b.sb, a.K, a.N, 64, 64)) return PQ_ERR_CUDA;
+    p.tdh = p.tdy; p.ta3 = p.tdy; p.tdl = p.tdy; p.twr = p.tdy;
+    if (hp) {
+      if (!map2d(&p.tdh, false, b.dhc, a.r, item_rows, 64, 128)) return PQ_ERR_CUDA;
+      if (!map3d(&p.ta3, a.A, a.K, a.r, a.E, 64, 64)) return PQ_ERR_CUDA;
+    }
+    if (hp && a.E > 1) {
+      if (!map2d(&p.tdl, false, b.dlc, 16, a.T, 64, 128)) return PQ_ERR_CUDA;
+      if (!map2d(&p.twr, false, a.Wr, a.K, a.E, 64, 64)) return PQ_ERR_CUDA;
+    }
+    p.rt = sv.rt; p.perm = (hp && a.E > 1) ? sv.perm : nullptr; p.w_scales = a.w_scales; p.beta = a.beta; p.dX = dX;
+    p.T = a.T; p.N = a.N; p.K = a.K; p.r = a.r; p.E = hp ? a.E : 1; p.sstride = a.scale_stride; p.ntk = ntk;
+    rc = launch_gemm<BwdDxProblem>(p, mtiles * ntk, st);
+    if (rc) return rc;
+  }
+  {
+    BwdDwProblem::Params p;
+    if (!map2d(&p.tdyT, false, b.dys, a.N, a.T, 64, 64)) return PQ_ERR_CUDA;
+    if (!map2d(&p.txt, false, sv.xt, a.K, a.T, 64, 64)) return PQ_ERR_CUDA;
+    p.s8 = w_s8; p.beta = a.beta; p.dW = dW; p.dbeta_partial = b.dbeta_partial;
+    p.T = a.T; p.N = a.N; p.K = a.K; p.sstride = a.scale_stride; p.ntk = ntk;
+    rc = launch_gemm<BwdDwProblem>(p, ntn128 * ntk, st);
+    if (rc) return rc;
+  }
+  if (hp) {
+    HpDbProblem::Params p;
+    if (!map2d(&p.tdyT, false, b.dys, a.N, a.T, 64, 64)) return PQ_ERR_CUDA;
+    if (!map2d(&p.tgh, false, b.gh, a.r, item_rows, 64, 64)) return PQ_ERR_CUDA;
+    p.rt = sv.rt; p.B = a.B; p.alpha = a.alpha; p.dB = dB; p.dalpha_partial = b.dalpha_partial;
+    p.N = a.N; p.r = a.r; p.E = a.E; p.bn = r64; p.sstride = a.scale_stride; p.ntn = ntn128;
+    rc = launch_gemm<HpDbProblem>(p, ntn128 * a.E, st);
+    if (rc) return rc;
+    HpDaProblem::Params q;
+    if (!map2d(&q.tdhT, false, b.dhc, a.r, item_rows, 64, 64)) return PQ_ERR_CUDA;
+    if (!map2d(&q.txs, false, b.xs, a.K, a.T, 64, 64)) return PQ_ERR_CUDA;
+    q.rt = sv.rt; q.w_scales = a.w_scales; q.beta = a.beta; q.dA = dA;
+    q.K = a.K; q.r = a.r; q.E = a.E; q.sstride = a.scale_stride; q.ntk = ntk;
+    rc = launch_gemm<HpDaProblem>(q, ntk * a.E, st);
+    if (rc) return rc;
+  }
+  return PQ_OK;
+}
+
 }  // namespace pq

@@ -1,0 +1,85 @@
+"""GPU parity tests (backward side): straight-through gradients of the layer
+through the C ABI against the CPU oracle (App. B.1)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import pquant_oracle as O
+from paper_2602_22592_b200 import binding as pqb
+from paper_2602_22592_b200 import inputs as I
+from paper_2602_22592_b200.layer import PQLinear
+from test_gpu_forward import CASES, TOL_BF16, check_status, f32, rel_err
+
+pytestmark = pytest.mark.gpu
+
+
+def run_fwd_bwd(c, scale_vector):
+    L = PQLinear(c["T"], c["K"], c["N"], c["r"], c["E"], scale_vector=scale_vector).load_case(c)
+    L.pack()
+    L.forward()
+    L.backward()
+    torch.cuda.synchronize()
+    check_status()
+    return L
+
+
+def check_backward(c, L, f, g, scale_vector):
+    errs = {}
+    errs["dX"] = rel_err(f32(L.dX), g["dX"])
+    errs["dW"] = rel_err(f32(L.dW), g["dW"])
+    red = (lambda v: v) if scale_vector else (lambda v: np.array([v.sum()]))
+    errs["dbeta"] = rel_err(f32(L.dbeta), red(g["dbeta"]))
+    if c["r"] > 0:
+        errs["dA"] = rel_err(f32(L.dA), g["dA"])
+        errs["dB"] = rel_err(f32(L.dB), g["dB"])
+        errs["dalpha"] = rel_err(f32(L.dalpha), red(g["dalpha"]))
+        if c["E"] > 1:
+            errs["dWr"] = rel_err(f32(L.dWr), g["dWr"])
+    bad = {k: v for k, v in errs.items() if not v <= TOL_BF16}
+    assert not bad, f"gradients outside tolerance: {bad} (all: {errs})"
+    return errs
+
+
+BWD_CASES = dict(CASES)
+BWD_CASES["routed8_vec"] = dict(T=700, K=512, N=512, r=64, E=8, scale_vector=True, alpha=1.3, beta=0.6)
+
+
+@pytest.mark.parametrize("name", list(BWD_CASES))
+def test_backward_matches_oracle(name):
+    kw = dict(BWD_CASES[name])
+    sv = kw.pop("scale_vector", False)
+    c = I.make_linear_case(kw.pop("T"), kw.pop("K"), kw.pop("N"), kw.pop("r"), kw.pop("E"), seed=11, scale_vector=sv, **kw)
+    if sv:   # distinct per-feature scales so that a misplaced index shows
+        c["alpha"] = (c["alpha"] * np.linspace(0.8, 1.2, c["N"])).astype(np.float32)
+        c["beta"] = (c["beta"] * np.linspace(1.2, 0.8, c["N"])).astype(np.float32)
+    f = O.linear_forward(c["X"], c["W"], c["A"], c["B"], c["Wr"], c["alpha"], c["beta"])
+    g = O.linear_backward(c["dY"], c["X"], f, c["A"], c["B"], c["Wr"], c["alpha"], c["beta"])
+    L = run_fwd_bwd(c, sv)
+    check_backward(c, L, f, g, sv)
+
+
+def test_backward_empty_experts_and_zero_beta():
+    # experts 1 and 3 receive no token: their gradients must be exactly zero;
+    # beta = 0 switches the 1-bit input gradient off without dividing by zero
+    c = I.make_linear_case(300, 256, 256, 32, 4, seed=9, zipf=False, beta=0.0)
+    c["X"][7] = 0.0
+    c["Wr"][:] = 0.0
+    c["Wr"][2] = I.bf16_values(np.full(256, 0.5, np.float32))
+    c["X"] = I.bf16_values(np.abs(c["X"]))
+    f = O.linear_forward(c["X"], c["W"], c["A"], c["B"], c["Wr"], c["alpha"], c["beta"])
+    g = O.linear_backward(c["dY"], c["X"], f, c["A"], c["B"], c["Wr"], c["alpha"], c["beta"])
+    L = run_fwd_bwd(c, False)
+    assert torch.all(L.dA[1] == 0) and torch.all(L.dA[3] == 0) and torch.all(L.dB[1] == 0) and torch.all(L.dB[3] == 0)
+    assert torch.all(L.dW == 0)
+    errs = {k: rel_err(f32(getattr(L, k)), g[k]) for k in ("dX", "dA", "dB", "dWr")}
+    assert all(v <= TOL_BF16 for v in errs.values()), errs
+
+
+def test_backward_is_deterministic():
+    c = I.make_linear_case(512, 512, 512, 64, 4, seed=3)
+    L = run_fwd_bwd(c, False)
+    keep = [t.clone() for t in (L.dX, L.dW, L.dA, L.dB, L.dWr, L.dalpha, L.dbeta)]
+    L.backward()
+    torch.cuda.synchronize()
+    for a, b in zip(keep, (L.dX, L.dW, L.dA, L.dB, L.dWr, L.dalpha, L.dbeta)):
+        assert torch.equal(a, b)
