@@ -1,0 +1,364 @@
+#!/usr/bin/env python
+"""Benchmark of the pQuant decoupled linear layer (pack + forward + STE backward).
+
+One "step" = the whole hot path over one batch of synthetic input: for each of
+the three 1.3B-shaped MLP projections (gate, up: 2048->5632; down: 5632->2048;
+8192 tokens, HP width 128) re-quantise the latent weights (pq_pack_weights),
+run pq_linear_forward and pq_linear_backward.  Metric: tokens/s.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload mlp_dense|mlp_e8|decode]
+  python bench.py --impl reference ...      # the CPU oracle on the host cores
+
+Prints ONE JSON line (rank 0).  With N > 1 (torchrun) every rank runs an
+independent replica of the workload on its own GPU -- the layer has no
+inter-GPU exchange -- and the slowest rank's time is used.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+METRIC = "pQuant linear fwd+bwd tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the
+# committed ncu capture (profiles/); None until a capture of this kernel exists.
+NCU_TRAFFIC_BYTES = {"bwd_dw": None}
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return d, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs (read only)."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thr = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {"hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+                 "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+                 "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+                 "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4)}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                get = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or nv.nvmlDeviceGetCurrentClocksThrottleReasons
+                mask = get(self.h)
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(0.02)
+
+    def __enter__(self):
+        if self.nv:
+            self._thr = threading.Thread(target=self._run, daemon=True)
+            self._thr.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thr:
+            self._thr.join()
+
+    def summary(self):
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# --------------------------------------------------------------------------- workloads
+def build_mlp(E: int, device, T=None):
+    from paper_2602_22592_b200 import inputs as I
+    from paper_2602_22592_b200.layer import PQLinear
+    cases = I.config_mlp(E, seed=1 if E == 1 else 2, T=T)
+    layers = []
+    for c in cases:
+        L = PQLinear(c["T"], c["K"], c["N"], c["r"], c["E"], device=device).load_case(c)
+        L.name = c["name"]
+        layers.append(L)
+    return layers, cases
+
+
+def step_device(layers):
+    for L in layers:
+        L.pack()
+        L.forward()
+        L.backward()
+
+
+def roofline_time_s(layers, peaks):
+    """t_min = 2TNK / P_i8 + (4TNK + 6Tr(K+N)) / P_bf16 with P_i8 = 2 P_bf16 (nominal ratio)."""
+    pb = peaks["bf16_tflops_sustained"] * 1e12
+    t = 0.0
+    for L in layers:
+        tnk = L.T * L.N * L.K
+        t += 2 * tnk / (2 * pb) + (4 * tnk + 6 * L.T * L.r * (L.K + L.N)) / pb
+    return t
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2602_22592_b200 import binding as pqb
+    from paper_2602_22592_b200 import build as pqbuild
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback for the product path")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+    if rank == 0:
+        pqbuild.build()
+    if world > 1:
+        dist.barrier()
+    pqb.lib()
+    peaks, peak_kind = measured_peaks()
+
+    E = 8 if args.workload == "mlp_e8" else 1
+    layers, cases = build_mlp(E, device)
+    tokens = layers[0].T
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step_device(layers)
+    barrier()
+    code, where = pqb.pq_device_status()
+    if code:
+        raise RuntimeError(f"device-side wait timed out during warm-up (where={where})")
+
+    # dominant kernel: the dW GEMM (contraction over tokens), timed live with events on the launch stream
+    kid = pqb.KERNEL_IDS["bwd_dw"]
+    ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in layers] for _ in range(args.steps)]
+    for row in ev:
+        for a, b in row:
+            a.record(); b.record()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = pqb.pq_kernel_launches()
+    barrier()
+    with ClockSampler(local) as clk:
+        t0.record()
+        for s in range(args.steps):
+            for i, L in enumerate(layers):
+                L.pack()
+                L.forward()
+                pqb.pq_profile_events(kid, *ev[s][i])
+                L.backward()
+        t1.record()
+        barrier()
+    pqb.pq_profile_events(kid, None, None)
+    launches = pqb.pq_kernel_launches() - launches0
+    elapsed_ms = t0.elapsed_time(t1)
+    if world > 1:
+        tt = torch.tensor([elapsed_ms], device=device)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(tt.item())
+    code, where = pqb.pq_device_status()
+    if code:
+        raise RuntimeError(f"device-side wait timed out (where={where})")
+    ms_per_step = elapsed_ms / args.steps
+    value = world * tokens / (ms_per_step * 1e-3)
+
+    dw_ms = float(np.mean([a.elapsed_time(b) for row in ev for a, b in row]))
+    dw_flops = float(np.mean([2.0 * L.T * L.N * L.K for L in layers]))
+    achieved = dw_flops / (dw_ms * 1e-3) / 1e12
+    peak = peaks["bf16_tflops_sustained"]
+    roofline = {"kernel": "bwd_dw (dW = dY^T . q/gamma, bf16 tcgen05, fp32 accumulate)", "bound": "tensor",
+                "achieved": round(achieved, 1), "peak": peak, "unit": "TFLOP/s", "frac": round(achieved / peak, 4),
+                "peak_source": f"{peak_kind} bf16_tflops_sustained", "avg_launch_ms": round(dw_ms, 4),
+                "traffic": NCU_TRAFFIC_BYTES["bwd_dw"]}
+    t_min = roofline_time_s(layers, peaks)
+    layer_frac = t_min / (ms_per_step * 1e-3)
+
+    # per-kernel breakdown of one extra (untimed) step
+    names = ["pack_sums", "binarize_pack", "router", "route_scan", "act_quant", "hp_up", "fwd", "scatter_rows", "scaled_sign",
+             "hp_dh", "bwd_dx", "bwd_dw", "hp_db", "hp_da", "router_wgrad"]
+    bev = {n: (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for n in names}
+    breakdown = {n: 0.0 for n in names}
+    for L in layers:
+        for n, (a, b) in bev.items():
+            a.record(); b.record()
+            pqb.pq_profile_events(pqb.KERNEL_IDS[n], a, b)
+        L.pack(); L.forward(); L.backward()
+        torch.cuda.synchronize()
+        for n, (a, b) in bev.items():
+            breakdown[n] += a.elapsed_time(b) * 1e3
+    for n in names:
+        pqb.pq_profile_events(pqb.KERNEL_IDS[n], None, None)
+    breakdown = {n: round(v, 1) for n, v in breakdown.items() if v > 0.5}
+
+    # end to end: inputs come from pinned host memory and results go back, every step
+    e2e = None
+    if not args.no_e2e:
+        hx = [L.X.cpu().pin_memory() for L in layers]
+        hdy = [L.dY.cpu().pin_memory() for L in layers]
+        hy = [torch.empty_like(L.Y, device="cpu").pin_memory() for L in layers]
+        hdx = [torch.empty_like(L.dX, device="cpu").pin_memory() for L in layers]
+
+        def step_e2e():
+            for i, L in enumerate(layers):
+                L.X.copy_(hx[i], non_blocking=True)
+                L.dY.copy_(hdy[i], non_blocking=True)
+                L.pack(); L.forward(); L.backward()
+                hy[i].copy_(L.Y, non_blocking=True)
+                hdx[i].copy_(L.dX, non_blocking=True)
+
+        n_e2e = max(3, min(args.steps, 10))
+        for _ in range(2):
+            step_e2e()
+        barrier()
+        t0.record()
+        for _ in range(n_e2e):
+            step_e2e()
+        t1.record()
+        barrier()
+        ms = t0.elapsed_time(t1)
+        if world > 1:
+            tt = torch.tensor([ms], device=device)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            ms = float(tt.item())
+        bi = sum(t.numel() * t.element_size() for t in hx + hdy)
+        bo = sum(t.numel() * t.element_size() for t in hy + hdx)
+        e2e = {"value": round(world * tokens / (ms / n_e2e * 1e-3), 1), "unit": "tokens/s", "h2d_bytes_per_step": bi,
+               "d2h_bytes_per_step": bo, "steps": n_e2e,
+               "note": "X and dY of each projection copied from pinned host memory, Y and dX copied back; weights stay resident"}
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        cpu_baseline = oracle_baseline(E, sample_tokens=args.cpu_tokens)
+
+    if rank == 0:
+        out = {
+            "metric": METRIC, "value": round(value, 1), "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "int8 x int8 -> int32 (forward 1-bit branch); bf16 -> fp32 (HP branch, backward)",
+            "data": "synthetic",
+            "config": {"workload": ("1.3B LLaMA MLP projections gate/up/down as pQuant linears, 8192 tokens, hidden 2048, FFN 5632, "
+                                    f"HP width 128, {E} expert(s)" + (", Zipf(1.1) routing" if E > 1 else "")),
+                       "tokens_per_step": tokens, "l2": "inputs larger than L2 (each projection moves > 400 MB per step)",
+                       "replicas": world},
+            "roofline": roofline,
+            "layer_roofline": {"t_min_ms": round(t_min * 1e3, 4), "frac": round(layer_frac, 4),
+                               "formula": "2TNK/P_i8 + (4TNK + 6Tr(K+N))/P_bf16, P_i8 = 2 P_bf16, sustained bf16 peak"},
+            "breakdown_us_per_step": breakdown,
+            "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": int(launches),
+            "clocks": clk.summary(),
+        }
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# --------------------------------------------------------------------------- oracle (CPU) arm
+def oracle_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info()]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def oracle_step(cases, sample_tokens):
+    """The oracle as it stands on the first `sample_tokens` tokens of each projection."""
+    from oracle import pquant_oracle as O
+    for c in cases:
+        X, dY = c["X"][:sample_tokens], c["dY"][:sample_tokens]
+        f = O.linear_forward(X, c["W"], c["A"], c["B"], c["Wr"], c["alpha"], c["beta"])
+        O.linear_backward(dY, X, f, c["A"], c["B"], c["Wr"], c["alpha"], c["beta"])
+
+
+def oracle_baseline(E, sample_tokens):
+    from paper_2602_22592_b200 import inputs as I
+    cases = I.config_mlp(E, seed=1 if E == 1 else 2, T=sample_tokens)
+    t = time.perf_counter()
+    oracle_step(cases, sample_tokens)
+    dt = time.perf_counter() - t
+    return {"value": round(sample_tokens / dt, 1), "unit": "tokens/s", "cores": oracle_threads(), "kind": "oracle",
+            "sample": (f"first {sample_tokens} of 8192 tokens through pack + forward + backward of the three projections "
+                       f"({dt:.1f} s; the per-matrix weight quantisation does not shrink with the sample, so this understates "
+                       "the full-batch rate)")}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2602_22592_b200 import inputs as I
+    E = 8 if args.workload == "mlp_e8" else 1
+    T = args.cpu_tokens
+    cases = I.config_mlp(E, seed=1 if E == 1 else 2, T=T)
+    for _ in range(min(args.warmup, 1)):
+        oracle_step(cases, T)
+    steps = max(1, min(args.steps, 5))
+    t = time.perf_counter()
+    for _ in range(steps):
+        oracle_step(cases, T)
+    dt = (time.perf_counter() - t) / steps
+    value = round(T / dt, 1)
+    out = {"impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+           "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": round(dt * 1e3, 2), "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+           "config": {"workload": f"1.3B LLaMA MLP projections as pQuant linears, {E} expert(s); CPU oracle on a {T}-token sample per step"},
+           "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": oracle_threads(), "kind": "oracle",
+                            "sample": f"{T} of 8192 tokens per step"},
+           "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(out))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="mlp_dense", choices=["mlp_dense", "mlp_e8"])
+    ap.add_argument("--cpu-tokens", type=int, default=4096)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -82,7 +82,8 @@ typedef struct pq_saved_view {
   int32_t* perm;      /* [T]    perm[p] = token at sorted position p                   */
   int32_t* pos;       /* [T]    inverse: pos[token] = p                                */
   int32_t* offsets;   /* [E+1]  sorted positions of expert e: offsets[e]..offsets[e+1] */
-  uint16_t* h;        /* [max_items*128, r] bf16 HP hidden activations, one 128-row block per item */
+  uint16_t* h;        /* [2][max_items*128, r] bf16 HP hidden activations as hi/lo planes (h = hi + lo),
+                         one 128-row block per item in each plane */
   /* Item table.  An item is the intersection of one 128-row tile of the sorted
    * order with one expert's range; rows of an item's block outside that range
    * are zero.  items[i] = {tile, expert, first row, end row} (rows relative to
@@ -148,6 +149,18 @@ int pq_debug_gemm(int mode, int M, int N, int K, const void* A, const void* B, v
  * Synchronises `stream`.  code = 0 when no wait failed; `where` identifies the
  * waiting role.  The word is cleared by the call. */
 int pq_device_status(void* stream, int* code, int* where);
+
+/* Cumulative number of kernels this library has launched in this process. */
+long long pq_kernel_launches(void);
+
+/* Measurement hook: from now on, every launch of the kernel with this id is
+ * bracketed by cudaEventRecord(start_event) / cudaEventRecord(stop_event) on
+ * the launching stream (both cudaEvent_t passed as void*; NULL, NULL clears).
+ * Ids: 0 weight sums, 1 binarize+pack, 2 router, 3 expert scan, 4 activation
+ * quantise, 5 HP up-projection, 6 fused forward tile, 7 row scatter, 8 scaled
+ * sign, 9 scaled B, 10 HP dH, 11 dX, 12 dW, 13 HP dB, 14 HP dA, 15 router
+ * weight gradient, 16 partial sums, 17 scalar sum, 18 debug GEMM. */
+int pq_profile_events(int kernel_id, void* start_event, void* stop_event);
 
 const char* pq_status_string(int status);
 

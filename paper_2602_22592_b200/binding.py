@@ -22,7 +22,11 @@ PQ_PHASE_PACK, PQ_PHASE_FWD, PQ_PHASE_BWD, PQ_PHASE_DECODE = 0, 1, 2, 3
 
 EXPORTS = ("pq_status_string", "pq_workspace_bytes", "pq_saved_bytes", "pq_saved_view_init",
            "pq_pack_weights", "pq_linear_forward", "pq_linear_backward", "pq_debug_gemm",
-           "pq_device_status")
+           "pq_device_status", "pq_kernel_launches", "pq_profile_events")
+
+KERNEL_IDS = dict(pack_sums=0, binarize_pack=1, router=2, route_scan=3, act_quant=4, hp_up=5, fwd=6, scatter_rows=7,
+                  scaled_sign=8, scaled_b=9, hp_dh=10, bwd_dx=11, bwd_dw=12, hp_db=13, hp_da=14, router_wgrad=15,
+                  sum_partials=16, sum_scalar=17, debug=18, decode_prep=19, decode_main=20)
 
 
 class PqError(RuntimeError):
@@ -73,6 +77,10 @@ def lib() -> ctypes.CDLL:
         L.pq_debug_gemm.argtypes = [ci, ci, ci, ci, vp, vp, vp, vp]
         L.pq_device_status.restype = ci
         L.pq_device_status.argtypes = [vp, ctypes.POINTER(ci), ctypes.POINTER(ci)]
+        L.pq_kernel_launches.restype = ctypes.c_longlong
+        L.pq_kernel_launches.argtypes = []
+        L.pq_profile_events.restype = ci
+        L.pq_profile_events.argtypes = [ci, vp, vp]
         _lib = L
     return _lib
 
@@ -134,7 +142,7 @@ def pq_saved_view_init(d: pq_desc, saved: torch.Tensor) -> dict:
         gate=view(v.gate, torch.float32, d.T), probs=view(v.probs, torch.float32, d.T, E),
         expert=view(v.expert, torch.int32, d.T), perm=view(v.perm, torch.int32, d.T),
         pos=view(v.pos, torch.int32, d.T), offsets=view(v.offsets, torch.int32, E + 1),
-        h=view(v.h, torch.bfloat16, v.max_items * 128, d.r) if d.r > 0 else None,
+        h=view(v.h, torch.bfloat16, 2, v.max_items * 128, d.r) if d.r > 0 else None,
         n_items=view(v.n_items, torch.int32, 1), items=view(v.items, torch.int32, v.max_items, 4),
         tile_item_begin=view(v.tile_item_begin, torch.int32, mt + 1),
         expert_item_begin=view(v.expert_item_begin, torch.int32, E + 1), max_items=v.max_items)
@@ -167,3 +175,16 @@ def pq_device_status(stream=None) -> tuple[int, int]:
     code, where = ctypes.c_int(0), ctypes.c_int(0)
     _check("pq_device_status", lib().pq_device_status(_stream(stream), ctypes.byref(code), ctypes.byref(where)))
     return code.value, where.value
+
+
+def pq_kernel_launches() -> int:
+    return lib().pq_kernel_launches()
+
+
+def pq_profile_events(kernel_id: int, start: "torch.cuda.Event | None", stop: "torch.cuda.Event | None"):
+    """Bracket every later launch of kernel `kernel_id` with the two events (None, None clears).
+    The events must have been created with enable_timing=True and recorded once already
+    (torch creates the underlying cudaEvent lazily)."""
+    s = None if start is None else ctypes.c_void_p(start.cuda_event)
+    e = None if stop is None else ctypes.c_void_p(stop.cuda_event)
+    _check("pq_profile_events", lib().pq_profile_events(kernel_id, s, e))

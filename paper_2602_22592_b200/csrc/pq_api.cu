@@ -54,7 +54,7 @@ static size_t carve_saved(const pq_desc* d, void* base, SavedPtrs* out) {
   s.perm = c.take<int>(T);
   s.pos = c.take<int>(T);
   s.offsets = c.take<int>(E + 1);
-  s.h = d->r > 0 ? c.take<uint16_t>((size_t)s.max_items * kTileRows * d->r) : nullptr;
+  s.h = d->r > 0 ? c.take<uint16_t>((size_t)2 * s.max_items * kTileRows * d->r) : nullptr;  // hi and lo planes
   s.rt.n_items = c.take<int>(1);
   s.rt.items = c.take<int4>(s.max_items);
   s.rt.tile_item_begin = c.take<int>(mtiles_of(d) + 1);
@@ -100,8 +100,8 @@ static size_t carve_bwd_scratch(const pq_desc* d, void* base, BwdScratch* out) {
   s.dys = routed(d) ? c.take<uint16_t>(T * N) : nullptr;
   s.sb = c.take<uint16_t>(N * K);
   s.ba = (r > 0 && vec) ? c.take<uint16_t>((size_t)E * N * r) : nullptr;
-  s.dhc = r > 0 ? c.take<uint16_t>((size_t)max_items_of(d) * kTileRows * r) : nullptr;
-  s.gh = r > 0 ? c.take<uint16_t>((size_t)max_items_of(d) * kTileRows * r) : nullptr;
+  s.dhc = r > 0 ? c.take<uint16_t>((size_t)2 * max_items_of(d) * kTileRows * r) : nullptr;
+  s.gh = r > 0 ? c.take<uint16_t>((size_t)2 * max_items_of(d) * kTileRows * r) : nullptr;
   s.dl = routed(d) ? c.take<float>(T * E) : nullptr;
   s.dlc = routed(d) ? c.take<uint16_t>(T * 16) : nullptr;
   s.dbeta_partial = c.take<float>(((K + 255) / 256) * N);
@@ -278,6 +278,15 @@ int pq_debug_gemm(int mode, int M, int N, int K, const void* A, const void* B, v
   if (M < 1 || N < 1 || K < 1 || M % 8 || N % 8 || K % (mode == 0 ? 16 : 8)) return PQ_ERR_SHAPE;
   if (misaligned(A) || misaligned(B) || misaligned(D)) return PQ_ERR_ALIGN;
   return gemm_debug(mode, M, N, K, A, B, D, static_cast<cudaStream_t>(stream));
+}
+
+long long pq_kernel_launches(void) { return g_launches; }
+
+int pq_profile_events(int kernel_id, void* start_event, void* stop_event) {
+  if (kernel_id < 0 || kernel_id >= KID_COUNT) return PQ_ERR_SHAPE;
+  g_profile[kernel_id].start = static_cast<cudaEvent_t>(start_event);
+  g_profile[kernel_id].stop = static_cast<cudaEvent_t>(stop_event);
+  return PQ_OK;
 }
 
 int pq_device_status(void* stream, int* code, int* where) {

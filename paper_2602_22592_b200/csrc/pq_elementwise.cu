@@ -6,6 +6,9 @@
 
 namespace pq {
 
+ProfileSlot g_profile[KID_COUNT] = {};
+long long g_launches = 0;
+
 // ---------------------------------------------------------------------------
 // K2a: partial sums of W and |W| in fp64 (Eq. 6).  Fixed grid and a fixed
 // reduction tree, so the result does not depend on scheduling.
@@ -420,8 +423,10 @@ static inline int grid_for(long long work, int per_block, int cap) {
 cudaError_t launch_pack(const float* W, int N, int K, uint32_t* bits, int8_t* s8, float* scales, double* partial, cudaStream_t st) {
   const long long n4 = (long long)N * K / 4;
   const int nparts = grid_for(n4, 256 * 8, kPackPartials);
-  k_weight_partial_sums<<<nparts, 256, 0, st>>>(reinterpret_cast<const float4*>(W), n4, partial);
+  { LaunchScope ls(KID_PACK_SUMS, st);
+  k_weight_partial_sums<<<nparts, 256, 0, st>>>(reinterpret_cast<const float4*>(W), n4, partial); }
   const int grid = grid_for(n4, 256 * 4, 148 * 8);
+  LaunchScope ls(KID_BINARIZE_PACK, st);
   k_binarize_pack<<<grid, 256, 0, st>>>(reinterpret_cast<const float4*>(W), n4, partial, nparts, 1.0 / ((double)N * K), bits,
                                         reinterpret_cast<uint32_t*>(s8), scales);
   return cudaGetLastError();
@@ -431,10 +436,13 @@ cudaError_t launch_route_and_quant(const uint16_t* X, const uint16_t* Wr, int T,
                                    cudaStream_t st) {
   const int nblocks = (T + kRouterTokensPerBlock - 1) / kRouterTokensPerBlock;
   if (E > 1) {
+    LaunchScope ls(KID_ROUTER, st);
     k_router<<<nblocks, 256, 0, st>>>(reinterpret_cast<const uint4*>(X), reinterpret_cast<const uint4*>(Wr), T, K, E, sv.expert, sc.gate_tok,
                                       sc.probs_tok, sc.block_counts);
   }
-  k_route_scan<<<1, 32, 0, st>>>(T, E, nblocks, sc.block_counts, sc.block_base, sv.offsets, sv.rt);
+  { LaunchScope ls(KID_ROUTE_SCAN, st);
+  k_route_scan<<<1, 32, 0, st>>>(T, E, nblocks, sc.block_counts, sc.block_base, sv.offsets, sv.rt); }
+  LaunchScope ls(KID_ACT_QUANT, st);
   k_act_quant<<<(T + 7) / 8, 256, 0, st>>>(reinterpret_cast<const uint4*>(X), T, K, E, sv.expert, sc.block_base, sv.offsets, sc.gate_tok,
                                            sc.probs_tok, reinterpret_cast<uint2*>(sv.q), reinterpret_cast<uint4*>(sv.xt),
                                            reinterpret_cast<uint4*>(sv.xs), sv.gamma, sv.gate, sv.probs, sv.perm, sv.pos);
@@ -442,12 +450,14 @@ cudaError_t launch_route_and_quant(const uint16_t* X, const uint16_t* Wr, int T,
 }
 
 cudaError_t launch_scatter_rows(const uint16_t* src, uint16_t* dst, const int* pos, int T, int row_elems, cudaStream_t st) {
+  LaunchScope ls(KID_SCATTER_ROWS, st);
   k_scatter_rows<<<(T + 7) / 8, 256, 0, st>>>(reinterpret_cast<const uint4*>(src), reinterpret_cast<uint4*>(dst), pos, T, row_elems / 8);
   return cudaGetLastError();
 }
 
 cudaError_t launch_scaled_sign(const int8_t* s8, uint16_t* out, const float* beta, int beta_stride, int N, int K, cudaStream_t st) {
   const long long n16 = (long long)N * K / 16;
+  LaunchScope ls(KID_SCALED_SIGN, st);
   k_scaled_sign<<<grid_for(n16, 256 * 2, 148 * 8), 256, 0, st>>>(reinterpret_cast<const uint4*>(s8), reinterpret_cast<uint4*>(out), beta,
                                                                beta_stride, N, K);
   return cudaGetLastError();
@@ -455,6 +465,7 @@ cudaError_t launch_scaled_sign(const int8_t* s8, uint16_t* out, const float* bet
 
 cudaError_t launch_scaled_b(const uint16_t* B, uint16_t* out, const float* alpha, int E, int N, int r, cudaStream_t st) {
   const long long n2 = (long long)E * N * r / 2;
+  LaunchScope ls(KID_SCALED_B, st);
   k_scaled_b<<<grid_for(n2, 256 * 4, 148 * 8), 256, 0, st>>>(reinterpret_cast<const uint32_t*>(B), reinterpret_cast<uint32_t*>(out), alpha, E, N, r);
   return cudaGetLastError();
 }
@@ -463,17 +474,21 @@ cudaError_t launch_router_wgrad(const uint16_t* xs, const float* dl, int T, int 
                                 cudaStream_t st) {
   const int chunks = (T + 255) / 256;
   dim3 grid((K / 2 + 127) / 128, chunks);
-  k_router_wgrad_partial<<<grid, 128, 0, st>>>(reinterpret_cast<const uint32_t*>(xs), dl, T, K, E, partial);
+  { LaunchScope ls(KID_ROUTER_WGRAD, st);
+  k_router_wgrad_partial<<<grid, 128, 0, st>>>(reinterpret_cast<const uint32_t*>(xs), dl, T, K, E, partial); }
+  LaunchScope ls(KID_SUM_PARTIALS, st);
   k_sum_partials<<<(E * K + 255) / 256, 256, 0, st>>>(partial, chunks, E * K, scale, dWr);
   return cudaGetLastError();
 }
 
 cudaError_t launch_sum_partials(const float* partial, int nparts, int n, const float* scale, float* out, cudaStream_t st) {
+  LaunchScope ls(KID_SUM_PARTIALS, st);
   k_sum_partials<<<(n + 255) / 256, 256, 0, st>>>(partial, nparts, n, scale, out);
   return cudaGetLastError();
 }
 
 cudaError_t launch_sum_to_scalar(const float* v, int n, float* out, cudaStream_t st) {
+  LaunchScope ls(KID_SUM_SCALAR, st);
   k_sum_to_scalar<<<1, 1024, 0, st>>>(v, n, out);
   return cudaGetLastError();
 }

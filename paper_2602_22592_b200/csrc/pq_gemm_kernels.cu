@@ -79,7 +79,7 @@ static int sm_count() {
 }
 
 template <class P>
-static int launch_gemm(const typename P::Params& p, int max_tiles, cudaStream_t st) {
+static int launch_gemm(int kernel_id, const typename P::Params& p, int max_tiles, cudaStream_t st) {
   static bool configured = false;
   if (!configured) {
     if (cudaFuncSetAttribute(gemm_kernel<P>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes) != cudaSuccess) return PQ_ERR_CUDA;
@@ -87,11 +87,22 @@ static int launch_gemm(const typename P::Params& p, int max_tiles, cudaStream_t 
   }
   int grid = max_tiles < sm_count() ? max_tiles : sm_count();
   if (grid < 1) grid = 1;
+  LaunchScope ls(kernel_id, st);
   gemm_kernel<P><<<grid, kGemmThreads, kGemmSmemBytes, st>>>(p);
   return cudaGetLastError() == cudaSuccess ? PQ_OK : PQ_ERR_CUDA;
 }
 
 __device__ __forceinline__ int round_up(int x, int m) { return (x + m - 1) / m * m; }
+
+// Intermediates that feed a second tensor-core product (H, g H, dH / c) are kept
+// as TWO bf16 planes, v ~= hi + lo with hi = bf16(v), lo = bf16(v - hi): about 16
+// significand bits, so their rounding does not show in the results.  The planes
+// are stacked along the row axis ([2][item_rows][r]); a product against such an
+// operand simply runs its contraction over both planes.
+__device__ __forceinline__ void split2(float a, float b, uint32_t& hi, uint32_t& lo) {
+  hi = pack_bf16x2(a, b);
+  lo = pack_bf16x2(a - bf16lo(hi), b - bf16hi(hi));
+}
 static inline int h_round_up(int x, int m) { return (x + m - 1) / m * m; }
 
 // ---------------------------------------------------------------------------
@@ -156,7 +167,7 @@ int gemm_debug(int mode, int M, int N, int K, const void* A, const void* B, void
       return PQ_ERR_UNSUPPORTED;
   }
   if (!ok) return PQ_ERR_CUDA;
-  return launch_gemm<DebugProblem>(p, ((M + 127) / 128) * p.ntn, st);
+  return launch_gemm<DebugProblem>(KID_DEBUG, p, ((M + 127) / 128) * p.ntn, st);
 }
 
 // ---------------------------------------------------------------------------
@@ -168,7 +179,7 @@ struct HpUpProblem {
     CUtensorMap tx, ta;  // X sorted [T,K]; A [E,r,K]
     RoutingTables rt;
     uint16_t* H;
-    int K, r, bn;
+    int K, r, bn, item_rows;
   };
   struct Tile { int item; int4 it; };
   __device__ static int num_tiles(const Params& p) { return p.rt.n_items[0]; }
@@ -183,7 +194,8 @@ struct HpUpProblem {
   __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane) {
     const int row = quad * 32 + lane;
     const bool live = row >= t.it.z && row < t.it.w;
-    uint4* out = reinterpret_cast<uint4*>(p.H + ((long long)t.item * 128 + row) * p.r);
+    uint4* out_hi = reinterpret_cast<uint4*>(p.H + ((long long)t.item * 128 + row) * p.r);
+    uint4* out_lo = reinterpret_cast<uint4*>(p.H + ((long long)p.item_rows + t.item * 128 + row) * p.r);
     for (int c = 0; c * 32 < p.r; ++c) {
       uint32_t v[32];
       tmem_ld32(taddr + c * 32, v);
@@ -191,14 +203,13 @@ struct HpUpProblem {
 #pragma unroll
       for (int g = 0; g < 4; ++g) {
         if (c * 32 + g * 8 < p.r) {
-          uint4 o = make_uint4(0, 0, 0, 0);
+          uint32_t hi[4] = {0, 0, 0, 0}, lo[4] = {0, 0, 0, 0};
           if (live) {
-            o.x = pack_bf16x2(__uint_as_float(v[8 * g + 0]), __uint_as_float(v[8 * g + 1]));
-            o.y = pack_bf16x2(__uint_as_float(v[8 * g + 2]), __uint_as_float(v[8 * g + 3]));
-            o.z = pack_bf16x2(__uint_as_float(v[8 * g + 4]), __uint_as_float(v[8 * g + 5]));
-            o.w = pack_bf16x2(__uint_as_float(v[8 * g + 6]), __uint_as_float(v[8 * g + 7]));
+#pragma unroll
+            for (int j = 0; j < 4; ++j) split2(__uint_as_float(v[8 * g + 2 * j]), __uint_as_float(v[8 * g + 2 * j + 1]), hi[j], lo[j]);
           }
-          out[c * 4 + g] = o;
+          out_hi[c * 4 + g] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+          out_lo[c * 4 + g] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
         }
       }
     }
@@ -223,7 +234,7 @@ struct FwdProblem {
     const float* alpha;
     const float* beta;
     uint16_t* Y;
-    int T, N, K, r, sstride, ntn;
+    int T, N, K, r, sstride, ntn, item_rows;
   };
   struct Tile { int m, n, ib, ie; };
   __device__ static int num_tiles(const Params& p) { return ((p.T + 127) / 128) * p.ntn; }
@@ -231,7 +242,7 @@ struct FwdProblem {
     t.m = i / p.ntn; t.n = i % p.ntn;
     if (HP) { t.ib = p.rt.tile_item_begin[t.m]; t.ie = p.rt.tile_item_begin[t.m + 1]; } else { t.ib = t.ie = 0; }
   }
-  __device__ static int num_segments(const Params&, const Tile& t) { return 1 + (t.ie - t.ib); }
+  __device__ static int num_segments(const Params&, const Tile& t) { return 1 + 2 * (t.ie - t.ib); }
   __device__ static void segment(const Params& p, const Tile& t, int i, Segment& s) {
     s.bn = 256; s.ksteps = 4; s.a_z = 0; s.b_z = 0; s.b_bytes = kStageBBytes;
     if (i == 0) {
@@ -239,10 +250,10 @@ struct FwdProblem {
       s.ta = &p.tq; s.a_rank = 2; s.a_x = 0; s.a_y = t.m * 128;
       s.tb = &p.ts; s.b_rank = 2; s.b_x = 0; s.b_y = t.n * 256;
     } else {
-      const int item = t.ib + i - 1;
+      const int item = t.ib + ((i - 1) >> 1), plane = (i - 1) & 1;
       const int e = p.rt.items[item].y;
       s.mode = MODE_BF_KK; s.acc = 1; s.nkb = (p.r + 63) / 64;
-      s.ta = &p.th; s.a_rank = 2; s.a_x = 0; s.a_y = item * 128;
+      s.ta = &p.th; s.a_rank = 2; s.a_x = 0; s.a_y = plane * p.item_rows + item * 128;
       s.tb = &p.tb; s.b_rank = 3; s.b_x = 0; s.b_y = t.n * 256; s.b_z = e;
     }
   }
@@ -284,20 +295,20 @@ int gemm_forward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, co
   const bool hp = a.r > 0;
   if (hp) {
     HpUpProblem::Params p;
-    p.rt = sv.rt; p.H = sv.h; p.K = a.K; p.r = a.r; p.bn = h_round_up(a.r, 16);
+    p.rt = sv.rt; p.H = sv.h; p.K = a.K; p.r = a.r; p.bn = h_round_up(a.r, 16); p.item_rows = sv.max_items * 128;
     if (!map2d(&p.tx, false, xs, a.K, a.T, 64, 128)) return PQ_ERR_CUDA;
     if (!map3d(&p.ta, a.A, a.K, a.r, a.E, 64, p.bn)) return PQ_ERR_CUDA;
-    int rc = launch_gemm<HpUpProblem>(p, sv.max_items, st);
+    int rc = launch_gemm<HpUpProblem>(KID_HP_UP, p, sv.max_items, st);
     if (rc) return rc;
     FwdProblem<true>::Params f;
     if (!map2d(&f.tq, true, sv.q, a.K, a.T, 128, 128)) return PQ_ERR_CUDA;
     if (!map2d(&f.ts, true, w_s8, a.K, a.N, 128, 256)) return PQ_ERR_CUDA;
-    if (!map2d(&f.th, false, sv.h, a.r, (uint64_t)sv.max_items * 128, 64, 128)) return PQ_ERR_CUDA;
+    if (!map2d(&f.th, false, sv.h, a.r, (uint64_t)sv.max_items * 256, 64, 128)) return PQ_ERR_CUDA;
     if (!map3d(&f.tb, a.B, a.r, a.N, a.E, 64, 256)) return PQ_ERR_CUDA;
     f.rt = sv.rt; f.perm = a.E > 1 ? sv.perm : nullptr; f.gamma = sv.gamma; f.gate = sv.gate; f.w_scales = a.w_scales;
     f.alpha = a.alpha; f.beta = a.beta; f.Y = Y; f.T = a.T; f.N = a.N; f.K = a.K; f.r = a.r; f.sstride = a.scale_stride;
-    f.ntn = (a.N + 255) / 256;
-    return launch_gemm<FwdProblem<true>>(f, mtiles * f.ntn, st);
+    f.ntn = (a.N + 255) / 256; f.item_rows = sv.max_items * 128;
+    return launch_gemm<FwdProblem<true>>(KID_FWD, f, mtiles * f.ntn, st);
   }
   FwdProblem<false>::Params f;
   if (!map2d(&f.tq, true, sv.q, a.K, a.T, 128, 128)) return PQ_ERR_CUDA;
@@ -305,8 +316,8 @@ int gemm_forward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, co
   f.th = f.tq; f.tb = f.tq;
   f.rt = sv.rt; f.perm = nullptr; f.gamma = sv.gamma; f.gate = sv.gate; f.w_scales = a.w_scales;
   f.alpha = a.alpha; f.beta = a.beta; f.Y = Y; f.T = a.T; f.N = a.N; f.K = a.K; f.r = 0; f.sstride = a.scale_stride;
-  f.ntn = (a.N + 255) / 256;
-  return launch_gemm<FwdProblem<false>>(f, mtiles * f.ntn, st);
+  f.ntn = (a.N + 255) / 256; f.item_rows = 0;
+  return launch_gemm<FwdProblem<false>>(KID_FWD, f, mtiles * f.ntn, st);
 }
 
 
@@ -343,7 +354,7 @@ struct HpDhProblem {
     uint16_t* gh;
     float* dl;
     uint16_t* dlc;
-    int T, N, r, E, bn, sstride;
+    int T, N, r, E, bn, sstride, item_rows;
   };
   struct Tile { int item; int4 it; };
   __device__ static int num_tiles(const Params& p) { return p.rt.n_items[0]; }
@@ -364,9 +375,13 @@ struct HpDhProblem {
     const float ca = p.sstride ? 1.0f : p.alpha[0];
     const float g = live ? p.gate[pos] : 0.f;
     const long long hrow = ((long long)t.item * 128 + row) * p.r;
+    const long long plane = (long long)p.item_rows * p.r;
     const uint4* hin = reinterpret_cast<const uint4*>(p.H + hrow);
+    const uint4* hin_lo = reinterpret_cast<const uint4*>(p.H + plane + hrow);
     uint4* dhc = reinterpret_cast<uint4*>(p.dhc + hrow);
+    uint4* dhc_lo = reinterpret_cast<uint4*>(p.dhc + plane + hrow);
     uint4* gh = reinterpret_cast<uint4*>(p.gh + hrow);
+    uint4* gh_lo = reinterpret_cast<uint4*>(p.gh + plane + hrow);
     float dg = 0.f;
     for (int c32 = 0; c32 * 32 < p.r; ++c32) {
       uint32_t v[32];
@@ -375,26 +390,25 @@ struct HpDhProblem {
 #pragma unroll
       for (int q8 = 0; q8 < 4; ++q8) {
         if (c32 * 32 + q8 * 8 < p.r) {
-          uint4 o1 = make_uint4(0, 0, 0, 0), o2 = make_uint4(0, 0, 0, 0);
+          uint32_t w1[4] = {0, 0, 0, 0}, w1l[4] = {0, 0, 0, 0}, w2[4] = {0, 0, 0, 0}, w2l[4] = {0, 0, 0, 0};
           if (live) {
-            const uint4 hv = hin[c32 * 4 + q8];
-            const uint32_t hw[4] = {hv.x, hv.y, hv.z, hv.w};
-            uint32_t w1[4], w2[4];
+            const uint4 hv = hin[c32 * 4 + q8], hl = hin_lo[c32 * 4 + q8];
+            const uint32_t hw[4] = {hv.x, hv.y, hv.z, hv.w}, hlw[4] = {hl.x, hl.y, hl.z, hl.w};
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-              const float h0 = bf16lo(hw[j]), h1 = bf16hi(hw[j]);
+              const float h0 = bf16lo(hw[j]) + bf16lo(hlw[j]), h1 = bf16hi(hw[j]) + bf16hi(hlw[j]);
               const float d0 = __uint_as_float(v[q8 * 8 + 2 * j]), d1 = __uint_as_float(v[q8 * 8 + 2 * j + 1]);
               dg = fmaf(h0, d0, dg);
               dg = fmaf(h1, d1, dg);
               const float sc = ca * g * inv_cc;
-              w1[j] = pack_bf16x2(sc * d0, sc * d1);
-              w2[j] = pack_bf16x2(g * h0, g * h1);
+              split2(sc * d0, sc * d1, w1[j], w1l[j]);
+              split2(g * h0, g * h1, w2[j], w2l[j]);
             }
-            o1 = make_uint4(w1[0], w1[1], w1[2], w1[3]);
-            o2 = make_uint4(w2[0], w2[1], w2[2], w2[3]);
           }
-          dhc[c32 * 4 + q8] = o1;
-          gh[c32 * 4 + q8] = o2;
+          dhc[c32 * 4 + q8] = make_uint4(w1[0], w1[1], w1[2], w1[3]);
+          dhc_lo[c32 * 4 + q8] = make_uint4(w1l[0], w1l[1], w1l[2], w1l[3]);
+          gh[c32 * 4 + q8] = make_uint4(w2[0], w2[1], w2[2], w2[3]);
+          gh_lo[c32 * 4 + q8] = make_uint4(w2l[0], w2l[1], w2l[2], w2l[3]);
         }
       }
     }
@@ -432,7 +446,7 @@ struct BwdDxProblem {
     const float* w_scales;
     const float* beta;
     uint16_t* dX;
-    int T, N, K, r, E, sstride, ntk;
+    int T, N, K, r, E, sstride, ntk, item_rows;
   };
   struct Tile { int m, kt, ib, ie, skip1; };
   __device__ static int num_tiles(const Params& p) { return ((p.T + 127) / 128) * p.ntk; }
@@ -441,7 +455,7 @@ struct BwdDxProblem {
     if (p.r > 0) { t.ib = p.rt.tile_item_begin[t.m]; t.ie = p.rt.tile_item_begin[t.m + 1]; } else { t.ib = t.ie = 0; }
     t.skip1 = dx_scale(p.w_scales, p.beta, p.sstride) == 0.f;
   }
-  __device__ static int num_segments(const Params& p, const Tile& t) { return (t.skip1 ? 0 : 1) + (t.ie - t.ib) + (p.E > 1 ? 1 : 0); }
+  __device__ static int num_segments(const Params& p, const Tile& t) { return (t.skip1 ? 0 : 1) + 2 * (t.ie - t.ib) + (p.E > 1 ? 1 : 0); }
   __device__ static void segment(const Params& p, const Tile& t, int i, Segment& s) {
     s.mode = MODE_BF_KM; s.acc = 0; s.bn = 256; s.ksteps = 4; s.a_rank = 2; s.a_x = 0; s.a_z = 0;
     s.b_x = t.kt * 256; s.b_y = 0; s.b_z = 0; s.b_bytes = kStageBBytes;
@@ -454,10 +468,10 @@ struct BwdDxProblem {
       }
       --i;
     }
-    if (i < t.ie - t.ib) {
-      const int item = t.ib + i;
+    if (i < 2 * (t.ie - t.ib)) {
+      const int item = t.ib + (i >> 1), plane = i & 1;
       s.nkb = (p.r + 63) / 64;
-      s.ta = &p.tdh; s.a_y = item * 128;
+      s.ta = &p.tdh; s.a_y = plane * p.item_rows + item * 128;
       s.tb = &p.ta3; s.b_rank = 3; s.b_z = p.rt.items[item].y;
       return;
     }
@@ -563,7 +577,7 @@ struct HpDbProblem {
     const float* alpha;
     float* dB;
     float* dalpha_partial;
-    int N, r, E, bn, sstride, ntn;
+    int N, r, E, bn, sstride, ntn, item_rows;
   };
   struct Tile { int nt, e, ib, ie; };
   __device__ static int num_tiles(const Params& p) { return p.ntn * p.E; }
@@ -571,12 +585,12 @@ struct HpDbProblem {
     t.e = i / p.ntn; t.nt = i % p.ntn;
     t.ib = p.rt.expert_item_begin[t.e]; t.ie = p.rt.expert_item_begin[t.e + 1];
   }
-  __device__ static int num_segments(const Params&, const Tile& t) { return t.ie - t.ib; }
+  __device__ static int num_segments(const Params&, const Tile& t) { return 2 * (t.ie - t.ib); }
   __device__ static void segment(const Params& p, const Tile& t, int i, Segment& s) {
-    const int item = t.ib + i;
+    const int item = t.ib + (i >> 1), plane = i & 1;
     s.mode = MODE_BF_MM; s.acc = 0; s.bn = p.bn; s.ksteps = 4; s.nkb = 2;
     s.ta = &p.tdyT; s.a_rank = 2; s.a_x = t.nt * 128; s.a_y = p.rt.items[item].x * 128; s.a_z = 0;
-    s.tb = &p.tgh; s.b_rank = 2; s.b_x = 0; s.b_y = item * 128; s.b_z = 0;
+    s.tb = &p.tgh; s.b_rank = 2; s.b_x = 0; s.b_y = plane * p.item_rows + item * 128; s.b_z = 0;
     s.b_bytes = (p.bn / 64) * kMnBoxBytes;
   }
   __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane) {
@@ -627,7 +641,7 @@ struct HpDaProblem {
     const float* w_scales;
     const float* beta;
     float* dA;
-    int K, r, E, sstride, ntk;
+    int K, r, E, sstride, ntk, item_rows;
   };
   struct Tile { int e, kt, ib, ie; };
   __device__ static int num_tiles(const Params& p) { return p.ntk * p.E; }
@@ -635,11 +649,11 @@ struct HpDaProblem {
     t.e = i / p.ntk; t.kt = i % p.ntk;
     t.ib = p.rt.expert_item_begin[t.e]; t.ie = p.rt.expert_item_begin[t.e + 1];
   }
-  __device__ static int num_segments(const Params&, const Tile& t) { return t.ie - t.ib; }
+  __device__ static int num_segments(const Params&, const Tile& t) { return 2 * (t.ie - t.ib); }
   __device__ static void segment(const Params& p, const Tile& t, int i, Segment& s) {
-    const int item = t.ib + i;
+    const int item = t.ib + (i >> 1), plane = i & 1;
     s.mode = MODE_BF_MM; s.acc = 0; s.bn = 256; s.ksteps = 4; s.nkb = 2;
-    s.ta = &p.tdhT; s.a_rank = 2; s.a_x = 0; s.a_y = item * 128; s.a_z = 0;
+    s.ta = &p.tdhT; s.a_rank = 2; s.a_x = 0; s.a_y = plane * p.item_rows + item * 128; s.a_z = 0;
     s.tb = &p.txs; s.b_rank = 2; s.b_x = t.kt * 256; s.b_y = p.rt.items[item].x * 128; s.b_z = 0;
     s.b_bytes = kStageBBytes;
   }
@@ -675,7 +689,7 @@ int gemm_backward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, c
   const int ntk = (a.K + 255) / 256, ntn128 = (a.N + 127) / 128;
   const bool hp = a.r > 0;
   const int r64 = h_round_up(a.r, 64);
-  const uint64_t item_rows = (uint64_t)sv.max_items * 128;
+  const uint64_t item_rows = (uint64_t)sv.max_items * 128;  // rows of one plane; buffers hold two
   int rc;
   if (hp) {
     HpDhProblem::Params p;
@@ -683,8 +697,8 @@ int gemm_backward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, c
     if (!map3d(&p.tba, b.ba, a.r, a.N, a.E, 64, 64)) return PQ_ERR_CUDA;
     p.rt = sv.rt; p.H = sv.h; p.gate = sv.gate; p.probs = sv.probs; p.w_scales = a.w_scales; p.alpha = a.alpha; p.beta = a.beta;
     p.dhc = b.dhc; p.gh = b.gh; p.dl = b.dl; p.dlc = b.dlc;
-    p.T = a.T; p.N = a.N; p.r = a.r; p.E = a.E; p.bn = r64; p.sstride = a.scale_stride;
-    rc = launch_gemm<HpDhProblem>(p, sv.max_items, st);
+    p.T = a.T; p.N = a.N; p.r = a.r; p.E = a.E; p.bn = r64; p.sstride = a.scale_stride; p.item_rows = (int)item_rows;
+    rc = launch_gemm<HpDhProblem>(KID_HP_DH, p, sv.max_items, st);
     if (rc) return rc;
   }
   {
@@ -693,7 +707,7 @@ int gemm_backward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, c
     if (!map2d(&p.tsb, false, b.sb, a.K, a.N, 64, 64)) return PQ_ERR_CUDA;
     p.tdh = p.tdy; p.ta3 = p.tdy; p.tdl = p.tdy; p.twr = p.tdy;
     if (hp) {
-      if (!map2d(&p.tdh, false, b.dhc, a.r, item_rows, 64, 128)) return PQ_ERR_CUDA;
+      if (!map2d(&p.tdh, false, b.dhc, a.r, 2 * item_rows, 64, 128)) return PQ_ERR_CUDA;
       if (!map3d(&p.ta3, a.A, a.K, a.r, a.E, 64, 64)) return PQ_ERR_CUDA;
     }
     if (hp && a.E > 1) {
@@ -701,8 +715,8 @@ int gemm_backward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, c
       if (!map2d(&p.twr, false, a.Wr, a.K, a.E, 64, 64)) return PQ_ERR_CUDA;
     }
     p.rt = sv.rt; p.perm = (hp && a.E > 1) ? sv.perm : nullptr; p.w_scales = a.w_scales; p.beta = a.beta; p.dX = dX;
-    p.T = a.T; p.N = a.N; p.K = a.K; p.r = a.r; p.E = hp ? a.E : 1; p.sstride = a.scale_stride; p.ntk = ntk;
-    rc = launch_gemm<BwdDxProblem>(p, mtiles * ntk, st);
+    p.T = a.T; p.N = a.N; p.K = a.K; p.r = a.r; p.E = hp ? a.E : 1; p.sstride = a.scale_stride; p.ntk = ntk; p.item_rows = (int)item_rows;
+    rc = launch_gemm<BwdDxProblem>(KID_BWD_DX, p, mtiles * ntk, st);
     if (rc) return rc;
   }
   {
@@ -711,23 +725,23 @@ int gemm_backward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, c
     if (!map2d(&p.txt, false, sv.xt, a.K, a.T, 64, 64)) return PQ_ERR_CUDA;
     p.s8 = w_s8; p.beta = a.beta; p.dW = dW; p.dbeta_partial = b.dbeta_partial;
     p.T = a.T; p.N = a.N; p.K = a.K; p.sstride = a.scale_stride; p.ntk = ntk;
-    rc = launch_gemm<BwdDwProblem>(p, ntn128 * ntk, st);
+    rc = launch_gemm<BwdDwProblem>(KID_BWD_DW, p, ntn128 * ntk, st);
     if (rc) return rc;
   }
   if (hp) {
     HpDbProblem::Params p;
     if (!map2d(&p.tdyT, false, b.dys, a.N, a.T, 64, 64)) return PQ_ERR_CUDA;
-    if (!map2d(&p.tgh, false, b.gh, a.r, item_rows, 64, 64)) return PQ_ERR_CUDA;
+    if (!map2d(&p.tgh, false, b.gh, a.r, 2 * item_rows, 64, 64)) return PQ_ERR_CUDA;
     p.rt = sv.rt; p.B = a.B; p.alpha = a.alpha; p.dB = dB; p.dalpha_partial = b.dalpha_partial;
-    p.N = a.N; p.r = a.r; p.E = a.E; p.bn = r64; p.sstride = a.scale_stride; p.ntn = ntn128;
-    rc = launch_gemm<HpDbProblem>(p, ntn128 * a.E, st);
+    p.N = a.N; p.r = a.r; p.E = a.E; p.bn = r64; p.sstride = a.scale_stride; p.ntn = ntn128; p.item_rows = (int)item_rows;
+    rc = launch_gemm<HpDbProblem>(KID_HP_DB, p, ntn128 * a.E, st);
     if (rc) return rc;
     HpDaProblem::Params q;
-    if (!map2d(&q.tdhT, false, b.dhc, a.r, item_rows, 64, 64)) return PQ_ERR_CUDA;
+    if (!map2d(&q.tdhT, false, b.dhc, a.r, 2 * item_rows, 64, 64)) return PQ_ERR_CUDA;
     if (!map2d(&q.txs, false, b.xs, a.K, a.T, 64, 64)) return PQ_ERR_CUDA;
     q.rt = sv.rt; q.w_scales = a.w_scales; q.beta = a.beta; q.dA = dA;
-    q.K = a.K; q.r = a.r; q.E = a.E; q.sstride = a.scale_stride; q.ntk = ntk;
-    rc = launch_gemm<HpDaProblem>(q, ntk * a.E, st);
+    q.K = a.K; q.r = a.r; q.E = a.E; q.sstride = a.scale_stride; q.ntk = ntk; q.item_rows = (int)item_rows;
+    rc = launch_gemm<HpDaProblem>(KID_HP_DA, q, ntk * a.E, st);
     if (rc) return rc;
   }
   return PQ_OK;

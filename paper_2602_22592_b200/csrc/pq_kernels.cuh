@@ -13,6 +13,25 @@ constexpr int kPackPartials = 1024;        // fp64 partial sums of the weight re
 constexpr float kActQmax = 128.0f;         // 2^7 of Eq. 9
 constexpr float kActAmaxFloor = 1e-5f;     // all-zero row guard
 
+// Kernel ids for launch counting and optional event timing (pq_profile_events).
+enum KernelId : int {
+  KID_PACK_SUMS = 0, KID_BINARIZE_PACK, KID_ROUTER, KID_ROUTE_SCAN, KID_ACT_QUANT, KID_HP_UP, KID_FWD, KID_SCATTER_ROWS,
+  KID_SCALED_SIGN, KID_SCALED_B, KID_HP_DH, KID_BWD_DX, KID_BWD_DW, KID_HP_DB, KID_HP_DA, KID_ROUTER_WGRAD, KID_SUM_PARTIALS,
+  KID_SUM_SCALAR, KID_DEBUG, KID_DECODE_PREP, KID_DECODE_MAIN, KID_COUNT
+};
+struct ProfileSlot { cudaEvent_t start, stop; };
+extern ProfileSlot g_profile[KID_COUNT];
+extern long long g_launches;
+// Brackets one kernel launch: counts it and, if events were registered for its id, records them.
+struct LaunchScope {
+  int id; cudaStream_t st;
+  LaunchScope(int id_, cudaStream_t st_) : id(id_), st(st_) {
+    ++g_launches;
+    if (g_profile[id].start) cudaEventRecord(g_profile[id].start, st);
+  }
+  ~LaunchScope() { if (g_profile[id].stop) cudaEventRecord(g_profile[id].stop, st); }
+};
+
 // Item table of the expert-sorted token order (built by k_route_scan).
 struct RoutingTables {
   int* n_items;            // [1]
@@ -78,8 +97,8 @@ struct BwdBuffers {
   const uint16_t* xs;    // [T,K] bf16 activations in sorted order
   const uint16_t* sb;    // [N,K] bf16 sign * (beta_n or 1)
   const uint16_t* ba;    // [E,N,r] bf16 B * (alpha_n or 1)
-  uint16_t* dhc;         // [items*128, r] bf16 dH / c
-  uint16_t* gh;          // [items*128, r] bf16 g * H
+  uint16_t* dhc;         // [2][items*128, r] bf16 hi/lo planes of dH / c
+  uint16_t* gh;          // [2][items*128, r] bf16 hi/lo planes of g * H
   float* dl;             // [T,E] fp32 router logit gradient (sorted order)
   uint16_t* dlc;         // [T,16] bf16 dl / c
   float* dbeta_partial;  // [ceil(K/256), N]
