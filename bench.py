@@ -208,7 +208,7 @@ def run_ours(args):
 
     # per-kernel breakdown of one extra (untimed) step
     names = ["pack_sums", "binarize_pack", "router", "route_scan", "act_quant", "hp_up", "fwd", "scatter_rows", "scaled_sign",
-             "hp_dh", "bwd_dx", "bwd_dw", "hp_db", "hp_da", "router_wgrad"]
+             "hp_dh", "bwd_dx", "bwd_dw", "hp_db", "reduce_db", "hp_da", "reduce_da", "router_wgrad", "sum_partials", "sum_scalar"]
     bev = {n: (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for n in names}
     breakdown = {n: 0.0 for n in names}
     for L in layers:

@@ -26,7 +26,7 @@ EXPORTS = ("pq_status_string", "pq_workspace_bytes", "pq_saved_bytes", "pq_saved
 
 KERNEL_IDS = dict(pack_sums=0, binarize_pack=1, router=2, route_scan=3, act_quant=4, hp_up=5, fwd=6, scatter_rows=7,
                   scaled_sign=8, scaled_b=9, hp_dh=10, bwd_dx=11, bwd_dw=12, hp_db=13, hp_da=14, router_wgrad=15,
-                  sum_partials=16, sum_scalar=17, debug=18, decode_prep=19, decode_main=20)
+                  sum_partials=16, sum_scalar=17, debug=18, decode_prep=19, decode_main=20, reduce_db=21, reduce_da=22)
 
 
 class PqError(RuntimeError):

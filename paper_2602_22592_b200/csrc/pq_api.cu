@@ -26,6 +26,16 @@ static inline int experts_of(const pq_desc* d) { return d->r > 0 ? (d->E < 1 ? 1
 static inline int max_items_of(const pq_desc* d) { return mtiles_of(d) + experts_of(d) - 1; }
 static inline bool routed(const pq_desc* d) { return d->r > 0 && d->E > 1; }
 
+// Items per chunk for the split token contraction of dA (table a) and dB (table b): small enough that
+// (chunks x output tiles) fills about two waves of 148 CTAs, large enough to keep the partial buffers small.
+static inline int chunk_items(int mtiles, int out_tiles) {
+  int c = mtiles * out_tiles / 296;
+  return c < 1 ? 1 : c;
+}
+static inline int chunk_a_of(const pq_desc* d) { return chunk_items(mtiles_of(d), (d->K + 255) / 256); }
+static inline int chunk_b_of(const pq_desc* d) { return chunk_items(mtiles_of(d), (d->N + 127) / 128); }
+static inline int max_chunks(const pq_desc* d, int chunk) { return (max_items_of(d) + chunk - 1) / chunk + experts_of(d); }
+
 static int check_desc(const pq_desc* d, bool training) {
   if (!d) return PQ_ERR_NULL;
   if (d->size != sizeof(pq_desc)) return PQ_ERR_SHAPE;
@@ -59,6 +69,14 @@ static size_t carve_saved(const pq_desc* d, void* base, SavedPtrs* out) {
   s.rt.items = c.take<int4>(s.max_items);
   s.rt.tile_item_begin = c.take<int>(mtiles_of(d) + 1);
   s.rt.expert_item_begin = c.take<int>(E + 1);
+  s.chunk_a = chunk_a_of(d); s.chunk_b = chunk_b_of(d);
+  s.max_chunks_a = max_chunks(d, s.chunk_a); s.max_chunks_b = max_chunks(d, s.chunk_b);
+  s.rt.n_chunks_a = c.take<int>(1);
+  s.rt.chunks_a = c.take<int4>(s.max_chunks_a);
+  s.rt.expert_chunk_begin_a = c.take<int>(E + 1);
+  s.rt.n_chunks_b = c.take<int>(1);
+  s.rt.chunks_b = c.take<int4>(s.max_chunks_b);
+  s.rt.expert_chunk_begin_b = c.take<int>(E + 1);
   if (out) *out = s;
   return c.off;
 }
@@ -89,6 +107,8 @@ struct BwdScratch {
   float* dwr_partial;
   float* dalpha_vec;
   float* dbeta_vec;
+  float* da_partial;
+  float* db_partial;
 };
 
 static size_t carve_bwd_scratch(const pq_desc* d, void* base, BwdScratch* out) {
@@ -109,6 +129,8 @@ static size_t carve_bwd_scratch(const pq_desc* d, void* base, BwdScratch* out) {
   s.dwr_partial = routed(d) ? c.take<float>(((T + 255) / 256) * E * K) : nullptr;
   s.dalpha_vec = c.take<float>(N);
   s.dbeta_vec = c.take<float>(N);
+  s.da_partial = r > 0 ? c.take<float>((size_t)max_chunks(d, chunk_a_of(d)) * r * K) : nullptr;
+  s.db_partial = r > 0 ? c.take<float>((size_t)max_chunks(d, chunk_b_of(d)) * N * r) : nullptr;
   if (out) *out = s;
   return c.off;
 }
@@ -254,6 +276,7 @@ int pq_linear_backward(const pq_desc* d, const uint16_t* dY, const uint16_t* X, 
   }
   b.dhc = sc.dhc; b.gh = sc.gh; b.dl = sc.dl; b.dlc = sc.dlc;
   b.dbeta_partial = sc.dbeta_partial; b.dalpha_partial = sc.dalpha_partial;
+  b.da_partial = sc.da_partial; b.db_partial = sc.db_partial;
   rc = gemm_backward(a, w_s8, sv, b, dX, dW, dA, dB, st);
   if (rc) return rc;
 

@@ -168,61 +168,93 @@ __global__ void __launch_bounds__(256) k_router(const uint4* __restrict__ X, con
 // table.  An item is the intersection of a 128-row tile of the sorted token
 // order with one expert's range: {tile, expert, first row, end row} (rows
 // relative to the tile).  Items are sorted by tile and therefore by expert.
-// One small block; the work is a few hundred integers.
+// Also groups each expert's items into chunks (two tables, two chunk sizes): the
+// units over which the token contraction of dA and dB is split across CTAs.
+// One block; the work is a few hundred integers.
 // ---------------------------------------------------------------------------
-__global__ void __launch_bounds__(32) k_route_scan(int T, int E, int nblocks, const int* __restrict__ block_counts,
-                                                   int* __restrict__ block_base, int* __restrict__ offsets, RoutingTables rt) {
-  __shared__ int off[kMaxExperts + 1];
-  const int lane = threadIdx.x;
-  if (E <= 1) {
-    if (lane == 0) { off[0] = 0; off[1] = T; offsets[0] = 0; offsets[1] = T; }
-  } else {
-    __shared__ int total[kMaxExperts];
-    if (lane < E) {
-      int run = 0;
-      for (int b = 0; b < nblocks; ++b) {
-        block_base[b * E + lane] = run;
-        run += block_counts[b * E + lane];
-      }
-      total[lane] = run;
-    }
-    __syncwarp();
-    if (lane == 0) {
-      int run = 0;
-      for (int e = 0; e < E; ++e) { off[e] = run; offsets[e] = run; run += total[e]; }
-      off[E] = run;
-      offsets[E] = run;
-    }
+// Builder of one chunk table: consecutive items of one expert, at most `size` items each.
+struct ChunkBuilder {
+  int4* out; int* begin; int size; int n = 0, cur_e = -1, cur_b = 0, cur_n = 0, next_e = 0;
+  __device__ void flush() {
+    if (cur_n > 0) { out[n] = make_int4(cur_e, cur_b, cur_b + cur_n, 0); ++n; }
+    cur_n = 0;
   }
-  __syncwarp();
-  if (lane == 0) {
+  __device__ void add(int item, int e) {
+    if (e != cur_e || cur_n == size) {
+      flush();
+      cur_b = item;
+      if (e != cur_e) {
+        for (; next_e <= e; ++next_e) begin[next_e] = n;  // experts without items get an empty range
+        cur_e = e;
+      }
+    }
+    ++cur_n;
+  }
+  __device__ void finish(int Ee, int* count) {
+    flush();
+    for (; next_e <= Ee; ++next_e) begin[next_e] = n;
+    count[0] = n;
+  }
+};
+
+__global__ void __launch_bounds__(512) k_route_scan(int T, int E, int nblocks, const int* __restrict__ block_counts,
+                                                    int* __restrict__ block_base, int* __restrict__ offsets, RoutingTables rt,
+                                                    int chunk_a, int chunk_b) {
+  __shared__ int off[kMaxExperts + 1];
+  __shared__ int total[kMaxExperts];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (E > 1 && warp < E) {
+    // exclusive scan of this expert's per-block counts, 32 blocks at a time
+    int carry = 0;
+    for (int b0 = 0; b0 < nblocks; b0 += 32) {
+      const int b = b0 + lane;
+      const int v = b < nblocks ? block_counts[b * E + warp] : 0;
+      int inc = v;
+      for (int d = 1; d < 32; d <<= 1) {
+        const int u = __shfl_up_sync(0xffffffffu, inc, d);
+        if (lane >= d) inc += u;
+      }
+      if (b < nblocks) block_base[b * E + warp] = carry + inc - v;
+      carry += __shfl_sync(0xffffffffu, inc, 31);
+    }
+    if (lane == 0) total[warp] = carry;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
     const int Ee = E < 1 ? 1 : E;
+    if (E <= 1) {
+      off[0] = 0; off[1] = T;
+    } else {
+      int run = 0;
+      for (int e = 0; e < E; ++e) { off[e] = run; run += total[e]; }
+      off[E] = run;
+    }
+    for (int e = 0; e <= Ee; ++e) offsets[e] = off[e];
     const int mtiles = (T + kTileRows - 1) / kTileRows;
+    int next_item_e = 0;  // experts whose first item index is still to be recorded
+    ChunkBuilder ca{rt.chunks_a, rt.expert_chunk_begin_a, chunk_a}, cb{rt.chunks_b, rt.expert_chunk_begin_b, chunk_b};
     int n = 0, e = 0;
-    for (int x = 0; x <= Ee; ++x) rt.expert_item_begin[x] = 0;
     for (int tile = 0; tile < mtiles; ++tile) {
       rt.tile_item_begin[tile] = n;
       const int r0 = tile * kTileRows, r1 = min(T, r0 + kTileRows);
       while (e < Ee && off[e + 1] <= r0) ++e;  // first expert reaching into this tile
-      int ee = e;
-      while (ee < Ee && off[ee] < r1) {
+      for (int ee = e; ee < Ee && off[ee] < r1; ++ee) {
         const int lo = max(off[ee], r0), hi = min(off[ee + 1], r1);
         if (hi > lo) {
           rt.items[n] = make_int4(tile, ee, lo - r0, hi - r0);
+          // first item of each expert (items ascend in expert)
+          for (; next_item_e <= ee; ++next_item_e) rt.expert_item_begin[next_item_e] = n;
+          ca.add(n, ee);
+          cb.add(n, ee);
           ++n;
         }
-        ++ee;
       }
     }
     rt.tile_item_begin[mtiles] = n;
     rt.n_items[0] = n;
-    // items are sorted by expert: first item of each expert
-    int i = 0;
-    for (int x = 0; x < Ee; ++x) {
-      while (i < n && rt.items[i].y < x) ++i;
-      rt.expert_item_begin[x] = i;
-    }
-    rt.expert_item_begin[Ee] = n;
+    for (; next_item_e <= Ee; ++next_item_e) rt.expert_item_begin[next_item_e] = n;
+    ca.finish(Ee, rt.n_chunks_a);
+    cb.finish(Ee, rt.n_chunks_b);
   }
 }
 
@@ -407,6 +439,51 @@ __global__ void __launch_bounds__(1024) k_sum_to_scalar(const float* __restrict_
   }
 }
 
+// dB[e,n,:] = alpha_n * sum over expert e's chunks of the raw partials (ascending chunk order);
+// dalpha partial[e,n] = sum_j B[e,n,j] * that sum.  One warp per (e, n) row.
+__global__ void __launch_bounds__(256) k_reduce_db(const float* __restrict__ partial, RoutingTables rt, const uint16_t* __restrict__ B,
+                                                   const float* __restrict__ alpha, int sstride, int E, int N, int r,
+                                                   float* __restrict__ dB, float* __restrict__ dalpha_partial) {
+  const int row = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (row >= E * N) return;
+  const int e = row / N, n = row % N;
+  const int c0 = rt.expert_chunk_begin_b[e], c1 = rt.expert_chunk_begin_b[e + 1];
+  const float al = alpha[n * sstride];
+  float part = 0.f;
+  for (int j = lane * 4; j < r; j += 128) {
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int c = c0; c < c1; ++c) {
+      const float4 v = *reinterpret_cast<const float4*>(partial + ((long long)c * N + n) * r + j);
+      s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+    }
+    const uint2 bv = *reinterpret_cast<const uint2*>(B + ((long long)e * N + n) * r + j);
+    part = fmaf(bf16lo(bv.x), s.x, part); part = fmaf(bf16hi(bv.x), s.y, part);
+    part = fmaf(bf16lo(bv.y), s.z, part); part = fmaf(bf16hi(bv.y), s.w, part);
+    *reinterpret_cast<float4*>(dB + ((long long)e * N + n) * r + j) = make_float4(al * s.x, al * s.y, al * s.z, al * s.w);
+  }
+  for (int d = 16; d > 0; d >>= 1) part += __shfl_xor_sync(0xffffffffu, part, d);
+  if (lane == 0) dalpha_partial[(long long)e * N + n] = part;
+}
+
+// dA[e,j,k] = c * sum over expert e's chunks of the raw partials; c as in the dX tile (lam*beta or lam, 1 if that is 0)
+__global__ void __launch_bounds__(256) k_reduce_da(const float* __restrict__ partial, RoutingTables rt, const float* __restrict__ w_scales,
+                                                   const float* __restrict__ beta, int sstride, int E, int r, int K, float* __restrict__ dA) {
+  const long long per_e = (long long)r * K / 4, total = per_e * E;
+  float c = sstride ? w_scales[0] : w_scales[0] * beta[0];
+  if (c == 0.f) c = 1.0f;
+  for (long long i = blockIdx.x * 256LL + threadIdx.x; i < total; i += gridDim.x * 256LL) {
+    const int e = (int)(i / per_e);
+    const long long w = i % per_e;
+    const int c0 = rt.expert_chunk_begin_a[e], c1 = rt.expert_chunk_begin_a[e + 1];
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int ch = c0; ch < c1; ++ch) {
+      const float4 v = reinterpret_cast<const float4*>(partial)[(long long)ch * per_e + w];
+      s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+    }
+    reinterpret_cast<float4*>(dA)[i] = make_float4(c * s.x, c * s.y, c * s.z, c * s.w);
+  }
+}
+
 __global__ void k_fill_zero(uint4* p, long long n16) {
   for (long long i = blockIdx.x * 256LL + threadIdx.x; i < n16; i += gridDim.x * 256LL) p[i] = make_uint4(0, 0, 0, 0);
 }
@@ -441,7 +518,7 @@ cudaError_t launch_route_and_quant(const uint16_t* X, const uint16_t* Wr, int T,
                                       sc.probs_tok, sc.block_counts);
   }
   { LaunchScope ls(KID_ROUTE_SCAN, st);
-  k_route_scan<<<1, 32, 0, st>>>(T, E, nblocks, sc.block_counts, sc.block_base, sv.offsets, sv.rt); }
+  k_route_scan<<<1, 512, 0, st>>>(T, E, nblocks, sc.block_counts, sc.block_base, sv.offsets, sv.rt, sv.chunk_a, sv.chunk_b); }
   LaunchScope ls(KID_ACT_QUANT, st);
   k_act_quant<<<(T + 7) / 8, 256, 0, st>>>(reinterpret_cast<const uint4*>(X), T, K, E, sv.expert, sc.block_base, sv.offsets, sc.gate_tok,
                                            sc.probs_tok, reinterpret_cast<uint2*>(sv.q), reinterpret_cast<uint4*>(sv.xt),
@@ -490,6 +567,21 @@ cudaError_t launch_sum_partials(const float* partial, int nparts, int n, const f
 cudaError_t launch_sum_to_scalar(const float* v, int n, float* out, cudaStream_t st) {
   LaunchScope ls(KID_SUM_SCALAR, st);
   k_sum_to_scalar<<<1, 1024, 0, st>>>(v, n, out);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_reduce_db(const float* partial, const RoutingTables& rt, const uint16_t* B, const float* alpha, int sstride, int E, int N,
+                             int r, float* dB, float* dalpha_partial, cudaStream_t st) {
+  LaunchScope ls(KID_REDUCE_DB, st);
+  k_reduce_db<<<(E * N + 7) / 8, 256, 0, st>>>(partial, rt, B, alpha, sstride, E, N, r, dB, dalpha_partial);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_reduce_da(const float* partial, const RoutingTables& rt, const float* w_scales, const float* beta, int sstride, int E, int r,
+                             int K, float* dA, cudaStream_t st) {
+  LaunchScope ls(KID_REDUCE_DA, st);
+  const long long total = (long long)E * r * K / 4;
+  k_reduce_da<<<grid_for(total, 256 * 2, 148 * 8), 256, 0, st>>>(partial, rt, w_scales, beta, sstride, E, r, K, dA);
   return cudaGetLastError();
 }
 

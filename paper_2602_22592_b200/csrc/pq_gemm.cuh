@@ -30,7 +30,9 @@ constexpr int kStageBytes = kStageABytes + kStageBBytes;
 constexpr int kMnBoxBytes = 64 * 128;    // one MN-major box: 64 k-rows of 64 bf16
 constexpr int kTmemCols = 512;
 constexpr int kAccCols = 256;            // TMEM columns reserved per accumulator
-constexpr int kGemmSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kEpiRowPitch = 144;                      // 128 payload bytes + 16 pad: conflict-free 16-byte accesses
+constexpr int kEpiWarpBytes = 32 * kEpiRowPitch;       // per epilogue warp: 32 rows of one 128-byte chunk
+constexpr int kGemmSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ + 4 * kEpiWarpBytes;
 
 enum OpMode : int {
   MODE_I8_KK = 0,  // int8, A[M,K] and B[N,K] K-contiguous
@@ -84,8 +86,29 @@ __device__ __forceinline__ bool pipe_wait(uint32_t bar, uint32_t parity, int whe
   return true;
 }
 
+// Coalescing store for epilogues.  Each lane holds 128 contiguous bytes (8 x 16 B) of ITS OWN output
+// row, and rows may live anywhere in global memory (row_ptr = 0 skips the row).  The warp transposes
+// through its staging buffer so that every store instruction writes 4 rows x 128 contiguous bytes
+// instead of 32 rows x 16 bytes.  Only the first valid_bytes of each row are written.
+__device__ __forceinline__ void warp_store_rows(uint8_t* stage, const uint4 (&v)[8], void* row_ptr, int valid_bytes, int lane) {
+  uint4* mine = reinterpret_cast<uint4*>(stage + lane * kEpiRowPitch);
+#pragma unroll
+  for (int j = 0; j < 8; ++j) mine[j] = v[j];
+  __syncwarp();
+  const unsigned long long my = reinterpret_cast<unsigned long long>(row_ptr);
+  const int c = lane & 7;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int row = 4 * i + (lane >> 3);
+    const unsigned long long dst = __shfl_sync(0xffffffffu, my, row);
+    const uint4 val = *reinterpret_cast<const uint4*>(stage + row * kEpiRowPitch + c * 16);
+    if (dst != 0ull && c * 16 < valid_bytes) *reinterpret_cast<uint4*>(dst + c * 16) = val;
+  }
+  __syncwarp();
+}
+
 template <class P>
-__global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_constant__ typename P::Params p) {
+__device__ __forceinline__ void gemm_body(const typename P::Params& p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t bar_base = smem_base + kStages * kStageBytes;
@@ -97,6 +120,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
   uint8_t* bar_generic = smem_raw + (bar_base - smem_u32(smem_raw));
   volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(bar_generic + 8 * (2 * kStages + 4));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_generic + 8 * (2 * kStages + 4) + 8);
+  uint8_t* epi_stage = bar_generic + 256;  // 4 x kEpiWarpBytes
 
   constexpr int kAccStages = (P::kAccPerTile == 1) ? 2 : 1;
   const int warp = threadIdx.x >> 5;
@@ -205,7 +229,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
       if (!pipe_wait(tfull_bar(ac.stage), ac.phase, WHERE_EPILOGUE, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + ac.stage * P::kAccPerTile * kAccCols + (static_cast<uint32_t>(quad * 32) << 16);
-      P::epilogue(p, t, taddr, quad, lane);
+      P::epilogue(p, t, taddr, quad, lane, epi_stage + (warp - 2) * kEpiWarpBytes);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(ac.stage));
@@ -226,5 +250,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_kernel(const __grid_cons
     tmem_dealloc(tmem_base, kTmemCols);
   }
 }
+
+// One named kernel per problem, so that profiler listings show which product ran.
+#define PQ_DEFINE_GEMM_KERNEL(name, Problem)                                                      \
+  __global__ void __launch_bounds__(kGemmThreads, 1) name(const __grid_constant__ typename Problem::Params p) { \
+    gemm_body<Problem>(p);                                                                        \
+  }
 
 }  // namespace pq

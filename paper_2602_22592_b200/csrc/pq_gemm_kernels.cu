@@ -78,17 +78,14 @@ static int sm_count() {
   return g_sm_count;
 }
 
-template <class P>
-static int launch_gemm(int kernel_id, const typename P::Params& p, int max_tiles, cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(gemm_kernel<P>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes) != cudaSuccess) return PQ_ERR_CUDA;
-    configured = true;
-  }
+template <class Params>
+static int launch_gemm(int kernel_id, void (*kernel)(Params), const Params& p, int max_tiles, cudaStream_t st) {
+  // (cudaFuncSetAttribute is cheap and idempotent; calling it per launch keeps this free of static state per kernel)
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes) != cudaSuccess) return PQ_ERR_CUDA;
   int grid = max_tiles < sm_count() ? max_tiles : sm_count();
   if (grid < 1) grid = 1;
   LaunchScope ls(kernel_id, st);
-  gemm_kernel<P><<<grid, kGemmThreads, kGemmSmemBytes, st>>>(p);
+  kernel<<<grid, kGemmThreads, kGemmSmemBytes, st>>>(p);
   return cudaGetLastError() == cudaSuccess ? PQ_OK : PQ_ERR_CUDA;
 }
 
@@ -128,7 +125,7 @@ struct DebugProblem {
     if (p.mode >= MODE_BF_KM) { s.b_x = t.n * 256; s.b_y = 0; } else { s.b_x = 0; s.b_y = t.n * 256; }
     s.b_bytes = kStageBBytes;
   }
-  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane) {
+  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane, uint8_t* stage) {
     const int row = t.m * 128 + quad * 32 + lane;
     uint32_t* D = reinterpret_cast<uint32_t*>(p.D);
     for (int c = 0; c < 8; ++c) {
@@ -137,14 +134,15 @@ struct DebugProblem {
       uint32_t v[32];
       tmem_ld32(taddr + c * 32, v);
       tmem_ld_wait();
-      if (row < p.M) {
+      uint4 o[8];
 #pragma unroll
-        for (int j = 0; j < 32; ++j)
-          if (n0 + j < p.N) D[(long long)row * p.N + n0 + j] = v[j];
-      }
+      for (int j = 0; j < 8; ++j) o[j] = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+      const int valid = min(32, p.N - n0) * 4;   // N is a multiple of 8 -> whole 16-byte pieces
+      warp_store_rows(stage, o, row < p.M ? D + (long long)row * p.N + n0 : nullptr, valid, lane);
     }
   }
 };
+PQ_DEFINE_GEMM_KERNEL(k_gemm_debug, DebugProblem)
 
 int gemm_debug(int mode, int M, int N, int K, const void* A, const void* B, void* D, cudaStream_t st) {
   DebugProblem::Params p;
@@ -167,7 +165,7 @@ int gemm_debug(int mode, int M, int N, int K, const void* A, const void* B, void
       return PQ_ERR_UNSUPPORTED;
   }
   if (!ok) return PQ_ERR_CUDA;
-  return launch_gemm<DebugProblem>(KID_DEBUG, p, ((M + 127) / 128) * p.ntn, st);
+  return launch_gemm(KID_DEBUG, k_gemm_debug, p, ((M + 127) / 128) * p.ntn, st);
 }
 
 // ---------------------------------------------------------------------------
@@ -191,7 +189,7 @@ struct HpUpProblem {
     s.tb = &p.ta; s.b_rank = 3; s.b_x = 0; s.b_y = 0; s.b_z = t.it.y;
     s.b_bytes = p.bn * 128;
   }
-  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane) {
+  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane, uint8_t* stage) {
     const int row = quad * 32 + lane;
     const bool live = row >= t.it.z && row < t.it.w;
     uint4* out_hi = reinterpret_cast<uint4*>(p.H + ((long long)t.item * 128 + row) * p.r);
@@ -215,6 +213,8 @@ struct HpUpProblem {
     }
   }
 };
+
+PQ_DEFINE_GEMM_KERNEL(k_gemm_hp_up, HpUpProblem)
 
 // ---------------------------------------------------------------------------
 // F2: fused output tile.  Accumulator 0 (int32): q S^T over K.  Accumulator 1
@@ -257,38 +257,48 @@ struct FwdProblem {
       s.tb = &p.tb; s.b_rank = 3; s.b_x = 0; s.b_y = t.n * 256; s.b_z = e;
     }
   }
-  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane) {
+  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane, uint8_t* stage) {
     const int pos = t.m * 128 + quad * 32 + lane;
     const bool live = pos < p.T;
     const int token = live ? (p.perm ? p.perm[pos] : pos) : 0;
     const float s1 = live ? __fdiv_rn(p.w_scales[0], p.gamma[pos]) : 0.f;
     const float g = (HP && live) ? p.gate[pos] : 0.f;
-    uint4* yrow = reinterpret_cast<uint4*>(p.Y + (long long)token * p.N);
-    for (int c = 0; c < 8; ++c) {
-      const int n0 = t.n * 256 + c * 32;
+    uint16_t* yrow = live ? p.Y + (long long)token * p.N : nullptr;
+    for (int c = 0; c < 4; ++c) {           // 64 output columns = 128 bytes of the row per pass
+      const int n0 = t.n * 256 + c * 64;
       if (n0 >= p.N) break;
-      uint32_t a[32], z[32];
-      tmem_ld32(taddr + c * 32, a);
-      if (HP) tmem_ld32(taddr + kAccCols + c * 32, z);
-      tmem_ld_wait();
-      if (live) {
+      uint4 o[8];
 #pragma unroll
-        for (int gq = 0; gq < 4; ++gq) {
-          float y[8];
+      for (int h = 0; h < 2; ++h) {
+        uint32_t a[32], z[32];
+        tmem_ld32(taddr + c * 64 + h * 32, a);
+        if (HP) tmem_ld32(taddr + kAccCols + c * 64 + h * 32, z);
+        tmem_ld_wait();
+        const int nb = n0 + h * 32;
+        if (nb < p.N) {
+          uint32_t w[16];
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const int n = n0 + gq * 8 + j;
-            const float be = __ldg(p.beta + n * p.sstride);
-            float v = be * s1 * (float)(int)a[gq * 8 + j];
-            if (HP) v += __ldg(p.alpha + n * p.sstride) * g * __uint_as_float(z[gq * 8 + j]);
-            y[j] = v;
+          for (int j = 0; j < 16; ++j) {
+            float y[2];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+              const int n = nb + 2 * j + u;
+              float v = __ldg(p.beta + n * p.sstride) * s1 * (float)(int)a[2 * j + u];
+              if (HP) v += __ldg(p.alpha + n * p.sstride) * g * __uint_as_float(z[2 * j + u]);
+              y[u] = v;
+            }
+            w[j] = pack_bf16x2(y[0], y[1]);
           }
-          yrow[(n0 >> 3) + gq] = make_uint4(pack_bf16x2(y[0], y[1]), pack_bf16x2(y[2], y[3]), pack_bf16x2(y[4], y[5]), pack_bf16x2(y[6], y[7]));
+#pragma unroll
+          for (int j = 0; j < 4; ++j) o[4 * h + j] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
         }
       }
+      warp_store_rows(stage, o, yrow ? yrow + n0 : nullptr, min(64, p.N - n0) * 2, lane);
     }
   }
 };
+PQ_DEFINE_GEMM_KERNEL(k_gemm_fwd_hp, FwdProblem<true>)
+PQ_DEFINE_GEMM_KERNEL(k_gemm_fwd_1bit, FwdProblem<false>)
 
 int gemm_forward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, const uint16_t* xs, uint16_t* Y, cudaStream_t st) {
   const int mtiles = (a.T + 127) / 128;
@@ -298,7 +308,7 @@ int gemm_forward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, co
     p.rt = sv.rt; p.H = sv.h; p.K = a.K; p.r = a.r; p.bn = h_round_up(a.r, 16); p.item_rows = sv.max_items * 128;
     if (!map2d(&p.tx, false, xs, a.K, a.T, 64, 128)) return PQ_ERR_CUDA;
     if (!map3d(&p.ta, a.A, a.K, a.r, a.E, 64, p.bn)) return PQ_ERR_CUDA;
-    int rc = launch_gemm<HpUpProblem>(KID_HP_UP, p, sv.max_items, st);
+    int rc = launch_gemm(KID_HP_UP, k_gemm_hp_up, p, sv.max_items, st);
     if (rc) return rc;
     FwdProblem<true>::Params f;
     if (!map2d(&f.tq, true, sv.q, a.K, a.T, 128, 128)) return PQ_ERR_CUDA;
@@ -308,7 +318,7 @@ int gemm_forward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, co
     f.rt = sv.rt; f.perm = a.E > 1 ? sv.perm : nullptr; f.gamma = sv.gamma; f.gate = sv.gate; f.w_scales = a.w_scales;
     f.alpha = a.alpha; f.beta = a.beta; f.Y = Y; f.T = a.T; f.N = a.N; f.K = a.K; f.r = a.r; f.sstride = a.scale_stride;
     f.ntn = (a.N + 255) / 256; f.item_rows = sv.max_items * 128;
-    return launch_gemm<FwdProblem<true>>(KID_FWD, f, mtiles * f.ntn, st);
+    return launch_gemm(KID_FWD, k_gemm_fwd_hp, f, mtiles * f.ntn, st);
   }
   FwdProblem<false>::Params f;
   if (!map2d(&f.tq, true, sv.q, a.K, a.T, 128, 128)) return PQ_ERR_CUDA;
@@ -317,7 +327,7 @@ int gemm_forward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, co
   f.rt = sv.rt; f.perm = nullptr; f.gamma = sv.gamma; f.gate = sv.gate; f.w_scales = a.w_scales;
   f.alpha = a.alpha; f.beta = a.beta; f.Y = Y; f.T = a.T; f.N = a.N; f.K = a.K; f.r = 0; f.sstride = a.scale_stride;
   f.ntn = (a.N + 255) / 256; f.item_rows = 0;
-  return launch_gemm<FwdProblem<false>>(KID_FWD, f, mtiles * f.ntn, st);
+  return launch_gemm(KID_FWD, k_gemm_fwd_1bit, f, mtiles * f.ntn, st);
 }
 
 
@@ -366,7 +376,7 @@ struct HpDhProblem {
     s.tb = &p.tba; s.b_rank = 3; s.b_x = 0; s.b_y = 0; s.b_z = t.it.y;
     s.b_bytes = (p.bn / 64) * kMnBoxBytes;
   }
-  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane) {
+  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane, uint8_t* stage) {
     const int row = quad * 32 + lane;
     const bool live = row >= t.it.z && row < t.it.w;
     const int pos = t.it.x * 128 + row;
@@ -433,6 +443,8 @@ struct HpDhProblem {
   }
 };
 
+PQ_DEFINE_GEMM_KERNEL(k_gemm_hp_dh, HpDhProblem)
+
 // ---------------------------------------------------------------------------
 // B2: dX tile = c * ( dYs . Sb  +  sum_items dhc . A_e  +  dlc . Wr ), rows
 // scattered back to token order.
@@ -479,33 +491,35 @@ struct BwdDxProblem {
     s.ta = &p.tdl; s.a_y = t.m * 128;
     s.tb = &p.twr; s.b_rank = 2;
   }
-  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane) {
+  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane, uint8_t* stage) {
     const int pos = t.m * 128 + quad * 32 + lane;
     const bool live = pos < p.T;
     const int token = live ? (p.perm ? p.perm[pos] : pos) : 0;
     const float c = dx_scale(p.w_scales, p.beta, p.sstride);
     const float cc = c != 0.f ? c : 1.0f;
     const bool has = num_segments(p, t) > 0;
-    uint4* xrow = reinterpret_cast<uint4*>(p.dX + (long long)token * p.K);
-    for (int c32 = 0; c32 < 8; ++c32) {
-      const int k0 = t.kt * 256 + c32 * 32;
+    uint16_t* xrow = live ? p.dX + (long long)token * p.K : nullptr;
+    for (int c64 = 0; c64 < 4; ++c64) {
+      const int k0 = t.kt * 256 + c64 * 64;
       if (k0 >= p.K) break;
-      uint32_t v[32];
-      tmem_ld32(taddr + c32 * 32, v);
-      tmem_ld_wait();
-      if (live) {
+      uint4 o[8];
 #pragma unroll
-        for (int q8 = 0; q8 < 4; ++q8) {
-          uint32_t w[4];
+      for (int h = 0; h < 2; ++h) {
+        uint32_t v[32];
+        tmem_ld32(taddr + c64 * 64 + h * 32, v);
+        tmem_ld_wait();
+        uint32_t w[16];
 #pragma unroll
-          for (int j = 0; j < 4; ++j)
-            w[j] = has ? pack_bf16x2(cc * __uint_as_float(v[q8 * 8 + 2 * j]), cc * __uint_as_float(v[q8 * 8 + 2 * j + 1])) : 0u;
-          xrow[(k0 >> 3) + q8] = make_uint4(w[0], w[1], w[2], w[3]);
-        }
+        for (int j = 0; j < 16; ++j)
+          w[j] = has ? pack_bf16x2(cc * __uint_as_float(v[2 * j]), cc * __uint_as_float(v[2 * j + 1])) : 0u;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) o[4 * h + j] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
       }
+      warp_store_rows(stage, o, xrow ? xrow + k0 : nullptr, min(64, p.K - k0) * 2, lane);
     }
   }
 };
+PQ_DEFINE_GEMM_KERNEL(k_gemm_bwd_dx, BwdDxProblem)
 
 // ---------------------------------------------------------------------------
 // B3: G = dYs^T . xt (contraction over tokens); dW = beta_n G; per-tile partial
@@ -531,11 +545,11 @@ struct BwdDwProblem {
     s.tb = &p.txt; s.b_rank = 2; s.b_x = t.kt * 256; s.b_y = 0; s.b_z = 0;
     s.b_bytes = kStageBBytes;
   }
-  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane) {
+  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane, uint8_t* stage) {
     const int n = t.nt * 128 + quad * 32 + lane;
     const bool live = n < p.N;
     const float be = live ? p.beta[n * p.sstride] : 0.f;
-    float4* wrow = reinterpret_cast<float4*>(p.dW + (long long)(live ? n : 0) * p.K);
+    float* wrow = live ? p.dW + (long long)n * p.K : nullptr;
     const uint4* srow = reinterpret_cast<const uint4*>(p.s8 + (long long)(live ? n : 0) * p.K);
     float part = 0.f;
     for (int c32 = 0; c32 < 8; ++c32) {
@@ -544,46 +558,50 @@ struct BwdDwProblem {
       uint32_t v[32];
       tmem_ld32(taddr + c32 * 32, v);
       tmem_ld_wait();
+      uint4 o[8];
+      uint32_t sw[8] = {0, 0, 0, 0, 0, 0, 0, 0};
       if (live) {
         const uint4 s0 = __ldg(srow + (k0 >> 4)), s1 = __ldg(srow + (k0 >> 4) + 1);
-        const uint32_t sw[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
-#pragma unroll
-        for (int q4 = 0; q4 < 8; ++q4) {
-          const float g0 = __uint_as_float(v[q4 * 4]), g1 = __uint_as_float(v[q4 * 4 + 1]);
-          const float g2 = __uint_as_float(v[q4 * 4 + 2]), g3 = __uint_as_float(v[q4 * 4 + 3]);
-          const uint32_t sb = sw[q4];  // four +-1 bytes: bit 7 set <-> -1
-          part += (sb & 0x80u) ? -g0 : g0;
-          part += (sb & 0x8000u) ? -g1 : g1;
-          part += (sb & 0x800000u) ? -g2 : g2;
-          part += (sb & 0x80000000u) ? -g3 : g3;
-          wrow[(k0 >> 2) + q4] = make_float4(be * g0, be * g1, be * g2, be * g3);
-        }
+        sw[0] = s0.x; sw[1] = s0.y; sw[2] = s0.z; sw[3] = s0.w; sw[4] = s1.x; sw[5] = s1.y; sw[6] = s1.z; sw[7] = s1.w;
       }
+#pragma unroll
+      for (int q4 = 0; q4 < 8; ++q4) {
+        const float g0 = __uint_as_float(v[q4 * 4]), g1 = __uint_as_float(v[q4 * 4 + 1]);
+        const float g2 = __uint_as_float(v[q4 * 4 + 2]), g3 = __uint_as_float(v[q4 * 4 + 3]);
+        const uint32_t sb = sw[q4];  // four +-1 bytes: bit 7 set <-> -1
+        part += (sb & 0x80u) ? -g0 : g0;
+        part += (sb & 0x8000u) ? -g1 : g1;
+        part += (sb & 0x800000u) ? -g2 : g2;
+        part += (sb & 0x80000000u) ? -g3 : g3;
+        o[q4] = make_uint4(__float_as_uint(be * g0), __float_as_uint(be * g1), __float_as_uint(be * g2), __float_as_uint(be * g3));
+      }
+      warp_store_rows(stage, o, wrow ? wrow + k0 : nullptr, 128, lane);
     }
     if (live) p.dbeta_partial[(long long)t.kt * p.N + n] = part;
   }
 };
+PQ_DEFINE_GEMM_KERNEL(k_gemm_bwd_dw, BwdDwProblem)
 
 // ---------------------------------------------------------------------------
-// B4: dBraw_e = dYs^T . (g H) over the items of expert e; dB = alpha_n dBraw;
-// partial of dalpha_n = sum_j B_e[n,j] dBraw_e[n,j].
+// B4: raw dB partials.  The token contraction of dBraw_e = dYs^T . (g H) is split
+// into chunks of expert e's items so that enough CTAs work on it; each tile
+// (chunk, 128 output features) writes its fp32 partial, and k_reduce_db sums a
+// expert's chunks in a fixed order, scales by alpha_n and forms the dalpha partials.
 // ---------------------------------------------------------------------------
 struct HpDbProblem {
   static constexpr int kAccPerTile = 1;
   struct Params {
     CUtensorMap tdyT, tgh;
     RoutingTables rt;
-    const uint16_t* B;
-    const float* alpha;
-    float* dB;
-    float* dalpha_partial;
-    int N, r, E, bn, sstride, ntn, item_rows;
+    float* partial;  // [chunks, N, r]
+    int N, r, bn, ntn, item_rows;
   };
-  struct Tile { int nt, e, ib, ie; };
-  __device__ static int num_tiles(const Params& p) { return p.ntn * p.E; }
+  struct Tile { int nt, chunk, ib, ie; };
+  __device__ static int num_tiles(const Params& p) { return p.ntn * p.rt.n_chunks_b[0]; }
   __device__ static void tile_init(const Params& p, int i, Tile& t) {
-    t.e = i / p.ntn; t.nt = i % p.ntn;
-    t.ib = p.rt.expert_item_begin[t.e]; t.ie = p.rt.expert_item_begin[t.e + 1];
+    t.chunk = i / p.ntn; t.nt = i % p.ntn;
+    const int4 c = p.rt.chunks_b[t.chunk];
+    t.ib = c.y; t.ie = c.z;
   }
   __device__ static int num_segments(const Params&, const Tile& t) { return 2 * (t.ie - t.ib); }
   __device__ static void segment(const Params& p, const Tile& t, int i, Segment& s) {
@@ -593,61 +611,40 @@ struct HpDbProblem {
     s.tb = &p.tgh; s.b_rank = 2; s.b_x = 0; s.b_y = plane * p.item_rows + item * 128; s.b_z = 0;
     s.b_bytes = (p.bn / 64) * kMnBoxBytes;
   }
-  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane) {
+  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane, uint8_t* stage) {
     const int n = t.nt * 128 + quad * 32 + lane;
-    const bool live = n < p.N;
-    const bool has = t.ie > t.ib;
-    const float al = live ? p.alpha[n * p.sstride] : 0.f;
-    const long long rowoff = ((long long)t.e * p.N + (live ? n : 0)) * p.r;
-    float4* out = reinterpret_cast<float4*>(p.dB + rowoff);
-    const uint4* bin = reinterpret_cast<const uint4*>(p.B + rowoff);
-    float part = 0.f;
+    float* out = n < p.N ? p.partial + ((long long)t.chunk * p.N + n) * p.r : nullptr;
     for (int c32 = 0; c32 * 32 < p.r; ++c32) {
       uint32_t v[32];
       tmem_ld32(taddr + c32 * 32, v);
       tmem_ld_wait();
-      if (live) {
+      uint4 o[8];
 #pragma unroll
-        for (int q8 = 0; q8 < 4; ++q8) {
-          if (c32 * 32 + q8 * 8 < p.r) {
-            const uint4 bv = __ldg(bin + c32 * 4 + q8);
-            const uint32_t bw[4] = {bv.x, bv.y, bv.z, bv.w};
-            float a[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) a[j] = has ? __uint_as_float(v[q8 * 8 + j]) : 0.f;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              part = fmaf(bf16lo(bw[j]), a[2 * j], part);
-              part = fmaf(bf16hi(bw[j]), a[2 * j + 1], part);
-            }
-            out[c32 * 8 + q8 * 2] = make_float4(al * a[0], al * a[1], al * a[2], al * a[3]);
-            out[c32 * 8 + q8 * 2 + 1] = make_float4(al * a[4], al * a[5], al * a[6], al * a[7]);
-          }
-        }
-      }
+      for (int j = 0; j < 8; ++j) o[j] = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+      warp_store_rows(stage, o, out ? out + c32 * 32 : nullptr, min(32, p.r - c32 * 32) * 4, lane);
     }
-    if (live) p.dalpha_partial[(long long)t.e * p.N + n] = part;
   }
 };
+PQ_DEFINE_GEMM_KERNEL(k_gemm_hp_db, HpDbProblem)
 
 // ---------------------------------------------------------------------------
-// B5: dA_e = c * dhc^T . Xs over the items of expert e.
+// B5: raw dA partials, dhc^T . Xs over one chunk of an expert's items; summed and
+// scaled by k_reduce_da.
 // ---------------------------------------------------------------------------
 struct HpDaProblem {
   static constexpr int kAccPerTile = 1;
   struct Params {
     CUtensorMap tdhT, txs;
     RoutingTables rt;
-    const float* w_scales;
-    const float* beta;
-    float* dA;
-    int K, r, E, sstride, ntk, item_rows;
+    float* partial;  // [chunks, r, K]
+    int K, r, ntk, item_rows;
   };
-  struct Tile { int e, kt, ib, ie; };
-  __device__ static int num_tiles(const Params& p) { return p.ntk * p.E; }
+  struct Tile { int chunk, kt, ib, ie; };
+  __device__ static int num_tiles(const Params& p) { return p.ntk * p.rt.n_chunks_a[0]; }
   __device__ static void tile_init(const Params& p, int i, Tile& t) {
-    t.e = i / p.ntk; t.kt = i % p.ntk;
-    t.ib = p.rt.expert_item_begin[t.e]; t.ie = p.rt.expert_item_begin[t.e + 1];
+    t.chunk = i / p.ntk; t.kt = i % p.ntk;
+    const int4 c = p.rt.chunks_a[t.chunk];
+    t.ib = c.y; t.ie = c.z;
   }
   __device__ static int num_segments(const Params&, const Tile& t) { return 2 * (t.ie - t.ib); }
   __device__ static void segment(const Params& p, const Tile& t, int i, Segment& s) {
@@ -657,31 +654,23 @@ struct HpDaProblem {
     s.tb = &p.txs; s.b_rank = 2; s.b_x = t.kt * 256; s.b_y = p.rt.items[item].x * 128; s.b_z = 0;
     s.b_bytes = kStageBBytes;
   }
-  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane) {
+  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane, uint8_t* stage) {
     const int j = quad * 32 + lane;
-    const bool live = j < p.r;
-    const bool has = t.ie > t.ib;
-    const float c = dx_scale(p.w_scales, p.beta, p.sstride);
-    const float cc = c != 0.f ? c : 1.0f;
-    float4* out = reinterpret_cast<float4*>(p.dA + ((long long)t.e * p.r + (live ? j : 0)) * p.K);
+    float* out = j < p.r ? p.partial + ((long long)t.chunk * p.r + j) * p.K : nullptr;
     for (int c32 = 0; c32 < 8; ++c32) {
       const int k0 = t.kt * 256 + c32 * 32;
       if (k0 >= p.K) break;
       uint32_t v[32];
       tmem_ld32(taddr + c32 * 32, v);
       tmem_ld_wait();
-      if (live) {
+      uint4 o[8];
 #pragma unroll
-        for (int q4 = 0; q4 < 8; ++q4) {
-          float a[4];
-#pragma unroll
-          for (int i = 0; i < 4; ++i) a[i] = has ? cc * __uint_as_float(v[q4 * 4 + i]) : 0.f;
-          out[(k0 >> 2) + q4] = make_float4(a[0], a[1], a[2], a[3]);
-        }
-      }
+      for (int q = 0; q < 8; ++q) o[q] = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+      warp_store_rows(stage, o, out ? out + k0 : nullptr, 128, lane);
     }
   }
 };
+PQ_DEFINE_GEMM_KERNEL(k_gemm_hp_da, HpDaProblem)
 
 int gemm_backward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, const BwdBuffers& b, uint16_t* dX, float* dW, float* dA,
                   float* dB, cudaStream_t st) {
@@ -698,7 +687,7 @@ int gemm_backward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, c
     p.rt = sv.rt; p.H = sv.h; p.gate = sv.gate; p.probs = sv.probs; p.w_scales = a.w_scales; p.alpha = a.alpha; p.beta = a.beta;
     p.dhc = b.dhc; p.gh = b.gh; p.dl = b.dl; p.dlc = b.dlc;
     p.T = a.T; p.N = a.N; p.r = a.r; p.E = a.E; p.bn = r64; p.sstride = a.scale_stride; p.item_rows = (int)item_rows;
-    rc = launch_gemm<HpDhProblem>(KID_HP_DH, p, sv.max_items, st);
+    rc = launch_gemm(KID_HP_DH, k_gemm_hp_dh, p, sv.max_items, st);
     if (rc) return rc;
   }
   {
@@ -716,7 +705,7 @@ int gemm_backward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, c
     }
     p.rt = sv.rt; p.perm = (hp && a.E > 1) ? sv.perm : nullptr; p.w_scales = a.w_scales; p.beta = a.beta; p.dX = dX;
     p.T = a.T; p.N = a.N; p.K = a.K; p.r = a.r; p.E = hp ? a.E : 1; p.sstride = a.scale_stride; p.ntk = ntk; p.item_rows = (int)item_rows;
-    rc = launch_gemm<BwdDxProblem>(KID_BWD_DX, p, mtiles * ntk, st);
+    rc = launch_gemm(KID_BWD_DX, k_gemm_bwd_dx, p, mtiles * ntk, st);
     if (rc) return rc;
   }
   {
@@ -725,24 +714,25 @@ int gemm_backward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, c
     if (!map2d(&p.txt, false, sv.xt, a.K, a.T, 64, 64)) return PQ_ERR_CUDA;
     p.s8 = w_s8; p.beta = a.beta; p.dW = dW; p.dbeta_partial = b.dbeta_partial;
     p.T = a.T; p.N = a.N; p.K = a.K; p.sstride = a.scale_stride; p.ntk = ntk;
-    rc = launch_gemm<BwdDwProblem>(KID_BWD_DW, p, ntn128 * ntk, st);
+    rc = launch_gemm(KID_BWD_DW, k_gemm_bwd_dw, p, ntn128 * ntk, st);
     if (rc) return rc;
   }
   if (hp) {
     HpDbProblem::Params p;
     if (!map2d(&p.tdyT, false, b.dys, a.N, a.T, 64, 64)) return PQ_ERR_CUDA;
     if (!map2d(&p.tgh, false, b.gh, a.r, 2 * item_rows, 64, 64)) return PQ_ERR_CUDA;
-    p.rt = sv.rt; p.B = a.B; p.alpha = a.alpha; p.dB = dB; p.dalpha_partial = b.dalpha_partial;
-    p.N = a.N; p.r = a.r; p.E = a.E; p.bn = r64; p.sstride = a.scale_stride; p.ntn = ntn128; p.item_rows = (int)item_rows;
-    rc = launch_gemm<HpDbProblem>(KID_HP_DB, p, ntn128 * a.E, st);
+    p.rt = sv.rt; p.partial = b.db_partial; p.N = a.N; p.r = a.r; p.bn = r64; p.ntn = ntn128; p.item_rows = (int)item_rows;
+    rc = launch_gemm(KID_HP_DB, k_gemm_hp_db, p, ntn128 * sv.max_chunks_b, st);
     if (rc) return rc;
+    if (launch_reduce_db(b.db_partial, sv.rt, a.B, a.alpha, a.scale_stride, a.E, a.N, a.r, dB, b.dalpha_partial, st) != cudaSuccess)
+      return PQ_ERR_CUDA;
     HpDaProblem::Params q;
     if (!map2d(&q.tdhT, false, b.dhc, a.r, 2 * item_rows, 64, 64)) return PQ_ERR_CUDA;
     if (!map2d(&q.txs, false, b.xs, a.K, a.T, 64, 64)) return PQ_ERR_CUDA;
-    q.rt = sv.rt; q.w_scales = a.w_scales; q.beta = a.beta; q.dA = dA;
-    q.K = a.K; q.r = a.r; q.E = a.E; q.sstride = a.scale_stride; q.ntk = ntk; q.item_rows = (int)item_rows;
-    rc = launch_gemm<HpDaProblem>(KID_HP_DA, q, ntk * a.E, st);
+    q.rt = sv.rt; q.partial = b.da_partial; q.K = a.K; q.r = a.r; q.ntk = ntk; q.item_rows = (int)item_rows;
+    rc = launch_gemm(KID_HP_DA, k_gemm_hp_da, q, ntk * sv.max_chunks_a, st);
     if (rc) return rc;
+    if (launch_reduce_da(b.da_partial, sv.rt, a.w_scales, a.beta, a.scale_stride, a.E, a.r, a.K, dA, st) != cudaSuccess) return PQ_ERR_CUDA;
   }
   return PQ_OK;
 }

@@ -17,7 +17,7 @@ constexpr float kActAmaxFloor = 1e-5f;     // all-zero row guard
 enum KernelId : int {
   KID_PACK_SUMS = 0, KID_BINARIZE_PACK, KID_ROUTER, KID_ROUTE_SCAN, KID_ACT_QUANT, KID_HP_UP, KID_FWD, KID_SCATTER_ROWS,
   KID_SCALED_SIGN, KID_SCALED_B, KID_HP_DH, KID_BWD_DX, KID_BWD_DW, KID_HP_DB, KID_HP_DA, KID_ROUTER_WGRAD, KID_SUM_PARTIALS,
-  KID_SUM_SCALAR, KID_DEBUG, KID_DECODE_PREP, KID_DECODE_MAIN, KID_COUNT
+  KID_SUM_SCALAR, KID_DEBUG, KID_DECODE_PREP, KID_DECODE_MAIN, KID_REDUCE_DB, KID_REDUCE_DA, KID_COUNT
 };
 struct ProfileSlot { cudaEvent_t start, stop; };
 extern ProfileSlot g_profile[KID_COUNT];
@@ -38,6 +38,13 @@ struct RoutingTables {
   int4* items;             // [max_items] {tile, expert, first row, end row}
   int* tile_item_begin;    // [mtiles + 1]
   int* expert_item_begin;  // [E + 1]
+  // chunk tables {expert, first item, end item, 0}: table a splits dA, table b splits dB
+  int* n_chunks_a;         // [1]
+  int4* chunks_a;          // [max_items + E]
+  int* expert_chunk_begin_a;  // [E + 1]
+  int* n_chunks_b;
+  int4* chunks_b;
+  int* expert_chunk_begin_b;
 };
 
 // Device pointers into the caller's `saved` buffer.
@@ -55,6 +62,8 @@ struct SavedPtrs {
   uint16_t* h;
   RoutingTables rt;
   int max_items;
+  int chunk_a, chunk_b;      // items per chunk of the two tables
+  int max_chunks_a, max_chunks_b;
 };
 
 struct FwdScratch {
@@ -76,6 +85,10 @@ cudaError_t launch_router_wgrad(const uint16_t* xs, const float* dl, int T, int 
 cudaError_t launch_sum_partials(const float* partial, int nparts, int n, const float* scale, float* out, cudaStream_t st);
 cudaError_t launch_sum_to_scalar(const float* v, int n, float* out, cudaStream_t st);
 cudaError_t launch_fill_zero(void* p, size_t bytes, cudaStream_t st);
+cudaError_t launch_reduce_db(const float* partial, const RoutingTables& rt, const uint16_t* B, const float* alpha, int sstride, int E, int N,
+                             int r, float* dB, float* dalpha_partial, cudaStream_t st);
+cudaError_t launch_reduce_da(const float* partial, const RoutingTables& rt, const float* w_scales, const float* beta, int sstride, int E, int r,
+                             int K, float* dA, cudaStream_t st);
 
 // tensor-core launchers (pq_gemm_kernels.cu).  All return a PQ_* status.
 struct LayerArgs {
@@ -103,6 +116,8 @@ struct BwdBuffers {
   uint16_t* dlc;         // [T,16] bf16 dl / c
   float* dbeta_partial;  // [ceil(K/256), N]
   float* dalpha_partial; // [E, N]
+  float* da_partial;     // [max_chunks_a, r, K] raw split-contraction partials of dA
+  float* db_partial;     // [max_chunks_b, N, r]
 };
 int gemm_backward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, const BwdBuffers& b, uint16_t* dX, float* dW, float* dA,
                   float* dB, cudaStream_t st);
