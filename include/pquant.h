@@ -47,7 +47,8 @@ enum {
   PQ_ERR_WORKSPACE = -4,   /* workspace / saved buffer too small                */
   PQ_ERR_UNSUPPORTED = -5, /* valid request this build does not implement       */
   PQ_ERR_CUDA = -6,        /* a CUDA runtime / driver call failed               */
-  PQ_ERR_TIMEOUT = -7      /* a device-side bounded wait ran out                */
+  PQ_ERR_TIMEOUT = -7,     /* a device-side bounded wait ran out                */
+  PQ_ERR_TOO_LARGE = -8    /* problem needs more scratch than a fixed-size buffer holds */
 };
 
 enum { PQ_SCALE_VECTOR = 1u }; /* pq_desc.flags: alpha, beta have N entries instead of 1 */
@@ -110,6 +111,35 @@ int pq_saved_view_init(const pq_desc* d, void* saved, pq_saved_view* out);
  * Only d->N and d->K are read. */
 int pq_pack_weights(const pq_desc* d, const float* W, uint32_t* w_bits, int8_t* w_s8,
                     float* w_scales, void* ws, size_t ws_bytes, void* stream);
+
+/* Weight quantisation for callers that cannot allocate device memory.
+ * (The paper has no counterpart: this is a packaging variant of pq_pack_weights.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a serving
+ * process whose device memory is handed out once at start-up by another
+ * component, a plug-in running inside someone else's memory pool, a section of
+ * a program that must not trigger the implicit synchronisation an allocation
+ * causes.  Such a caller still owns W and the three outputs, but has nowhere to
+ * get the reduction workspace pq_pack_weights asks for.  Here that workspace is a
+ * fixed 64 KiB array inside the library (a file-scope device array: every GPU
+ * that loads the library holds those 64 KiB until the process exits).
+ *
+ * Same inputs, outputs and results as pq_pack_weights, minus ws / ws_bytes.
+ *   - Limit: N * K <= 67,108,864 elements (4096 slabs of 16384 elements, one
+ *     pair of fp64 partial sums each).  Larger matrices get PQ_ERR_TOO_LARGE and
+ *     nothing is launched.
+ *   - The call makes no cudaMalloc / cudaFree and uses no allocating routine.
+ *   - The first call on each device looks up the array's device address (a
+ *     one-off host-side query); make that first call outside any stream capture.
+ *   - All calls share the one array.  Nothing in it has to start at zero -- each
+ *     call overwrites the slots it later reads -- but two calls whose kernels
+ *     overlap on the GPU (different streams) would overwrite each other's
+ *     partial sums: keep calls on one device in stream order.
+ *   - lam and mu are summed slab by slab instead of grid-strided, so they can
+ *     differ from pq_pack_weights in the last fp64 bit before the one rounding to
+ *     fp32; in practice the outputs are identical. */
+int pq_pack_weights_static(const pq_desc* d, const float* W, uint32_t* w_bits, int8_t* w_s8,
+                           float* w_scales, void* stream);
 
 /* Forward of the layer (Eq. 10-11, Sec. 3.3).
  *   training (w_s8 != NULL): tensor-core path; fills `saved` (may be NULL when

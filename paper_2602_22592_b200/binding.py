@@ -16,12 +16,12 @@ LIB_PATH = os.path.join(_HERE, "libpquant.so")
 
 PQ_OK = 0
 PQ_ERR_NULL, PQ_ERR_SHAPE, PQ_ERR_ALIGN, PQ_ERR_WORKSPACE = -1, -2, -3, -4
-PQ_ERR_UNSUPPORTED, PQ_ERR_CUDA, PQ_ERR_TIMEOUT = -5, -6, -7
+PQ_ERR_UNSUPPORTED, PQ_ERR_CUDA, PQ_ERR_TIMEOUT, PQ_ERR_TOO_LARGE = -5, -6, -7, -8
 PQ_SCALE_VECTOR = 1
 PQ_PHASE_PACK, PQ_PHASE_FWD, PQ_PHASE_BWD, PQ_PHASE_DECODE = 0, 1, 2, 3
 
 EXPORTS = ("pq_status_string", "pq_workspace_bytes", "pq_saved_bytes", "pq_saved_view_init",
-           "pq_pack_weights", "pq_linear_forward", "pq_linear_backward", "pq_debug_gemm",
+           "pq_pack_weights", "pq_pack_weights_static", "pq_linear_forward", "pq_linear_backward", "pq_debug_gemm",
            "pq_device_status", "pq_kernel_launches", "pq_profile_events")
 
 KERNEL_IDS = dict(pack_sums=0, binarize_pack=1, router=2, route_scan=3, act_quant=4, hp_up=5, fwd=6, scatter_rows=7,
@@ -69,6 +69,8 @@ def lib() -> ctypes.CDLL:
         L.pq_saved_view_init.argtypes = [dp, vp, ctypes.POINTER(pq_saved_view)]
         L.pq_pack_weights.restype = ci
         L.pq_pack_weights.argtypes = [dp, vp, vp, vp, vp, vp, sz, vp]
+        L.pq_pack_weights_static.restype = ci
+        L.pq_pack_weights_static.argtypes = [dp, vp, vp, vp, vp, vp]
         L.pq_linear_forward.restype = ci
         L.pq_linear_forward.argtypes = [dp] + [vp] * 10 + [vp, sz, vp, sz, vp]
         L.pq_linear_backward.restype = ci
@@ -151,6 +153,13 @@ def pq_saved_view_init(d: pq_desc, saved: torch.Tensor) -> dict:
 def pq_pack_weights(d, W, w_bits, w_s8, w_scales, ws, stream=None):
     _check("pq_pack_weights", lib().pq_pack_weights(ctypes.byref(d), _ptr(W), _ptr(w_bits), _ptr(w_s8), _ptr(w_scales),
                                                      _ptr(ws), _nbytes(ws), _stream(stream)))
+
+
+def pq_pack_weights_static(d, W, w_bits, w_s8, w_scales, stream=None):
+    """pq_pack_weights without a workspace argument: for callers that cannot allocate device memory
+    (the reduction scratch is a fixed 64 KiB array inside the library; N * K <= 67,108,864)."""
+    _check("pq_pack_weights_static", lib().pq_pack_weights_static(ctypes.byref(d), _ptr(W), _ptr(w_bits), _ptr(w_s8),
+                                                                   _ptr(w_scales), _stream(stream)))
 
 
 def pq_linear_forward(d, X, w_bits, w_s8, w_scales, A, B, Wr, alpha, beta, Y, saved, ws, stream=None):

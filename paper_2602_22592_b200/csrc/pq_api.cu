@@ -137,6 +137,78 @@ static size_t carve_bwd_scratch(const pq_desc* d, void* base, BwdScratch* out) {
 
 static inline bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) != 0; }
 
+// ---------------------------------------------------------------------------
+// Allocation-free weight pack: the fp64 partial sums live in a fixed device array
+// owned by the library instead of a caller-provided workspace.
+// ---------------------------------------------------------------------------
+constexpr int kStaticSlabElems = 16384;    // elements summed into one pair of partials
+constexpr int kStaticMaxSlabs = 4096;      // 4096 x 2 doubles = 64 KiB
+static __device__ __align__(256) double g_pack_scratch[2 * kStaticMaxSlabs];
+
+// One block per slab of kStaticSlabElems consecutive elements: {sum, sum of |.|} in fp64,
+// a fixed order inside the block, so the result does not depend on scheduling.
+__global__ void __launch_bounds__(256) k_weight_slab_sums(const float4* __restrict__ W4, long long n4, double* __restrict__ partial) {
+  const long long base = (long long)blockIdx.x * (kStaticSlabElems / 4);
+  double s = 0.0, a = 0.0;
+  for (int i = threadIdx.x; i < kStaticSlabElems / 4; i += 256) {
+    if (base + i < n4) {
+      const float4 v = __ldg(W4 + base + i);
+      s += (double)v.x + (double)v.y + (double)v.z + (double)v.w;
+      a += (double)fabsf(v.x) + (double)fabsf(v.y) + (double)fabsf(v.z) + (double)fabsf(v.w);
+    }
+  }
+  for (int d = 16; d > 0; d >>= 1) {
+    s += __shfl_xor_sync(0xffffffffu, s, d);
+    a += __shfl_xor_sync(0xffffffffu, a, d);
+  }
+  __shared__ double sh[2][8];
+  if ((threadIdx.x & 31) == 0) { sh[0][threadIdx.x >> 5] = s; sh[1][threadIdx.x >> 5] = a; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double ts = 0.0, ta = 0.0;
+    for (int w = 0; w < 8; ++w) { ts += sh[0][w]; ta += sh[1][w]; }
+    partial[2 * blockIdx.x] = ts;      // every slot that k_binarize_pack reads is written here first:
+    partial[2 * blockIdx.x + 1] = ta;  // nothing left over from an earlier call is ever used
+  }
+}
+
+// In host code the name g_pack_scratch is only a handle for the device array, not a device
+// address (handing it to a kernel would make the kernel touch the wrong memory).  The real
+// address is asked for once per device, with that device current, and cached.
+static int static_scratch_ptr(double** out) {
+  constexpr int kMaxDevices = 64;
+  static double* cache[kMaxDevices] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return PQ_ERR_CUDA;
+  if (!cache[dev]) {
+    double* ptr = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_pack_scratch) != cudaSuccess || !ptr) return PQ_ERR_CUDA;
+    cache[dev] = ptr;
+  }
+  *out = cache[dev];
+  return PQ_OK;
+}
+
+static int pack_static(const float* W, int N, int K, uint32_t* bits, int8_t* s8, float* scales, cudaStream_t st) {
+  const long long elems = (long long)N * K;
+  const long long slabs = (elems + kStaticSlabElems - 1) / kStaticSlabElems;
+  if (slabs > kStaticMaxSlabs) return PQ_ERR_TOO_LARGE;
+  double* scratch = nullptr;
+  int rc = static_scratch_ptr(&scratch);
+  if (rc) return rc;
+  const long long n4 = elems / 4;
+  {
+    LaunchScope ls(KID_PACK_SUMS, st);
+    k_weight_slab_sums<<<(int)slabs, 256, 0, st>>>(reinterpret_cast<const float4*>(W), n4, scratch);
+  }
+  long long g = (n4 + 1023) / 1024;
+  const int grid = (int)(g < 1 ? 1 : (g > 148 * 8 ? 148 * 8 : g));
+  LaunchScope ls(KID_BINARIZE_PACK, st);
+  k_binarize_pack<<<grid, 256, 0, st>>>(reinterpret_cast<const float4*>(W), n4, scratch, (int)slabs, 1.0 / (double)elems, bits,
+                                        reinterpret_cast<uint32_t*>(s8), scales);
+  return cudaGetLastError() == cudaSuccess ? PQ_OK : PQ_ERR_CUDA;
+}
+
 }  // namespace pq
 
 using namespace pq;
@@ -153,6 +225,7 @@ const char* pq_status_string(int s) {
     case PQ_ERR_UNSUPPORTED: return "request not supported";
     case PQ_ERR_CUDA: return "a CUDA call failed";
     case PQ_ERR_TIMEOUT: return "a device-side bounded wait ran out";
+    case PQ_ERR_TOO_LARGE: return "the problem needs more scratch than the library's fixed-size buffer holds";
     default: return "unknown status";
   }
 }
@@ -199,6 +272,13 @@ int pq_pack_weights(const pq_desc* d, const float* W, uint32_t* w_bits, int8_t* 
   if (ws_bytes < pq_workspace_bytes(d, PQ_PHASE_PACK)) return PQ_ERR_WORKSPACE;
   cudaError_t e = launch_pack(W, d->N, d->K, w_bits, w_s8, w_scales, static_cast<double*>(ws), static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? PQ_OK : PQ_ERR_CUDA;
+}
+
+int pq_pack_weights_static(const pq_desc* d, const float* W, uint32_t* w_bits, int8_t* w_s8, float* w_scales, void* stream) {
+  if (!d || !W || !w_bits || !w_scales) return PQ_ERR_NULL;
+  if (d->size != sizeof(pq_desc) || d->N < 1 || d->K < 32 || d->K % 32) return PQ_ERR_SHAPE;
+  if (misaligned(W) || misaligned(w_bits) || misaligned(w_s8)) return PQ_ERR_ALIGN;
+  return pack_static(W, d->N, d->K, w_bits, w_s8, w_scales, static_cast<cudaStream_t>(stream));
 }
 
 int pq_linear_forward(const pq_desc* d, const uint16_t* X, const uint32_t* w_bits, const int8_t* w_s8, const float* w_scales,
