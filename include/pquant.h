@@ -174,6 +174,11 @@ int pq_linear_backward(const pq_desc* d, const uint16_t* dY, const uint16_t* X,
  * M, N, K multiples of 8 (bf16) / 16 (int8). */
 int pq_debug_gemm(int mode, int M, int N, int K, const void* A, const void* B, void* D,
                   void* stream);
+/* Same with the width of the output tiles chosen by the caller (the layer's kernels
+ * use 256, 160 for the forward tile with an HP branch, and narrower pieces in the last
+ * wave): tile_n a multiple of 32 (modes 0, 1) or 64 (modes 2, 3), at most 256. */
+int pq_debug_gemm_tile(int mode, int M, int N, int K, const void* A, const void* B, void* D,
+                       int tile_n, void* stream);
 
 /* Reads the device status word written by a kernel whose bounded wait ran out.
  * Synchronises `stream`.  code = 0 when no wait failed; `where` identifies the

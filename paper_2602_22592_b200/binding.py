@@ -21,7 +21,7 @@ PQ_SCALE_VECTOR = 1
 PQ_PHASE_PACK, PQ_PHASE_FWD, PQ_PHASE_BWD, PQ_PHASE_DECODE = 0, 1, 2, 3
 
 EXPORTS = ("pq_status_string", "pq_workspace_bytes", "pq_saved_bytes", "pq_saved_view_init",
-           "pq_pack_weights", "pq_pack_weights_static", "pq_linear_forward", "pq_linear_backward", "pq_debug_gemm",
+           "pq_pack_weights", "pq_pack_weights_static", "pq_linear_forward", "pq_linear_backward", "pq_debug_gemm", "pq_debug_gemm_tile",
            "pq_device_status", "pq_kernel_launches", "pq_profile_events")
 
 KERNEL_IDS = dict(pack_sums=0, binarize_pack=1, router=2, route_scan=3, act_quant=4, hp_up=5, fwd=6, scatter_rows=7,
@@ -77,6 +77,8 @@ def lib() -> ctypes.CDLL:
         L.pq_linear_backward.argtypes = [dp] + [vp] * 9 + [vp, sz] + [vp] * 7 + [vp, sz, vp]
         L.pq_debug_gemm.restype = ci
         L.pq_debug_gemm.argtypes = [ci, ci, ci, ci, vp, vp, vp, vp]
+        L.pq_debug_gemm_tile.restype = ci
+        L.pq_debug_gemm_tile.argtypes = [ci, ci, ci, ci, vp, vp, vp, ci, vp]
         L.pq_device_status.restype = ci
         L.pq_device_status.argtypes = [vp, ctypes.POINTER(ci), ctypes.POINTER(ci)]
         L.pq_kernel_launches.restype = ctypes.c_longlong
@@ -178,6 +180,10 @@ def pq_linear_backward(d, dY, X, w_s8, w_scales, A, B, Wr, alpha, beta, saved, d
 
 def pq_debug_gemm(mode, M, N, K, A, B, D, stream=None):
     _check("pq_debug_gemm", lib().pq_debug_gemm(mode, M, N, K, _ptr(A), _ptr(B), _ptr(D), _stream(stream)))
+
+
+def pq_debug_gemm_tile(mode, M, N, K, A, B, D, tile_n, stream=None):
+    _check("pq_debug_gemm_tile", lib().pq_debug_gemm_tile(mode, M, N, K, _ptr(A), _ptr(B), _ptr(D), tile_n, _stream(stream)))
 
 
 def pq_device_status(stream=None) -> tuple[int, int]:

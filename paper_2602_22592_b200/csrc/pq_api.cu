@@ -124,7 +124,7 @@ static size_t carve_bwd_scratch(const pq_desc* d, void* base, BwdScratch* out) {
   s.gh = r > 0 ? c.take<uint16_t>((size_t)2 * max_items_of(d) * kTileRows * r) : nullptr;
   s.dl = routed(d) ? c.take<float>(T * E) : nullptr;
   s.dlc = routed(d) ? c.take<uint16_t>(T * 16) : nullptr;
-  s.dbeta_partial = c.take<float>(((K + 255) / 256) * N);
+  s.dbeta_partial = c.take<float>(((K + 31) / 32) * N);   // one slot per 32 columns of K
   s.dalpha_partial = r > 0 ? c.take<float>((size_t)E * N) : nullptr;
   s.dwr_partial = routed(d) ? c.take<float>(((T + 255) / 256) * E * K) : nullptr;
   s.dalpha_vec = c.take<float>(N);
@@ -363,9 +363,9 @@ int pq_linear_backward(const pq_desc* d, const uint16_t* dY, const uint16_t* X, 
   if (routed(d)) {
     if (launch_router_wgrad(sv.xs, sc.dl, d->T, d->K, E, sc.dwr_partial, dWr, nullptr, st) != cudaSuccess) return PQ_ERR_CUDA;
   }
-  // dbeta_n = lam * sum over k-tiles of the partial sign-weighted row sums; scalar form sums over n
-  const int ntk = (d->K + 255) / 256;
-  if (launch_sum_partials(sc.dbeta_partial, ntk, d->N, w_scales, vec ? dbeta : sc.dbeta_vec, st) != cudaSuccess) return PQ_ERR_CUDA;
+  // dbeta_n = lam * sum over the 32-column slots of the partial sign-weighted row sums; scalar form sums over n
+  const int nslots = (d->K + 31) / 32;
+  if (launch_sum_partials(sc.dbeta_partial, nslots, d->N, w_scales, vec ? dbeta : sc.dbeta_vec, st) != cudaSuccess) return PQ_ERR_CUDA;
   if (!vec && launch_sum_to_scalar(sc.dbeta_vec, d->N, dbeta, st) != cudaSuccess) return PQ_ERR_CUDA;
   if (hp) {
     if (launch_sum_partials(sc.dalpha_partial, E, d->N, nullptr, vec ? dalpha : sc.dalpha_vec, st) != cudaSuccess) return PQ_ERR_CUDA;
@@ -380,7 +380,14 @@ int pq_debug_gemm(int mode, int M, int N, int K, const void* A, const void* B, v
   if (!A || !B || !D) return PQ_ERR_NULL;
   if (M < 1 || N < 1 || K < 1 || M % 8 || N % 8 || K % (mode == 0 ? 16 : 8)) return PQ_ERR_SHAPE;
   if (misaligned(A) || misaligned(B) || misaligned(D)) return PQ_ERR_ALIGN;
-  return gemm_debug(mode, M, N, K, A, B, D, static_cast<cudaStream_t>(stream));
+  return gemm_debug(mode, M, N, K, A, B, D, 256, static_cast<cudaStream_t>(stream));
+}
+
+int pq_debug_gemm_tile(int mode, int M, int N, int K, const void* A, const void* B, void* D, int tile_n, void* stream) {
+  if (!A || !B || !D) return PQ_ERR_NULL;
+  if (M < 1 || N < 1 || K < 1 || M % 8 || N % 8 || K % (mode == 0 ? 16 : 8)) return PQ_ERR_SHAPE;
+  if (misaligned(A) || misaligned(B) || misaligned(D)) return PQ_ERR_ALIGN;
+  return gemm_debug(mode, M, N, K, A, B, D, tile_n, static_cast<cudaStream_t>(stream));
 }
 
 long long pq_kernel_launches(void) { return g_launches; }

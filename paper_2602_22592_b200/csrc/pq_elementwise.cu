@@ -15,7 +15,19 @@ long long g_launches = 0;
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) k_weight_partial_sums(const float4* __restrict__ W4, long long n4, double* __restrict__ partial) {
   double s = 0.0, a = 0.0;
-  for (long long i = blockIdx.x * 256LL + threadIdx.x; i < n4; i += gridDim.x * 256LL) {
+  const long long stride = gridDim.x * 256LL;
+  long long i = blockIdx.x * 256LL + threadIdx.x;
+  // four loads in flight per thread; the order of the additions is fixed by the launch shape alone
+  for (; i + 3 * stride < n4; i += 4 * stride) {
+    const float4 v0 = __ldg(W4 + i), v1 = __ldg(W4 + i + stride), v2 = __ldg(W4 + i + 2 * stride), v3 = __ldg(W4 + i + 3 * stride);
+    s += ((double)v0.x + (double)v0.y + (double)v0.z + (double)v0.w) + ((double)v1.x + (double)v1.y + (double)v1.z + (double)v1.w);
+    s += ((double)v2.x + (double)v2.y + (double)v2.z + (double)v2.w) + ((double)v3.x + (double)v3.y + (double)v3.z + (double)v3.w);
+    a += ((double)fabsf(v0.x) + (double)fabsf(v0.y) + (double)fabsf(v0.z) + (double)fabsf(v0.w)) +
+         ((double)fabsf(v1.x) + (double)fabsf(v1.y) + (double)fabsf(v1.z) + (double)fabsf(v1.w));
+    a += ((double)fabsf(v2.x) + (double)fabsf(v2.y) + (double)fabsf(v2.z) + (double)fabsf(v2.w)) +
+         ((double)fabsf(v3.x) + (double)fabsf(v3.y) + (double)fabsf(v3.z) + (double)fabsf(v3.w));
+  }
+  for (; i < n4; i += stride) {
     const float4 v = __ldg(W4 + i);
     s += (double)v.x + (double)v.y + (double)v.z + (double)v.w;
     a += (double)fabsf(v.x) + (double)fabsf(v.y) + (double)fabsf(v.z) + (double)fabsf(v.w);
@@ -66,21 +78,32 @@ __global__ void __launch_bounds__(256) k_binarize_pack(const float4* __restrict_
   if (blockIdx.x == 0 && threadIdx.x == 0) { scales[0] = lam; scales[1] = mu; }
   // n4 is a multiple of 8 (K % 32 == 0), so whole groups of 8 lanes stay together
   const long long n4_pad = (n4 + 31) & ~31LL;
-  for (long long i = blockIdx.x * 256LL + threadIdx.x; i < n4_pad; i += gridDim.x * 256LL) {
-    uint32_t nib = 0, bytes = 0;
-    if (i < n4) {
-      const float4 v = __ldg(W4 + i);
-      const uint32_t b0 = v.x >= mu, b1 = v.y >= mu, b2 = v.z >= mu, b3 = v.w >= mu;
-      nib = b0 | (b1 << 1) | (b2 << 2) | (b3 << 3);
-      // +1 -> 0x01, -1 -> 0xFF, little endian: byte j <-> k + j
-      bytes = (b0 ? 0x01u : 0xFFu) | (b1 ? 0x0100u : 0xFF00u) | (b2 ? 0x010000u : 0xFF0000u) | (b3 ? 0x01000000u : 0xFF000000u);
-      if (s8x4) s8x4[i] = bytes;
+  const long long stride = gridDim.x * 256LL;
+  for (long long i0 = blockIdx.x * 256LL + threadIdx.x; i0 < n4_pad; i0 += 2 * stride) {
+    float4 v[2];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const long long i = i0 + u * stride;
+      v[u] = i < n4 ? __ldg(W4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
-    uint32_t word = nib << (4 * (threadIdx.x & 7));
-    word |= __shfl_xor_sync(0xffffffffu, word, 1);
-    word |= __shfl_xor_sync(0xffffffffu, word, 2);
-    word |= __shfl_xor_sync(0xffffffffu, word, 4);
-    if ((threadIdx.x & 7) == 0 && i < n4) bits[i >> 3] = word;
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const long long i = i0 + u * stride;
+      if (i >= n4_pad) break;          // uniform over the warp: stride and n4_pad are multiples of 32
+      uint32_t nib = 0;
+      if (i < n4) {
+        const uint32_t b0 = v[u].x >= mu, b1 = v[u].y >= mu, b2 = v[u].z >= mu, b3 = v[u].w >= mu;
+        nib = b0 | (b1 << 1) | (b2 << 2) | (b3 << 3);
+        // +1 -> 0x01, -1 -> 0xFF, little endian: byte j <-> k + j
+        const uint32_t bytes = (b0 ? 0x01u : 0xFFu) | (b1 ? 0x0100u : 0xFF00u) | (b2 ? 0x010000u : 0xFF0000u) | (b3 ? 0x01000000u : 0xFF000000u);
+        if (s8x4) s8x4[i] = bytes;
+      }
+      uint32_t word = nib << (4 * (threadIdx.x & 7));
+      word |= __shfl_xor_sync(0xffffffffu, word, 1);
+      word |= __shfl_xor_sync(0xffffffffu, word, 2);
+      word |= __shfl_xor_sync(0xffffffffu, word, 4);
+      if ((threadIdx.x & 7) == 0 && i < n4) bits[i >> 3] = word;
+    }
   }
 }
 
@@ -172,37 +195,53 @@ __global__ void __launch_bounds__(256) k_router(const uint4* __restrict__ X, con
 // units over which the token contraction of dA and dB is split across CTAs.
 // One block; the work is a few hundred integers.
 // ---------------------------------------------------------------------------
-// Builder of one chunk table: consecutive items of one expert, at most `size` items each.
-struct ChunkBuilder {
-  int4* out; int* begin; int size; int n = 0, cur_e = -1, cur_b = 0, cur_n = 0, next_e = 0;
-  __device__ void flush() {
-    if (cur_n > 0) { out[n] = make_int4(cur_e, cur_b, cur_b + cur_n, 0); ++n; }
-    cur_n = 0;
+// Items of one 128-row tile [r0, r1) of the sorted order: experts e0 <= e < E whose non-empty range
+// [off[e], off[e+1]) meets the tile.  Returns the number of items; calls f(k, e, lo, hi) for the k-th.
+template <class F>
+__device__ __forceinline__ int tile_items(const int* off, int Ee, int r0, int r1, F f) {
+  int n = 0;
+  for (int e = 0; e < Ee; ++e) {
+    const int lo = max(off[e], r0), hi = min(off[e + 1], r1);
+    if (hi > lo) { f(n, e, lo, hi); ++n; }
   }
-  __device__ void add(int item, int e) {
-    if (e != cur_e || cur_n == size) {
-      flush();
-      cur_b = item;
-      if (e != cur_e) {
-        for (; next_e <= e; ++next_e) begin[next_e] = n;  // experts without items get an empty range
-        cur_e = e;
-      }
+  return n;
+}
+
+// One chunk table: consecutive items of one expert, at most `size` items each.  Thread 0 lays out the
+// experts' chunk ranges (<= 16 experts), then all threads fill the entries.
+__device__ __forceinline__ void build_chunks(int Ee, const int* item_begin /*shared, Ee+1*/, int size, int4* out, int* begin, int* count,
+                                             int* sh_begin /*shared, Ee+1*/) {
+  if (threadIdx.x == 0) {
+    int n = 0;
+    for (int e = 0; e < Ee; ++e) {
+      sh_begin[e] = n;
+      n += (item_begin[e + 1] - item_begin[e] + size - 1) / size;
     }
-    ++cur_n;
-  }
-  __device__ void finish(int Ee, int* count) {
-    flush();
-    for (; next_e <= Ee; ++next_e) begin[next_e] = n;
+    sh_begin[Ee] = n;
     count[0] = n;
   }
-};
+  __syncthreads();
+  if (threadIdx.x <= Ee) begin[threadIdx.x] = sh_begin[threadIdx.x];
+  for (int c = threadIdx.x; c < sh_begin[Ee]; c += blockDim.x) {
+    int e = 0;
+    while (sh_begin[e + 1] <= c) ++e;
+    const int first = item_begin[e] + (c - sh_begin[e]) * size;
+    out[c] = make_int4(e, first, min(first + size, item_begin[e + 1]), 0);
+  }
+  __syncthreads();
+}
 
 __global__ void __launch_bounds__(512) k_route_scan(int T, int E, int nblocks, const int* __restrict__ block_counts,
                                                     int* __restrict__ block_base, int* __restrict__ offsets, RoutingTables rt,
                                                     int chunk_a, int chunk_b) {
   __shared__ int off[kMaxExperts + 1];
   __shared__ int total[kMaxExperts];
+  __shared__ int item_begin[kMaxExperts + 1];
+  __shared__ int chunk_begin[kMaxExperts + 1];
+  __shared__ int warp_sums[16];
+  __shared__ int carry_sh;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int Ee = E < 1 ? 1 : E;
   if (E > 1 && warp < E) {
     // exclusive scan of this expert's per-block counts, 32 blocks at a time
     int carry = 0;
@@ -221,7 +260,6 @@ __global__ void __launch_bounds__(512) k_route_scan(int T, int E, int nblocks, c
   }
   __syncthreads();
   if (threadIdx.x == 0) {
-    const int Ee = E < 1 ? 1 : E;
     if (E <= 1) {
       off[0] = 0; off[1] = T;
     } else {
@@ -229,33 +267,55 @@ __global__ void __launch_bounds__(512) k_route_scan(int T, int E, int nblocks, c
       for (int e = 0; e < E; ++e) { off[e] = run; run += total[e]; }
       off[E] = run;
     }
-    for (int e = 0; e <= Ee; ++e) offsets[e] = off[e];
-    const int mtiles = (T + kTileRows - 1) / kTileRows;
-    int next_item_e = 0;  // experts whose first item index is still to be recorded
-    ChunkBuilder ca{rt.chunks_a, rt.expert_chunk_begin_a, chunk_a}, cb{rt.chunks_b, rt.expert_chunk_begin_b, chunk_b};
-    int n = 0, e = 0;
-    for (int tile = 0; tile < mtiles; ++tile) {
-      rt.tile_item_begin[tile] = n;
-      const int r0 = tile * kTileRows, r1 = min(T, r0 + kTileRows);
-      while (e < Ee && off[e + 1] <= r0) ++e;  // first expert reaching into this tile
-      for (int ee = e; ee < Ee && off[ee] < r1; ++ee) {
-        const int lo = max(off[ee], r0), hi = min(off[ee + 1], r1);
-        if (hi > lo) {
-          rt.items[n] = make_int4(tile, ee, lo - r0, hi - r0);
-          // first item of each expert (items ascend in expert)
-          for (; next_item_e <= ee; ++next_item_e) rt.expert_item_begin[next_item_e] = n;
-          ca.add(n, ee);
-          cb.add(n, ee);
-          ++n;
-        }
-      }
-    }
-    rt.tile_item_begin[mtiles] = n;
-    rt.n_items[0] = n;
-    for (; next_item_e <= Ee; ++next_item_e) rt.expert_item_begin[next_item_e] = n;
-    ca.finish(Ee, rt.n_chunks_a);
-    cb.finish(Ee, rt.n_chunks_b);
+    carry_sh = 0;
   }
+  __syncthreads();
+  if (threadIdx.x <= Ee) offsets[threadIdx.x] = off[threadIdx.x];
+
+  // items: one thread per tile counts its items, a block-wide scan places them
+  const int mtiles = (T + kTileRows - 1) / kTileRows;
+  for (int base = 0; base < mtiles; base += blockDim.x) {
+    const int tile = base + threadIdx.x;
+    const int r0 = tile * kTileRows, r1 = min(T, r0 + kTileRows);
+    const int cnt = tile < mtiles ? tile_items(off, Ee, r0, r1, [](int, int, int, int) {}) : 0;
+    int inc = cnt;
+    for (int d = 1; d < 32; d <<= 1) {
+      const int u = __shfl_up_sync(0xffffffffu, inc, d);
+      if (lane >= d) inc += u;
+    }
+    if (lane == 31) warp_sums[warp] = inc;
+    __syncthreads();
+    int before = carry_sh;
+    for (int w = 0; w < warp; ++w) before += warp_sums[w];
+    const int first = before + inc - cnt;
+    if (tile < mtiles) {
+      rt.tile_item_begin[tile] = first;
+      tile_items(off, Ee, r0, r1, [&](int k, int e, int lo, int hi) { rt.items[first + k] = make_int4(tile, e, lo - r0, hi - r0); });
+    }
+    __syncthreads();
+    if (threadIdx.x == blockDim.x - 1) carry_sh = first + cnt;
+    __syncthreads();
+  }
+  const int n_items = carry_sh;
+  if (threadIdx.x == 0) { rt.tile_item_begin[mtiles] = n_items; rt.n_items[0] = n_items; }
+  // first item of each expert: the first item of the tile holding its first row, plus the items of the
+  // non-empty experts below it in that tile; an empty expert points at its successor's first item
+  if (threadIdx.x <= Ee) {
+    int e = threadIdx.x;
+    while (e < Ee && off[e + 1] == off[e]) ++e;
+    int idx = n_items;
+    if (e < Ee) {
+      const int tile = off[e] / kTileRows, r0 = tile * kTileRows;
+      idx = rt.tile_item_begin[tile];   // written above by this block, ordered by the barriers of the loop
+      for (int f = 0; f < e; ++f)
+        if (min(off[f + 1], r0 + kTileRows) > max(off[f], r0)) ++idx;
+    }
+    item_begin[threadIdx.x] = idx;
+    rt.expert_item_begin[threadIdx.x] = idx;
+  }
+  __syncthreads();
+  build_chunks(Ee, item_begin, chunk_a, rt.chunks_a, rt.expert_chunk_begin_a, rt.n_chunks_a, chunk_begin);
+  build_chunks(Ee, item_begin, chunk_b, rt.chunks_b, rt.expert_chunk_begin_b, rt.n_chunks_b, chunk_begin);
 }
 
 // ---------------------------------------------------------------------------
@@ -265,15 +325,42 @@ __global__ void __launch_bounds__(512) k_route_scan(int T, int E, int nblocks, c
 // stable): q (int8), xt = q / gamma (bf16, the backward's operand) and, with
 // routing, a bf16 copy of the row itself plus its gate and probabilities.
 // ---------------------------------------------------------------------------
+// WPR warps share one token row.  CH > 0: every lane keeps its CH 16-byte pieces of the row in registers
+// between the absmax pass and the quantising pass (rows of up to 256 * CH * WPR elements), so X is read
+// once; CH = 0 reads the row twice.
+template <int CH, int WPR>
 __global__ void __launch_bounds__(256) k_act_quant(const uint4* __restrict__ X, int T, int K, int E, const int* __restrict__ expert,
                                                    const int* __restrict__ block_base, const int* __restrict__ offsets,
                                                    const float* __restrict__ gate_tok, const float* __restrict__ probs_tok,
                                                    uint2* __restrict__ q, uint4* __restrict__ xt, uint4* __restrict__ xs,
                                                    float* __restrict__ gamma_s, float* __restrict__ gate_s, float* __restrict__ probs_s,
                                                    int* __restrict__ perm, int* __restrict__ pos) {
+  __shared__ float amax_sh[8];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int t = blockIdx.x * 8 + warp;
-  if (t >= T) return;
+  const int sub = warp % WPR, slot = sub * 32 + lane;   // this lane's first 16-byte piece of the row
+  const int t_raw = blockIdx.x * (8 / WPR) + warp / WPR;
+  const bool valid = t_raw < T;
+  if (WPR == 1 && !valid) return;
+  const int t = valid ? t_raw : T - 1;                  // idle warps of a shared row keep the barrier company
+  const int chunks = K >> 3;
+  const uint4* xrow = X + (long long)t * chunks;
+  uint4 held[CH > 0 ? CH : 1];
+  float amax = 0.f;
+  auto fold = [&](const uint4& v) {
+    amax = fmaxf(amax, fmaxf(fmaxf(fabsf(bf16lo(v.x)), fabsf(bf16hi(v.x))), fmaxf(fabsf(bf16lo(v.y)), fabsf(bf16hi(v.y)))));
+    amax = fmaxf(amax, fmaxf(fmaxf(fabsf(bf16lo(v.z)), fabsf(bf16hi(v.z))), fmaxf(fabsf(bf16lo(v.w)), fabsf(bf16hi(v.w)))));
+  };
+  if (CH > 0) {
+#pragma unroll
+    for (int i = 0; i < CH; ++i) {
+      const int c = slot + 32 * WPR * i;
+      held[i] = c < chunks ? __ldg(xrow + c) : make_uint4(0u, 0u, 0u, 0u);
+    }
+#pragma unroll
+    for (int i = 0; i < CH; ++i) fold(held[i]);
+  } else {
+    for (int c = slot; c < chunks; c += 32 * WPR) fold(__ldg(xrow + c));
+  }
   int p = t;
   if (E > 1) {
     const int e = expert[t];
@@ -283,29 +370,28 @@ __global__ void __launch_bounds__(256) k_act_quant(const uint4* __restrict__ X, 
     const int rank = __popc(same & ((1u << (t - first)) - 1u));
     p = offsets[e] + block_base[blk * E + e] + rank;
   }
-  const int chunks = K >> 3;
-  const uint4* xrow = X + (long long)t * chunks;
-  float amax = 0.f;
-  for (int c = lane; c < chunks; c += 32) {
-    const uint4 v = __ldg(xrow + c);
-    amax = fmaxf(amax, fmaxf(fmaxf(fabsf(bf16lo(v.x)), fabsf(bf16hi(v.x))), fmaxf(fabsf(bf16lo(v.y)), fabsf(bf16hi(v.y)))));
-    amax = fmaxf(amax, fmaxf(fmaxf(fabsf(bf16lo(v.z)), fabsf(bf16hi(v.z))), fmaxf(fabsf(bf16lo(v.w)), fabsf(bf16hi(v.w)))));
-  }
   for (int d = 16; d > 0; d >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, d));
+  if (WPR > 1) {
+    if (lane == 0) amax_sh[warp] = amax;
+    __syncthreads();
+    const int w0 = warp - sub;
+#pragma unroll
+    for (int w = 0; w < WPR; ++w) amax = fmaxf(amax, amax_sh[w0 + w]);
+    if (!valid) return;
+  }
   const float gamma = __fdiv_rn(kActQmax, fmaxf(amax, kActAmaxFloor));
   const float inv_gamma = __fdiv_rn(1.0f, gamma);
-  if (lane == 0) {
+  if (lane == 0 && sub == 0) {
     gamma_s[p] = gamma;
     perm[p] = t;
     pos[t] = p;
     gate_s[p] = (E > 1) ? gate_tok[t] : 1.0f;
   }
-  if (E > 1 && lane < E) probs_s[(long long)p * E + lane] = probs_tok[(long long)t * E + lane];
+  if (E > 1 && sub == 0 && lane < E) probs_s[(long long)p * E + lane] = probs_tok[(long long)t * E + lane];
   uint2* qrow = q + (long long)p * chunks;
   uint4* xtrow = xt ? xt + (long long)p * chunks : nullptr;
   uint4* xsrow = xs ? xs + (long long)p * chunks : nullptr;
-  for (int c = lane; c < chunks; c += 32) {
-    const uint4 v = __ldg(xrow + c);
+  auto emit = [&](int c, const uint4& v) {
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
     int qi[8];
 #pragma unroll
@@ -327,6 +413,15 @@ __global__ void __launch_bounds__(256) k_act_quant(const uint4* __restrict__ X, 
       xtrow[c] = o;
     }
     if (xsrow) xsrow[c] = v;
+  };
+  if (CH > 0) {
+#pragma unroll
+    for (int i = 0; i < CH; ++i) {
+      const int c = slot + 32 * WPR * i;
+      if (c < chunks) emit(c, held[i]);
+    }
+  } else {
+    for (int c = slot; c < chunks; c += 32 * WPR) emit(c, __ldg(xrow + c));
   }
 }
 
@@ -520,9 +615,17 @@ cudaError_t launch_route_and_quant(const uint16_t* X, const uint16_t* Wr, int T,
   { LaunchScope ls(KID_ROUTE_SCAN, st);
   k_route_scan<<<1, 512, 0, st>>>(T, E, nblocks, sc.block_counts, sc.block_base, sv.offsets, sv.rt, sv.chunk_a, sv.chunk_b); }
   LaunchScope ls(KID_ACT_QUANT, st);
-  k_act_quant<<<(T + 7) / 8, 256, 0, st>>>(reinterpret_cast<const uint4*>(X), T, K, E, sv.expert, sc.block_base, sv.offsets, sc.gate_tok,
-                                           sc.probs_tok, reinterpret_cast<uint2*>(sv.q), reinterpret_cast<uint4*>(sv.xt),
-                                           reinterpret_cast<uint4*>(sv.xs), sv.gamma, sv.gate, sv.probs, sv.perm, sv.pos);
+  const int per_lane = (K / 8 + 31) / 32;   // 16-byte pieces of a row per lane if one warp took the whole row
+  auto kern = k_act_quant<0, 1>;
+  int wpr = 1;
+  if (per_lane <= 4) kern = k_act_quant<4, 1>;
+  else if (per_lane <= 8) kern = k_act_quant<8, 1>;
+  else if (per_lane <= 16) { kern = k_act_quant<8, 2>; wpr = 2; }
+  else if (per_lane <= 32) { kern = k_act_quant<8, 4>; wpr = 4; }
+  const int rows_per_block = 8 / wpr;
+  kern<<<(T + rows_per_block - 1) / rows_per_block, 256, 0, st>>>(reinterpret_cast<const uint4*>(X), T, K, E, sv.expert, sc.block_base, sv.offsets, sc.gate_tok,
+                                    sc.probs_tok, reinterpret_cast<uint2*>(sv.q), reinterpret_cast<uint4*>(sv.xt),
+                                    reinterpret_cast<uint4*>(sv.xs), sv.gamma, sv.gate, sv.probs, sv.perm, sv.pos);
   return cudaGetLastError();
 }
 

@@ -3,6 +3,8 @@
 //              Y = alpha g (H B_e^T) + beta (lam/gamma) (q S^T)      (Eq. 10, 11)
 //   backward : dH, dX, dW, dB, dA of the straight-through estimator  (App. B.1)
 //   debug    : raw accumulators of one contraction, for bit-exact tests
+#include <type_traits>
+
 #include "pq_gemm.cuh"
 #include "pq_kernels.cuh"
 
@@ -35,9 +37,9 @@ static bool make_map(CUtensorMap* m, bool is_i8, const void* base, int rank, con
   const int eb = is_i8 ? 1 : 2;
   if ((reinterpret_cast<uintptr_t>(base) & 15) != 0) return false;
   if (box[0] * eb != 128) return false;
-  cuuint64_t gd[3];
-  cuuint64_t gs[2];
-  cuuint32_t bx[3], es[3];
+  cuuint64_t gd[4];
+  cuuint64_t gs[3];
+  cuuint32_t bx[4], es[4];
   for (int i = 0; i < rank; ++i) {
     gd[i] = dims[i];
     bx[i] = box[i];
@@ -67,6 +69,22 @@ static bool map3d(CUtensorMap* m, const void* base, uint64_t inner, uint64_t mid
   return make_map(m, false, base, 3, dims, strides, box);
 }
 
+// MN-major operand: matrix [batch][k_total][mn_total] with mn contiguous, read in 64 (mn) x 64 (k) boxes.
+// When mn_total is a multiple of 64 the map views the 64-wide column blocks as a dimension of their own,
+// (64, k_total, mn_total / 64[, batch]) -- base_rank 2 or 3 says whether the operand has the batch dimension --, so that ONE load delivers `nblk` boxes back to back; *blk = nblk.
+// Otherwise (a narrower last block would alias the next row) a plain map with one box per load; *blk = 0.
+static bool map_mn(CUtensorMap* m, int* blk, const void* base, uint64_t mn_total, uint64_t k_total, int base_rank, uint64_t batch, int nblk) {
+  if (mn_total % 64 == 0) {
+    *blk = nblk;
+    const uint64_t dims[4] = {64, k_total, mn_total / 64, batch};
+    const uint64_t strides[3] = {mn_total * 2, 128, mn_total * k_total * 2};
+    const uint32_t box[4] = {64, 64, (uint32_t)nblk, 1};
+    return make_map(m, false, base, base_rank + 1, dims, strides, box);
+  }
+  *blk = 0;
+  return base_rank == 3 ? map3d(m, base, mn_total, k_total, batch, 64, 64) : map2d(m, false, base, mn_total, k_total, 64, 64);
+}
+
 static int g_sm_count = 0;
 static int sm_count() {
   if (!g_sm_count) {
@@ -78,18 +96,27 @@ static int sm_count() {
   return g_sm_count;
 }
 
+static int grid_for_tiles(int max_tiles) {
+  int grid = max_tiles < sm_count() ? max_tiles : sm_count();
+  return grid < 1 ? 1 : grid;
+}
+
 template <class Params>
 static int launch_gemm(int kernel_id, void (*kernel)(Params), const Params& p, int max_tiles, cudaStream_t st) {
   // (cudaFuncSetAttribute is cheap and idempotent; calling it per launch keeps this free of static state per kernel)
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes) != cudaSuccess) return PQ_ERR_CUDA;
-  int grid = max_tiles < sm_count() ? max_tiles : sm_count();
-  if (grid < 1) grid = 1;
+  const int grid = grid_for_tiles(max_tiles);
   LaunchScope ls(kernel_id, st);
   kernel<<<grid, kGemmThreads, kGemmSmemBytes, st>>>(p);
   return cudaGetLastError() == cudaSuccess ? PQ_OK : PQ_ERR_CUDA;
 }
 
 __device__ __forceinline__ int round_up(int x, int m) { return (x + m - 1) / m * m; }
+// width actually contracted for a tile that starts at n0: the tile's width, cut at the matrix edge
+__device__ __forceinline__ int clip_bn(int bn, int n0, int n_total, int granule) {
+  const int left = round_up(n_total - n0, granule);
+  return left < bn ? (left > 0 ? left : granule) : bn;
+}
 
 // Intermediates that feed a second tensor-core product (H, g H, dH / c) are kept
 // as TWO bf16 planes, v ~= hi + lo with hi = bf16(v), lo = bf16(v - hi): about 16
@@ -106,33 +133,34 @@ static inline int h_round_up(int x, int m) { return (x + m - 1) / m * m; }
 // debug: D[M,N] = contraction of A and B in one of the four operand forms
 // ---------------------------------------------------------------------------
 struct DebugProblem {
-  static constexpr int kAccPerTile = 1;
+  using Acc = AccDouble;
   struct Params {
     CUtensorMap ta, tb;
-    int mode, M, N, K, ntn;
+    TileGrid g;
+    int mode, M, N, K, a_blk, b_blk;
     void* D;
   };
-  struct Tile { int m, n; };
-  __device__ static int num_tiles(const Params& p) { return ((p.M + 127) / 128) * p.ntn; }
-  __device__ static void tile_init(const Params& p, int i, Tile& t) { t.m = i / p.ntn; t.n = i % p.ntn; }
+  struct Tile { TileCoord c; };
+  __device__ static int num_tiles(const Params& p) { return p.g.total; }
+  __device__ static void tile_init(const Params& p, int i, Tile& t) { t.c = tile_coord(p.g, i); }
   __device__ static int num_segments(const Params&, const Tile&) { return 1; }
   __device__ static void segment(const Params& p, const Tile& t, int, Segment& s) {
-    s.mode = p.mode; s.acc = 0; s.bn = 256; s.ksteps = 4;
+    s.mode = p.mode; s.acc = 0; s.ksteps = 4; s.b_box = p.g.bn; s.a_blk = p.a_blk; s.b_blk = p.b_blk;
+    s.bn = clip_bn(t.c.bn, t.c.n0, p.N, p.mode >= MODE_BF_KM ? 64 : 32);
     const int bk = p.mode == MODE_I8_KK ? 128 : 64;
     s.nkb = (p.K + bk - 1) / bk;
     s.ta = &p.ta; s.tb = &p.tb; s.a_rank = 2; s.b_rank = 2; s.a_z = 0; s.b_z = 0;
-    if (p.mode == MODE_BF_MM) { s.a_x = t.m * 128; s.a_y = 0; } else { s.a_x = 0; s.a_y = t.m * 128; }
-    if (p.mode >= MODE_BF_KM) { s.b_x = t.n * 256; s.b_y = 0; } else { s.b_x = 0; s.b_y = t.n * 256; }
-    s.b_bytes = kStageBBytes;
+    if (p.mode == MODE_BF_MM) { s.a_x = t.c.m * 128; s.a_y = 0; } else { s.a_x = 0; s.a_y = t.c.m * 128; }
+    if (p.mode >= MODE_BF_KM) { s.b_x = t.c.n0; s.b_y = 0; } else { s.b_x = 0; s.b_y = t.c.n0; }
   }
-  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane, uint8_t* stage) {
-    const int row = t.m * 128 + quad * 32 + lane;
+  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t tacc, uint32_t, int quad, int half, int lane, uint8_t* stage) {
+    const int row = t.c.m * 128 + quad * 32 + lane;
     uint32_t* D = reinterpret_cast<uint32_t*>(p.D);
-    for (int c = 0; c < 8; ++c) {
-      const int n0 = t.n * 256 + c * 32;
+    for (int c = half; c * 32 < t.c.bn; c += 2) {
+      const int n0 = t.c.n0 + c * 32;
       if (n0 >= p.N) break;
       uint32_t v[32];
-      tmem_ld32(taddr + c * 32, v);
+      tmem_ld32(tacc + c * 32, v);
       tmem_ld_wait();
       uint4 o[8];
 #pragma unroll
@@ -144,35 +172,40 @@ struct DebugProblem {
 };
 PQ_DEFINE_GEMM_KERNEL(k_gemm_debug, DebugProblem)
 
-int gemm_debug(int mode, int M, int N, int K, const void* A, const void* B, void* D, cudaStream_t st) {
+int gemm_debug(int mode, int M, int N, int K, const void* A, const void* B, void* D, int tile_n, cudaStream_t st) {
   DebugProblem::Params p;
-  p.mode = mode; p.M = M; p.N = N; p.K = K; p.D = D; p.ntn = (N + 255) / 256;
+  p.mode = mode; p.M = M; p.N = N; p.K = K; p.D = D; p.a_blk = 0; p.b_blk = 0;
+  const int granule = mode >= MODE_BF_KM ? 64 : 32;
+  if (tile_n <= 0) tile_n = 256;
+  if (tile_n > 256 || tile_n % granule) return PQ_ERR_SHAPE;
+  const int mt = (M + 127) / 128, nt = (N + tile_n - 1) / tile_n;
+  p.g = make_tile_grid(mt, nt, tile_n);
   bool ok = true;
   switch (mode) {
     case MODE_I8_KK:
-      ok = map2d(&p.ta, true, A, K, M, 128, 128) && map2d(&p.tb, true, B, K, N, 128, 256);
+      ok = map2d(&p.ta, true, A, K, M, 128, 128) && map2d(&p.tb, true, B, K, N, 128, tile_n);
       break;
     case MODE_BF_KK:
-      ok = map2d(&p.ta, false, A, K, M, 64, 128) && map2d(&p.tb, false, B, K, N, 64, 256);
+      ok = map2d(&p.ta, false, A, K, M, 64, 128) && map2d(&p.tb, false, B, K, N, 64, tile_n);
       break;
     case MODE_BF_KM:
-      ok = map2d(&p.ta, false, A, K, M, 64, 128) && map2d(&p.tb, false, B, N, K, 64, 64);
+      ok = map2d(&p.ta, false, A, K, M, 64, 128) && map_mn(&p.tb, &p.b_blk, B, N, K, 2, 1, tile_n / 64);
       break;
     case MODE_BF_MM:
-      ok = map2d(&p.ta, false, A, M, K, 64, 64) && map2d(&p.tb, false, B, N, K, 64, 64);
+      ok = map_mn(&p.ta, &p.a_blk, A, M, K, 2, 1, 2) && map_mn(&p.tb, &p.b_blk, B, N, K, 2, 1, tile_n / 64);
       break;
     default:
       return PQ_ERR_UNSUPPORTED;
   }
   if (!ok) return PQ_ERR_CUDA;
-  return launch_gemm(KID_DEBUG, k_gemm_debug, p, ((M + 127) / 128) * p.ntn, st);
+  return launch_gemm(KID_DEBUG, k_gemm_debug, p, p.g.total, st);
 }
 
 // ---------------------------------------------------------------------------
 // F1: hidden activations of the HP branch, H = X_sorted A_e^T, one tile per item
 // ---------------------------------------------------------------------------
 struct HpUpProblem {
-  static constexpr int kAccPerTile = 1;
+  using Acc = AccDouble;
   struct Params {
     CUtensorMap tx, ta;  // X sorted [T,K]; A [E,r,K]
     RoutingTables rt;
@@ -187,14 +220,14 @@ struct HpUpProblem {
     s.mode = MODE_BF_KK; s.acc = 0; s.bn = p.bn; s.ksteps = 4; s.nkb = (p.K + 63) / 64;
     s.ta = &p.tx; s.a_rank = 2; s.a_x = 0; s.a_y = t.it.x * 128; s.a_z = 0;
     s.tb = &p.ta; s.b_rank = 3; s.b_x = 0; s.b_y = 0; s.b_z = t.it.y;
-    s.b_bytes = p.bn * 128;
+    s.b_box = p.bn; s.a_blk = 0; s.b_blk = 0;
   }
-  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane, uint8_t* stage) {
+  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, uint32_t, int quad, int half, int lane, uint8_t* stage) {
     const int row = quad * 32 + lane;
     const bool live = row >= t.it.z && row < t.it.w;
     uint4* out_hi = reinterpret_cast<uint4*>(p.H + ((long long)t.item * 128 + row) * p.r);
     uint4* out_lo = reinterpret_cast<uint4*>(p.H + ((long long)p.item_rows + t.item * 128 + row) * p.r);
-    for (int c = 0; c * 32 < p.r; ++c) {
+    for (int c = half; c * 32 < p.r; c += 2) {
       uint32_t v[32];
       tmem_ld32(taddr + c * 32, v);
       tmem_ld_wait();
@@ -223,10 +256,12 @@ PQ_DEFINE_GEMM_KERNEL(k_gemm_hp_up, HpUpProblem)
 // ---------------------------------------------------------------------------
 template <bool HP>
 struct FwdProblem {
-  static constexpr int kAccPerTile = HP ? 2 : 1;
+  // with the HP branch a tile holds an int32 and an fp32 accumulator of 256 columns each: all of TMEM
+  using Acc = typename std::conditional<HP, AccPair, AccDouble>::type;
   struct Params {
     CUtensorMap tq, ts, th, tb;  // q [T,K] s8; S [N,K] s8; H [items*128,r]; B [E,N,r]
     RoutingTables rt;
+    TileGrid g;
     const int* perm;
     const float* gamma;
     const float* gate;
@@ -234,76 +269,113 @@ struct FwdProblem {
     const float* alpha;
     const float* beta;
     uint16_t* Y;
-    int T, N, K, r, sstride, ntn, item_rows;
+    int T, N, K, r, sstride, item_rows;
   };
-  struct Tile { int m, n, ib, ie; };
-  __device__ static int num_tiles(const Params& p) { return ((p.T + 127) / 128) * p.ntn; }
+  struct Tile { TileCoord c; int bn, ib, ie; };
+  __device__ static int num_tiles(const Params& p) { return p.g.total; }
   __device__ static void tile_init(const Params& p, int i, Tile& t) {
-    t.m = i / p.ntn; t.n = i % p.ntn;
-    if (HP) { t.ib = p.rt.tile_item_begin[t.m]; t.ie = p.rt.tile_item_begin[t.m + 1]; } else { t.ib = t.ie = 0; }
+    t.c = tile_coord(p.g, i);
+    t.bn = clip_bn(t.c.bn, t.c.n0, p.N, 32);
+    if (HP) { t.ib = p.rt.tile_item_begin[t.c.m]; t.ie = p.rt.tile_item_begin[t.c.m + 1]; } else { t.ib = t.ie = 0; }
   }
-  __device__ static int num_segments(const Params&, const Tile& t) { return 1 + 2 * (t.ie - t.ib); }
+  // The HP product uses the leading bf16 plane of H only: its 2^-9 relative rounding is of the size of the
+  // output's own rounding to bf16; the second plane serves the backward pass, whose sums are longer.
+  __device__ static int num_segments(const Params&, const Tile& t) { return 1 + (t.ie - t.ib); }
   __device__ static void segment(const Params& p, const Tile& t, int i, Segment& s) {
-    s.bn = 256; s.ksteps = 4; s.a_z = 0; s.b_z = 0; s.b_bytes = kStageBBytes;
+    s.bn = t.bn; s.ksteps = 4; s.a_z = 0; s.b_z = 0; s.b_box = 256; s.a_blk = 0; s.b_blk = 0;
     if (i == 0) {
       s.mode = MODE_I8_KK; s.acc = 0; s.nkb = (p.K + 127) / 128;
-      s.ta = &p.tq; s.a_rank = 2; s.a_x = 0; s.a_y = t.m * 128;
-      s.tb = &p.ts; s.b_rank = 2; s.b_x = 0; s.b_y = t.n * 256;
+      s.ta = &p.tq; s.a_rank = 2; s.a_x = 0; s.a_y = t.c.m * 128;
+      s.tb = &p.ts; s.b_rank = 2; s.b_x = 0; s.b_y = t.c.n0;
     } else {
-      const int item = t.ib + ((i - 1) >> 1), plane = (i - 1) & 1;
+      const int item = t.ib + (i - 1);
       const int e = p.rt.items[item].y;
       s.mode = MODE_BF_KK; s.acc = 1; s.nkb = (p.r + 63) / 64;
-      s.ta = &p.th; s.a_rank = 2; s.a_x = 0; s.a_y = plane * p.item_rows + item * 128;
-      s.tb = &p.tb; s.b_rank = 3; s.b_x = 0; s.b_y = t.n * 256; s.b_z = e;
+      s.ta = &p.th; s.a_rank = 2; s.a_x = 0; s.a_y = item * 128;
+      s.tb = &p.tb; s.b_rank = 3; s.b_x = 0; s.b_y = t.c.n0; s.b_z = e;
     }
   }
-  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane, uint8_t* stage) {
-    const int pos = t.m * 128 + quad * 32 + lane;
+  // y = cb_n * acc + ca_n * z for 32 consecutive columns starting at n, packed to 16 bf16 pairs
+  template <bool VEC>
+  __device__ static __forceinline__ void combine32(const Params& p, int n, float cb, float ca, const uint32_t (&a)[32], const uint32_t (&z)[32],
+                                                  uint4* out) {
+    uint32_t w[16];
+#pragma unroll
+    for (int q4 = 0; q4 < 8; ++q4) {
+      float b4[4] = {cb, cb, cb, cb}, a4[4] = {ca, ca, ca, ca};
+      if (VEC) {
+        const float4 bv = __ldg(reinterpret_cast<const float4*>(p.beta + n) + q4);
+        b4[0] *= bv.x; b4[1] *= bv.y; b4[2] *= bv.z; b4[3] *= bv.w;
+        if (HP) {
+          const float4 av = __ldg(reinterpret_cast<const float4*>(p.alpha + n) + q4);
+          a4[0] *= av.x; a4[1] *= av.y; a4[2] *= av.z; a4[3] *= av.w;
+        }
+      }
+      float y[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        y[u] = b4[u] * (float)(int)a[4 * q4 + u];
+        if (HP) y[u] = fmaf(a4[u], __uint_as_float(z[4 * q4 + u]), y[u]);
+      }
+      w[2 * q4] = pack_bf16x2(y[0], y[1]);
+      w[2 * q4 + 1] = pack_bf16x2(y[2], y[3]);
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) out[j] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+  }
+  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t tacc, uint32_t tz, int quad, int half, int lane, uint8_t* stage) {
+    const int pos = t.c.m * 128 + quad * 32 + lane;
     const bool live = pos < p.T;
     const int token = live ? (p.perm ? p.perm[pos] : pos) : 0;
-    const float s1 = live ? __fdiv_rn(p.w_scales[0], p.gamma[pos]) : 0.f;
-    const float g = (HP && live) ? p.gate[pos] : 0.f;
+    // per-row factors: 1-bit branch lam / gamma_t (Eq. 10), HP branch g_t; scalar feature scales folded in
+    float cb = live ? __fdiv_rn(p.w_scales[0], p.gamma[pos]) : 0.f;
+    float ca = (HP && live) ? p.gate[pos] : 0.f;
+    const bool vec = p.sstride != 0;
+    if (!vec) { cb *= p.beta[0]; if (HP) ca *= p.alpha[0]; }
     uint16_t* yrow = live ? p.Y + (long long)token * p.N : nullptr;
-    for (int c = 0; c < 4; ++c) {           // 64 output columns = 128 bytes of the row per pass
-      const int n0 = t.n * 256 + c * 64;
+    for (int c = half; c * 64 < t.bn; c += 2) {     // 64 output columns = 128 bytes of the row per pass
+      const int n0 = t.c.n0 + c * 64;
       if (n0 >= p.N) break;
       uint4 o[8];
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
-        uint32_t a[32], z[32];
-        tmem_ld32(taddr + c * 64 + h * 32, a);
-        if (HP) tmem_ld32(taddr + kAccCols + c * 64 + h * 32, z);
-        tmem_ld_wait();
         const int nb = n0 + h * 32;
-        if (nb < p.N) {
-          uint32_t w[16];
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            float y[2];
-#pragma unroll
-            for (int u = 0; u < 2; ++u) {
-              const int n = nb + 2 * j + u;
-              float v = __ldg(p.beta + n * p.sstride) * s1 * (float)(int)a[2 * j + u];
-              if (HP) v += __ldg(p.alpha + n * p.sstride) * g * __uint_as_float(z[2 * j + u]);
-              y[u] = v;
-            }
-            w[j] = pack_bf16x2(y[0], y[1]);
-          }
-#pragma unroll
-          for (int j = 0; j < 4; ++j) o[4 * h + j] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+        if (c * 64 + h * 32 < t.bn && nb < p.N) {
+          uint32_t a[32], z[32];
+          tmem_ld32(tacc + c * 64 + h * 32, a);
+          if (HP) tmem_ld32(tz + c * 64 + h * 32, z);
+          tmem_ld_wait();
+          if (vec) combine32<true>(p, nb, cb, ca, a, z, o + 4 * h);
+          else combine32<false>(p, nb, cb, ca, a, z, o + 4 * h);
         }
       }
-      warp_store_rows(stage, o, yrow ? yrow + n0 : nullptr, min(64, p.N - n0) * 2, lane);
+      warp_store_rows(stage, o, yrow ? yrow + n0 : nullptr, min(64, min(t.bn - c * 64, p.N - n0)) * 2, lane);
     }
   }
 };
 PQ_DEFINE_GEMM_KERNEL(k_gemm_fwd_hp, FwdProblem<true>)
 PQ_DEFINE_GEMM_KERNEL(k_gemm_fwd_1bit, FwdProblem<false>)
 
-int gemm_forward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, const uint16_t* xs, uint16_t* Y, cudaStream_t st) {
+template <bool HP>
+static int fill_forward_params(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, uint16_t* Y, typename FwdProblem<HP>::Params& f) {
+  using P = FwdProblem<HP>;
   const int mtiles = (a.T + 127) / 128;
-  const bool hp = a.r > 0;
-  if (hp) {
+  if (!map2d(&f.tq, true, sv.q, a.K, a.T, 128, 128)) return PQ_ERR_CUDA;
+  if (!map2d(&f.ts, true, w_s8, a.K, a.N, 128, 256)) return PQ_ERR_CUDA;
+  f.th = f.tq; f.tb = f.tq;
+  if (HP) {
+    if (!map2d(&f.th, false, sv.h, a.r, (uint64_t)sv.max_items * 256, 64, 128)) return PQ_ERR_CUDA;
+    if (!map3d(&f.tb, a.B, a.r, a.N, a.E, 64, 256)) return PQ_ERR_CUDA;
+  }
+  f.rt = sv.rt; f.perm = (HP && a.E > 1) ? sv.perm : nullptr; f.gamma = sv.gamma; f.gate = sv.gate; f.w_scales = a.w_scales;
+  f.alpha = a.alpha; f.beta = a.beta; f.Y = Y; f.T = a.T; f.N = a.N; f.K = a.K; f.r = a.r; f.sstride = a.scale_stride;
+  f.item_rows = sv.max_items * 128;
+  f.g = make_tile_grid(mtiles, (a.N + 255) / 256, 256);
+  return PQ_OK;
+}
+
+int gemm_forward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, const uint16_t* xs, uint16_t* Y, cudaStream_t st) {
+  if (a.r > 0) {
     HpUpProblem::Params p;
     p.rt = sv.rt; p.H = sv.h; p.K = a.K; p.r = a.r; p.bn = h_round_up(a.r, 16); p.item_rows = sv.max_items * 128;
     if (!map2d(&p.tx, false, xs, a.K, a.T, 64, 128)) return PQ_ERR_CUDA;
@@ -311,23 +383,14 @@ int gemm_forward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, co
     int rc = launch_gemm(KID_HP_UP, k_gemm_hp_up, p, sv.max_items, st);
     if (rc) return rc;
     FwdProblem<true>::Params f;
-    if (!map2d(&f.tq, true, sv.q, a.K, a.T, 128, 128)) return PQ_ERR_CUDA;
-    if (!map2d(&f.ts, true, w_s8, a.K, a.N, 128, 256)) return PQ_ERR_CUDA;
-    if (!map2d(&f.th, false, sv.h, a.r, (uint64_t)sv.max_items * 256, 64, 128)) return PQ_ERR_CUDA;
-    if (!map3d(&f.tb, a.B, a.r, a.N, a.E, 64, 256)) return PQ_ERR_CUDA;
-    f.rt = sv.rt; f.perm = a.E > 1 ? sv.perm : nullptr; f.gamma = sv.gamma; f.gate = sv.gate; f.w_scales = a.w_scales;
-    f.alpha = a.alpha; f.beta = a.beta; f.Y = Y; f.T = a.T; f.N = a.N; f.K = a.K; f.r = a.r; f.sstride = a.scale_stride;
-    f.ntn = (a.N + 255) / 256; f.item_rows = sv.max_items * 128;
-    return launch_gemm(KID_FWD, k_gemm_fwd_hp, f, mtiles * f.ntn, st);
+    rc = fill_forward_params<true>(a, w_s8, sv, Y, f);
+    if (rc) return rc;
+    return launch_gemm(KID_FWD, k_gemm_fwd_hp, f, f.g.total, st);
   }
   FwdProblem<false>::Params f;
-  if (!map2d(&f.tq, true, sv.q, a.K, a.T, 128, 128)) return PQ_ERR_CUDA;
-  if (!map2d(&f.ts, true, w_s8, a.K, a.N, 128, 256)) return PQ_ERR_CUDA;
-  f.th = f.tq; f.tb = f.tq;
-  f.rt = sv.rt; f.perm = nullptr; f.gamma = sv.gamma; f.gate = sv.gate; f.w_scales = a.w_scales;
-  f.alpha = a.alpha; f.beta = a.beta; f.Y = Y; f.T = a.T; f.N = a.N; f.K = a.K; f.r = 0; f.sstride = a.scale_stride;
-  f.ntn = (a.N + 255) / 256; f.item_rows = 0;
-  return launch_gemm(KID_FWD, k_gemm_fwd_1bit, f, mtiles * f.ntn, st);
+  int rc = fill_forward_params<false>(a, w_s8, sv, Y, f);
+  if (rc) return rc;
+  return launch_gemm(KID_FWD, k_gemm_fwd_1bit, f, f.g.total, st);
 }
 
 
@@ -350,7 +413,7 @@ __device__ __forceinline__ float dx_scale(const float* w_scales, const float* be
 //   gh = g H (bf16, masked),  dl[t,j] = dg g (delta_je - p_tj),  dlc = dl / c
 // ---------------------------------------------------------------------------
 struct HpDhProblem {
-  static constexpr int kAccPerTile = 1;
+  using Acc = AccDouble;
   struct Params {
     CUtensorMap tdy, tba;  // dYs [T,N]; (alpha) B [E,N,r]
     RoutingTables rt;
@@ -364,19 +427,21 @@ struct HpDhProblem {
     uint16_t* gh;
     float* dl;
     uint16_t* dlc;
-    int T, N, r, E, bn, sstride, item_rows;
+    int T, N, r, E, bn, sstride, item_rows, ba_blk;
   };
   struct Tile { int item; int4 it; };
   __device__ static int num_tiles(const Params& p) { return p.rt.n_items[0]; }
   __device__ static void tile_init(const Params& p, int i, Tile& t) { t.item = i; t.it = p.rt.items[i]; }
   __device__ static int num_segments(const Params&, const Tile&) { return 1; }
   __device__ static void segment(const Params& p, const Tile& t, int, Segment& s) {
+    s.a_blk = 0; s.b_blk = p.ba_blk;
     s.mode = MODE_BF_KM; s.acc = 0; s.bn = p.bn; s.ksteps = 4; s.nkb = (p.N + 63) / 64;
     s.ta = &p.tdy; s.a_rank = 2; s.a_x = 0; s.a_y = t.it.x * 128; s.a_z = 0;
     s.tb = &p.tba; s.b_rank = 3; s.b_x = 0; s.b_y = 0; s.b_z = t.it.y;
-    s.b_bytes = (p.bn / 64) * kMnBoxBytes;
+    s.b_box = 0;
   }
-  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane, uint8_t* stage) {
+  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, uint32_t, int quad, int half, int lane, uint8_t* stage) {
+    if (half) return;   // each row's sum over all r columns stays in one thread
     const int row = quad * 32 + lane;
     const bool live = row >= t.it.z && row < t.it.w;
     const int pos = t.it.x * 128 + row;
@@ -450,7 +515,7 @@ PQ_DEFINE_GEMM_KERNEL(k_gemm_hp_dh, HpDhProblem)
 // scattered back to token order.
 // ---------------------------------------------------------------------------
 struct BwdDxProblem {
-  static constexpr int kAccPerTile = 1;
+  using Acc = AccDouble;
   struct Params {
     CUtensorMap tdy, tsb, tdh, ta3, tdl, twr;
     RoutingTables rt;
@@ -458,24 +523,27 @@ struct BwdDxProblem {
     const float* w_scales;
     const float* beta;
     uint16_t* dX;
-    int T, N, K, r, E, sstride, ntk, item_rows;
+    TileGrid g;
+    int T, N, K, r, E, sstride, item_rows, sb_blk, a3_blk, wr_blk;
   };
-  struct Tile { int m, kt, ib, ie, skip1; };
-  __device__ static int num_tiles(const Params& p) { return ((p.T + 127) / 128) * p.ntk; }
+  struct Tile { TileCoord c; int m, bn, ib, ie, skip1; };
+  __device__ static int num_tiles(const Params& p) { return p.g.total; }
   __device__ static void tile_init(const Params& p, int i, Tile& t) {
-    t.m = i / p.ntk; t.kt = i % p.ntk;
+    t.c = tile_coord(p.g, i);
+    t.m = t.c.m;
+    t.bn = clip_bn(t.c.bn, t.c.n0, p.K, 64);
     if (p.r > 0) { t.ib = p.rt.tile_item_begin[t.m]; t.ie = p.rt.tile_item_begin[t.m + 1]; } else { t.ib = t.ie = 0; }
     t.skip1 = dx_scale(p.w_scales, p.beta, p.sstride) == 0.f;
   }
   __device__ static int num_segments(const Params& p, const Tile& t) { return (t.skip1 ? 0 : 1) + 2 * (t.ie - t.ib) + (p.E > 1 ? 1 : 0); }
   __device__ static void segment(const Params& p, const Tile& t, int i, Segment& s) {
-    s.mode = MODE_BF_KM; s.acc = 0; s.bn = 256; s.ksteps = 4; s.a_rank = 2; s.a_x = 0; s.a_z = 0;
-    s.b_x = t.kt * 256; s.b_y = 0; s.b_z = 0; s.b_bytes = kStageBBytes;
+    s.mode = MODE_BF_KM; s.acc = 0; s.bn = t.bn; s.ksteps = 4; s.a_rank = 2; s.a_x = 0; s.a_z = 0;
+    s.b_x = t.c.n0; s.b_y = 0; s.b_z = 0; s.b_box = 0; s.a_blk = 0;
     if (!t.skip1) {
       if (i == 0) {
         s.nkb = (p.N + 63) / 64;
         s.ta = &p.tdy; s.a_y = t.m * 128;
-        s.tb = &p.tsb; s.b_rank = 2;
+        s.tb = &p.tsb; s.b_rank = 2; s.b_blk = p.sb_blk;
         return;
       }
       --i;
@@ -484,14 +552,14 @@ struct BwdDxProblem {
       const int item = t.ib + (i >> 1), plane = i & 1;
       s.nkb = (p.r + 63) / 64;
       s.ta = &p.tdh; s.a_y = plane * p.item_rows + item * 128;
-      s.tb = &p.ta3; s.b_rank = 3; s.b_z = p.rt.items[item].y;
+      s.tb = &p.ta3; s.b_rank = 3; s.b_z = p.rt.items[item].y; s.b_blk = p.a3_blk;
       return;
     }
     s.nkb = 1; s.ksteps = 1;
     s.ta = &p.tdl; s.a_y = t.m * 128;
-    s.tb = &p.twr; s.b_rank = 2;
+    s.tb = &p.twr; s.b_rank = 2; s.b_blk = p.wr_blk;
   }
-  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane, uint8_t* stage) {
+  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, uint32_t, int quad, int half, int lane, uint8_t* stage) {
     const int pos = t.m * 128 + quad * 32 + lane;
     const bool live = pos < p.T;
     const int token = live ? (p.perm ? p.perm[pos] : pos) : 0;
@@ -499,8 +567,8 @@ struct BwdDxProblem {
     const float cc = c != 0.f ? c : 1.0f;
     const bool has = num_segments(p, t) > 0;
     uint16_t* xrow = live ? p.dX + (long long)token * p.K : nullptr;
-    for (int c64 = 0; c64 < 4; ++c64) {
-      const int k0 = t.kt * 256 + c64 * 64;
+    for (int c64 = half; c64 * 64 < t.bn; c64 += 2) {
+      const int k0 = t.c.n0 + c64 * 64;
       if (k0 >= p.K) break;
       uint4 o[8];
 #pragma unroll
@@ -526,34 +594,39 @@ PQ_DEFINE_GEMM_KERNEL(k_gemm_bwd_dx, BwdDxProblem)
 // of dbeta_n = lam * sum_k S[n,k] G[n,k].
 // ---------------------------------------------------------------------------
 struct BwdDwProblem {
-  static constexpr int kAccPerTile = 1;
+  using Acc = AccDouble;
   struct Params {
     CUtensorMap tdyT, txt;
     const int8_t* s8;
     const float* beta;
     float* dW;
     float* dbeta_partial;
-    int T, N, K, sstride, ntk;
+    TileGrid g;
+    int T, N, K, sstride, dy_blk, xt_blk;
   };
-  struct Tile { int nt, kt; };
-  __device__ static int num_tiles(const Params& p) { return ((p.N + 127) / 128) * p.ntk; }
-  __device__ static void tile_init(const Params& p, int i, Tile& t) { t.nt = i / p.ntk; t.kt = i % p.ntk; }
+  struct Tile { TileCoord c; int nt, bn; };
+  __device__ static int num_tiles(const Params& p) { return p.g.total; }
+  __device__ static void tile_init(const Params& p, int i, Tile& t) {
+    t.c = tile_coord(p.g, i);
+    t.nt = t.c.m;
+    t.bn = clip_bn(t.c.bn, t.c.n0, p.K, 64);
+  }
   __device__ static int num_segments(const Params&, const Tile&) { return 1; }
   __device__ static void segment(const Params& p, const Tile& t, int, Segment& s) {
-    s.mode = MODE_BF_MM; s.acc = 0; s.bn = 256; s.ksteps = 4; s.nkb = (p.T + 63) / 64;
+    s.mode = MODE_BF_MM; s.acc = 0; s.bn = t.bn; s.ksteps = 4; s.nkb = (p.T + 63) / 64;
     s.ta = &p.tdyT; s.a_rank = 2; s.a_x = t.nt * 128; s.a_y = 0; s.a_z = 0;
-    s.tb = &p.txt; s.b_rank = 2; s.b_x = t.kt * 256; s.b_y = 0; s.b_z = 0;
-    s.b_bytes = kStageBBytes;
+    s.tb = &p.txt; s.b_rank = 2; s.b_x = t.c.n0; s.b_y = 0; s.b_z = 0;
+    s.b_box = 0; s.a_blk = p.dy_blk; s.b_blk = p.xt_blk;
   }
-  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane, uint8_t* stage) {
+  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, uint32_t, int quad, int half, int lane, uint8_t* stage) {
     const int n = t.nt * 128 + quad * 32 + lane;
     const bool live = n < p.N;
     const float be = live ? p.beta[n * p.sstride] : 0.f;
     float* wrow = live ? p.dW + (long long)n * p.K : nullptr;
     const uint4* srow = reinterpret_cast<const uint4*>(p.s8 + (long long)(live ? n : 0) * p.K);
     float part = 0.f;
-    for (int c32 = 0; c32 < 8; ++c32) {
-      const int k0 = t.kt * 256 + c32 * 32;
+    for (int c32 = half; c32 * 32 < t.bn; c32 += 2) {
+      const int k0 = t.c.n0 + c32 * 32;
       if (k0 >= p.K) break;
       uint32_t v[32];
       tmem_ld32(taddr + c32 * 32, v);
@@ -577,7 +650,12 @@ struct BwdDwProblem {
       }
       warp_store_rows(stage, o, wrow ? wrow + k0 : nullptr, 128, lane);
     }
-    if (live) p.dbeta_partial[(long long)t.kt * p.N + n] = part;
+    if (live) {
+      // one slot per 32 columns of K; each of the two warps of a row fills its first slot and clears its others
+      const int slot = t.c.n0 / 32 + half;
+      p.dbeta_partial[(long long)slot * p.N + n] = part;
+      for (int j = 2; (half + j) * 32 < t.bn; j += 2) p.dbeta_partial[(long long)(slot + j) * p.N + n] = 0.f;
+    }
   }
 };
 PQ_DEFINE_GEMM_KERNEL(k_gemm_bwd_dw, BwdDwProblem)
@@ -589,12 +667,12 @@ PQ_DEFINE_GEMM_KERNEL(k_gemm_bwd_dw, BwdDwProblem)
 // expert's chunks in a fixed order, scales by alpha_n and forms the dalpha partials.
 // ---------------------------------------------------------------------------
 struct HpDbProblem {
-  static constexpr int kAccPerTile = 1;
+  using Acc = AccDouble;
   struct Params {
     CUtensorMap tdyT, tgh;
     RoutingTables rt;
     float* partial;  // [chunks, N, r]
-    int N, r, bn, ntn, item_rows;
+    int N, r, bn, ntn, item_rows, dy_blk, gh_blk;
   };
   struct Tile { int nt, chunk, ib, ie; };
   __device__ static int num_tiles(const Params& p) { return p.ntn * p.rt.n_chunks_b[0]; }
@@ -609,12 +687,12 @@ struct HpDbProblem {
     s.mode = MODE_BF_MM; s.acc = 0; s.bn = p.bn; s.ksteps = 4; s.nkb = 2;
     s.ta = &p.tdyT; s.a_rank = 2; s.a_x = t.nt * 128; s.a_y = p.rt.items[item].x * 128; s.a_z = 0;
     s.tb = &p.tgh; s.b_rank = 2; s.b_x = 0; s.b_y = plane * p.item_rows + item * 128; s.b_z = 0;
-    s.b_bytes = (p.bn / 64) * kMnBoxBytes;
+    s.b_box = 0; s.a_blk = p.dy_blk; s.b_blk = p.gh_blk;
   }
-  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane, uint8_t* stage) {
+  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, uint32_t, int quad, int half, int lane, uint8_t* stage) {
     const int n = t.nt * 128 + quad * 32 + lane;
     float* out = n < p.N ? p.partial + ((long long)t.chunk * p.N + n) * p.r : nullptr;
-    for (int c32 = 0; c32 * 32 < p.r; ++c32) {
+    for (int c32 = half; c32 * 32 < p.r; c32 += 2) {
       uint32_t v[32];
       tmem_ld32(taddr + c32 * 32, v);
       tmem_ld_wait();
@@ -632,12 +710,12 @@ PQ_DEFINE_GEMM_KERNEL(k_gemm_hp_db, HpDbProblem)
 // scaled by k_reduce_da.
 // ---------------------------------------------------------------------------
 struct HpDaProblem {
-  static constexpr int kAccPerTile = 1;
+  using Acc = AccDouble;
   struct Params {
     CUtensorMap tdhT, txs;
     RoutingTables rt;
     float* partial;  // [chunks, r, K]
-    int K, r, ntk, item_rows;
+    int K, r, ntk, item_rows, dh_blk, xs_blk;
   };
   struct Tile { int chunk, kt, ib, ie; };
   __device__ static int num_tiles(const Params& p) { return p.ntk * p.rt.n_chunks_a[0]; }
@@ -652,12 +730,12 @@ struct HpDaProblem {
     s.mode = MODE_BF_MM; s.acc = 0; s.bn = 256; s.ksteps = 4; s.nkb = 2;
     s.ta = &p.tdhT; s.a_rank = 2; s.a_x = 0; s.a_y = plane * p.item_rows + item * 128; s.a_z = 0;
     s.tb = &p.txs; s.b_rank = 2; s.b_x = t.kt * 256; s.b_y = p.rt.items[item].x * 128; s.b_z = 0;
-    s.b_bytes = kStageBBytes;
+    s.b_box = 0; s.a_blk = p.dh_blk; s.b_blk = p.xs_blk;
   }
-  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, int quad, int lane, uint8_t* stage) {
+  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, uint32_t, int quad, int half, int lane, uint8_t* stage) {
     const int j = quad * 32 + lane;
     float* out = j < p.r ? p.partial + ((long long)t.chunk * p.r + j) * p.K : nullptr;
-    for (int c32 = 0; c32 < 8; ++c32) {
+    for (int c32 = half; c32 < 8; c32 += 2) {
       const int k0 = t.kt * 256 + c32 * 32;
       if (k0 >= p.K) break;
       uint32_t v[32];
@@ -683,7 +761,7 @@ int gemm_backward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, c
   if (hp) {
     HpDhProblem::Params p;
     if (!map2d(&p.tdy, false, b.dys, a.N, a.T, 64, 128)) return PQ_ERR_CUDA;
-    if (!map3d(&p.tba, b.ba, a.r, a.N, a.E, 64, 64)) return PQ_ERR_CUDA;
+    if (!map_mn(&p.tba, &p.ba_blk, b.ba, a.r, a.N, 3, a.E, r64 / 64)) return PQ_ERR_CUDA;
     p.rt = sv.rt; p.H = sv.h; p.gate = sv.gate; p.probs = sv.probs; p.w_scales = a.w_scales; p.alpha = a.alpha; p.beta = a.beta;
     p.dhc = b.dhc; p.gh = b.gh; p.dl = b.dl; p.dlc = b.dlc;
     p.T = a.T; p.N = a.N; p.r = a.r; p.E = a.E; p.bn = r64; p.sstride = a.scale_stride; p.item_rows = (int)item_rows;
@@ -693,42 +771,44 @@ int gemm_backward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, c
   {
     BwdDxProblem::Params p;
     if (!map2d(&p.tdy, false, b.dys, a.N, a.T, 64, 128)) return PQ_ERR_CUDA;
-    if (!map2d(&p.tsb, false, b.sb, a.K, a.N, 64, 64)) return PQ_ERR_CUDA;
-    p.tdh = p.tdy; p.ta3 = p.tdy; p.tdl = p.tdy; p.twr = p.tdy;
+    if (!map_mn(&p.tsb, &p.sb_blk, b.sb, a.K, a.N, 2, 1, 4)) return PQ_ERR_CUDA;
+    p.tdh = p.tdy; p.ta3 = p.tdy; p.tdl = p.tdy; p.twr = p.tdy; p.a3_blk = 0; p.wr_blk = 0;
     if (hp) {
       if (!map2d(&p.tdh, false, b.dhc, a.r, 2 * item_rows, 64, 128)) return PQ_ERR_CUDA;
-      if (!map3d(&p.ta3, a.A, a.K, a.r, a.E, 64, 64)) return PQ_ERR_CUDA;
+      if (!map_mn(&p.ta3, &p.a3_blk, a.A, a.K, a.r, 3, a.E, 4)) return PQ_ERR_CUDA;
     }
     if (hp && a.E > 1) {
       if (!map2d(&p.tdl, false, b.dlc, 16, a.T, 64, 128)) return PQ_ERR_CUDA;
-      if (!map2d(&p.twr, false, a.Wr, a.K, a.E, 64, 64)) return PQ_ERR_CUDA;
+      if (!map_mn(&p.twr, &p.wr_blk, a.Wr, a.K, a.E, 2, 1, 4)) return PQ_ERR_CUDA;
     }
     p.rt = sv.rt; p.perm = (hp && a.E > 1) ? sv.perm : nullptr; p.w_scales = a.w_scales; p.beta = a.beta; p.dX = dX;
-    p.T = a.T; p.N = a.N; p.K = a.K; p.r = a.r; p.E = hp ? a.E : 1; p.sstride = a.scale_stride; p.ntk = ntk; p.item_rows = (int)item_rows;
-    rc = launch_gemm(KID_BWD_DX, k_gemm_bwd_dx, p, mtiles * ntk, st);
+    p.T = a.T; p.N = a.N; p.K = a.K; p.r = a.r; p.E = hp ? a.E : 1; p.sstride = a.scale_stride; p.item_rows = (int)item_rows;
+    p.g = make_tile_grid(mtiles, ntk, 256);
+    rc = launch_gemm(KID_BWD_DX, k_gemm_bwd_dx, p, p.g.total, st);
     if (rc) return rc;
   }
   {
     BwdDwProblem::Params p;
-    if (!map2d(&p.tdyT, false, b.dys, a.N, a.T, 64, 64)) return PQ_ERR_CUDA;
-    if (!map2d(&p.txt, false, sv.xt, a.K, a.T, 64, 64)) return PQ_ERR_CUDA;
+    if (!map_mn(&p.tdyT, &p.dy_blk, b.dys, a.N, a.T, 2, 1, 2)) return PQ_ERR_CUDA;
+    if (!map_mn(&p.txt, &p.xt_blk, sv.xt, a.K, a.T, 2, 1, 4)) return PQ_ERR_CUDA;
     p.s8 = w_s8; p.beta = a.beta; p.dW = dW; p.dbeta_partial = b.dbeta_partial;
-    p.T = a.T; p.N = a.N; p.K = a.K; p.sstride = a.scale_stride; p.ntk = ntk;
-    rc = launch_gemm(KID_BWD_DW, k_gemm_bwd_dw, p, ntn128 * ntk, st);
+    p.T = a.T; p.N = a.N; p.K = a.K; p.sstride = a.scale_stride;
+    p.g = make_tile_grid(ntn128, ntk, 256);
+    rc = launch_gemm(KID_BWD_DW, k_gemm_bwd_dw, p, p.g.total, st);
     if (rc) return rc;
   }
   if (hp) {
     HpDbProblem::Params p;
-    if (!map2d(&p.tdyT, false, b.dys, a.N, a.T, 64, 64)) return PQ_ERR_CUDA;
-    if (!map2d(&p.tgh, false, b.gh, a.r, 2 * item_rows, 64, 64)) return PQ_ERR_CUDA;
+    if (!map_mn(&p.tdyT, &p.dy_blk, b.dys, a.N, a.T, 2, 1, 2)) return PQ_ERR_CUDA;
+    if (!map_mn(&p.tgh, &p.gh_blk, b.gh, a.r, 2 * item_rows, 2, 1, r64 / 64)) return PQ_ERR_CUDA;
     p.rt = sv.rt; p.partial = b.db_partial; p.N = a.N; p.r = a.r; p.bn = r64; p.ntn = ntn128; p.item_rows = (int)item_rows;
     rc = launch_gemm(KID_HP_DB, k_gemm_hp_db, p, ntn128 * sv.max_chunks_b, st);
     if (rc) return rc;
     if (launch_reduce_db(b.db_partial, sv.rt, a.B, a.alpha, a.scale_stride, a.E, a.N, a.r, dB, b.dalpha_partial, st) != cudaSuccess)
       return PQ_ERR_CUDA;
     HpDaProblem::Params q;
-    if (!map2d(&q.tdhT, false, b.dhc, a.r, 2 * item_rows, 64, 64)) return PQ_ERR_CUDA;
-    if (!map2d(&q.txs, false, b.xs, a.K, a.T, 64, 64)) return PQ_ERR_CUDA;
+    if (!map_mn(&q.tdhT, &q.dh_blk, b.dhc, a.r, 2 * item_rows, 2, 1, 2)) return PQ_ERR_CUDA;
+    if (!map_mn(&q.txs, &q.xs_blk, b.xs, a.K, a.T, 2, 1, 4)) return PQ_ERR_CUDA;
     q.rt = sv.rt; q.partial = b.da_partial; q.K = a.K; q.r = a.r; q.ntk = ntk; q.item_rows = (int)item_rows;
     rc = launch_gemm(KID_HP_DA, k_gemm_hp_da, q, ntk * sv.max_chunks_a, st);
     if (rc) return rc;

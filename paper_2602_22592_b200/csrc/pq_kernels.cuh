@@ -102,7 +102,7 @@ struct LayerArgs {
   const uint16_t* Wr;  // [E,K]
 };
 
-int gemm_debug(int mode, int M, int N, int K, const void* A, const void* B, void* D, cudaStream_t st);
+int gemm_debug(int mode, int M, int N, int K, const void* A, const void* B, void* D, int tile_n, cudaStream_t st);
 int gemm_forward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, const uint16_t* xs, uint16_t* Y, cudaStream_t st);
 
 struct BwdBuffers {
@@ -114,7 +114,7 @@ struct BwdBuffers {
   uint16_t* gh;          // [2][items*128, r] bf16 hi/lo planes of g * H
   float* dl;             // [T,E] fp32 router logit gradient (sorted order)
   uint16_t* dlc;         // [T,16] bf16 dl / c
-  float* dbeta_partial;  // [ceil(K/256), N]
+  float* dbeta_partial;  // [ceil(K/32), N]
   float* dalpha_partial; // [E, N]
   float* da_partial;     // [max_chunks_a, r, K] raw split-contraction partials of dA
   float* db_partial;     // [max_chunks_b, N, r]

@@ -74,6 +74,38 @@ def test_engine_int8_accumulators_bit_exact(M, N, K):
     assert np.array_equal(D.cpu().numpy().astype(np.int64), O.onebit_gemm(A, B))
 
 
+@pytest.mark.parametrize("tile_n", [32, 64, 128, 160, 256])
+@pytest.mark.parametrize("M,N,K", [(392, 520, 1040), (2048, 4096, 256), (128, 2400, 128)])
+def test_engine_int8_tile_widths_bit_exact(tile_n, M, N, K):
+    # narrow tiles, the 160-wide forward tile, and shapes whose last wave is cut into pieces
+    rng = np.random.default_rng(tile_n + M + N + K)
+    A = rng.integers(-128, 128, (M, K)).astype(np.int8)
+    B = rng.choice([-1, 1], (N, K)).astype(np.int8)
+    D = torch.full((M, N), 0x7FFFFFFF, dtype=torch.int32, device="cuda")
+    pqb.pq_debug_gemm_tile(0, M, N, K, torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda(), D, tile_n)
+    torch.cuda.synchronize()
+    check_status()
+    assert np.array_equal(D.cpu().numpy().astype(np.int64), O.onebit_gemm(A, B))
+
+
+@pytest.mark.parametrize("mode,tile_n", [(1, 96), (2, 64), (2, 128), (3, 64), (3, 192)])
+def test_engine_bf16_tile_widths(mode, tile_n):
+    M, N, K = 392, 1096, 520
+    rng = np.random.default_rng(mode * 1000 + tile_n)
+    A = I.bf16_values(rng.standard_normal((M, K)).astype(np.float32))
+    B = I.bf16_values(rng.standard_normal((N, K)).astype(np.float32))
+    ref = A.astype(np.float64) @ B.astype(np.float64).T
+    At = torch.from_numpy(A if mode != 3 else np.ascontiguousarray(A.T)).cuda().to(torch.bfloat16)
+    Bt = torch.from_numpy(B if mode == 1 else np.ascontiguousarray(B.T)).cuda().to(torch.bfloat16)
+    D = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+    pqb.pq_debug_gemm_tile(mode, M, N, K, At, Bt, D, tile_n)
+    torch.cuda.synchronize()
+    check_status()
+    got = D.cpu().numpy()
+    assert np.all(np.isfinite(got))
+    assert np.max(np.abs(got - ref)) <= 1e-4 * np.sqrt(K) * 4
+
+
 @pytest.mark.parametrize("mode", [1, 2, 3])
 @pytest.mark.parametrize("M,N,K", [(128, 256, 64), (256, 512, 512), (392, 520, 1000), (8, 16, 16)])
 def test_engine_bf16_operand_forms(mode, M, N, K):
@@ -143,6 +175,11 @@ CASES = {
     "dense_hp_ragged": dict(T=333, K=384, N=544, r=64, E=1),
     "routed8": dict(T=1000, K=512, N=768, r=128, E=8),
     "routed4_small_r": dict(T=520, K=256, N=256, r=16, E=4, scale_vector=True, alpha=1.5, beta=0.4),
+    # long rows: the activation quantiser keeps a row in registers of 1, 2 or 4 warps, or re-reads it
+    "k2048": dict(T=70, K=2048, N=64, r=0, E=0),
+    "k4096_routed": dict(T=200, K=4096, N=64, r=16, E=4),
+    "k5632": dict(T=130, K=5632, N=96, r=0, E=0),
+    "k8704": dict(T=40, K=8704, N=64, r=0, E=0),
 }
 
 
