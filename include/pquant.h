@@ -51,7 +51,10 @@ enum {
   PQ_ERR_TOO_LARGE = -8    /* problem needs more scratch than a fixed-size buffer holds */
 };
 
-enum { PQ_SCALE_VECTOR = 1u }; /* pq_desc.flags: alpha, beta have N entries instead of 1 */
+enum {
+  PQ_SCALE_VECTOR = 1u,    /* pq_desc.flags: alpha, beta have N entries instead of 1                      */
+  PQ_DECODE_DUMP_ACC = 2u  /* decode only, test hook: also write the exact int32 sums of the 1-bit product */
+};
 
 enum { PQ_PHASE_PACK = 0, PQ_PHASE_FWD = 1, PQ_PHASE_BWD = 2, PQ_PHASE_DECODE = 3 };
 
@@ -144,13 +147,32 @@ int pq_pack_weights_static(const pq_desc* d, const float* W, uint32_t* w_bits, i
 /* Forward of the layer (Eq. 10-11, Sec. 3.3).
  *   training (w_s8 != NULL): tensor-core path; fills `saved` (may be NULL when
  *     no backward follows).  A, B may be NULL iff r == 0; Wr NULL iff E <= 1.
- *   decode (w_s8 == NULL): small-T path straight from the packed bits
- *     (T <= 16), nothing is saved. */
+ *   decode (w_s8 == NULL): T <= 16 tokens straight from the packed bits w_bits
+ *     (App. A): two kernels bound by the bytes of the weights.  `saved` is ignored,
+ *     ws needs pq_workspace_bytes(d, PQ_PHASE_DECODE) bytes.  r <= 256; K and N such
+ *     that one SM's share of the bits and expert rows fits its shared memory
+ *     (PQ_ERR_UNSUPPORTED otherwise; the 3B-shaped 3200 x 8640 layers fit).  The two
+ *     kernels are launched with programmatic stream serialisation, so consecutive
+ *     decode calls on one stream overlap their prologues. */
 int pq_linear_forward(const pq_desc* d, const uint16_t* X, const uint32_t* w_bits,
                       const int8_t* w_s8, const float* w_scales, const uint16_t* A,
                       const uint16_t* B, const uint16_t* Wr, const float* alpha,
                       const float* beta, uint16_t* Y, void* saved, size_t saved_bytes, void* ws,
                       size_t ws_bytes, void* stream);
+
+/* What the decode path leaves in its workspace, for tests and diagnostics.  One entry per
+ * token: the routed expert, its gate g_t, gamma_t (Eq. 9) and the sum over k of the int8 codes. */
+typedef struct pq_decode_token {
+  int32_t expert;
+  float gate;
+  float gamma;
+  int32_t code_sum;
+} pq_decode_token;
+typedef struct pq_decode_view {
+  pq_decode_token* tokens; /* [T] (device)                                                        */
+  int32_t* acc;            /* [T,N] sum_k S[n,k] q[t,k] when PQ_DECODE_DUMP_ACC is set, else NULL */
+} pq_decode_view;
+int pq_decode_view_init(const pq_desc* d, void* ws, pq_decode_view* out);
 
 /* Straight-through backward (App. B.1): Sign, Round and Clip pass the gradient
  * unchanged; mu, lam, gamma are constants.  Every gradient is OVERWRITTEN.
@@ -194,8 +216,8 @@ long long pq_kernel_launches(void);
  * Ids: 0 weight sums, 1 binarize+pack, 2 router, 3 expert scan, 4 activation
  * quantise, 5 HP up-projection, 6 fused forward tile, 7 row scatter, 8 scaled
  * sign, 9 scaled B, 10 HP dH, 11 dX, 12 dW, 13 HP dB, 14 HP dA, 15 router
- * weight gradient, 16 partial sums, 17 scalar sum, 18 debug GEMM, 21 dB chunk
- * reduction, 22 dA chunk reduction. */
+ * weight gradient, 16 partial sums, 17 scalar sum, 18 debug GEMM, 19 decode
+ * token preparation, 20 decode main, 21 dB chunk reduction, 22 dA chunk reduction. */
 int pq_profile_events(int kernel_id, void* start_event, void* stop_event);
 
 const char* pq_status_string(int status);

@@ -18,10 +18,11 @@ PQ_OK = 0
 PQ_ERR_NULL, PQ_ERR_SHAPE, PQ_ERR_ALIGN, PQ_ERR_WORKSPACE = -1, -2, -3, -4
 PQ_ERR_UNSUPPORTED, PQ_ERR_CUDA, PQ_ERR_TIMEOUT, PQ_ERR_TOO_LARGE = -5, -6, -7, -8
 PQ_SCALE_VECTOR = 1
+PQ_DECODE_DUMP_ACC = 2
 PQ_PHASE_PACK, PQ_PHASE_FWD, PQ_PHASE_BWD, PQ_PHASE_DECODE = 0, 1, 2, 3
 
 EXPORTS = ("pq_status_string", "pq_workspace_bytes", "pq_saved_bytes", "pq_saved_view_init",
-           "pq_pack_weights", "pq_pack_weights_static", "pq_linear_forward", "pq_linear_backward", "pq_debug_gemm", "pq_debug_gemm_tile",
+           "pq_decode_view_init", "pq_pack_weights", "pq_pack_weights_static", "pq_linear_forward", "pq_linear_backward", "pq_debug_gemm", "pq_debug_gemm_tile",
            "pq_device_status", "pq_kernel_launches", "pq_profile_events")
 
 KERNEL_IDS = dict(pack_sums=0, binarize_pack=1, router=2, route_scan=3, act_quant=4, hp_up=5, fwd=6, scatter_rows=7,
@@ -47,6 +48,10 @@ class pq_saved_view(ctypes.Structure):
                  "n_items", "items", "tile_item_begin", "expert_item_begin")] + [("max_items", ctypes.c_int32)]
 
 
+class pq_decode_view(ctypes.Structure):
+    _fields_ = [("tokens", ctypes.c_void_p), ("acc", ctypes.c_void_p)]
+
+
 _lib = None
 
 
@@ -67,6 +72,8 @@ def lib() -> ctypes.CDLL:
         L.pq_saved_bytes.argtypes = [dp]
         L.pq_saved_view_init.restype = ci
         L.pq_saved_view_init.argtypes = [dp, vp, ctypes.POINTER(pq_saved_view)]
+        L.pq_decode_view_init.restype = ci
+        L.pq_decode_view_init.argtypes = [dp, vp, ctypes.POINTER(pq_decode_view)]
         L.pq_pack_weights.restype = ci
         L.pq_pack_weights.argtypes = [dp, vp, vp, vp, vp, vp, sz, vp]
         L.pq_pack_weights_static.restype = ci
@@ -107,8 +114,9 @@ def _check(fn, status):
         raise PqError(fn, status)
 
 
-def make_desc(T, K, N, r=0, E=0, top_k=1, scale_vector=False) -> pq_desc:
-    return pq_desc(ctypes.sizeof(pq_desc), PQ_SCALE_VECTOR if scale_vector else 0, T, K, N, r, E, top_k)
+def make_desc(T, K, N, r=0, E=0, top_k=1, scale_vector=False, dump_acc=False) -> pq_desc:
+    flags = (PQ_SCALE_VECTOR if scale_vector else 0) | (PQ_DECODE_DUMP_ACC if dump_acc else 0)
+    return pq_desc(ctypes.sizeof(pq_desc), flags, T, K, N, r, E, top_k)
 
 
 def pq_status_string(status: int) -> str:
@@ -150,6 +158,19 @@ def pq_saved_view_init(d: pq_desc, saved: torch.Tensor) -> dict:
         n_items=view(v.n_items, torch.int32, 1), items=view(v.items, torch.int32, v.max_items, 4),
         tile_item_begin=view(v.tile_item_begin, torch.int32, mt + 1),
         expert_item_begin=view(v.expert_item_begin, torch.int32, E + 1), max_items=v.max_items)
+
+
+def pq_decode_view_init(d: pq_desc, ws: torch.Tensor) -> dict:
+    """Views into the decode workspace: per-token expert / gate / gamma / code sum, and the int32 sums if dumped."""
+    v = pq_decode_view()
+    _check("pq_decode_view_init", lib().pq_decode_view_init(ctypes.byref(d), _ptr(ws), ctypes.byref(v)))
+    base = ws.data_ptr()
+    raw = ws[v.tokens - base: v.tokens - base + 16 * d.T]
+    out = dict(expert=raw.view(torch.int32).view(d.T, 4)[:, 0], gate=raw.view(torch.float32).view(d.T, 4)[:, 1],
+               gamma=raw.view(torch.float32).view(d.T, 4)[:, 2], code_sum=raw.view(torch.int32).view(d.T, 4)[:, 3], acc=None)
+    if v.acc:
+        out["acc"] = ws[v.acc - base: v.acc - base + 4 * d.T * d.N].view(torch.int32).view(d.T, d.N)
+    return out
 
 
 def pq_pack_weights(d, W, w_bits, w_s8, w_scales, ws, stream=None):

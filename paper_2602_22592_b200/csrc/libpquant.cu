@@ -2,4 +2,5 @@
 // word and are compiled together (no relocatable device code needed).
 #include "pq_elementwise.cu"
 #include "pq_gemm_kernels.cu"
+#include "pq_decode.cu"
 #include "pq_api.cu"

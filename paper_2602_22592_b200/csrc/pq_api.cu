@@ -245,7 +245,9 @@ size_t pq_workspace_bytes(const pq_desc* d, int phase) {
     case PQ_PHASE_BWD:
       if (check_desc(d, true) != PQ_OK) return 0;
       return carve_bwd_scratch(d, nullptr, nullptr);
-    case PQ_PHASE_DECODE: return 0;
+    case PQ_PHASE_DECODE:
+      if (check_desc(d, false) != PQ_OK || d->T > 16) return 0;
+      return decode_workspace_bytes(d->T, d->K, d->N, d->r, (d->flags & PQ_DECODE_DUMP_ACC) != 0);
     default: return 0;
   }
 }
@@ -261,6 +263,17 @@ int pq_saved_view_init(const pq_desc* d, void* saved, pq_saved_view* out) {
   out->n_items = s.rt.n_items; out->items = reinterpret_cast<int32_t*>(s.rt.items);
   out->tile_item_begin = s.rt.tile_item_begin; out->expert_item_begin = s.rt.expert_item_begin;
   out->max_items = s.max_items;
+  return PQ_OK;
+}
+
+int pq_decode_view_init(const pq_desc* d, void* ws, pq_decode_view* out) {
+  if (!d || !ws || !out) return PQ_ERR_NULL;
+  int rc = check_desc(d, false);
+  if (rc) return rc;
+  if (d->T > 16) return PQ_ERR_SHAPE;
+  const DecodeViewPtrs v = decode_view(d->T, d->K, d->N, d->r, ws, (d->flags & PQ_DECODE_DUMP_ACC) != 0);
+  out->tokens = static_cast<pq_decode_token*>(v.tokens);
+  out->acc = v.acc;
   return PQ_OK;
 }
 
@@ -285,7 +298,20 @@ int pq_linear_forward(const pq_desc* d, const uint16_t* X, const uint32_t* w_bit
                       const uint16_t* A, const uint16_t* B, const uint16_t* Wr, const float* alpha, const float* beta, uint16_t* Y,
                       void* saved, size_t saved_bytes, void* ws, size_t ws_bytes, void* stream) {
   if (!d || !X || !w_scales || !beta || !Y) return PQ_ERR_NULL;
-  if (!w_s8) return PQ_ERR_UNSUPPORTED;  // decode path: see pq_decode_forward
+  if (!w_s8) {
+    // decode: a few tokens straight from the packed sign bits
+    if (!w_bits || !ws) return PQ_ERR_NULL;
+    int rc = check_desc(d, false);
+    if (rc) return rc;
+    if (d->T > 16) return PQ_ERR_SHAPE;
+    if (d->r > 0 && (!A || !B || !alpha)) return PQ_ERR_NULL;
+    if (routed(d) && !Wr) return PQ_ERR_NULL;
+    if (misaligned(X) || misaligned(w_bits) || misaligned(A) || misaligned(B) || misaligned(Wr) || misaligned(ws)) return PQ_ERR_ALIGN;
+    const bool dump = (d->flags & PQ_DECODE_DUMP_ACC) != 0;
+    if (ws_bytes < decode_workspace_bytes(d->T, d->K, d->N, d->r, dump)) return PQ_ERR_WORKSPACE;
+    LayerArgs a{d->T, d->K, d->N, d->r, experts_of(d), (d->flags & PQ_SCALE_VECTOR) ? 1 : 0, w_scales, alpha, beta, A, B, Wr};
+    return decode_forward(a, X, w_bits, Y, ws, dump, static_cast<cudaStream_t>(stream));
+  }
   int rc = check_desc(d, true);
   if (rc) return rc;
   (void)w_bits;

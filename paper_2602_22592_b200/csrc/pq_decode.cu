@@ -1,0 +1,499 @@
+// Decode path of the pQuant layer (App. A): M <= 16 tokens against weights stored as
+// packed sign bits.  The work is bound by the bytes of the weights (N K / 8 bytes of bits,
+// 2 r (K + N) bytes per expert in use), so the kernels are built around streaming them once:
+//
+//   k_decode_prep  one CTA per (token, slice of the r hidden rows): absmax quantisation of the
+//                  token (Eq. 7-9), router (Sec. 3.3), and its slice of h = A_e x.
+//   k_decode_main  one CTA per SM, each owning a contiguous range of output features: the sign
+//                  bits and the expert rows B_e of that range arrive by bulk copies into shared
+//                  memory; the 1-bit product runs on mma.sync (u8 bit masks x s8 activations,
+//                  exact in int32), the expert product on bf16 mma.sync, and the epilogue forms
+//                  Y = alpha g (B_e h) + beta (lam / gamma) (q . S)  (Eq. 10-11).
+//
+// The sum over k of q S is evaluated as 2 * (sum over the set bits of q) - (sum of q): the bit
+// words feed the tensor cores as 0/1 masks without expansion to +-1.
+#include "pq_kernels.cuh"
+
+namespace pq {
+
+constexpr int kDecodeMainThreads = 512;
+constexpr int kDecodeMaxTokens = 16;
+constexpr int kDecodeRing = 3;          // expert-row buffers in flight per CTA
+
+struct DecodeTokInfo {  // one per token, written by k_decode_prep
+  int expert;
+  float gate;
+  float gamma;
+  int rowsum;           // sum over k of q[k]
+};
+
+// programmatic dependent launch: let the next kernel in the stream start early / wait for the previous one
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void mma_u8s8(int (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// ---------------------------------------------------------------------------
+// Layout of the quantised activations handed from prep to main ("q fragments").
+// The contraction index k is walked in pairs of 32-bit weight words (64 values of k).  For pair
+// ip, the thread of a warp with quad index c (lane & 3) takes from a weight word w the bits
+// c + 8 j (mask 0x01010101 of w >> c) and c + 4 + 8 j (mask 0x10101010, i.e. the value 16), j = 0..3.
+// Its four 4-byte operand registers for the tokens' side therefore hold, for token g = lane >> 2,
+//   r0: q[64 ip      + c     + 8 j]   r1: q[64 ip + 32 + c     + 8 j]      (weight-1 masks)
+//   r2: q[64 ip      + c + 4 + 8 j]   r3: q[64 ip + 32 + c + 4 + 8 j]      (weight-16 masks)
+// stored as 16 bytes at ((group * npairs + ip) * 32 + lane) * 16, group = token / 8.
+// ---------------------------------------------------------------------------
+
+// grid (slices, M), 256 threads, dynamic shared memory: K bf16 values of the token
+__global__ void __launch_bounds__(256) k_decode_prep(const uint4* __restrict__ X, const uint4* __restrict__ Wr, const uint16_t* __restrict__ A,
+                                                     int M, int K, int E, int r, int rows_per_slice, DecodeTokInfo* __restrict__ info,
+                                                     uint4* __restrict__ qfrag, float* __restrict__ H) {
+  extern __shared__ uint4 xs4[];
+  __shared__ float red_f[8];
+  __shared__ int red_i[8];
+  __shared__ float logit_sh[kMaxExperts];
+  pdl_launch_dependents();
+  pdl_wait();   // X may come from the previous kernel; the buffers written here may still be read by it
+  const int m = blockIdx.y, slice = blockIdx.x;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int chunks = K >> 3;
+  const uint4* xrow = X + (long long)m * chunks;
+  float amax = 0.f;
+  for (int c = threadIdx.x; c < chunks; c += 256) {
+    const uint4 v = __ldg(xrow + c);
+    xs4[c] = v;
+    amax = fmaxf(amax, fmaxf(fmaxf(fabsf(bf16lo(v.x)), fabsf(bf16hi(v.x))), fmaxf(fabsf(bf16lo(v.y)), fabsf(bf16hi(v.y)))));
+    amax = fmaxf(amax, fmaxf(fmaxf(fabsf(bf16lo(v.z)), fabsf(bf16hi(v.z))), fmaxf(fabsf(bf16lo(v.w)), fabsf(bf16hi(v.w)))));
+  }
+  for (int d = 16; d > 0; d >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, d));
+  if (lane == 0) red_f[warp] = amax;
+  __syncthreads();   // also publishes xs4
+  amax = red_f[0];
+#pragma unroll
+  for (int w = 1; w < 8; ++w) amax = fmaxf(amax, red_f[w]);
+  const float gamma = __fdiv_rn(kActQmax, fmaxf(amax, kActAmaxFloor));
+
+  // router: the same pinned fp32 order as the training path (lane j owns the chunks c = j mod 32, ascending,
+  // fused multiply-add; butterfly 16, 8, 4, 2, 1), one warp per expert
+  int best = 0;
+  float gate = 1.0f;
+  if (E > 1) {
+    for (int e = warp; e < E; e += 8) {
+      float acc = 0.f;
+      for (int c = lane; c < chunks; c += 32) {
+        const uint4 xv = xs4[c];
+        const uint4 wv = __ldg(Wr + (long long)e * chunks + c);
+        acc = fmaf(bf16lo(xv.x), bf16lo(wv.x), acc); acc = fmaf(bf16hi(xv.x), bf16hi(wv.x), acc);
+        acc = fmaf(bf16lo(xv.y), bf16lo(wv.y), acc); acc = fmaf(bf16hi(xv.y), bf16hi(wv.y), acc);
+        acc = fmaf(bf16lo(xv.z), bf16lo(wv.z), acc); acc = fmaf(bf16hi(xv.z), bf16hi(wv.z), acc);
+        acc = fmaf(bf16lo(xv.w), bf16lo(wv.w), acc); acc = fmaf(bf16hi(xv.w), bf16hi(wv.w), acc);
+      }
+      for (int d = 16; d > 0; d >>= 1) acc = acc + __shfl_xor_sync(0xffffffffu, acc, d);
+      if (lane == 0) logit_sh[e] = acc;
+    }
+    __syncthreads();
+    float lmax = logit_sh[0];
+    for (int e = 1; e < E; ++e)
+      if (logit_sh[e] > lmax) { lmax = logit_sh[e]; best = e; }
+    float den = 0.f, pbest = 0.f;
+    for (int e = 0; e < E; ++e) {
+      const float pe = expf(logit_sh[e] - lmax);
+      den += pe;
+      if (e == best) pbest = pe;
+    }
+    gate = pbest * (1.0f / den);
+  }
+
+  if (slice == 0) {
+    // Eq. 7-9 for this token; every thread turns pairs of weight words (64 values of k) into fragment order
+    const int npairs = (K + 63) >> 6;
+    const int group = m >> 3, g = m & 7;
+    int rowsum = 0;
+    for (int ip = threadIdx.x; ip < npairs; ip += 256) {
+      int qv[64];
+#pragma unroll
+      for (int ch = 0; ch < 8; ++ch) {
+        const bool in = 8 * ip + ch < chunks;
+        const uint4 v = in ? xs4[8 * ip + ch] : make_uint4(0u, 0u, 0u, 0u);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int q0 = in ? max(-128, min(127, __float2int_rn(__fmul_rn(bf16lo(w[u]), gamma)))) : 0;
+          const int q1 = in ? max(-128, min(127, __float2int_rn(__fmul_rn(bf16hi(w[u]), gamma)))) : 0;
+          qv[8 * ch + 2 * u] = q0;
+          qv[8 * ch + 2 * u + 1] = q1;
+          rowsum += q0 + q1;
+        }
+      }
+      uint4 out[4];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t w[4];
+#pragma unroll
+        for (int reg = 0; reg < 4; ++reg) {
+          const int base = (reg & 1) * 32 + c + (reg >> 1) * 4;
+          w[reg] = (qv[base] & 0xFF) | ((qv[base + 8] & 0xFF) << 8) | ((qv[base + 16] & 0xFF) << 16) | ((qv[base + 24] & 0xFF) << 24);
+        }
+        out[c] = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+      uint4* dst = qfrag + ((long long)(group * npairs + ip) * 32 + g * 4);
+#pragma unroll
+      for (int c = 0; c < 4; ++c) dst[c] = out[c];
+    }
+    for (int d = 16; d > 0; d >>= 1) rowsum += __shfl_xor_sync(0xffffffffu, rowsum, d);
+    if (lane == 0) red_i[warp] = rowsum;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int tot = 0;
+      for (int w = 0; w < 8; ++w) tot += red_i[w];
+      info[m] = DecodeTokInfo{best, gate, gamma, tot};
+    }
+  }
+
+  // this slice of h = A_e x (fp32 accumulation over the bf16 operands), one warp per row
+  if (r > 0) {
+    const int j0 = slice * rows_per_slice, j1 = min(r, j0 + rows_per_slice);
+    for (int j = j0 + warp; j < j1; j += 8) {
+      const uint4* arow = reinterpret_cast<const uint4*>(A + ((long long)best * r + j) * K);
+      float a0 = 0.f, a1 = 0.f;
+      for (int c = lane; c < chunks; c += 32) {
+        const uint4 xv = xs4[c];
+        const uint4 wv = __ldg(arow + c);
+        a0 = fmaf(bf16lo(xv.x), bf16lo(wv.x), a0); a1 = fmaf(bf16hi(xv.x), bf16hi(wv.x), a1);
+        a0 = fmaf(bf16lo(xv.y), bf16lo(wv.y), a0); a1 = fmaf(bf16hi(xv.y), bf16hi(wv.y), a1);
+        a0 = fmaf(bf16lo(xv.z), bf16lo(wv.z), a0); a1 = fmaf(bf16hi(xv.z), bf16hi(wv.z), a1);
+        a0 = fmaf(bf16lo(xv.w), bf16lo(wv.w), a0); a1 = fmaf(bf16hi(xv.w), bf16hi(wv.w), a1);
+      }
+      float a = a0 + a1;
+      for (int d = 16; d > 0; d >>= 1) a += __shfl_xor_sync(0xffffffffu, a, d);
+      if (lane == 0) H[m * r + j] = a;
+    }
+  }
+}
+
+struct DecodeMainParams {
+  const uint32_t* bits;     // [N, K/32]
+  const uint16_t* B;        // [E, N, r]
+  const DecodeTokInfo* info;
+  const uint4* qfrag;
+  const float* H;           // [M, r]
+  const float* w_scales;
+  const float* alpha;
+  const float* beta;
+  uint16_t* Y;              // [M, N]
+  int* acc_dump;            // [M, N] exact 1-bit accumulators (test hook) or null
+  int M, K, N, r, sstride;
+  // shared-memory carve-up (bytes from the 128-byte aligned base)
+  int off_q, off_ring, off_h, off_red, ring_stage_bytes;
+};
+
+// Range of output features of CTA b: whole groups of 8, spread evenly.
+__device__ __forceinline__ void decode_range(int b, int nctas, int N, int& n_lo, int& n_hi) {
+  const int groups = N >> 3;
+  n_lo = (int)((long long)b * groups / nctas) << 3;
+  n_hi = (int)((long long)(b + 1) * groups / nctas) << 3;
+}
+
+__global__ void __launch_bounds__(kDecodeMainThreads, 1) k_decode_main(const __grid_constant__ DecodeMainParams p) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  __shared__ __align__(8) uint64_t bars[1 + kDecodeRing];
+  __shared__ DecodeTokInfo tok[kDecodeMaxTokens];
+  __shared__ int distinct[2][8], ndistinct[2];
+  __shared__ int fail;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, c = lane & 3;
+  int n_lo, n_hi;
+  decode_range(blockIdx.x, gridDim.x, p.N, n_lo, n_hi);
+  const int ncols = n_hi - n_lo;
+  const int nks = p.K >> 5, npairs = (nks + 1) >> 1;
+  const uint32_t bits_bytes = (uint32_t)ncols * (uint32_t)(p.K >> 3);
+  uint32_t* bits_s = reinterpret_cast<uint32_t*>(smem);
+  const uint32_t bar_bits = smem_u32(&bars[0]);
+
+  if (threadIdx.x == 0) {
+    fail = 0;
+    mbar_init(bar_bits, 1);
+    for (int s = 0; s < kDecodeRing; ++s) mbar_init(smem_u32(&bars[1 + s]), 1);
+    mbar_fence_init();
+    // the sign bits do not depend on the previous kernel: start them before waiting for it
+    if (ncols > 0) {
+      mbar_expect_tx(bar_bits, bits_bytes);
+      bulk_load(smem_u32(bits_s), p.bits + (long long)n_lo * nks, bits_bytes, bar_bits);
+    }
+  }
+  pdl_launch_dependents();
+  pdl_wait();
+  if (threadIdx.x < p.M) tok[threadIdx.x] = p.info[threadIdx.x];
+  __syncthreads();
+  const int ngroups = (p.M + 7) >> 3;
+  if (threadIdx.x < ngroups) {
+    // distinct experts of the tokens of this group, in order of first appearance
+    const int G = threadIdx.x;
+    int n = 0;
+    for (int t = 8 * G; t < min(p.M, 8 * G + 8); ++t) {
+      bool seen = false;
+      for (int i = 0; i < n; ++i) seen |= distinct[G][i] == tok[t].expert;
+      if (!seen) distinct[G][n++] = tok[t].expert;
+    }
+    ndistinct[G] = p.r > 0 ? n : 0;
+  }
+  __syncthreads();
+  if (ncols == 0) return;
+
+  const int ntile = (ncols + 15) >> 4;                 // 16-feature tiles of this CTA (<= 8)
+  const int kslices = (kDecodeMainThreads / 32) / ntile; // warps sharing one tile split the contraction
+  const int my_tile = warp % ntile, my_slice = warp / ntile;
+  const bool active = my_slice < kslices;
+  const int row0 = 16 * my_tile + g, row1 = row0 + 8;   // this thread's two features (local index)
+  const bool has0 = row0 < ncols, has1 = row1 < ncols;
+  uint4* q_s = reinterpret_cast<uint4*>(smem + p.off_q);
+  uint8_t* ring = smem + p.off_ring;
+  uint4* h_s = reinterpret_cast<uint4*>(smem + p.off_h);
+  int* red = reinterpret_cast<int*>(smem + p.off_red);
+  const int rsteps = (p.r + 31) >> 5;                   // 32 hidden values per step of the expert product
+  const uint32_t row_bytes = (uint32_t)p.r * 2u;
+  int ring_use = 0;                                      // expert-row loads consumed so far (all groups)
+  int ring_issued = 0;
+
+  for (int G = 0; G < ngroups; ++G) {
+    const int nd = ndistinct[G];
+    if (threadIdx.x == 0) {
+      // first expert rows of this group
+      for (; ring_issued < ring_use + min(nd, kDecodeRing); ++ring_issued) {
+        const int e = distinct[G][ring_issued - ring_use];
+        const uint32_t bar = smem_u32(&bars[1 + ring_issued % kDecodeRing]);
+        mbar_expect_tx(bar, (uint32_t)ncols * row_bytes);
+        bulk_load(smem_u32(ring + (ring_issued % kDecodeRing) * p.ring_stage_bytes), p.B + ((long long)e * p.N + n_lo) * p.r,
+                  (uint32_t)ncols * row_bytes, bar);
+      }
+    }
+    // activations of this group in fragment order; hidden activations as bf16 hi + lo fragments
+    {
+      const uint4* src = p.qfrag + (long long)G * npairs * 32;
+      for (int i = threadIdx.x; i < npairs * 32; i += kDecodeMainThreads) q_s[i] = __ldg(src + i);
+      for (int i = threadIdx.x; i < rsteps * 32; i += kDecodeMainThreads) {
+        const int s = i >> 5, ln = i & 31, tg = ln >> 2, tc = ln & 3;
+        const int t = 8 * G + tg, j0 = 8 * (4 * s + tc);
+        uint32_t hi[4] = {0, 0, 0, 0}, lo[4] = {0, 0, 0, 0};
+        if (t < p.M) {
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const int j = j0 + 2 * u;
+            const float v0 = j < p.r ? p.H[t * p.r + j] : 0.f, v1 = j + 1 < p.r ? p.H[t * p.r + j + 1] : 0.f;
+            hi[u] = pack_bf16x2(v0, v1);
+            lo[u] = pack_bf16x2(v0 - bf16lo(hi[u]), v1 - bf16hi(hi[u]));
+          }
+        }
+        h_s[i] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+        h_s[rsteps * 32 + i] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+      }
+    }
+    __syncthreads();
+    if (G == 0 && !mbar_wait(bar_bits, 0, WHERE_OTHER)) fail = 1;
+    __syncthreads();
+    if (fail) return;
+
+    // ---- 1-bit product: masked sums, weight 1 and weight 16
+    int acc1[4] = {0, 0, 0, 0}, acc16[4] = {0, 0, 0, 0};
+    if (active) {
+      const int p0 = (int)((long long)my_slice * npairs / kslices), p1 = (int)((long long)(my_slice + 1) * npairs / kslices);
+      const uint32_t* w0 = bits_s + (long long)(has0 ? row0 : 0) * nks;
+      const uint32_t* w1 = bits_s + (long long)(has1 ? row1 : 0) * nks;
+      for (int ip = p0; ip < p1; ++ip) {
+        const uint4 qv = q_s[ip * 32 + lane];
+        const int i0 = 2 * ip, i1 = min(2 * ip + 1, nks - 1);   // an odd word count pairs the last word with zeros of q
+        const uint32_t t00 = w0[i0] >> c, t01 = w0[i1] >> c, t10 = w1[i0] >> c, t11 = w1[i1] >> c;
+        const uint32_t a1[4] = {t00 & 0x01010101u, t10 & 0x01010101u, t01 & 0x01010101u, t11 & 0x01010101u};
+        const uint32_t a16[4] = {t00 & 0x10101010u, t10 & 0x10101010u, t01 & 0x10101010u, t11 & 0x10101010u};
+        mma_u8s8(acc1, a1, qv.x, qv.y);
+        mma_u8s8(acc16, a16, qv.z, qv.w);
+      }
+    }
+    // ---- expert product z = B_e h, tokens of other experts masked out
+    float z[4] = {0.f, 0.f, 0.f, 0.f};
+    const int my_tok = 8 * G + g;                          // the token whose h this thread feeds
+    const int my_tok_e = my_tok < p.M ? tok[my_tok].expert : -1;
+    for (int d = 0; d < nd; ++d) {
+      const int use = ring_use + d, stage = use % kDecodeRing;
+      if (!mbar_wait(smem_u32(&bars[1 + stage]), (use / kDecodeRing) & 1, WHERE_OTHER)) fail = 1;
+      const int e = distinct[G][d];
+      if (active && !fail) {
+        const uint8_t* rows = ring + stage * p.ring_stage_bytes;
+        const uint4* r0p = reinterpret_cast<const uint4*>(rows + (long long)(has0 ? row0 : 0) * row_bytes);
+        const uint4* r1p = reinterpret_cast<const uint4*>(rows + (long long)(has1 ? row1 : 0) * row_bytes);
+        const bool mine = my_tok_e == e;
+        for (int s = my_slice; s < rsteps; s += kslices) {
+          const int chunk = 4 * s + c;
+          uint4 b0 = make_uint4(0, 0, 0, 0), b1 = b0;
+          if (chunk * 8 < p.r) { b0 = r0p[chunk]; b1 = r1p[chunk]; }
+          uint4 hh = h_s[s * 32 + lane], hl = h_s[rsteps * 32 + s * 32 + lane];
+          if (!mine) { hh = make_uint4(0, 0, 0, 0); hl = hh; }
+          mma_bf16(z, b0.x, b1.x, b0.y, b1.y, hh.x, hh.y);
+          mma_bf16(z, b0.z, b1.z, b0.w, b1.w, hh.z, hh.w);
+          mma_bf16(z, b0.x, b1.x, b0.y, b1.y, hl.x, hl.y);
+          mma_bf16(z, b0.z, b1.z, b0.w, b1.w, hl.z, hl.w);
+        }
+      }
+      __syncthreads();   // every warp is done with this buffer
+      if (fail) return;
+      if (threadIdx.x == 0 && ring_issued < ring_use + nd) {
+        const int en = distinct[G][ring_issued - ring_use];
+        const uint32_t bar = smem_u32(&bars[1 + ring_issued % kDecodeRing]);
+        mbar_expect_tx(bar, (uint32_t)ncols * row_bytes);
+        bulk_load(smem_u32(ring + (ring_issued % kDecodeRing) * p.ring_stage_bytes), p.B + ((long long)en * p.N + n_lo) * p.r,
+                  (uint32_t)ncols * row_bytes, bar);
+        ++ring_issued;
+      }
+    }
+    ring_use += nd;
+
+    // ---- sum the contraction slices of a tile, then the epilogue (Eq. 10-11)
+    if (active) {
+      int* mine = red + ((my_slice * ntile + my_tile) * 32 + lane) * 8;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        mine[u] = acc1[u] + (acc16[u] >> 4);   // the weight-16 sums are exact multiples of 16
+        mine[4 + u] = __float_as_int(z[u]);
+      }
+    }
+    __syncthreads();
+    if (active && my_slice == 0) {
+      int ms[4] = {0, 0, 0, 0};
+      float zz[4] = {0.f, 0.f, 0.f, 0.f};
+      for (int s = 0; s < kslices; ++s) {
+        const int* part = red + ((s * ntile + my_tile) * 32 + lane) * 8;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) { ms[u] += part[u]; zz[u] += __int_as_float(part[4 + u]); }
+      }
+      const float lam = p.w_scales[0];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        // accumulator u: feature row0 (u < 2) or row1, token 8G + 2c + (u & 1)
+        const int nl = (u < 2) ? row0 : row1, t = 8 * G + 2 * c + (u & 1);
+        if (nl < ncols && t < p.M) {
+          const int n = n_lo + nl;
+          const int acc = 2 * ms[u] - tok[t].rowsum;
+          float y = p.beta[n * p.sstride] * __fdiv_rn(lam, tok[t].gamma) * (float)acc;
+          if (p.r > 0) y = fmaf(p.alpha[n * p.sstride] * tok[t].gate, zz[u], y);
+          p.Y[(long long)t * p.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(y));
+          if (p.acc_dump) p.acc_dump[(long long)t * p.N + n] = acc;
+        }
+      }
+    }
+    __syncthreads();   // q, h and the reduction buffer are rewritten by the next group
+  }
+}
+
+// ---------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------
+static inline size_t up256(size_t x) { return (x + 255) / 256 * 256; }
+
+size_t decode_workspace_bytes(int M, int K, int N, int r, bool dump) {
+  const size_t npairs = ((size_t)K / 32 + 1) / 2;
+  size_t b = up256(sizeof(DecodeTokInfo) * kDecodeMaxTokens);
+  b += up256(2 * npairs * 32 * sizeof(uint4));
+  b += up256(sizeof(float) * kDecodeMaxTokens * (size_t)(r > 0 ? r : 1));
+  if (dump) b += up256(sizeof(int) * (size_t)M * N);
+  return b;
+}
+
+DecodeViewPtrs decode_view(int M, int K, int N, int r, void* ws, bool dump) {
+  uint8_t* w = static_cast<uint8_t*>(ws);
+  const size_t npairs = ((size_t)K / 32 + 1) / 2;
+  DecodeViewPtrs v{w, nullptr};
+  w += up256(sizeof(DecodeTokInfo) * kDecodeMaxTokens) + up256(2 * npairs * 32 * sizeof(uint4)) +
+       up256(sizeof(float) * kDecodeMaxTokens * (size_t)(r > 0 ? r : 1));
+  if (dump) v.acc = reinterpret_cast<int*>(w);
+  (void)M; (void)N;
+  return v;
+}
+
+static int decode_sm_count() {
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
+  return n;
+}
+
+int decode_forward(const LayerArgs& a, const uint16_t* X, const uint32_t* bits, uint16_t* Y, void* ws, bool dump, cudaStream_t st) {
+  const int M = a.T, K = a.K, N = a.N, r = a.r, E = a.E;
+  uint8_t* w = static_cast<uint8_t*>(ws);
+  const size_t npairs = ((size_t)K / 32 + 1) / 2;
+  DecodeTokInfo* info = reinterpret_cast<DecodeTokInfo*>(w);
+  w += up256(sizeof(DecodeTokInfo) * kDecodeMaxTokens);
+  uint4* qfrag = reinterpret_cast<uint4*>(w);
+  w += up256(2 * npairs * 32 * sizeof(uint4));
+  float* H = reinterpret_cast<float*>(w);
+  w += up256(sizeof(float) * kDecodeMaxTokens * (size_t)(r > 0 ? r : 1));
+  int* acc_dump = dump ? reinterpret_cast<int*>(w) : nullptr;
+
+  static int sms = decode_sm_count();
+  const int groups = N / 8;
+  const int nctas = groups < sms ? groups : sms;
+  const int max_cols = ((groups + nctas - 1) / nctas) * 8;
+  if (max_cols > 128) return PQ_ERR_UNSUPPORTED;   // 16 warps cover at most 8 tiles of 16 features
+
+  DecodeMainParams p{};
+  p.bits = bits; p.B = a.B; p.info = info; p.qfrag = qfrag; p.H = H; p.w_scales = a.w_scales; p.alpha = a.alpha; p.beta = a.beta;
+  p.Y = Y; p.acc_dump = acc_dump; p.M = M; p.K = K; p.N = N; p.r = r; p.sstride = a.scale_stride;
+  size_t off = up256((size_t)max_cols * (K / 8));
+  p.off_q = (int)off; off += up256(npairs * 32 * sizeof(uint4));
+  p.ring_stage_bytes = (int)up256((size_t)max_cols * r * 2);
+  p.off_ring = (int)off; off += (size_t)kDecodeRing * p.ring_stage_bytes;
+  const int rsteps = (r + 31) / 32;
+  p.off_h = (int)off; off += up256((size_t)2 * (rsteps > 0 ? rsteps : 1) * 32 * sizeof(uint4));
+  p.off_red = (int)off; off += (size_t)(kDecodeMainThreads / 32) * 32 * 8 * sizeof(int);
+  const size_t smem_main = off + 128;
+  if (smem_main > 227 * 1024) return PQ_ERR_UNSUPPORTED;
+  const size_t smem_prep = (size_t)K * 2;
+  if (smem_prep > 200 * 1024) return PQ_ERR_UNSUPPORTED;
+  if (cudaFuncSetAttribute(k_decode_main, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_main) != cudaSuccess) return PQ_ERR_CUDA;
+  if (cudaFuncSetAttribute(k_decode_prep, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_prep) != cudaSuccess) return PQ_ERR_CUDA;
+
+  // slices of the hidden rows: enough CTAs to pull A_e at full rate, at least one row per warp
+  int slices = 1, rows_per_slice = 1;
+  if (r > 0) {
+    slices = 2 * sms / M;
+    const int max_slices = (r + 7) / 8;
+    if (slices > max_slices) slices = max_slices;
+    if (slices < 1) slices = 1;
+    rows_per_slice = (r + slices - 1) / slices;
+    slices = (r + rows_per_slice - 1) / rows_per_slice;
+  }
+
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg{};
+  cfg.stream = st; cfg.attrs = attr; cfg.numAttrs = 1;
+  {
+    cfg.gridDim = dim3(slices, M, 1); cfg.blockDim = dim3(256, 1, 1); cfg.dynamicSmemBytes = smem_prep;
+    LaunchScope ls(KID_DECODE_PREP, st);
+    if (cudaLaunchKernelEx(&cfg, k_decode_prep, reinterpret_cast<const uint4*>(X), reinterpret_cast<const uint4*>(a.Wr), a.A, M, K,
+                           (r > 0 && E > 1) ? E : 1, r, rows_per_slice, info, qfrag, H) != cudaSuccess)
+      return PQ_ERR_CUDA;
+  }
+  {
+    cfg.gridDim = dim3(nctas, 1, 1); cfg.blockDim = dim3(kDecodeMainThreads, 1, 1); cfg.dynamicSmemBytes = smem_main;
+    LaunchScope ls(KID_DECODE_MAIN, st);
+    if (cudaLaunchKernelEx(&cfg, k_decode_main, p) != cudaSuccess) return PQ_ERR_CUDA;
+  }
+  return PQ_OK;
+}
+
+}  // namespace pq

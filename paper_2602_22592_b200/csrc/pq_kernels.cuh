@@ -105,6 +105,12 @@ struct LayerArgs {
 int gemm_debug(int mode, int M, int N, int K, const void* A, const void* B, void* D, int tile_n, cudaStream_t st);
 int gemm_forward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, const uint16_t* xs, uint16_t* Y, cudaStream_t st);
 
+// decode path (pq_decode.cu)
+size_t decode_workspace_bytes(int M, int K, int N, int r, bool dump);
+int decode_forward(const LayerArgs& a, const uint16_t* X, const uint32_t* bits, uint16_t* Y, void* ws, bool dump, cudaStream_t st);
+struct DecodeViewPtrs { void* tokens; int* acc; };
+DecodeViewPtrs decode_view(int M, int K, int N, int r, void* ws, bool dump);
+
 struct BwdBuffers {
   const uint16_t* dys;   // [T,N] bf16 upstream gradient in sorted order
   const uint16_t* xs;    // [T,K] bf16 activations in sorted order

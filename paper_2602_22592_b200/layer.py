@@ -23,7 +23,7 @@ def _f32(a, dev):
 class PQLinear:
     """One decoupled linear layer of fixed shape on one CUDA device."""
 
-    def __init__(self, T, K, N, r=0, E=0, scale_vector=False, device="cuda:0", training=True):
+    def __init__(self, T, K, N, r=0, E=0, scale_vector=False, device="cuda:0", training=True, dump_acc=False):
         self.dev = torch.device(device)
         self.T, self.K, self.N, self.r, self.E = T, K, N, r, (E if r > 0 else 0)
         self.scale_vector = scale_vector
@@ -55,6 +55,12 @@ class PQLinear:
                 self.dWr = torch.empty((Ee, K), dtype=torch.float32, device=dev) if Ee > 1 else None
             else:
                 self.dA = self.dB = self.dWr = None
+        else:
+            # decode: T <= 16 tokens straight from the packed bits
+            self.desc = pqb.make_desc(T, K, N, r, self.E, 1, scale_vector, dump_acc=dump_acc)
+            nb = pqb.pq_workspace_bytes(self.desc, pqb.PQ_PHASE_DECODE)
+            self.ws_decode = torch.zeros(max(nb, 16), **u8) if T <= 16 else None
+            self.Y = torch.empty((T, N), dtype=torch.bfloat16, device=dev)
         self.X = self.W = self.A = self.B = self.Wr = self.alpha = self.beta = self.dY = None
 
     # -- data ---------------------------------------------------------------
@@ -72,8 +78,17 @@ class PQLinear:
         return self
 
     # -- calls --------------------------------------------------------------
-    def pack(self):
-        pqb.pq_pack_weights(self.desc, self.W, self.w_bits, self.w_s8, self.w_scales, self.ws_pack)
+    def pack(self, bits_only=False):
+        pqb.pq_pack_weights(self.desc, self.W, self.w_bits, None if bits_only else self.w_s8, self.w_scales, self.ws_pack)
+
+    def decode(self, X=None, Y=None):
+        """Inference forward from the packed sign bits (w_s8 is not used)."""
+        pqb.pq_linear_forward(self.desc, self.X if X is None else X, self.w_bits, None, self.w_scales, self.A, self.B, self.Wr,
+                              self.alpha, self.beta, self.Y if Y is None else Y, None, self.ws_decode)
+        return self.Y if Y is None else Y
+
+    def decode_view(self) -> dict:
+        return pqb.pq_decode_view_init(self.desc, self.ws_decode)
 
     def forward(self, X=None, Y=None):
         pqb.pq_linear_forward(self.desc, self.X if X is None else X, self.w_bits, self.w_s8, self.w_scales, self.A, self.B,

@@ -1,0 +1,101 @@
+"""GPU parity tests of the decode path (App. A): a few tokens against the packed sign bits,
+through the C ABI, against the CPU oracle reading the same bits back."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import pquant_oracle as O
+from paper_2602_22592_b200 import binding as pqb
+from paper_2602_22592_b200 import inputs as I
+from paper_2602_22592_b200.layer import PQLinear
+from test_gpu_forward import TOL_BF16, check_status, f32, rel_err
+
+pytestmark = pytest.mark.gpu
+
+
+def run_decode(c, scale_vector=False):
+    L = PQLinear(c["T"], c["K"], c["N"], c["r"], c["E"], scale_vector=scale_vector, training=False, dump_acc=True).load_case(c)
+    L.pack(bits_only=True)
+    L.decode()
+    torch.cuda.synchronize()
+    check_status()
+    return L
+
+
+def check_decode(c, L):
+    mu, lam = O.weight_scales(c["W"])
+    bits = O.pack_bits(O.binarize(c["W"], mu))
+    assert np.array_equal(L.w_bits.cpu().numpy().view(np.uint32), bits)
+    f = O.decode_forward(c["X"], bits, lam, c["A"], c["B"], c["Wr"], c["alpha"], c["beta"])
+    v = L.decode_view()
+    # integers: router index, int8 codes (through their sum), the 1-bit product itself
+    assert np.array_equal(v["expert"].cpu().numpy(), f["idx"])
+    assert np.array_equal(f32(v["gamma"]), f["gamma"])
+    assert np.array_equal(v["code_sum"].cpu().numpy(), f["q"].astype(np.int64).sum(axis=1))
+    assert np.array_equal(v["acc"].cpu().numpy().astype(np.int64), f["acc"])
+    assert rel_err(f32(v["gate"]), f["gate"]) <= 1e-5
+    assert rel_err(f32(L.Y), f["Y"]) <= TOL_BF16
+    return f
+
+
+DECODE_CASES = {
+    "m1_small": dict(T=1, K=256, N=96, r=32, E=4),
+    "m5_odd_words": dict(T=5, K=2080, N=992, r=40, E=3),          # 65 weight words per row, r not a multiple of 32
+    "m16_two_groups": dict(T=16, K=512, N=2048, r=64, E=8),
+    "m9_dense_hp": dict(T=9, K=384, N=320, r=160, E=1),
+    "m3_pure_1bit": dict(T=3, K=1024, N=64, r=0, E=0),
+    "m12_vector_scales": dict(T=12, K=320, N=4736, r=16, E=2, scale_vector=True, alpha=1.5, beta=0.4),
+}
+
+
+@pytest.mark.parametrize("name", list(DECODE_CASES))
+def test_decode_matches_oracle(name):
+    kw = dict(DECODE_CASES[name])
+    sv = kw.pop("scale_vector", False)
+    c = I.make_linear_case(kw.pop("T"), kw.pop("K"), kw.pop("N"), kw.pop("r"), kw.pop("E"), seed=21, scale_vector=sv,
+                           exact_quota=False, with_grad=False, **kw)
+    if sv:
+        c["alpha"] = (c["alpha"] * np.linspace(0.8, 1.2, c["N"])).astype(np.float32)
+        c["beta"] = (c["beta"] * np.linspace(1.2, 0.8, c["N"])).astype(np.float32)
+    check_decode(c, run_decode(c, sv))
+
+
+@pytest.mark.parametrize("M", [1, 4, 16])
+@pytest.mark.parametrize("proj", [0, 2])
+def test_decode_3b_shapes(M, proj):
+    # the 3B-shaped layers the decode benchmark streams: 3200 -> 8640 (gate) and 8640 -> 3200 (down)
+    c = I.config_decode(M, seed=4)[proj]
+    check_decode(c, run_decode(c))
+
+
+def test_decode_agrees_with_training_forward():
+    c = I.make_linear_case(16, 512, 768, 64, 4, seed=5, exact_quota=False, with_grad=False)
+    Ld = run_decode(c)
+    Lt = PQLinear(16, 512, 768, 64, 4).load_case(c)
+    Lt.pack(); Lt.forward()
+    torch.cuda.synchronize()
+    assert rel_err(f32(Ld.Y), f32(Lt.Y)) <= TOL_BF16
+    assert np.array_equal(Ld.decode_view()["expert"].cpu().numpy(), Lt.saved_view()["expert"].cpu().numpy())
+
+
+def test_decode_is_deterministic_and_repeatable():
+    c = I.make_linear_case(7, 640, 1280, 96, 8, seed=6, exact_quota=False, with_grad=False)
+    L = run_decode(c)
+    y = L.Y.clone()
+    for _ in range(3):
+        L.decode()
+    torch.cuda.synchronize()
+    check_status()
+    assert torch.equal(y, L.Y)
+
+
+def test_decode_rejects_too_many_tokens():
+    L = PQLinear(32, 256, 256, 32, 2, training=False)
+    c = I.make_linear_case(32, 256, 256, 32, 2, seed=1, with_grad=False)
+    L.load_case(c)
+    L.pack(bits_only=True)
+    assert pqb.pq_workspace_bytes(L.desc, pqb.PQ_PHASE_DECODE) == 0
+    ws = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
+    with pytest.raises(pqb.PqError) as ei:
+        pqb.pq_linear_forward(L.desc, L.X, L.w_bits, None, L.w_scales, L.A, L.B, L.Wr, L.alpha, L.beta, L.Y, None, ws)
+    assert ei.value.status == pqb.PQ_ERR_SHAPE
