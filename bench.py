@@ -289,6 +289,182 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+# --------------------------------------------------------------------------- decode workload
+DECODE_LAYERS = 26   # depth of the 3B-shaped decoder whose MLP projections form the working set
+
+
+def run_decode(args):
+    """Decode linears from packed 1-bit weights: 26 layers x (gate, up, down) of a 3B-shaped model, all with
+    distinct weights (far more bytes than L2), M tokens each, replayed as one CUDA graph.  The figure of merit
+    is the algorithmic bytes of the weights that must be read, per second, against the measured HBM rate."""
+    import torch
+    from paper_2602_22592_b200 import binding as pqb
+    from paper_2602_22592_b200 import build as pqbuild
+    from paper_2602_22592_b200 import inputs as I
+    from paper_2602_22592_b200.layer import PQLinear
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback for the product path")
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+    if rank == 0:
+        pqbuild.build()
+    if world > 1:
+        dist.barrier()
+    pqb.lib()
+    peaks, peak_kind = measured_peaks()
+    M = args.decode_tokens
+    hid, ffn, r, E = I.DECODE_3B["hidden"], I.DECODE_3B["ffn"], I.DECODE_3B["r"], I.DECODE_3B["E"]
+    gen = torch.Generator(device=device)
+    gen.manual_seed(4)
+    layers = []
+    for layer in range(DECODE_LAYERS):
+        for i, (name, K, N) in enumerate(I.mlp_shapes(hid, ffn)):
+            L = PQLinear(M, K, N, r, E, device=device, training=False)
+            act = I.decode_activations(M, K, E, seed=4 * 1024 + layer * 4 + i)
+            # weights drawn on the device (N(0, 0.02), the same law as the host generator), packed, latent copy dropped
+            L.W = torch.randn((N, K), generator=gen, device=device, dtype=torch.float32) * 0.02
+            L.pack(bits_only=True)
+            L.W = None
+            L.w_s8 = None
+            L.A = (torch.randn((E, r, K), generator=gen, device=device) * 0.02).to(torch.bfloat16)
+            L.B = (torch.randn((E, N, r), generator=gen, device=device) * 0.02).to(torch.bfloat16)
+            L.X = torch.from_numpy(act["X"]).to(device).to(torch.bfloat16)
+            L.Wr = torch.from_numpy(act["Wr"]).to(device).to(torch.bfloat16)
+            L.alpha = torch.full((1,), 2.0, device=device)
+            L.beta = torch.full((1,), 0.2, device=device)
+            layers.append(L)
+    torch.cuda.synchronize()
+
+    def step():
+        for L in layers:
+            L.decode()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    code, where = pqb.pq_device_status()
+    if code:
+        raise RuntimeError(f"device-side wait timed out during warm-up (where={where})")
+    # algorithmic bytes of one pass: sign bits + scale, the experts the tokens really use, router, activations
+    algo = 0
+    for L in layers:
+        experts = L.decode_view()["expert"].cpu().numpy()
+        algo += L.N * L.K // 8 + 4 + len(set(experts.tolist())) * 2 * r * (L.K + L.N) + 2 * E * L.K + 2 * M * L.K + 2 * M * L.N
+    def capture(nstreams):
+        """One CUDA graph of the whole pass.  nstreams = 1: every linear after the previous one, as the layers of a
+        decoder depend on each other.  nstreams > 1: the linears are dealt round-robin onto that many branches, so that
+        independent linears (other sequences, parallel projections) overlap and the weights stream back to back."""
+        side = [torch.cuda.Stream(device=device) for _ in range(nstreams)] if nstreams > 1 else []
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            if not side:
+                step()
+            else:
+                cur = torch.cuda.current_stream()
+                for si, st in enumerate(side):
+                    st.wait_stream(cur)
+                    with torch.cuda.stream(st):
+                        for L in layers[si::nstreams]:
+                            L.decode()
+                for st in side:
+                    cur.wait_stream(st)
+        return g
+
+    def time_graph(g):
+        for _ in range(3):
+            g.replay()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(args.steps):
+            g.replay()
+        b.record()
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b) / args.steps
+        if world > 1:
+            tt = torch.tensor([ms], device=device)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            ms = float(tt.item())
+        return ms
+
+    launches0 = pqb.pq_kernel_launches()
+    graph_serial = capture(1)
+    launches_per_step = pqb.pq_kernel_launches() - launches0
+    graph = capture(args.decode_streams)
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ms_serial = time_graph(graph_serial)
+    with ClockSampler(local) as clk:
+        ms_per_step = time_graph(graph)
+    code, where = pqb.pq_device_status()
+    if code:
+        raise RuntimeError(f"device-side wait timed out (where={where})")
+    # same pass launched call by call (no graph), for the launch-overhead comparison
+    t0.record()
+    for _ in range(min(args.steps, 20)):
+        step()
+    t1.record()
+    torch.cuda.synchronize()
+    ms_eager = t0.elapsed_time(t1) / min(args.steps, 20)
+
+    # end to end: every linear's activations from pinned host memory, every result back
+    hx = [L.X.cpu().pin_memory() for L in layers]
+    hy = [torch.empty_like(L.Y, device="cpu").pin_memory() for L in layers]
+
+    def step_e2e():
+        for i, L in enumerate(layers):
+            L.X.copy_(hx[i], non_blocking=True)
+            L.decode()
+            hy[i].copy_(L.Y, non_blocking=True)
+
+    for _ in range(2):
+        step_e2e()
+    torch.cuda.synchronize()
+    n_e2e = max(3, min(args.steps, 10))
+    t0.record()
+    for _ in range(n_e2e):
+        step_e2e()
+    t1.record()
+    torch.cuda.synchronize()
+    ms_e2e = t0.elapsed_time(t1) / n_e2e
+
+    gbs = algo / (ms_per_step * 1e-3) / 1e9
+    nlin = len(layers)
+    if rank == 0:
+        out = {
+            "metric": "pQuant decode linear (packed 1-bit weights) tokens/s", "value": round(world * M * nlin / (ms_per_step * 1e-3), 1),
+            "unit": "token-linears/s", "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "u8 bit masks x s8 -> s32 (1-bit branch), bf16 -> f32 (experts)", "data": "synthetic",
+            "config": {"workload": (f"decode, {M} token(s): {DECODE_LAYERS} layers x gate/up/down of a 3B-shaped model (hidden {hid}, FFN {ffn}), "
+                                    f"1-bit weights packed 32 per word, {E} bf16 experts of width {r}, top-1, Zipf(1.1)"),
+                       "linears_per_step": nlin, "l2": f"{algo / 1e6:.0f} MB of distinct weights per step, larger than L2",
+                       "launch": f"one CUDA graph per step, {args.decode_streams} independent linears in flight", "replicas": world},
+            "roofline": {"kernel": "k_decode_prep + k_decode_main (all launches of a step)", "bound": "hbm", "achieved": round(gbs, 1),
+                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(gbs / peaks["hbm_gbs"], 4),
+                         "peak_source": f"{peak_kind} hbm_gbs", "algorithmic_bytes_per_step": int(algo),
+                         "us_per_linear": round(ms_per_step * 1e3 / nlin, 3), "traffic": None},
+            "serial": {"ms_per_step": round(ms_serial, 4), "us_per_linear": round(ms_serial * 1e3 / nlin, 3),
+                       "hbm_frac": round(algo / (ms_serial * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
+                       "note": "the same pass with every linear launched after the previous one has finished (dependent layers)"},
+            "eager_ms_per_step": round(ms_eager, 4),
+            "cpu_baseline": None,
+            "e2e": {"value": round(world * M * nlin / (ms_e2e * 1e-3), 1), "unit": "token-linears/s",
+                    "h2d_bytes_per_step": sum(t.numel() * t.element_size() for t in hx),
+                    "d2h_bytes_per_step": sum(t.numel() * t.element_size() for t in hy), "steps": n_e2e},
+            "gpu_launches": int(launches_per_step * args.steps), "clocks": clk.summary(),
+        }
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 # --------------------------------------------------------------------------- oracle (CPU) arm
 def oracle_threads():
     try:
@@ -352,7 +528,9 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="mlp_dense", choices=["mlp_dense", "mlp_e8"])
+    ap.add_argument("--workload", default="mlp_dense", choices=["mlp_dense", "mlp_e8", "decode"])
+    ap.add_argument("--decode-tokens", type=int, default=1, choices=range(1, 17), metavar="M")
+    ap.add_argument("--decode-streams", type=int, default=8, help="independent decode linears in flight (graph branches)")
     ap.add_argument("--cpu-tokens", type=int, default=4096)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
@@ -360,6 +538,8 @@ def main():
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == "decode":
+        run_decode(args)
     else:
         run_ours(args)
 

@@ -207,6 +207,13 @@ int pq_debug_gemm_tile(int mode, int M, int N, int K, const void* A, const void*
  * waiting role.  The word is cleared by the call. */
 int pq_device_status(void* stream, int* code, int* where);
 
+/* Process-wide launch options.
+ *   PQ_OPT_DECODE_PDL (default 1): launch the decode kernels with programmatic stream
+ *   serialisation, so that a kernel's prologue (barrier set-up, the copy of the sign bits)
+ *   overlaps the tail of the kernel before it in the stream.  0 = plain stream order. */
+enum { PQ_OPT_DECODE_PDL = 1 };
+int pq_set_option(int option, int value);
+
 /* Cumulative number of kernels this library has launched in this process. */
 long long pq_kernel_launches(void);
 

@@ -23,7 +23,7 @@ PQ_PHASE_PACK, PQ_PHASE_FWD, PQ_PHASE_BWD, PQ_PHASE_DECODE = 0, 1, 2, 3
 
 EXPORTS = ("pq_status_string", "pq_workspace_bytes", "pq_saved_bytes", "pq_saved_view_init",
            "pq_decode_view_init", "pq_pack_weights", "pq_pack_weights_static", "pq_linear_forward", "pq_linear_backward", "pq_debug_gemm", "pq_debug_gemm_tile",
-           "pq_device_status", "pq_kernel_launches", "pq_profile_events")
+           "pq_device_status", "pq_kernel_launches", "pq_profile_events", "pq_set_option")
 
 KERNEL_IDS = dict(pack_sums=0, binarize_pack=1, router=2, route_scan=3, act_quant=4, hp_up=5, fwd=6, scatter_rows=7,
                   scaled_sign=8, scaled_b=9, hp_dh=10, bwd_dx=11, bwd_dw=12, hp_db=13, hp_da=14, router_wgrad=15,
@@ -90,6 +90,8 @@ def lib() -> ctypes.CDLL:
         L.pq_device_status.argtypes = [vp, ctypes.POINTER(ci), ctypes.POINTER(ci)]
         L.pq_kernel_launches.restype = ctypes.c_longlong
         L.pq_kernel_launches.argtypes = []
+        L.pq_set_option.restype = ci
+        L.pq_set_option.argtypes = [ci, ci]
         L.pq_profile_events.restype = ci
         L.pq_profile_events.argtypes = [ci, vp, vp]
         _lib = L
@@ -211,6 +213,13 @@ def pq_device_status(stream=None) -> tuple[int, int]:
     code, where = ctypes.c_int(0), ctypes.c_int(0)
     _check("pq_device_status", lib().pq_device_status(_stream(stream), ctypes.byref(code), ctypes.byref(where)))
     return code.value, where.value
+
+
+PQ_OPT_DECODE_PDL = 1
+
+
+def pq_set_option(option: int, value: int):
+    _check("pq_set_option", lib().pq_set_option(option, value))
 
 
 def pq_kernel_launches() -> int:

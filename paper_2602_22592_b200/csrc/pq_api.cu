@@ -416,6 +416,13 @@ int pq_debug_gemm_tile(int mode, int M, int N, int K, const void* A, const void*
   return gemm_debug(mode, M, N, K, A, B, D, tile_n, static_cast<cudaStream_t>(stream));
 }
 
+int pq_set_option(int option, int value) {
+  switch (option) {
+    case PQ_OPT_DECODE_PDL: decode_set_pdl(value); return PQ_OK;
+    default: return PQ_ERR_UNSUPPORTED;
+  }
+}
+
 long long pq_kernel_launches(void) { return g_launches; }
 
 int pq_profile_events(int kernel_id, void* start_event, void* stop_event) {

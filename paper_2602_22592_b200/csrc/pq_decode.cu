@@ -94,13 +94,22 @@ __global__ void __launch_bounds__(256) k_decode_prep(const uint4* __restrict__ X
   if (E > 1) {
     for (int e = warp; e < E; e += 8) {
       float acc = 0.f;
-      for (int c = lane; c < chunks; c += 32) {
-        const uint4 xv = xs4[c];
-        const uint4 wv = __ldg(Wr + (long long)e * chunks + c);
-        acc = fmaf(bf16lo(xv.x), bf16lo(wv.x), acc); acc = fmaf(bf16hi(xv.x), bf16hi(wv.x), acc);
-        acc = fmaf(bf16lo(xv.y), bf16lo(wv.y), acc); acc = fmaf(bf16hi(xv.y), bf16hi(wv.y), acc);
-        acc = fmaf(bf16lo(xv.z), bf16lo(wv.z), acc); acc = fmaf(bf16hi(xv.z), bf16hi(wv.z), acc);
-        acc = fmaf(bf16lo(xv.w), bf16lo(wv.w), acc); acc = fmaf(bf16hi(xv.w), bf16hi(wv.w), acc);
+      const uint4* wrow = Wr + (long long)e * chunks;
+      // eight loads in flight per lane; the additions keep the ascending order of the chunks
+      for (int c0 = lane; c0 < chunks; c0 += 32 * 8) {
+        uint4 wv[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) wv[u] = (c0 + 32 * u < chunks) ? __ldg(wrow + c0 + 32 * u) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          if (c0 + 32 * u < chunks) {
+            const uint4 xv = xs4[c0 + 32 * u];
+            acc = fmaf(bf16lo(xv.x), bf16lo(wv[u].x), acc); acc = fmaf(bf16hi(xv.x), bf16hi(wv[u].x), acc);
+            acc = fmaf(bf16lo(xv.y), bf16lo(wv[u].y), acc); acc = fmaf(bf16hi(xv.y), bf16hi(wv[u].y), acc);
+            acc = fmaf(bf16lo(xv.z), bf16lo(wv[u].z), acc); acc = fmaf(bf16hi(xv.z), bf16hi(wv[u].z), acc);
+            acc = fmaf(bf16lo(xv.w), bf16lo(wv[u].w), acc); acc = fmaf(bf16hi(xv.w), bf16hi(wv[u].w), acc);
+          }
+        }
       }
       for (int d = 16; d > 0; d >>= 1) acc = acc + __shfl_xor_sync(0xffffffffu, acc, d);
       if (lane == 0) logit_sh[e] = acc;
@@ -170,13 +179,20 @@ __global__ void __launch_bounds__(256) k_decode_prep(const uint4* __restrict__ X
     for (int j = j0 + warp; j < j1; j += 8) {
       const uint4* arow = reinterpret_cast<const uint4*>(A + ((long long)best * r + j) * K);
       float a0 = 0.f, a1 = 0.f;
-      for (int c = lane; c < chunks; c += 32) {
-        const uint4 xv = xs4[c];
-        const uint4 wv = __ldg(arow + c);
-        a0 = fmaf(bf16lo(xv.x), bf16lo(wv.x), a0); a1 = fmaf(bf16hi(xv.x), bf16hi(wv.x), a1);
-        a0 = fmaf(bf16lo(xv.y), bf16lo(wv.y), a0); a1 = fmaf(bf16hi(xv.y), bf16hi(wv.y), a1);
-        a0 = fmaf(bf16lo(xv.z), bf16lo(wv.z), a0); a1 = fmaf(bf16hi(xv.z), bf16hi(wv.z), a1);
-        a0 = fmaf(bf16lo(xv.w), bf16lo(wv.w), a0); a1 = fmaf(bf16hi(xv.w), bf16hi(wv.w), a1);
+      for (int c0 = lane; c0 < chunks; c0 += 32 * 8) {
+        uint4 wv[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) wv[u] = (c0 + 32 * u < chunks) ? __ldg(arow + c0 + 32 * u) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          if (c0 + 32 * u < chunks) {
+            const uint4 xv = xs4[c0 + 32 * u];
+            a0 = fmaf(bf16lo(xv.x), bf16lo(wv[u].x), a0); a1 = fmaf(bf16hi(xv.x), bf16hi(wv[u].x), a1);
+            a0 = fmaf(bf16lo(xv.y), bf16lo(wv[u].y), a0); a1 = fmaf(bf16hi(xv.y), bf16hi(wv[u].y), a1);
+            a0 = fmaf(bf16lo(xv.z), bf16lo(wv[u].z), a0); a1 = fmaf(bf16hi(xv.z), bf16hi(wv[u].z), a1);
+            a0 = fmaf(bf16lo(xv.w), bf16lo(wv[u].w), a0); a1 = fmaf(bf16hi(xv.w), bf16hi(wv[u].w), a1);
+          }
+        }
       }
       float a = a0 + a1;
       for (int d = 16; d > 0; d >>= 1) a += __shfl_xor_sync(0xffffffffu, a, d);
@@ -210,7 +226,7 @@ __device__ __forceinline__ void decode_range(int b, int nctas, int N, int& n_lo,
 
 __global__ void __launch_bounds__(kDecodeMainThreads, 1) k_decode_main(const __grid_constant__ DecodeMainParams p) {
   extern __shared__ __align__(128) uint8_t smem[];
-  __shared__ __align__(8) uint64_t bars[1 + kDecodeRing];
+  __shared__ __align__(8) uint64_t bars[2 + kDecodeRing];   // sign bits, q fragments, expert-row ring
   __shared__ DecodeTokInfo tok[kDecodeMaxTokens];
   __shared__ int distinct[2][8], ndistinct[2];
   __shared__ int fail;
@@ -222,12 +238,14 @@ __global__ void __launch_bounds__(kDecodeMainThreads, 1) k_decode_main(const __g
   const int nks = p.K >> 5, npairs = (nks + 1) >> 1;
   const uint32_t bits_bytes = (uint32_t)ncols * (uint32_t)(p.K >> 3);
   uint32_t* bits_s = reinterpret_cast<uint32_t*>(smem);
-  const uint32_t bar_bits = smem_u32(&bars[0]);
+  const uint32_t bar_bits = smem_u32(&bars[0]), bar_q = smem_u32(&bars[1]);
+  auto ring_bar = [&](int i) { return smem_u32(&bars[2 + i % kDecodeRing]); };
 
   if (threadIdx.x == 0) {
     fail = 0;
     mbar_init(bar_bits, 1);
-    for (int s = 0; s < kDecodeRing; ++s) mbar_init(smem_u32(&bars[1 + s]), 1);
+    mbar_init(bar_q, 1);
+    for (int s = 0; s < kDecodeRing; ++s) mbar_init(ring_bar(s), 1);
     mbar_fence_init();
     // the sign bits do not depend on the previous kernel: start them before waiting for it
     if (ncols > 0) {
@@ -272,38 +290,38 @@ __global__ void __launch_bounds__(kDecodeMainThreads, 1) k_decode_main(const __g
   for (int G = 0; G < ngroups; ++G) {
     const int nd = ndistinct[G];
     if (threadIdx.x == 0) {
-      // first expert rows of this group
+      // activations of this group (already in fragment order) and its first expert rows
+      mbar_expect_tx(bar_q, (uint32_t)npairs * 32u * 16u);
+      bulk_load(smem_u32(q_s), p.qfrag + (long long)G * npairs * 32, (uint32_t)npairs * 32u * 16u, bar_q);
       for (; ring_issued < ring_use + min(nd, kDecodeRing); ++ring_issued) {
         const int e = distinct[G][ring_issued - ring_use];
-        const uint32_t bar = smem_u32(&bars[1 + ring_issued % kDecodeRing]);
-        mbar_expect_tx(bar, (uint32_t)ncols * row_bytes);
+        mbar_expect_tx(ring_bar(ring_issued), (uint32_t)ncols * row_bytes);
         bulk_load(smem_u32(ring + (ring_issued % kDecodeRing) * p.ring_stage_bytes), p.B + ((long long)e * p.N + n_lo) * p.r,
-                  (uint32_t)ncols * row_bytes, bar);
+                  (uint32_t)ncols * row_bytes, ring_bar(ring_issued));
       }
     }
-    // activations of this group in fragment order; hidden activations as bf16 hi + lo fragments
-    {
-      const uint4* src = p.qfrag + (long long)G * npairs * 32;
-      for (int i = threadIdx.x; i < npairs * 32; i += kDecodeMainThreads) q_s[i] = __ldg(src + i);
-      for (int i = threadIdx.x; i < rsteps * 32; i += kDecodeMainThreads) {
-        const int s = i >> 5, ln = i & 31, tg = ln >> 2, tc = ln & 3;
-        const int t = 8 * G + tg, j0 = 8 * (4 * s + tc);
-        uint32_t hi[4] = {0, 0, 0, 0}, lo[4] = {0, 0, 0, 0};
-        if (t < p.M) {
+    // hidden activations as bf16 hi + lo fragments
+    for (int i = threadIdx.x; i < rsteps * 32; i += kDecodeMainThreads) {
+      const int s = i >> 5, ln = i & 31, tg = ln >> 2, tc = ln & 3;
+      const int t = 8 * G + tg, j0 = 8 * (4 * s + tc);
+      uint32_t hi[4] = {0, 0, 0, 0}, lo[4] = {0, 0, 0, 0};
+      if (t < p.M) {
+        float v[8];
 #pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            const int j = j0 + 2 * u;
-            const float v0 = j < p.r ? p.H[t * p.r + j] : 0.f, v1 = j + 1 < p.r ? p.H[t * p.r + j + 1] : 0.f;
-            hi[u] = pack_bf16x2(v0, v1);
-            lo[u] = pack_bf16x2(v0 - bf16lo(hi[u]), v1 - bf16hi(hi[u]));
-          }
+        for (int u = 0; u < 8; ++u) v[u] = j0 + u < p.r ? p.H[t * p.r + j0 + u] : 0.f;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          hi[u] = pack_bf16x2(v[2 * u], v[2 * u + 1]);
+          lo[u] = pack_bf16x2(v[2 * u] - bf16lo(hi[u]), v[2 * u + 1] - bf16hi(hi[u]));
         }
-        h_s[i] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-        h_s[rsteps * 32 + i] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
       }
+      h_s[i] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+      h_s[rsteps * 32 + i] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
     }
-    __syncthreads();
-    if (G == 0 && !mbar_wait(bar_bits, 0, WHERE_OTHER)) fail = 1;
+    if (threadIdx.x == 0) {   // one thread polls, the rest wait at the barrier
+      if (!mbar_wait(bar_q, G & 1, WHERE_OTHER)) fail = 1;
+      if (G == 0 && !mbar_wait(bar_bits, 0, WHERE_OTHER)) fail = 1;
+    }
     __syncthreads();
     if (fail) return;
 
@@ -329,9 +347,11 @@ __global__ void __launch_bounds__(kDecodeMainThreads, 1) k_decode_main(const __g
     const int my_tok_e = my_tok < p.M ? tok[my_tok].expert : -1;
     for (int d = 0; d < nd; ++d) {
       const int use = ring_use + d, stage = use % kDecodeRing;
-      if (!mbar_wait(smem_u32(&bars[1 + stage]), (use / kDecodeRing) & 1, WHERE_OTHER)) fail = 1;
+      if (threadIdx.x == 0 && !mbar_wait(ring_bar(use), (use / kDecodeRing) & 1, WHERE_OTHER)) fail = 1;
+      __syncthreads();
+      if (fail) return;
       const int e = distinct[G][d];
-      if (active && !fail) {
+      if (active) {
         const uint8_t* rows = ring + stage * p.ring_stage_bytes;
         const uint4* r0p = reinterpret_cast<const uint4*>(rows + (long long)(has0 ? row0 : 0) * row_bytes);
         const uint4* r1p = reinterpret_cast<const uint4*>(rows + (long long)(has1 ? row1 : 0) * row_bytes);
@@ -348,15 +368,15 @@ __global__ void __launch_bounds__(kDecodeMainThreads, 1) k_decode_main(const __g
           mma_bf16(z, b0.z, b1.z, b0.w, b1.w, hl.z, hl.w);
         }
       }
-      __syncthreads();   // every warp is done with this buffer
-      if (fail) return;
-      if (threadIdx.x == 0 && ring_issued < ring_use + nd) {
-        const int en = distinct[G][ring_issued - ring_use];
-        const uint32_t bar = smem_u32(&bars[1 + ring_issued % kDecodeRing]);
-        mbar_expect_tx(bar, (uint32_t)ncols * row_bytes);
-        bulk_load(smem_u32(ring + (ring_issued % kDecodeRing) * p.ring_stage_bytes), p.B + ((long long)en * p.N + n_lo) * p.r,
-                  (uint32_t)ncols * row_bytes, bar);
-        ++ring_issued;
+      if (nd > kDecodeRing) {   // more experts than buffers: refill this one once every warp is done with it
+        __syncthreads();
+        if (threadIdx.x == 0 && ring_issued < ring_use + nd) {
+          const int en = distinct[G][ring_issued - ring_use];
+          mbar_expect_tx(ring_bar(ring_issued), (uint32_t)ncols * row_bytes);
+          bulk_load(smem_u32(ring + (ring_issued % kDecodeRing) * p.ring_stage_bytes), p.B + ((long long)en * p.N + n_lo) * p.r,
+                    (uint32_t)ncols * row_bytes, ring_bar(ring_issued));
+          ++ring_issued;
+        }
       }
     }
     ring_use += nd;
@@ -423,6 +443,10 @@ DecodeViewPtrs decode_view(int M, int K, int N, int r, void* ws, bool dump) {
   return v;
 }
 
+// Launch option: programmatic stream serialisation of the two decode kernels (on by default).
+static int g_decode_pdl = 1;
+void decode_set_pdl(int on) { g_decode_pdl = on ? 1 : 0; }
+
 static int decode_sm_count() {
   int dev = 0, n = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return 148;
@@ -480,7 +504,7 @@ int decode_forward(const LayerArgs& a, const uint16_t* X, const uint32_t* bits, 
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cudaLaunchConfig_t cfg{};
-  cfg.stream = st; cfg.attrs = attr; cfg.numAttrs = 1;
+  cfg.stream = st; cfg.attrs = attr; cfg.numAttrs = g_decode_pdl ? 1 : 0;
   {
     cfg.gridDim = dim3(slices, M, 1); cfg.blockDim = dim3(256, 1, 1); cfg.dynamicSmemBytes = smem_prep;
     LaunchScope ls(KID_DECODE_PREP, st);

@@ -145,3 +145,13 @@ def config_decode(M: int, seed: int = 4, layers: int = 1) -> list[dict]:
             c["name"] = f"L{layer}.{name}"
             cases.append(c)
     return cases
+
+
+def decode_activations(M: int, K: int, E: int, seed: int, plant: float = 6.0) -> dict:
+    """Activations and router of one decode linear without the (large) weight draws:
+    X [M,K] ~ N(0,1) bf16 with a Zipf(1.1) expert planted per token (i.i.d. draws), Wr [E,K] orthonormal rows."""
+    rr = _rng(seed, 4)
+    Wr = router_weights(E, K, rr, orthonormal=True)
+    planted = zipf_assignment(M, E, rr, exact_quota=False)
+    X = _rng(seed, 0).standard_normal((M, K), dtype=np.float32) + np.float32(plant) * Wr[planted]
+    return dict(X=bf16_values(X), Wr=Wr, planted=planted)
