@@ -196,10 +196,11 @@ def run_ours(args):
     value = world * tokens / (ms_per_step * 1e-3)
 
     dw_ms = float(np.mean([a.elapsed_time(b) for row in ev for a, b in row]))
-    dw_flops = float(np.mean([2.0 * L.T * L.N * L.K for L in layers]))
+    # algorithmic flops of the launch: dW = dY^T . (q/gamma) and, in the same launch, dB_e = dY^T . (g H)
+    dw_flops = float(np.mean([2.0 * L.T * L.N * L.K + 2.0 * L.T * L.N * L.r for L in layers]))
     achieved = dw_flops / (dw_ms * 1e-3) / 1e12
     peak = peaks["bf16_tflops_sustained"]
-    roofline = {"kernel": "bwd_dw (dW = dY^T . q/gamma, bf16 tcgen05, fp32 accumulate)", "bound": "tensor",
+    roofline = {"kernel": "k_gemm_bwd_dw (dW = dY^T . q/gamma and dB = dY^T . gH, bf16 tcgen05, fp32 accumulate)", "bound": "tensor",
                 "achieved": round(achieved, 1), "peak": peak, "unit": "TFLOP/s", "frac": round(achieved / peak, 4),
                 "peak_source": f"{peak_kind} bf16_tflops_sustained", "avg_launch_ms": round(dw_ms, 4),
                 "traffic": NCU_TRAFFIC_BYTES["bwd_dw"]}

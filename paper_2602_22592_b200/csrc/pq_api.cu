@@ -26,14 +26,13 @@ static inline int experts_of(const pq_desc* d) { return d->r > 0 ? (d->E < 1 ? 1
 static inline int max_items_of(const pq_desc* d) { return mtiles_of(d) + experts_of(d) - 1; }
 static inline bool routed(const pq_desc* d) { return d->r > 0 && d->E > 1; }
 
-// Items per chunk for the split token contraction of dA (table a) and dB (table b): small enough that
-// (chunks x output tiles) fills about two waves of 148 CTAs, large enough to keep the partial buffers small.
+// Items per chunk for the split token contraction of dA: (chunks x output tiles)
+// should fill about one wave of 148 CTAs; more chunks only add fp32 partial results to write and re-read.
 static inline int chunk_items(int mtiles, int out_tiles) {
-  int c = mtiles * out_tiles / 296;
+  int c = (mtiles * out_tiles + 147) / 148;
   return c < 1 ? 1 : c;
 }
 static inline int chunk_a_of(const pq_desc* d) { return chunk_items(mtiles_of(d), (d->K + 255) / 256); }
-static inline int chunk_b_of(const pq_desc* d) { return chunk_items(mtiles_of(d), (d->N + 127) / 128); }
 static inline int max_chunks(const pq_desc* d, int chunk) { return (max_items_of(d) + chunk - 1) / chunk + experts_of(d); }
 
 static int check_desc(const pq_desc* d, bool training) {
@@ -69,14 +68,11 @@ static size_t carve_saved(const pq_desc* d, void* base, SavedPtrs* out) {
   s.rt.items = c.take<int4>(s.max_items);
   s.rt.tile_item_begin = c.take<int>(mtiles_of(d) + 1);
   s.rt.expert_item_begin = c.take<int>(E + 1);
-  s.chunk_a = chunk_a_of(d); s.chunk_b = chunk_b_of(d);
-  s.max_chunks_a = max_chunks(d, s.chunk_a); s.max_chunks_b = max_chunks(d, s.chunk_b);
+  s.chunk_a = chunk_a_of(d);
+  s.max_chunks_a = max_chunks(d, s.chunk_a);
   s.rt.n_chunks_a = c.take<int>(1);
   s.rt.chunks_a = c.take<int4>(s.max_chunks_a);
   s.rt.expert_chunk_begin_a = c.take<int>(E + 1);
-  s.rt.n_chunks_b = c.take<int>(1);
-  s.rt.chunks_b = c.take<int4>(s.max_chunks_b);
-  s.rt.expert_chunk_begin_b = c.take<int>(E + 1);
   if (out) *out = s;
   return c.off;
 }
@@ -108,7 +104,6 @@ struct BwdScratch {
   float* dalpha_vec;
   float* dbeta_vec;
   float* da_partial;
-  float* db_partial;
 };
 
 static size_t carve_bwd_scratch(const pq_desc* d, void* base, BwdScratch* out) {
@@ -124,13 +119,12 @@ static size_t carve_bwd_scratch(const pq_desc* d, void* base, BwdScratch* out) {
   s.gh = r > 0 ? c.take<uint16_t>((size_t)2 * max_items_of(d) * kTileRows * r) : nullptr;
   s.dl = routed(d) ? c.take<float>(T * E) : nullptr;
   s.dlc = routed(d) ? c.take<uint16_t>(T * 16) : nullptr;
-  s.dbeta_partial = c.take<float>(((K + 31) / 32) * N);   // one slot per 32 columns of K
-  s.dalpha_partial = r > 0 ? c.take<float>((size_t)E * N) : nullptr;
+  s.dbeta_partial = c.take<float>(2 * ((K + 255) / 256) * N);   // two slots per 256-column tile of K
+  s.dalpha_partial = r > 0 ? c.take<float>((size_t)2 * E * N) : nullptr;
   s.dwr_partial = routed(d) ? c.take<float>(((T + 255) / 256) * E * K) : nullptr;
   s.dalpha_vec = c.take<float>(N);
   s.dbeta_vec = c.take<float>(N);
   s.da_partial = r > 0 ? c.take<float>((size_t)max_chunks(d, chunk_a_of(d)) * r * K) : nullptr;
-  s.db_partial = r > 0 ? c.take<float>((size_t)max_chunks(d, chunk_b_of(d)) * N * r) : nullptr;
   if (out) *out = s;
   return c.off;
 }
@@ -382,23 +376,19 @@ int pq_linear_backward(const pq_desc* d, const uint16_t* dY, const uint16_t* X, 
   }
   b.dhc = sc.dhc; b.gh = sc.gh; b.dl = sc.dl; b.dlc = sc.dlc;
   b.dbeta_partial = sc.dbeta_partial; b.dalpha_partial = sc.dalpha_partial;
-  b.da_partial = sc.da_partial; b.db_partial = sc.db_partial;
+  b.da_partial = sc.da_partial;
   rc = gemm_backward(a, w_s8, sv, b, dX, dW, dA, dB, st);
   if (rc) return rc;
 
   if (routed(d)) {
     if (launch_router_wgrad(sv.xs, sc.dl, d->T, d->K, E, sc.dwr_partial, dWr, nullptr, st) != cudaSuccess) return PQ_ERR_CUDA;
   }
-  // dbeta_n = lam * sum over the 32-column slots of the partial sign-weighted row sums; scalar form sums over n
-  const int nslots = (d->K + 31) / 32;
-  if (launch_sum_partials(sc.dbeta_partial, nslots, d->N, w_scales, vec ? dbeta : sc.dbeta_vec, st) != cudaSuccess) return PQ_ERR_CUDA;
-  if (!vec && launch_sum_to_scalar(sc.dbeta_vec, d->N, dbeta, st) != cudaSuccess) return PQ_ERR_CUDA;
-  if (hp) {
-    if (launch_sum_partials(sc.dalpha_partial, E, d->N, nullptr, vec ? dalpha : sc.dalpha_vec, st) != cudaSuccess) return PQ_ERR_CUDA;
-    if (!vec && launch_sum_to_scalar(sc.dalpha_vec, d->N, dalpha, st) != cudaSuccess) return PQ_ERR_CUDA;
-  } else if (dalpha) {
-    if (cudaMemsetAsync(dalpha, 0, sizeof(float) * (vec ? d->N : 1), st) != cudaSuccess) return PQ_ERR_CUDA;
-  }
+  // dbeta_n = lam * sum over the column tiles of the partial sign-weighted row sums, dalpha_n = sum over experts
+  // of the dB-weighted row sums; the scalar form sums over n as well
+  if (dalpha && !hp && cudaMemsetAsync(dalpha, 0, sizeof(float) * (vec ? d->N : 1), st) != cudaSuccess) return PQ_ERR_CUDA;
+  if (launch_finalize_scales(sc.dbeta_partial, 2 * ((d->K + 255) / 256), hp ? sc.dalpha_partial : nullptr, 2 * E, d->N, w_scales, vec, dbeta,
+                             hp ? dalpha : nullptr, sc.dbeta_vec, sc.dalpha_vec, st) != cudaSuccess)
+    return PQ_ERR_CUDA;
   return PQ_OK;
 }
 

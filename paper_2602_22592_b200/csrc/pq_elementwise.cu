@@ -47,18 +47,23 @@ __global__ void __launch_bounds__(256) k_weight_partial_sums(const float4* __res
   }
 }
 
-// Every block re-reduces the (few hundred) partials in the same order, so all
-// blocks agree on mu without a grid-wide barrier.
+// Every block re-reduces the (few hundred) partials in the same order, so all blocks agree on mu without
+// a grid-wide barrier: thread t sums partials t, t + 256, ... (ascending), then a fixed tree over the block.
 __device__ __forceinline__ void reduce_partials(const double* partial, int nparts, double inv_count, float* mu, float* lam) {
+  __shared__ double sh[2][8];
   __shared__ double fin[2];
-  if (threadIdx.x < 32) {
-    double s = 0.0, a = 0.0;
-    for (int i = threadIdx.x; i < nparts; i += 32) { s += partial[2 * i]; a += partial[2 * i + 1]; }
-    for (int d = 16; d > 0; d >>= 1) {
-      s += __shfl_xor_sync(0xffffffffu, s, d);
-      a += __shfl_xor_sync(0xffffffffu, a, d);
-    }
-    if (threadIdx.x == 0) { fin[0] = s; fin[1] = a; }
+  double s = 0.0, a = 0.0;
+  for (int i = threadIdx.x; i < nparts; i += 256) { s += partial[2 * i]; a += partial[2 * i + 1]; }
+  for (int d = 16; d > 0; d >>= 1) {
+    s += __shfl_xor_sync(0xffffffffu, s, d);
+    a += __shfl_xor_sync(0xffffffffu, a, d);
+  }
+  if ((threadIdx.x & 31) == 0) { sh[0][threadIdx.x >> 5] = s; sh[1][threadIdx.x >> 5] = a; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double ts = 0.0, ta = 0.0;
+    for (int w = 0; w < 8; ++w) { ts += sh[0][w]; ta += sh[1][w]; }
+    fin[0] = ts; fin[1] = ta;
   }
   __syncthreads();
   *mu = (float)(fin[0] * inv_count);
@@ -191,8 +196,8 @@ __global__ void __launch_bounds__(256) k_router(const uint4* __restrict__ X, con
 // table.  An item is the intersection of a 128-row tile of the sorted token
 // order with one expert's range: {tile, expert, first row, end row} (rows
 // relative to the tile).  Items are sorted by tile and therefore by expert.
-// Also groups each expert's items into chunks (two tables, two chunk sizes): the
-// units over which the token contraction of dA and dB is split across CTAs.
+// Also groups each expert's items into chunks: the units over which the token
+// contraction of dA is split across CTAs.
 // One block; the work is a few hundred integers.
 // ---------------------------------------------------------------------------
 // Items of one 128-row tile [r0, r1) of the sorted order: experts e0 <= e < E whose non-empty range
@@ -233,7 +238,7 @@ __device__ __forceinline__ void build_chunks(int Ee, const int* item_begin /*sha
 
 __global__ void __launch_bounds__(512) k_route_scan(int T, int E, int nblocks, const int* __restrict__ block_counts,
                                                     int* __restrict__ block_base, int* __restrict__ offsets, RoutingTables rt,
-                                                    int chunk_a, int chunk_b) {
+                                                    int chunk_a) {
   __shared__ int off[kMaxExperts + 1];
   __shared__ int total[kMaxExperts];
   __shared__ int item_begin[kMaxExperts + 1];
@@ -315,7 +320,6 @@ __global__ void __launch_bounds__(512) k_route_scan(int T, int E, int nblocks, c
   }
   __syncthreads();
   build_chunks(Ee, item_begin, chunk_a, rt.chunks_a, rt.expert_chunk_begin_a, rt.n_chunks_a, chunk_begin);
-  build_chunks(Ee, item_begin, chunk_b, rt.chunks_b, rt.expert_chunk_begin_b, rt.n_chunks_b, chunk_begin);
 }
 
 // ---------------------------------------------------------------------------
@@ -519,45 +523,53 @@ __global__ void __launch_bounds__(256) k_sum_partials(const float* __restrict__ 
   out[i] = s * (scale_ptr ? scale_ptr[0] : 1.0f);
 }
 
-// out[0] = sum_i v[i]  (scalar feature scales), one block, fixed tree
-__global__ void __launch_bounds__(1024) k_sum_to_scalar(const float* __restrict__ v, int n, float* __restrict__ out) {
-  __shared__ double sh[32];
-  double s = 0.0;
-  for (int i = threadIdx.x; i < n; i += 1024) s += (double)v[i];
-  for (int d = 16; d > 0; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
-  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = s;
-  __syncthreads();
-  if (threadIdx.x < 32) {
-    s = sh[threadIdx.x];
-    for (int d = 16; d > 0; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
-    if (threadIdx.x == 0) out[0] = (float)s;
+// Feature-scale gradients from their per-tile partials, one thread per output feature:
+//   dbeta_n = lam * sum_s dbeta_partial[s, n]      dalpha_n = sum_e dalpha_partial[e, n]   (slots / experts ascending)
+__global__ void __launch_bounds__(128) k_finalize_scales(const float* __restrict__ dbeta_partial, int nslots,
+                                                         const float* __restrict__ dalpha_partial, int E, int N,
+                                                         const float* __restrict__ w_scales, float* __restrict__ dbeta,
+                                                         float* __restrict__ dalpha) {
+  const int n = blockIdx.x * 128 + threadIdx.x;
+  if (n >= N) return;
+  float b = 0.f;
+#pragma unroll 8
+  for (int s = 0; s < nslots; ++s) b += dbeta_partial[(long long)s * N + n];
+  dbeta[n] = b * w_scales[0];
+  if (dalpha_partial) {
+    float a = 0.f;
+#pragma unroll 8
+    for (int e = 0; e < E; ++e) a += dalpha_partial[(long long)e * N + n];
+    dalpha[n] = a;
   }
 }
 
-// dB[e,n,:] = alpha_n * sum over expert e's chunks of the raw partials (ascending chunk order);
-// dalpha partial[e,n] = sum_j B[e,n,j] * that sum.  One warp per (e, n) row.
-__global__ void __launch_bounds__(256) k_reduce_db(const float* __restrict__ partial, RoutingTables rt, const uint16_t* __restrict__ B,
-                                                   const float* __restrict__ alpha, int sstride, int E, int N, int r,
-                                                   float* __restrict__ dB, float* __restrict__ dalpha_partial) {
-  const int row = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
-  if (row >= E * N) return;
-  const int e = row / N, n = row % N;
-  const int c0 = rt.expert_chunk_begin_b[e], c1 = rt.expert_chunk_begin_b[e + 1];
-  const float al = alpha[n * sstride];
-  float part = 0.f;
-  for (int j = lane * 4; j < r; j += 128) {
-    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int c = c0; c < c1; ++c) {
-      const float4 v = *reinterpret_cast<const float4*>(partial + ((long long)c * N + n) * r + j);
-      s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
-    }
-    const uint2 bv = *reinterpret_cast<const uint2*>(B + ((long long)e * N + n) * r + j);
-    part = fmaf(bf16lo(bv.x), s.x, part); part = fmaf(bf16hi(bv.x), s.y, part);
-    part = fmaf(bf16lo(bv.y), s.z, part); part = fmaf(bf16hi(bv.y), s.w, part);
-    *reinterpret_cast<float4*>(dB + ((long long)e * N + n) * r + j) = make_float4(al * s.x, al * s.y, al * s.z, al * s.w);
+// Scalar feature scales: out_b[0] = sum_n vb[n], out_a[0] = sum_n va[n] (va may be null); one block, fp64, fixed tree.
+__global__ void __launch_bounds__(1024) k_sum_scales(const float* __restrict__ vb, const float* __restrict__ va, int N,
+                                                     float* __restrict__ out_b, float* __restrict__ out_a) {
+  __shared__ double sh[2][32];
+  double sb = 0.0, sa = 0.0;
+  for (int n = threadIdx.x; n < N; n += 1024) {
+    sb += (double)vb[n];
+    if (va) sa += (double)va[n];
   }
-  for (int d = 16; d > 0; d >>= 1) part += __shfl_xor_sync(0xffffffffu, part, d);
-  if (lane == 0) dalpha_partial[(long long)e * N + n] = part;
+  for (int d = 16; d > 0; d >>= 1) {
+    sb += __shfl_xor_sync(0xffffffffu, sb, d);
+    sa += __shfl_xor_sync(0xffffffffu, sa, d);
+  }
+  if ((threadIdx.x & 31) == 0) { sh[0][threadIdx.x >> 5] = sb; sh[1][threadIdx.x >> 5] = sa; }
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    sb = sh[0][threadIdx.x];
+    sa = sh[1][threadIdx.x];
+    for (int d = 16; d > 0; d >>= 1) {
+      sb += __shfl_xor_sync(0xffffffffu, sb, d);
+      sa += __shfl_xor_sync(0xffffffffu, sa, d);
+    }
+    if (threadIdx.x == 0) {
+      out_b[0] = (float)sb;
+      if (va) out_a[0] = (float)sa;
+    }
+  }
 }
 
 // dA[e,j,k] = c * sum over expert e's chunks of the raw partials; c as in the dX tile (lam*beta or lam, 1 if that is 0)
@@ -594,7 +606,7 @@ static inline int grid_for(long long work, int per_block, int cap) {
 
 cudaError_t launch_pack(const float* W, int N, int K, uint32_t* bits, int8_t* s8, float* scales, double* partial, cudaStream_t st) {
   const long long n4 = (long long)N * K / 4;
-  const int nparts = grid_for(n4, 256 * 8, kPackPartials);
+  const int nparts = grid_for(n4, 256 * 8, 2 * 148);   // two blocks per SM, each thread keeps four loads in flight
   { LaunchScope ls(KID_PACK_SUMS, st);
   k_weight_partial_sums<<<nparts, 256, 0, st>>>(reinterpret_cast<const float4*>(W), n4, partial); }
   const int grid = grid_for(n4, 256 * 4, 148 * 8);
@@ -613,7 +625,7 @@ cudaError_t launch_route_and_quant(const uint16_t* X, const uint16_t* Wr, int T,
                                       sc.probs_tok, sc.block_counts);
   }
   { LaunchScope ls(KID_ROUTE_SCAN, st);
-  k_route_scan<<<1, 512, 0, st>>>(T, E, nblocks, sc.block_counts, sc.block_base, sv.offsets, sv.rt, sv.chunk_a, sv.chunk_b); }
+  k_route_scan<<<1, 512, 0, st>>>(T, E, nblocks, sc.block_counts, sc.block_base, sv.offsets, sv.rt, sv.chunk_a); }
   LaunchScope ls(KID_ACT_QUANT, st);
   const int per_lane = (K / 8 + 31) / 32;   // 16-byte pieces of a row per lane if one warp took the whole row
   auto kern = k_act_quant<0, 1>;
@@ -667,16 +679,17 @@ cudaError_t launch_sum_partials(const float* partial, int nparts, int n, const f
   return cudaGetLastError();
 }
 
-cudaError_t launch_sum_to_scalar(const float* v, int n, float* out, cudaStream_t st) {
-  LaunchScope ls(KID_SUM_SCALAR, st);
-  k_sum_to_scalar<<<1, 1024, 0, st>>>(v, n, out);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_reduce_db(const float* partial, const RoutingTables& rt, const uint16_t* B, const float* alpha, int sstride, int E, int N,
-                             int r, float* dB, float* dalpha_partial, cudaStream_t st) {
-  LaunchScope ls(KID_REDUCE_DB, st);
-  k_reduce_db<<<(E * N + 7) / 8, 256, 0, st>>>(partial, rt, B, alpha, sstride, E, N, r, dB, dalpha_partial);
+cudaError_t launch_finalize_scales(const float* dbeta_partial, int nslots, const float* dalpha_partial, int E, int N, const float* w_scales,
+                                   int vec, float* dbeta, float* dalpha, float* tmp_b, float* tmp_a, cudaStream_t st) {
+  {
+    LaunchScope ls(KID_SUM_PARTIALS, st);
+    k_finalize_scales<<<(N + 127) / 128, 128, 0, st>>>(dbeta_partial, nslots, dalpha_partial, E, N, w_scales, vec ? dbeta : tmp_b,
+                                                       vec ? dalpha : tmp_a);
+  }
+  if (!vec) {
+    LaunchScope ls(KID_SUM_SCALAR, st);
+    k_sum_scales<<<1, 1024, 0, st>>>(tmp_b, dalpha_partial ? tmp_a : nullptr, N, dbeta, dalpha);
+  }
   return cudaGetLastError();
 }
 

@@ -55,6 +55,8 @@ struct Segment {
   int a_rank, b_rank;       // tensor-map rank (2 or 3)
   int b_box;                // K-major B: rows one TMA load delivers (box height of tb); bn is covered by
                             // ceil(bn / b_box) loads.  Per k-block B always occupies bn * 128 bytes.
+  int b2_y;                 // MN-major B only, -1 = unused: the columns [bn/2, bn) of B come from a second row range of
+                            // tb starting at k row b2_y (same columns b_x), e.g. the second bf16 plane of an operand
   int a_blk, b_blk;         // MN-major operand read through a "blocked" tensor map (64-wide column blocks as an
                             // extra dimension): number of blocks one load delivers; 0 = one 64 x 64 box per load
 };
@@ -188,6 +190,7 @@ __device__ __forceinline__ void gemm_body(const typename P::Params& p) {
         const int nseg = P::num_segments(p, t);
         for (int s = 0; ok && s < nseg; ++s) {
           Segment sg;
+          sg.b2_y = -1;
           P::segment(p, t, s, sg);
           const int a_step = (sg.mode == MODE_I8_KK) ? 128 : 64;
           // both operands of k-block kb into the stage at sa
@@ -204,12 +207,16 @@ __device__ __forceinline__ void gemm_body(const typename P::Params& p) {
               tma_fetch(sa, sg.ta, bar, sg.a_rank, sg.a_x + kb * a_step, sg.a_y, sg.a_z);
             }
             if (b_is_mn(sg.mode)) {
-              if (sg.b_blk) {
-                tma_fetch_blocked(sb, sg.tb, bar, sg.b_rank, sg.b_y + kb * 64, sg.b_x >> 6, sg.b_z);
-              } else {
-                const int nbox = sg.bn / 64;
-                for (int b = 0; b < nbox; ++b)
-                  tma_fetch(sb + b * kMnBoxBytes, sg.tb, bar, sg.b_rank, sg.b_x + 64 * b, sg.b_y + kb * 64, sg.b_z);
+              const int parts = sg.b2_y >= 0 ? 2 : 1;
+              for (int part = 0; part < parts; ++part) {
+                const int krow = (part ? sg.b2_y : sg.b_y) + kb * 64;
+                if (sg.b_blk) {
+                  tma_fetch_blocked(sb + part * sg.b_blk * kMnBoxBytes, sg.tb, bar, sg.b_rank, krow, sg.b_x >> 6, sg.b_z);
+                } else {
+                  const int nbox = sg.bn / (64 * parts);
+                  for (int b = 0; b < nbox; ++b)
+                    tma_fetch(sb + (part * nbox + b) * kMnBoxBytes, sg.tb, bar, sg.b_rank, sg.b_x + 64 * b, krow, sg.b_z);
+                }
               }
             } else {
               for (int row = 0; row < sg.bn; row += sg.b_box)
@@ -221,7 +228,7 @@ __device__ __forceinline__ void gemm_body(const typename P::Params& p) {
             const uint32_t bar = full_bar(st.stage);
             const uint32_t sa = smem_base + st.stage * kStageBytes;
             if (b_is_mn(sg.mode)) {
-              mbar_expect_tx(bar, kStageABytes + (sg.b_blk ? sg.b_blk * kMnBoxBytes : sg.bn * 128));
+              mbar_expect_tx(bar, kStageABytes + (sg.b_blk ? (sg.b2_y >= 0 ? 2 : 1) * sg.b_blk * kMnBoxBytes : sg.bn * 128));
             } else {
               const int nload = (sg.bn + sg.b_box - 1) / sg.b_box;
               mbar_expect_tx(bar, kStageABytes + nload * sg.b_box * 128);
@@ -246,6 +253,7 @@ __device__ __forceinline__ void gemm_body(const typename P::Params& p) {
         uint32_t started[2] = {0u, 0u};
         for (int s = 0; ok && s < nseg; ++s) {
           Segment sg;
+          sg.b2_y = -1;
           P::segment(p, t, s, sg);
           const uint32_t d_tmem = tmem_base + Acc::col(ac.stage, sg.acc);
           const bool amn = a_is_mn(sg.mode), bmn = b_is_mn(sg.mode);

@@ -590,37 +590,93 @@ struct BwdDxProblem {
 PQ_DEFINE_GEMM_KERNEL(k_gemm_bwd_dx, BwdDxProblem)
 
 // ---------------------------------------------------------------------------
-// B3: G = dYs^T . xt (contraction over tokens); dW = beta_n G; per-tile partial
-// of dbeta_n = lam * sum_k S[n,k] G[n,k].
+// B3: the two products that contract dYs^T over tokens, in one launch.
+//   dW tiles: G = dYs^T . xt; dW = beta_n G; per-tile partial of dbeta_n = lam * sum_k S[n,k] G[n,k].
+//   dB tiles (one per expert and 128 output features, after the dW tiles): dBraw_e = dYs^T . (g H) over
+//     the expert's items, the hi and lo planes of g H side by side as the two halves of the tile's
+//     columns; dB = alpha_n dBraw, and the partial of dalpha_n = sum_j B[e,n,j] dBraw[n,j].
 // ---------------------------------------------------------------------------
 struct BwdDwProblem {
   using Acc = AccDouble;
   struct Params {
-    CUtensorMap tdyT, txt;
+    CUtensorMap tdyT, txt, tgh;
+    RoutingTables rt;
     const int8_t* s8;
     const float* beta;
+    const float* alpha;
+    const uint16_t* B;       // [E, N, r]
     float* dW;
-    float* dbeta_partial;
+    float* dB;               // [E, N, r]
+    float* dbeta_partial;    // [2 * ceil(K/256), N]
+    float* dalpha_partial;   // [2 * E, N]
     TileGrid g;
-    int T, N, K, sstride, dy_blk, xt_blk;
+    int T, N, K, r, r64, E, sstride, dy_blk, xt_blk, gh_blk, item_rows, ntn, db_tiles;
   };
-  struct Tile { TileCoord c; int nt, bn; };
-  __device__ static int num_tiles(const Params& p) { return p.g.total; }
+  struct Tile { TileCoord c; int nt, bn, e, ib, ie; };   // e < 0: dW tile
+  __device__ static int num_tiles(const Params& p) { return p.g.total + p.db_tiles; }
   __device__ static void tile_init(const Params& p, int i, Tile& t) {
-    t.c = tile_coord(p.g, i);
-    t.nt = t.c.m;
-    t.bn = clip_bn(t.c.bn, t.c.n0, p.K, 64);
+    if (i < p.g.total) {
+      t.c = tile_coord(p.g, i);
+      t.nt = t.c.m; t.e = -1; t.ib = t.ie = 0;
+      t.bn = clip_bn(t.c.bn, t.c.n0, p.K, 64);
+    } else {
+      const int j = i - p.g.total;
+      t.e = j / p.ntn; t.nt = j % p.ntn;
+      t.ib = p.rt.expert_item_begin[t.e]; t.ie = p.rt.expert_item_begin[t.e + 1];
+      t.bn = 2 * p.r64;
+      t.c.m = t.nt; t.c.n0 = 0; t.c.bn = t.bn;
+    }
   }
-  __device__ static int num_segments(const Params&, const Tile&) { return 1; }
-  __device__ static void segment(const Params& p, const Tile& t, int, Segment& s) {
-    s.mode = MODE_BF_MM; s.acc = 0; s.bn = t.bn; s.ksteps = 4; s.nkb = (p.T + 63) / 64;
-    s.ta = &p.tdyT; s.a_rank = 2; s.a_x = t.nt * 128; s.a_y = 0; s.a_z = 0;
-    s.tb = &p.txt; s.b_rank = 2; s.b_x = t.c.n0; s.b_y = 0; s.b_z = 0;
-    s.b_box = 0; s.a_blk = p.dy_blk; s.b_blk = p.xt_blk;
+  __device__ static int num_segments(const Params&, const Tile& t) { return t.e < 0 ? 1 : t.ie - t.ib; }
+  __device__ static void segment(const Params& p, const Tile& t, int i, Segment& s) {
+    s.mode = MODE_BF_MM; s.acc = 0; s.bn = t.bn; s.ksteps = 4; s.b_box = 0;
+    s.ta = &p.tdyT; s.a_rank = 2; s.a_x = t.nt * 128; s.a_z = 0; s.a_blk = p.dy_blk;
+    s.b_rank = 2; s.b_z = 0;
+    if (t.e < 0) {
+      s.nkb = (p.T + 63) / 64; s.a_y = 0;
+      s.tb = &p.txt; s.b_x = t.c.n0; s.b_y = 0; s.b_blk = p.xt_blk;
+    } else {
+      const int item = t.ib + i;
+      s.nkb = 2; s.a_y = p.rt.items[item].x * 128;      // the 128 tokens of the item's tile (rows outside the item are zero in g H)
+      s.tb = &p.tgh; s.b_x = 0; s.b_y = item * 128; s.b2_y = p.item_rows + item * 128; s.b_blk = p.gh_blk;
+    }
   }
   __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, uint32_t, int quad, int half, int lane, uint8_t* stage) {
     const int n = t.nt * 128 + quad * 32 + lane;
     const bool live = n < p.N;
+    if (t.e >= 0) {
+      // ---- dB tile: columns [0, r64) hold the hi-plane product, [r64, 2 r64) the lo-plane product
+      const bool any = t.ie > t.ib;                     // an expert without tokens: exact zeros
+      const float al = live ? p.alpha[n * p.sstride] : 0.f;
+      const long long row = ((long long)t.e * p.N + (live ? n : 0)) * p.r;
+      float part = 0.f;
+      for (int c32 = half; c32 * 32 < p.r; c32 += 2) {
+        uint32_t vh[32], vl[32];
+        if (any) {
+          tmem_ld32(taddr + c32 * 32, vh);
+          tmem_ld32(taddr + p.r64 + c32 * 32, vl);
+          tmem_ld_wait();
+        }
+        uint4 o[8];
+#pragma unroll
+        for (int q4 = 0; q4 < 8; ++q4) {
+          float gsum[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) gsum[u] = any ? __uint_as_float(vh[4 * q4 + u]) + __uint_as_float(vl[4 * q4 + u]) : 0.f;
+          const int j = c32 * 32 + q4 * 4;
+          if (live && j < p.r) {
+            const uint2 bv = *reinterpret_cast<const uint2*>(p.B + row + j);
+            part = fmaf(bf16lo(bv.x), gsum[0], part); part = fmaf(bf16hi(bv.x), gsum[1], part);
+            part = fmaf(bf16lo(bv.y), gsum[2], part); part = fmaf(bf16hi(bv.y), gsum[3], part);
+          }
+          o[q4] = make_uint4(__float_as_uint(al * gsum[0]), __float_as_uint(al * gsum[1]), __float_as_uint(al * gsum[2]),
+                             __float_as_uint(al * gsum[3]));
+        }
+        warp_store_rows(stage, o, live ? p.dB + row + c32 * 32 : nullptr, min(32, p.r - c32 * 32) * 4, lane);
+      }
+      if (live) p.dalpha_partial[(long long)(2 * t.e + half) * p.N + n] = part;
+      return;
+    }
     const float be = live ? p.beta[n * p.sstride] : 0.f;
     float* wrow = live ? p.dW + (long long)n * p.K : nullptr;
     const uint4* srow = reinterpret_cast<const uint4*>(p.s8 + (long long)(live ? n : 0) * p.K);
@@ -650,60 +706,11 @@ struct BwdDwProblem {
       }
       warp_store_rows(stage, o, wrow ? wrow + k0 : nullptr, 128, lane);
     }
-    if (live) {
-      // one slot per 32 columns of K; each of the two warps of a row fills its first slot and clears its others
-      const int slot = t.c.n0 / 32 + half;
-      p.dbeta_partial[(long long)slot * p.N + n] = part;
-      for (int j = 2; (half + j) * 32 < t.bn; j += 2) p.dbeta_partial[(long long)(slot + j) * p.N + n] = 0.f;
-    }
+    // one slot per (column tile, warp of the row pair)
+    if (live) p.dbeta_partial[(long long)(2 * (t.c.n0 / 256) + half) * p.N + n] = part;
   }
 };
 PQ_DEFINE_GEMM_KERNEL(k_gemm_bwd_dw, BwdDwProblem)
-
-// ---------------------------------------------------------------------------
-// B4: raw dB partials.  The token contraction of dBraw_e = dYs^T . (g H) is split
-// into chunks of expert e's items so that enough CTAs work on it; each tile
-// (chunk, 128 output features) writes its fp32 partial, and k_reduce_db sums a
-// expert's chunks in a fixed order, scales by alpha_n and forms the dalpha partials.
-// ---------------------------------------------------------------------------
-struct HpDbProblem {
-  using Acc = AccDouble;
-  struct Params {
-    CUtensorMap tdyT, tgh;
-    RoutingTables rt;
-    float* partial;  // [chunks, N, r]
-    int N, r, bn, ntn, item_rows, dy_blk, gh_blk;
-  };
-  struct Tile { int nt, chunk, ib, ie; };
-  __device__ static int num_tiles(const Params& p) { return p.ntn * p.rt.n_chunks_b[0]; }
-  __device__ static void tile_init(const Params& p, int i, Tile& t) {
-    t.chunk = i / p.ntn; t.nt = i % p.ntn;
-    const int4 c = p.rt.chunks_b[t.chunk];
-    t.ib = c.y; t.ie = c.z;
-  }
-  __device__ static int num_segments(const Params&, const Tile& t) { return 2 * (t.ie - t.ib); }
-  __device__ static void segment(const Params& p, const Tile& t, int i, Segment& s) {
-    const int item = t.ib + (i >> 1), plane = i & 1;
-    s.mode = MODE_BF_MM; s.acc = 0; s.bn = p.bn; s.ksteps = 4; s.nkb = 2;
-    s.ta = &p.tdyT; s.a_rank = 2; s.a_x = t.nt * 128; s.a_y = p.rt.items[item].x * 128; s.a_z = 0;
-    s.tb = &p.tgh; s.b_rank = 2; s.b_x = 0; s.b_y = plane * p.item_rows + item * 128; s.b_z = 0;
-    s.b_box = 0; s.a_blk = p.dy_blk; s.b_blk = p.gh_blk;
-  }
-  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, uint32_t, int quad, int half, int lane, uint8_t* stage) {
-    const int n = t.nt * 128 + quad * 32 + lane;
-    float* out = n < p.N ? p.partial + ((long long)t.chunk * p.N + n) * p.r : nullptr;
-    for (int c32 = half; c32 * 32 < p.r; c32 += 2) {
-      uint32_t v[32];
-      tmem_ld32(taddr + c32 * 32, v);
-      tmem_ld_wait();
-      uint4 o[8];
-#pragma unroll
-      for (int j = 0; j < 8; ++j) o[j] = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-      warp_store_rows(stage, o, out ? out + c32 * 32 : nullptr, min(32, p.r - c32 * 32) * 4, lane);
-    }
-  }
-};
-PQ_DEFINE_GEMM_KERNEL(k_gemm_hp_db, HpDbProblem)
 
 // ---------------------------------------------------------------------------
 // B5: raw dA partials, dhc^T . Xs over one chunk of an expert's items; summed and
@@ -791,21 +798,17 @@ int gemm_backward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, c
     BwdDwProblem::Params p;
     if (!map_mn(&p.tdyT, &p.dy_blk, b.dys, a.N, a.T, 2, 1, 2)) return PQ_ERR_CUDA;
     if (!map_mn(&p.txt, &p.xt_blk, sv.xt, a.K, a.T, 2, 1, 4)) return PQ_ERR_CUDA;
-    p.s8 = w_s8; p.beta = a.beta; p.dW = dW; p.dbeta_partial = b.dbeta_partial;
-    p.T = a.T; p.N = a.N; p.K = a.K; p.sstride = a.scale_stride;
+    p.tgh = p.txt; p.gh_blk = 0;
+    if (hp && !map_mn(&p.tgh, &p.gh_blk, b.gh, a.r, 2 * item_rows, 2, 1, r64 / 64)) return PQ_ERR_CUDA;
+    p.rt = sv.rt; p.s8 = w_s8; p.beta = a.beta; p.alpha = a.alpha; p.B = a.B; p.dW = dW; p.dB = dB;
+    p.dbeta_partial = b.dbeta_partial; p.dalpha_partial = b.dalpha_partial;
+    p.T = a.T; p.N = a.N; p.K = a.K; p.r = a.r; p.r64 = r64; p.E = a.E; p.sstride = a.scale_stride; p.item_rows = (int)item_rows;
+    p.ntn = ntn128; p.db_tiles = hp ? a.E * ntn128 : 0;
     p.g = make_tile_grid(ntn128, ntk, 256);
-    rc = launch_gemm(KID_BWD_DW, k_gemm_bwd_dw, p, p.g.total, st);
+    rc = launch_gemm(KID_BWD_DW, k_gemm_bwd_dw, p, p.g.total + p.db_tiles, st);
     if (rc) return rc;
   }
   if (hp) {
-    HpDbProblem::Params p;
-    if (!map_mn(&p.tdyT, &p.dy_blk, b.dys, a.N, a.T, 2, 1, 2)) return PQ_ERR_CUDA;
-    if (!map_mn(&p.tgh, &p.gh_blk, b.gh, a.r, 2 * item_rows, 2, 1, r64 / 64)) return PQ_ERR_CUDA;
-    p.rt = sv.rt; p.partial = b.db_partial; p.N = a.N; p.r = a.r; p.bn = r64; p.ntn = ntn128; p.item_rows = (int)item_rows;
-    rc = launch_gemm(KID_HP_DB, k_gemm_hp_db, p, ntn128 * sv.max_chunks_b, st);
-    if (rc) return rc;
-    if (launch_reduce_db(b.db_partial, sv.rt, a.B, a.alpha, a.scale_stride, a.E, a.N, a.r, dB, b.dalpha_partial, st) != cudaSuccess)
-      return PQ_ERR_CUDA;
     HpDaProblem::Params q;
     if (!map_mn(&q.tdhT, &q.dh_blk, b.dhc, a.r, 2 * item_rows, 2, 1, 2)) return PQ_ERR_CUDA;
     if (!map_mn(&q.txs, &q.xs_blk, b.xs, a.K, a.T, 2, 1, 4)) return PQ_ERR_CUDA;

@@ -38,13 +38,10 @@ struct RoutingTables {
   int4* items;             // [max_items] {tile, expert, first row, end row}
   int* tile_item_begin;    // [mtiles + 1]
   int* expert_item_begin;  // [E + 1]
-  // chunk tables {expert, first item, end item, 0}: table a splits dA, table b splits dB
+  // chunk table {expert, first item, end item, 0}: the units the token contraction of dA is split into
   int* n_chunks_a;         // [1]
   int4* chunks_a;          // [max_items + E]
   int* expert_chunk_begin_a;  // [E + 1]
-  int* n_chunks_b;
-  int4* chunks_b;
-  int* expert_chunk_begin_b;
 };
 
 // Device pointers into the caller's `saved` buffer.
@@ -62,8 +59,8 @@ struct SavedPtrs {
   uint16_t* h;
   RoutingTables rt;
   int max_items;
-  int chunk_a, chunk_b;      // items per chunk of the two tables
-  int max_chunks_a, max_chunks_b;
+  int chunk_a;               // items per chunk
+  int max_chunks_a;
 };
 
 struct FwdScratch {
@@ -83,10 +80,9 @@ cudaError_t launch_scaled_b(const uint16_t* B, uint16_t* out, const float* alpha
 cudaError_t launch_router_wgrad(const uint16_t* xs, const float* dl, int T, int K, int E, float* partial, float* dWr, const float* scale,
                                 cudaStream_t st);
 cudaError_t launch_sum_partials(const float* partial, int nparts, int n, const float* scale, float* out, cudaStream_t st);
-cudaError_t launch_sum_to_scalar(const float* v, int n, float* out, cudaStream_t st);
+cudaError_t launch_finalize_scales(const float* dbeta_partial, int nslots, const float* dalpha_partial, int E, int N, const float* w_scales,
+                                   int vec, float* dbeta, float* dalpha, float* tmp_b, float* tmp_a, cudaStream_t st);
 cudaError_t launch_fill_zero(void* p, size_t bytes, cudaStream_t st);
-cudaError_t launch_reduce_db(const float* partial, const RoutingTables& rt, const uint16_t* B, const float* alpha, int sstride, int E, int N,
-                             int r, float* dB, float* dalpha_partial, cudaStream_t st);
 cudaError_t launch_reduce_da(const float* partial, const RoutingTables& rt, const float* w_scales, const float* beta, int sstride, int E, int r,
                              int K, float* dA, cudaStream_t st);
 
@@ -121,10 +117,9 @@ struct BwdBuffers {
   uint16_t* gh;          // [2][items*128, r] bf16 hi/lo planes of g * H
   float* dl;             // [T,E] fp32 router logit gradient (sorted order)
   uint16_t* dlc;         // [T,16] bf16 dl / c
-  float* dbeta_partial;  // [ceil(K/32), N]
-  float* dalpha_partial; // [E, N]
+  float* dbeta_partial;  // [2 * ceil(K/256), N]
+  float* dalpha_partial; // [2 * E, N]
   float* da_partial;     // [max_chunks_a, r, K] raw split-contraction partials of dA
-  float* db_partial;     // [max_chunks_b, N, r]
 };
 int gemm_backward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, const BwdBuffers& b, uint16_t* dX, float* dW, float* dA,
                   float* dB, cudaStream_t st);
