@@ -30,9 +30,10 @@ import numpy as np
 
 METRIC = "pQuant linear fwd+bwd tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the
-# committed ncu capture (profiles/); None until a capture of this kernel exists.
-NCU_TRAFFIC_BYTES = {"bwd_dw": None}
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel (the 2048 -> 5632
+# projection) from the committed ncu capture (profiles/gemm_kernels_up_projection_ncu.md); set to None
+# whenever the kernel changes until it is captured again.
+NCU_TRAFFIC_BYTES = {"bwd_dw": 324611072}
 
 
 def measured_peaks():
