@@ -130,6 +130,9 @@ __device__ __forceinline__ void warp_store_rows(uint8_t* stage, const uint4 (&v)
   __syncwarp();
 }
 
+// Problems whose epilogue needs nothing fetched ahead of the accumulator
+struct NoPre {};
+
 // Accumulator layouts in TMEM (column of accumulator `acc` of pipeline stage `stage`).
 //   AccDouble     : one accumulator per tile, two stages of 256 columns.
 //   AccPair       : two accumulators of 256 columns per tile (all of TMEM), one stage: the epilogue of
@@ -288,10 +291,12 @@ __device__ __forceinline__ void gemm_body(const typename P::Params& p) {
     for (int tile = blockIdx.x; ok && tile < ntiles; tile += gridDim.x) {
       typename P::Tile t;
       P::tile_init(p, tile, t);
+      // per-row factors and addresses are fetched while the contraction is still running
+      const typename P::Pre pre = P::prepare(p, t, quad, lane);
       if (!pipe_wait(tfull_bar(ac.stage), ac.phase, WHERE_EPILOGUE, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const uint32_t tlane = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
-      P::epilogue(p, t, tlane + Acc::col(ac.stage, 0), tlane + Acc::col(ac.stage, 1), quad, half, lane, epi_stage + (warp - 2) * kEpiWarpBytes);
+      P::epilogue(p, t, pre, tlane + Acc::col(ac.stage, 0), tlane + Acc::col(ac.stage, 1), quad, half, lane, epi_stage + (warp - 2) * kEpiWarpBytes);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(ac.stage));

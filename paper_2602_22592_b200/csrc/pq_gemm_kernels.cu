@@ -153,7 +153,9 @@ struct DebugProblem {
     if (p.mode == MODE_BF_MM) { s.a_x = t.c.m * 128; s.a_y = 0; } else { s.a_x = 0; s.a_y = t.c.m * 128; }
     if (p.mode >= MODE_BF_KM) { s.b_x = t.c.n0; s.b_y = 0; } else { s.b_x = 0; s.b_y = t.c.n0; }
   }
-  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t tacc, uint32_t, int quad, int half, int lane, uint8_t* stage) {
+  using Pre = NoPre;
+  __device__ static Pre prepare(const Params&, const Tile&, int, int) { return Pre{}; }
+  __device__ static void epilogue(const Params& p, const Tile& t, const Pre& pre, uint32_t tacc, uint32_t, int quad, int half, int lane, uint8_t* stage) {
     const int row = t.c.m * 128 + quad * 32 + lane;
     uint32_t* D = reinterpret_cast<uint32_t*>(p.D);
     for (int c = half; c * 32 < t.c.bn; c += 2) {
@@ -222,7 +224,9 @@ struct HpUpProblem {
     s.tb = &p.ta; s.b_rank = 3; s.b_x = 0; s.b_y = 0; s.b_z = t.it.y;
     s.b_box = p.bn; s.a_blk = 0; s.b_blk = 0;
   }
-  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, uint32_t, int quad, int half, int lane, uint8_t* stage) {
+  using Pre = NoPre;
+  __device__ static Pre prepare(const Params&, const Tile&, int, int) { return Pre{}; }
+  __device__ static void epilogue(const Params& p, const Tile& t, const Pre& pre, uint32_t taddr, uint32_t, int quad, int half, int lane, uint8_t* stage) {
     const int row = quad * 32 + lane;
     const bool live = row >= t.it.z && row < t.it.w;
     uint4* out_hi = reinterpret_cast<uint4*>(p.H + ((long long)t.item * 128 + row) * p.r);
@@ -323,16 +327,22 @@ struct FwdProblem {
 #pragma unroll
     for (int j = 0; j < 4; ++j) out[j] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
   }
-  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t tacc, uint32_t tz, int quad, int half, int lane, uint8_t* stage) {
+  // per-row factors: 1-bit branch lam / gamma_t (Eq. 10), HP branch g_t; scalar feature scales folded in
+  struct Pre { uint16_t* yrow; float cb, ca; };
+  __device__ static Pre prepare(const Params& p, const Tile& t, int quad, int lane) {
     const int pos = t.c.m * 128 + quad * 32 + lane;
-    const bool live = pos < p.T;
-    const int token = live ? (p.perm ? p.perm[pos] : pos) : 0;
-    // per-row factors: 1-bit branch lam / gamma_t (Eq. 10), HP branch g_t; scalar feature scales folded in
-    float cb = live ? __fdiv_rn(p.w_scales[0], p.gamma[pos]) : 0.f;
-    float ca = (HP && live) ? p.gate[pos] : 0.f;
+    Pre r{nullptr, 0.f, 0.f};
+    if (pos < p.T) {
+      const int token = p.perm ? p.perm[pos] : pos;
+      r.yrow = p.Y + (long long)token * p.N;
+      r.cb = __fdiv_rn(p.w_scales[0], p.gamma[pos]);
+      if (HP) r.ca = p.gate[pos];
+      if (!p.sstride) { r.cb *= p.beta[0]; if (HP) r.ca *= p.alpha[0]; }
+    }
+    return r;
+  }
+  __device__ static void epilogue(const Params& p, const Tile& t, const Pre& pre, uint32_t tacc, uint32_t tz, int quad, int half, int lane, uint8_t* stage) {
     const bool vec = p.sstride != 0;
-    if (!vec) { cb *= p.beta[0]; if (HP) ca *= p.alpha[0]; }
-    uint16_t* yrow = live ? p.Y + (long long)token * p.N : nullptr;
     for (int c = half; c * 64 < t.bn; c += 2) {     // 64 output columns = 128 bytes of the row per pass
       const int n0 = t.c.n0 + c * 64;
       if (n0 >= p.N) break;
@@ -345,11 +355,11 @@ struct FwdProblem {
           tmem_ld32(tacc + c * 64 + h * 32, a);
           if (HP) tmem_ld32(tz + c * 64 + h * 32, z);
           tmem_ld_wait();
-          if (vec) combine32<true>(p, nb, cb, ca, a, z, o + 4 * h);
-          else combine32<false>(p, nb, cb, ca, a, z, o + 4 * h);
+          if (vec) combine32<true>(p, nb, pre.cb, pre.ca, a, z, o + 4 * h);
+          else combine32<false>(p, nb, pre.cb, pre.ca, a, z, o + 4 * h);
         }
       }
-      warp_store_rows(stage, o, yrow ? yrow + n0 : nullptr, min(64, min(t.bn - c * 64, p.N - n0)) * 2, lane);
+      warp_store_rows(stage, o, pre.yrow ? pre.yrow + n0 : nullptr, min(64, min(t.bn - c * 64, p.N - n0)) * 2, lane);
     }
   }
 };
@@ -440,7 +450,9 @@ struct HpDhProblem {
     s.tb = &p.tba; s.b_rank = 3; s.b_x = 0; s.b_y = 0; s.b_z = t.it.y;
     s.b_box = 0;
   }
-  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, uint32_t, int quad, int half, int lane, uint8_t* stage) {
+  using Pre = NoPre;
+  __device__ static Pre prepare(const Params&, const Tile&, int, int) { return Pre{}; }
+  __device__ static void epilogue(const Params& p, const Tile& t, const Pre& pre, uint32_t taddr, uint32_t, int quad, int half, int lane, uint8_t* stage) {
     if (half) return;   // each row's sum over all r columns stays in one thread
     const int row = quad * 32 + lane;
     const bool live = row >= t.it.z && row < t.it.w;
@@ -559,31 +571,34 @@ struct BwdDxProblem {
     s.ta = &p.tdl; s.a_y = t.m * 128;
     s.tb = &p.twr; s.b_rank = 2; s.b_blk = p.wr_blk;
   }
-  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, uint32_t, int quad, int half, int lane, uint8_t* stage) {
+  struct Pre { uint16_t* xrow; float cc; };
+  __device__ static Pre prepare(const Params& p, const Tile& t, int quad, int lane) {
     const int pos = t.m * 128 + quad * 32 + lane;
-    const bool live = pos < p.T;
-    const int token = live ? (p.perm ? p.perm[pos] : pos) : 0;
     const float c = dx_scale(p.w_scales, p.beta, p.sstride);
-    const float cc = c != 0.f ? c : 1.0f;
+    Pre r{nullptr, c != 0.f ? c : 1.0f};
+    if (pos < p.T) r.xrow = p.dX + (long long)(p.perm ? p.perm[pos] : pos) * p.K;
+    return r;
+  }
+  __device__ static void epilogue(const Params& p, const Tile& t, const Pre& pre, uint32_t taddr, uint32_t, int quad, int half, int lane, uint8_t* stage) {
+    const float cc = pre.cc;
     const bool has = num_segments(p, t) > 0;
-    uint16_t* xrow = live ? p.dX + (long long)token * p.K : nullptr;
     for (int c64 = half; c64 * 64 < t.bn; c64 += 2) {
       const int k0 = t.c.n0 + c64 * 64;
       if (k0 >= p.K) break;
+      uint32_t v0[32], v1[32];
+      tmem_ld32(taddr + c64 * 64, v0);
+      tmem_ld32(taddr + c64 * 64 + 32, v1);
+      tmem_ld_wait();
       uint4 o[8];
+      uint32_t w[32];
 #pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        uint32_t v[32];
-        tmem_ld32(taddr + c64 * 64 + h * 32, v);
-        tmem_ld_wait();
-        uint32_t w[16];
-#pragma unroll
-        for (int j = 0; j < 16; ++j)
-          w[j] = has ? pack_bf16x2(cc * __uint_as_float(v[2 * j]), cc * __uint_as_float(v[2 * j + 1])) : 0u;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) o[4 * h + j] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+      for (int j = 0; j < 16; ++j) {
+        w[j] = has ? pack_bf16x2(cc * __uint_as_float(v0[2 * j]), cc * __uint_as_float(v0[2 * j + 1])) : 0u;
+        w[16 + j] = has ? pack_bf16x2(cc * __uint_as_float(v1[2 * j]), cc * __uint_as_float(v1[2 * j + 1])) : 0u;
       }
-      warp_store_rows(stage, o, xrow ? xrow + k0 : nullptr, min(64, p.K - k0) * 2, lane);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) o[j] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+      warp_store_rows(stage, o, pre.xrow ? pre.xrow + k0 : nullptr, min(64, p.K - k0) * 2, lane);
     }
   }
 };
@@ -641,7 +656,9 @@ struct BwdDwProblem {
       s.tb = &p.tgh; s.b_x = 0; s.b_y = item * 128; s.b2_y = p.item_rows + item * 128; s.b_blk = p.gh_blk;
     }
   }
-  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, uint32_t, int quad, int half, int lane, uint8_t* stage) {
+  using Pre = NoPre;
+  __device__ static Pre prepare(const Params&, const Tile&, int, int) { return Pre{}; }
+  __device__ static void epilogue(const Params& p, const Tile& t, const Pre& pre, uint32_t taddr, uint32_t, int quad, int half, int lane, uint8_t* stage) {
     const int n = t.nt * 128 + quad * 32 + lane;
     const bool live = n < p.N;
     if (t.e >= 0) {
@@ -739,7 +756,9 @@ struct HpDaProblem {
     s.tb = &p.txs; s.b_rank = 2; s.b_x = t.kt * 256; s.b_y = p.rt.items[item].x * 128; s.b_z = 0;
     s.b_box = 0; s.a_blk = p.dh_blk; s.b_blk = p.xs_blk;
   }
-  __device__ static void epilogue(const Params& p, const Tile& t, uint32_t taddr, uint32_t, int quad, int half, int lane, uint8_t* stage) {
+  using Pre = NoPre;
+  __device__ static Pre prepare(const Params&, const Tile&, int, int) { return Pre{}; }
+  __device__ static void epilogue(const Params& p, const Tile& t, const Pre& pre, uint32_t taddr, uint32_t, int quad, int half, int lane, uint8_t* stage) {
     const int j = quad * 32 + lane;
     float* out = j < p.r ? p.partial + ((long long)t.chunk * p.r + j) * p.K : nullptr;
     for (int c32 = half; c32 < 8; c32 += 2) {
