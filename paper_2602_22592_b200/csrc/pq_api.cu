@@ -100,7 +100,6 @@ struct BwdScratch {
   uint16_t* dlc;
   float* dbeta_partial;
   float* dalpha_partial;
-  float* dwr_partial;
   float* dalpha_vec;
   float* dbeta_vec;
   float* da_partial;
@@ -121,7 +120,6 @@ static size_t carve_bwd_scratch(const pq_desc* d, void* base, BwdScratch* out) {
   s.dlc = routed(d) ? c.take<uint16_t>(T * 16) : nullptr;
   s.dbeta_partial = c.take<float>(2 * ((K + 255) / 256) * N);   // two slots per 256-column tile of K
   s.dalpha_partial = r > 0 ? c.take<float>((size_t)2 * E * N) : nullptr;
-  s.dwr_partial = routed(d) ? c.take<float>(((T + 255) / 256) * E * K) : nullptr;
   s.dalpha_vec = c.take<float>(N);
   s.dbeta_vec = c.take<float>(N);
   s.da_partial = r > 0 ? c.take<float>((size_t)max_chunks(d, chunk_a_of(d)) * r * K) : nullptr;
@@ -377,12 +375,9 @@ int pq_linear_backward(const pq_desc* d, const uint16_t* dY, const uint16_t* X, 
   b.dhc = sc.dhc; b.gh = sc.gh; b.dl = sc.dl; b.dlc = sc.dlc;
   b.dbeta_partial = sc.dbeta_partial; b.dalpha_partial = sc.dalpha_partial;
   b.da_partial = sc.da_partial;
-  rc = gemm_backward(a, w_s8, sv, b, dX, dW, dA, dB, st);
+  rc = gemm_backward(a, w_s8, sv, b, dX, dW, dA, dB, dWr, st);
   if (rc) return rc;
 
-  if (routed(d)) {
-    if (launch_router_wgrad(sv.xs, sc.dl, d->T, d->K, E, sc.dwr_partial, dWr, nullptr, st) != cudaSuccess) return PQ_ERR_CUDA;
-  }
   // dbeta_n = lam * sum over the column tiles of the partial sign-weighted row sums, dalpha_n = sum over experts
   // of the dB-weighted row sums; the scalar form sums over n as well
   if (dalpha && !hp && cudaMemsetAsync(dalpha, 0, sizeof(float) * (vec ? d->N : 1), st) != cudaSuccess) return PQ_ERR_CUDA;

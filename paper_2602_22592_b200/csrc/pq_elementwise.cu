@@ -120,23 +120,21 @@ __global__ void __launch_bounds__(256) k_binarize_pack(const float4* __restrict_
 // Softmax in fp32; ties go to the lowest index.  Also counts tokens per
 // expert for each block of kRouterTokensPerBlock consecutive tokens.
 // ---------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) k_router(const uint4* __restrict__ X, const uint4* __restrict__ Wr, int T, int K, int E,
-                                                int* __restrict__ expert, float* __restrict__ gate_tok,
-                                                float* __restrict__ probs_tok, int* __restrict__ block_counts) {
+__global__ void __launch_bounds__(1024) k_router(const uint4* __restrict__ X, const uint4* __restrict__ Wr, int T, int K, int E,
+                                                 int* __restrict__ expert, float* __restrict__ gate_tok,
+                                                 float* __restrict__ probs_tok, int* __restrict__ block_counts) {
   __shared__ int cnt[kMaxExperts];
   if (threadIdx.x < kMaxExperts) cnt[threadIdx.x] = 0;
   __syncthreads();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int chunks = K >> 3;
-  for (int it = 0; it < kRouterTokensPerBlock / 8; ++it) {
-    const int t = blockIdx.x * kRouterTokensPerBlock + it * 8 + warp;
-    if (t >= T) break;
+  const int t = blockIdx.x * kRouterTokensPerBlock + warp;   // one warp per token
+  if (t < T) {
     float acc[kMaxExperts];
 #pragma unroll
     for (int e = 0; e < kMaxExperts; ++e) acc[e] = 0.f;
     const uint4* xrow = X + (long long)t * chunks;
-    for (int c = lane; c < chunks; c += 32) {
-      const uint4 xv = __ldg(xrow + c);
+    auto fold = [&](const uint4& xv, int c) {
       const float x0 = bf16lo(xv.x), x1 = bf16hi(xv.x), x2 = bf16lo(xv.y), x3 = bf16hi(xv.y);
       const float x4 = bf16lo(xv.z), x5 = bf16hi(xv.z), x6 = bf16lo(xv.w), x7 = bf16hi(xv.w);
 #pragma unroll
@@ -151,7 +149,15 @@ __global__ void __launch_bounds__(256) k_router(const uint4* __restrict__ X, con
           acc[e] = a;
         }
       }
+    };
+    // the token's chunks in ascending order, two loads of X in flight (the 32 warps of the block hide the rest)
+    int c = lane;
+    for (; c + 32 < chunks; c += 64) {
+      const uint4 xa = __ldg(xrow + c), xb = __ldg(xrow + c + 32);
+      fold(xa, c);
+      fold(xb, c + 32);
     }
+    if (c < chunks) fold(__ldg(xrow + c), c);
 #pragma unroll
     for (int e = 0; e < kMaxExperts; ++e) {
       if (e < E) {
@@ -475,54 +481,6 @@ __global__ void __launch_bounds__(256) k_scaled_b(const uint32_t* __restrict__ B
   }
 }
 
-// ---------------------------------------------------------------------------
-// Router weight gradient dWr[e,k] = sum_p dl[p,e] * x[p,k]  (Sec. 3.3, "trained
-// end-to-end").  CUDA cores: E <= 16 outputs per k.  Partial sums per chunk of
-// 256 tokens, reduced afterwards in a fixed order.
-// ---------------------------------------------------------------------------
-__global__ void __launch_bounds__(128) k_router_wgrad_partial(const uint32_t* __restrict__ xs2, const float* __restrict__ dl, int T, int K, int E,
-                                                              float* __restrict__ partial) {
-  __shared__ float sdl[256 * kMaxExperts];
-  const int t0 = blockIdx.y * 256, nt = min(256, T - t0);
-  for (int i = threadIdx.x; i < nt * E; i += 128) sdl[i] = dl[(long long)t0 * E + i];
-  __syncthreads();
-  const int k2 = blockIdx.x * 128 + threadIdx.x;  // pair of k
-  if (2 * k2 >= K) return;
-  float a0[kMaxExperts], a1[kMaxExperts];
-#pragma unroll
-  for (int e = 0; e < kMaxExperts; ++e) { a0[e] = 0.f; a1[e] = 0.f; }
-  for (int t = 0; t < nt; ++t) {
-    const uint32_t v = __ldg(xs2 + (long long)(t0 + t) * (K / 2) + k2);
-    const float x0 = bf16lo(v), x1 = bf16hi(v);
-#pragma unroll
-    for (int e = 0; e < kMaxExperts; ++e) {
-      if (e < E) {
-        const float d = sdl[t * E + e];
-        a0[e] = fmaf(d, x0, a0[e]);
-        a1[e] = fmaf(d, x1, a1[e]);
-      }
-    }
-  }
-#pragma unroll
-  for (int e = 0; e < kMaxExperts; ++e) {
-    if (e < E) {
-      float* o = partial + ((long long)blockIdx.y * E + e) * K + 2 * k2;
-      o[0] = a0[e];
-      o[1] = a1[e];
-    }
-  }
-}
-
-// out[i] = scale * sum_c partial[c * n + i], c ascending
-__global__ void __launch_bounds__(256) k_sum_partials(const float* __restrict__ partial, int nparts, int n, const float* __restrict__ scale_ptr,
-                                                      float* __restrict__ out) {
-  const int i = blockIdx.x * 256 + threadIdx.x;
-  if (i >= n) return;
-  float s = 0.f;
-  for (int c = 0; c < nparts; ++c) s += partial[(long long)c * n + i];
-  out[i] = s * (scale_ptr ? scale_ptr[0] : 1.0f);
-}
-
 // Feature-scale gradients from their per-tile partials, one thread per output feature:
 //   dbeta_n = lam * sum_s dbeta_partial[s, n]      dalpha_n = sum_e dalpha_partial[e, n]   (slots / experts ascending)
 __global__ void __launch_bounds__(128) k_finalize_scales(const float* __restrict__ dbeta_partial, int nslots,
@@ -621,7 +579,7 @@ cudaError_t launch_route_and_quant(const uint16_t* X, const uint16_t* Wr, int T,
   const int nblocks = (T + kRouterTokensPerBlock - 1) / kRouterTokensPerBlock;
   if (E > 1) {
     LaunchScope ls(KID_ROUTER, st);
-    k_router<<<nblocks, 256, 0, st>>>(reinterpret_cast<const uint4*>(X), reinterpret_cast<const uint4*>(Wr), T, K, E, sv.expert, sc.gate_tok,
+    k_router<<<nblocks, 32 * kRouterTokensPerBlock, 0, st>>>(reinterpret_cast<const uint4*>(X), reinterpret_cast<const uint4*>(Wr), T, K, E, sv.expert, sc.gate_tok,
                                       sc.probs_tok, sc.block_counts);
   }
   { LaunchScope ls(KID_ROUTE_SCAN, st);
@@ -659,23 +617,6 @@ cudaError_t launch_scaled_b(const uint16_t* B, uint16_t* out, const float* alpha
   const long long n2 = (long long)E * N * r / 2;
   LaunchScope ls(KID_SCALED_B, st);
   k_scaled_b<<<grid_for(n2, 256 * 4, 148 * 8), 256, 0, st>>>(reinterpret_cast<const uint32_t*>(B), reinterpret_cast<uint32_t*>(out), alpha, E, N, r);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_router_wgrad(const uint16_t* xs, const float* dl, int T, int K, int E, float* partial, float* dWr, const float* scale,
-                                cudaStream_t st) {
-  const int chunks = (T + 255) / 256;
-  dim3 grid((K / 2 + 127) / 128, chunks);
-  { LaunchScope ls(KID_ROUTER_WGRAD, st);
-  k_router_wgrad_partial<<<grid, 128, 0, st>>>(reinterpret_cast<const uint32_t*>(xs), dl, T, K, E, partial); }
-  LaunchScope ls(KID_SUM_PARTIALS, st);
-  k_sum_partials<<<(E * K + 255) / 256, 256, 0, st>>>(partial, chunks, E * K, scale, dWr);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_sum_partials(const float* partial, int nparts, int n, const float* scale, float* out, cudaStream_t st) {
-  LaunchScope ls(KID_SUM_PARTIALS, st);
-  k_sum_partials<<<(n + 255) / 256, 256, 0, st>>>(partial, nparts, n, scale, out);
   return cudaGetLastError();
 }
 

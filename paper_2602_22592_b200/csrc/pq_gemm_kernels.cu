@@ -610,32 +610,41 @@ PQ_DEFINE_GEMM_KERNEL(k_gemm_bwd_dx, BwdDxProblem)
 //   dB tiles (one per expert and 128 output features, after the dW tiles): dBraw_e = dYs^T . (g H) over
 //     the expert's items, the hi and lo planes of g H side by side as the two halves of the tile's
 //     columns; dB = alpha_n dBraw, and the partial of dalpha_n = sum_j B[e,n,j] dBraw[n,j].
+//   router tiles (one per 256 columns of K, last): dWr = c * (dl / c)^T . Xs, the logit gradient in the
+//     bf16 form the dX tile also uses, rows >= E of the tile unused (Sec. 3.3, "trained end-to-end").
 // ---------------------------------------------------------------------------
 struct BwdDwProblem {
   using Acc = AccDouble;
   struct Params {
-    CUtensorMap tdyT, txt, tgh;
+    CUtensorMap tdyT, txt, tgh, tdlT, txs;
     RoutingTables rt;
     const int8_t* s8;
     const float* beta;
     const float* alpha;
+    const float* w_scales;
+    float* dWr;              // [E, K]
     const uint16_t* B;       // [E, N, r]
     float* dW;
     float* dB;               // [E, N, r]
     float* dbeta_partial;    // [2 * ceil(K/256), N]
     float* dalpha_partial;   // [2 * E, N]
     TileGrid g;
-    int T, N, K, r, r64, E, sstride, dy_blk, xt_blk, gh_blk, item_rows, ntn, db_tiles;
+    int T, N, K, r, r64, E, sstride, dy_blk, xt_blk, gh_blk, xs_blk, item_rows, ntn, db_tiles, wr_tiles;
   };
-  struct Tile { TileCoord c; int nt, bn, e, ib, ie; };   // e < 0: dW tile
-  __device__ static int num_tiles(const Params& p) { return p.g.total + p.db_tiles; }
+  struct Tile { TileCoord c; int nt, bn, e, ib, ie; };   // e == -1: dW tile, e == -2: router tile
+  __device__ static int num_tiles(const Params& p) { return p.g.total + p.db_tiles + p.wr_tiles; }
+  // order: router tiles and dW tiles (full-length contractions) first, the short dB tiles last
   __device__ static void tile_init(const Params& p, int i, Tile& t) {
-    if (i < p.g.total) {
-      t.c = tile_coord(p.g, i);
+    if (i < p.wr_tiles) {
+      t.e = -2; t.nt = 0; t.ib = t.ie = 0;
+      t.c.m = 0; t.c.n0 = i * 256; t.c.bn = 256;
+      t.bn = clip_bn(256, t.c.n0, p.K, 64);
+    } else if (i < p.wr_tiles + p.g.total) {
+      t.c = tile_coord(p.g, i - p.wr_tiles);
       t.nt = t.c.m; t.e = -1; t.ib = t.ie = 0;
       t.bn = clip_bn(t.c.bn, t.c.n0, p.K, 64);
     } else {
-      const int j = i - p.g.total;
+      const int j = i - p.wr_tiles - p.g.total;
       t.e = j / p.ntn; t.nt = j % p.ntn;
       t.ib = p.rt.expert_item_begin[t.e]; t.ie = p.rt.expert_item_begin[t.e + 1];
       t.bn = 2 * p.r64;
@@ -647,7 +656,11 @@ struct BwdDwProblem {
     s.mode = MODE_BF_MM; s.acc = 0; s.bn = t.bn; s.ksteps = 4; s.b_box = 0;
     s.ta = &p.tdyT; s.a_rank = 2; s.a_x = t.nt * 128; s.a_z = 0; s.a_blk = p.dy_blk;
     s.b_rank = 2; s.b_z = 0;
-    if (t.e < 0) {
+    if (t.e == -2) {
+      s.nkb = (p.T + 63) / 64; s.a_y = 0;
+      s.ta = &p.tdlT; s.a_x = 0; s.a_blk = 0;          // 16 columns: plain boxes, zero beyond
+      s.tb = &p.txs; s.b_x = t.c.n0; s.b_y = 0; s.b_blk = p.xs_blk;
+    } else if (t.e < 0) {
       s.nkb = (p.T + 63) / 64; s.a_y = 0;
       s.tb = &p.txt; s.b_x = t.c.n0; s.b_y = 0; s.b_blk = p.xt_blk;
     } else {
@@ -659,6 +672,27 @@ struct BwdDwProblem {
   using Pre = NoPre;
   __device__ static Pre prepare(const Params&, const Tile&, int, int) { return Pre{}; }
   __device__ static void epilogue(const Params& p, const Tile& t, const Pre& pre, uint32_t taddr, uint32_t, int quad, int half, int lane, uint8_t* stage) {
+    if (t.e == -2) {
+      // ---- router tile: row j < E of the accumulator is dWr[j, :] / c
+      const int j = quad * 32 + lane;
+      const float c = dx_scale(p.w_scales, p.beta, p.sstride);
+      const float cc = c != 0.f ? c : 1.0f;
+      float* out = j < p.E ? p.dWr + (long long)j * p.K : nullptr;
+      for (int c32 = half; c32 * 32 < t.bn; c32 += 2) {
+        const int k0 = t.c.n0 + c32 * 32;
+        if (k0 >= p.K) break;
+        uint32_t v[32];
+        tmem_ld32(taddr + c32 * 32, v);
+        tmem_ld_wait();
+        uint4 o[8];
+#pragma unroll
+        for (int q4 = 0; q4 < 8; ++q4)
+          o[q4] = make_uint4(__float_as_uint(cc * __uint_as_float(v[4 * q4])), __float_as_uint(cc * __uint_as_float(v[4 * q4 + 1])),
+                             __float_as_uint(cc * __uint_as_float(v[4 * q4 + 2])), __float_as_uint(cc * __uint_as_float(v[4 * q4 + 3])));
+        warp_store_rows(stage, o, out ? out + k0 : nullptr, min(32, p.K - k0) * 4, lane);
+      }
+      return;
+    }
     const int n = t.nt * 128 + quad * 32 + lane;
     const bool live = n < p.N;
     if (t.e >= 0) {
@@ -777,7 +811,7 @@ struct HpDaProblem {
 PQ_DEFINE_GEMM_KERNEL(k_gemm_hp_da, HpDaProblem)
 
 int gemm_backward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, const BwdBuffers& b, uint16_t* dX, float* dW, float* dA,
-                  float* dB, cudaStream_t st) {
+                  float* dB, float* dWr, cudaStream_t st) {
   const int mtiles = (a.T + 127) / 128;
   const int ntk = (a.K + 255) / 256, ntn128 = (a.N + 127) / 128;
   const bool hp = a.r > 0;
@@ -823,8 +857,15 @@ int gemm_backward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, c
     p.dbeta_partial = b.dbeta_partial; p.dalpha_partial = b.dalpha_partial;
     p.T = a.T; p.N = a.N; p.K = a.K; p.r = a.r; p.r64 = r64; p.E = a.E; p.sstride = a.scale_stride; p.item_rows = (int)item_rows;
     p.ntn = ntn128; p.db_tiles = hp ? a.E * ntn128 : 0;
+    p.tdlT = p.txt; p.txs = p.txt; p.xs_blk = 0; p.wr_tiles = 0; p.w_scales = a.w_scales; p.dWr = dWr;
+    if (hp && a.E > 1) {
+      int unused = 0;
+      if (!map_mn(&p.tdlT, &unused, b.dlc, 16, a.T, 2, 1, 2)) return PQ_ERR_CUDA;
+      if (!map_mn(&p.txs, &p.xs_blk, b.xs, a.K, a.T, 2, 1, 4)) return PQ_ERR_CUDA;
+      p.wr_tiles = ntk;
+    }
     p.g = make_tile_grid(ntn128, ntk, 256);
-    rc = launch_gemm(KID_BWD_DW, k_gemm_bwd_dw, p, p.g.total + p.db_tiles, st);
+    rc = launch_gemm(KID_BWD_DW, k_gemm_bwd_dw, p, p.g.total + p.db_tiles + p.wr_tiles, st);
     if (rc) return rc;
   }
   if (hp) {

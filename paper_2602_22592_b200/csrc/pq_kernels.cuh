@@ -77,9 +77,6 @@ cudaError_t launch_route_and_quant(const uint16_t* X, const uint16_t* Wr, int T,
 cudaError_t launch_scatter_rows(const uint16_t* src, uint16_t* dst, const int* pos, int T, int row_elems, cudaStream_t st);
 cudaError_t launch_scaled_sign(const int8_t* s8, uint16_t* out, const float* beta, int beta_stride, int N, int K, cudaStream_t st);
 cudaError_t launch_scaled_b(const uint16_t* B, uint16_t* out, const float* alpha, int E, int N, int r, cudaStream_t st);
-cudaError_t launch_router_wgrad(const uint16_t* xs, const float* dl, int T, int K, int E, float* partial, float* dWr, const float* scale,
-                                cudaStream_t st);
-cudaError_t launch_sum_partials(const float* partial, int nparts, int n, const float* scale, float* out, cudaStream_t st);
 cudaError_t launch_finalize_scales(const float* dbeta_partial, int nslots, const float* dalpha_partial, int E, int N, const float* w_scales,
                                    int vec, float* dbeta, float* dalpha, float* tmp_b, float* tmp_a, cudaStream_t st);
 cudaError_t launch_fill_zero(void* p, size_t bytes, cudaStream_t st);
@@ -115,13 +112,13 @@ struct BwdBuffers {
   const uint16_t* ba;    // [E,N,r] bf16 B * (alpha_n or 1)
   uint16_t* dhc;         // [2][items*128, r] bf16 hi/lo planes of dH / c
   uint16_t* gh;          // [2][items*128, r] bf16 hi/lo planes of g * H
-  float* dl;             // [T,E] fp32 router logit gradient (sorted order)
+  float* dl;             // [T,E] fp32 router logit gradient (sorted order), kept for inspection
   uint16_t* dlc;         // [T,16] bf16 dl / c
   float* dbeta_partial;  // [2 * ceil(K/256), N]
   float* dalpha_partial; // [2 * E, N]
   float* da_partial;     // [max_chunks_a, r, K] raw split-contraction partials of dA
 };
 int gemm_backward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, const BwdBuffers& b, uint16_t* dX, float* dW, float* dA,
-                  float* dB, cudaStream_t st);
+                  float* dB, float* dWr, cudaStream_t st);
 
 }  // namespace pq
