@@ -26,15 +26,6 @@ static inline int experts_of(const pq_desc* d) { return d->r > 0 ? (d->E < 1 ? 1
 static inline int max_items_of(const pq_desc* d) { return mtiles_of(d) + experts_of(d) - 1; }
 static inline bool routed(const pq_desc* d) { return d->r > 0 && d->E > 1; }
 
-// Items per chunk for the split token contraction of dA: (chunks x output tiles)
-// should fill about one wave of 148 CTAs; more chunks only add fp32 partial results to write and re-read.
-static inline int chunk_items(int mtiles, int out_tiles) {
-  int c = (mtiles * out_tiles + 147) / 148;
-  return c < 1 ? 1 : c;
-}
-static inline int chunk_a_of(const pq_desc* d) { return chunk_items(mtiles_of(d), (d->K + 255) / 256); }
-static inline int max_chunks(const pq_desc* d, int chunk) { return (max_items_of(d) + chunk - 1) / chunk + experts_of(d); }
-
 static int check_desc(const pq_desc* d, bool training) {
   if (!d) return PQ_ERR_NULL;
   if (d->size != sizeof(pq_desc)) return PQ_ERR_SHAPE;
@@ -68,11 +59,6 @@ static size_t carve_saved(const pq_desc* d, void* base, SavedPtrs* out) {
   s.rt.items = c.take<int4>(s.max_items);
   s.rt.tile_item_begin = c.take<int>(mtiles_of(d) + 1);
   s.rt.expert_item_begin = c.take<int>(E + 1);
-  s.chunk_a = chunk_a_of(d);
-  s.max_chunks_a = max_chunks(d, s.chunk_a);
-  s.rt.n_chunks_a = c.take<int>(1);
-  s.rt.chunks_a = c.take<int4>(s.max_chunks_a);
-  s.rt.expert_chunk_begin_a = c.take<int>(E + 1);
   if (out) *out = s;
   return c.off;
 }
@@ -102,7 +88,6 @@ struct BwdScratch {
   float* dalpha_partial;
   float* dalpha_vec;
   float* dbeta_vec;
-  float* da_partial;
 };
 
 static size_t carve_bwd_scratch(const pq_desc* d, void* base, BwdScratch* out) {
@@ -122,7 +107,6 @@ static size_t carve_bwd_scratch(const pq_desc* d, void* base, BwdScratch* out) {
   s.dalpha_partial = r > 0 ? c.take<float>((size_t)2 * E * N) : nullptr;
   s.dalpha_vec = c.take<float>(N);
   s.dbeta_vec = c.take<float>(N);
-  s.da_partial = r > 0 ? c.take<float>((size_t)max_chunks(d, chunk_a_of(d)) * r * K) : nullptr;
   if (out) *out = s;
   return c.off;
 }
@@ -374,7 +358,6 @@ int pq_linear_backward(const pq_desc* d, const uint16_t* dY, const uint16_t* X, 
   }
   b.dhc = sc.dhc; b.gh = sc.gh; b.dl = sc.dl; b.dlc = sc.dlc;
   b.dbeta_partial = sc.dbeta_partial; b.dalpha_partial = sc.dalpha_partial;
-  b.da_partial = sc.da_partial;
   rc = gemm_backward(a, w_s8, sv, b, dX, dW, dA, dB, dWr, st);
   if (rc) return rc;
 

@@ -202,8 +202,6 @@ __global__ void __launch_bounds__(1024) k_router(const uint4* __restrict__ X, co
 // table.  An item is the intersection of a 128-row tile of the sorted token
 // order with one expert's range: {tile, expert, first row, end row} (rows
 // relative to the tile).  Items are sorted by tile and therefore by expert.
-// Also groups each expert's items into chunks: the units over which the token
-// contraction of dA is split across CTAs.
 // One block; the work is a few hundred integers.
 // ---------------------------------------------------------------------------
 // Items of one 128-row tile [r0, r1) of the sorted order: experts e0 <= e < E whose non-empty range
@@ -218,37 +216,10 @@ __device__ __forceinline__ int tile_items(const int* off, int Ee, int r0, int r1
   return n;
 }
 
-// One chunk table: consecutive items of one expert, at most `size` items each.  Thread 0 lays out the
-// experts' chunk ranges (<= 16 experts), then all threads fill the entries.
-__device__ __forceinline__ void build_chunks(int Ee, const int* item_begin /*shared, Ee+1*/, int size, int4* out, int* begin, int* count,
-                                             int* sh_begin /*shared, Ee+1*/) {
-  if (threadIdx.x == 0) {
-    int n = 0;
-    for (int e = 0; e < Ee; ++e) {
-      sh_begin[e] = n;
-      n += (item_begin[e + 1] - item_begin[e] + size - 1) / size;
-    }
-    sh_begin[Ee] = n;
-    count[0] = n;
-  }
-  __syncthreads();
-  if (threadIdx.x <= Ee) begin[threadIdx.x] = sh_begin[threadIdx.x];
-  for (int c = threadIdx.x; c < sh_begin[Ee]; c += blockDim.x) {
-    int e = 0;
-    while (sh_begin[e + 1] <= c) ++e;
-    const int first = item_begin[e] + (c - sh_begin[e]) * size;
-    out[c] = make_int4(e, first, min(first + size, item_begin[e + 1]), 0);
-  }
-  __syncthreads();
-}
-
 __global__ void __launch_bounds__(512) k_route_scan(int T, int E, int nblocks, const int* __restrict__ block_counts,
-                                                    int* __restrict__ block_base, int* __restrict__ offsets, RoutingTables rt,
-                                                    int chunk_a) {
+                                                    int* __restrict__ block_base, int* __restrict__ offsets, RoutingTables rt) {
   __shared__ int off[kMaxExperts + 1];
   __shared__ int total[kMaxExperts];
-  __shared__ int item_begin[kMaxExperts + 1];
-  __shared__ int chunk_begin[kMaxExperts + 1];
   __shared__ int warp_sums[16];
   __shared__ int carry_sh;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -321,11 +292,8 @@ __global__ void __launch_bounds__(512) k_route_scan(int T, int E, int nblocks, c
       for (int f = 0; f < e; ++f)
         if (min(off[f + 1], r0 + kTileRows) > max(off[f], r0)) ++idx;
     }
-    item_begin[threadIdx.x] = idx;
     rt.expert_item_begin[threadIdx.x] = idx;
   }
-  __syncthreads();
-  build_chunks(Ee, item_begin, chunk_a, rt.chunks_a, rt.expert_chunk_begin_a, rt.n_chunks_a, chunk_begin);
 }
 
 // ---------------------------------------------------------------------------
@@ -530,25 +498,6 @@ __global__ void __launch_bounds__(1024) k_sum_scales(const float* __restrict__ v
   }
 }
 
-// dA[e,j,k] = c * sum over expert e's chunks of the raw partials; c as in the dX tile (lam*beta or lam, 1 if that is 0)
-__global__ void __launch_bounds__(256) k_reduce_da(const float* __restrict__ partial, RoutingTables rt, const float* __restrict__ w_scales,
-                                                   const float* __restrict__ beta, int sstride, int E, int r, int K, float* __restrict__ dA) {
-  const long long per_e = (long long)r * K / 4, total = per_e * E;
-  float c = sstride ? w_scales[0] : w_scales[0] * beta[0];
-  if (c == 0.f) c = 1.0f;
-  for (long long i = blockIdx.x * 256LL + threadIdx.x; i < total; i += gridDim.x * 256LL) {
-    const int e = (int)(i / per_e);
-    const long long w = i % per_e;
-    const int c0 = rt.expert_chunk_begin_a[e], c1 = rt.expert_chunk_begin_a[e + 1];
-    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int ch = c0; ch < c1; ++ch) {
-      const float4 v = reinterpret_cast<const float4*>(partial)[(long long)ch * per_e + w];
-      s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
-    }
-    reinterpret_cast<float4*>(dA)[i] = make_float4(c * s.x, c * s.y, c * s.z, c * s.w);
-  }
-}
-
 __global__ void k_fill_zero(uint4* p, long long n16) {
   for (long long i = blockIdx.x * 256LL + threadIdx.x; i < n16; i += gridDim.x * 256LL) p[i] = make_uint4(0, 0, 0, 0);
 }
@@ -583,7 +532,7 @@ cudaError_t launch_route_and_quant(const uint16_t* X, const uint16_t* Wr, int T,
                                       sc.probs_tok, sc.block_counts);
   }
   { LaunchScope ls(KID_ROUTE_SCAN, st);
-  k_route_scan<<<1, 512, 0, st>>>(T, E, nblocks, sc.block_counts, sc.block_base, sv.offsets, sv.rt, sv.chunk_a); }
+  k_route_scan<<<1, 512, 0, st>>>(T, E, nblocks, sc.block_counts, sc.block_base, sv.offsets, sv.rt); }
   LaunchScope ls(KID_ACT_QUANT, st);
   const int per_lane = (K / 8 + 31) / 32;   // 16-byte pieces of a row per lane if one warp took the whole row
   auto kern = k_act_quant<0, 1>;
@@ -631,14 +580,6 @@ cudaError_t launch_finalize_scales(const float* dbeta_partial, int nslots, const
     LaunchScope ls(KID_SUM_SCALAR, st);
     k_sum_scales<<<1, 1024, 0, st>>>(tmp_b, dalpha_partial ? tmp_a : nullptr, N, dbeta, dalpha);
   }
-  return cudaGetLastError();
-}
-
-cudaError_t launch_reduce_da(const float* partial, const RoutingTables& rt, const float* w_scales, const float* beta, int sstride, int E, int r,
-                             int K, float* dA, cudaStream_t st) {
-  LaunchScope ls(KID_REDUCE_DA, st);
-  const long long total = (long long)E * r * K / 4;
-  k_reduce_da<<<grid_for(total, 256 * 2, 148 * 8), 256, 0, st>>>(partial, rt, w_scales, beta, sstride, E, r, K, dA);
   return cudaGetLastError();
 }
 

@@ -610,80 +610,120 @@ PQ_DEFINE_GEMM_KERNEL(k_gemm_bwd_dx, BwdDxProblem)
 //   dB tiles (one per expert and 128 output features, after the dW tiles): dBraw_e = dYs^T . (g H) over
 //     the expert's items, the hi and lo planes of g H side by side as the two halves of the tile's
 //     columns; dB = alpha_n dBraw, and the partial of dalpha_n = sum_j B[e,n,j] dBraw[n,j].
-//   router tiles (one per 256 columns of K, last): dWr = c * (dl / c)^T . Xs, the logit gradient in the
+//   router tiles (one per 256 columns of K): dWr = c * (dl / c)^T . Xs, the logit gradient in the
 //     bf16 form the dX tile also uses, rows >= E of the tile unused (Sec. 3.3, "trained end-to-end").
+//   dA tiles (one per expert and 256 columns of K): dA_e = c * (dH / c)^T . Xs over the expert's items, with the
+//     leading bf16 plane of dH / c (its 2^-9 rounding averages out over the tokens of the sum).
 // ---------------------------------------------------------------------------
 struct BwdDwProblem {
   using Acc = AccDouble;
+  enum Kind : int { KIND_DW = 0, KIND_DB = 1, KIND_DWR = 2, KIND_DA = 3 };
   struct Params {
-    CUtensorMap tdyT, txt, tgh, tdlT, txs;
+    CUtensorMap tdyT, txt, tgh, tdlT, txs, tdhT;
     RoutingTables rt;
     const int8_t* s8;
     const float* beta;
     const float* alpha;
     const float* w_scales;
     float* dWr;              // [E, K]
+    float* dA;               // [E, r, K]
     const uint16_t* B;       // [E, N, r]
     float* dW;
     float* dB;               // [E, N, r]
     float* dbeta_partial;    // [2 * ceil(K/256), N]
     float* dalpha_partial;   // [2 * E, N]
     TileGrid g;
-    int T, N, K, r, r64, E, sstride, dy_blk, xt_blk, gh_blk, xs_blk, item_rows, ntn, db_tiles, wr_tiles;
+    int T, N, K, r, r64, E, sstride, dy_blk, xt_blk, gh_blk, xs_blk, dh_blk, item_rows, ntn, ntk, db_tiles, wr_tiles, da_tiles;
   };
-  struct Tile { TileCoord c; int nt, bn, e, ib, ie; };   // e == -1: dW tile, e == -2: router tile
-  __device__ static int num_tiles(const Params& p) { return p.g.total + p.db_tiles + p.wr_tiles; }
-  // order: router tiles and dW tiles (full-length contractions) first, the short dB tiles last
+  struct Tile { TileCoord c; int kind, nt, bn, e, ib, ie; };
+  __device__ static int num_tiles(const Params& p) { return p.wr_tiles + p.da_tiles + p.g.total + p.db_tiles; }
+  // order: the tiles whose contraction runs over all tokens first (router, dA with one expert, dW), the short ones last
   __device__ static void tile_init(const Params& p, int i, Tile& t) {
+    t.ib = t.ie = 0; t.e = 0; t.nt = 0;
     if (i < p.wr_tiles) {
-      t.e = -2; t.nt = 0; t.ib = t.ie = 0;
+      t.kind = KIND_DWR;
       t.c.m = 0; t.c.n0 = i * 256; t.c.bn = 256;
       t.bn = clip_bn(256, t.c.n0, p.K, 64);
-    } else if (i < p.wr_tiles + p.g.total) {
-      t.c = tile_coord(p.g, i - p.wr_tiles);
-      t.nt = t.c.m; t.e = -1; t.ib = t.ie = 0;
-      t.bn = clip_bn(t.c.bn, t.c.n0, p.K, 64);
-    } else {
-      const int j = i - p.wr_tiles - p.g.total;
-      t.e = j / p.ntn; t.nt = j % p.ntn;
-      t.ib = p.rt.expert_item_begin[t.e]; t.ie = p.rt.expert_item_begin[t.e + 1];
-      t.bn = 2 * p.r64;
-      t.c.m = t.nt; t.c.n0 = 0; t.c.bn = t.bn;
+      return;
     }
+    i -= p.wr_tiles;
+    if (i < p.da_tiles) {
+      t.kind = KIND_DA;
+      t.e = i / p.ntk;
+      t.ib = p.rt.expert_item_begin[t.e]; t.ie = p.rt.expert_item_begin[t.e + 1];
+      t.c.m = 0; t.c.n0 = (i % p.ntk) * 256; t.c.bn = 256;
+      t.bn = clip_bn(256, t.c.n0, p.K, 64);
+      return;
+    }
+    i -= p.da_tiles;
+    if (i < p.g.total) {
+      t.kind = KIND_DW;
+      t.c = tile_coord(p.g, i);
+      t.nt = t.c.m;
+      t.bn = clip_bn(t.c.bn, t.c.n0, p.K, 64);
+      return;
+    }
+    i -= p.g.total;
+    t.kind = KIND_DB;
+    t.e = i / p.ntn; t.nt = i % p.ntn;
+    t.ib = p.rt.expert_item_begin[t.e]; t.ie = p.rt.expert_item_begin[t.e + 1];
+    t.bn = 2 * p.r64;
+    t.c.m = t.nt; t.c.n0 = 0; t.c.bn = t.bn;
   }
-  __device__ static int num_segments(const Params&, const Tile& t) { return t.e < 0 ? 1 : t.ie - t.ib; }
+  __device__ static int num_segments(const Params&, const Tile& t) { return (t.kind == KIND_DW || t.kind == KIND_DWR) ? 1 : t.ie - t.ib; }
   __device__ static void segment(const Params& p, const Tile& t, int i, Segment& s) {
     s.mode = MODE_BF_MM; s.acc = 0; s.bn = t.bn; s.ksteps = 4; s.b_box = 0;
-    s.ta = &p.tdyT; s.a_rank = 2; s.a_x = t.nt * 128; s.a_z = 0; s.a_blk = p.dy_blk;
-    s.b_rank = 2; s.b_z = 0;
-    if (t.e == -2) {
-      s.nkb = (p.T + 63) / 64; s.a_y = 0;
-      s.ta = &p.tdlT; s.a_x = 0; s.a_blk = 0;          // 16 columns: plain boxes, zero beyond
-      s.tb = &p.txs; s.b_x = t.c.n0; s.b_y = 0; s.b_blk = p.xs_blk;
-    } else if (t.e < 0) {
-      s.nkb = (p.T + 63) / 64; s.a_y = 0;
-      s.tb = &p.txt; s.b_x = t.c.n0; s.b_y = 0; s.b_blk = p.xt_blk;
-    } else {
-      const int item = t.ib + i;
-      s.nkb = 2; s.a_y = p.rt.items[item].x * 128;      // the 128 tokens of the item's tile (rows outside the item are zero in g H)
-      s.tb = &p.tgh; s.b_x = 0; s.b_y = item * 128; s.b2_y = p.item_rows + item * 128; s.b_blk = p.gh_blk;
+    s.a_rank = 2; s.a_z = 0; s.b_rank = 2; s.b_z = 0;
+    switch (t.kind) {
+      case KIND_DW:
+        s.nkb = (p.T + 63) / 64;
+        s.ta = &p.tdyT; s.a_x = t.nt * 128; s.a_y = 0; s.a_blk = p.dy_blk;
+        s.tb = &p.txt; s.b_x = t.c.n0; s.b_y = 0; s.b_blk = p.xt_blk;
+        break;
+      case KIND_DWR:
+        s.nkb = (p.T + 63) / 64;
+        s.ta = &p.tdlT; s.a_x = 0; s.a_y = 0; s.a_blk = 0;          // 16 columns: plain boxes, zero beyond
+        s.tb = &p.txs; s.b_x = t.c.n0; s.b_y = 0; s.b_blk = p.xs_blk;
+        break;
+      case KIND_DB: {
+        const int item = t.ib + i;
+        s.nkb = 2;                                        // the 128 tokens of the item's tile (rows outside the item are zero in g H)
+        s.ta = &p.tdyT; s.a_x = t.nt * 128; s.a_y = p.rt.items[item].x * 128; s.a_blk = p.dy_blk;
+        s.tb = &p.tgh; s.b_x = 0; s.b_y = item * 128; s.b2_y = p.item_rows + item * 128; s.b_blk = p.gh_blk;
+        break;
+      }
+      default: {                                          // KIND_DA: (dH / c)^T . Xs over the expert's items, leading plane of dH / c
+        const int item = t.ib + i;
+        s.nkb = 2;
+        s.ta = &p.tdhT; s.a_x = 0; s.a_y = item * 128; s.a_blk = p.dh_blk;
+        s.tb = &p.txs; s.b_x = t.c.n0; s.b_y = p.rt.items[item].x * 128; s.b_blk = p.xs_blk;
+        break;
+      }
     }
   }
   using Pre = NoPre;
   __device__ static Pre prepare(const Params&, const Tile&, int, int) { return Pre{}; }
   __device__ static void epilogue(const Params& p, const Tile& t, const Pre& pre, uint32_t taddr, uint32_t, int quad, int half, int lane, uint8_t* stage) {
-    if (t.e == -2) {
-      // ---- router tile: row j < E of the accumulator is dWr[j, :] / c
+    if (t.kind == KIND_DWR || t.kind == KIND_DA) {
+      // ---- router tile: row j < E of the accumulator is dWr[j, :] / c;  dA tile: row j < r is dA[e, j, :] / c
       const int j = quad * 32 + lane;
       const float c = dx_scale(p.w_scales, p.beta, p.sstride);
       const float cc = c != 0.f ? c : 1.0f;
-      float* out = j < p.E ? p.dWr + (long long)j * p.K : nullptr;
+      const bool any = t.kind == KIND_DWR || t.ie > t.ib;    // an expert without tokens: exact zeros
+      float* out = nullptr;
+      if (t.kind == KIND_DWR) { if (j < p.E) out = p.dWr + (long long)j * p.K; }
+      else if (j < p.r) out = p.dA + ((long long)t.e * p.r + j) * p.K;
       for (int c32 = half; c32 * 32 < t.bn; c32 += 2) {
         const int k0 = t.c.n0 + c32 * 32;
         if (k0 >= p.K) break;
         uint32_t v[32];
-        tmem_ld32(taddr + c32 * 32, v);
-        tmem_ld_wait();
+        if (any) {
+          tmem_ld32(taddr + c32 * 32, v);
+          tmem_ld_wait();
+        } else {
+#pragma unroll
+          for (int u = 0; u < 32; ++u) v[u] = 0u;
+        }
         uint4 o[8];
 #pragma unroll
         for (int q4 = 0; q4 < 8; ++q4)
@@ -695,7 +735,7 @@ struct BwdDwProblem {
     }
     const int n = t.nt * 128 + quad * 32 + lane;
     const bool live = n < p.N;
-    if (t.e >= 0) {
+    if (t.kind == KIND_DB) {
       // ---- dB tile: columns [0, r64) hold the hi-plane product, [r64, 2 r64) the lo-plane product
       const bool any = t.ie > t.ib;                     // an expert without tokens: exact zeros
       const float al = live ? p.alpha[n * p.sstride] : 0.f;
@@ -763,53 +803,6 @@ struct BwdDwProblem {
 };
 PQ_DEFINE_GEMM_KERNEL(k_gemm_bwd_dw, BwdDwProblem)
 
-// ---------------------------------------------------------------------------
-// B5: raw dA partials, dhc^T . Xs over one chunk of an expert's items; summed and
-// scaled by k_reduce_da.
-// ---------------------------------------------------------------------------
-struct HpDaProblem {
-  using Acc = AccDouble;
-  struct Params {
-    CUtensorMap tdhT, txs;
-    RoutingTables rt;
-    float* partial;  // [chunks, r, K]
-    int K, r, ntk, item_rows, dh_blk, xs_blk;
-  };
-  struct Tile { int chunk, kt, ib, ie; };
-  __device__ static int num_tiles(const Params& p) { return p.ntk * p.rt.n_chunks_a[0]; }
-  __device__ static void tile_init(const Params& p, int i, Tile& t) {
-    t.chunk = i / p.ntk; t.kt = i % p.ntk;
-    const int4 c = p.rt.chunks_a[t.chunk];
-    t.ib = c.y; t.ie = c.z;
-  }
-  __device__ static int num_segments(const Params&, const Tile& t) { return 2 * (t.ie - t.ib); }
-  __device__ static void segment(const Params& p, const Tile& t, int i, Segment& s) {
-    const int item = t.ib + (i >> 1), plane = i & 1;
-    s.mode = MODE_BF_MM; s.acc = 0; s.bn = 256; s.ksteps = 4; s.nkb = 2;
-    s.ta = &p.tdhT; s.a_rank = 2; s.a_x = 0; s.a_y = plane * p.item_rows + item * 128; s.a_z = 0;
-    s.tb = &p.txs; s.b_rank = 2; s.b_x = t.kt * 256; s.b_y = p.rt.items[item].x * 128; s.b_z = 0;
-    s.b_box = 0; s.a_blk = p.dh_blk; s.b_blk = p.xs_blk;
-  }
-  using Pre = NoPre;
-  __device__ static Pre prepare(const Params&, const Tile&, int, int) { return Pre{}; }
-  __device__ static void epilogue(const Params& p, const Tile& t, const Pre& pre, uint32_t taddr, uint32_t, int quad, int half, int lane, uint8_t* stage) {
-    const int j = quad * 32 + lane;
-    float* out = j < p.r ? p.partial + ((long long)t.chunk * p.r + j) * p.K : nullptr;
-    for (int c32 = half; c32 < 8; c32 += 2) {
-      const int k0 = t.kt * 256 + c32 * 32;
-      if (k0 >= p.K) break;
-      uint32_t v[32];
-      tmem_ld32(taddr + c32 * 32, v);
-      tmem_ld_wait();
-      uint4 o[8];
-#pragma unroll
-      for (int q = 0; q < 8; ++q) o[q] = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
-      warp_store_rows(stage, o, out ? out + k0 : nullptr, 128, lane);
-    }
-  }
-};
-PQ_DEFINE_GEMM_KERNEL(k_gemm_hp_da, HpDaProblem)
-
 int gemm_backward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, const BwdBuffers& b, uint16_t* dX, float* dW, float* dA,
                   float* dB, float* dWr, cudaStream_t st) {
   const int mtiles = (a.T + 127) / 128;
@@ -856,26 +849,21 @@ int gemm_backward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, c
     p.rt = sv.rt; p.s8 = w_s8; p.beta = a.beta; p.alpha = a.alpha; p.B = a.B; p.dW = dW; p.dB = dB;
     p.dbeta_partial = b.dbeta_partial; p.dalpha_partial = b.dalpha_partial;
     p.T = a.T; p.N = a.N; p.K = a.K; p.r = a.r; p.r64 = r64; p.E = a.E; p.sstride = a.scale_stride; p.item_rows = (int)item_rows;
-    p.ntn = ntn128; p.db_tiles = hp ? a.E * ntn128 : 0;
-    p.tdlT = p.txt; p.txs = p.txt; p.xs_blk = 0; p.wr_tiles = 0; p.w_scales = a.w_scales; p.dWr = dWr;
+    p.ntn = ntn128; p.ntk = ntk; p.db_tiles = hp ? a.E * ntn128 : 0; p.da_tiles = hp ? a.E * ntk : 0;
+    p.tdlT = p.txt; p.txs = p.txt; p.tdhT = p.txt; p.xs_blk = 0; p.dh_blk = 0; p.wr_tiles = 0;
+    p.w_scales = a.w_scales; p.dWr = dWr; p.dA = dA;
+    if (hp) {
+      if (!map_mn(&p.txs, &p.xs_blk, b.xs, a.K, a.T, 2, 1, 4)) return PQ_ERR_CUDA;
+      if (!map_mn(&p.tdhT, &p.dh_blk, b.dhc, a.r, 2 * item_rows, 2, 1, 2)) return PQ_ERR_CUDA;
+    }
     if (hp && a.E > 1) {
       int unused = 0;
       if (!map_mn(&p.tdlT, &unused, b.dlc, 16, a.T, 2, 1, 2)) return PQ_ERR_CUDA;
-      if (!map_mn(&p.txs, &p.xs_blk, b.xs, a.K, a.T, 2, 1, 4)) return PQ_ERR_CUDA;
       p.wr_tiles = ntk;
     }
     p.g = make_tile_grid(ntn128, ntk, 256);
-    rc = launch_gemm(KID_BWD_DW, k_gemm_bwd_dw, p, p.g.total + p.db_tiles + p.wr_tiles, st);
+    rc = launch_gemm(KID_BWD_DW, k_gemm_bwd_dw, p, p.wr_tiles + p.da_tiles + p.g.total + p.db_tiles, st);
     if (rc) return rc;
-  }
-  if (hp) {
-    HpDaProblem::Params q;
-    if (!map_mn(&q.tdhT, &q.dh_blk, b.dhc, a.r, 2 * item_rows, 2, 1, 2)) return PQ_ERR_CUDA;
-    if (!map_mn(&q.txs, &q.xs_blk, b.xs, a.K, a.T, 2, 1, 4)) return PQ_ERR_CUDA;
-    q.rt = sv.rt; q.partial = b.da_partial; q.K = a.K; q.r = a.r; q.ntk = ntk; q.item_rows = (int)item_rows;
-    rc = launch_gemm(KID_HP_DA, k_gemm_hp_da, q, ntk * sv.max_chunks_a, st);
-    if (rc) return rc;
-    if (launch_reduce_da(b.da_partial, sv.rt, a.w_scales, a.beta, a.scale_stride, a.E, a.r, a.K, dA, st) != cudaSuccess) return PQ_ERR_CUDA;
   }
   return PQ_OK;
 }

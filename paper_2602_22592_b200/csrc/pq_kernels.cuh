@@ -38,10 +38,6 @@ struct RoutingTables {
   int4* items;             // [max_items] {tile, expert, first row, end row}
   int* tile_item_begin;    // [mtiles + 1]
   int* expert_item_begin;  // [E + 1]
-  // chunk table {expert, first item, end item, 0}: the units the token contraction of dA is split into
-  int* n_chunks_a;         // [1]
-  int4* chunks_a;          // [max_items + E]
-  int* expert_chunk_begin_a;  // [E + 1]
 };
 
 // Device pointers into the caller's `saved` buffer.
@@ -59,8 +55,6 @@ struct SavedPtrs {
   uint16_t* h;
   RoutingTables rt;
   int max_items;
-  int chunk_a;               // items per chunk
-  int max_chunks_a;
 };
 
 struct FwdScratch {
@@ -80,8 +74,6 @@ cudaError_t launch_scaled_b(const uint16_t* B, uint16_t* out, const float* alpha
 cudaError_t launch_finalize_scales(const float* dbeta_partial, int nslots, const float* dalpha_partial, int E, int N, const float* w_scales,
                                    int vec, float* dbeta, float* dalpha, float* tmp_b, float* tmp_a, cudaStream_t st);
 cudaError_t launch_fill_zero(void* p, size_t bytes, cudaStream_t st);
-cudaError_t launch_reduce_da(const float* partial, const RoutingTables& rt, const float* w_scales, const float* beta, int sstride, int E, int r,
-                             int K, float* dA, cudaStream_t st);
 
 // tensor-core launchers (pq_gemm_kernels.cu).  All return a PQ_* status.
 struct LayerArgs {
@@ -116,7 +108,6 @@ struct BwdBuffers {
   uint16_t* dlc;         // [T,16] bf16 dl / c
   float* dbeta_partial;  // [2 * ceil(K/256), N]
   float* dalpha_partial; // [2 * E, N]
-  float* da_partial;     // [max_chunks_a, r, K] raw split-contraction partials of dA
 };
 int gemm_backward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, const BwdBuffers& b, uint16_t* dX, float* dW, float* dA,
                   float* dB, float* dWr, cudaStream_t st);
