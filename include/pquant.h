@@ -174,6 +174,29 @@ typedef struct pq_decode_view {
 } pq_decode_view;
 int pq_decode_view_init(const pq_desc* d, void* ws, pq_decode_view* out);
 
+/* Decode forward of several INDEPENDENT linears in one launch pair (App. A: at batch size
+ * one the weights' bytes are the cost, so linears that do not depend on each other -- the
+ * gate and up projections of a block, the q/k/v projections, other sequences -- should
+ * stream their weights back to back instead of paying a launch and a pipeline fill each).
+ * Each item is what pq_linear_forward takes in its decode form; results are identical to n
+ * separate calls.  `items` is a HOST array, read before the call returns.  Any n >= 1
+ * (launched in groups of 16); every item needs its own ws. */
+typedef struct pq_decode_item {
+  pq_desc desc;            /* T <= 16 */
+  const uint16_t* X;       /* [T,K] bf16 */
+  const uint32_t* w_bits;  /* [N,K/32] */
+  const float* w_scales;   /* {lam, mu} */
+  const uint16_t* A;       /* [E,r,K] */
+  const uint16_t* B;       /* [E,N,r] */
+  const uint16_t* Wr;      /* [E,K], NULL if E <= 1 */
+  const float* alpha;
+  const float* beta;
+  uint16_t* Y;             /* [T,N] bf16 (out) */
+  void* ws;                /* pq_workspace_bytes(&desc, PQ_PHASE_DECODE) bytes */
+  size_t ws_bytes;
+} pq_decode_item;
+int pq_decode_batch(const pq_decode_item* items, int n, void* stream);
+
 /* Straight-through backward (App. B.1): Sign, Round and Clip pass the gradient
  * unchanged; mu, lam, gamma are constants.  Every gradient is OVERWRITTEN.
  *   dY [T,N] bf16 (in);  dX [T,K] bf16;  dW [N,K] fp32 (w.r.t. the latent W);

@@ -22,7 +22,7 @@ PQ_DECODE_DUMP_ACC = 2
 PQ_PHASE_PACK, PQ_PHASE_FWD, PQ_PHASE_BWD, PQ_PHASE_DECODE = 0, 1, 2, 3
 
 EXPORTS = ("pq_status_string", "pq_workspace_bytes", "pq_saved_bytes", "pq_saved_view_init",
-           "pq_decode_view_init", "pq_pack_weights", "pq_pack_weights_static", "pq_linear_forward", "pq_linear_backward", "pq_debug_gemm", "pq_debug_gemm_tile",
+           "pq_decode_view_init", "pq_decode_batch", "pq_pack_weights", "pq_pack_weights_static", "pq_linear_forward", "pq_linear_backward", "pq_debug_gemm", "pq_debug_gemm_tile",
            "pq_device_status", "pq_kernel_launches", "pq_profile_events", "pq_set_option")
 
 KERNEL_IDS = dict(pack_sums=0, binarize_pack=1, router=2, route_scan=3, act_quant=4, hp_up=5, fwd=6, scatter_rows=7,
@@ -46,6 +46,11 @@ class pq_saved_view(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in
                 ("q", "xt", "xs", "gamma", "gate", "probs", "expert", "perm", "pos", "offsets", "h",
                  "n_items", "items", "tile_item_begin", "expert_item_begin")] + [("max_items", ctypes.c_int32)]
+
+
+class pq_decode_item(ctypes.Structure):
+    _fields_ = [("desc", pq_desc)] + [(n, ctypes.c_void_p) for n in
+                                      ("X", "w_bits", "w_scales", "A", "B", "Wr", "alpha", "beta", "Y", "ws")] + [("ws_bytes", ctypes.c_size_t)]
 
 
 class pq_decode_view(ctypes.Structure):
@@ -74,6 +79,8 @@ def lib() -> ctypes.CDLL:
         L.pq_saved_view_init.argtypes = [dp, vp, ctypes.POINTER(pq_saved_view)]
         L.pq_decode_view_init.restype = ci
         L.pq_decode_view_init.argtypes = [dp, vp, ctypes.POINTER(pq_decode_view)]
+        L.pq_decode_batch.restype = ci
+        L.pq_decode_batch.argtypes = [ctypes.POINTER(pq_decode_item), ci, vp]
         L.pq_pack_weights.restype = ci
         L.pq_pack_weights.argtypes = [dp, vp, vp, vp, vp, vp, sz, vp]
         L.pq_pack_weights_static.restype = ci
@@ -191,6 +198,24 @@ def pq_linear_forward(d, X, w_bits, w_s8, w_scales, A, B, Wr, alpha, beta, Y, sa
     _check("pq_linear_forward", lib().pq_linear_forward(
         ctypes.byref(d), _ptr(X), _ptr(w_bits), _ptr(w_s8), _ptr(w_scales), _ptr(A), _ptr(B), _ptr(Wr), _ptr(alpha),
         _ptr(beta), _ptr(Y), _ptr(saved), _nbytes(saved), _ptr(ws), _nbytes(ws), _stream(stream)))
+
+
+def make_decode_items(entries):
+    """ctypes array of pq_decode_item from (desc, X, w_bits, w_scales, A, B, Wr, alpha, beta, Y, ws) tuples of tensors.
+    The array only holds pointers: keep the tensors alive while it is in use."""
+    arr = (pq_decode_item * len(entries))()
+    for i, (d, X, w_bits, w_scales, A, B, Wr, alpha, beta, Y, ws) in enumerate(entries):
+        arr[i].desc = d
+        for name, t in (("X", X), ("w_bits", w_bits), ("w_scales", w_scales), ("A", A), ("B", B), ("Wr", Wr), ("alpha", alpha),
+                        ("beta", beta), ("Y", Y), ("ws", ws)):
+            setattr(arr[i], name, None if t is None else t.data_ptr())
+        arr[i].ws_bytes = _nbytes(ws)
+    return arr
+
+
+def pq_decode_batch(items, stream=None):
+    """Decode forward of independent linears in one launch pair; `items` comes from make_decode_items."""
+    _check("pq_decode_batch", lib().pq_decode_batch(items, len(items), _stream(stream)))
 
 
 def pq_linear_backward(d, dY, X, w_s8, w_scales, A, B, Wr, alpha, beta, saved, dX, dW, dA, dB, dWr, dalpha, dbeta, ws,

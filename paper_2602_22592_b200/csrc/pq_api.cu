@@ -2,6 +2,7 @@
 // workspace buffers, launch sequencing.  No device allocation, no device
 // synchronisation (except pq_device_status, which says so).
 #include <cstring>
+#include <new>
 
 #include "pq_kernels.cuh"
 
@@ -270,21 +271,29 @@ int pq_pack_weights_static(const pq_desc* d, const float* W, uint32_t* w_bits, i
   return pack_static(W, d->N, d->K, w_bits, w_s8, w_scales, static_cast<cudaStream_t>(stream));
 }
 
+static int check_decode_item(const pq_desc* d, const uint16_t* X, const uint32_t* w_bits, const float* w_scales, const uint16_t* A,
+                             const uint16_t* B, const uint16_t* Wr, const float* alpha, const float* beta, const uint16_t* Y, const void* ws,
+                             size_t ws_bytes) {
+  if (!d || !X || !w_scales || !beta || !Y || !w_bits || !ws) return PQ_ERR_NULL;
+  int rc = check_desc(d, false);
+  if (rc) return rc;
+  if (d->T > 16) return PQ_ERR_SHAPE;
+  if (d->r > 0 && (!A || !B || !alpha)) return PQ_ERR_NULL;
+  if (routed(d) && !Wr) return PQ_ERR_NULL;
+  if (misaligned(X) || misaligned(w_bits) || misaligned(A) || misaligned(B) || misaligned(Wr) || misaligned(ws)) return PQ_ERR_ALIGN;
+  if (ws_bytes < decode_workspace_bytes(d->T, d->K, d->N, d->r, (d->flags & PQ_DECODE_DUMP_ACC) != 0)) return PQ_ERR_WORKSPACE;
+  return PQ_OK;
+}
+
 int pq_linear_forward(const pq_desc* d, const uint16_t* X, const uint32_t* w_bits, const int8_t* w_s8, const float* w_scales,
                       const uint16_t* A, const uint16_t* B, const uint16_t* Wr, const float* alpha, const float* beta, uint16_t* Y,
                       void* saved, size_t saved_bytes, void* ws, size_t ws_bytes, void* stream) {
   if (!d || !X || !w_scales || !beta || !Y) return PQ_ERR_NULL;
   if (!w_s8) {
     // decode: a few tokens straight from the packed sign bits
-    if (!w_bits || !ws) return PQ_ERR_NULL;
-    int rc = check_desc(d, false);
+    int rc = check_decode_item(d, X, w_bits, w_scales, A, B, Wr, alpha, beta, Y, ws, ws_bytes);
     if (rc) return rc;
-    if (d->T > 16) return PQ_ERR_SHAPE;
-    if (d->r > 0 && (!A || !B || !alpha)) return PQ_ERR_NULL;
-    if (routed(d) && !Wr) return PQ_ERR_NULL;
-    if (misaligned(X) || misaligned(w_bits) || misaligned(A) || misaligned(B) || misaligned(Wr) || misaligned(ws)) return PQ_ERR_ALIGN;
     const bool dump = (d->flags & PQ_DECODE_DUMP_ACC) != 0;
-    if (ws_bytes < decode_workspace_bytes(d->T, d->K, d->N, d->r, dump)) return PQ_ERR_WORKSPACE;
     LayerArgs a{d->T, d->K, d->N, d->r, experts_of(d), (d->flags & PQ_SCALE_VECTOR) ? 1 : 0, w_scales, alpha, beta, A, B, Wr};
     return decode_forward(a, X, w_bits, Y, ws, dump, static_cast<cudaStream_t>(stream));
   }
@@ -313,6 +322,26 @@ int pq_linear_forward(const pq_desc* d, const uint16_t* X, const uint32_t* w_bit
   if (launch_route_and_quant(X, Wr, d->T, d->K, routed(d) ? E : 1, sv, sc, st) != cudaSuccess) return PQ_ERR_CUDA;
   const uint16_t* xs = routed(d) ? sv.xs : X;
   return gemm_forward(a, w_s8, sv, xs, Y, st);
+}
+
+int pq_decode_batch(const pq_decode_item* items, int n, void* stream) {
+  if (!items) return PQ_ERR_NULL;
+  if (n < 1 || n > 4096) return PQ_ERR_SHAPE;
+  DecodeItemArgs* args = new (std::nothrow) DecodeItemArgs[n];
+  if (!args) return PQ_ERR_CUDA;
+  int rc = PQ_OK;
+  for (int i = 0; i < n && rc == PQ_OK; ++i) {
+    const pq_decode_item& it = items[i];
+    rc = check_decode_item(&it.desc, it.X, it.w_bits, it.w_scales, it.A, it.B, it.Wr, it.alpha, it.beta, it.Y, it.ws, it.ws_bytes);
+    if (rc) break;
+    const pq_desc* d = &it.desc;
+    args[i].a = LayerArgs{d->T, d->K, d->N, d->r, experts_of(d), (d->flags & PQ_SCALE_VECTOR) ? 1 : 0, it.w_scales, it.alpha, it.beta, it.A, it.B, it.Wr};
+    args[i].X = it.X; args[i].bits = it.w_bits; args[i].Y = it.Y; args[i].ws = it.ws;
+    args[i].dump = (d->flags & PQ_DECODE_DUMP_ACC) != 0;
+  }
+  if (rc == PQ_OK) rc = decode_batch(args, n, static_cast<cudaStream_t>(stream));
+  delete[] args;
+  return rc;
 }
 
 int pq_linear_backward(const pq_desc* d, const uint16_t* dY, const uint16_t* X, const int8_t* w_s8, const float* w_scales,

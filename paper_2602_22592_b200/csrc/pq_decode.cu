@@ -2,23 +2,32 @@
 // packed sign bits.  The work is bound by the bytes of the weights (N K / 8 bytes of bits,
 // 2 r (K + N) bytes per expert in use), so the kernels are built around streaming them once:
 //
-//   k_decode_prep  one CTA per (token, slice of the r hidden rows): absmax quantisation of the
-//                  token (Eq. 7-9), router (Sec. 3.3), and its slice of h = A_e x.
-//   k_decode_main  one CTA per SM, each owning a contiguous range of output features: the sign
-//                  bits and the expert rows B_e of that range arrive by bulk copies into shared
-//                  memory; the 1-bit product runs on mma.sync (u8 bit masks x s8 activations,
-//                  exact in int32), the expert product on bf16 mma.sync, and the epilogue forms
+//   k_decode_prep  one CTA per (linear, token, slice of the r hidden rows): absmax quantisation
+//                  of the token (Eq. 7-9), router (Sec. 3.3), and its slice of h = A_e x.
+//   k_decode_main  one CTA per SM, each owning a contiguous range of output features of every
+//                  linear of the batch.  A producer warp streams, linear after linear, the sign
+//                  bits, the activations and the expert rows B_e of that range into shared memory
+//                  by bulk copies (mbarrier full/empty pairs), running ahead of sixteen consumer
+//                  warps: 1-bit product on mma.sync (u8 bit masks x s8 activations, exact in
+//                  int32), expert product on bf16 mma.sync, epilogue
 //                  Y = alpha g (B_e h) + beta (lam / gamma) (q . S)  (Eq. 10-11).
+// A batch is a set of INDEPENDENT linears (the gate and up projections of one block, the q/k/v
+// projections, other sequences): their weights then stream back to back.
 //
 // The sum over k of q S is evaluated as 2 * (sum over the set bits of q) - (sum of q): the bit
 // words feed the tensor cores as 0/1 masks without expansion to +-1.
+#include <algorithm>
+
 #include "pq_kernels.cuh"
 
 namespace pq {
 
-constexpr int kDecodeMainThreads = 512;
+constexpr int kDecodeConsumerWarps = 16;
+constexpr int kDecodeConsumers = 32 * kDecodeConsumerWarps;
+constexpr int kDecodeMainThreads = kDecodeConsumers + 32;   // + the producer warp
 constexpr int kDecodeMaxTokens = 16;
 constexpr int kDecodeRing = 3;          // expert-row buffers in flight per CTA
+constexpr int kDecodeMaxBatch = 16;     // linears per launch (their descriptors travel as kernel parameters)
 
 struct DecodeTokInfo {  // one per token, written by k_decode_prep
   int expert;
@@ -58,17 +67,44 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1
 // stored as 16 bytes at ((group * npairs + ip) * 32 + lane) * 16, group = token / 8.
 // ---------------------------------------------------------------------------
 
-// grid (slices, M), 256 threads, dynamic shared memory: K bf16 values of the token
-__global__ void __launch_bounds__(256) k_decode_prep(const uint4* __restrict__ X, const uint4* __restrict__ Wr, const uint16_t* __restrict__ A,
-                                                     int M, int K, int E, int r, int rows_per_slice, DecodeTokInfo* __restrict__ info,
-                                                     uint4* __restrict__ qfrag, float* __restrict__ H) {
+// One linear of a batch: device pointers and sizes (the workspace pointers are carved by the host).
+struct DecodeLinear {
+  const uint4* X;           // [M, K] bf16
+  const uint4* Wr;          // [E, K] bf16 or null
+  const uint16_t* A;        // [E, r, K]
+  const uint16_t* B;        // [E, N, r]
+  const uint32_t* bits;     // [N, K/32]
+  const float* w_scales;
+  const float* alpha;
+  const float* beta;
+  uint16_t* Y;              // [M, N]
+  DecodeTokInfo* info;      // [16]
+  uint4* qfrag;             // [2, npairs, 32] fragments
+  float* H;                 // [M, r]
+  int* acc_dump;            // [M, N] exact 1-bit accumulators (test hook) or null
+  int M, K, N, r, E, sstride, slices, rows_per_slice;
+};
+struct DecodeBatch {
+  DecodeLinear lin[kDecodeMaxBatch];
+  int n;
+  // shared-memory carve-up of k_decode_main (bytes from the 128-byte aligned base)
+  int slot_bytes, off_slot_h, off_q, off_ring, off_hfrag, off_red, ring_stage_bytes;
+};
+
+// grid (slices, M, linears), 256 threads, dynamic shared memory: K bf16 values of the token
+__global__ void __launch_bounds__(256) k_decode_prep(const __grid_constant__ DecodeBatch bp) {
   extern __shared__ uint4 xs4[];
   __shared__ float red_f[8];
   __shared__ int red_i[8];
   __shared__ float logit_sh[kMaxExperts];
   pdl_launch_dependents();
   pdl_wait();   // X may come from the previous kernel; the buffers written here may still be read by it
+  const DecodeLinear& L = bp.lin[blockIdx.z];
   const int m = blockIdx.y, slice = blockIdx.x;
+  if (m >= L.M || slice >= L.slices) return;
+  const int K = L.K, E = L.E, r = L.r;
+  const uint4* __restrict__ X = L.X;
+  const uint4* __restrict__ Wr = L.Wr;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int chunks = K >> 3;
   const uint4* xrow = X + (long long)m * chunks;
@@ -159,7 +195,7 @@ __global__ void __launch_bounds__(256) k_decode_prep(const uint4* __restrict__ X
         }
         out[c] = make_uint4(w[0], w[1], w[2], w[3]);
       }
-      uint4* dst = qfrag + ((long long)(group * npairs + ip) * 32 + g * 4);
+      uint4* dst = L.qfrag + ((long long)(group * npairs + ip) * 32 + g * 4);
 #pragma unroll
       for (int c = 0; c < 4; ++c) dst[c] = out[c];
     }
@@ -169,15 +205,15 @@ __global__ void __launch_bounds__(256) k_decode_prep(const uint4* __restrict__ X
     if (threadIdx.x == 0) {
       int tot = 0;
       for (int w = 0; w < 8; ++w) tot += red_i[w];
-      info[m] = DecodeTokInfo{best, gate, gamma, tot};
+      L.info[m] = DecodeTokInfo{best, gate, gamma, tot};
     }
   }
 
   // this slice of h = A_e x (fp32 accumulation over the bf16 operands), one warp per row
   if (r > 0) {
-    const int j0 = slice * rows_per_slice, j1 = min(r, j0 + rows_per_slice);
+    const int j0 = slice * L.rows_per_slice, j1 = min(r, j0 + L.rows_per_slice);
     for (int j = j0 + warp; j < j1; j += 8) {
-      const uint4* arow = reinterpret_cast<const uint4*>(A + ((long long)best * r + j) * K);
+      const uint4* arow = reinterpret_cast<const uint4*>(L.A + ((long long)best * r + j) * K);
       float a0 = 0.f, a1 = 0.f;
       for (int c0 = lane; c0 < chunks; c0 += 32 * 8) {
         uint4 wv[8];
@@ -196,26 +232,10 @@ __global__ void __launch_bounds__(256) k_decode_prep(const uint4* __restrict__ X
       }
       float a = a0 + a1;
       for (int d = 16; d > 0; d >>= 1) a += __shfl_xor_sync(0xffffffffu, a, d);
-      if (lane == 0) H[m * r + j] = a;
+      if (lane == 0) L.H[m * r + j] = a;
     }
   }
 }
-
-struct DecodeMainParams {
-  const uint32_t* bits;     // [N, K/32]
-  const uint16_t* B;        // [E, N, r]
-  const DecodeTokInfo* info;
-  const uint4* qfrag;
-  const float* H;           // [M, r]
-  const float* w_scales;
-  const float* alpha;
-  const float* beta;
-  uint16_t* Y;              // [M, N]
-  int* acc_dump;            // [M, N] exact 1-bit accumulators (test hook) or null
-  int M, K, N, r, sstride;
-  // shared-memory carve-up (bytes from the 128-byte aligned base)
-  int off_q, off_ring, off_h, off_red, ring_stage_bytes;
-};
 
 // Range of output features of CTA b: whole groups of 8, spread evenly.
 __device__ __forceinline__ void decode_range(int b, int nctas, int N, int& n_lo, int& n_hi) {
@@ -224,197 +244,265 @@ __device__ __forceinline__ void decode_range(int b, int nctas, int N, int& n_lo,
   n_hi = (int)((long long)(b + 1) * groups / nctas) << 3;
 }
 
-__global__ void __launch_bounds__(kDecodeMainThreads, 1) k_decode_main(const __grid_constant__ DecodeMainParams p) {
-  extern __shared__ __align__(128) uint8_t smem[];
-  __shared__ __align__(8) uint64_t bars[2 + kDecodeRing];   // sign bits, q fragments, expert-row ring
-  __shared__ DecodeTokInfo tok[kDecodeMaxTokens];
-  __shared__ int distinct[2][8], ndistinct[2];
-  __shared__ int fail;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int g = lane >> 2, c = lane & 3;
-  int n_lo, n_hi;
-  decode_range(blockIdx.x, gridDim.x, p.N, n_lo, n_hi);
-  const int ncols = n_hi - n_lo;
-  const int nks = p.K >> 5, npairs = (nks + 1) >> 1;
-  const uint32_t bits_bytes = (uint32_t)ncols * (uint32_t)(p.K >> 3);
-  uint32_t* bits_s = reinterpret_cast<uint32_t*>(smem);
-  const uint32_t bar_bits = smem_u32(&bars[0]), bar_q = smem_u32(&bars[1]);
-  auto ring_bar = [&](int i) { return smem_u32(&bars[2 + i % kDecodeRing]); };
+// Per-linear header the producer leaves in a slot for the consumers.
+struct DecodeMeta {
+  DecodeTokInfo tok[kDecodeMaxTokens];
+  int distinct[2][8];
+  int ndistinct[2];
+};
 
-  if (threadIdx.x == 0) {
-    fail = 0;
-    mbar_init(bar_bits, 1);
-    mbar_init(bar_q, 1);
-    for (int s = 0; s < kDecodeRing; ++s) mbar_init(ring_bar(s), 1);
-    mbar_fence_init();
-    // the sign bits do not depend on the previous kernel: start them before waiting for it
-    if (ncols > 0) {
-      mbar_expect_tx(bar_bits, bits_bytes);
-      bulk_load(smem_u32(bits_s), p.bits + (long long)n_lo * nks, bits_bytes, bar_bits);
+constexpr int kDecodeMetaBytes = 512;   // the header's place at the start of a slot (keeps what follows 16-byte aligned)
+static_assert(sizeof(DecodeMeta) <= kDecodeMetaBytes, "slot header");
+
+// Wait with a bound.  Once any wait of the CTA has run out, every later wait returns at once, so that
+// all threads keep the same control flow and the kernel ends (with an error status and undefined output).
+__device__ __forceinline__ void decode_wait(uint32_t bar, uint32_t parity, volatile int* fail) {
+  if (mbar_try_wait(bar, parity)) return;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (*fail) return;
+    if (clock64() - t0 > kSpinCycles) {
+      report_timeout(WHERE_OTHER);
+      *fail = 1;
+      return;
     }
+  }
+}
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kDecodeConsumers) : "memory"); }
+
+__global__ void __launch_bounds__(kDecodeMainThreads, 1) k_decode_main(const __grid_constant__ DecodeBatch bp) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  // barriers: slot full/empty [2], q full/empty, ring full/empty [kDecodeRing]
+  __shared__ __align__(8) uint64_t bars[4 + 2 + 2 * kDecodeRing];
+  __shared__ int fail_sh;
+  volatile int* fail = &fail_sh;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  auto slot_full = [&](int s) { return smem_u32(&bars[s]); };
+  auto slot_empty = [&](int s) { return smem_u32(&bars[2 + s]); };
+  const uint32_t q_full = smem_u32(&bars[4]), q_empty = smem_u32(&bars[5]);
+  auto ring_full = [&](int i) { return smem_u32(&bars[6 + i % kDecodeRing]); };
+  auto ring_empty = [&](int i) { return smem_u32(&bars[6 + kDecodeRing + i % kDecodeRing]); };
+  if (threadIdx.x == 0) {
+    fail_sh = 0;
+    for (int s = 0; s < 2; ++s) { mbar_init(slot_full(s), 1); mbar_init(slot_empty(s), kDecodeConsumerWarps); }
+    mbar_init(q_full, 1); mbar_init(q_empty, kDecodeConsumerWarps);
+    for (int s = 0; s < kDecodeRing; ++s) { mbar_init(ring_full(s), 1); mbar_init(ring_empty(s), kDecodeConsumerWarps); }
+    mbar_fence_init();
   }
   pdl_launch_dependents();
   pdl_wait();
-  if (threadIdx.x < p.M) tok[threadIdx.x] = p.info[threadIdx.x];
   __syncthreads();
-  const int ngroups = (p.M + 7) >> 3;
-  if (threadIdx.x < ngroups) {
-    // distinct experts of the tokens of this group, in order of first appearance
-    const int G = threadIdx.x;
-    int n = 0;
-    for (int t = 8 * G; t < min(p.M, 8 * G + 8); ++t) {
-      bool seen = false;
-      for (int i = 0; i < n; ++i) seen |= distinct[G][i] == tok[t].expert;
-      if (!seen) distinct[G][n++] = tok[t].expert;
-    }
-    ndistinct[G] = p.r > 0 ? n : 0;
-  }
-  __syncthreads();
-  if (ncols == 0) return;
 
-  const int ntile = (ncols + 15) >> 4;                 // 16-feature tiles of this CTA (<= 8)
-  const int kslices = (kDecodeMainThreads / 32) / ntile; // warps sharing one tile split the contraction
-  const int my_tile = warp % ntile, my_slice = warp / ntile;
-  const bool active = my_slice < kslices;
-  const int row0 = 16 * my_tile + g, row1 = row0 + 8;   // this thread's two features (local index)
-  const bool has0 = row0 < ncols, has1 = row1 < ncols;
-  uint4* q_s = reinterpret_cast<uint4*>(smem + p.off_q);
-  uint8_t* ring = smem + p.off_ring;
-  uint4* h_s = reinterpret_cast<uint4*>(smem + p.off_h);
-  int* red = reinterpret_cast<int*>(smem + p.off_red);
-  const int rsteps = (p.r + 31) >> 5;                   // 32 hidden values per step of the expert product
-  const uint32_t row_bytes = (uint32_t)p.r * 2u;
-  int ring_use = 0;                                      // expert-row loads consumed so far (all groups)
-  int ring_issued = 0;
+  auto slot_ptr = [&](int s) { return smem + (size_t)s * bp.slot_bytes; };   // [meta][bits][H]
+  uint4* q_s = reinterpret_cast<uint4*>(smem + bp.off_q);
+  uint8_t* ring = smem + bp.off_ring;
 
-  for (int G = 0; G < ngroups; ++G) {
-    const int nd = ndistinct[G];
-    if (threadIdx.x == 0) {
-      // activations of this group (already in fragment order) and its first expert rows
-      mbar_expect_tx(bar_q, (uint32_t)npairs * 32u * 16u);
-      bulk_load(smem_u32(q_s), p.qfrag + (long long)G * npairs * 32, (uint32_t)npairs * 32u * 16u, bar_q);
-      for (; ring_issued < ring_use + min(nd, kDecodeRing); ++ring_issued) {
-        const int e = distinct[G][ring_issued - ring_use];
-        mbar_expect_tx(ring_bar(ring_issued), (uint32_t)ncols * row_bytes);
-        bulk_load(smem_u32(ring + (ring_issued % kDecodeRing) * p.ring_stage_bytes), p.B + ((long long)e * p.N + n_lo) * p.r,
-                  (uint32_t)ncols * row_bytes, ring_bar(ring_issued));
+  if (warp == kDecodeConsumerWarps) {
+    // ------------------------------------------------------------------ producer
+    int q_use = 0, ring_use = 0, slot_use[2] = {0, 0};
+    // issue of the slot of linear l: header (token info, distinct experts), sign bits, hidden activations
+    auto issue_slot = [&](int l) {
+      const DecodeLinear& L = bp.lin[l];
+      int n_lo, n_hi;
+      decode_range(blockIdx.x, gridDim.x, L.N, n_lo, n_hi);
+      const int ncols = n_hi - n_lo;
+      if (ncols == 0) return;
+      const int s = l & 1;
+      decode_wait(slot_empty(s), (slot_use[s] & 1) ^ 1, fail);
+      ++slot_use[s];
+      DecodeMeta* meta = reinterpret_cast<DecodeMeta*>(slot_ptr(s));
+      if (lane < L.M) meta->tok[lane] = L.info[lane];
+      __syncwarp();
+      if (lane < 2) {
+        int n = 0;
+        for (int t = 8 * lane; t < min(L.M, 8 * lane + 8); ++t) {
+          bool seen = false;
+          for (int i = 0; i < n; ++i) seen |= meta->distinct[lane][i] == meta->tok[t].expert;
+          if (!seen) meta->distinct[lane][n++] = meta->tok[t].expert;
+        }
+        meta->ndistinct[lane] = L.r > 0 ? n : 0;
+      }
+      __syncwarp();
+      if (lane == 0) {
+        const uint32_t bits_bytes = (uint32_t)ncols * (uint32_t)(L.K >> 3);
+        const uint32_t h_bytes = L.r > 0 ? (uint32_t)(L.M * L.r) * 4u : 0u;
+        mbar_expect_tx(slot_full(s), bits_bytes + h_bytes);     // release: the header written above is visible to the waiters
+        bulk_load(smem_u32(slot_ptr(s) + kDecodeMetaBytes), L.bits + (long long)n_lo * (L.K >> 5), bits_bytes, slot_full(s));
+        if (h_bytes) bulk_load(smem_u32(slot_ptr(s) + bp.off_slot_h), L.H, h_bytes, slot_full(s));
+      }
+    };
+    if (bp.n > 0) issue_slot(0);
+    for (int l = 0; l < bp.n; ++l) {
+      if (l + 1 < bp.n) issue_slot(l + 1);       // the next linear's bits are in flight while this one is consumed
+      const DecodeLinear& L = bp.lin[l];
+      int n_lo, n_hi;
+      decode_range(blockIdx.x, gridDim.x, L.N, n_lo, n_hi);
+      const int ncols = n_hi - n_lo;
+      if (ncols == 0) continue;
+      const DecodeMeta* meta = reinterpret_cast<const DecodeMeta*>(slot_ptr(l & 1));
+      const int npairs = ((L.K >> 5) + 1) >> 1;
+      const uint32_t q_bytes = (uint32_t)npairs * 32u * 16u, row_bytes = (uint32_t)L.r * 2u;
+      const int ngroups = (L.M + 7) >> 3;
+      for (int G = 0; G < ngroups; ++G) {
+        decode_wait(q_empty, (q_use & 1) ^ 1, fail);
+        ++q_use;
+        if (lane == 0) {
+          mbar_expect_tx(q_full, q_bytes);
+          bulk_load(smem_u32(q_s), L.qfrag + (long long)G * npairs * 32, q_bytes, q_full);
+        }
+        const int nd = meta->ndistinct[G];
+        for (int d = 0; d < nd; ++d) {
+          decode_wait(ring_empty(ring_use), ((ring_use / kDecodeRing) & 1) ^ 1, fail);
+          if (lane == 0) {
+            const int e = meta->distinct[G][d];
+            mbar_expect_tx(ring_full(ring_use), (uint32_t)ncols * row_bytes);
+            bulk_load(smem_u32(ring + (ring_use % kDecodeRing) * bp.ring_stage_bytes), L.B + ((long long)e * L.N + n_lo) * L.r,
+                      (uint32_t)ncols * row_bytes, ring_full(ring_use));
+          }
+          ++ring_use;
+        }
       }
     }
-    // hidden activations as bf16 hi + lo fragments
-    for (int i = threadIdx.x; i < rsteps * 32; i += kDecodeMainThreads) {
-      const int s = i >> 5, ln = i & 31, tg = ln >> 2, tc = ln & 3;
-      const int t = 8 * G + tg, j0 = 8 * (4 * s + tc);
-      uint32_t hi[4] = {0, 0, 0, 0}, lo[4] = {0, 0, 0, 0};
-      if (t < p.M) {
-        float v[8];
+    return;
+  }
+
+  // -------------------------------------------------------------------- consumers
+  const int g = lane >> 2, c = lane & 3;
+  uint4* h_s = reinterpret_cast<uint4*>(smem + bp.off_hfrag);
+  int* red = reinterpret_cast<int*>(smem + bp.off_red);
+  int q_use = 0, ring_use = 0, slot_use[2] = {0, 0};
+  for (int l = 0; l < bp.n; ++l) {
+    const DecodeLinear& L = bp.lin[l];
+    int n_lo, n_hi;
+    decode_range(blockIdx.x, gridDim.x, L.N, n_lo, n_hi);
+    const int ncols = n_hi - n_lo;
+    if (ncols == 0) continue;
+    const int s = l & 1;
+    decode_wait(slot_full(s), slot_use[s] & 1, fail);
+    ++slot_use[s];
+    const DecodeMeta* meta = reinterpret_cast<const DecodeMeta*>(slot_ptr(s));
+    const uint32_t* bits_s = reinterpret_cast<const uint32_t*>(slot_ptr(s) + kDecodeMetaBytes);
+    const float* H_s = reinterpret_cast<const float*>(slot_ptr(s) + bp.off_slot_h);
+    const int nks = L.K >> 5, npairs = (nks + 1) >> 1;
+    const int ntile = (ncols + 15) >> 4;                   // 16-feature tiles of this CTA (<= 8)
+    const int kslices = kDecodeConsumerWarps / ntile;      // warps sharing one tile split the contraction
+    const int my_tile = warp % ntile, my_slice = warp / ntile;
+    const bool active = my_slice < kslices;
+    const int row0 = 16 * my_tile + g, row1 = row0 + 8;    // this thread's two features (local index)
+    const bool has0 = row0 < ncols, has1 = row1 < ncols;
+    const int rsteps = (L.r + 31) >> 5;                    // 32 hidden values per step of the expert product
+    const uint32_t row_bytes = (uint32_t)L.r * 2u;
+    const int ngroups = (L.M + 7) >> 3;
+
+    for (int G = 0; G < ngroups; ++G) {
+      const int nd = meta->ndistinct[G];
+      // hidden activations of this group as bf16 hi + lo fragments
+      for (int i = threadIdx.x; i < rsteps * 32; i += kDecodeConsumers) {
+        const int st = i >> 5, ln = i & 31, tg = ln >> 2, tc = ln & 3;
+        const int t = 8 * G + tg, j0 = 8 * (4 * st + tc);
+        uint32_t hi[4] = {0, 0, 0, 0}, lo[4] = {0, 0, 0, 0};
+        if (t < L.M) {
+          float v[8];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) v[u] = j0 + u < p.r ? p.H[t * p.r + j0 + u] : 0.f;
+          for (int u = 0; u < 8; ++u) v[u] = j0 + u < L.r ? H_s[t * L.r + j0 + u] : 0.f;
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            hi[u] = pack_bf16x2(v[2 * u], v[2 * u + 1]);
+            lo[u] = pack_bf16x2(v[2 * u] - bf16lo(hi[u]), v[2 * u + 1] - bf16hi(hi[u]));
+          }
+        }
+        h_s[i] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+        h_s[rsteps * 32 + i] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+      }
+      decode_wait(q_full, q_use & 1, fail);
+      ++q_use;
+
+      // ---- 1-bit product: masked sums, weight 1 and weight 16
+      int acc1[4] = {0, 0, 0, 0}, acc16[4] = {0, 0, 0, 0};
+      if (active) {
+        const int p0 = (int)((long long)my_slice * npairs / kslices), p1 = (int)((long long)(my_slice + 1) * npairs / kslices);
+        const uint32_t* w0 = bits_s + (long long)(has0 ? row0 : 0) * nks;
+        const uint32_t* w1 = bits_s + (long long)(has1 ? row1 : 0) * nks;
+        for (int ip = p0; ip < p1; ++ip) {
+          const uint4 qv = q_s[ip * 32 + lane];
+          const int i0 = 2 * ip, i1 = min(2 * ip + 1, nks - 1);   // an odd word count pairs the last word with zeros of q
+          const uint32_t t00 = w0[i0] >> c, t01 = w0[i1] >> c, t10 = w1[i0] >> c, t11 = w1[i1] >> c;
+          const uint32_t a1[4] = {t00 & 0x01010101u, t10 & 0x01010101u, t01 & 0x01010101u, t11 & 0x01010101u};
+          const uint32_t a16[4] = {t00 & 0x10101010u, t10 & 0x10101010u, t01 & 0x10101010u, t11 & 0x10101010u};
+          mma_u8s8(acc1, a1, qv.x, qv.y);
+          mma_u8s8(acc16, a16, qv.z, qv.w);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(q_empty);                  // this warp is done with the q fragments
+      consumer_sync();                                      // the h fragments are complete
+      // ---- expert product z = B_e h, tokens of other experts masked out
+      float z[4] = {0.f, 0.f, 0.f, 0.f};
+      const int my_tok = 8 * G + g;                          // the token whose h this thread feeds
+      const int my_tok_e = my_tok < L.M ? meta->tok[my_tok].expert : -1;
+      for (int d = 0; d < nd; ++d) {
+        const int stage = ring_use % kDecodeRing;
+        decode_wait(ring_full(ring_use), (ring_use / kDecodeRing) & 1, fail);
+        const int e = meta->distinct[G][d];
+        if (active) {
+          const uint8_t* rows = ring + stage * bp.ring_stage_bytes;
+          const uint4* r0p = reinterpret_cast<const uint4*>(rows + (long long)(has0 ? row0 : 0) * row_bytes);
+          const uint4* r1p = reinterpret_cast<const uint4*>(rows + (long long)(has1 ? row1 : 0) * row_bytes);
+          const bool mine = my_tok_e == e;
+          for (int st = my_slice; st < rsteps; st += kslices) {
+            const int chunk = 4 * st + c;
+            uint4 b0 = make_uint4(0, 0, 0, 0), b1 = b0;
+            if (chunk * 8 < L.r) { b0 = r0p[chunk]; b1 = r1p[chunk]; }
+            uint4 hh = h_s[st * 32 + lane], hl = h_s[rsteps * 32 + st * 32 + lane];
+            if (!mine) { hh = make_uint4(0, 0, 0, 0); hl = hh; }
+            mma_bf16(z, b0.x, b1.x, b0.y, b1.y, hh.x, hh.y);
+            mma_bf16(z, b0.z, b1.z, b0.w, b1.w, hh.z, hh.w);
+            mma_bf16(z, b0.x, b1.x, b0.y, b1.y, hl.x, hl.y);
+            mma_bf16(z, b0.z, b1.z, b0.w, b1.w, hl.z, hl.w);
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(ring_empty(ring_use));   // this warp is done with the buffer
+        ++ring_use;
+      }
+
+      // ---- sum the contraction slices of a tile, then the epilogue (Eq. 10-11)
+      if (active) {
+        int* mine = red + ((my_slice * ntile + my_tile) * 32 + lane) * 8;
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-          hi[u] = pack_bf16x2(v[2 * u], v[2 * u + 1]);
-          lo[u] = pack_bf16x2(v[2 * u] - bf16lo(hi[u]), v[2 * u + 1] - bf16hi(hi[u]));
+          mine[u] = acc1[u] + (acc16[u] >> 4);   // the weight-16 sums are exact multiples of 16
+          mine[4 + u] = __float_as_int(z[u]);
         }
       }
-      h_s[i] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-      h_s[rsteps * 32 + i] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-    }
-    if (threadIdx.x == 0) {   // one thread polls, the rest wait at the barrier
-      if (!mbar_wait(bar_q, G & 1, WHERE_OTHER)) fail = 1;
-      if (G == 0 && !mbar_wait(bar_bits, 0, WHERE_OTHER)) fail = 1;
-    }
-    __syncthreads();
-    if (fail) return;
-
-    // ---- 1-bit product: masked sums, weight 1 and weight 16
-    int acc1[4] = {0, 0, 0, 0}, acc16[4] = {0, 0, 0, 0};
-    if (active) {
-      const int p0 = (int)((long long)my_slice * npairs / kslices), p1 = (int)((long long)(my_slice + 1) * npairs / kslices);
-      const uint32_t* w0 = bits_s + (long long)(has0 ? row0 : 0) * nks;
-      const uint32_t* w1 = bits_s + (long long)(has1 ? row1 : 0) * nks;
-      for (int ip = p0; ip < p1; ++ip) {
-        const uint4 qv = q_s[ip * 32 + lane];
-        const int i0 = 2 * ip, i1 = min(2 * ip + 1, nks - 1);   // an odd word count pairs the last word with zeros of q
-        const uint32_t t00 = w0[i0] >> c, t01 = w0[i1] >> c, t10 = w1[i0] >> c, t11 = w1[i1] >> c;
-        const uint32_t a1[4] = {t00 & 0x01010101u, t10 & 0x01010101u, t01 & 0x01010101u, t11 & 0x01010101u};
-        const uint32_t a16[4] = {t00 & 0x10101010u, t10 & 0x10101010u, t01 & 0x10101010u, t11 & 0x10101010u};
-        mma_u8s8(acc1, a1, qv.x, qv.y);
-        mma_u8s8(acc16, a16, qv.z, qv.w);
-      }
-    }
-    // ---- expert product z = B_e h, tokens of other experts masked out
-    float z[4] = {0.f, 0.f, 0.f, 0.f};
-    const int my_tok = 8 * G + g;                          // the token whose h this thread feeds
-    const int my_tok_e = my_tok < p.M ? tok[my_tok].expert : -1;
-    for (int d = 0; d < nd; ++d) {
-      const int use = ring_use + d, stage = use % kDecodeRing;
-      if (threadIdx.x == 0 && !mbar_wait(ring_bar(use), (use / kDecodeRing) & 1, WHERE_OTHER)) fail = 1;
-      __syncthreads();
-      if (fail) return;
-      const int e = distinct[G][d];
-      if (active) {
-        const uint8_t* rows = ring + stage * p.ring_stage_bytes;
-        const uint4* r0p = reinterpret_cast<const uint4*>(rows + (long long)(has0 ? row0 : 0) * row_bytes);
-        const uint4* r1p = reinterpret_cast<const uint4*>(rows + (long long)(has1 ? row1 : 0) * row_bytes);
-        const bool mine = my_tok_e == e;
-        for (int s = my_slice; s < rsteps; s += kslices) {
-          const int chunk = 4 * s + c;
-          uint4 b0 = make_uint4(0, 0, 0, 0), b1 = b0;
-          if (chunk * 8 < p.r) { b0 = r0p[chunk]; b1 = r1p[chunk]; }
-          uint4 hh = h_s[s * 32 + lane], hl = h_s[rsteps * 32 + s * 32 + lane];
-          if (!mine) { hh = make_uint4(0, 0, 0, 0); hl = hh; }
-          mma_bf16(z, b0.x, b1.x, b0.y, b1.y, hh.x, hh.y);
-          mma_bf16(z, b0.z, b1.z, b0.w, b1.w, hh.z, hh.w);
-          mma_bf16(z, b0.x, b1.x, b0.y, b1.y, hl.x, hl.y);
-          mma_bf16(z, b0.z, b1.z, b0.w, b1.w, hl.z, hl.w);
-        }
-      }
-      if (nd > kDecodeRing) {   // more experts than buffers: refill this one once every warp is done with it
-        __syncthreads();
-        if (threadIdx.x == 0 && ring_issued < ring_use + nd) {
-          const int en = distinct[G][ring_issued - ring_use];
-          mbar_expect_tx(ring_bar(ring_issued), (uint32_t)ncols * row_bytes);
-          bulk_load(smem_u32(ring + (ring_issued % kDecodeRing) * p.ring_stage_bytes), p.B + ((long long)en * p.N + n_lo) * p.r,
-                    (uint32_t)ncols * row_bytes, ring_bar(ring_issued));
-          ++ring_issued;
-        }
-      }
-    }
-    ring_use += nd;
-
-    // ---- sum the contraction slices of a tile, then the epilogue (Eq. 10-11)
-    if (active) {
-      int* mine = red + ((my_slice * ntile + my_tile) * 32 + lane) * 8;
+      consumer_sync();
+      if (active && my_slice == 0) {
+        int ms[4] = {0, 0, 0, 0};
+        float zz[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int sl = 0; sl < kslices; ++sl) {
+          const int* part = red + ((sl * ntile + my_tile) * 32 + lane) * 8;
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        mine[u] = acc1[u] + (acc16[u] >> 4);   // the weight-16 sums are exact multiples of 16
-        mine[4 + u] = __float_as_int(z[u]);
-      }
-    }
-    __syncthreads();
-    if (active && my_slice == 0) {
-      int ms[4] = {0, 0, 0, 0};
-      float zz[4] = {0.f, 0.f, 0.f, 0.f};
-      for (int s = 0; s < kslices; ++s) {
-        const int* part = red + ((s * ntile + my_tile) * 32 + lane) * 8;
+          for (int u = 0; u < 4; ++u) { ms[u] += part[u]; zz[u] += __int_as_float(part[4 + u]); }
+        }
+        const float lam = L.w_scales[0];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) { ms[u] += part[u]; zz[u] += __int_as_float(part[4 + u]); }
-      }
-      const float lam = p.w_scales[0];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        // accumulator u: feature row0 (u < 2) or row1, token 8G + 2c + (u & 1)
-        const int nl = (u < 2) ? row0 : row1, t = 8 * G + 2 * c + (u & 1);
-        if (nl < ncols && t < p.M) {
-          const int n = n_lo + nl;
-          const int acc = 2 * ms[u] - tok[t].rowsum;
-          float y = p.beta[n * p.sstride] * __fdiv_rn(lam, tok[t].gamma) * (float)acc;
-          if (p.r > 0) y = fmaf(p.alpha[n * p.sstride] * tok[t].gate, zz[u], y);
-          p.Y[(long long)t * p.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(y));
-          if (p.acc_dump) p.acc_dump[(long long)t * p.N + n] = acc;
+        for (int u = 0; u < 4; ++u) {
+          // accumulator u: feature row0 (u < 2) or row1, token 8G + 2c + (u & 1)
+          const int nl = (u < 2) ? row0 : row1, t = 8 * G + 2 * c + (u & 1);
+          if (nl < ncols && t < L.M) {
+            const int n = n_lo + nl;
+            const int acc = 2 * ms[u] - meta->tok[t].rowsum;
+            float y = L.beta[n * L.sstride] * __fdiv_rn(lam, meta->tok[t].gamma) * (float)acc;
+            if (L.r > 0) y = fmaf(L.alpha[n * L.sstride] * meta->tok[t].gate, zz[u], y);
+            L.Y[(long long)t * L.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(y));
+            if (L.acc_dump) L.acc_dump[(long long)t * L.N + n] = acc;
+          }
         }
       }
+      consumer_sync();   // the h fragments and the reduction buffer are rewritten by the next group
     }
-    __syncthreads();   // q, h and the reduction buffer are rewritten by the next group
+    __syncwarp();
+    if (lane == 0) mbar_arrive(slot_empty(s));               // this warp is done with the slot of linear l
   }
 }
 
@@ -454,51 +542,61 @@ static int decode_sm_count() {
   return n;
 }
 
-int decode_forward(const LayerArgs& a, const uint16_t* X, const uint32_t* bits, uint16_t* Y, void* ws, bool dump, cudaStream_t st) {
-  const int M = a.T, K = a.K, N = a.N, r = a.r, E = a.E;
-  uint8_t* w = static_cast<uint8_t*>(ws);
-  const size_t npairs = ((size_t)K / 32 + 1) / 2;
-  DecodeTokInfo* info = reinterpret_cast<DecodeTokInfo*>(w);
-  w += up256(sizeof(DecodeTokInfo) * kDecodeMaxTokens);
-  uint4* qfrag = reinterpret_cast<uint4*>(w);
-  w += up256(2 * npairs * 32 * sizeof(uint4));
-  float* H = reinterpret_cast<float*>(w);
-  w += up256(sizeof(float) * kDecodeMaxTokens * (size_t)(r > 0 ? r : 1));
-  int* acc_dump = dump ? reinterpret_cast<int*>(w) : nullptr;
-
+// One launch pair for up to kDecodeMaxBatch independent linears.
+static int decode_launch(const DecodeItemArgs* items, int n, cudaStream_t st) {
   static int sms = decode_sm_count();
-  const int groups = N / 8;
-  const int nctas = groups < sms ? groups : sms;
-  const int max_cols = ((groups + nctas - 1) / nctas) * 8;
-  if (max_cols > 128) return PQ_ERR_UNSUPPORTED;   // 16 warps cover at most 8 tiles of 16 features
-
-  DecodeMainParams p{};
-  p.bits = bits; p.B = a.B; p.info = info; p.qfrag = qfrag; p.H = H; p.w_scales = a.w_scales; p.alpha = a.alpha; p.beta = a.beta;
-  p.Y = Y; p.acc_dump = acc_dump; p.M = M; p.K = K; p.N = N; p.r = r; p.sstride = a.scale_stride;
-  size_t off = up256((size_t)max_cols * (K / 8));
-  p.off_q = (int)off; off += up256(npairs * 32 * sizeof(uint4));
-  p.ring_stage_bytes = (int)up256((size_t)max_cols * r * 2);
-  p.off_ring = (int)off; off += (size_t)kDecodeRing * p.ring_stage_bytes;
-  const int rsteps = (r + 31) / 32;
-  p.off_h = (int)off; off += up256((size_t)2 * (rsteps > 0 ? rsteps : 1) * 32 * sizeof(uint4));
-  p.off_red = (int)off; off += (size_t)(kDecodeMainThreads / 32) * 32 * 8 * sizeof(int);
-  const size_t smem_main = off + 128;
-  if (smem_main > 227 * 1024) return PQ_ERR_UNSUPPORTED;
-  const size_t smem_prep = (size_t)K * 2;
-  if (smem_prep > 200 * 1024) return PQ_ERR_UNSUPPORTED;
-  if (cudaFuncSetAttribute(k_decode_main, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_main) != cudaSuccess) return PQ_ERR_CUDA;
-  if (cudaFuncSetAttribute(k_decode_prep, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_prep) != cudaSuccess) return PQ_ERR_CUDA;
-
-  // slices of the hidden rows: enough CTAs to pull A_e at full rate, at least one row per warp
-  int slices = 1, rows_per_slice = 1;
-  if (r > 0) {
-    slices = 2 * sms / M;
-    const int max_slices = (r + 7) / 8;
-    if (slices > max_slices) slices = max_slices;
-    if (slices < 1) slices = 1;
-    rows_per_slice = (r + slices - 1) / slices;
-    slices = (r + rows_per_slice - 1) / rows_per_slice;
+  DecodeBatch bp{};
+  bp.n = n;
+  size_t slot_bits = 0, slot_h = 0, q_bytes = 0, ring_stage = 0, hfrag = 0, prep_smem = 0;
+  int max_slices = 1, max_m = 1;
+  for (int i = 0; i < n; ++i) {
+    const DecodeItemArgs& it = items[i];
+    const int M = it.a.T, K = it.a.K, N = it.a.N, r = it.a.r;
+    DecodeLinear& L = bp.lin[i];
+    uint8_t* w = static_cast<uint8_t*>(it.ws);
+    const size_t npairs = ((size_t)K / 32 + 1) / 2;
+    L.info = reinterpret_cast<DecodeTokInfo*>(w); w += up256(sizeof(DecodeTokInfo) * kDecodeMaxTokens);
+    L.qfrag = reinterpret_cast<uint4*>(w); w += up256(2 * npairs * 32 * sizeof(uint4));
+    L.H = reinterpret_cast<float*>(w); w += up256(sizeof(float) * kDecodeMaxTokens * (size_t)(r > 0 ? r : 1));
+    L.acc_dump = it.dump ? reinterpret_cast<int*>(w) : nullptr;
+    L.X = reinterpret_cast<const uint4*>(it.X); L.Wr = reinterpret_cast<const uint4*>(it.a.Wr); L.A = it.a.A; L.B = it.a.B;
+    L.bits = it.bits; L.w_scales = it.a.w_scales; L.alpha = it.a.alpha; L.beta = it.a.beta; L.Y = it.Y;
+    L.M = M; L.K = K; L.N = N; L.r = r; L.E = (r > 0 && it.a.E > 1) ? it.a.E : 1; L.sstride = it.a.scale_stride;
+    // slices of the hidden rows: enough CTAs to pull A_e at full rate, at least one row per warp
+    L.slices = 1; L.rows_per_slice = 1;
+    if (r > 0) {
+      int slices = 2 * sms / (M * n);
+      const int most = (r + 7) / 8;
+      if (slices > most) slices = most;
+      if (slices < 1) slices = 1;
+      L.rows_per_slice = (r + slices - 1) / slices;
+      L.slices = (r + L.rows_per_slice - 1) / L.rows_per_slice;
+    }
+    if (L.slices > max_slices) max_slices = L.slices;
+    if (M > max_m) max_m = M;
+    const int groups = N / 8;
+    const int max_cols = ((groups + sms - 1) / sms) * 8;
+    if (max_cols > 128) return PQ_ERR_UNSUPPORTED;   // 16 warps cover at most 8 tiles of 16 features
+    slot_bits = std::max(slot_bits, up256((size_t)max_cols * (K / 8)));
+    slot_h = std::max(slot_h, up256((size_t)kDecodeMaxTokens * (r > 0 ? r : 1) * 4));
+    q_bytes = std::max(q_bytes, up256(npairs * 32 * sizeof(uint4)));
+    ring_stage = std::max(ring_stage, up256((size_t)max_cols * r * 2));
+    hfrag = std::max(hfrag, up256((size_t)2 * std::max((r + 31) / 32, 1) * 32 * sizeof(uint4)));
+    prep_smem = std::max(prep_smem, (size_t)K * 2);
   }
+  const size_t meta = kDecodeMetaBytes;
+  bp.off_slot_h = (int)(meta + slot_bits);
+  bp.slot_bytes = (int)(meta + slot_bits + slot_h);
+  size_t off = 2 * (size_t)bp.slot_bytes;
+  bp.off_q = (int)off; off += q_bytes;
+  bp.ring_stage_bytes = (int)ring_stage;
+  bp.off_ring = (int)off; off += kDecodeRing * ring_stage;
+  bp.off_hfrag = (int)off; off += hfrag;
+  bp.off_red = (int)off; off += (size_t)kDecodeConsumerWarps * 32 * 8 * sizeof(int);
+  const size_t smem_main = off + 128;
+  if (smem_main > 227 * 1024 || prep_smem > 200 * 1024) return PQ_ERR_UNSUPPORTED;
+  if (cudaFuncSetAttribute(k_decode_main, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_main) != cudaSuccess) return PQ_ERR_CUDA;
+  if (cudaFuncSetAttribute(k_decode_prep, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)prep_smem) != cudaSuccess) return PQ_ERR_CUDA;
 
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -506,18 +604,30 @@ int decode_forward(const LayerArgs& a, const uint16_t* X, const uint32_t* bits, 
   cudaLaunchConfig_t cfg{};
   cfg.stream = st; cfg.attrs = attr; cfg.numAttrs = g_decode_pdl ? 1 : 0;
   {
-    cfg.gridDim = dim3(slices, M, 1); cfg.blockDim = dim3(256, 1, 1); cfg.dynamicSmemBytes = smem_prep;
+    cfg.gridDim = dim3(max_slices, max_m, n); cfg.blockDim = dim3(256, 1, 1); cfg.dynamicSmemBytes = prep_smem;
     LaunchScope ls(KID_DECODE_PREP, st);
-    if (cudaLaunchKernelEx(&cfg, k_decode_prep, reinterpret_cast<const uint4*>(X), reinterpret_cast<const uint4*>(a.Wr), a.A, M, K,
-                           (r > 0 && E > 1) ? E : 1, r, rows_per_slice, info, qfrag, H) != cudaSuccess)
-      return PQ_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, k_decode_prep, bp) != cudaSuccess) return PQ_ERR_CUDA;
   }
   {
-    cfg.gridDim = dim3(nctas, 1, 1); cfg.blockDim = dim3(kDecodeMainThreads, 1, 1); cfg.dynamicSmemBytes = smem_main;
+    cfg.gridDim = dim3(sms, 1, 1); cfg.blockDim = dim3(kDecodeMainThreads, 1, 1); cfg.dynamicSmemBytes = smem_main;
     LaunchScope ls(KID_DECODE_MAIN, st);
-    if (cudaLaunchKernelEx(&cfg, k_decode_main, p) != cudaSuccess) return PQ_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, k_decode_main, bp) != cudaSuccess) return PQ_ERR_CUDA;
   }
   return PQ_OK;
+}
+
+int decode_batch(const DecodeItemArgs* items, int n, cudaStream_t st) {
+  for (int i = 0; i < n; i += kDecodeMaxBatch) {
+    const int m = n - i < kDecodeMaxBatch ? n - i : kDecodeMaxBatch;
+    const int rc = decode_launch(items + i, m, st);
+    if (rc) return rc;
+  }
+  return PQ_OK;
+}
+
+int decode_forward(const LayerArgs& a, const uint16_t* X, const uint32_t* bits, uint16_t* Y, void* ws, bool dump, cudaStream_t st) {
+  DecodeItemArgs it{a, X, bits, Y, ws, dump};
+  return decode_launch(&it, 1, st);
 }
 
 }  // namespace pq

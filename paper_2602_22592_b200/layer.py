@@ -87,6 +87,10 @@ class PQLinear:
                               self.alpha, self.beta, self.Y if Y is None else Y, None, self.ws_decode)
         return self.Y if Y is None else Y
 
+    def decode_entry(self):
+        """This layer's arguments as one entry for binding.make_decode_items."""
+        return (self.desc, self.X, self.w_bits, self.w_scales, self.A, self.B, self.Wr, self.alpha, self.beta, self.Y, self.ws_decode)
+
     def decode_view(self) -> dict:
         return pqb.pq_decode_view_init(self.desc, self.ws_decode)
 

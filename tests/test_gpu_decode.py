@@ -89,6 +89,35 @@ def test_decode_is_deterministic_and_repeatable():
     assert torch.equal(y, L.Y)
 
 
+def test_decode_batch_of_independent_linears():
+    # a mixed batch (different shapes, token counts, expert counts; more than one launch group of 16)
+    # gives exactly what the separate calls give, and matches the oracle
+    shapes = [dict(T=1, K=256, N=96, r=32, E=4), dict(T=16, K=512, N=2048, r=64, E=8), dict(T=5, K=2080, N=992, r=40, E=3),
+              dict(T=3, K=1024, N=64, r=0, E=0), dict(T=9, K=384, N=320, r=160, E=1)]
+    layers, cases = [], []
+    for i in range(19):
+        kw = dict(shapes[i % len(shapes)])
+        c = I.make_linear_case(kw["T"], kw["K"], kw["N"], kw["r"], kw["E"], seed=40 + i, exact_quota=False, with_grad=False)
+        L = PQLinear(c["T"], c["K"], c["N"], c["r"], c["E"], training=False, dump_acc=True).load_case(c)
+        L.pack(bits_only=True)
+        layers.append(L)
+        cases.append(c)
+    singles = []
+    for L in layers:
+        L.decode()
+        torch.cuda.synchronize()
+        singles.append(L.Y.clone())
+        L.Y.zero_()
+    items = pqb.make_decode_items([L.decode_entry() for L in layers])
+    pqb.pq_decode_batch(items)
+    torch.cuda.synchronize()
+    check_status()
+    for L, y, c in zip(layers, singles, cases):
+        assert torch.equal(L.Y, y)
+    for L, c in list(zip(layers, cases))[:5]:
+        check_decode(c, L)
+
+
 def test_decode_rejects_too_many_tokens():
     L = PQLinear(32, 256, 256, 32, 2, training=False)
     c = I.make_linear_case(32, 256, 256, 32, 2, seed=1, with_grad=False)
