@@ -298,7 +298,9 @@ DECODE_LAYERS = 26   # depth of the 3B-shaped decoder whose MLP projections form
 def run_decode(args):
     """Decode linears from packed 1-bit weights: 26 layers x (gate, up, down) of a 3B-shaped model, all with
     distinct weights (far more bytes than L2), M tokens each, replayed as one CUDA graph.  The figure of merit
-    is the algorithmic bytes of the weights that must be read, per second, against the measured HBM rate."""
+    is the algorithmic bytes of the weights that must be read, per second, against the measured HBM rate.
+    Headline: the linears treated as independent and handed to pq_decode_batch in groups; beside it the same
+    pass with one call per linear (dependent layers) and in groups of two."""
     import torch
     from paper_2602_22592_b200 import binding as pqb
     from paper_2602_22592_b200 import build as pqbuild
@@ -359,24 +361,20 @@ def run_decode(args):
     for L in layers:
         experts = L.decode_view()["expert"].cpu().numpy()
         algo += L.N * L.K // 8 + 4 + len(set(experts.tolist())) * 2 * r * (L.K + L.N) + 2 * E * L.K + 2 * M * L.K + 2 * M * L.N
-    def capture(nstreams):
-        """One CUDA graph of the whole pass.  nstreams = 1: every linear after the previous one, as the layers of a
-        decoder depend on each other.  nstreams > 1: the linears are dealt round-robin onto that many branches, so that
-        independent linears (other sequences, parallel projections) overlap and the weights stream back to back."""
-        side = [torch.cuda.Stream(device=device) for _ in range(nstreams)] if nstreams > 1 else []
+    def capture(batch):
+        """One CUDA graph of the whole pass.  batch = 1: one call per linear, each after the previous one, as the
+        layers of a decoder depend on each other.  batch > 1: pq_decode_batch over groups of `batch` consecutive
+        linears, treated as independent (other sequences, parallel projections), so their weights stream back to back."""
         g = torch.cuda.CUDAGraph()
+        keep = []
         with torch.cuda.graph(g):
-            if not side:
+            if batch <= 1:
                 step()
             else:
-                cur = torch.cuda.current_stream()
-                for si, st in enumerate(side):
-                    st.wait_stream(cur)
-                    with torch.cuda.stream(st):
-                        for L in layers[si::nstreams]:
-                            L.decode()
-                for st in side:
-                    cur.wait_stream(st)
+                for i in range(0, len(layers), batch):
+                    items = pqb.make_decode_items([L.decode_entry() for L in layers[i:i + batch]])
+                    keep.append(items)
+                    pqb.pq_decode_batch(items)
         return g
 
     def time_graph(g):
@@ -397,11 +395,13 @@ def run_decode(args):
         return ms
 
     launches0 = pqb.pq_kernel_launches()
-    graph_serial = capture(1)
+    graph = capture(args.decode_batch)
     launches_per_step = pqb.pq_kernel_launches() - launches0
-    graph = capture(args.decode_streams)
+    graph_serial = capture(1)
+    graph_pairs = capture(2)
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ms_serial = time_graph(graph_serial)
+    ms_pairs = time_graph(graph_pairs)
     with ClockSampler(local) as clk:
         ms_per_step = time_graph(graph)
     code, where = pqb.pq_device_status()
@@ -447,14 +447,17 @@ def run_decode(args):
             "config": {"workload": (f"decode, {M} token(s): {DECODE_LAYERS} layers x gate/up/down of a 3B-shaped model (hidden {hid}, FFN {ffn}), "
                                     f"1-bit weights packed 32 per word, {E} bf16 experts of width {r}, top-1, Zipf(1.1)"),
                        "linears_per_step": nlin, "l2": f"{algo / 1e6:.0f} MB of distinct weights per step, larger than L2",
-                       "launch": f"one CUDA graph per step, {args.decode_streams} independent linears in flight", "replicas": world},
+                       "launch": f"one CUDA graph per step, pq_decode_batch over groups of {args.decode_batch} independent linears", "replicas": world},
             "roofline": {"kernel": "k_decode_prep + k_decode_main (all launches of a step)", "bound": "hbm", "achieved": round(gbs, 1),
                          "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(gbs / peaks["hbm_gbs"], 4),
                          "peak_source": f"{peak_kind} hbm_gbs", "algorithmic_bytes_per_step": int(algo),
                          "us_per_linear": round(ms_per_step * 1e3 / nlin, 3), "traffic": None},
             "serial": {"ms_per_step": round(ms_serial, 4), "us_per_linear": round(ms_serial * 1e3 / nlin, 3),
                        "hbm_frac": round(algo / (ms_serial * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
-                       "note": "the same pass with every linear launched after the previous one has finished (dependent layers)"},
+                       "note": "the same pass with one call per linear, each after the previous one has finished (dependent layers)"},
+            "pairs": {"ms_per_step": round(ms_pairs, 4), "us_per_linear": round(ms_pairs * 1e3 / nlin, 3),
+                      "hbm_frac": round(algo / (ms_pairs * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
+                      "note": "batches of two (what the gate and up projections of one block allow)"},
             "eager_ms_per_step": round(ms_eager, 4),
             "cpu_baseline": None,
             "e2e": {"value": round(world * M * nlin / (ms_e2e * 1e-3), 1), "unit": "token-linears/s",
@@ -532,7 +535,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="mlp_dense", choices=["mlp_dense", "mlp_e8", "decode"])
     ap.add_argument("--decode-tokens", type=int, default=1, choices=range(1, 17), metavar="M")
-    ap.add_argument("--decode-streams", type=int, default=8, help="independent decode linears in flight (graph branches)")
+    ap.add_argument("--decode-batch", type=int, default=16, help="independent decode linears per pq_decode_batch call")
     ap.add_argument("--cpu-tokens", type=int, default=4096)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")

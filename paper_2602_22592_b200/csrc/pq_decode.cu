@@ -80,7 +80,7 @@ struct DecodeLinear {
   uint16_t* Y;              // [M, N]
   DecodeTokInfo* info;      // [16]
   uint4* qfrag;             // [2, npairs, 32] fragments
-  float* H;                 // [M, r]
+  uint4* hfrag;             // [2 groups][2 planes (hi, lo)][ceil(r/32)][32] fragments of h = A_e x
   int* acc_dump;            // [M, N] exact 1-bit accumulators (test hook) or null
   int M, K, N, r, E, sstride, slices, rows_per_slice;
 };
@@ -88,7 +88,7 @@ struct DecodeBatch {
   DecodeLinear lin[kDecodeMaxBatch];
   int n;
   // shared-memory carve-up of k_decode_main (bytes from the 128-byte aligned base)
-  int slot_bytes, off_slot_h, off_q, off_ring, off_hfrag, off_red, ring_stage_bytes;
+  int slot_bytes, off_slot_h, off_q, off_ring, off_red, ring_stage_bytes;
 };
 
 // grid (slices, M, linears), 256 threads, dynamic shared memory: K bf16 values of the token
@@ -232,7 +232,16 @@ __global__ void __launch_bounds__(256) k_decode_prep(const __grid_constant__ Dec
       }
       float a = a0 + a1;
       for (int d = 16; d > 0; d >>= 1) a += __shfl_xor_sync(0xffffffffu, a, d);
-      if (lane == 0) L.H[m * r + j] = a;
+      if (lane == 0) {
+        // element (token m, hidden index j) of the expert product's token-side operand: step j / 32, lane
+        // 4 (m % 8) + (j % 32) / 8, 16-bit slot j % 8; hi = bf16(a), lo = bf16(a - hi)
+        const int rsteps = (r + 31) >> 5;
+        const __nv_bfloat16 hi = __float2bfloat16_rn(a), lo = __float2bfloat16_rn(a - __bfloat162float(hi));
+        uint16_t* base = reinterpret_cast<uint16_t*>(L.hfrag);
+        const long long pos = ((long long)((m >> 3) * 2 * rsteps + (j >> 5)) * 32 + (m & 7) * 4 + ((j & 31) >> 3)) * 8 + (j & 7);
+        base[pos] = __bfloat16_as_ushort(hi);
+        base[pos + (long long)rsteps * 32 * 8] = __bfloat16_as_ushort(lo);
+      }
     }
   }
 }
@@ -244,15 +253,7 @@ __device__ __forceinline__ void decode_range(int b, int nctas, int N, int& n_lo,
   n_hi = (int)((long long)(b + 1) * groups / nctas) << 3;
 }
 
-// Per-linear header the producer leaves in a slot for the consumers.
-struct DecodeMeta {
-  DecodeTokInfo tok[kDecodeMaxTokens];
-  int distinct[2][8];
-  int ndistinct[2];
-};
-
-constexpr int kDecodeMetaBytes = 512;   // the header's place at the start of a slot (keeps what follows 16-byte aligned)
-static_assert(sizeof(DecodeMeta) <= kDecodeMetaBytes, "slot header");
+constexpr int kDecodeMetaBytes = 256;   // token info at the start of a slot
 
 // Wait with a bound.  Once any wait of the CTA has run out, every later wait returns at once, so that
 // all threads keep the same control flow and the kernel ends (with an error status and undefined output).
@@ -269,6 +270,23 @@ __device__ __forceinline__ void decode_wait(uint32_t bar, uint32_t parity, volat
   }
 }
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kDecodeConsumers) : "memory"); }
+
+// Distinct experts of the tokens [8 G, 8 G + 8) in order of first appearance (every thread computes its own copy).
+__device__ __forceinline__ int decode_distinct(const DecodeTokInfo* tok, int M, int G, int (&list)[8]) {
+  int n = 0;
+  for (int t = 8 * G; t < min(M, 8 * G + 8); ++t) {
+    const int e = tok[t].expert;
+    bool seen = false;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) seen |= (i < n) && list[i] == e;
+    if (!seen) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) if (i == n) list[i] = e;
+      ++n;
+    }
+  }
+  return n;
+}
 
 __global__ void __launch_bounds__(kDecodeMainThreads, 1) k_decode_main(const __grid_constant__ DecodeBatch bp) {
   extern __shared__ __align__(128) uint8_t smem[];
@@ -293,14 +311,15 @@ __global__ void __launch_bounds__(kDecodeMainThreads, 1) k_decode_main(const __g
   pdl_wait();
   __syncthreads();
 
-  auto slot_ptr = [&](int s) { return smem + (size_t)s * bp.slot_bytes; };   // [meta][bits][H]
+  // a slot holds, for one linear: token info | sign bits of this CTA's features | h fragments (both groups)
+  auto slot_ptr = [&](int s) { return smem + (size_t)s * bp.slot_bytes; };
   uint4* q_s = reinterpret_cast<uint4*>(smem + bp.off_q);
   uint8_t* ring = smem + bp.off_ring;
 
   if (warp == kDecodeConsumerWarps) {
-    // ------------------------------------------------------------------ producer
-    int q_use = 0, ring_use = 0, slot_use[2] = {0, 0};
-    // issue of the slot of linear l: header (token info, distinct experts), sign bits, hidden activations
+    // ------------------------------------------------------------------ producer (one thread issues everything)
+    if (lane != 0) return;
+    int q_use = 0, ring_use = 0, slot_use[2] = {0, 0}, slot_seen[2] = {0, 0};
     auto issue_slot = [&](int l) {
       const DecodeLinear& L = bp.lin[l];
       int n_lo, n_hi;
@@ -310,57 +329,51 @@ __global__ void __launch_bounds__(kDecodeMainThreads, 1) k_decode_main(const __g
       const int s = l & 1;
       decode_wait(slot_empty(s), (slot_use[s] & 1) ^ 1, fail);
       ++slot_use[s];
-      DecodeMeta* meta = reinterpret_cast<DecodeMeta*>(slot_ptr(s));
-      if (lane < L.M) meta->tok[lane] = L.info[lane];
-      __syncwarp();
-      if (lane < 2) {
-        int n = 0;
-        for (int t = 8 * lane; t < min(L.M, 8 * lane + 8); ++t) {
-          bool seen = false;
-          for (int i = 0; i < n; ++i) seen |= meta->distinct[lane][i] == meta->tok[t].expert;
-          if (!seen) meta->distinct[lane][n++] = meta->tok[t].expert;
-        }
-        meta->ndistinct[lane] = L.r > 0 ? n : 0;
-      }
-      __syncwarp();
-      if (lane == 0) {
-        const uint32_t bits_bytes = (uint32_t)ncols * (uint32_t)(L.K >> 3);
-        const uint32_t h_bytes = L.r > 0 ? (uint32_t)(L.M * L.r) * 4u : 0u;
-        mbar_expect_tx(slot_full(s), bits_bytes + h_bytes);     // release: the header written above is visible to the waiters
-        bulk_load(smem_u32(slot_ptr(s) + kDecodeMetaBytes), L.bits + (long long)n_lo * (L.K >> 5), bits_bytes, slot_full(s));
-        if (h_bytes) bulk_load(smem_u32(slot_ptr(s) + bp.off_slot_h), L.H, h_bytes, slot_full(s));
-      }
+      const uint32_t bits_bytes = (uint32_t)ncols * (uint32_t)(L.K >> 3);
+      const uint32_t h_bytes = L.r > 0 ? (uint32_t)(((L.M + 7) >> 3) * 2 * ((L.r + 31) >> 5)) * 512u : 0u;
+      mbar_expect_tx(slot_full(s), kDecodeMetaBytes + bits_bytes + h_bytes);
+      bulk_load(smem_u32(slot_ptr(s)), L.info, kDecodeMetaBytes, slot_full(s));
+      bulk_load(smem_u32(slot_ptr(s) + kDecodeMetaBytes), L.bits + (long long)n_lo * (L.K >> 5), bits_bytes, slot_full(s));
+      if (h_bytes) bulk_load(smem_u32(slot_ptr(s) + bp.off_slot_h), L.hfrag, h_bytes, slot_full(s));
     };
     if (bp.n > 0) issue_slot(0);
     for (int l = 0; l < bp.n; ++l) {
-      if (l + 1 < bp.n) issue_slot(l + 1);       // the next linear's bits are in flight while this one is consumed
       const DecodeLinear& L = bp.lin[l];
       int n_lo, n_hi;
       decode_range(blockIdx.x, gridDim.x, L.N, n_lo, n_hi);
       const int ncols = n_hi - n_lo;
-      if (ncols == 0) continue;
-      const DecodeMeta* meta = reinterpret_cast<const DecodeMeta*>(slot_ptr(l & 1));
-      const int npairs = ((L.K >> 5) + 1) >> 1;
-      const uint32_t q_bytes = (uint32_t)npairs * 32u * 16u, row_bytes = (uint32_t)L.r * 2u;
-      const int ngroups = (L.M + 7) >> 3;
-      for (int G = 0; G < ngroups; ++G) {
-        decode_wait(q_empty, (q_use & 1) ^ 1, fail);
-        ++q_use;
-        if (lane == 0) {
+      if (ncols > 0) {
+        const int s = l & 1;
+        const int npairs = ((L.K >> 5) + 1) >> 1;
+        const uint32_t q_bytes = (uint32_t)npairs * 32u * 16u, row_bytes = (uint32_t)L.r * 2u;
+        const int ngroups = (L.M + 7) >> 3;
+        for (int G = 0; G < ngroups; ++G) {
+          decode_wait(q_empty, (q_use & 1) ^ 1, fail);
+          ++q_use;
           mbar_expect_tx(q_full, q_bytes);
           bulk_load(smem_u32(q_s), L.qfrag + (long long)G * npairs * 32, q_bytes, q_full);
-        }
-        const int nd = meta->ndistinct[G];
-        for (int d = 0; d < nd; ++d) {
-          decode_wait(ring_empty(ring_use), ((ring_use / kDecodeRing) & 1) ^ 1, fail);
-          if (lane == 0) {
-            const int e = meta->distinct[G][d];
+          if (G == 0) {
+            // the routing of this linear's tokens (needed to pick the expert rows) arrived with its slot
+            decode_wait(slot_full(s), slot_seen[s] & 1, fail);
+            ++slot_seen[s];
+          }
+          int list[8];
+          const int nd = L.r > 0 ? decode_distinct(reinterpret_cast<const DecodeTokInfo*>(slot_ptr(s)), L.M, G, list) : 0;
+          for (int d = 0; d < nd; ++d) {
+            int e = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) if (i == d) e = list[i];
+            decode_wait(ring_empty(ring_use), ((ring_use / kDecodeRing) & 1) ^ 1, fail);
             mbar_expect_tx(ring_full(ring_use), (uint32_t)ncols * row_bytes);
             bulk_load(smem_u32(ring + (ring_use % kDecodeRing) * bp.ring_stage_bytes), L.B + ((long long)e * L.N + n_lo) * L.r,
                       (uint32_t)ncols * row_bytes, ring_full(ring_use));
+            ++ring_use;
           }
-          ++ring_use;
+          // the next linear's slot goes out as soon as this linear's first loads are on their way
+          if (G == 0 && l + 1 < bp.n) issue_slot(l + 1);
         }
+      } else if (l + 1 < bp.n) {
+        issue_slot(l + 1);
       }
     }
     return;
@@ -368,7 +381,6 @@ __global__ void __launch_bounds__(kDecodeMainThreads, 1) k_decode_main(const __g
 
   // -------------------------------------------------------------------- consumers
   const int g = lane >> 2, c = lane & 3;
-  uint4* h_s = reinterpret_cast<uint4*>(smem + bp.off_hfrag);
   int* red = reinterpret_cast<int*>(smem + bp.off_red);
   int q_use = 0, ring_use = 0, slot_use[2] = {0, 0};
   for (int l = 0; l < bp.n; ++l) {
@@ -378,11 +390,6 @@ __global__ void __launch_bounds__(kDecodeMainThreads, 1) k_decode_main(const __g
     const int ncols = n_hi - n_lo;
     if (ncols == 0) continue;
     const int s = l & 1;
-    decode_wait(slot_full(s), slot_use[s] & 1, fail);
-    ++slot_use[s];
-    const DecodeMeta* meta = reinterpret_cast<const DecodeMeta*>(slot_ptr(s));
-    const uint32_t* bits_s = reinterpret_cast<const uint32_t*>(slot_ptr(s) + kDecodeMetaBytes);
-    const float* H_s = reinterpret_cast<const float*>(slot_ptr(s) + bp.off_slot_h);
     const int nks = L.K >> 5, npairs = (nks + 1) >> 1;
     const int ntile = (ncols + 15) >> 4;                   // 16-feature tiles of this CTA (<= 8)
     const int kslices = kDecodeConsumerWarps / ntile;      // warps sharing one tile split the contraction
@@ -393,57 +400,59 @@ __global__ void __launch_bounds__(kDecodeMainThreads, 1) k_decode_main(const __g
     const int rsteps = (L.r + 31) >> 5;                    // 32 hidden values per step of the expert product
     const uint32_t row_bytes = (uint32_t)L.r * 2u;
     const int ngroups = (L.M + 7) >> 3;
+    // per-feature factors of the epilogue, fetched before anything is waited for
+    const bool finisher = active && my_slice == 0;
+    float lam = 0.f, be0 = 0.f, be1 = 0.f, al0 = 0.f, al1 = 0.f;
+    if (finisher) {
+      lam = L.w_scales[0];
+      if (has0) { be0 = L.beta[(n_lo + row0) * L.sstride]; if (L.r > 0) al0 = L.alpha[(n_lo + row0) * L.sstride]; }
+      if (has1) { be1 = L.beta[(n_lo + row1) * L.sstride]; if (L.r > 0) al1 = L.alpha[(n_lo + row1) * L.sstride]; }
+    }
+    decode_wait(slot_full(s), slot_use[s] & 1, fail);
+    ++slot_use[s];
+    const DecodeTokInfo* tok = reinterpret_cast<const DecodeTokInfo*>(slot_ptr(s));
+    const uint32_t* bits_s = reinterpret_cast<const uint32_t*>(slot_ptr(s) + kDecodeMetaBytes);
+    const uint4* h_all = reinterpret_cast<const uint4*>(slot_ptr(s) + bp.off_slot_h);
 
     for (int G = 0; G < ngroups; ++G) {
-      const int nd = meta->ndistinct[G];
-      // hidden activations of this group as bf16 hi + lo fragments
-      for (int i = threadIdx.x; i < rsteps * 32; i += kDecodeConsumers) {
-        const int st = i >> 5, ln = i & 31, tg = ln >> 2, tc = ln & 3;
-        const int t = 8 * G + tg, j0 = 8 * (4 * st + tc);
-        uint32_t hi[4] = {0, 0, 0, 0}, lo[4] = {0, 0, 0, 0};
-        if (t < L.M) {
-          float v[8];
-#pragma unroll
-          for (int u = 0; u < 8; ++u) v[u] = j0 + u < L.r ? H_s[t * L.r + j0 + u] : 0.f;
-#pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            hi[u] = pack_bf16x2(v[2 * u], v[2 * u + 1]);
-            lo[u] = pack_bf16x2(v[2 * u] - bf16lo(hi[u]), v[2 * u + 1] - bf16hi(hi[u]));
-          }
-        }
-        h_s[i] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-        h_s[rsteps * 32 + i] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-      }
+      int list[8];
+      const int nd = L.r > 0 ? decode_distinct(tok, L.M, G, list) : 0;
       decode_wait(q_full, q_use & 1, fail);
       ++q_use;
 
-      // ---- 1-bit product: masked sums, weight 1 and weight 16
-      int acc1[4] = {0, 0, 0, 0}, acc16[4] = {0, 0, 0, 0};
+      // ---- 1-bit product: masked sums, weight 1 and weight 16; two independent chains of accumulators
+      int acc1[4] = {0, 0, 0, 0}, acc16[4] = {0, 0, 0, 0}, bcc1[4] = {0, 0, 0, 0}, bcc16[4] = {0, 0, 0, 0};
       if (active) {
         const int p0 = (int)((long long)my_slice * npairs / kslices), p1 = (int)((long long)(my_slice + 1) * npairs / kslices);
         const uint32_t* w0 = bits_s + (long long)(has0 ? row0 : 0) * nks;
         const uint32_t* w1 = bits_s + (long long)(has1 ? row1 : 0) * nks;
-        for (int ip = p0; ip < p1; ++ip) {
+        auto step = [&](int ip, int (&x1)[4], int (&x16)[4]) {
           const uint4 qv = q_s[ip * 32 + lane];
           const int i0 = 2 * ip, i1 = min(2 * ip + 1, nks - 1);   // an odd word count pairs the last word with zeros of q
           const uint32_t t00 = w0[i0] >> c, t01 = w0[i1] >> c, t10 = w1[i0] >> c, t11 = w1[i1] >> c;
           const uint32_t a1[4] = {t00 & 0x01010101u, t10 & 0x01010101u, t01 & 0x01010101u, t11 & 0x01010101u};
           const uint32_t a16[4] = {t00 & 0x10101010u, t10 & 0x10101010u, t01 & 0x10101010u, t11 & 0x10101010u};
-          mma_u8s8(acc1, a1, qv.x, qv.y);
-          mma_u8s8(acc16, a16, qv.z, qv.w);
-        }
+          mma_u8s8(x1, a1, qv.x, qv.y);
+          mma_u8s8(x16, a16, qv.z, qv.w);
+        };
+        int ip = p0;
+        for (; ip + 1 < p1; ip += 2) { step(ip, acc1, acc16); step(ip + 1, bcc1, bcc16); }
+        if (ip < p1) step(ip, acc1, acc16);
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(q_empty);                  // this warp is done with the q fragments
-      consumer_sync();                                      // the h fragments are complete
-      // ---- expert product z = B_e h, tokens of other experts masked out
-      float z[4] = {0.f, 0.f, 0.f, 0.f};
+      // ---- expert product z = B_e h, tokens of other experts masked out; four independent chains
+      float z0[4] = {0.f, 0.f, 0.f, 0.f}, z1[4] = {0.f, 0.f, 0.f, 0.f}, z2[4] = {0.f, 0.f, 0.f, 0.f}, z3[4] = {0.f, 0.f, 0.f, 0.f};
       const int my_tok = 8 * G + g;                          // the token whose h this thread feeds
-      const int my_tok_e = my_tok < L.M ? meta->tok[my_tok].expert : -1;
+      const int my_tok_e = my_tok < L.M ? tok[my_tok].expert : -1;
+      const uint4* h_hi = h_all + (size_t)(G * 2) * rsteps * 32;
+      const uint4* h_lo = h_hi + (size_t)rsteps * 32;
       for (int d = 0; d < nd; ++d) {
+        int e = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) if (i == d) e = list[i];
         const int stage = ring_use % kDecodeRing;
         decode_wait(ring_full(ring_use), (ring_use / kDecodeRing) & 1, fail);
-        const int e = meta->distinct[G][d];
         if (active) {
           const uint8_t* rows = ring + stage * bp.ring_stage_bytes;
           const uint4* r0p = reinterpret_cast<const uint4*>(rows + (long long)(has0 ? row0 : 0) * row_bytes);
@@ -451,14 +460,14 @@ __global__ void __launch_bounds__(kDecodeMainThreads, 1) k_decode_main(const __g
           const bool mine = my_tok_e == e;
           for (int st = my_slice; st < rsteps; st += kslices) {
             const int chunk = 4 * st + c;
-            uint4 b0 = make_uint4(0, 0, 0, 0), b1 = b0;
-            if (chunk * 8 < L.r) { b0 = r0p[chunk]; b1 = r1p[chunk]; }
-            uint4 hh = h_s[st * 32 + lane], hl = h_s[rsteps * 32 + st * 32 + lane];
-            if (!mine) { hh = make_uint4(0, 0, 0, 0); hl = hh; }
-            mma_bf16(z, b0.x, b1.x, b0.y, b1.y, hh.x, hh.y);
-            mma_bf16(z, b0.z, b1.z, b0.w, b1.w, hh.z, hh.w);
-            mma_bf16(z, b0.x, b1.x, b0.y, b1.y, hl.x, hl.y);
-            mma_bf16(z, b0.z, b1.z, b0.w, b1.w, hl.z, hl.w);
+            const bool in = chunk * 8 < L.r;
+            uint4 b0 = make_uint4(0, 0, 0, 0), b1 = b0, hh = b0, hl = b0;
+            if (in) { b0 = r0p[chunk]; b1 = r1p[chunk]; }
+            if (mine && in) { hh = h_hi[st * 32 + lane]; hl = h_lo[st * 32 + lane]; }
+            mma_bf16(z0, b0.x, b1.x, b0.y, b1.y, hh.x, hh.y);
+            mma_bf16(z1, b0.z, b1.z, b0.w, b1.w, hh.z, hh.w);
+            mma_bf16(z2, b0.x, b1.x, b0.y, b1.y, hl.x, hl.y);
+            mma_bf16(z3, b0.z, b1.z, b0.w, b1.w, hl.z, hl.w);
           }
         }
         __syncwarp();
@@ -471,12 +480,12 @@ __global__ void __launch_bounds__(kDecodeMainThreads, 1) k_decode_main(const __g
         int* mine = red + ((my_slice * ntile + my_tile) * 32 + lane) * 8;
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-          mine[u] = acc1[u] + (acc16[u] >> 4);   // the weight-16 sums are exact multiples of 16
-          mine[4 + u] = __float_as_int(z[u]);
+          mine[u] = (acc1[u] + bcc1[u]) + ((acc16[u] + bcc16[u]) >> 4);   // the weight-16 sums are exact multiples of 16
+          mine[4 + u] = __float_as_int((z0[u] + z1[u]) + (z2[u] + z3[u]));
         }
       }
       consumer_sync();
-      if (active && my_slice == 0) {
+      if (finisher) {
         int ms[4] = {0, 0, 0, 0};
         float zz[4] = {0.f, 0.f, 0.f, 0.f};
         for (int sl = 0; sl < kslices; ++sl) {
@@ -484,22 +493,21 @@ __global__ void __launch_bounds__(kDecodeMainThreads, 1) k_decode_main(const __g
 #pragma unroll
           for (int u = 0; u < 4; ++u) { ms[u] += part[u]; zz[u] += __int_as_float(part[4 + u]); }
         }
-        const float lam = L.w_scales[0];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
           // accumulator u: feature row0 (u < 2) or row1, token 8G + 2c + (u & 1)
           const int nl = (u < 2) ? row0 : row1, t = 8 * G + 2 * c + (u & 1);
           if (nl < ncols && t < L.M) {
             const int n = n_lo + nl;
-            const int acc = 2 * ms[u] - meta->tok[t].rowsum;
-            float y = L.beta[n * L.sstride] * __fdiv_rn(lam, meta->tok[t].gamma) * (float)acc;
-            if (L.r > 0) y = fmaf(L.alpha[n * L.sstride] * meta->tok[t].gate, zz[u], y);
+            const int acc = 2 * ms[u] - tok[t].rowsum;
+            float y = ((u < 2) ? be0 : be1) * __fdiv_rn(lam, tok[t].gamma) * (float)acc;
+            if (L.r > 0) y = fmaf(((u < 2) ? al0 : al1) * tok[t].gate, zz[u], y);
             L.Y[(long long)t * L.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(y));
             if (L.acc_dump) L.acc_dump[(long long)t * L.N + n] = acc;
           }
         }
       }
-      consumer_sync();   // the h fragments and the reduction buffer are rewritten by the next group
+      consumer_sync();   // the reduction buffer is rewritten by the next group
     }
     __syncwarp();
     if (lane == 0) mbar_arrive(slot_empty(s));               // this warp is done with the slot of linear l
@@ -515,7 +523,7 @@ size_t decode_workspace_bytes(int M, int K, int N, int r, bool dump) {
   const size_t npairs = ((size_t)K / 32 + 1) / 2;
   size_t b = up256(sizeof(DecodeTokInfo) * kDecodeMaxTokens);
   b += up256(2 * npairs * 32 * sizeof(uint4));
-  b += up256(sizeof(float) * kDecodeMaxTokens * (size_t)(r > 0 ? r : 1));
+  b += up256((size_t)2 * 2 * ((r + 31) / 32 > 0 ? (r + 31) / 32 : 1) * 512);
   if (dump) b += up256(sizeof(int) * (size_t)M * N);
   return b;
 }
@@ -525,7 +533,7 @@ DecodeViewPtrs decode_view(int M, int K, int N, int r, void* ws, bool dump) {
   const size_t npairs = ((size_t)K / 32 + 1) / 2;
   DecodeViewPtrs v{w, nullptr};
   w += up256(sizeof(DecodeTokInfo) * kDecodeMaxTokens) + up256(2 * npairs * 32 * sizeof(uint4)) +
-       up256(sizeof(float) * kDecodeMaxTokens * (size_t)(r > 0 ? r : 1));
+       up256((size_t)2 * 2 * ((r + 31) / 32 > 0 ? (r + 31) / 32 : 1) * 512);
   if (dump) v.acc = reinterpret_cast<int*>(w);
   (void)M; (void)N;
   return v;
@@ -547,7 +555,7 @@ static int decode_launch(const DecodeItemArgs* items, int n, cudaStream_t st) {
   static int sms = decode_sm_count();
   DecodeBatch bp{};
   bp.n = n;
-  size_t slot_bits = 0, slot_h = 0, q_bytes = 0, ring_stage = 0, hfrag = 0, prep_smem = 0;
+  size_t slot_bits = 0, slot_h = 0, q_bytes = 0, ring_stage = 0, prep_smem = 0;
   int max_slices = 1, max_m = 1;
   for (int i = 0; i < n; ++i) {
     const DecodeItemArgs& it = items[i];
@@ -557,7 +565,7 @@ static int decode_launch(const DecodeItemArgs* items, int n, cudaStream_t st) {
     const size_t npairs = ((size_t)K / 32 + 1) / 2;
     L.info = reinterpret_cast<DecodeTokInfo*>(w); w += up256(sizeof(DecodeTokInfo) * kDecodeMaxTokens);
     L.qfrag = reinterpret_cast<uint4*>(w); w += up256(2 * npairs * 32 * sizeof(uint4));
-    L.H = reinterpret_cast<float*>(w); w += up256(sizeof(float) * kDecodeMaxTokens * (size_t)(r > 0 ? r : 1));
+    L.hfrag = reinterpret_cast<uint4*>(w); w += up256((size_t)2 * 2 * ((r + 31) / 32 > 0 ? (r + 31) / 32 : 1) * 512);
     L.acc_dump = it.dump ? reinterpret_cast<int*>(w) : nullptr;
     L.X = reinterpret_cast<const uint4*>(it.X); L.Wr = reinterpret_cast<const uint4*>(it.a.Wr); L.A = it.a.A; L.B = it.a.B;
     L.bits = it.bits; L.w_scales = it.a.w_scales; L.alpha = it.a.alpha; L.beta = it.a.beta; L.Y = it.Y;
@@ -578,10 +586,9 @@ static int decode_launch(const DecodeItemArgs* items, int n, cudaStream_t st) {
     const int max_cols = ((groups + sms - 1) / sms) * 8;
     if (max_cols > 128) return PQ_ERR_UNSUPPORTED;   // 16 warps cover at most 8 tiles of 16 features
     slot_bits = std::max(slot_bits, up256((size_t)max_cols * (K / 8)));
-    slot_h = std::max(slot_h, up256((size_t)kDecodeMaxTokens * (r > 0 ? r : 1) * 4));
+    slot_h = std::max(slot_h, up256((size_t)2 * 2 * std::max((r + 31) / 32, 1) * 512));
     q_bytes = std::max(q_bytes, up256(npairs * 32 * sizeof(uint4)));
     ring_stage = std::max(ring_stage, up256((size_t)max_cols * r * 2));
-    hfrag = std::max(hfrag, up256((size_t)2 * std::max((r + 31) / 32, 1) * 32 * sizeof(uint4)));
     prep_smem = std::max(prep_smem, (size_t)K * 2);
   }
   const size_t meta = kDecodeMetaBytes;
@@ -591,7 +598,6 @@ static int decode_launch(const DecodeItemArgs* items, int n, cudaStream_t st) {
   bp.off_q = (int)off; off += q_bytes;
   bp.ring_stage_bytes = (int)ring_stage;
   bp.off_ring = (int)off; off += kDecodeRing * ring_stage;
-  bp.off_hfrag = (int)off; off += hfrag;
   bp.off_red = (int)off; off += (size_t)kDecodeConsumerWarps * 32 * 8 * sizeof(int);
   const size_t smem_main = off + 128;
   if (smem_main > 227 * 1024 || prep_smem > 200 * 1024) return PQ_ERR_UNSUPPORTED;
