@@ -22,9 +22,8 @@
 
 namespace pq {
 
-constexpr int kDecodeConsumerWarps = 16;
-constexpr int kDecodeConsumers = 32 * kDecodeConsumerWarps;
-constexpr int kDecodeMainThreads = kDecodeConsumers + 32;   // + the producer warp
+constexpr int kDecodeMaxConsumerWarps = 16;                 // 16 with one CTA per SM, 8 when two CTAs fit an SM
+constexpr int kDecodeMainThreads = 32 * kDecodeMaxConsumerWarps + 32;   // + the producer warp
 constexpr int kDecodeMaxTokens = 16;
 constexpr int kDecodeRing = 3;          // expert-row buffers in flight per CTA
 constexpr int kDecodeMaxBatch = 16;     // linears per launch (their descriptors travel as kernel parameters)
@@ -64,7 +63,8 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1
 // Its four 4-byte operand registers for the tokens' side therefore hold, for token g = lane >> 2,
 //   r0: q[64 ip      + c     + 8 j]   r1: q[64 ip + 32 + c     + 8 j]      (weight-1 masks)
 //   r2: q[64 ip      + c + 4 + 8 j]   r3: q[64 ip + 32 + c + 4 + 8 j]      (weight-16 masks)
-// stored as 16 bytes at ((group * npairs + ip) * 32 + lane) * 16, group = token / 8.
+// stored as 16 bytes; only the tokens that exist are stored: with Mg = min(8, M - 8 group) tokens in the group,
+// the piece of (pair ip, token g, quad index c) sits at uint4 index group * npairs * 32 + (ip * Mg + g) * 4 + c.
 // ---------------------------------------------------------------------------
 
 // One linear of a batch: device pointers and sizes (the workspace pointers are carved by the host).
@@ -88,7 +88,8 @@ struct DecodeBatch {
   DecodeLinear lin[kDecodeMaxBatch];
   int n;
   // shared-memory carve-up of k_decode_main (bytes from the 128-byte aligned base)
-  int slot_bytes, off_slot_h, off_q, off_ring, off_red, ring_stage_bytes;
+  int nwarps;               // consumer warps per CTA
+  int slot_bytes, off_slot_h, off_q, q_bytes, nq, off_ring, off_red, ring_stage_bytes;
 };
 
 // grid (slices, M, linears), 256 threads, dynamic shared memory: K bf16 values of the token
@@ -166,7 +167,7 @@ __global__ void __launch_bounds__(256) k_decode_prep(const __grid_constant__ Dec
   if (slice == 0) {
     // Eq. 7-9 for this token; every thread turns pairs of weight words (64 values of k) into fragment order
     const int npairs = (K + 63) >> 6;
-    const int group = m >> 3, g = m & 7;
+    const int group = m >> 3, g = m & 7, mg = min(8, L.M - 8 * group);
     int rowsum = 0;
     for (int ip = threadIdx.x; ip < npairs; ip += 256) {
       int qv[64];
@@ -195,7 +196,7 @@ __global__ void __launch_bounds__(256) k_decode_prep(const __grid_constant__ Dec
         }
         out[c] = make_uint4(w[0], w[1], w[2], w[3]);
       }
-      uint4* dst = L.qfrag + ((long long)(group * npairs + ip) * 32 + g * 4);
+      uint4* dst = L.qfrag + ((long long)group * npairs * 32 + (long long)(ip * mg + g) * 4);
 #pragma unroll
       for (int c = 0; c < 4; ++c) dst[c] = out[c];
     }
@@ -248,9 +249,9 @@ __global__ void __launch_bounds__(256) k_decode_prep(const __grid_constant__ Dec
 
 // Range of output features of CTA b: whole groups of 8, spread evenly.
 __device__ __forceinline__ void decode_range(int b, int nctas, int N, int& n_lo, int& n_hi) {
-  const int groups = N >> 3;
-  n_lo = (int)((long long)b * groups / nctas) << 3;
-  n_hi = (int)((long long)(b + 1) * groups / nctas) << 3;
+  const unsigned groups = (unsigned)N >> 3;   // b * groups stays far below 2^32
+  n_lo = (int)(((unsigned)b * groups / (unsigned)nctas) << 3);
+  n_hi = (int)(((unsigned)(b + 1) * groups / (unsigned)nctas) << 3);
 }
 
 constexpr int kDecodeMetaBytes = 256;   // token info at the start of a slot
@@ -269,7 +270,7 @@ __device__ __forceinline__ void decode_wait(uint32_t bar, uint32_t parity, volat
     }
   }
 }
-__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kDecodeConsumers) : "memory"); }
+__device__ __forceinline__ void consumer_sync(int nthreads) { asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory"); }
 
 // Distinct experts of the tokens [8 G, 8 G + 8) in order of first appearance (every thread computes its own copy).
 __device__ __forceinline__ int decode_distinct(const DecodeTokInfo* tok, int M, int G, int (&list)[8]) {
@@ -288,23 +289,24 @@ __device__ __forceinline__ int decode_distinct(const DecodeTokInfo* tok, int M, 
   return n;
 }
 
-__global__ void __launch_bounds__(kDecodeMainThreads, 1) k_decode_main(const __grid_constant__ DecodeBatch bp) {
+__global__ void __launch_bounds__(kDecodeMainThreads) k_decode_main(const __grid_constant__ DecodeBatch bp) {
   extern __shared__ __align__(128) uint8_t smem[];
-  // barriers: slot full/empty [2], q full/empty, ring full/empty [kDecodeRing]
-  __shared__ __align__(8) uint64_t bars[4 + 2 + 2 * kDecodeRing];
+  // barriers: slot full/empty [2], q full/empty [2], ring full/empty [kDecodeRing]
+  __shared__ __align__(8) uint64_t bars[4 + 4 + 2 * kDecodeRing];
   __shared__ int fail_sh;
   volatile int* fail = &fail_sh;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   auto slot_full = [&](int s) { return smem_u32(&bars[s]); };
   auto slot_empty = [&](int s) { return smem_u32(&bars[2 + s]); };
-  const uint32_t q_full = smem_u32(&bars[4]), q_empty = smem_u32(&bars[5]);
-  auto ring_full = [&](int i) { return smem_u32(&bars[6 + i % kDecodeRing]); };
-  auto ring_empty = [&](int i) { return smem_u32(&bars[6 + kDecodeRing + i % kDecodeRing]); };
+  auto q_full = [&](int i) { return smem_u32(&bars[4 + i]); };
+  auto q_empty = [&](int i) { return smem_u32(&bars[6 + i]); };
+  auto ring_full = [&](int i) { return smem_u32(&bars[8 + i % kDecodeRing]); };
+  auto ring_empty = [&](int i) { return smem_u32(&bars[8 + kDecodeRing + i % kDecodeRing]); };
   if (threadIdx.x == 0) {
     fail_sh = 0;
-    for (int s = 0; s < 2; ++s) { mbar_init(slot_full(s), 1); mbar_init(slot_empty(s), kDecodeConsumerWarps); }
-    mbar_init(q_full, 1); mbar_init(q_empty, kDecodeConsumerWarps);
-    for (int s = 0; s < kDecodeRing; ++s) { mbar_init(ring_full(s), 1); mbar_init(ring_empty(s), kDecodeConsumerWarps); }
+    for (int s = 0; s < 2; ++s) { mbar_init(slot_full(s), 1); mbar_init(slot_empty(s), bp.nwarps); }
+    for (int s = 0; s < 2; ++s) { mbar_init(q_full(s), 1); mbar_init(q_empty(s), bp.nwarps); }
+    for (int s = 0; s < kDecodeRing; ++s) { mbar_init(ring_full(s), 1); mbar_init(ring_empty(s), bp.nwarps); }
     mbar_fence_init();
   }
   pdl_launch_dependents();
@@ -316,7 +318,7 @@ __global__ void __launch_bounds__(kDecodeMainThreads, 1) k_decode_main(const __g
   uint4* q_s = reinterpret_cast<uint4*>(smem + bp.off_q);
   uint8_t* ring = smem + bp.off_ring;
 
-  if (warp == kDecodeConsumerWarps) {
+  if (warp == bp.nwarps) {
     // ------------------------------------------------------------------ producer (one thread issues everything)
     if (lane != 0) return;
     int q_use = 0, ring_use = 0, slot_use[2] = {0, 0}, slot_seen[2] = {0, 0};
@@ -345,13 +347,15 @@ __global__ void __launch_bounds__(kDecodeMainThreads, 1) k_decode_main(const __g
       if (ncols > 0) {
         const int s = l & 1;
         const int npairs = ((L.K >> 5) + 1) >> 1;
-        const uint32_t q_bytes = (uint32_t)npairs * 32u * 16u, row_bytes = (uint32_t)L.r * 2u;
+        const uint32_t row_bytes = (uint32_t)L.r * 2u;
         const int ngroups = (L.M + 7) >> 3;
         for (int G = 0; G < ngroups; ++G) {
-          decode_wait(q_empty, (q_use & 1) ^ 1, fail);
+          const uint32_t q_bytes = (uint32_t)(npairs * min(8, L.M - 8 * G)) * 64u;
+          const int qb = q_use % bp.nq;
+          decode_wait(q_empty(qb), ((q_use / bp.nq) & 1) ^ 1, fail);
+          mbar_expect_tx(q_full(qb), q_bytes);
+          bulk_load(smem_u32(q_s) + qb * bp.q_bytes, L.qfrag + (long long)G * npairs * 32, q_bytes, q_full(qb));
           ++q_use;
-          mbar_expect_tx(q_full, q_bytes);
-          bulk_load(smem_u32(q_s), L.qfrag + (long long)G * npairs * 32, q_bytes, q_full);
           if (G == 0) {
             // the routing of this linear's tokens (needed to pick the expert rows) arrived with its slot
             decode_wait(slot_full(s), slot_seen[s] & 1, fail);
@@ -392,7 +396,7 @@ __global__ void __launch_bounds__(kDecodeMainThreads, 1) k_decode_main(const __g
     const int s = l & 1;
     const int nks = L.K >> 5, npairs = (nks + 1) >> 1;
     const int ntile = (ncols + 15) >> 4;                   // 16-feature tiles of this CTA (<= 8)
-    const int kslices = kDecodeConsumerWarps / ntile;      // warps sharing one tile split the contraction
+    const int kslices = bp.nwarps / ntile;                 // warps sharing one tile split the contraction
     const int my_tile = warp % ntile, my_slice = warp / ntile;
     const bool active = my_slice < kslices;
     const int row0 = 16 * my_tile + g, row1 = row0 + 8;    // this thread's two features (local index)
@@ -417,17 +421,19 @@ __global__ void __launch_bounds__(kDecodeMainThreads, 1) k_decode_main(const __g
     for (int G = 0; G < ngroups; ++G) {
       int list[8];
       const int nd = L.r > 0 ? decode_distinct(tok, L.M, G, list) : 0;
-      decode_wait(q_full, q_use & 1, fail);
+      const int qb = q_use % bp.nq, mg = min(8, L.M - 8 * G);
+      decode_wait(q_full(qb), (q_use / bp.nq) & 1, fail);
       ++q_use;
+      const uint4* q_g = reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(q_s) + qb * bp.q_bytes);
 
       // ---- 1-bit product: masked sums, weight 1 and weight 16; two independent chains of accumulators
       int acc1[4] = {0, 0, 0, 0}, acc16[4] = {0, 0, 0, 0}, bcc1[4] = {0, 0, 0, 0}, bcc16[4] = {0, 0, 0, 0};
       if (active) {
-        const int p0 = (int)((long long)my_slice * npairs / kslices), p1 = (int)((long long)(my_slice + 1) * npairs / kslices);
+        const int p0 = my_slice * npairs / kslices, p1 = (my_slice + 1) * npairs / kslices;
         const uint32_t* w0 = bits_s + (long long)(has0 ? row0 : 0) * nks;
         const uint32_t* w1 = bits_s + (long long)(has1 ? row1 : 0) * nks;
         auto step = [&](int ip, int (&x1)[4], int (&x16)[4]) {
-          const uint4 qv = q_s[ip * 32 + lane];
+          const uint4 qv = g < mg ? q_g[(ip * mg + g) * 4 + c] : make_uint4(0u, 0u, 0u, 0u);
           const int i0 = 2 * ip, i1 = min(2 * ip + 1, nks - 1);   // an odd word count pairs the last word with zeros of q
           const uint32_t t00 = w0[i0] >> c, t01 = w0[i1] >> c, t10 = w1[i0] >> c, t11 = w1[i1] >> c;
           const uint32_t a1[4] = {t00 & 0x01010101u, t10 & 0x01010101u, t01 & 0x01010101u, t11 & 0x01010101u};
@@ -440,7 +446,7 @@ __global__ void __launch_bounds__(kDecodeMainThreads, 1) k_decode_main(const __g
         if (ip < p1) step(ip, acc1, acc16);
       }
       __syncwarp();
-      if (lane == 0) mbar_arrive(q_empty);                  // this warp is done with the q fragments
+      if (lane == 0) mbar_arrive(q_empty(qb));              // this warp is done with the q fragments
       // ---- expert product z = B_e h, tokens of other experts masked out; four independent chains
       float z0[4] = {0.f, 0.f, 0.f, 0.f}, z1[4] = {0.f, 0.f, 0.f, 0.f}, z2[4] = {0.f, 0.f, 0.f, 0.f}, z3[4] = {0.f, 0.f, 0.f, 0.f};
       const int my_tok = 8 * G + g;                          // the token whose h this thread feeds
@@ -477,21 +483,26 @@ __global__ void __launch_bounds__(kDecodeMainThreads, 1) k_decode_main(const __g
 
       // ---- sum the contraction slices of a tile, then the epilogue (Eq. 10-11)
       if (active) {
-        int* mine = red + ((my_slice * ntile + my_tile) * 32 + lane) * 8;
+        // lane-interleaved int4 rows: [slice][tile][2][32 lanes]
+        int4* mine = reinterpret_cast<int4*>(red) + (my_slice * ntile + my_tile) * 64 + lane;
+        int m4[4], z4[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-          mine[u] = (acc1[u] + bcc1[u]) + ((acc16[u] + bcc16[u]) >> 4);   // the weight-16 sums are exact multiples of 16
-          mine[4 + u] = __float_as_int((z0[u] + z1[u]) + (z2[u] + z3[u]));
+          m4[u] = (acc1[u] + bcc1[u]) + ((acc16[u] + bcc16[u]) >> 4);   // the weight-16 sums are exact multiples of 16
+          z4[u] = __float_as_int((z0[u] + z1[u]) + (z2[u] + z3[u]));
         }
+        mine[0] = make_int4(m4[0], m4[1], m4[2], m4[3]);
+        mine[32] = make_int4(z4[0], z4[1], z4[2], z4[3]);
       }
-      consumer_sync();
+      consumer_sync(32 * bp.nwarps);
       if (finisher) {
         int ms[4] = {0, 0, 0, 0};
         float zz[4] = {0.f, 0.f, 0.f, 0.f};
         for (int sl = 0; sl < kslices; ++sl) {
-          const int* part = red + ((sl * ntile + my_tile) * 32 + lane) * 8;
-#pragma unroll
-          for (int u = 0; u < 4; ++u) { ms[u] += part[u]; zz[u] += __int_as_float(part[4 + u]); }
+          const int4* part = reinterpret_cast<const int4*>(red) + (sl * ntile + my_tile) * 64 + lane;
+          const int4 pm = part[0], pz = part[32];
+          ms[0] += pm.x; ms[1] += pm.y; ms[2] += pm.z; ms[3] += pm.w;
+          zz[0] += __int_as_float(pz.x); zz[1] += __int_as_float(pz.y); zz[2] += __int_as_float(pz.z); zz[3] += __int_as_float(pz.w);
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
@@ -507,7 +518,7 @@ __global__ void __launch_bounds__(kDecodeMainThreads, 1) k_decode_main(const __g
           }
         }
       }
-      consumer_sync();   // the reduction buffer is rewritten by the next group
+      consumer_sync(32 * bp.nwarps);   // the reduction buffer is rewritten by the next group
     }
     __syncwarp();
     if (lane == 0) mbar_arrive(slot_empty(s));               // this warp is done with the slot of linear l
@@ -551,10 +562,13 @@ static int decode_sm_count() {
 }
 
 // One launch pair for up to kDecodeMaxBatch independent linears.
-static int decode_launch(const DecodeItemArgs* items, int n, cudaStream_t st) {
+static int decode_launch_with(const DecodeItemArgs* items, int n, int ctas_per_sm, cudaStream_t st) {
   static int sms = decode_sm_count();
+  // two CTAs of 8 consumer warps per SM (their phases interleave) when the shared memory of both fits, else one of 16
+  const int nctas = sms * ctas_per_sm, nwarps = ctas_per_sm == 2 ? 8 : 16;
+  const size_t smem_limit = ctas_per_sm == 2 ? 112 * 1024 : 227 * 1024;
   DecodeBatch bp{};
-  bp.n = n;
+  bp.n = n; bp.nwarps = nwarps;
   size_t slot_bits = 0, slot_h = 0, q_bytes = 0, ring_stage = 0, prep_smem = 0;
   int max_slices = 1, max_m = 1;
   for (int i = 0; i < n; ++i) {
@@ -583,11 +597,11 @@ static int decode_launch(const DecodeItemArgs* items, int n, cudaStream_t st) {
     if (L.slices > max_slices) max_slices = L.slices;
     if (M > max_m) max_m = M;
     const int groups = N / 8;
-    const int max_cols = ((groups + sms - 1) / sms) * 8;
-    if (max_cols > 128) return PQ_ERR_UNSUPPORTED;   // 16 warps cover at most 8 tiles of 16 features
+    const int max_cols = ((groups + nctas - 1) / nctas) * 8;
+    if (max_cols > 16 * nwarps / 2) return PQ_ERR_UNSUPPORTED;   // at least two warps per tile of 16 features
     slot_bits = std::max(slot_bits, up256((size_t)max_cols * (K / 8)));
     slot_h = std::max(slot_h, up256((size_t)2 * 2 * std::max((r + 31) / 32, 1) * 512));
-    q_bytes = std::max(q_bytes, up256(npairs * 32 * sizeof(uint4)));
+    q_bytes = std::max(q_bytes, up256(npairs * (size_t)std::min(M, 8) * 64));
     ring_stage = std::max(ring_stage, up256((size_t)max_cols * r * 2));
     prep_smem = std::max(prep_smem, (size_t)K * 2);
   }
@@ -595,12 +609,19 @@ static int decode_launch(const DecodeItemArgs* items, int n, cudaStream_t st) {
   bp.off_slot_h = (int)(meta + slot_bits);
   bp.slot_bytes = (int)(meta + slot_bits + slot_h);
   size_t off = 2 * (size_t)bp.slot_bytes;
-  bp.off_q = (int)off; off += q_bytes;
+  const size_t fixed = off + kDecodeRing * ring_stage + (size_t)nwarps * 32 * 8 * sizeof(int) + 128;
+  bp.nq = fixed + 2 * q_bytes <= smem_limit ? 2 : 1;     // the activations of two (linear, token group) steps in flight if they fit
+  bp.q_bytes = (int)q_bytes;
+  bp.off_q = (int)off; off += bp.nq * q_bytes;
   bp.ring_stage_bytes = (int)ring_stage;
   bp.off_ring = (int)off; off += kDecodeRing * ring_stage;
-  bp.off_red = (int)off; off += (size_t)kDecodeConsumerWarps * 32 * 8 * sizeof(int);
+  bp.off_red = (int)off; off += (size_t)nwarps * 32 * 8 * sizeof(int);
   const size_t smem_main = off + 128;
-  if (smem_main > 227 * 1024 || prep_smem > 200 * 1024) return PQ_ERR_UNSUPPORTED;
+  if (smem_main > smem_limit) {
+    if (ctas_per_sm == 2) return PQ_ERR_WORKSPACE;   // caller retries with one CTA per SM
+    return PQ_ERR_UNSUPPORTED;
+  }
+  if (prep_smem > 200 * 1024) return PQ_ERR_UNSUPPORTED;
   if (cudaFuncSetAttribute(k_decode_main, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_main) != cudaSuccess) return PQ_ERR_CUDA;
   if (cudaFuncSetAttribute(k_decode_prep, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)prep_smem) != cudaSuccess) return PQ_ERR_CUDA;
 
@@ -615,11 +636,16 @@ static int decode_launch(const DecodeItemArgs* items, int n, cudaStream_t st) {
     if (cudaLaunchKernelEx(&cfg, k_decode_prep, bp) != cudaSuccess) return PQ_ERR_CUDA;
   }
   {
-    cfg.gridDim = dim3(sms, 1, 1); cfg.blockDim = dim3(kDecodeMainThreads, 1, 1); cfg.dynamicSmemBytes = smem_main;
+    cfg.gridDim = dim3(nctas, 1, 1); cfg.blockDim = dim3(32 * nwarps + 32, 1, 1); cfg.dynamicSmemBytes = smem_main;
     LaunchScope ls(KID_DECODE_MAIN, st);
     if (cudaLaunchKernelEx(&cfg, k_decode_main, bp) != cudaSuccess) return PQ_ERR_CUDA;
   }
   return PQ_OK;
+}
+
+static int decode_launch(const DecodeItemArgs* items, int n, cudaStream_t st) {
+  const int rc = decode_launch_with(items, n, 2, st);
+  return rc == PQ_ERR_WORKSPACE ? decode_launch_with(items, n, 1, st) : rc;
 }
 
 int decode_batch(const DecodeItemArgs* items, int n, cudaStream_t st) {
