@@ -83,6 +83,8 @@ struct DecodeLinear {
   uint4* hfrag;             // [2 groups][2 planes (hi, lo)][ceil(r/32)][32] fragments of h = A_e x
   int* acc_dump;            // [M, N] exact 1-bit accumulators (test hook) or null
   int M, K, N, r, E, sstride, slices, rows_per_slice;
+  // partition of the N / 8 feature groups over the CTAs of k_decode_main: the first `grp_rem` CTAs own grp_base + 1 groups
+  int grp_base, grp_rem;
 };
 struct DecodeBatch {
   DecodeLinear lin[kDecodeMaxBatch];
@@ -247,11 +249,20 @@ __global__ void __launch_bounds__(256) k_decode_prep(const __grid_constant__ Dec
   }
 }
 
-// Range of output features of CTA b: whole groups of 8, spread evenly.
-__device__ __forceinline__ void decode_range(int b, int nctas, int N, int& n_lo, int& n_hi) {
-  const unsigned groups = (unsigned)N >> 3;   // b * groups stays far below 2^32
-  n_lo = (int)(((unsigned)b * groups / (unsigned)nctas) << 3);
-  n_hi = (int)(((unsigned)(b + 1) * groups / (unsigned)nctas) << 3);
+// Range of output features of CTA b: whole groups of 8, spread evenly (no division on the device).
+__device__ __forceinline__ void decode_range(int b, const DecodeLinear& L, int& n_lo, int& n_hi) {
+  n_lo = (b * L.grp_base + min(b, L.grp_rem)) << 3;
+  n_hi = n_lo + ((L.grp_base + (b < L.grp_rem ? 1 : 0)) << 3);
+}
+// Split of the consumer warps over the 16-feature tiles of a CTA: warp -> (tile, contraction slice).
+struct DecodeSplit { int ntile, kslices, my_tile, my_slice; };
+__device__ __forceinline__ DecodeSplit decode_split(int ncols, int nwarps, int warp) {
+  DecodeSplit d;
+  d.ntile = (ncols + 15) >> 4;
+  d.kslices = 0; d.my_slice = 0; d.my_tile = warp;
+  for (int w = d.ntile; w <= nwarps; w += d.ntile) ++d.kslices;              // nwarps / ntile
+  while (d.my_tile >= d.ntile) { d.my_tile -= d.ntile; ++d.my_slice; }       // warp / ntile, warp % ntile
+  return d;
 }
 
 constexpr int kDecodeMetaBytes = 256;   // token info at the start of a slot
@@ -272,21 +283,11 @@ __device__ __forceinline__ void decode_wait(uint32_t bar, uint32_t parity, volat
 }
 __device__ __forceinline__ void consumer_sync(int nthreads) { asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory"); }
 
-// Distinct experts of the tokens [8 G, 8 G + 8) in order of first appearance (every thread computes its own copy).
-__device__ __forceinline__ int decode_distinct(const DecodeTokInfo* tok, int M, int G, int (&list)[8]) {
-  int n = 0;
-  for (int t = 8 * G; t < min(M, 8 * G + 8); ++t) {
-    const int e = tok[t].expert;
-    bool seen = false;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) seen |= (i < n) && list[i] == e;
-    if (!seen) {
-#pragma unroll
-      for (int i = 0; i < 8; ++i) if (i == n) list[i] = e;
-      ++n;
-    }
-  }
-  return n;
+// Experts used by the tokens [8 G, 8 G + 8) as a bit mask; producer and consumers walk it in ascending order.
+__device__ __forceinline__ unsigned decode_expert_mask(const DecodeTokInfo* tok, int M, int G) {
+  unsigned mask = 0u;
+  for (int t = 8 * G; t < min(M, 8 * G + 8); ++t) mask |= 1u << tok[t].expert;
+  return mask;
 }
 
 __global__ void __launch_bounds__(kDecodeMainThreads) k_decode_main(const __grid_constant__ DecodeBatch bp) {
@@ -325,7 +326,7 @@ __global__ void __launch_bounds__(kDecodeMainThreads) k_decode_main(const __grid
     auto issue_slot = [&](int l) {
       const DecodeLinear& L = bp.lin[l];
       int n_lo, n_hi;
-      decode_range(blockIdx.x, gridDim.x, L.N, n_lo, n_hi);
+      decode_range(blockIdx.x, L, n_lo, n_hi);
       const int ncols = n_hi - n_lo;
       if (ncols == 0) return;
       const int s = l & 1;
@@ -342,7 +343,7 @@ __global__ void __launch_bounds__(kDecodeMainThreads) k_decode_main(const __grid
     for (int l = 0; l < bp.n; ++l) {
       const DecodeLinear& L = bp.lin[l];
       int n_lo, n_hi;
-      decode_range(blockIdx.x, gridDim.x, L.N, n_lo, n_hi);
+      decode_range(blockIdx.x, L, n_lo, n_hi);
       const int ncols = n_hi - n_lo;
       if (ncols > 0) {
         const int s = l & 1;
@@ -361,12 +362,9 @@ __global__ void __launch_bounds__(kDecodeMainThreads) k_decode_main(const __grid
             decode_wait(slot_full(s), slot_seen[s] & 1, fail);
             ++slot_seen[s];
           }
-          int list[8];
-          const int nd = L.r > 0 ? decode_distinct(reinterpret_cast<const DecodeTokInfo*>(slot_ptr(s)), L.M, G, list) : 0;
-          for (int d = 0; d < nd; ++d) {
-            int e = 0;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) if (i == d) e = list[i];
+          unsigned emask = L.r > 0 ? decode_expert_mask(reinterpret_cast<const DecodeTokInfo*>(slot_ptr(s)), L.M, G) : 0u;
+          for (; emask; emask &= emask - 1) {
+            const int e = __ffs(emask) - 1;
             decode_wait(ring_empty(ring_use), ((ring_use / kDecodeRing) & 1) ^ 1, fail);
             mbar_expect_tx(ring_full(ring_use), (uint32_t)ncols * row_bytes);
             bulk_load(smem_u32(ring + (ring_use % kDecodeRing) * bp.ring_stage_bytes), L.B + ((long long)e * L.N + n_lo) * L.r,
@@ -387,17 +385,20 @@ __global__ void __launch_bounds__(kDecodeMainThreads) k_decode_main(const __grid
   const int g = lane >> 2, c = lane & 3;
   int* red = reinterpret_cast<int*>(smem + bp.off_red);
   int q_use = 0, ring_use = 0, slot_use[2] = {0, 0};
+  DecodeSplit split{1, 1, 0, 0};
+  int split_cols = -1, chunk = 0, chunk_pairs = -1, chunk_slices = -1;
   for (int l = 0; l < bp.n; ++l) {
     const DecodeLinear& L = bp.lin[l];
     int n_lo, n_hi;
-    decode_range(blockIdx.x, gridDim.x, L.N, n_lo, n_hi);
+    decode_range(blockIdx.x, L, n_lo, n_hi);
     const int ncols = n_hi - n_lo;
     if (ncols == 0) continue;
     const int s = l & 1;
     const int nks = L.K >> 5, npairs = (nks + 1) >> 1;
-    const int ntile = (ncols + 15) >> 4;                   // 16-feature tiles of this CTA (<= 8)
-    const int kslices = bp.nwarps / ntile;                 // warps sharing one tile split the contraction
-    const int my_tile = warp % ntile, my_slice = warp / ntile;
+    if (ncols != split_cols) { split = decode_split(ncols, bp.nwarps, warp); split_cols = ncols; }
+    const int ntile = split.ntile;                         // 16-feature tiles of this CTA (<= 8)
+    const int kslices = split.kslices;                     // warps sharing one tile split the contraction
+    const int my_tile = split.my_tile, my_slice = split.my_slice;
     const bool active = my_slice < kslices;
     const int row0 = 16 * my_tile + g, row1 = row0 + 8;    // this thread's two features (local index)
     const bool has0 = row0 < ncols, has1 = row1 < ncols;
@@ -419,8 +420,7 @@ __global__ void __launch_bounds__(kDecodeMainThreads) k_decode_main(const __grid
     const uint4* h_all = reinterpret_cast<const uint4*>(slot_ptr(s) + bp.off_slot_h);
 
     for (int G = 0; G < ngroups; ++G) {
-      int list[8];
-      const int nd = L.r > 0 ? decode_distinct(tok, L.M, G, list) : 0;
+      unsigned emask = L.r > 0 ? decode_expert_mask(tok, L.M, G) : 0u;
       const int qb = q_use % bp.nq, mg = min(8, L.M - 8 * G);
       decode_wait(q_full(qb), (q_use / bp.nq) & 1, fail);
       ++q_use;
@@ -429,7 +429,11 @@ __global__ void __launch_bounds__(kDecodeMainThreads) k_decode_main(const __grid
       // ---- 1-bit product: masked sums, weight 1 and weight 16; two independent chains of accumulators
       int acc1[4] = {0, 0, 0, 0}, acc16[4] = {0, 0, 0, 0}, bcc1[4] = {0, 0, 0, 0}, bcc16[4] = {0, 0, 0, 0};
       if (active) {
-        const int p0 = my_slice * npairs / kslices, p1 = (my_slice + 1) * npairs / kslices;
+        if (npairs != chunk_pairs || kslices != chunk_slices) {          // ceil(npairs / kslices), recomputed only on change
+          chunk = (int)(((unsigned)npairs + (unsigned)kslices - 1u) / (unsigned)kslices);
+          chunk_pairs = npairs; chunk_slices = kslices;
+        }
+        const int p0 = min(npairs, my_slice * chunk), p1 = min(npairs, p0 + chunk);
         const uint32_t* w0 = bits_s + (long long)(has0 ? row0 : 0) * nks;
         const uint32_t* w1 = bits_s + (long long)(has1 ? row1 : 0) * nks;
         auto step = [&](int ip, int (&x1)[4], int (&x16)[4]) {
@@ -453,10 +457,8 @@ __global__ void __launch_bounds__(kDecodeMainThreads) k_decode_main(const __grid
       const int my_tok_e = my_tok < L.M ? tok[my_tok].expert : -1;
       const uint4* h_hi = h_all + (size_t)(G * 2) * rsteps * 32;
       const uint4* h_lo = h_hi + (size_t)rsteps * 32;
-      for (int d = 0; d < nd; ++d) {
-        int e = 0;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) if (i == d) e = list[i];
+      for (; emask; emask &= emask - 1) {
+        const int e = __ffs(emask) - 1;
         const int stage = ring_use % kDecodeRing;
         decode_wait(ring_full(ring_use), (ring_use / kDecodeRing) & 1, fail);
         if (active) {
@@ -597,6 +599,7 @@ static int decode_launch_with(const DecodeItemArgs* items, int n, int ctas_per_s
     if (L.slices > max_slices) max_slices = L.slices;
     if (M > max_m) max_m = M;
     const int groups = N / 8;
+    L.grp_base = groups / nctas; L.grp_rem = groups % nctas;
     const int max_cols = ((groups + nctas - 1) / nctas) * 8;
     if (max_cols > 16 * nwarps / 2) return PQ_ERR_UNSUPPORTED;   // at least two warps per tile of 16 features
     slot_bits = std::max(slot_bits, up256((size_t)max_cols * (K / 8)));
