@@ -33,7 +33,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel (the 2048 -> 5632
 # projection) from the committed ncu capture (profiles/gemm_kernels_up_projection_ncu.md); set to None
 # whenever the kernel changes until it is captured again.
-NCU_TRAFFIC_BYTES = {"bwd_dw": 324611072}
+NCU_TRAFFIC_BYTES = {"bwd_dw": 359938816}
 
 
 def measured_peaks():
@@ -397,23 +397,26 @@ def run_decode(args):
     launches0 = pqb.pq_kernel_launches()
     graph = capture(args.decode_batch)
     launches_per_step = pqb.pq_kernel_launches() - launches0
-    graph_serial = capture(1)
-    graph_pairs = capture(2)
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ms_serial = time_graph(graph_serial)
-    ms_pairs = time_graph(graph_pairs)
+    if args.decode_skip_serial:      # profiling runs: only the batched graph
+        ms_serial = ms_pairs = float("nan")
+    else:
+        ms_serial = time_graph(capture(1))
+        ms_pairs = time_graph(capture(2))
     with ClockSampler(local) as clk:
         ms_per_step = time_graph(graph)
     code, where = pqb.pq_device_status()
     if code:
         raise RuntimeError(f"device-side wait timed out (where={where})")
     # same pass launched call by call (no graph), for the launch-overhead comparison
-    t0.record()
-    for _ in range(min(args.steps, 20)):
-        step()
-    t1.record()
-    torch.cuda.synchronize()
-    ms_eager = t0.elapsed_time(t1) / min(args.steps, 20)
+    ms_eager = float("nan")
+    if not args.decode_skip_serial:
+        t0.record()
+        for _ in range(min(args.steps, 20)):
+            step()
+        t1.record()
+        torch.cuda.synchronize()
+        ms_eager = t0.elapsed_time(t1) / min(args.steps, 20)
 
     # end to end: every linear's activations from pinned host memory, every result back
     hx = [L.X.cpu().pin_memory() for L in layers]
@@ -535,6 +538,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="mlp_dense", choices=["mlp_dense", "mlp_e8", "decode"])
     ap.add_argument("--decode-tokens", type=int, default=1, choices=range(1, 17), metavar="M")
+    ap.add_argument("--decode-skip-serial", action="store_true", help="time only the batched graph (shorter runs under a profiler)")
     ap.add_argument("--decode-batch", type=int, default=16, help="independent decode linears per pq_decode_batch call")
     ap.add_argument("--cpu-tokens", type=int, default=4096)
     ap.add_argument("--no-e2e", action="store_true")
