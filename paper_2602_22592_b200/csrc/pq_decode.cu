@@ -25,7 +25,9 @@ namespace pq {
 constexpr int kDecodeMaxConsumerWarps = 16;                 // 16 with one CTA per SM, 8 when two CTAs fit an SM
 constexpr int kDecodeMainThreads = 32 * kDecodeMaxConsumerWarps + 32;   // + the producer warp
 constexpr int kDecodeMaxTokens = 16;
-constexpr int kDecodeRing = 3;          // expert-row buffers in flight per CTA
+constexpr int kDecodeMaxSlots = 4;      // linears whose sign bits are in flight or in use per CTA
+constexpr int kDecodeMaxQ = 4;          // activation buffers
+constexpr int kDecodeMaxRing = 8;       // expert-row buffers
 constexpr int kDecodeMaxBatch = 16;     // linears per launch (their descriptors travel as kernel parameters)
 
 struct DecodeTokInfo {  // one per token, written by k_decode_prep
@@ -91,7 +93,15 @@ struct DecodeBatch {
   int n;
   // shared-memory carve-up of k_decode_main (bytes from the 128-byte aligned base)
   int nwarps;               // consumer warps per CTA
-  int slot_bytes, off_slot_h, off_q, q_bytes, nq, off_ring, off_red, ring_stage_bytes;
+  int nslot, nq, nring;     // depths of the three buffer rings
+  int off_slots, slot_bytes, off_slot_h, off_q, q_bytes, off_ring, off_red, ring_stage_bytes;
+};
+// position in a ring of buffers with mbarrier full/empty pairs: the producer waits for empty(idx) with
+// parity phase ^ 1, a consumer for full(idx) with parity phase
+struct DecodeCursor {
+  int idx = 0;
+  uint32_t phase = 0;
+  __device__ __forceinline__ void next(int n) { if (++idx == n) { idx = 0; phase ^= 1u; } }
 };
 
 // grid (slices, M, linears), 256 threads, dynamic shared memory: K bf16 values of the token
@@ -292,90 +302,80 @@ __device__ __forceinline__ unsigned decode_expert_mask(const DecodeTokInfo* tok,
 
 __global__ void __launch_bounds__(kDecodeMainThreads) k_decode_main(const __grid_constant__ DecodeBatch bp) {
   extern __shared__ __align__(128) uint8_t smem[];
-  // barriers: slot full/empty [2], q full/empty [2], ring full/empty [kDecodeRing]
-  __shared__ __align__(8) uint64_t bars[4 + 4 + 2 * kDecodeRing];
+  // barriers: token info; slot, q and expert-row rings, a full/empty pair per buffer
+  __shared__ __align__(8) uint64_t bars[1 + 2 * kDecodeMaxSlots + 2 * kDecodeMaxQ + 2 * kDecodeMaxRing];
   __shared__ int fail_sh;
   volatile int* fail = &fail_sh;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  auto slot_full = [&](int s) { return smem_u32(&bars[s]); };
-  auto slot_empty = [&](int s) { return smem_u32(&bars[2 + s]); };
-  auto q_full = [&](int i) { return smem_u32(&bars[4 + i]); };
-  auto q_empty = [&](int i) { return smem_u32(&bars[6 + i]); };
-  auto ring_full = [&](int i) { return smem_u32(&bars[8 + i % kDecodeRing]); };
-  auto ring_empty = [&](int i) { return smem_u32(&bars[8 + kDecodeRing + i % kDecodeRing]); };
+  const uint32_t bar0 = smem_u32(&bars[0]);
+  const uint32_t info_full = bar0;
+  auto slot_full = [&](int s) { return bar0 + 8u * (1 + s); };
+  auto slot_empty = [&](int s) { return bar0 + 8u * (1 + kDecodeMaxSlots + s); };
+  auto q_full = [&](int i) { return bar0 + 8u * (1 + 2 * kDecodeMaxSlots + i); };
+  auto q_empty = [&](int i) { return bar0 + 8u * (1 + 2 * kDecodeMaxSlots + kDecodeMaxQ + i); };
+  auto ring_full = [&](int i) { return bar0 + 8u * (1 + 2 * kDecodeMaxSlots + 2 * kDecodeMaxQ + i); };
+  auto ring_empty = [&](int i) { return bar0 + 8u * (1 + 2 * kDecodeMaxSlots + 2 * kDecodeMaxQ + kDecodeMaxRing + i); };
   if (threadIdx.x == 0) {
     fail_sh = 0;
-    for (int s = 0; s < 2; ++s) { mbar_init(slot_full(s), 1); mbar_init(slot_empty(s), bp.nwarps); }
-    for (int s = 0; s < 2; ++s) { mbar_init(q_full(s), 1); mbar_init(q_empty(s), bp.nwarps); }
-    for (int s = 0; s < kDecodeRing; ++s) { mbar_init(ring_full(s), 1); mbar_init(ring_empty(s), bp.nwarps); }
+    mbar_init(info_full, 1);
+    for (int s = 0; s < bp.nslot; ++s) { mbar_init(slot_full(s), 1); mbar_init(slot_empty(s), bp.nwarps); }
+    for (int s = 0; s < bp.nq; ++s) { mbar_init(q_full(s), 1); mbar_init(q_empty(s), bp.nwarps); }
+    for (int s = 0; s < bp.nring; ++s) { mbar_init(ring_full(s), 1); mbar_init(ring_empty(s), bp.nwarps); }
     mbar_fence_init();
   }
   pdl_launch_dependents();
   pdl_wait();
   __syncthreads();
 
-  // a slot holds, for one linear: token info | sign bits of this CTA's features | h fragments (both groups)
-  auto slot_ptr = [&](int s) { return smem + (size_t)s * bp.slot_bytes; };
+  // token info of every linear of the batch sits at the start; a slot holds, for one linear, the sign bits
+  // of this CTA's features | the h fragments (both groups)
+  auto info_ptr = [&](int l) { return reinterpret_cast<const DecodeTokInfo*>(smem + l * kDecodeMetaBytes); };
+  auto slot_ptr = [&](int s) { return smem + bp.off_slots + (size_t)s * bp.slot_bytes; };
   uint4* q_s = reinterpret_cast<uint4*>(smem + bp.off_q);
   uint8_t* ring = smem + bp.off_ring;
 
   if (warp == bp.nwarps) {
     // ------------------------------------------------------------------ producer (one thread issues everything)
     if (lane != 0) return;
-    int q_use = 0, ring_use = 0, slot_use[2] = {0, 0}, slot_seen[2] = {0, 0};
-    auto issue_slot = [&](int l) {
-      const DecodeLinear& L = bp.lin[l];
-      int n_lo, n_hi;
-      decode_range(blockIdx.x, L, n_lo, n_hi);
-      const int ncols = n_hi - n_lo;
-      if (ncols == 0) return;
-      const int s = l & 1;
-      decode_wait(slot_empty(s), (slot_use[s] & 1) ^ 1, fail);
-      ++slot_use[s];
-      const uint32_t bits_bytes = (uint32_t)ncols * (uint32_t)(L.K >> 3);
-      const uint32_t h_bytes = L.r > 0 ? (uint32_t)(((L.M + 7) >> 3) * 2 * ((L.r + 31) >> 5)) * 512u : 0u;
-      mbar_expect_tx(slot_full(s), kDecodeMetaBytes + bits_bytes + h_bytes);
-      bulk_load(smem_u32(slot_ptr(s)), L.info, kDecodeMetaBytes, slot_full(s));
-      bulk_load(smem_u32(slot_ptr(s) + kDecodeMetaBytes), L.bits + (long long)n_lo * (L.K >> 5), bits_bytes, slot_full(s));
-      if (h_bytes) bulk_load(smem_u32(slot_ptr(s) + bp.off_slot_h), L.hfrag, h_bytes, slot_full(s));
-    };
-    if (bp.n > 0) issue_slot(0);
+    // The routing of every linear's tokens first: it decides which expert rows are fetched, and with it in
+    // hand nothing below waits for data, only for free buffers, so the loads run as far ahead as the rings allow.
+    mbar_expect_tx(info_full, (uint32_t)bp.n * kDecodeMetaBytes);
+    for (int l = 0; l < bp.n; ++l) bulk_load(smem_u32(smem + l * kDecodeMetaBytes), bp.lin[l].info, kDecodeMetaBytes, info_full);
+    decode_wait(info_full, 0, fail);
+    DecodeCursor cs, cq, cr;
     for (int l = 0; l < bp.n; ++l) {
       const DecodeLinear& L = bp.lin[l];
       int n_lo, n_hi;
       decode_range(blockIdx.x, L, n_lo, n_hi);
       const int ncols = n_hi - n_lo;
-      if (ncols > 0) {
-        const int s = l & 1;
-        const int npairs = ((L.K >> 5) + 1) >> 1;
-        const uint32_t row_bytes = (uint32_t)L.r * 2u;
-        const int ngroups = (L.M + 7) >> 3;
-        for (int G = 0; G < ngroups; ++G) {
-          const uint32_t q_bytes = (uint32_t)(npairs * min(8, L.M - 8 * G)) * 64u;
-          const int qb = q_use % bp.nq;
-          decode_wait(q_empty(qb), ((q_use / bp.nq) & 1) ^ 1, fail);
-          mbar_expect_tx(q_full(qb), q_bytes);
-          bulk_load(smem_u32(q_s) + qb * bp.q_bytes, L.qfrag + (long long)G * npairs * 32, q_bytes, q_full(qb));
-          ++q_use;
-          if (G == 0) {
-            // the routing of this linear's tokens (needed to pick the expert rows) arrived with its slot
-            decode_wait(slot_full(s), slot_seen[s] & 1, fail);
-            ++slot_seen[s];
-          }
-          unsigned emask = L.r > 0 ? decode_expert_mask(reinterpret_cast<const DecodeTokInfo*>(slot_ptr(s)), L.M, G) : 0u;
-          for (; emask; emask &= emask - 1) {
-            const int e = __ffs(emask) - 1;
-            decode_wait(ring_empty(ring_use), ((ring_use / kDecodeRing) & 1) ^ 1, fail);
-            mbar_expect_tx(ring_full(ring_use), (uint32_t)ncols * row_bytes);
-            bulk_load(smem_u32(ring + (ring_use % kDecodeRing) * bp.ring_stage_bytes), L.B + ((long long)e * L.N + n_lo) * L.r,
-                      (uint32_t)ncols * row_bytes, ring_full(ring_use));
-            ++ring_use;
-          }
-          // the next linear's slot goes out as soon as this linear's first loads are on their way
-          if (G == 0 && l + 1 < bp.n) issue_slot(l + 1);
+      if (ncols == 0) continue;
+      {
+        decode_wait(slot_empty(cs.idx), cs.phase ^ 1u, fail);
+        const uint32_t bits_bytes = (uint32_t)ncols * (uint32_t)(L.K >> 3);
+        const uint32_t h_bytes = L.r > 0 ? (uint32_t)(((L.M + 7) >> 3) * 2 * ((L.r + 31) >> 5)) * 512u : 0u;
+        mbar_expect_tx(slot_full(cs.idx), bits_bytes + h_bytes);
+        bulk_load(smem_u32(slot_ptr(cs.idx)), L.bits + (long long)n_lo * (L.K >> 5), bits_bytes, slot_full(cs.idx));
+        if (h_bytes) bulk_load(smem_u32(slot_ptr(cs.idx) + bp.off_slot_h), L.hfrag, h_bytes, slot_full(cs.idx));
+        cs.next(bp.nslot);
+      }
+      const int npairs = ((L.K >> 5) + 1) >> 1;
+      const uint32_t row_bytes = (uint32_t)L.r * 2u;
+      const int ngroups = (L.M + 7) >> 3;
+      for (int G = 0; G < ngroups; ++G) {
+        const uint32_t q_bytes = (uint32_t)(npairs * min(8, L.M - 8 * G)) * 64u;
+        decode_wait(q_empty(cq.idx), cq.phase ^ 1u, fail);
+        mbar_expect_tx(q_full(cq.idx), q_bytes);
+        bulk_load(smem_u32(q_s) + cq.idx * bp.q_bytes, L.qfrag + (long long)G * npairs * 32, q_bytes, q_full(cq.idx));
+        cq.next(bp.nq);
+        unsigned emask = L.r > 0 ? decode_expert_mask(info_ptr(l), L.M, G) : 0u;
+        for (; emask; emask &= emask - 1) {
+          const int e = __ffs(emask) - 1;
+          decode_wait(ring_empty(cr.idx), cr.phase ^ 1u, fail);
+          mbar_expect_tx(ring_full(cr.idx), (uint32_t)ncols * row_bytes);
+          bulk_load(smem_u32(ring + cr.idx * bp.ring_stage_bytes), L.B + ((long long)e * L.N + n_lo) * L.r,
+                    (uint32_t)ncols * row_bytes, ring_full(cr.idx));
+          cr.next(bp.nring);
         }
-      } else if (l + 1 < bp.n) {
-        issue_slot(l + 1);
       }
     }
     return;
@@ -384,8 +384,9 @@ __global__ void __launch_bounds__(kDecodeMainThreads) k_decode_main(const __grid
   // -------------------------------------------------------------------- consumers
   const int g = lane >> 2, c = lane & 3;
   int* red = reinterpret_cast<int*>(smem + bp.off_red);
-  int q_use = 0, ring_use = 0, slot_use[2] = {0, 0};
+  DecodeCursor cs, cq, cr;
   DecodeSplit split{1, 1, 0, 0};
+  decode_wait(info_full, 0, fail);
   int split_cols = -1, chunk = 0, chunk_pairs = -1, chunk_slices = -1;
   for (int l = 0; l < bp.n; ++l) {
     const DecodeLinear& L = bp.lin[l];
@@ -393,7 +394,6 @@ __global__ void __launch_bounds__(kDecodeMainThreads) k_decode_main(const __grid
     decode_range(blockIdx.x, L, n_lo, n_hi);
     const int ncols = n_hi - n_lo;
     if (ncols == 0) continue;
-    const int s = l & 1;
     const int nks = L.K >> 5, npairs = (nks + 1) >> 1;
     if (ncols != split_cols) { split = decode_split(ncols, bp.nwarps, warp); split_cols = ncols; }
     const int ntile = split.ntile;                         // 16-feature tiles of this CTA (<= 8)
@@ -413,17 +413,18 @@ __global__ void __launch_bounds__(kDecodeMainThreads) k_decode_main(const __grid
       if (has0) { be0 = L.beta[(n_lo + row0) * L.sstride]; if (L.r > 0) al0 = L.alpha[(n_lo + row0) * L.sstride]; }
       if (has1) { be1 = L.beta[(n_lo + row1) * L.sstride]; if (L.r > 0) al1 = L.alpha[(n_lo + row1) * L.sstride]; }
     }
-    decode_wait(slot_full(s), slot_use[s] & 1, fail);
-    ++slot_use[s];
-    const DecodeTokInfo* tok = reinterpret_cast<const DecodeTokInfo*>(slot_ptr(s));
-    const uint32_t* bits_s = reinterpret_cast<const uint32_t*>(slot_ptr(s) + kDecodeMetaBytes);
+    decode_wait(slot_full(cs.idx), cs.phase, fail);
+    const int s = cs.idx;
+    cs.next(bp.nslot);
+    const DecodeTokInfo* tok = info_ptr(l);
+    const uint32_t* bits_s = reinterpret_cast<const uint32_t*>(slot_ptr(s));
     const uint4* h_all = reinterpret_cast<const uint4*>(slot_ptr(s) + bp.off_slot_h);
 
     for (int G = 0; G < ngroups; ++G) {
       unsigned emask = L.r > 0 ? decode_expert_mask(tok, L.M, G) : 0u;
-      const int qb = q_use % bp.nq, mg = min(8, L.M - 8 * G);
-      decode_wait(q_full(qb), (q_use / bp.nq) & 1, fail);
-      ++q_use;
+      const int qb = cq.idx, mg = min(8, L.M - 8 * G);
+      decode_wait(q_full(qb), cq.phase, fail);
+      cq.next(bp.nq);
       const uint4* q_g = reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(q_s) + qb * bp.q_bytes);
 
       // ---- 1-bit product: masked sums, weight 1 and weight 16; two independent chains of accumulators
@@ -459,8 +460,9 @@ __global__ void __launch_bounds__(kDecodeMainThreads) k_decode_main(const __grid
       const uint4* h_lo = h_hi + (size_t)rsteps * 32;
       for (; emask; emask &= emask - 1) {
         const int e = __ffs(emask) - 1;
-        const int stage = ring_use % kDecodeRing;
-        decode_wait(ring_full(ring_use), (ring_use / kDecodeRing) & 1, fail);
+        const int stage = cr.idx;
+        decode_wait(ring_full(stage), cr.phase, fail);
+        cr.next(bp.nring);
         if (active) {
           const uint8_t* rows = ring + stage * bp.ring_stage_bytes;
           const uint4* r0p = reinterpret_cast<const uint4*>(rows + (long long)(has0 ? row0 : 0) * row_bytes);
@@ -479,8 +481,7 @@ __global__ void __launch_bounds__(kDecodeMainThreads) k_decode_main(const __grid
           }
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(ring_empty(ring_use));   // this warp is done with the buffer
-        ++ring_use;
+        if (lane == 0) mbar_arrive(ring_empty(stage));      // this warp is done with the buffer
       }
 
       // ---- sum the contraction slices of a tile, then the epilogue (Eq. 10-11)
@@ -608,16 +609,26 @@ static int decode_launch_with(const DecodeItemArgs* items, int n, int ctas_per_s
     ring_stage = std::max(ring_stage, up256((size_t)max_cols * r * 2));
     prep_smem = std::max(prep_smem, (size_t)K * 2);
   }
-  const size_t meta = kDecodeMetaBytes;
-  bp.off_slot_h = (int)(meta + slot_bits);
-  bp.slot_bytes = (int)(meta + slot_bits + slot_h);
-  size_t off = 2 * (size_t)bp.slot_bytes;
-  const size_t fixed = off + kDecodeRing * ring_stage + (size_t)nwarps * 32 * 8 * sizeof(int) + 128;
-  bp.nq = fixed + 2 * q_bytes <= smem_limit ? 2 : 1;     // the activations of two (linear, token group) steps in flight if they fit
+  // Buffer rings: at least two slots, one activation buffer and (with experts) two expert-row buffers; then
+  // deeper, in turn, while shared memory lasts, so that the loads of several linears are in flight at once.
+  const size_t slot_bytes = slot_bits + slot_h;
+  const size_t fixed = (size_t)n * kDecodeMetaBytes + (size_t)nwarps * 32 * 8 * sizeof(int) + 128;
+  const bool experts = ring_stage > 0;
+  bp.nslot = 2; bp.nq = 1; bp.nring = experts ? 2 : 1;
+  auto total = [&](int ns, int nq, int nr) { return fixed + ns * slot_bytes + nq * q_bytes + nr * ring_stage; };
+  for (bool grew = true; grew;) {
+    grew = false;
+    if (bp.nslot < kDecodeMaxSlots && total(bp.nslot + 1, bp.nq, bp.nring) <= smem_limit) { ++bp.nslot; grew = true; }
+    if (experts && bp.nring < kDecodeMaxRing && total(bp.nslot, bp.nq, bp.nring + 1) <= smem_limit) { ++bp.nring; grew = true; }
+    if (bp.nq < kDecodeMaxQ && bp.nq < bp.nslot * ((max_m + 7) / 8) && total(bp.nslot, bp.nq + 1, bp.nring) <= smem_limit) { ++bp.nq; grew = true; }
+  }
+  size_t off = (size_t)n * kDecodeMetaBytes;
+  bp.off_slots = (int)off; bp.off_slot_h = (int)slot_bits; bp.slot_bytes = (int)slot_bytes;
+  off += bp.nslot * slot_bytes;
   bp.q_bytes = (int)q_bytes;
   bp.off_q = (int)off; off += bp.nq * q_bytes;
   bp.ring_stage_bytes = (int)ring_stage;
-  bp.off_ring = (int)off; off += kDecodeRing * ring_stage;
+  bp.off_ring = (int)off; off += bp.nring * ring_stage;
   bp.off_red = (int)off; off += (size_t)nwarps * 32 * 8 * sizeof(int);
   const size_t smem_main = off + 128;
   if (smem_main > smem_limit) {
