@@ -94,7 +94,7 @@ struct DecodeBatch {
   // shared-memory carve-up of k_decode_main (bytes from the 128-byte aligned base)
   int nwarps;               // consumer warps per CTA
   int nslot, nq, nring;     // depths of the three buffer rings
-  int off_slots, slot_bytes, off_slot_h, off_q, q_bytes, off_ring, off_red, ring_stage_bytes;
+  int off_slots, slot_bytes, off_slot_h, off_q, q_bytes, off_ring, ring_stage_bytes;
 };
 // position in a ring of buffers with mbarrier full/empty pairs: the producer waits for empty(idx) with
 // parity phase ^ 1, a consumer for full(idx) with parity phase
@@ -264,17 +264,6 @@ __device__ __forceinline__ void decode_range(int b, const DecodeLinear& L, int& 
   n_lo = (b * L.grp_base + min(b, L.grp_rem)) << 3;
   n_hi = n_lo + ((L.grp_base + (b < L.grp_rem ? 1 : 0)) << 3);
 }
-// Split of the consumer warps over the 16-feature tiles of a CTA: warp -> (tile, contraction slice).
-struct DecodeSplit { int ntile, kslices, my_tile, my_slice; };
-__device__ __forceinline__ DecodeSplit decode_split(int ncols, int nwarps, int warp) {
-  DecodeSplit d;
-  d.ntile = (ncols + 15) >> 4;
-  d.kslices = 0; d.my_slice = 0; d.my_tile = warp;
-  for (int w = d.ntile; w <= nwarps; w += d.ntile) ++d.kslices;              // nwarps / ntile
-  while (d.my_tile >= d.ntile) { d.my_tile -= d.ntile; ++d.my_slice; }       // warp / ntile, warp % ntile
-  return d;
-}
-
 constexpr int kDecodeMetaBytes = 256;   // token info at the start of a slot
 
 // Wait with a bound.  Once any wait of the CTA has run out, every later wait returns at once, so that
@@ -291,7 +280,6 @@ __device__ __forceinline__ void decode_wait(uint32_t bar, uint32_t parity, volat
     }
   }
 }
-__device__ __forceinline__ void consumer_sync(int nthreads) { asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory"); }
 
 // Experts used by the tokens [8 G, 8 G + 8) as a bit mask; producer and consumers walk it in ascending order.
 __device__ __forceinline__ unsigned decode_expert_mask(const DecodeTokInfo* tok, int M, int G) {
@@ -382,73 +370,99 @@ __global__ void __launch_bounds__(kDecodeMainThreads) k_decode_main(const __grid
   }
 
   // -------------------------------------------------------------------- consumers
+  // The work of a CTA is a list of items (linear, token group, tile of 16 features), in that order; item i
+  // belongs to warp i mod nwarps, which contracts over all of K, adds the expert product and writes the 16 x 8
+  // outputs: no warp waits for another.  Every warp walks every buffer of the three rings in the producer's
+  // order, waits for it to be full and hands it back exactly once (the empty barriers count nwarps arrivals),
+  // whether it used it or not: a warp that skipped ahead without waiting could arrive twice in one phase.
   const int g = lane >> 2, c = lane & 3;
-  int* red = reinterpret_cast<int*>(smem + bp.off_red);
   DecodeCursor cs, cq, cr;
-  DecodeSplit split{1, 1, 0, 0};
   decode_wait(info_full, 0, fail);
-  int split_cols = -1, chunk = 0, chunk_pairs = -1, chunk_slices = -1;
+  int base_mod = 0;                                          // (items before the current (linear, group)) mod nwarps
   for (int l = 0; l < bp.n; ++l) {
     const DecodeLinear& L = bp.lin[l];
     int n_lo, n_hi;
     decode_range(blockIdx.x, L, n_lo, n_hi);
     const int ncols = n_hi - n_lo;
     if (ncols == 0) continue;
+    const int ntile = (ncols + 15) >> 4;                     // <= nwarps (checked by the host)
     const int nks = L.K >> 5, npairs = (nks + 1) >> 1;
-    if (ncols != split_cols) { split = decode_split(ncols, bp.nwarps, warp); split_cols = ncols; }
-    const int ntile = split.ntile;                         // 16-feature tiles of this CTA (<= 8)
-    const int kslices = split.kslices;                     // warps sharing one tile split the contraction
-    const int my_tile = split.my_tile, my_slice = split.my_slice;
-    const bool active = my_slice < kslices;
-    const int row0 = 16 * my_tile + g, row1 = row0 + 8;    // this thread's two features (local index)
-    const bool has0 = row0 < ncols, has1 = row1 < ncols;
-    const int rsteps = (L.r + 31) >> 5;                    // 32 hidden values per step of the expert product
+    const int rsteps = (L.r + 31) >> 5;                      // 32 hidden values per step of the expert product
     const uint32_t row_bytes = (uint32_t)L.r * 2u;
     const int ngroups = (L.M + 7) >> 3;
-    // per-feature factors of the epilogue, fetched before anything is waited for
-    const bool finisher = active && my_slice == 0;
-    float lam = 0.f, be0 = 0.f, be1 = 0.f, al0 = 0.f, al1 = 0.f;
-    if (finisher) {
-      lam = L.w_scales[0];
-      if (has0) { be0 = L.beta[(n_lo + row0) * L.sstride]; if (L.r > 0) al0 = L.alpha[(n_lo + row0) * L.sstride]; }
-      if (has1) { be1 = L.beta[(n_lo + row1) * L.sstride]; if (L.r > 0) al1 = L.alpha[(n_lo + row1) * L.sstride]; }
-    }
-    decode_wait(slot_full(cs.idx), cs.phase, fail);
-    const int s = cs.idx;
-    cs.next(bp.nslot);
     const DecodeTokInfo* tok = info_ptr(l);
+    const int s = cs.idx;
+    decode_wait(slot_full(s), cs.phase, fail);
+    cs.next(bp.nslot);
     const uint32_t* bits_s = reinterpret_cast<const uint32_t*>(slot_ptr(s));
     const uint4* h_all = reinterpret_cast<const uint4*>(slot_ptr(s) + bp.off_slot_h);
 
     for (int G = 0; G < ngroups; ++G) {
+      int my_tile = warp - base_mod;                         // tile j of this (linear, group) is item base + j
+      if (my_tile < 0) my_tile += bp.nwarps;
+      const bool mine = my_tile < ntile;
+      base_mod += ntile;
+      if (base_mod >= bp.nwarps) base_mod -= bp.nwarps;
       unsigned emask = L.r > 0 ? decode_expert_mask(tok, L.M, G) : 0u;
-      const int qb = cq.idx, mg = min(8, L.M - 8 * G);
-      decode_wait(q_full(qb), cq.phase, fail);
+      const int qb = cq.idx;
+      const uint32_t q_phase = cq.phase;
       cq.next(bp.nq);
-      const uint4* q_g = reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(q_s) + qb * bp.q_bytes);
-
-      // ---- 1-bit product: masked sums, weight 1 and weight 16; two independent chains of accumulators
-      int acc1[4] = {0, 0, 0, 0}, acc16[4] = {0, 0, 0, 0}, bcc1[4] = {0, 0, 0, 0}, bcc16[4] = {0, 0, 0, 0};
-      if (active) {
-        if (npairs != chunk_pairs || kslices != chunk_slices) {          // ceil(npairs / kslices), recomputed only on change
-          chunk = (int)(((unsigned)npairs + (unsigned)kslices - 1u) / (unsigned)kslices);
-          chunk_pairs = npairs; chunk_slices = kslices;
+      if (!mine) {
+        // nothing of this group is this warp's: hand its buffers back as they arrive
+        decode_wait(q_full(qb), q_phase, fail);
+        if (lane == 0) mbar_arrive(q_empty(qb));
+        for (; emask; emask &= emask - 1) {
+          decode_wait(ring_full(cr.idx), cr.phase, fail);
+          if (lane == 0) mbar_arrive(ring_empty(cr.idx));
+          cr.next(bp.nring);
         }
-        const int p0 = min(npairs, my_slice * chunk), p1 = min(npairs, p0 + chunk);
-        const uint32_t* w0 = bits_s + (long long)(has0 ? row0 : 0) * nks;
-        const uint32_t* w1 = bits_s + (long long)(has1 ? row1 : 0) * nks;
-        auto step = [&](int ip, int (&x1)[4], int (&x16)[4]) {
-          const uint4 qv = g < mg ? q_g[(ip * mg + g) * 4 + c] : make_uint4(0u, 0u, 0u, 0u);
-          const int i0 = 2 * ip, i1 = min(2 * ip + 1, nks - 1);   // an odd word count pairs the last word with zeros of q
-          const uint32_t t00 = w0[i0] >> c, t01 = w0[i1] >> c, t10 = w1[i0] >> c, t11 = w1[i1] >> c;
+        continue;
+      }
+      const int row0 = 16 * my_tile + g, row1 = row0 + 8;    // this thread's two features (local index)
+      const bool has0 = row0 < ncols, has1 = row1 < ncols;
+      // per-feature factors of the epilogue, fetched before anything is waited for
+      const float lam = L.w_scales[0];
+      float be0 = 0.f, be1 = 0.f, al0 = 0.f, al1 = 0.f;
+      if (has0) { be0 = L.beta[(n_lo + row0) * L.sstride]; if (L.r > 0) al0 = L.alpha[(n_lo + row0) * L.sstride]; }
+      if (has1) { be1 = L.beta[(n_lo + row1) * L.sstride]; if (L.r > 0) al1 = L.alpha[(n_lo + row1) * L.sstride]; }
+      const int mg = min(8, L.M - 8 * G);
+      decode_wait(q_full(qb), q_phase, fail);
+
+      // ---- 1-bit product: masked sums, weight 1 and weight 16; two independent chains of accumulators.
+      // Threads of tokens that do not exist read the last token's fragments (their results are never stored),
+      // threads of features beyond the range read feature 0.
+      int acc1[4] = {0, 0, 0, 0}, acc16[4] = {0, 0, 0, 0}, bcc1[4] = {0, 0, 0, 0}, bcc16[4] = {0, 0, 0, 0};
+      {
+        const uint4* qp = reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(q_s) + qb * bp.q_bytes) + min(g, mg - 1) * 4 + c;
+        const int qstep = mg * 4;
+        const uint32_t* w0 = bits_s + (has0 ? row0 : 0) * nks;
+        const uint32_t* w1 = bits_s + (has1 ? row1 : 0) * nks;
+        auto mac = [&](uint32_t x00, uint32_t x01, uint32_t x10, uint32_t x11, const uint4& qv, int (&x1)[4], int (&x16)[4]) {
+          const uint32_t t00 = x00 >> c, t01 = x01 >> c, t10 = x10 >> c, t11 = x11 >> c;
           const uint32_t a1[4] = {t00 & 0x01010101u, t10 & 0x01010101u, t01 & 0x01010101u, t11 & 0x01010101u};
           const uint32_t a16[4] = {t00 & 0x10101010u, t10 & 0x10101010u, t01 & 0x10101010u, t11 & 0x10101010u};
           mma_u8s8(x1, a1, qv.x, qv.y);
           mma_u8s8(x16, a16, qv.z, qv.w);
         };
-        int ip = p0;
-        for (; ip + 1 < p1; ip += 2) { step(ip, acc1, acc16); step(ip + 1, bcc1, bcc16); }
-        if (ip < p1) step(ip, acc1, acc16);
+        if ((nks & 1) == 0) {
+          // rows are 8-byte aligned: one load per pair of weight words
+          const uint2* v0 = reinterpret_cast<const uint2*>(w0);
+          const uint2* v1 = reinterpret_cast<const uint2*>(w1);
+          int ip = 0;
+#pragma unroll 2
+          for (; ip + 1 < npairs; ip += 2) {
+            const uint2 a = v0[ip], b = v1[ip], a2 = v0[ip + 1], b2 = v1[ip + 1];
+            const uint4 qa = qp[ip * qstep], qb2 = qp[(ip + 1) * qstep];
+            mac(a.x, a.y, b.x, b.y, qa, acc1, acc16);
+            mac(a2.x, a2.y, b2.x, b2.y, qb2, bcc1, bcc16);
+          }
+          if (ip < npairs) { const uint2 a = v0[ip], b = v1[ip]; mac(a.x, a.y, b.x, b.y, qp[ip * qstep], acc1, acc16); }
+        } else {
+          for (int ip = 0; ip < npairs; ++ip) {
+            const int i0 = 2 * ip, i1 = min(2 * ip + 1, nks - 1);   // the odd last word pairs with zeros of q
+            mac(w0[i0], w0[i1], w1[i0], w1[i1], qp[ip * qstep], acc1, acc16);
+          }
+        }
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(q_empty(qb));              // this warp is done with the q fragments
@@ -463,65 +477,40 @@ __global__ void __launch_bounds__(kDecodeMainThreads) k_decode_main(const __grid
         const int stage = cr.idx;
         decode_wait(ring_full(stage), cr.phase, fail);
         cr.next(bp.nring);
-        if (active) {
-          const uint8_t* rows = ring + stage * bp.ring_stage_bytes;
-          const uint4* r0p = reinterpret_cast<const uint4*>(rows + (long long)(has0 ? row0 : 0) * row_bytes);
-          const uint4* r1p = reinterpret_cast<const uint4*>(rows + (long long)(has1 ? row1 : 0) * row_bytes);
-          const bool mine = my_tok_e == e;
-          for (int st = my_slice; st < rsteps; st += kslices) {
-            const int chunk = 4 * st + c;
-            const bool in = chunk * 8 < L.r;
-            uint4 b0 = make_uint4(0, 0, 0, 0), b1 = b0, hh = b0, hl = b0;
-            if (in) { b0 = r0p[chunk]; b1 = r1p[chunk]; }
-            if (mine && in) { hh = h_hi[st * 32 + lane]; hl = h_lo[st * 32 + lane]; }
-            mma_bf16(z0, b0.x, b1.x, b0.y, b1.y, hh.x, hh.y);
-            mma_bf16(z1, b0.z, b1.z, b0.w, b1.w, hh.z, hh.w);
-            mma_bf16(z2, b0.x, b1.x, b0.y, b1.y, hl.x, hl.y);
-            mma_bf16(z3, b0.z, b1.z, b0.w, b1.w, hl.z, hl.w);
-          }
+        const uint8_t* rows = ring + stage * bp.ring_stage_bytes;
+        const uint4* r0p = reinterpret_cast<const uint4*>(rows + (has0 ? row0 : 0) * row_bytes);
+        const uint4* r1p = reinterpret_cast<const uint4*>(rows + (has1 ? row1 : 0) * row_bytes);
+        const bool feeds = my_tok_e == e;
+        for (int st = 0; st < rsteps; ++st) {
+          const int chunk = 4 * st + c;
+          const bool in = chunk * 8 < L.r;
+          uint4 b0 = make_uint4(0, 0, 0, 0), b1 = b0, hh = b0, hl = b0;
+          if (in) { b0 = r0p[chunk]; b1 = r1p[chunk]; }
+          if (feeds && in) { hh = h_hi[st * 32 + lane]; hl = h_lo[st * 32 + lane]; }
+          mma_bf16(z0, b0.x, b1.x, b0.y, b1.y, hh.x, hh.y);
+          mma_bf16(z1, b0.z, b1.z, b0.w, b1.w, hh.z, hh.w);
+          mma_bf16(z2, b0.x, b1.x, b0.y, b1.y, hl.x, hl.y);
+          mma_bf16(z3, b0.z, b1.z, b0.w, b1.w, hl.z, hl.w);
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(ring_empty(stage));      // this warp is done with the buffer
       }
 
-      // ---- sum the contraction slices of a tile, then the epilogue (Eq. 10-11)
-      if (active) {
-        // lane-interleaved int4 rows: [slice][tile][2][32 lanes]
-        int4* mine = reinterpret_cast<int4*>(red) + (my_slice * ntile + my_tile) * 64 + lane;
-        int m4[4], z4[4];
+      // ---- epilogue (Eq. 10-11)
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          m4[u] = (acc1[u] + bcc1[u]) + ((acc16[u] + bcc16[u]) >> 4);   // the weight-16 sums are exact multiples of 16
-          z4[u] = __float_as_int((z0[u] + z1[u]) + (z2[u] + z3[u]));
-        }
-        mine[0] = make_int4(m4[0], m4[1], m4[2], m4[3]);
-        mine[32] = make_int4(z4[0], z4[1], z4[2], z4[3]);
-      }
-      consumer_sync(32 * bp.nwarps);
-      if (finisher) {
-        int ms[4] = {0, 0, 0, 0};
-        float zz[4] = {0.f, 0.f, 0.f, 0.f};
-        for (int sl = 0; sl < kslices; ++sl) {
-          const int4* part = reinterpret_cast<const int4*>(red) + (sl * ntile + my_tile) * 64 + lane;
-          const int4 pm = part[0], pz = part[32];
-          ms[0] += pm.x; ms[1] += pm.y; ms[2] += pm.z; ms[3] += pm.w;
-          zz[0] += __int_as_float(pz.x); zz[1] += __int_as_float(pz.y); zz[2] += __int_as_float(pz.z); zz[3] += __int_as_float(pz.w);
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          // accumulator u: feature row0 (u < 2) or row1, token 8G + 2c + (u & 1)
-          const int nl = (u < 2) ? row0 : row1, t = 8 * G + 2 * c + (u & 1);
-          if (nl < ncols && t < L.M) {
-            const int n = n_lo + nl;
-            const int acc = 2 * ms[u] - tok[t].rowsum;
-            float y = ((u < 2) ? be0 : be1) * __fdiv_rn(lam, tok[t].gamma) * (float)acc;
-            if (L.r > 0) y = fmaf(((u < 2) ? al0 : al1) * tok[t].gate, zz[u], y);
-            L.Y[(long long)t * L.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(y));
-            if (L.acc_dump) L.acc_dump[(long long)t * L.N + n] = acc;
-          }
+      for (int u = 0; u < 4; ++u) {
+        // accumulator u: feature row0 (u < 2) or row1, token 8G + 2c + (u & 1)
+        const int nl = (u < 2) ? row0 : row1, t = 8 * G + 2 * c + (u & 1);
+        if (nl < ncols && t < L.M) {
+          const int n = n_lo + nl;
+          const int m = (acc1[u] + bcc1[u]) + ((acc16[u] + bcc16[u]) >> 4);   // the weight-16 sums are exact multiples of 16
+          const int acc = 2 * m - tok[t].rowsum;
+          float y = ((u < 2) ? be0 : be1) * __fdiv_rn(lam, tok[t].gamma) * (float)acc;
+          if (L.r > 0) y = fmaf(((u < 2) ? al0 : al1) * tok[t].gate, (z0[u] + z1[u]) + (z2[u] + z3[u]), y);
+          L.Y[(long long)t * L.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(y));
+          if (L.acc_dump) L.acc_dump[(long long)t * L.N + n] = acc;
         }
       }
-      consumer_sync(32 * bp.nwarps);   // the reduction buffer is rewritten by the next group
     }
     __syncwarp();
     if (lane == 0) mbar_arrive(slot_empty(s));               // this warp is done with the slot of linear l
@@ -569,7 +558,7 @@ static int decode_launch_with(const DecodeItemArgs* items, int n, int ctas_per_s
   static int sms = decode_sm_count();
   // two CTAs of 8 consumer warps per SM (their phases interleave) when the shared memory of both fits, else one of 16
   const int nctas = sms * ctas_per_sm, nwarps = ctas_per_sm == 2 ? 8 : 16;
-  const size_t smem_limit = ctas_per_sm == 2 ? 112 * 1024 : 227 * 1024;
+  const size_t smem_limit = ctas_per_sm == 2 ? 112 * 1024 : 226 * 1024;   // dynamic part; the barriers are static
   DecodeBatch bp{};
   bp.n = n; bp.nwarps = nwarps;
   size_t slot_bits = 0, slot_h = 0, q_bytes = 0, ring_stage = 0, prep_smem = 0;
@@ -602,7 +591,7 @@ static int decode_launch_with(const DecodeItemArgs* items, int n, int ctas_per_s
     const int groups = N / 8;
     L.grp_base = groups / nctas; L.grp_rem = groups % nctas;
     const int max_cols = ((groups + nctas - 1) / nctas) * 8;
-    if (max_cols > 16 * nwarps / 2) return PQ_ERR_UNSUPPORTED;   // at least two warps per tile of 16 features
+    if (max_cols > 16 * nwarps) return PQ_ERR_UNSUPPORTED;       // at most one tile of 16 features per warp and token group
     slot_bits = std::max(slot_bits, up256((size_t)max_cols * (K / 8)));
     slot_h = std::max(slot_h, up256((size_t)2 * 2 * std::max((r + 31) / 32, 1) * 512));
     q_bytes = std::max(q_bytes, up256(npairs * (size_t)std::min(M, 8) * 64));
@@ -612,7 +601,7 @@ static int decode_launch_with(const DecodeItemArgs* items, int n, int ctas_per_s
   // Buffer rings: at least two slots, one activation buffer and (with experts) two expert-row buffers; then
   // deeper, in turn, while shared memory lasts, so that the loads of several linears are in flight at once.
   const size_t slot_bytes = slot_bits + slot_h;
-  const size_t fixed = (size_t)n * kDecodeMetaBytes + (size_t)nwarps * 32 * 8 * sizeof(int) + 128;
+  const size_t fixed = (size_t)n * kDecodeMetaBytes + 128;
   const bool experts = ring_stage > 0;
   bp.nslot = 2; bp.nq = 1; bp.nring = experts ? 2 : 1;
   auto total = [&](int ns, int nq, int nr) { return fixed + ns * slot_bytes + nq * q_bytes + nr * ring_stage; };
@@ -629,7 +618,6 @@ static int decode_launch_with(const DecodeItemArgs* items, int n, int ctas_per_s
   bp.off_q = (int)off; off += bp.nq * q_bytes;
   bp.ring_stage_bytes = (int)ring_stage;
   bp.off_ring = (int)off; off += bp.nring * ring_stage;
-  bp.off_red = (int)off; off += (size_t)nwarps * 32 * 8 * sizeof(int);
   const size_t smem_main = off + 128;
   if (smem_main > smem_limit) {
     if (ctas_per_sm == 2) return PQ_ERR_WORKSPACE;   // caller retries with one CTA per SM
