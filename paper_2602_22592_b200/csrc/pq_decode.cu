@@ -5,12 +5,14 @@
 //   k_decode_prep  one CTA per (linear, token, slice of the r hidden rows): absmax quantisation
 //                  of the token (Eq. 7-9), router (Sec. 3.3), and its slice of h = A_e x.
 //   k_decode_main  one CTA per SM, each owning a contiguous range of output features of every
-//                  linear of the batch.  A producer warp streams, linear after linear, the sign
-//                  bits, the activations and the expert rows B_e of that range into shared memory
-//                  by bulk copies (mbarrier full/empty pairs), running ahead of sixteen consumer
-//                  warps: 1-bit product on mma.sync (u8 bit masks x s8 activations, exact in
-//                  int32), expert product on bf16 mma.sync, epilogue
-//                  Y = alpha g (B_e h) + beta (lam / gamma) (q . S)  (Eq. 10-11).
+//                  linear of the batch.  A producer warp first fetches the routing of all linears,
+//                  then streams, linear after linear, the sign bits, the activations and the expert
+//                  rows B_e of that range into rings of shared-memory buffers by bulk copies
+//                  (mbarrier full/empty pairs), as far ahead as the rings allow.  Each consumer warp
+//                  owns whole (linear, token group, 16-feature tile) items: 1-bit product on mma.sync
+//                  (u8 bit masks x s8 activations, exact in int32) over all of K, expert product on
+//                  bf16 mma.sync, epilogue Y = alpha g (B_e h) + beta (lam / gamma) (q . S)
+//                  (Eq. 10-11) straight from its registers; warps never wait for one another.
 // A batch is a set of INDEPENDENT linears (the gate and up projections of one block, the q/k/v
 // projections, other sequences): their weights then stream back to back.
 //
@@ -22,7 +24,7 @@
 
 namespace pq {
 
-constexpr int kDecodeMaxConsumerWarps = 16;                 // 16 with one CTA per SM, 8 when two CTAs fit an SM
+constexpr int kDecodeMaxConsumerWarps = 16;                 // 8 are launched unless a CTA owns more than 128 features
 constexpr int kDecodeMainThreads = 32 * kDecodeMaxConsumerWarps + 32;   // + the producer warp
 constexpr int kDecodeMaxTokens = 16;
 constexpr int kDecodeMaxSlots = 4;      // linears whose sign bits are in flight or in use per CTA
@@ -104,6 +106,8 @@ struct DecodeCursor {
   __device__ __forceinline__ void next(int n) { if (++idx == n) { idx = 0; phase ^= 1u; } }
 };
 
+constexpr int kPrepLoads = 16;   // 16-byte loads a lane keeps in flight while it walks a row of Wr or A_e
+
 // grid (slices, M, linears), 256 threads, dynamic shared memory: K bf16 values of the token
 __global__ void __launch_bounds__(256) k_decode_prep(const __grid_constant__ DecodeBatch bp) {
   extern __shared__ uint4 xs4[];
@@ -144,13 +148,13 @@ __global__ void __launch_bounds__(256) k_decode_prep(const __grid_constant__ Dec
     for (int e = warp; e < E; e += 8) {
       float acc = 0.f;
       const uint4* wrow = Wr + (long long)e * chunks;
-      // eight loads in flight per lane; the additions keep the ascending order of the chunks
-      for (int c0 = lane; c0 < chunks; c0 += 32 * 8) {
-        uint4 wv[8];
+      // sixteen loads in flight per lane; the additions keep the ascending order of the chunks
+      for (int c0 = lane; c0 < chunks; c0 += 32 * kPrepLoads) {
+        uint4 wv[kPrepLoads];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) wv[u] = (c0 + 32 * u < chunks) ? __ldg(wrow + c0 + 32 * u) : make_uint4(0u, 0u, 0u, 0u);
+        for (int u = 0; u < kPrepLoads; ++u) wv[u] = (c0 + 32 * u < chunks) ? __ldg(wrow + c0 + 32 * u) : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
+        for (int u = 0; u < kPrepLoads; ++u) {
           if (c0 + 32 * u < chunks) {
             const uint4 xv = xs4[c0 + 32 * u];
             acc = fmaf(bf16lo(xv.x), bf16lo(wv[u].x), acc); acc = fmaf(bf16hi(xv.x), bf16hi(wv[u].x), acc);
@@ -228,12 +232,12 @@ __global__ void __launch_bounds__(256) k_decode_prep(const __grid_constant__ Dec
     for (int j = j0 + warp; j < j1; j += 8) {
       const uint4* arow = reinterpret_cast<const uint4*>(L.A + ((long long)best * r + j) * K);
       float a0 = 0.f, a1 = 0.f;
-      for (int c0 = lane; c0 < chunks; c0 += 32 * 8) {
-        uint4 wv[8];
+      for (int c0 = lane; c0 < chunks; c0 += 32 * kPrepLoads) {
+        uint4 wv[kPrepLoads];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) wv[u] = (c0 + 32 * u < chunks) ? __ldg(arow + c0 + 32 * u) : make_uint4(0u, 0u, 0u, 0u);
+        for (int u = 0; u < kPrepLoads; ++u) wv[u] = (c0 + 32 * u < chunks) ? __ldg(arow + c0 + 32 * u) : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
+        for (int u = 0; u < kPrepLoads; ++u) {
           if (c0 + 32 * u < chunks) {
             const uint4 xv = xs4[c0 + 32 * u];
             a0 = fmaf(bf16lo(xv.x), bf16lo(wv[u].x), a0); a1 = fmaf(bf16hi(xv.x), bf16hi(wv[u].x), a1);
@@ -266,12 +270,27 @@ __device__ __forceinline__ void decode_range(int b, const DecodeLinear& L, int& 
 }
 constexpr int kDecodeMetaBytes = 256;   // token info at the start of a slot
 
+// mbarrier.try_wait with a suspend-time hint: a warp whose phase is not complete is parked by the hardware for up
+// to `ns` nanoseconds (it resumes at once when the phase completes) instead of coming back to poll after the short
+// default limit.  Most consumer warps of a CTA are waiting at any time; polling, they took most of the issue slots.
+__device__ __forceinline__ bool mbar_try_wait_parked(uint32_t bar, uint32_t parity, uint32_t ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(ns)
+      : "memory");
+  return ok != 0;
+}
+
 // Wait with a bound.  Once any wait of the CTA has run out, every later wait returns at once, so that
 // all threads keep the same control flow and the kernel ends (with an error status and undefined output).
 __device__ __forceinline__ void decode_wait(uint32_t bar, uint32_t parity, volatile int* fail) {
   if (mbar_try_wait(bar, parity)) return;
   const long long t0 = clock64();
-  while (!mbar_try_wait(bar, parity)) {
+  while (!mbar_try_wait_parked(bar, parity, 20000u)) {
     if (*fail) return;
     if (clock64() - t0 > kSpinCycles) {
       report_timeout(WHERE_OTHER);
@@ -312,8 +331,8 @@ __global__ void __launch_bounds__(kDecodeMainThreads) k_decode_main(const __grid
     mbar_fence_init();
   }
   pdl_launch_dependents();
-  pdl_wait();
   __syncthreads();
+  if (warp != bp.nwarps) pdl_wait();   // the producer waits later: weights do not depend on the previous kernel
 
   // token info of every linear of the batch sits at the start; a slot holds, for one linear, the sign bits
   // of this CTA's features | the h fragments (both groups)
@@ -325,6 +344,26 @@ __global__ void __launch_bounds__(kDecodeMainThreads) k_decode_main(const __grid
   if (warp == bp.nwarps) {
     // ------------------------------------------------------------------ producer (one thread issues everything)
     if (lane != 0) return;
+    // The sign bits of the first linears (as many as there are slots) go out before the previous kernel, which
+    // prepares this one's tokens, is known to have finished: weights are not its output.
+    int early = 0;
+    {
+      DecodeCursor c0;
+      for (int l = 0; l < bp.n && early < bp.nslot; ++l) {
+        const DecodeLinear& L = bp.lin[l];
+        int n_lo, n_hi;
+        decode_range(blockIdx.x, L, n_lo, n_hi);
+        const int ncols = n_hi - n_lo;
+        if (ncols == 0) continue;
+        const uint32_t bits_bytes = (uint32_t)ncols * (uint32_t)(L.K >> 3);
+        const uint32_t h_bytes = L.r > 0 ? (uint32_t)(((L.M + 7) >> 3) * 2 * ((L.r + 31) >> 5)) * 512u : 0u;
+        mbar_expect_tx(slot_full(c0.idx), bits_bytes + h_bytes);
+        bulk_load(smem_u32(slot_ptr(c0.idx)), L.bits + (long long)n_lo * (L.K >> 5), bits_bytes, slot_full(c0.idx));
+        c0.next(bp.nslot);
+        ++early;
+      }
+    }
+    pdl_wait();
     // The routing of every linear's tokens first: it decides which expert rows are fetched, and with it in
     // hand nothing below waits for data, only for free buffers, so the loads run as far ahead as the rings allow.
     mbar_expect_tx(info_full, (uint32_t)bp.n * kDecodeMetaBytes);
@@ -338,11 +377,15 @@ __global__ void __launch_bounds__(kDecodeMainThreads) k_decode_main(const __grid
       const int ncols = n_hi - n_lo;
       if (ncols == 0) continue;
       {
-        decode_wait(slot_empty(cs.idx), cs.phase ^ 1u, fail);
         const uint32_t bits_bytes = (uint32_t)ncols * (uint32_t)(L.K >> 3);
         const uint32_t h_bytes = L.r > 0 ? (uint32_t)(((L.M + 7) >> 3) * 2 * ((L.r + 31) >> 5)) * 512u : 0u;
-        mbar_expect_tx(slot_full(cs.idx), bits_bytes + h_bytes);
-        bulk_load(smem_u32(slot_ptr(cs.idx)), L.bits + (long long)n_lo * (L.K >> 5), bits_bytes, slot_full(cs.idx));
+        if (early > 0) {
+          --early;                                          // bits already on their way
+        } else {
+          decode_wait(slot_empty(cs.idx), cs.phase ^ 1u, fail);
+          mbar_expect_tx(slot_full(cs.idx), bits_bytes + h_bytes);
+          bulk_load(smem_u32(slot_ptr(cs.idx)), L.bits + (long long)n_lo * (L.K >> 5), bits_bytes, slot_full(cs.idx));
+        }
         if (h_bytes) bulk_load(smem_u32(slot_ptr(cs.idx) + bp.off_slot_h), L.hfrag, h_bytes, slot_full(cs.idx));
         cs.next(bp.nslot);
       }
@@ -445,18 +488,42 @@ __global__ void __launch_bounds__(kDecodeMainThreads) k_decode_main(const __grid
           mma_u8s8(x16, a16, qv.z, qv.w);
         };
         if ((nks & 1) == 0) {
-          // rows are 8-byte aligned: one load per pair of weight words
+          // Rows are 8-byte aligned: one load per pair of weight words.  Software pipeline without branches:
+          // two register sets of four steps each; while one is multiplied the other is being loaded (the
+          // loads past the end are clamped to the last step and never used).
           const uint2* v0 = reinterpret_cast<const uint2*>(w0);
           const uint2* v1 = reinterpret_cast<const uint2*>(w1);
+          struct Set { uint2 a[4], b[4]; uint4 q[4]; };
+          const int last = npairs - 1;
+          auto fetch = [&](Set& f, int ip) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const int i = min(ip + j, last);
+              f.a[j] = v0[i]; f.b[j] = v1[i]; f.q[j] = qp[i * qstep];
+            }
+          };
+          auto macs = [&](const Set& f) {
+            mac(f.a[0].x, f.a[0].y, f.b[0].x, f.b[0].y, f.q[0], acc1, acc16);
+            mac(f.a[1].x, f.a[1].y, f.b[1].x, f.b[1].y, f.q[1], bcc1, bcc16);
+            mac(f.a[2].x, f.a[2].y, f.b[2].x, f.b[2].y, f.q[2], acc1, acc16);
+            mac(f.a[3].x, f.a[3].y, f.b[3].x, f.b[3].y, f.q[3], bcc1, bcc16);
+          };
+          Set A, B;
           int ip = 0;
-#pragma unroll 2
-          for (; ip + 1 < npairs; ip += 2) {
-            const uint2 a = v0[ip], b = v1[ip], a2 = v0[ip + 1], b2 = v1[ip + 1];
-            const uint4 qa = qp[ip * qstep], qb2 = qp[(ip + 1) * qstep];
-            mac(a.x, a.y, b.x, b.y, qa, acc1, acc16);
-            mac(a2.x, a2.y, b2.x, b2.y, qb2, bcc1, bcc16);
+          fetch(A, 0);
+          for (; ip + 8 <= npairs; ip += 8) {
+            fetch(B, ip + 4);
+            macs(A);
+            fetch(A, ip + 8);
+            macs(B);
           }
-          if (ip < npairs) { const uint2 a = v0[ip], b = v1[ip]; mac(a.x, a.y, b.x, b.y, qp[ip * qstep], acc1, acc16); }
+          // fewer than eight steps left; A holds steps ip .. ip + 3 (clamped)
+          if (ip + 4 <= npairs) { macs(A); ip += 4; fetch(A, ip); }
+          for (int j = 0; ip + j < npairs; ++j) {
+            if (j == 0) mac(A.a[0].x, A.a[0].y, A.b[0].x, A.b[0].y, A.q[0], acc1, acc16);
+            if (j == 1) mac(A.a[1].x, A.a[1].y, A.b[1].x, A.b[1].y, A.q[1], bcc1, bcc16);
+            if (j == 2) mac(A.a[2].x, A.a[2].y, A.b[2].x, A.b[2].y, A.q[2], acc1, acc16);
+          }
         } else {
           for (int ip = 0; ip < npairs; ++ip) {
             const int i0 = 2 * ip, i1 = min(2 * ip + 1, nks - 1);   // the odd last word pairs with zeros of q
@@ -554,11 +621,12 @@ static int decode_sm_count() {
 }
 
 // One launch pair for up to kDecodeMaxBatch independent linears.
-static int decode_launch_with(const DecodeItemArgs* items, int n, int ctas_per_sm, cudaStream_t st) {
+static int decode_launch_with(const DecodeItemArgs* items, int n, int nwarps, cudaStream_t st) {
   static int sms = decode_sm_count();
-  // two CTAs of 8 consumer warps per SM (their phases interleave) when the shared memory of both fits, else one of 16
-  const int nctas = sms * ctas_per_sm, nwarps = ctas_per_sm == 2 ? 8 : 16;
-  const size_t smem_limit = ctas_per_sm == 2 ? 112 * 1024 : 226 * 1024;   // dynamic part; the barriers are static
+  // One CTA per SM.  Eight consumer warps keep up with what the buffer rings can hold in flight (measured: more warps,
+  // or two smaller CTAs per SM, are not faster); sixteen only when a CTA's feature range needs more than eight tiles.
+  const int nctas = sms;
+  const size_t smem_limit = 226 * 1024;   // dynamic part; the barriers are static
   DecodeBatch bp{};
   bp.n = n; bp.nwarps = nwarps;
   size_t slot_bits = 0, slot_h = 0, q_bytes = 0, ring_stage = 0, prep_smem = 0;
@@ -576,14 +644,15 @@ static int decode_launch_with(const DecodeItemArgs* items, int n, int ctas_per_s
     L.X = reinterpret_cast<const uint4*>(it.X); L.Wr = reinterpret_cast<const uint4*>(it.a.Wr); L.A = it.a.A; L.B = it.a.B;
     L.bits = it.bits; L.w_scales = it.a.w_scales; L.alpha = it.a.alpha; L.beta = it.a.beta; L.Y = it.Y;
     L.M = M; L.K = K; L.N = N; L.r = r; L.E = (r > 0 && it.a.E > 1) ? it.a.E : 1; L.sstride = it.a.scale_stride;
-    // slices of the hidden rows: enough CTAs to pull A_e at full rate, at least one row per warp
+    // Slices of the hidden rows: whole rounds of eight rows (one per warp), and enough CTAs in the grid (about
+    // eight per SM) that the rows of A_e stream at full rate; every slice repeats the token's absmax and router.
     L.slices = 1; L.rows_per_slice = 1;
     if (r > 0) {
-      int slices = 2 * sms / (M * n);
+      int slices = (8 * sms + M * n - 1) / (M * n);
       const int most = (r + 7) / 8;
       if (slices > most) slices = most;
       if (slices < 1) slices = 1;
-      L.rows_per_slice = (r + slices - 1) / slices;
+      L.rows_per_slice = ((r + slices - 1) / slices + 7) / 8 * 8;
       L.slices = (r + L.rows_per_slice - 1) / L.rows_per_slice;
     }
     if (L.slices > max_slices) max_slices = L.slices;
@@ -593,7 +662,7 @@ static int decode_launch_with(const DecodeItemArgs* items, int n, int ctas_per_s
     const int max_cols = ((groups + nctas - 1) / nctas) * 8;
     if (max_cols > 16 * nwarps) return PQ_ERR_UNSUPPORTED;       // at most one tile of 16 features per warp and token group
     slot_bits = std::max(slot_bits, up256((size_t)max_cols * (K / 8)));
-    slot_h = std::max(slot_h, up256((size_t)2 * 2 * std::max((r + 31) / 32, 1) * 512));
+    slot_h = std::max(slot_h, r > 0 ? up256((size_t)((M + 7) / 8) * 2 * ((r + 31) / 32) * 512) : (size_t)0);   // token groups in use only
     q_bytes = std::max(q_bytes, up256(npairs * (size_t)std::min(M, 8) * 64));
     ring_stage = std::max(ring_stage, up256((size_t)max_cols * r * 2));
     prep_smem = std::max(prep_smem, (size_t)K * 2);
@@ -620,7 +689,6 @@ static int decode_launch_with(const DecodeItemArgs* items, int n, int ctas_per_s
   bp.off_ring = (int)off; off += bp.nring * ring_stage;
   const size_t smem_main = off + 128;
   if (smem_main > smem_limit) {
-    if (ctas_per_sm == 2) return PQ_ERR_WORKSPACE;   // caller retries with one CTA per SM
     return PQ_ERR_UNSUPPORTED;
   }
   if (prep_smem > 200 * 1024) return PQ_ERR_UNSUPPORTED;
@@ -646,8 +714,8 @@ static int decode_launch_with(const DecodeItemArgs* items, int n, int ctas_per_s
 }
 
 static int decode_launch(const DecodeItemArgs* items, int n, cudaStream_t st) {
-  const int rc = decode_launch_with(items, n, 2, st);
-  return rc == PQ_ERR_WORKSPACE ? decode_launch_with(items, n, 1, st) : rc;
+  const int rc = decode_launch_with(items, n, 8, st);
+  return rc == PQ_ERR_UNSUPPORTED ? decode_launch_with(items, n, kDecodeMaxConsumerWarps, st) : rc;
 }
 
 int decode_batch(const DecodeItemArgs* items, int n, cudaStream_t st) {
