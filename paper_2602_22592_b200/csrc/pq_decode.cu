@@ -270,27 +270,12 @@ __device__ __forceinline__ void decode_range(int b, const DecodeLinear& L, int& 
 }
 constexpr int kDecodeMetaBytes = 256;   // token info at the start of a slot
 
-// mbarrier.try_wait with a suspend-time hint: a warp whose phase is not complete is parked by the hardware for up
-// to `ns` nanoseconds (it resumes at once when the phase completes) instead of coming back to poll after the short
-// default limit.  Most consumer warps of a CTA are waiting at any time; polling, they took most of the issue slots.
-__device__ __forceinline__ bool mbar_try_wait_parked(uint32_t bar, uint32_t parity, uint32_t ns) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity), "r"(ns)
-      : "memory");
-  return ok != 0;
-}
-
 // Wait with a bound.  Once any wait of the CTA has run out, every later wait returns at once, so that
 // all threads keep the same control flow and the kernel ends (with an error status and undefined output).
 __device__ __forceinline__ void decode_wait(uint32_t bar, uint32_t parity, volatile int* fail) {
   if (mbar_try_wait(bar, parity)) return;
   const long long t0 = clock64();
-  while (!mbar_try_wait_parked(bar, parity, 20000u)) {
+  while (!mbar_try_wait(bar, parity)) {
     if (*fail) return;
     if (clock64() - t0 > kSpinCycles) {
       report_timeout(WHERE_OTHER);
@@ -620,13 +605,16 @@ static int decode_sm_count() {
   return n;
 }
 
+constexpr size_t kDecodeMainSmemLimit = 226 * 1024;   // dynamic shared memory of k_decode_main (its barriers are static)
+constexpr size_t kDecodePrepSmemLimit = 200 * 1024;   // K bf16 values of one token
+
 // One launch pair for up to kDecodeMaxBatch independent linears.
 static int decode_launch_with(const DecodeItemArgs* items, int n, int nwarps, cudaStream_t st) {
   static int sms = decode_sm_count();
   // One CTA per SM.  Eight consumer warps keep up with what the buffer rings can hold in flight (measured: more warps,
   // or two smaller CTAs per SM, are not faster); sixteen only when a CTA's feature range needs more than eight tiles.
   const int nctas = sms;
-  const size_t smem_limit = 226 * 1024;   // dynamic part; the barriers are static
+  const size_t smem_limit = kDecodeMainSmemLimit;
   DecodeBatch bp{};
   bp.n = n; bp.nwarps = nwarps;
   size_t slot_bits = 0, slot_h = 0, q_bytes = 0, ring_stage = 0, prep_smem = 0;
@@ -691,9 +679,13 @@ static int decode_launch_with(const DecodeItemArgs* items, int n, int nwarps, cu
   if (smem_main > smem_limit) {
     return PQ_ERR_UNSUPPORTED;
   }
-  if (prep_smem > 200 * 1024) return PQ_ERR_UNSUPPORTED;
-  if (cudaFuncSetAttribute(k_decode_main, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_main) != cudaSuccess) return PQ_ERR_CUDA;
-  if (cudaFuncSetAttribute(k_decode_prep, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)prep_smem) != cudaSuccess) return PQ_ERR_CUDA;
+  if (prep_smem > kDecodePrepSmemLimit) return PQ_ERR_UNSUPPORTED;
+  // The opt-in limits are set once, to the largest request this file can make: a launch recorded in a CUDA graph
+  // keeps its own shared-memory size, and a later call with a smaller one must not lower the limit under it.
+  static const bool limits_set =
+      cudaFuncSetAttribute(k_decode_main, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDecodeMainSmemLimit) == cudaSuccess &&
+      cudaFuncSetAttribute(k_decode_prep, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDecodePrepSmemLimit) == cudaSuccess;
+  if (!limits_set) return PQ_ERR_CUDA;
 
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
