@@ -128,23 +128,20 @@ def roofline_time_s(layers, peaks):
 
 def run_ours(args):
     import torch
-    import torch.distributed as dist
     from paper_2602_22592_b200 import binding as pqb
     from paper_2602_22592_b200 import build as pqbuild
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
+    from paper_2602_22592_b200 import replicas
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback for the product path")
     torch.cuda.set_device(local)
     device = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=device)
+    reps = replicas.from_env("nccl", device)   # one replica per GPU, no collective on the data path
+    world, rank = reps.world, reps.rank
     if rank == 0:
         pqbuild.build()
-    if world > 1:
-        dist.barrier()
+    reps.barrier()
     pqb.lib()
     peaks, peak_kind = measured_peaks()
 
@@ -153,8 +150,7 @@ def run_ours(args):
     tokens = layers[0].T
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        reps.barrier()
         torch.cuda.synchronize()
 
     for _ in range(args.warmup):
@@ -185,16 +181,12 @@ def run_ours(args):
         barrier()
     pqb.pq_profile_events(kid, None, None)
     launches = pqb.pq_kernel_launches() - launches0
-    elapsed_ms = t0.elapsed_time(t1)
-    if world > 1:
-        tt = torch.tensor([elapsed_ms], device=device)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(tt.item())
+    elapsed_ms = reps.max_over_ranks(t0.elapsed_time(t1), device)
     code, where = pqb.pq_device_status()
     if code:
         raise RuntimeError(f"device-side wait timed out (where={where})")
     ms_per_step = elapsed_ms / args.steps
-    value = world * tokens / (ms_per_step * 1e-3)
+    value = reps.whole_job_rate(tokens, ms_per_step)
 
     dw_ms = float(np.mean([a.elapsed_time(b) for row in ev for a, b in row]))
     # algorithmic flops of the launch: dW = dY^T . (q/gamma) and, in the same launch, dB_e = dY^T . (g H)
@@ -280,14 +272,10 @@ def run_ours(args):
         drain()
         t1.record()
         barrier()
-        ms = t0.elapsed_time(t1)
-        if world > 1:
-            tt = torch.tensor([ms], device=device)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            ms = float(tt.item())
+        ms = reps.max_over_ranks(t0.elapsed_time(t1), device)
         bi = sum(t.numel() * t.element_size() for t in hx + hdy)
         bo = sum(t.numel() * t.element_size() for t in hy + hdx)
-        e2e = {"value": round(world * tokens / (ms / n_e2e * 1e-3), 1), "unit": "tokens/s", "h2d_bytes_per_step": bi,
+        e2e = {"value": round(reps.whole_job_rate(tokens, ms / n_e2e), 1), "unit": "tokens/s", "h2d_bytes_per_step": bi,
                "d2h_bytes_per_step": bo, "steps": n_e2e,
                "note": "X and dY of each projection copied from pinned host memory, Y and dX copied back, copies on their own streams overlapping the kernels; weights stay resident"}
 
@@ -313,8 +301,7 @@ def run_ours(args):
             "clocks": clk.summary(),
         }
         print(json.dumps(out))
-    if world > 1:
-        dist.destroy_process_group()
+    reps.close()
 
 
 # --------------------------------------------------------------------------- decode workload
@@ -335,18 +322,15 @@ def run_decode(args):
 
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback for the product path")
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
+    from paper_2602_22592_b200 import replicas
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
     device = torch.device("cuda", local)
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=device)
+    reps = replicas.from_env("nccl", device)   # one replica per GPU, no collective on the data path
+    world, rank = reps.world, reps.rank
     if rank == 0:
         pqbuild.build()
-    if world > 1:
-        dist.barrier()
+    reps.barrier()
     pqb.lib()
     peaks, peak_kind = measured_peaks()
     M = args.decode_tokens
@@ -413,12 +397,7 @@ def run_decode(args):
             g.replay()
         b.record()
         torch.cuda.synchronize()
-        ms = a.elapsed_time(b) / args.steps
-        if world > 1:
-            tt = torch.tensor([ms], device=device)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            ms = float(tt.item())
-        return ms
+        return reps.max_over_ranks(a.elapsed_time(b) / args.steps, device)
 
     launches0 = pqb.pq_kernel_launches()
     graph = capture(args.decode_batch)
@@ -469,7 +448,7 @@ def run_decode(args):
     nlin = len(layers)
     if rank == 0:
         out = {
-            "metric": "pQuant decode linear (packed 1-bit weights) tokens/s", "value": round(world * M * nlin / (ms_per_step * 1e-3), 1),
+            "metric": "pQuant decode linear (packed 1-bit weights) tokens/s", "value": round(reps.whole_job_rate(M * nlin, ms_per_step), 1),
             "unit": "token-linears/s", "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "u8 bit masks x s8 -> s32 (1-bit branch), bf16 -> f32 (experts)", "data": "synthetic",
@@ -489,14 +468,13 @@ def run_decode(args):
                       "note": "batches of two (what the gate and up projections of one block allow)"},
             "eager_ms_per_step": round(ms_eager, 4),
             "cpu_baseline": None,
-            "e2e": {"value": round(world * M * nlin / (ms_e2e * 1e-3), 1), "unit": "token-linears/s",
+            "e2e": {"value": round(reps.whole_job_rate(M * nlin, ms_e2e), 1), "unit": "token-linears/s",
                     "h2d_bytes_per_step": sum(t.numel() * t.element_size() for t in hx),
                     "d2h_bytes_per_step": sum(t.numel() * t.element_size() for t in hy), "steps": n_e2e},
             "gpu_launches": int(launches_per_step * args.steps), "clocks": clk.summary(),
         }
         print(json.dumps(out))
-    if world > 1:
-        dist.destroy_process_group()
+    reps.close()
 
 
 # --------------------------------------------------------------------------- oracle (CPU) arm
