@@ -95,6 +95,7 @@ struct DecodeBatch {
   int n;
   // shared-memory carve-up of k_decode_main (bytes from the 128-byte aligned base)
   int nwarps;               // consumer warps per CTA
+  int prep_rows;            // rows of K values k_decode_prep keeps in shared memory beside the token (2..8, two buffers)
   int nslot, nq, nring;     // depths of the three buffer rings
   int off_slots, slot_bytes, off_slot_h, off_q, q_bytes, off_ring, ring_stage_bytes;
 };
@@ -106,68 +107,118 @@ struct DecodeCursor {
   __device__ __forceinline__ void next(int n) { if (++idx == n) { idx = 0; phase ^= 1u; } }
 };
 
-constexpr int kPrepLoads = 16;   // 16-byte loads a lane keeps in flight while it walks a row of Wr or A_e
+// Wait with a bound.  Once any wait of the CTA has run out, every later wait returns at once, so that
+// all threads keep the same control flow and the kernel ends (with an error status and undefined output).
+__device__ __forceinline__ void decode_wait(uint32_t bar, uint32_t parity, volatile int* fail) {
+  if (mbar_try_wait(bar, parity)) return;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (*fail) return;
+    if (clock64() - t0 > kSpinCycles) {
+      report_timeout(WHERE_OTHER);
+      *fail = 1;
+      return;
+    }
+  }
+}
 
-// grid (slices, M, linears), 256 threads, dynamic shared memory: K bf16 values of the token
+// grid (slices, M, linears), 256 threads.  Dynamic shared memory: the token's K bf16 values, then two buffers of
+// `prep_rows` / 2 rows of K bf16 values each (router rows first, rows of A_e afterwards).  Whole rows arrive by bulk
+// copies, a round of rows at a time, the next round in flight while one is used, and the dot products run out of
+// shared memory: with plain loads every lane went to memory several times in a row for a long row, and that
+// latency was most of the kernel.
 __global__ void __launch_bounds__(256) k_decode_prep(const __grid_constant__ DecodeBatch bp) {
-  extern __shared__ uint4 xs4[];
+  extern __shared__ __align__(128) uint4 xs4[];
+  __shared__ __align__(8) uint64_t pbar[3];   // token; the two row buffers
   __shared__ float red_f[8];
   __shared__ int red_i[8];
   __shared__ float logit_sh[kMaxExperts];
+  __shared__ int fail_sh;
+  volatile int* fail = &fail_sh;
+  if (threadIdx.x == 0) {
+    fail_sh = 0;
+    for (int i = 0; i < 3; ++i) mbar_init(smem_u32(&pbar[i]), 1);
+    mbar_fence_init();
+  }
   pdl_launch_dependents();
   pdl_wait();   // X may come from the previous kernel; the buffers written here may still be read by it
+  __syncthreads();
   const DecodeLinear& L = bp.lin[blockIdx.z];
   const int m = blockIdx.y, slice = blockIdx.x;
   if (m >= L.M || slice >= L.slices) return;
   const int K = L.K, E = L.E, r = L.r;
-  const uint4* __restrict__ X = L.X;
-  const uint4* __restrict__ Wr = L.Wr;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int chunks = K >> 3;
-  const uint4* xrow = X + (long long)m * chunks;
+  const uint32_t row_bytes = (uint32_t)K * 2u;
+  const int R = bp.prep_rows >> 1;                             // rows of one buffer (<= 4, one per warp)
+  const uint4* rows4 = xs4 + chunks;
+  const uint32_t rows_s = smem_u32(xs4) + row_bytes;
+  // rounds of up to R rows of a [*, K] bf16 matrix alternate between the two buffers; all threads count them
+  int issued = 0, taken = 0;
+  uint32_t phase0 = 0, phase1 = 0;
+  auto issue = [&](const uint16_t* base, long long row0, int n) {
+    const int b = issued & 1;
+    if (threadIdx.x == 0) {
+      mbar_expect_tx(smem_u32(&pbar[1 + b]), (uint32_t)n * row_bytes);
+      for (int i = 0; i < n; ++i) bulk_load(rows_s + (uint32_t)(b * R + i) * row_bytes, base + (row0 + i) * K, row_bytes, smem_u32(&pbar[1 + b]));
+    }
+    ++issued;
+  };
+  auto take = [&]() {   // waits for the oldest round in flight and returns its buffer's first row
+    const int b = taken & 1;
+    decode_wait(smem_u32(&pbar[1 + b]), b ? phase1 : phase0, fail);
+    if (b) phase1 ^= 1u; else phase0 ^= 1u;
+    ++taken;
+    return rows4 + (size_t)(b * R) * chunks;
+  };
+
+  // the token, and with it the first two rounds of router rows
+  if (threadIdx.x == 0) {
+    mbar_expect_tx(smem_u32(&pbar[0]), row_bytes);
+    bulk_load(smem_u32(xs4), reinterpret_cast<const uint16_t*>(L.X) + (long long)m * K, row_bytes, smem_u32(&pbar[0]));
+  }
+  const uint16_t* Wr = reinterpret_cast<const uint16_t*>(L.Wr);
+  const int router_rounds = E > 1 ? (E + R - 1) / R : 0;
+  for (int k = 0; k < min(2, router_rounds); ++k) issue(Wr, k * R, min(R, E - k * R));
+  decode_wait(smem_u32(&pbar[0]), 0, fail);
   float amax = 0.f;
   for (int c = threadIdx.x; c < chunks; c += 256) {
-    const uint4 v = __ldg(xrow + c);
-    xs4[c] = v;
+    const uint4 v = xs4[c];
     amax = fmaxf(amax, fmaxf(fmaxf(fabsf(bf16lo(v.x)), fabsf(bf16hi(v.x))), fmaxf(fabsf(bf16lo(v.y)), fabsf(bf16hi(v.y)))));
     amax = fmaxf(amax, fmaxf(fmaxf(fabsf(bf16lo(v.z)), fabsf(bf16hi(v.z))), fmaxf(fabsf(bf16lo(v.w)), fabsf(bf16hi(v.w)))));
   }
   for (int d = 16; d > 0; d >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, d));
   if (lane == 0) red_f[warp] = amax;
-  __syncthreads();   // also publishes xs4
+  __syncthreads();
   amax = red_f[0];
 #pragma unroll
   for (int w = 1; w < 8; ++w) amax = fmaxf(amax, red_f[w]);
   const float gamma = __fdiv_rn(kActQmax, fmaxf(amax, kActAmaxFloor));
 
   // router: the same pinned fp32 order as the training path (lane j owns the chunks c = j mod 32, ascending,
-  // fused multiply-add; butterfly 16, 8, 4, 2, 1), one warp per expert
+  // fused multiply-add; butterfly 16, 8, 4, 2, 1), one warp per expert of the round
   int best = 0;
   float gate = 1.0f;
   if (E > 1) {
-    for (int e = warp; e < E; e += 8) {
-      float acc = 0.f;
-      const uint4* wrow = Wr + (long long)e * chunks;
-      // sixteen loads in flight per lane; the additions keep the ascending order of the chunks
-      for (int c0 = lane; c0 < chunks; c0 += 32 * kPrepLoads) {
-        uint4 wv[kPrepLoads];
-#pragma unroll
-        for (int u = 0; u < kPrepLoads; ++u) wv[u] = (c0 + 32 * u < chunks) ? __ldg(wrow + c0 + 32 * u) : make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll
-        for (int u = 0; u < kPrepLoads; ++u) {
-          if (c0 + 32 * u < chunks) {
-            const uint4 xv = xs4[c0 + 32 * u];
-            acc = fmaf(bf16lo(xv.x), bf16lo(wv[u].x), acc); acc = fmaf(bf16hi(xv.x), bf16hi(wv[u].x), acc);
-            acc = fmaf(bf16lo(xv.y), bf16lo(wv[u].y), acc); acc = fmaf(bf16hi(xv.y), bf16hi(wv[u].y), acc);
-            acc = fmaf(bf16lo(xv.z), bf16lo(wv[u].z), acc); acc = fmaf(bf16hi(xv.z), bf16hi(wv[u].z), acc);
-            acc = fmaf(bf16lo(xv.w), bf16lo(wv[u].w), acc); acc = fmaf(bf16hi(xv.w), bf16hi(wv[u].w), acc);
-          }
+    for (int k = 0; k < router_rounds; ++k) {
+      const int n = min(R, E - k * R);
+      const uint4* buf = take();
+      if (warp < n) {
+        float acc = 0.f;
+        const uint4* wrow = buf + (size_t)warp * chunks;
+        for (int c = lane; c < chunks; c += 32) {
+          const uint4 xv = xs4[c], wv = wrow[c];
+          acc = fmaf(bf16lo(xv.x), bf16lo(wv.x), acc); acc = fmaf(bf16hi(xv.x), bf16hi(wv.x), acc);
+          acc = fmaf(bf16lo(xv.y), bf16lo(wv.y), acc); acc = fmaf(bf16hi(xv.y), bf16hi(wv.y), acc);
+          acc = fmaf(bf16lo(xv.z), bf16lo(wv.z), acc); acc = fmaf(bf16hi(xv.z), bf16hi(wv.z), acc);
+          acc = fmaf(bf16lo(xv.w), bf16lo(wv.w), acc); acc = fmaf(bf16hi(xv.w), bf16hi(wv.w), acc);
         }
+        for (int d = 16; d > 0; d >>= 1) acc = acc + __shfl_xor_sync(0xffffffffu, acc, d);
+        if (lane == 0) logit_sh[k * R + warp] = acc;
       }
-      for (int d = 16; d > 0; d >>= 1) acc = acc + __shfl_xor_sync(0xffffffffu, acc, d);
-      if (lane == 0) logit_sh[e] = acc;
+      __syncthreads();                                         // this buffer is free, its logits are visible
+      if (k + 2 < router_rounds) issue(Wr, (k + 2) * R, min(R, E - (k + 2) * R));
     }
-    __syncthreads();
     float lmax = logit_sh[0];
     for (int e = 1; e < E; ++e)
       if (logit_sh[e] > lmax) { lmax = logit_sh[e]; best = e; }
@@ -179,6 +230,11 @@ __global__ void __launch_bounds__(256) k_decode_prep(const __grid_constant__ Dec
     }
     gate = pbest * (1.0f / den);
   }
+  // the first two rounds of this slice's rows of A_e are on their way while slice 0 quantises the token
+  const int j0 = slice * L.rows_per_slice, j1 = min(r, j0 + L.rows_per_slice);
+  const int h_rounds = (r > 0 && j0 < j1) ? (j1 - j0 + R - 1) / R : 0;
+  const long long arow0 = (long long)best * r + j0;
+  for (int k = 0; k < min(2, h_rounds); ++k) issue(L.A, arow0 + k * R, min(R, j1 - j0 - k * R));
 
   if (slice == 0) {
     // Eq. 7-9 for this token; every thread turns pairs of weight words (64 values of k) into fragment order
@@ -226,26 +282,20 @@ __global__ void __launch_bounds__(256) k_decode_prep(const __grid_constant__ Dec
     }
   }
 
-  // this slice of h = A_e x (fp32 accumulation over the bf16 operands), one warp per row
-  if (r > 0) {
-    const int j0 = slice * L.rows_per_slice, j1 = min(r, j0 + L.rows_per_slice);
-    for (int j = j0 + warp; j < j1; j += 8) {
-      const uint4* arow = reinterpret_cast<const uint4*>(L.A + ((long long)best * r + j) * K);
+  // this slice of h = A_e x (fp32 accumulation over the bf16 operands), one warp per row of the round
+  for (int k = 0; k < h_rounds; ++k) {
+    const int n = min(R, j1 - j0 - k * R);
+    const uint4* buf = take();
+    if (warp < n) {
+      const int j = j0 + k * R + warp;
+      const uint4* arow = buf + (size_t)warp * chunks;
       float a0 = 0.f, a1 = 0.f;
-      for (int c0 = lane; c0 < chunks; c0 += 32 * kPrepLoads) {
-        uint4 wv[kPrepLoads];
-#pragma unroll
-        for (int u = 0; u < kPrepLoads; ++u) wv[u] = (c0 + 32 * u < chunks) ? __ldg(arow + c0 + 32 * u) : make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll
-        for (int u = 0; u < kPrepLoads; ++u) {
-          if (c0 + 32 * u < chunks) {
-            const uint4 xv = xs4[c0 + 32 * u];
-            a0 = fmaf(bf16lo(xv.x), bf16lo(wv[u].x), a0); a1 = fmaf(bf16hi(xv.x), bf16hi(wv[u].x), a1);
-            a0 = fmaf(bf16lo(xv.y), bf16lo(wv[u].y), a0); a1 = fmaf(bf16hi(xv.y), bf16hi(wv[u].y), a1);
-            a0 = fmaf(bf16lo(xv.z), bf16lo(wv[u].z), a0); a1 = fmaf(bf16hi(xv.z), bf16hi(wv[u].z), a1);
-            a0 = fmaf(bf16lo(xv.w), bf16lo(wv[u].w), a0); a1 = fmaf(bf16hi(xv.w), bf16hi(wv[u].w), a1);
-          }
-        }
+      for (int c = lane; c < chunks; c += 32) {
+        const uint4 xv = xs4[c], wv = arow[c];
+        a0 = fmaf(bf16lo(xv.x), bf16lo(wv.x), a0); a1 = fmaf(bf16hi(xv.x), bf16hi(wv.x), a1);
+        a0 = fmaf(bf16lo(xv.y), bf16lo(wv.y), a0); a1 = fmaf(bf16hi(xv.y), bf16hi(wv.y), a1);
+        a0 = fmaf(bf16lo(xv.z), bf16lo(wv.z), a0); a1 = fmaf(bf16hi(xv.z), bf16hi(wv.z), a1);
+        a0 = fmaf(bf16lo(xv.w), bf16lo(wv.w), a0); a1 = fmaf(bf16hi(xv.w), bf16hi(wv.w), a1);
       }
       float a = a0 + a1;
       for (int d = 16; d > 0; d >>= 1) a += __shfl_xor_sync(0xffffffffu, a, d);
@@ -260,6 +310,10 @@ __global__ void __launch_bounds__(256) k_decode_prep(const __grid_constant__ Dec
         base[pos + (long long)rsteps * 32 * 8] = __bfloat16_as_ushort(lo);
       }
     }
+    if (k + 2 < h_rounds) {
+      __syncthreads();                                         // this buffer is free
+      issue(L.A, arow0 + (k + 2) * R, min(R, j1 - j0 - (k + 2) * R));
+    }
   }
 }
 
@@ -269,21 +323,6 @@ __device__ __forceinline__ void decode_range(int b, const DecodeLinear& L, int& 
   n_hi = n_lo + ((L.grp_base + (b < L.grp_rem ? 1 : 0)) << 3);
 }
 constexpr int kDecodeMetaBytes = 256;   // token info at the start of a slot
-
-// Wait with a bound.  Once any wait of the CTA has run out, every later wait returns at once, so that
-// all threads keep the same control flow and the kernel ends (with an error status and undefined output).
-__device__ __forceinline__ void decode_wait(uint32_t bar, uint32_t parity, volatile int* fail) {
-  if (mbar_try_wait(bar, parity)) return;
-  const long long t0 = clock64();
-  while (!mbar_try_wait(bar, parity)) {
-    if (*fail) return;
-    if (clock64() - t0 > kSpinCycles) {
-      report_timeout(WHERE_OTHER);
-      *fail = 1;
-      return;
-    }
-  }
-}
 
 // Experts used by the tokens [8 G, 8 G + 8) as a bit mask; producer and consumers walk it in ascending order.
 __device__ __forceinline__ unsigned decode_expert_mask(const DecodeTokInfo* tok, int M, int G) {
@@ -618,7 +657,7 @@ static int decode_launch_with(const DecodeItemArgs* items, int n, int nwarps, cu
   DecodeBatch bp{};
   bp.n = n; bp.nwarps = nwarps;
   size_t slot_bits = 0, slot_h = 0, q_bytes = 0, ring_stage = 0, prep_smem = 0;
-  int max_slices = 1, max_m = 1;
+  int max_slices = 1, max_m = 1, max_k = 0;
   for (int i = 0; i < n; ++i) {
     const DecodeItemArgs& it = items[i];
     const int M = it.a.T, K = it.a.K, N = it.a.N, r = it.a.r;
@@ -632,18 +671,6 @@ static int decode_launch_with(const DecodeItemArgs* items, int n, int nwarps, cu
     L.X = reinterpret_cast<const uint4*>(it.X); L.Wr = reinterpret_cast<const uint4*>(it.a.Wr); L.A = it.a.A; L.B = it.a.B;
     L.bits = it.bits; L.w_scales = it.a.w_scales; L.alpha = it.a.alpha; L.beta = it.a.beta; L.Y = it.Y;
     L.M = M; L.K = K; L.N = N; L.r = r; L.E = (r > 0 && it.a.E > 1) ? it.a.E : 1; L.sstride = it.a.scale_stride;
-    // Slices of the hidden rows: whole rounds of eight rows (one per warp), and enough CTAs in the grid (about
-    // eight per SM) that the rows of A_e stream at full rate; every slice repeats the token's absmax and router.
-    L.slices = 1; L.rows_per_slice = 1;
-    if (r > 0) {
-      int slices = (8 * sms + M * n - 1) / (M * n);
-      const int most = (r + 7) / 8;
-      if (slices > most) slices = most;
-      if (slices < 1) slices = 1;
-      L.rows_per_slice = ((r + slices - 1) / slices + 7) / 8 * 8;
-      L.slices = (r + L.rows_per_slice - 1) / L.rows_per_slice;
-    }
-    if (L.slices > max_slices) max_slices = L.slices;
     if (M > max_m) max_m = M;
     const int groups = N / 8;
     L.grp_base = groups / nctas; L.grp_rem = groups % nctas;
@@ -653,7 +680,7 @@ static int decode_launch_with(const DecodeItemArgs* items, int n, int nwarps, cu
     slot_h = std::max(slot_h, r > 0 ? up256((size_t)((M + 7) / 8) * 2 * ((r + 31) / 32) * 512) : (size_t)0);   // token groups in use only
     q_bytes = std::max(q_bytes, up256(npairs * (size_t)std::min(M, 8) * 64));
     ring_stage = std::max(ring_stage, up256((size_t)max_cols * r * 2));
-    prep_smem = std::max(prep_smem, (size_t)K * 2);
+    max_k = std::max(max_k, K);
   }
   // Buffer rings: at least two slots, one activation buffer and (with experts) two expert-row buffers; then
   // deeper, in turn, while shared memory lasts, so that the loads of several linears are in flight at once.
@@ -679,7 +706,27 @@ static int decode_launch_with(const DecodeItemArgs* items, int n, int nwarps, cu
   if (smem_main > smem_limit) {
     return PQ_ERR_UNSUPPORTED;
   }
-  if (prep_smem > kDecodePrepSmemLimit) return PQ_ERR_UNSUPPORTED;
+  // token preparation: the token and up to eight rows (router rows, then rows of A_e) of K bf16 values each
+  bp.prep_rows = (int)std::min<size_t>(8, (kDecodePrepSmemLimit - (size_t)max_k * 2) / ((size_t)max_k * 2)) & ~1;   // two buffers
+  if (bp.prep_rows < 2) return PQ_ERR_UNSUPPORTED;
+  prep_smem = (size_t)max_k * 2 * (1 + bp.prep_rows);
+  // Slices of the hidden rows: whole rounds of rows, as many slices as keep the grid within
+  // one wave of resident CTAs (every slice repeats the token's absmax and router, and rounds run one after another).
+  const int resident = sms * std::max<int>(1, (int)((227 * 1024) / (prep_smem + 1024)));
+  int total_tokens = 0;
+  for (int i = 0; i < n; ++i) total_tokens += items[i].a.T;
+  for (int i = 0; i < n; ++i) {
+    DecodeLinear& L = bp.lin[i];
+    L.slices = 1; L.rows_per_slice = 1;
+    if (L.r > 0) {
+      int slices = std::max(1, resident / std::max(1, total_tokens));
+      slices = std::min(slices, (L.r + 7) / 8);
+      const int round_rows = bp.prep_rows / 2;
+      L.rows_per_slice = ((L.r + slices - 1) / slices + round_rows - 1) / round_rows * round_rows;
+      L.slices = (L.r + L.rows_per_slice - 1) / L.rows_per_slice;
+    }
+    max_slices = std::max(max_slices, L.slices);
+  }
   // The opt-in limits are set once, to the largest request this file can make: a launch recorded in a CUDA graph
   // keeps its own shared-memory size, and a later call with a smaller one must not lower the limit under it.
   static const bool limits_set =
