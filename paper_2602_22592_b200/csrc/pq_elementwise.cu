@@ -17,20 +17,28 @@ __global__ void __launch_bounds__(256) k_weight_partial_sums(const float4* __res
   double s = 0.0, a = 0.0;
   const long long stride = gridDim.x * 256LL;
   long long i = blockIdx.x * 256LL + threadIdx.x;
-  // four loads in flight per thread; the order of the additions is fixed by the launch shape alone
+  // One conversion to fp64 per element (the conversion is the slow instruction here); |x| is taken on the double,
+  // which is the same number as the double of |x|.  The order of the additions is fixed by the launch shape alone.
+  auto sums = [](const float4& v, double& ts, double& ta) {
+    const double d0 = (double)v.x, d1 = (double)v.y, d2 = (double)v.z, d3 = (double)v.w;
+    ts = d0 + d1 + d2 + d3;
+    ta = fabs(d0) + fabs(d1) + fabs(d2) + fabs(d3);
+  };
+  // four loads in flight per thread
   for (; i + 3 * stride < n4; i += 4 * stride) {
     const float4 v0 = __ldg(W4 + i), v1 = __ldg(W4 + i + stride), v2 = __ldg(W4 + i + 2 * stride), v3 = __ldg(W4 + i + 3 * stride);
-    s += ((double)v0.x + (double)v0.y + (double)v0.z + (double)v0.w) + ((double)v1.x + (double)v1.y + (double)v1.z + (double)v1.w);
-    s += ((double)v2.x + (double)v2.y + (double)v2.z + (double)v2.w) + ((double)v3.x + (double)v3.y + (double)v3.z + (double)v3.w);
-    a += ((double)fabsf(v0.x) + (double)fabsf(v0.y) + (double)fabsf(v0.z) + (double)fabsf(v0.w)) +
-         ((double)fabsf(v1.x) + (double)fabsf(v1.y) + (double)fabsf(v1.z) + (double)fabsf(v1.w));
-    a += ((double)fabsf(v2.x) + (double)fabsf(v2.y) + (double)fabsf(v2.z) + (double)fabsf(v2.w)) +
-         ((double)fabsf(v3.x) + (double)fabsf(v3.y) + (double)fabsf(v3.z) + (double)fabsf(v3.w));
+    double s0, a0, s1, a1, s2, a2, s3, a3;
+    sums(v0, s0, a0); sums(v1, s1, a1); sums(v2, s2, a2); sums(v3, s3, a3);
+    s += s0 + s1;
+    s += s2 + s3;
+    a += a0 + a1;
+    a += a2 + a3;
   }
   for (; i < n4; i += stride) {
-    const float4 v = __ldg(W4 + i);
-    s += (double)v.x + (double)v.y + (double)v.z + (double)v.w;
-    a += (double)fabsf(v.x) + (double)fabsf(v.y) + (double)fabsf(v.z) + (double)fabsf(v.w);
+    double s0, a0;
+    sums(__ldg(W4 + i), s0, a0);
+    s += s0;
+    a += a0;
   }
   for (int d = 16; d > 0; d >>= 1) {
     s += __shfl_xor_sync(0xffffffffu, s, d);
@@ -513,7 +521,8 @@ static inline int grid_for(long long work, int per_block, int cap) {
 
 cudaError_t launch_pack(const float* W, int N, int K, uint32_t* bits, int8_t* s8, float* scales, double* partial, cudaStream_t st) {
   const long long n4 = (long long)N * K / 4;
-  const int nparts = grid_for(n4, 256 * 8, 2 * 148);   // two blocks per SM, each thread keeps four loads in flight
+  const int nparts = grid_for(n4, 256 * 8, 6 * 148);   // six blocks per SM, each thread keeps four loads in flight (~14 MB in all)
+  static_assert(6 * 148 <= kPackPartials, "partial sums of the weight reduction");
   { LaunchScope ls(KID_PACK_SUMS, st);
   k_weight_partial_sums<<<nparts, 256, 0, st>>>(reinterpret_cast<const float4*>(W), n4, partial); }
   const int grid = grid_for(n4, 256 * 4, 148 * 8);
