@@ -2,7 +2,7 @@
 //
 // One CTA per SM, 320 threads: warp 0 = TMA producer, warp 1 = MMA issuer
 // (also owns the TMEM allocation), warps 2-9 = epilogue (two per TMEM lane
-// quadrant, which take alternate column chunks of the tile).  Operands travel global -> shared by TMA into a 4-stage ring of
+// quadrant, which take alternate column chunks of the tile).  Operands travel global -> shared by TMA into a ring (4 stages of 48 KB; more, smaller ones for narrow tiles) of
 // 128-byte-swizzled tiles; tcgen05.mma accumulates 128 x (<=256) tiles in
 // TMEM; the epilogue reads them back with tcgen05.ld.
 //
@@ -17,22 +17,24 @@
 #pragma once
 #include <cuda.h>
 
+#include <type_traits>
+
 #include "pq_common.cuh"
 
 namespace pq {
 
 constexpr int kEpiWarps = 8;
 constexpr int kGemmThreads = 64 + 32 * kEpiWarps;
-constexpr int kStages = 4;
+constexpr int kMaxStages = 8;             // barrier pairs reserved for the operand ring
 constexpr int kTileM = 128;
 constexpr int kStageABytes = 128 * 128;  // 128 rows x 128 B, or two 64x64 bf16 MN boxes
 constexpr int kStageBBytes = 256 * 128;  // up to 256 rows x 128 B, or four MN boxes
-constexpr int kStageBytes = kStageABytes + kStageBBytes;
+constexpr int kRingBytes = 4 * (kStageABytes + kStageBBytes);   // operand ring: four stages of a 256-column tile
 constexpr int kMnBoxBytes = 64 * 128;    // one MN-major box: 64 k-rows of 64 bf16
 constexpr int kTmemCols = 512;
 constexpr int kAccCols = 256;            // TMEM columns of one accumulator stage in the default layout
 constexpr int kEpiWarpBytes = 32 * 128;                // per epilogue warp: 32 rows of one 128-byte chunk (xor-swizzled)
-constexpr int kGemmSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ + kEpiWarps * kEpiWarpBytes;
+constexpr int kGemmSmemBytes = kRingBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ + kEpiWarps * kEpiWarpBytes;
 static_assert(kGemmSmemBytes <= 227 * 1024, "shared memory of one CTA");
 
 enum OpMode : int {
@@ -133,6 +135,17 @@ __device__ __forceinline__ void warp_store_rows(uint8_t* stage, const uint4 (&v)
 // Problems whose epilogue needs nothing fetched ahead of the accumulator
 struct NoPre {};
 
+// Widest B operand of a launch, in tile columns (B takes that many x 128 bytes of a stage): the ring holds as many
+// stages as fit, so a launch of narrow tiles keeps more k-blocks in flight.  Problems without `stage_cols` use 256.
+template <class P, class = void>
+struct stage_cols_of {
+  __device__ static int get(const typename P::Params&) { return 256; }
+};
+template <class P>
+struct stage_cols_of<P, std::void_t<decltype(&P::stage_cols)>> {
+  __device__ static int get(const typename P::Params& p) { return P::stage_cols(p); }
+};
+
 // Accumulator layouts in TMEM (column of accumulator `acc` of pipeline stage `stage`).
 //   AccDouble     : one accumulator per tile, two stages of 256 columns.
 //   AccPair       : two accumulators of 256 columns per tile (all of TMEM), one stage: the epilogue of
@@ -151,15 +164,17 @@ __device__ __forceinline__ void gemm_body(const typename P::Params& p) {
   extern __shared__ uint8_t smem_raw[];
   using Acc = typename P::Acc;
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t bar_base = smem_base + kStages * kStageBytes;
-  // barrier block: full[4] empty[4] tfull[2] tempty[2] (8 B each), then tmem ptr, abort flag
+  const uint32_t kStageBytes = kStageABytes + (uint32_t)stage_cols_of<P>::get(p) * 128u;   // a multiple of 1024
+  const int kStages = min(kMaxStages, (int)(kRingBytes / kStageBytes));
+  const uint32_t bar_base = smem_base + kRingBytes;
+  // barrier block: full[8] empty[8] tfull[2] tempty[2] (8 B each), then tmem ptr, abort flag
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
-  auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
-  auto tfull_bar = [&](int s) { return bar_base + 8u * (2 * kStages + s); };
-  auto tempty_bar = [&](int s) { return bar_base + 8u * (2 * kStages + 2 + s); };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (kMaxStages + s); };
+  auto tfull_bar = [&](int s) { return bar_base + 8u * (2 * kMaxStages + s); };
+  auto tempty_bar = [&](int s) { return bar_base + 8u * (2 * kMaxStages + 2 + s); };
   uint8_t* bar_generic = smem_raw + (bar_base - smem_u32(smem_raw));
-  volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(bar_generic + 8 * (2 * kStages + 5));
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_generic + 8 * (2 * kStages + 5) + 8);
+  volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(bar_generic + 8 * (2 * kMaxStages + 5));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_generic + 8 * (2 * kMaxStages + 5) + 8);
   uint8_t* epi_stage = bar_generic + 256;  // kEpiWarps x kEpiWarpBytes
 
   constexpr int kAccStages = Acc::kStages;

@@ -215,6 +215,7 @@ struct HpUpProblem {
     int K, r, bn, item_rows;
   };
   struct Tile { int item; int4 it; };
+  __device__ static int stage_cols(const Params& p) { return p.bn <= 128 ? 128 : 256; }
   __device__ static int num_tiles(const Params& p) { return p.rt.n_items[0]; }
   __device__ static void tile_init(const Params& p, int i, Tile& t) { t.item = i; t.it = p.rt.items[i]; }
   __device__ static int num_segments(const Params&, const Tile&) { return 1; }
@@ -440,6 +441,7 @@ struct HpDhProblem {
     int T, N, r, E, bn, sstride, item_rows, ba_blk;
   };
   struct Tile { int item; int4 it; };
+  __device__ static int stage_cols(const Params& p) { return p.bn <= 128 ? 128 : 256; }
   __device__ static int num_tiles(const Params& p) { return p.rt.n_items[0]; }
   __device__ static void tile_init(const Params& p, int i, Tile& t) { t.item = i; t.it = p.rt.items[i]; }
   __device__ static int num_segments(const Params&, const Tile&) { return 1; }
