@@ -446,6 +446,9 @@ def run_decode(args):
 
     gbs = algo / (ms_per_step * 1e-3) / 1e9
     nlin = len(layers)
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        cpu_baseline = oracle_decode_baseline(M, hid, ffn, r, E)
     if rank == 0:
         out = {
             "metric": "pQuant decode linear (packed 1-bit weights) tokens/s", "value": round(reps.whole_job_rate(M * nlin, ms_per_step), 1),
@@ -467,7 +470,7 @@ def run_decode(args):
                       "hbm_frac": round(algo / (ms_pairs * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
                       "note": "batches of two (what the gate and up projections of one block allow)"},
             "eager_ms_per_step": round(ms_eager, 4),
-            "cpu_baseline": None,
+            "cpu_baseline": cpu_baseline,
             "e2e": {"value": round(reps.whole_job_rate(M * nlin, ms_e2e), 1), "unit": "token-linears/s",
                     "h2d_bytes_per_step": sum(t.numel() * t.element_size() for t in hx),
                     "d2h_bytes_per_step": sum(t.numel() * t.element_size() for t in hy), "steps": n_e2e},
@@ -506,6 +509,28 @@ def oracle_baseline(E, sample_tokens):
             "sample": (f"first {sample_tokens} of 8192 tokens through pack + forward + backward of the three projections "
                        f"({dt:.1f} s; the per-matrix weight quantisation does not shrink with the sample, so this understates "
                        "the full-batch rate)")}
+
+
+def oracle_decode_baseline(M, hid, ffn, r, E):
+    """The oracle's decode forward as it stands on one layer's three linears (weights packed beforehand, as on the GPU)."""
+    from oracle import pquant_oracle as O
+    from paper_2602_22592_b200 import inputs as I
+    rng = np.random.default_rng(7)
+    prepared = []
+    for i, (_, K, N) in enumerate(I.mlp_shapes(hid, ffn)):
+        W = (rng.standard_normal((N, K), dtype=np.float32) * np.float32(0.02))
+        mu, lam = O.weight_scales(W)
+        bits = O.pack_bits(O.binarize(W, mu))
+        A = I.bf16_values(rng.standard_normal((E, r, K), dtype=np.float32) * np.float32(0.02))
+        B = I.bf16_values(rng.standard_normal((E, N, r), dtype=np.float32) * np.float32(0.02))
+        act = I.decode_activations(M, K, E, seed=9000 + i)
+        prepared.append((act["X"], bits, lam, A, B, act["Wr"]))
+    t = time.perf_counter()
+    for X, bits, lam, A, B, Wr in prepared:
+        O.decode_forward(X, bits, lam, A, B, Wr, 2.0, 0.2)
+    dt = time.perf_counter() - t
+    return {"value": round(M * len(prepared) / dt, 1), "unit": "token-linears/s", "cores": oracle_threads(), "kind": "oracle",
+            "sample": f"the three linears of one layer ({M} token(s) each, {dt:.1f} s), weights packed beforehand"}
 
 
 def run_reference(args):
