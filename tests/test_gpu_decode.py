@@ -89,6 +89,49 @@ def test_decode_is_deterministic_and_repeatable():
     assert torch.equal(y, L.Y)
 
 
+def test_decode_in_a_cuda_graph_and_without_dependent_launch():
+    # Launches of different shapes (hence different shared-memory sizes) recorded in one CUDA graph replay to the
+    # same bits as the eager calls, also after a later, smaller call; and the plain-launch option gives the same.
+    shapes = [dict(T=2, K=2048, N=4096, r=64, E=4), dict(T=1, K=256, N=96, r=32, E=4), dict(T=11, K=1024, N=2560, r=160, E=8)]
+    layers = []
+    for i, kw in enumerate(shapes):
+        c = I.make_linear_case(kw["T"], kw["K"], kw["N"], kw["r"], kw["E"], seed=70 + i, exact_quota=False, with_grad=False)
+        L = PQLinear(c["T"], c["K"], c["N"], c["r"], c["E"], training=False, dump_acc=True).load_case(c)
+        L.pack(bits_only=True)
+        layers.append(L)
+    eager = []
+    for L in layers:
+        L.decode()
+        torch.cuda.synchronize()
+        eager.append(L.Y.clone())
+    stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream):
+            for L in layers:
+                L.decode()
+    layers[1].decode()                               # a small call after the capture
+    torch.cuda.synchronize()
+    for L in layers:
+        L.Y.zero_()
+    for _ in range(2):
+        graph.replay()
+    torch.cuda.synchronize()
+    check_status()
+    for L, y in zip(layers, eager):
+        assert torch.equal(L.Y, y)
+    pqb.pq_set_option(pqb.PQ_OPT_DECODE_PDL, 0)
+    try:
+        for L, y in zip(layers, eager):
+            L.Y.zero_()
+            L.decode()
+            torch.cuda.synchronize()
+            assert torch.equal(L.Y, y)
+    finally:
+        pqb.pq_set_option(pqb.PQ_OPT_DECODE_PDL, 1)
+    check_status()
+
+
 def test_decode_batch_of_independent_linears():
     # a mixed batch (different shapes, token counts, expert counts; more than one launch group of 16)
     # gives exactly what the separate calls give, and matches the oracle
