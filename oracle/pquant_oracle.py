@@ -349,8 +349,29 @@ def linear_backward(dY, X, fwd, A=None, B=None, Wr=None, alpha=1.0, beta=1.0):
     return g
 
 
-def decode_forward(X, bits, lam, A=None, B=None, Wr=None, alpha=1.0, beta=1.0):
+def rmsnorm(X, weight, eps):
+    """RMSNorm in front of the activation quantiser (App. A: at inference the norm is
+    fused with the quantisation; the equations write it as LayerNorm(X)).
+
+    Per token row: x / sqrt(mean_k x^2 + eps) * weight.  The paper fixes no
+    precision; the reading taken is: the mean of squares and the reciprocal
+    square root in fp64, that factor rounded once to fp32, then two fp32
+    multiplies per element (by the factor, then by the gain), and one rounding
+    to bf16 -- the values a separate bf16 norm layer would have handed over.
+    """
+    X32 = np.asarray(X, dtype=np.float32)
+    w32 = np.asarray(weight, dtype=np.float32)
+    ms = np.mean(np.square(X32.astype(np.float64)), axis=1)
+    rinv = (1.0 / np.sqrt(ms + np.float64(np.float32(eps)))).astype(np.float32)
+    y = ((X32 * rinv[:, None]).astype(np.float32) * w32[None, :]).astype(np.float32)
+    return round_to_bf16(y.astype(np.float64)).astype(np.float32)
+
+
+def decode_forward(X, bits, lam, A=None, B=None, Wr=None, alpha=1.0, beta=1.0, norm_weight=None, norm_eps=1e-6):
     """Inference path (App. A): same forward, with S read back out of the
-    packed 1-bit words instead of the latent weights."""
+    packed 1-bit words instead of the latent weights; with `norm_weight` the
+    input is the un-normalised activation and RMSNorm comes first."""
+    if norm_weight is not None:
+        X = rmsnorm(X, norm_weight, norm_eps)
     K = np.asarray(X).shape[1]
     return linear_forward(X, None, A, B, Wr, alpha, beta, S=unpack_bits(bits, K), lam=lam)

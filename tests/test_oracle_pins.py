@@ -341,3 +341,47 @@ def test_library_matmul_special_case():
     assert np.array_equal(acc.numpy().astype(np.int64), f["acc"])
     h = torch.from_numpy(c["X"].astype(np.float64)) @ torch.from_numpy(c["A"][0].astype(np.float64)).T
     assert np.allclose(h.numpy(), f["h"], rtol=1e-13)
+
+
+def test_rmsnorm_closed_forms_and_library_routine():
+    # App. A / Sec. 4.5: RMSNorm fused with the activation quantiser at inference.
+    rng = np.random.default_rng(11)
+    K = 384
+    X = O.round_to_bf16(rng.standard_normal((5, K)) * 3.0)
+    w = O.round_to_bf16(1.0 + 0.1 * rng.standard_normal(K))
+    # constant rows: c / sqrt(c^2 + eps) * w
+    for c in (0.5, -2.0, 8.0):
+        y = O.rmsnorm(np.full((1, K), c), np.ones(K), 1e-6)
+        assert np.allclose(y, c / np.sqrt(c * c + 1e-6), rtol=2.0 ** -8)
+    # a power-of-two rescaling of the input changes nothing when eps = 0
+    assert np.array_equal(O.rmsnorm(X, w, 0.0), O.rmsnorm(4.0 * X, w, 0.0))
+    # unit mean square before the gain (within the bf16 rounding of the outputs)
+    y1 = O.rmsnorm(X, np.ones(K), 0.0).astype(np.float64)
+    assert np.allclose(np.mean(y1 * y1, axis=1), 1.0, rtol=2.0 ** -7)
+    # the library routine in fp64, rounded to bf16, differs by at most one bf16 step
+    import torch
+    ref = torch.nn.functional.rms_norm(torch.from_numpy(np.asarray(X, np.float64)), (K,), torch.from_numpy(np.asarray(w, np.float64)), 1e-5).numpy()
+    y = O.rmsnorm(X, w, 1e-5).astype(np.float64)
+    assert np.all(np.abs(y - ref) <= 2.0 ** -7 * np.abs(ref) + 1e-30)
+    # planted mistakes are caught by the same comparison: eps dropped into the wrong place, mean of |x| instead of x^2
+    wrong1 = X / (np.sqrt(np.mean(X * X, axis=1, keepdims=True)) + 1e-1) * w
+    wrong2 = X / np.mean(np.abs(X), axis=1, keepdims=True) * w
+    for wrong in (wrong1, wrong2):
+        assert not np.all(np.abs(wrong - ref) <= 2.0 ** -7 * np.abs(ref) + 1e-30)
+    # every output is a bf16 value
+    assert np.array_equal(O.round_to_bf16(y), y)
+
+
+def test_decode_with_fused_norm_is_norm_then_decode():
+    rng = np.random.default_rng(12)
+    K, N = 128, 64
+    X = O.round_to_bf16(rng.standard_normal((3, K)) * 2.0)
+    w = O.round_to_bf16(1.0 + 0.2 * rng.standard_normal(K))
+    W = rng.standard_normal((N, K)).astype(np.float32)
+    mu, lam = O.weight_scales(W)
+    bits = O.pack_bits(O.binarize(W, mu))
+    a = O.decode_forward(X, bits, lam, norm_weight=w, norm_eps=1e-5)
+    b = O.decode_forward(O.rmsnorm(X, w, 1e-5), bits, lam)
+    assert np.array_equal(a["Y"], b["Y"]) and np.array_equal(a["q"], b["q"])
+    c = O.decode_forward(X, bits, lam)
+    assert not np.array_equal(a["q"], c["q"])
