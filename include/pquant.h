@@ -194,6 +194,14 @@ typedef struct pq_decode_item {
   uint16_t* Y;             /* [T,N] bf16 (out) */
   void* ws;                /* pq_workspace_bytes(&desc, PQ_PHASE_DECODE) bytes */
   size_t ws_bytes;
+  /* RMSNorm fused in front of the activation quantiser (App. A, Sec. 4.5: at inference the
+   * norm is fused with the quantisation).  norm_weight [K] bf16 (device) or NULL: X arrives
+   * normalised.  With it, X is the un-normalised activation and every use of the token (its
+   * quantisation, the router, the expert branch) sees
+   *   bf16( fp32( fp32(x * s) * norm_weight ) ),   s = fp32( 1 / sqrt(mean_k x^2 + norm_eps) ),
+   * the mean and the reciprocal square root taken in fp64. */
+  const uint16_t* norm_weight;
+  float norm_eps;
 } pq_decode_item;
 int pq_decode_batch(const pq_decode_item* items, int n, void* stream);
 
@@ -220,8 +228,8 @@ int pq_linear_backward(const pq_desc* d, const uint16_t* dY, const uint16_t* X,
 int pq_debug_gemm(int mode, int M, int N, int K, const void* A, const void* B, void* D,
                   void* stream);
 /* Same with the width of the output tiles chosen by the caller (the layer's kernels
- * use 256, 160 for the forward tile with an HP branch, and narrower pieces in the last
- * wave): tile_n a multiple of 32 (modes 0, 1) or 64 (modes 2, 3), at most 256. */
+ * use 256, or 128 for the two small products of the HP branch): tile_n a multiple of 32
+ * (modes 0, 1) or 64 (modes 2, 3), at most 256. */
 int pq_debug_gemm_tile(int mode, int M, int N, int K, const void* A, const void* B, void* D,
                        int tile_n, void* stream);
 

@@ -50,7 +50,8 @@ class pq_saved_view(ctypes.Structure):
 
 class pq_decode_item(ctypes.Structure):
     _fields_ = [("desc", pq_desc)] + [(n, ctypes.c_void_p) for n in
-                                      ("X", "w_bits", "w_scales", "A", "B", "Wr", "alpha", "beta", "Y", "ws")] + [("ws_bytes", ctypes.c_size_t)]
+                                      ("X", "w_bits", "w_scales", "A", "B", "Wr", "alpha", "beta", "Y", "ws")] + [
+        ("ws_bytes", ctypes.c_size_t), ("norm_weight", ctypes.c_void_p), ("norm_eps", ctypes.c_float)]
 
 
 class pq_decode_view(ctypes.Structure):
@@ -201,10 +202,15 @@ def pq_linear_forward(d, X, w_bits, w_s8, w_scales, A, B, Wr, alpha, beta, Y, sa
 
 
 def make_decode_items(entries):
-    """ctypes array of pq_decode_item from (desc, X, w_bits, w_scales, A, B, Wr, alpha, beta, Y, ws) tuples of tensors.
+    """ctypes array of pq_decode_item from (desc, X, w_bits, w_scales, A, B, Wr, alpha, beta, Y, ws[, norm_weight, norm_eps])
+    tuples of tensors (the last two: bf16 RMSNorm gain [K] and its epsilon, for un-normalised X).
     The array only holds pointers: keep the tensors alive while it is in use."""
     arr = (pq_decode_item * len(entries))()
-    for i, (d, X, w_bits, w_scales, A, B, Wr, alpha, beta, Y, ws) in enumerate(entries):
+    for i, entry in enumerate(entries):
+        d, X, w_bits, w_scales, A, B, Wr, alpha, beta, Y, ws = entry[:11]
+        norm_weight, norm_eps = (entry[11], entry[12]) if len(entry) > 11 else (None, 0.0)
+        arr[i].norm_weight = None if norm_weight is None else norm_weight.data_ptr()
+        arr[i].norm_eps = float(norm_eps)
         arr[i].desc = d
         for name, t in (("X", X), ("w_bits", w_bits), ("w_scales", w_scales), ("A", A), ("B", B), ("Wr", Wr), ("alpha", alpha),
                         ("beta", beta), ("Y", Y), ("ws", ws)):

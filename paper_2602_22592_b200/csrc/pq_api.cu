@@ -338,6 +338,9 @@ int pq_decode_batch(const pq_decode_item* items, int n, void* stream) {
     args[i].a = LayerArgs{d->T, d->K, d->N, d->r, experts_of(d), (d->flags & PQ_SCALE_VECTOR) ? 1 : 0, it.w_scales, it.alpha, it.beta, it.A, it.B, it.Wr};
     args[i].X = it.X; args[i].bits = it.w_bits; args[i].Y = it.Y; args[i].ws = it.ws;
     args[i].dump = (d->flags & PQ_DECODE_DUMP_ACC) != 0;
+    if (misaligned(it.norm_weight)) { rc = PQ_ERR_ALIGN; break; }
+    if (it.norm_weight && !(it.norm_eps >= 0.f)) { rc = PQ_ERR_SHAPE; break; }
+    args[i].norm_weight = it.norm_weight; args[i].norm_eps = it.norm_eps;
   }
   if (rc == PQ_OK) rc = decode_batch(args, n, static_cast<cudaStream_t>(stream));
   delete[] args;

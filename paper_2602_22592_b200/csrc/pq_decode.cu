@@ -86,6 +86,8 @@ struct DecodeLinear {
   uint4* qfrag;             // [2, npairs, 32] fragments
   uint4* hfrag;             // [2 groups][2 planes (hi, lo)][ceil(r/32)][32] fragments of h = A_e x
   int* acc_dump;            // [M, N] exact 1-bit accumulators (test hook) or null
+  const uint4* norm_w;      // [K] bf16 RMSNorm gain or null
+  float norm_eps;
   int M, K, N, r, E, sstride, slices, rows_per_slice;
   // partition of the N / 8 feature groups over the CTAs of k_decode_main: the first `grp_rem` CTAs own grp_base + 1 groups
   int grp_base, grp_rem;
@@ -181,6 +183,36 @@ __global__ void __launch_bounds__(256) k_decode_prep(const __grid_constant__ Dec
   const int router_rounds = E > 1 ? (E + R - 1) / R : 0;
   for (int k = 0; k < min(2, router_rounds); ++k) issue(Wr, k * R, min(R, E - k * R));
   decode_wait(smem_u32(&pbar[0]), 0, fail);
+  if (L.norm_w) {
+    // RMSNorm fused in front of the quantiser (App. A): mean of squares and its reciprocal root in fp64 (thread sums
+    // in ascending chunk order, then a fixed tree), the factor rounded once to fp32; the token in shared memory is
+    // replaced by bf16(fp32(fp32(x s) w)), which every later step reads.
+    __shared__ double red_d[8];
+    double ss = 0.0;
+    for (int c = threadIdx.x; c < chunks; c += 256) {
+      const uint4 v = xs4[c];
+      const double d0 = bf16lo(v.x), d1 = bf16hi(v.x), d2 = bf16lo(v.y), d3 = bf16hi(v.y);
+      const double d4 = bf16lo(v.z), d5 = bf16hi(v.z), d6 = bf16lo(v.w), d7 = bf16hi(v.w);
+      ss += ((d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3)) + ((d4 * d4 + d5 * d5) + (d6 * d6 + d7 * d7));
+    }
+    for (int d = 16; d > 0; d >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, d);
+    if (lane == 0) red_d[warp] = ss;
+    __syncthreads();
+    double tot = 0.0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) tot += red_d[w];
+    const float s = (float)(1.0 / sqrt(tot / (double)K + (double)L.norm_eps));
+    for (int c = threadIdx.x; c < chunks; c += 256) {
+      const uint4 v = xs4[c], g = __ldg(L.norm_w + c);
+      uint4 o;
+      o.x = pack_bf16x2(__fmul_rn(__fmul_rn(bf16lo(v.x), s), bf16lo(g.x)), __fmul_rn(__fmul_rn(bf16hi(v.x), s), bf16hi(g.x)));
+      o.y = pack_bf16x2(__fmul_rn(__fmul_rn(bf16lo(v.y), s), bf16lo(g.y)), __fmul_rn(__fmul_rn(bf16hi(v.y), s), bf16hi(g.y)));
+      o.z = pack_bf16x2(__fmul_rn(__fmul_rn(bf16lo(v.z), s), bf16lo(g.z)), __fmul_rn(__fmul_rn(bf16hi(v.z), s), bf16hi(g.z)));
+      o.w = pack_bf16x2(__fmul_rn(__fmul_rn(bf16lo(v.w), s), bf16lo(g.w)), __fmul_rn(__fmul_rn(bf16hi(v.w), s), bf16hi(g.w)));
+      xs4[c] = o;
+    }
+    // each thread reads back only the chunks it wrote itself in the pass below; the barrier after it publishes them
+  }
   float amax = 0.f;
   for (int c = threadIdx.x; c < chunks; c += 256) {
     const uint4 v = xs4[c];
@@ -670,6 +702,7 @@ static int decode_launch_with(const DecodeItemArgs* items, int n, int nwarps, cu
     L.acc_dump = it.dump ? reinterpret_cast<int*>(w) : nullptr;
     L.X = reinterpret_cast<const uint4*>(it.X); L.Wr = reinterpret_cast<const uint4*>(it.a.Wr); L.A = it.a.A; L.B = it.a.B;
     L.bits = it.bits; L.w_scales = it.a.w_scales; L.alpha = it.a.alpha; L.beta = it.a.beta; L.Y = it.Y;
+    L.norm_w = reinterpret_cast<const uint4*>(it.norm_weight); L.norm_eps = it.norm_eps;
     L.M = M; L.K = K; L.N = N; L.r = r; L.E = (r > 0 && it.a.E > 1) ? it.a.E : 1; L.sstride = it.a.scale_stride;
     if (M > max_m) max_m = M;
     const int groups = N / 8;

@@ -94,7 +94,11 @@ int gemm_forward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, co
 size_t decode_workspace_bytes(int M, int K, int N, int r, bool dump);
 int decode_forward(const LayerArgs& a, const uint16_t* X, const uint32_t* bits, uint16_t* Y, void* ws, bool dump, cudaStream_t st);
 struct DecodeViewPtrs { void* tokens; int* acc; };
-struct DecodeItemArgs { LayerArgs a; const uint16_t* X; const uint32_t* bits; uint16_t* Y; void* ws; bool dump; };
+struct DecodeItemArgs {
+  LayerArgs a; const uint16_t* X; const uint32_t* bits; uint16_t* Y; void* ws; bool dump;
+  const uint16_t* norm_weight = nullptr;   // RMSNorm gain [K] bf16, or null: X arrives normalised
+  float norm_eps = 0.f;
+};
 int decode_batch(const DecodeItemArgs* items, int n, cudaStream_t st);   // independent linears, launched together
 void decode_set_pdl(int on);
 DecodeViewPtrs decode_view(int M, int K, int N, int r, void* ws, bool dump);

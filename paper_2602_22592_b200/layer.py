@@ -82,14 +82,23 @@ class PQLinear:
         pqb.pq_pack_weights(self.desc, self.W, self.w_bits, None if bits_only else self.w_s8, self.w_scales, self.ws_pack)
 
     def decode(self, X=None, Y=None):
-        """Inference forward from the packed sign bits (w_s8 is not used)."""
+        """Inference forward from the packed sign bits (w_s8 is not used).  With `norm_weight` set, X is the
+        un-normalised activation and RMSNorm is fused in front of the quantiser (a batch of one)."""
+        if getattr(self, "norm_weight", None) is not None:
+            entry = list(self.decode_entry())
+            if X is not None: entry[1] = X
+            if Y is not None: entry[9] = Y
+            items = pqb.make_decode_items([tuple(entry)])
+            pqb.pq_decode_batch(items)
+            return self.Y if Y is None else Y
         pqb.pq_linear_forward(self.desc, self.X if X is None else X, self.w_bits, None, self.w_scales, self.A, self.B, self.Wr,
                               self.alpha, self.beta, self.Y if Y is None else Y, None, self.ws_decode)
         return self.Y if Y is None else Y
 
     def decode_entry(self):
         """This layer's arguments as one entry for binding.make_decode_items."""
-        return (self.desc, self.X, self.w_bits, self.w_scales, self.A, self.B, self.Wr, self.alpha, self.beta, self.Y, self.ws_decode)
+        return (self.desc, self.X, self.w_bits, self.w_scales, self.A, self.B, self.Wr, self.alpha, self.beta, self.Y, self.ws_decode,
+                getattr(self, "norm_weight", None), getattr(self, "norm_eps", 0.0))
 
     def decode_view(self) -> dict:
         return pqb.pq_decode_view_init(self.desc, self.ws_decode)

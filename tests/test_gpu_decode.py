@@ -68,6 +68,39 @@ def test_decode_3b_shapes(M, proj):
     check_decode(c, run_decode(c))
 
 
+@pytest.mark.parametrize("name", ["m1_small", "m5_odd_words", "m16_two_groups", "m12_vector_scales", "m3_pure_1bit"])
+def test_decode_with_fused_rmsnorm(name):
+    # App. A: RMSNorm fused in front of the activation quantiser.  X is the un-normalised activation (here the case's
+    # tokens stretched row by row); codes, routing and the 1-bit sums must still agree exactly with the oracle.
+    kw = dict(DECODE_CASES[name])
+    scale_vector = kw.pop("scale_vector", False)
+    c = I.make_linear_case(kw.pop("T"), kw.pop("K"), kw.pop("N"), kw.pop("r"), kw.pop("E"), seed=31, exact_quota=False, with_grad=False,
+                           scale_vector=scale_vector, **kw)
+    rng = np.random.default_rng(5)
+    c["X"] = I.bf16_values(c["X"] * rng.uniform(0.25, 6.0, size=(c["T"], 1)).astype(np.float32))
+    w = I.bf16_values(1.0 + 0.1 * rng.standard_normal(c["K"]).astype(np.float32))
+    eps = 1e-5
+    L = PQLinear(c["T"], c["K"], c["N"], c["r"], c["E"], scale_vector=scale_vector, training=False, dump_acc=True).load_case(c)
+    L.norm_weight = torch.from_numpy(w).to(L.X.device).to(torch.bfloat16)
+    L.norm_eps = eps
+    L.pack(bits_only=True)
+    L.decode()
+    torch.cuda.synchronize()
+    check_status()
+    mu, lam = O.weight_scales(c["W"])
+    bits = O.pack_bits(O.binarize(c["W"], mu))
+    f = O.decode_forward(c["X"], bits, lam, c["A"], c["B"], c["Wr"], c["alpha"], c["beta"], norm_weight=w, norm_eps=eps)
+    v = L.decode_view()
+    assert np.array_equal(v["expert"].cpu().numpy(), f["idx"])
+    assert np.array_equal(f32(v["gamma"]), f["gamma"])
+    assert np.array_equal(v["code_sum"].cpu().numpy(), f["q"].astype(np.int64).sum(axis=1))
+    assert np.array_equal(v["acc"].cpu().numpy().astype(np.int64), f["acc"])
+    assert rel_err(f32(L.Y), f["Y"]) <= TOL_BF16
+    # and it is not the un-normalised result
+    g = O.decode_forward(c["X"], bits, lam, c["A"], c["B"], c["Wr"], c["alpha"], c["beta"])
+    assert not np.array_equal(g["q"], f["q"])
+
+
 def test_decode_agrees_with_training_forward():
     c = I.make_linear_case(16, 512, 768, 64, 4, seed=5, exact_quota=False, with_grad=False)
     Ld = run_decode(c)
