@@ -353,6 +353,9 @@ def run_decode(args):
             L.Wr = torch.from_numpy(act["Wr"]).to(device).to(torch.bfloat16)
             L.alpha = torch.full((1,), 2.0, device=device)
             L.beta = torch.full((1,), 0.2, device=device)
+            if args.decode_rmsnorm:
+                L.norm_weight = (1.0 + 0.1 * torch.randn((K,), generator=gen, device=device)).to(torch.bfloat16)
+                L.norm_eps = 1e-5
             layers.append(L)
     torch.cuda.synchronize()
 
@@ -456,7 +459,8 @@ def run_decode(args):
             "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "u8 bit masks x s8 -> s32 (1-bit branch), bf16 -> f32 (experts)", "data": "synthetic",
             "config": {"workload": (f"decode, {M} token(s): {DECODE_LAYERS} layers x gate/up/down of a 3B-shaped model (hidden {hid}, FFN {ffn}), "
-                                    f"1-bit weights packed 32 per word, {E} bf16 experts of width {r}, top-1, Zipf(1.1)"),
+                                    f"1-bit weights packed 32 per word, {E} bf16 experts of width {r}, top-1, Zipf(1.1)"
+                                    + (", RMSNorm fused in front of the quantiser" if args.decode_rmsnorm else "")),
                        "linears_per_step": nlin, "l2": f"{algo / 1e6:.0f} MB of distinct weights per step, larger than L2",
                        "launch": f"one CUDA graph per step, pq_decode_batch over groups of {args.decode_batch} independent linears", "replicas": world},
             "roofline": {"kernel": "k_decode_prep + k_decode_main (all launches of a step)", "bound": "hbm", "achieved": round(gbs, 1),
@@ -569,6 +573,7 @@ def main():
     ap.add_argument("--decode-tokens", type=int, default=1, choices=range(1, 17), metavar="M")
     ap.add_argument("--decode-skip-serial", action="store_true", help="time only the batched graph (shorter runs under a profiler)")
     ap.add_argument("--decode-batch", type=int, default=16, help="independent decode linears per pq_decode_batch call")
+    ap.add_argument("--decode-rmsnorm", action="store_true", help="decode from un-normalised activations, RMSNorm fused into the token preparation")
     ap.add_argument("--cpu-tokens", type=int, default=4096)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
