@@ -520,12 +520,15 @@ __global__ void __launch_bounds__(kDecodeMainThreads) k_decode_main(const __grid
       const int row0 = 16 * my_tile + g, row1 = row0 + 8;    // this thread's two features (local index)
       const bool has0 = row0 < ncols, has1 = row1 < ncols;
       // per-feature factors of the epilogue, fetched before anything is waited for
-      const float lam = L.w_scales[0];
+      float lam = L.w_scales[0];
       float be0 = 0.f, be1 = 0.f, al0 = 0.f, al1 = 0.f;
       if (has0) { be0 = L.beta[(n_lo + row0) * L.sstride]; if (L.r > 0) al0 = L.alpha[(n_lo + row0) * L.sstride]; }
       if (has1) { be1 = L.beta[(n_lo + row1) * L.sstride]; if (L.r > 0) al1 = L.alpha[(n_lo + row1) * L.sstride]; }
       const int mg = min(8, L.M - 8 * G);
       decode_wait(q_full(qb), q_phase, fail);
+      // the epilogue's factors are in registers from here on: their loads were issued before the wait and must not
+      // be moved down to their first use, where a warp would sit out a trip to global memory per tile
+      asm volatile("" : "+f"(lam), "+f"(be0), "+f"(be1), "+f"(al0), "+f"(al1));
 
       // ---- 1-bit product: masked sums, weight 1 and weight 16; two independent chains of accumulators.
       // Threads of tokens that do not exist read the last token's fragments (their results are never stored),
