@@ -199,7 +199,8 @@ typedef struct pq_decode_item {
    * normalised.  With it, X is the un-normalised activation and every use of the token (its
    * quantisation, the router, the expert branch) sees
    *   bf16( fp32( fp32(x * s) * norm_weight ) ),   s = fp32( 1 / sqrt(mean_k x^2 + norm_eps) ),
-   * the mean and the reciprocal square root taken in fp64. */
+   * the mean and the reciprocal square root taken in fp64.  norm_eps > 0 (PQ_ERR_SHAPE otherwise:
+   * an all-zero token would divide by zero). */
   const uint16_t* norm_weight;
   float norm_eps;
 } pq_decode_item;

@@ -339,7 +339,7 @@ int pq_decode_batch(const pq_decode_item* items, int n, void* stream) {
     args[i].X = it.X; args[i].bits = it.w_bits; args[i].Y = it.Y; args[i].ws = it.ws;
     args[i].dump = (d->flags & PQ_DECODE_DUMP_ACC) != 0;
     if (misaligned(it.norm_weight)) { rc = PQ_ERR_ALIGN; break; }
-    if (it.norm_weight && !(it.norm_eps >= 0.f)) { rc = PQ_ERR_SHAPE; break; }
+    if (it.norm_weight && !(it.norm_eps > 0.f)) { rc = PQ_ERR_SHAPE; break; }   // an all-zero token needs it
     args[i].norm_weight = it.norm_weight; args[i].norm_eps = it.norm_eps;
   }
   if (rc == PQ_OK) rc = decode_batch(args, n, static_cast<cudaStream_t>(stream));

@@ -101,6 +101,29 @@ def test_decode_with_fused_rmsnorm(name):
     assert not np.array_equal(g["q"], f["q"])
 
 
+def test_fused_rmsnorm_zero_token_and_bad_epsilon():
+    c = I.make_linear_case(3, 256, 96, 32, 4, seed=33, exact_quota=False, with_grad=False)
+    c["X"][1, :] = 0.0                                  # an all-zero token: normalised to zeros, codes all zero
+    w = I.bf16_values(np.linspace(0.5, 1.5, c["K"]).astype(np.float32))
+    L = PQLinear(c["T"], c["K"], c["N"], c["r"], c["E"], training=False, dump_acc=True).load_case(c)
+    L.norm_weight = torch.from_numpy(w).to(L.X.device).to(torch.bfloat16)
+    L.norm_eps = 1e-6
+    L.pack(bits_only=True)
+    L.decode()
+    torch.cuda.synchronize()
+    check_status()
+    mu, lam = O.weight_scales(c["W"])
+    bits = O.pack_bits(O.binarize(c["W"], mu))
+    f = O.decode_forward(c["X"], bits, lam, c["A"], c["B"], c["Wr"], c["alpha"], c["beta"], norm_weight=w, norm_eps=1e-6)
+    v = L.decode_view()
+    assert np.array_equal(v["acc"].cpu().numpy().astype(np.int64), f["acc"])
+    assert int(v["code_sum"][1]) == 0 and np.array_equal(f32(v["gamma"]), f["gamma"])
+    assert rel_err(f32(L.Y), f["Y"]) <= TOL_BF16
+    L.norm_eps = 0.0
+    with pytest.raises(pqb.PqError):
+        L.decode()
+
+
 def test_decode_agrees_with_training_forward():
     c = I.make_linear_case(16, 512, 768, 64, 4, seed=5, exact_quota=False, with_grad=False)
     Ld = run_decode(c)
