@@ -125,6 +125,8 @@ static __device__ __align__(256) double g_pack_scratch[2 * kStaticMaxSlabs];
 // One block per slab of kStaticSlabElems consecutive elements: {sum, sum of |.|} in fp64,
 // a fixed order inside the block, so the result does not depend on scheduling.
 __global__ void __launch_bounds__(256) k_weight_slab_sums(const float4* __restrict__ W4, long long n4, double* __restrict__ partial) {
+  pdl_launch_dependents();   // launched with programmatic stream serialisation: see launch_pdl
+  pdl_wait();
   const long long base = (long long)blockIdx.x * (kStaticSlabElems / 4);
   double s = 0.0, a = 0.0;
   for (int i = threadIdx.x; i < kStaticSlabElems / 4; i += 256) {
@@ -176,12 +178,12 @@ static int pack_static(const float* W, int N, int K, uint32_t* bits, int8_t* s8,
   const long long n4 = elems / 4;
   {
     LaunchScope ls(KID_PACK_SUMS, st);
-    k_weight_slab_sums<<<(int)slabs, 256, 0, st>>>(reinterpret_cast<const float4*>(W), n4, scratch);
+    launch_pdl(k_weight_slab_sums, (int)slabs, 256, 0, st, reinterpret_cast<const float4*>(W), n4, scratch);
   }
   long long g = (n4 + 1023) / 1024;
   const int grid = (int)(g < 1 ? 1 : (g > 148 * 8 ? 148 * 8 : g));
   LaunchScope ls(KID_BINARIZE_PACK, st);
-  k_binarize_pack<<<grid, 256, 0, st>>>(reinterpret_cast<const float4*>(W), n4, scratch, (int)slabs, 1.0 / (double)elems, bits,
+  launch_pdl(k_binarize_pack, grid, 256, 0, st, reinterpret_cast<const float4*>(W), n4, scratch, (int)slabs, 1.0 / (double)elems, bits,
                                         reinterpret_cast<uint32_t*>(s8), scales);
   return cudaGetLastError() == cudaSuccess ? PQ_OK : PQ_ERR_CUDA;
 }

@@ -79,6 +79,10 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int whe
   return true;
 }
 
+// programmatic dependent launch: let the next kernel in the stream start early / wait for the previous one
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---------------------------------------------------------------------------
 // TMA (cp.async.bulk.tensor), loads only, no multicast
 // ---------------------------------------------------------------------------

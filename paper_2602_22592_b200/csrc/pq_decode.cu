@@ -39,9 +39,6 @@ struct DecodeTokInfo {  // one per token, written by k_decode_prep
   int rowsum;           // sum over k of q[k]
 };
 
-// programmatic dependent launch: let the next kernel in the stream start early / wait for the previous one
-__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"

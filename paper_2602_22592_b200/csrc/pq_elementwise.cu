@@ -14,6 +14,8 @@ long long g_launches = 0;
 // reduction tree, so the result does not depend on scheduling.
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) k_weight_partial_sums(const float4* __restrict__ W4, long long n4, double* __restrict__ partial) {
+  pdl_launch_dependents();   // launched with programmatic stream serialisation: see launch_pdl
+  pdl_wait();
   double s = 0.0, a = 0.0;
   const long long stride = gridDim.x * 256LL;
   long long i = blockIdx.x * 256LL + threadIdx.x;
@@ -86,6 +88,8 @@ __device__ __forceinline__ void reduce_partials(const double* partial, int npart
 __global__ void __launch_bounds__(256) k_binarize_pack(const float4* __restrict__ W4, long long n4, const double* __restrict__ partial,
                                                        int nparts, double inv_count, uint32_t* __restrict__ bits,
                                                        uint32_t* __restrict__ s8x4, float* __restrict__ scales) {
+  pdl_launch_dependents();   // launched with programmatic stream serialisation: see launch_pdl
+  pdl_wait();
   float mu, lam;
   reduce_partials(partial, nparts, inv_count, &mu, &lam);
   if (blockIdx.x == 0 && threadIdx.x == 0) { scales[0] = lam; scales[1] = mu; }
@@ -131,6 +135,8 @@ __global__ void __launch_bounds__(256) k_binarize_pack(const float4* __restrict_
 __global__ void __launch_bounds__(1024) k_router(const uint4* __restrict__ X, const uint4* __restrict__ Wr, int T, int K, int E,
                                                  int* __restrict__ expert, float* __restrict__ gate_tok,
                                                  float* __restrict__ probs_tok, int* __restrict__ block_counts) {
+  pdl_launch_dependents();   // launched with programmatic stream serialisation: see launch_pdl
+  pdl_wait();
   __shared__ int cnt[kMaxExperts];
   if (threadIdx.x < kMaxExperts) cnt[threadIdx.x] = 0;
   __syncthreads();
@@ -226,6 +232,8 @@ __device__ __forceinline__ int tile_items(const int* off, int Ee, int r0, int r1
 
 __global__ void __launch_bounds__(512) k_route_scan(int T, int E, int nblocks, const int* __restrict__ block_counts,
                                                     int* __restrict__ block_base, int* __restrict__ offsets, RoutingTables rt) {
+  pdl_launch_dependents();   // launched with programmatic stream serialisation: see launch_pdl
+  pdl_wait();
   __shared__ int off[kMaxExperts + 1];
   __shared__ int total[kMaxExperts];
   __shared__ int warp_sums[16];
@@ -321,6 +329,8 @@ __global__ void __launch_bounds__(256) k_act_quant(const uint4* __restrict__ X, 
                                                    uint2* __restrict__ q, uint4* __restrict__ xt, uint4* __restrict__ xs,
                                                    float* __restrict__ gamma_s, float* __restrict__ gate_s, float* __restrict__ probs_s,
                                                    int* __restrict__ perm, int* __restrict__ pos) {
+  pdl_launch_dependents();   // launched with programmatic stream serialisation: see launch_pdl
+  pdl_wait();
   __shared__ float amax_sh[8];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int sub = warp % WPR, slot = sub * 32 + lane;   // this lane's first 16-byte piece of the row
@@ -414,6 +424,8 @@ __global__ void __launch_bounds__(256) k_act_quant(const uint4* __restrict__ X, 
 // dst[pos[t], :] = src[t, :]  (rows of `chunks` 16-byte pieces), one warp per row
 __global__ void __launch_bounds__(256) k_scatter_rows(const uint4* __restrict__ src, uint4* __restrict__ dst, const int* __restrict__ pos,
                                                       int T, int chunks) {
+  pdl_launch_dependents();   // launched with programmatic stream serialisation: see launch_pdl
+  pdl_wait();
   const int t = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
   if (t >= T) return;
   const uint4* s = src + (long long)t * chunks;
@@ -424,6 +436,8 @@ __global__ void __launch_bounds__(256) k_scatter_rows(const uint4* __restrict__ 
 // Sb[n,k] = bf16(scale_n) * S[n,k]; scale_n = beta_n (vector form) or 1
 __global__ void __launch_bounds__(256) k_scaled_sign(const uint4* __restrict__ s8, uint4* __restrict__ out, const float* __restrict__ beta,
                                                      int beta_stride, int N, int K) {
+  pdl_launch_dependents();   // launched with programmatic stream serialisation: see launch_pdl
+  pdl_wait();
   const long long n16 = (long long)N * K / 16;
   const int per_row = K / 16;
   for (long long i = blockIdx.x * 256LL + threadIdx.x; i < n16; i += gridDim.x * 256LL) {
@@ -448,6 +462,8 @@ __global__ void __launch_bounds__(256) k_scaled_sign(const uint4* __restrict__ s
 // Ba[e,n,j] = bf16(alpha_n * B[e,n,j])  (vector alpha only)
 __global__ void __launch_bounds__(256) k_scaled_b(const uint32_t* __restrict__ B2, uint32_t* __restrict__ out, const float* __restrict__ alpha,
                                                   int E, int N, int r) {
+  pdl_launch_dependents();   // launched with programmatic stream serialisation: see launch_pdl
+  pdl_wait();
   const long long n2 = (long long)E * N * r / 2;
   const int per_row = r / 2;
   for (long long i = blockIdx.x * 256LL + threadIdx.x; i < n2; i += gridDim.x * 256LL) {
@@ -463,6 +479,8 @@ __global__ void __launch_bounds__(128) k_finalize_scales(const float* __restrict
                                                          const float* __restrict__ dalpha_partial, int E, int N,
                                                          const float* __restrict__ w_scales, float* __restrict__ dbeta,
                                                          float* __restrict__ dalpha) {
+  pdl_launch_dependents();   // launched with programmatic stream serialisation: see launch_pdl
+  pdl_wait();
   const int n = blockIdx.x * 128 + threadIdx.x;
   if (n >= N) return;
   float b = 0.f;
@@ -480,6 +498,8 @@ __global__ void __launch_bounds__(128) k_finalize_scales(const float* __restrict
 // Scalar feature scales: out_b[0] = sum_n vb[n], out_a[0] = sum_n va[n] (va may be null); one block, fp64, fixed tree.
 __global__ void __launch_bounds__(1024) k_sum_scales(const float* __restrict__ vb, const float* __restrict__ va, int N,
                                                      float* __restrict__ out_b, float* __restrict__ out_a) {
+  pdl_launch_dependents();   // launched with programmatic stream serialisation: see launch_pdl
+  pdl_wait();
   __shared__ double sh[2][32];
   double sb = 0.0, sa = 0.0;
   for (int n = threadIdx.x; n < N; n += 1024) {
@@ -507,6 +527,8 @@ __global__ void __launch_bounds__(1024) k_sum_scales(const float* __restrict__ v
 }
 
 __global__ void k_fill_zero(uint4* p, long long n16) {
+  pdl_launch_dependents();   // launched with programmatic stream serialisation: see launch_pdl
+  pdl_wait();
   for (long long i = blockIdx.x * 256LL + threadIdx.x; i < n16; i += gridDim.x * 256LL) p[i] = make_uint4(0, 0, 0, 0);
 }
 
@@ -524,10 +546,10 @@ cudaError_t launch_pack(const float* W, int N, int K, uint32_t* bits, int8_t* s8
   const int nparts = grid_for(n4, 256 * 8, 6 * 148);   // six blocks per SM, each thread keeps four loads in flight (~14 MB in all)
   static_assert(6 * 148 <= kPackPartials, "partial sums of the weight reduction");
   { LaunchScope ls(KID_PACK_SUMS, st);
-  k_weight_partial_sums<<<nparts, 256, 0, st>>>(reinterpret_cast<const float4*>(W), n4, partial); }
+  launch_pdl(k_weight_partial_sums, nparts, 256, 0, st, reinterpret_cast<const float4*>(W), n4, partial); }
   const int grid = grid_for(n4, 256 * 4, 148 * 8);
   LaunchScope ls(KID_BINARIZE_PACK, st);
-  k_binarize_pack<<<grid, 256, 0, st>>>(reinterpret_cast<const float4*>(W), n4, partial, nparts, 1.0 / ((double)N * K), bits,
+  launch_pdl(k_binarize_pack, grid, 256, 0, st, reinterpret_cast<const float4*>(W), n4, partial, nparts, 1.0 / ((double)N * K), bits,
                                         reinterpret_cast<uint32_t*>(s8), scales);
   return cudaGetLastError();
 }
@@ -537,11 +559,11 @@ cudaError_t launch_route_and_quant(const uint16_t* X, const uint16_t* Wr, int T,
   const int nblocks = (T + kRouterTokensPerBlock - 1) / kRouterTokensPerBlock;
   if (E > 1) {
     LaunchScope ls(KID_ROUTER, st);
-    k_router<<<nblocks, 32 * kRouterTokensPerBlock, 0, st>>>(reinterpret_cast<const uint4*>(X), reinterpret_cast<const uint4*>(Wr), T, K, E, sv.expert, sc.gate_tok,
+    launch_pdl(k_router, nblocks, 32 * kRouterTokensPerBlock, 0, st, reinterpret_cast<const uint4*>(X), reinterpret_cast<const uint4*>(Wr), T, K, E, sv.expert, sc.gate_tok,
                                       sc.probs_tok, sc.block_counts);
   }
   { LaunchScope ls(KID_ROUTE_SCAN, st);
-  k_route_scan<<<1, 512, 0, st>>>(T, E, nblocks, sc.block_counts, sc.block_base, sv.offsets, sv.rt); }
+  launch_pdl(k_route_scan, 1, 512, 0, st, T, E, nblocks, sc.block_counts, sc.block_base, sv.offsets, sv.rt); }
   LaunchScope ls(KID_ACT_QUANT, st);
   const int per_lane = (K / 8 + 31) / 32;   // 16-byte pieces of a row per lane if one warp took the whole row
   auto kern = k_act_quant<0, 1>;
@@ -551,7 +573,7 @@ cudaError_t launch_route_and_quant(const uint16_t* X, const uint16_t* Wr, int T,
   else if (per_lane <= 16) { kern = k_act_quant<8, 2>; wpr = 2; }
   else if (per_lane <= 32) { kern = k_act_quant<8, 4>; wpr = 4; }
   const int rows_per_block = 8 / wpr;
-  kern<<<(T + rows_per_block - 1) / rows_per_block, 256, 0, st>>>(reinterpret_cast<const uint4*>(X), T, K, E, sv.expert, sc.block_base, sv.offsets, sc.gate_tok,
+  launch_pdl(kern, (T + rows_per_block - 1) / rows_per_block, 256, 0, st, reinterpret_cast<const uint4*>(X), T, K, E, sv.expert, sc.block_base, sv.offsets, sc.gate_tok,
                                     sc.probs_tok, reinterpret_cast<uint2*>(sv.q), reinterpret_cast<uint4*>(sv.xt),
                                     reinterpret_cast<uint4*>(sv.xs), sv.gamma, sv.gate, sv.probs, sv.perm, sv.pos);
   return cudaGetLastError();
@@ -559,14 +581,14 @@ cudaError_t launch_route_and_quant(const uint16_t* X, const uint16_t* Wr, int T,
 
 cudaError_t launch_scatter_rows(const uint16_t* src, uint16_t* dst, const int* pos, int T, int row_elems, cudaStream_t st) {
   LaunchScope ls(KID_SCATTER_ROWS, st);
-  k_scatter_rows<<<(T + 7) / 8, 256, 0, st>>>(reinterpret_cast<const uint4*>(src), reinterpret_cast<uint4*>(dst), pos, T, row_elems / 8);
+  launch_pdl(k_scatter_rows, (T + 7) / 8, 256, 0, st, reinterpret_cast<const uint4*>(src), reinterpret_cast<uint4*>(dst), pos, T, row_elems / 8);
   return cudaGetLastError();
 }
 
 cudaError_t launch_scaled_sign(const int8_t* s8, uint16_t* out, const float* beta, int beta_stride, int N, int K, cudaStream_t st) {
   const long long n16 = (long long)N * K / 16;
   LaunchScope ls(KID_SCALED_SIGN, st);
-  k_scaled_sign<<<grid_for(n16, 256 * 2, 148 * 8), 256, 0, st>>>(reinterpret_cast<const uint4*>(s8), reinterpret_cast<uint4*>(out), beta,
+  launch_pdl(k_scaled_sign, grid_for(n16, 256 * 2, 148 * 8), 256, 0, st, reinterpret_cast<const uint4*>(s8), reinterpret_cast<uint4*>(out), beta,
                                                                beta_stride, N, K);
   return cudaGetLastError();
 }
@@ -574,7 +596,7 @@ cudaError_t launch_scaled_sign(const int8_t* s8, uint16_t* out, const float* bet
 cudaError_t launch_scaled_b(const uint16_t* B, uint16_t* out, const float* alpha, int E, int N, int r, cudaStream_t st) {
   const long long n2 = (long long)E * N * r / 2;
   LaunchScope ls(KID_SCALED_B, st);
-  k_scaled_b<<<grid_for(n2, 256 * 4, 148 * 8), 256, 0, st>>>(reinterpret_cast<const uint32_t*>(B), reinterpret_cast<uint32_t*>(out), alpha, E, N, r);
+  launch_pdl(k_scaled_b, grid_for(n2, 256 * 4, 148 * 8), 256, 0, st, reinterpret_cast<const uint32_t*>(B), reinterpret_cast<uint32_t*>(out), alpha, E, N, r);
   return cudaGetLastError();
 }
 
@@ -582,12 +604,12 @@ cudaError_t launch_finalize_scales(const float* dbeta_partial, int nslots, const
                                    int vec, float* dbeta, float* dalpha, float* tmp_b, float* tmp_a, cudaStream_t st) {
   {
     LaunchScope ls(KID_SUM_PARTIALS, st);
-    k_finalize_scales<<<(N + 127) / 128, 128, 0, st>>>(dbeta_partial, nslots, dalpha_partial, E, N, w_scales, vec ? dbeta : tmp_b,
+    launch_pdl(k_finalize_scales, (N + 127) / 128, 128, 0, st, dbeta_partial, nslots, dalpha_partial, E, N, w_scales, vec ? dbeta : tmp_b,
                                                        vec ? dalpha : tmp_a);
   }
   if (!vec) {
     LaunchScope ls(KID_SUM_SCALAR, st);
-    k_sum_scales<<<1, 1024, 0, st>>>(tmp_b, dalpha_partial ? tmp_a : nullptr, N, dbeta, dalpha);
+    launch_pdl(k_sum_scales, 1, 1024, 0, st, tmp_b, dalpha_partial ? tmp_a : nullptr, N, dbeta, dalpha);
   }
   return cudaGetLastError();
 }
@@ -595,7 +617,7 @@ cudaError_t launch_finalize_scales(const float* dbeta_partial, int nslots, const
 cudaError_t launch_fill_zero(void* p, size_t bytes, cudaStream_t st) {
   const long long n16 = (long long)(bytes / 16);
   if (n16 == 0) return cudaSuccess;
-  k_fill_zero<<<grid_for(n16, 256 * 4, 148 * 4), 256, 0, st>>>(reinterpret_cast<uint4*>(p), n16);
+  launch_pdl(k_fill_zero, grid_for(n16, 256 * 4, 148 * 4), 256, 0, st, reinterpret_cast<uint4*>(p), n16);
   return cudaGetLastError();
 }
 

@@ -191,9 +191,13 @@ __device__ __forceinline__ void gemm_body(const typename P::Params& p) {
     tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_holder)), kTmemCols);
     tmem_relinquish();
   }
+  // Launched with programmatic stream serialisation: the next kernel's CTAs may start (and do their own set-up)
+  // while this one's last tiles run; nothing of global memory is touched before the previous kernel has finished.
+  pdl_launch_dependents();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  pdl_wait();
   const uint32_t tmem_base = *tmem_holder;
   const int ntiles = P::num_tiles(p);
 

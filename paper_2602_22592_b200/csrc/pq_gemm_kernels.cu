@@ -107,8 +107,13 @@ static int launch_gemm(int kernel_id, void (*kernel)(Params), const Params& p, i
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes) != cudaSuccess) return PQ_ERR_CUDA;
   const int grid = grid_for_tiles(max_tiles);
   LaunchScope ls(kernel_id, st);
-  kernel<<<grid, kGemmThreads, kGemmSmemBytes, st>>>(p);
-  return cudaGetLastError() == cudaSuccess ? PQ_OK : PQ_ERR_CUDA;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(grid, 1, 1); cfg.blockDim = dim3(kGemmThreads, 1, 1); cfg.dynamicSmemBytes = kGemmSmemBytes;
+  cfg.stream = st; cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, p) == cudaSuccess ? PQ_OK : PQ_ERR_CUDA;
 }
 
 __device__ __forceinline__ int round_up(int x, int m) { return (x + m - 1) / m * m; }

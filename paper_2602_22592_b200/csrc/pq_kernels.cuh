@@ -64,6 +64,21 @@ struct FwdScratch {
   int* block_base;
 };
 
+// Launch with programmatic stream serialisation: the kernel may be scheduled while its predecessor in the stream is
+// still draining, which hides its launch latency and set-up.  Every kernel launched this way starts with
+// griddepcontrol.launch_dependents and griddepcontrol.wait, i.e. touches no global memory before the predecessor
+// has completed; the result of the launch is picked up by the caller's cudaGetLastError().
+template <class... KArgs, class... Args>
+inline void launch_pdl(void (*kernel)(KArgs...), int grid, int block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)grid, 1, 1); cfg.blockDim = dim3((unsigned)block, 1, 1); cfg.dynamicSmemBytes = smem;
+  cfg.stream = st; cfg.attrs = attr; cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // elementwise launchers (pq_elementwise.cu)
 cudaError_t launch_pack(const float* W, int N, int K, uint32_t* bits, int8_t* s8, float* scales, double* partial, cudaStream_t st);
 cudaError_t launch_route_and_quant(const uint16_t* X, const uint16_t* Wr, int T, int K, int E, const SavedPtrs& sv, const FwdScratch& sc,
