@@ -200,6 +200,40 @@ def run_ours(args):
     t_min = roofline_time_s(layers, peaks)
     layer_frac = t_min / (ms_per_step * 1e-3)
 
+    # The same step with each projection's pack + forward + backward on a stream of its own (the three linears are
+    # independent): tails of one projection's kernels and its memory-bound kernels overlap the others' GEMMs.
+    # Reported beside the headline, which stays the single-stream figure the roofline numbers belong to.
+    n_conc = max(3, min(args.steps, 50))
+    side = [torch.cuda.Stream(device=device) for _ in layers]
+    main_stream = torch.cuda.current_stream(device)
+
+    def step_concurrent():
+        fork = torch.cuda.Event()
+        fork.record(main_stream)
+        for L, st in zip(layers, side):
+            st.wait_event(fork)
+            with torch.cuda.stream(st):
+                L.pack()
+                L.forward()
+                L.backward()
+            done = torch.cuda.Event()
+            done.record(st)
+            main_stream.wait_event(done)
+
+    for _ in range(2):
+        step_concurrent()
+    barrier()
+    c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    c0.record()
+    for _ in range(n_conc):
+        step_concurrent()
+    c1.record()
+    barrier()
+    conc_ms = reps.max_over_ranks(c0.elapsed_time(c1), device) / n_conc
+    concurrent = {"streams": len(side), "steps": n_conc, "ms_per_step": round(conc_ms, 4),
+                  "value": round(reps.whole_job_rate(tokens, conc_ms), 1), "unit": "tokens/s",
+                  "note": "each projection on its own stream; not the headline"}
+
     # per-kernel breakdown: mean over a few extra (untimed) steps
     names = ["pack_sums", "binarize_pack", "router", "route_scan", "act_quant", "hp_up", "fwd", "scatter_rows", "scaled_sign",
              "hp_dh", "bwd_dx", "bwd_dw", "hp_db", "reduce_db", "hp_da", "reduce_da", "router_wgrad", "sum_partials", "sum_scalar"]
@@ -296,7 +330,7 @@ def run_ours(args):
             "roofline": roofline,
             "layer_roofline": {"t_min_ms": round(t_min * 1e3, 4), "frac": round(layer_frac, 4),
                                "formula": "2TNK/P_i8 + (4TNK + 6Tr(K+N))/P_bf16, P_i8 = 2 P_bf16, sustained bf16 peak"},
-            "breakdown_us_per_step": breakdown,
+            "breakdown_us_per_step": breakdown, "concurrent_streams": concurrent,
             "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": int(launches),
             "clocks": clk.summary(),
         }
