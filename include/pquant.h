@@ -242,8 +242,13 @@ int pq_device_status(void* stream, int* code, int* where);
 /* Process-wide launch options.
  *   PQ_OPT_DECODE_PDL (default 1): launch the decode kernels with programmatic stream
  *   serialisation, so that a kernel's prologue (barrier set-up, the copy of the sign bits)
- *   overlaps the tail of the kernel before it in the stream.  0 = plain stream order. */
-enum { PQ_OPT_DECODE_PDL = 1 };
+ *   overlaps the tail of the kernel before it in the stream.  0 = plain stream order.
+ *   PQ_OPT_SIDE_STREAM (default 1): pq_linear_forward and pq_linear_backward of a layer with
+ *   an HP branch run kernels that do not depend on one another side by side, on a helper
+ *   stream the library keeps per caller stream (created on first use); the helper's work is
+ *   joined back inside the same call, so the caller's stream order is unchanged and a stream
+ *   capture records one graph with a fork and a join.  0 = every kernel on the caller's stream. */
+enum { PQ_OPT_DECODE_PDL = 1, PQ_OPT_SIDE_STREAM = 2 };
 int pq_set_option(int option, int value);
 
 /* Cumulative number of kernels this library has launched in this process. */

@@ -247,6 +247,7 @@ def pq_device_status(stream=None) -> tuple[int, int]:
 
 
 PQ_OPT_DECODE_PDL = 1
+PQ_OPT_SIDE_STREAM = 2
 
 
 def pq_set_option(option: int, value: int):

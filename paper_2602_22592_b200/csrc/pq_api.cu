@@ -2,7 +2,10 @@
 // workspace buffers, launch sequencing.  No device allocation, no device
 // synchronisation (except pq_device_status, which says so).
 #include <cstring>
+#include <map>
+#include <mutex>
 #include <new>
+#include <utility>
 
 #include "pq_kernels.cuh"
 
@@ -113,6 +116,54 @@ static size_t carve_bwd_scratch(const pq_desc* d, void* base, BwdScratch* out) {
 }
 
 static inline bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) != 0; }
+
+// ---------------------------------------------------------------------------
+// Helper stream: kernels of one call that do not depend on one another (the
+// activation quantisation and the HP up-projection of a dense layer; the scaled
+// sign matrix and the HP gradient GEMM) run side by side.  Every caller stream
+// gets one non-blocking helper stream and two events, created on first use and
+// kept; work forked to the helper is always joined back before the call's last
+// kernel, so the caller sees plain stream order.  Event record and wait are
+// legal under stream capture and become edges of the captured graph.
+// ---------------------------------------------------------------------------
+static int g_side_streams = 1;
+
+struct SideCtx {
+  cudaStream_t side = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr;
+};
+
+static SideCtx* side_for(cudaStream_t st) {
+  if (!g_side_streams) return nullptr;
+  static std::mutex mu;
+  static std::map<std::pair<int, cudaStream_t>, SideCtx> ctxs;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return nullptr;
+  std::lock_guard<std::mutex> lock(mu);
+  SideCtx& c = ctxs[std::make_pair(dev, st)];
+  if (!c.side) {
+    // nothing is created while the caller's stream is being captured: such a call keeps plain stream order
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) {
+      cudaGetLastError();
+      return nullptr;
+    }
+    SideCtx n;
+    if (cudaStreamCreateWithFlags(&n.side, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&n.fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&n.join, cudaEventDisableTiming) != cudaSuccess) {
+      cudaGetLastError();
+      return nullptr;   // the caller falls back to plain stream order
+    }
+    c = n;
+  }
+  return &c;
+}
+
+// helper stream ordered after everything already in st
+static bool side_fork(SideCtx* c, cudaStream_t st) {
+  return cudaEventRecord(c->fork, st) == cudaSuccess && cudaStreamWaitEvent(c->side, c->fork, 0) == cudaSuccess;
+}
 
 // ---------------------------------------------------------------------------
 // Allocation-free weight pack: the fp64 partial sums live in a fixed device array
@@ -321,9 +372,13 @@ int pq_linear_forward(const pq_desc* d, const uint16_t* X, const uint32_t* w_bit
   if (ws_bytes < used) return PQ_ERR_WORKSPACE;
   const int E = experts_of(d);
   LayerArgs a{d->T, d->K, d->N, d->r, E, (d->flags & PQ_SCALE_VECTOR) ? 1 : 0, w_scales, alpha, beta, A, B, Wr};
-  if (launch_route_and_quant(X, Wr, d->T, d->K, routed(d) ? E : 1, sv, sc, st) != cudaSuccess) return PQ_ERR_CUDA;
+  // dense layer with an HP branch: the quantisation runs on the helper stream next to scan -> up-projection
+  SideCtx* side = (d->r > 0 && !routed(d)) ? side_for(st) : nullptr;
+  if (side && !side_fork(side, st)) return PQ_ERR_CUDA;
+  if (launch_route_and_quant(X, Wr, d->T, d->K, routed(d) ? E : 1, sv, sc, st, side ? side->side : st) != cudaSuccess) return PQ_ERR_CUDA;
+  if (side && cudaEventRecord(side->join, side->side) != cudaSuccess) return PQ_ERR_CUDA;
   const uint16_t* xs = routed(d) ? sv.xs : X;
-  return gemm_forward(a, w_s8, sv, xs, Y, st);
+  return gemm_forward(a, w_s8, sv, xs, Y, st, side ? side->join : nullptr);
 }
 
 int pq_decode_batch(const pq_decode_item* items, int n, void* stream) {
@@ -373,6 +428,13 @@ int pq_linear_backward(const pq_desc* d, const uint16_t* dY, const uint16_t* X, 
   const int vec = (d->flags & PQ_SCALE_VECTOR) ? 1 : 0;
   LayerArgs a{d->T, d->K, d->N, d->r, E, vec, w_scales, alpha, beta, A, B, Wr};
 
+  // with an HP branch the scaled sign matrix is made on the helper stream while the HP gradient GEMM runs
+  SideCtx* side = hp ? side_for(st) : nullptr;
+  if (side) {
+    if (!side_fork(side, st)) return PQ_ERR_CUDA;
+    if (launch_scaled_sign(w_s8, sc.sb, beta, vec, d->N, d->K, side->side) != cudaSuccess) return PQ_ERR_CUDA;
+    if (cudaEventRecord(side->join, side->side) != cudaSuccess) return PQ_ERR_CUDA;
+  }
   BwdBuffers b{};
   if (routed(d)) {
     if (launch_scatter_rows(dY, sc.dys, sv.pos, d->T, d->N, st) != cudaSuccess) return PQ_ERR_CUDA;
@@ -382,7 +444,7 @@ int pq_linear_backward(const pq_desc* d, const uint16_t* dY, const uint16_t* X, 
     b.dys = dY;
     b.xs = X;
   }
-  if (launch_scaled_sign(w_s8, sc.sb, beta, vec, d->N, d->K, st) != cudaSuccess) return PQ_ERR_CUDA;
+  if (!side && launch_scaled_sign(w_s8, sc.sb, beta, vec, d->N, d->K, st) != cudaSuccess) return PQ_ERR_CUDA;
   b.sb = sc.sb;
   if (hp && vec) {
     if (launch_scaled_b(B, sc.ba, alpha, E, d->N, d->r, st) != cudaSuccess) return PQ_ERR_CUDA;
@@ -392,7 +454,7 @@ int pq_linear_backward(const pq_desc* d, const uint16_t* dY, const uint16_t* X, 
   }
   b.dhc = sc.dhc; b.gh = sc.gh; b.dl = sc.dl; b.dlc = sc.dlc;
   b.dbeta_partial = sc.dbeta_partial; b.dalpha_partial = sc.dalpha_partial;
-  rc = gemm_backward(a, w_s8, sv, b, dX, dW, dA, dB, dWr, st);
+  rc = gemm_backward(a, w_s8, sv, b, dX, dW, dA, dB, dWr, st, side ? side->join : nullptr);
   if (rc) return rc;
 
   // dbeta_n = lam * sum over the column tiles of the partial sign-weighted row sums, dalpha_n = sum over experts
@@ -421,6 +483,7 @@ int pq_debug_gemm_tile(int mode, int M, int N, int K, const void* A, const void*
 int pq_set_option(int option, int value) {
   switch (option) {
     case PQ_OPT_DECODE_PDL: decode_set_pdl(value); return PQ_OK;
+    case PQ_OPT_SIDE_STREAM: g_side_streams = value ? 1 : 0; return PQ_OK;
     default: return PQ_ERR_UNSUPPORTED;
   }
 }

@@ -555,7 +555,8 @@ cudaError_t launch_pack(const float* W, int N, int K, uint32_t* bits, int8_t* s8
 }
 
 cudaError_t launch_route_and_quant(const uint16_t* X, const uint16_t* Wr, int T, int K, int E, const SavedPtrs& sv, const FwdScratch& sc,
-                                   cudaStream_t st) {
+                                   cudaStream_t st, cudaStream_t st_quant) {
+  if (E > 1) st_quant = st;   // the sorted position of a token comes from the router and the scan
   const int nblocks = (T + kRouterTokensPerBlock - 1) / kRouterTokensPerBlock;
   if (E > 1) {
     LaunchScope ls(KID_ROUTER, st);
@@ -564,7 +565,7 @@ cudaError_t launch_route_and_quant(const uint16_t* X, const uint16_t* Wr, int T,
   }
   { LaunchScope ls(KID_ROUTE_SCAN, st);
   launch_pdl(k_route_scan, 1, 512, 0, st, T, E, nblocks, sc.block_counts, sc.block_base, sv.offsets, sv.rt); }
-  LaunchScope ls(KID_ACT_QUANT, st);
+  LaunchScope ls(KID_ACT_QUANT, st_quant);
   const int per_lane = (K / 8 + 31) / 32;   // 16-byte pieces of a row per lane if one warp took the whole row
   auto kern = k_act_quant<0, 1>;
   int wpr = 1;
@@ -573,7 +574,7 @@ cudaError_t launch_route_and_quant(const uint16_t* X, const uint16_t* Wr, int T,
   else if (per_lane <= 16) { kern = k_act_quant<8, 2>; wpr = 2; }
   else if (per_lane <= 32) { kern = k_act_quant<8, 4>; wpr = 4; }
   const int rows_per_block = 8 / wpr;
-  launch_pdl(kern, (T + rows_per_block - 1) / rows_per_block, 256, 0, st, reinterpret_cast<const uint4*>(X), T, K, E, sv.expert, sc.block_base, sv.offsets, sc.gate_tok,
+  launch_pdl(kern, (T + rows_per_block - 1) / rows_per_block, 256, 0, st_quant, reinterpret_cast<const uint4*>(X), T, K, E, sv.expert, sc.block_base, sv.offsets, sc.gate_tok,
                                     sc.probs_tok, reinterpret_cast<uint2*>(sv.q), reinterpret_cast<uint4*>(sv.xt),
                                     reinterpret_cast<uint4*>(sv.xs), sv.gamma, sv.gate, sv.probs, sv.perm, sv.pos);
   return cudaGetLastError();

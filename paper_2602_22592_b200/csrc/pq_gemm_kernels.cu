@@ -390,7 +390,8 @@ static int fill_forward_params(const LayerArgs& a, const int8_t* w_s8, const Sav
   return PQ_OK;
 }
 
-int gemm_forward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, const uint16_t* xs, uint16_t* Y, cudaStream_t st) {
+int gemm_forward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, const uint16_t* xs, uint16_t* Y, cudaStream_t st,
+                 cudaEvent_t before_main) {
   if (a.r > 0) {
     HpUpProblem::Params p;
     p.rt = sv.rt; p.H = sv.h; p.K = a.K; p.r = a.r; p.bn = h_round_up(a.r, 16); p.item_rows = sv.max_items * 128;
@@ -401,11 +402,13 @@ int gemm_forward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, co
     FwdProblem<true>::Params f;
     rc = fill_forward_params<true>(a, w_s8, sv, Y, f);
     if (rc) return rc;
+    if (before_main && cudaStreamWaitEvent(st, before_main, 0) != cudaSuccess) return PQ_ERR_CUDA;
     return launch_gemm(KID_FWD, k_gemm_fwd_hp, f, f.g.total, st);
   }
   FwdProblem<false>::Params f;
   int rc = fill_forward_params<false>(a, w_s8, sv, Y, f);
   if (rc) return rc;
+  if (before_main && cudaStreamWaitEvent(st, before_main, 0) != cudaSuccess) return PQ_ERR_CUDA;
   return launch_gemm(KID_FWD, k_gemm_fwd_1bit, f, f.g.total, st);
 }
 
@@ -811,7 +814,7 @@ struct BwdDwProblem {
 PQ_DEFINE_GEMM_KERNEL(k_gemm_bwd_dw, BwdDwProblem)
 
 int gemm_backward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, const BwdBuffers& b, uint16_t* dX, float* dW, float* dA,
-                  float* dB, float* dWr, cudaStream_t st) {
+                  float* dB, float* dWr, cudaStream_t st, cudaEvent_t before_dx) {
   const int mtiles = (a.T + 127) / 128;
   const int ntk = (a.K + 255) / 256, ntn128 = (a.N + 127) / 128;
   const bool hp = a.r > 0;
@@ -844,6 +847,7 @@ int gemm_backward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, c
     p.rt = sv.rt; p.perm = (hp && a.E > 1) ? sv.perm : nullptr; p.w_scales = a.w_scales; p.beta = a.beta; p.dX = dX;
     p.T = a.T; p.N = a.N; p.K = a.K; p.r = a.r; p.E = hp ? a.E : 1; p.sstride = a.scale_stride; p.item_rows = (int)item_rows;
     p.g = make_tile_grid(mtiles, ntk, 256);
+    if (before_dx && cudaStreamWaitEvent(st, before_dx, 0) != cudaSuccess) return PQ_ERR_CUDA;
     rc = launch_gemm(KID_BWD_DX, k_gemm_bwd_dx, p, p.g.total, st);
     if (rc) return rc;
   }

@@ -81,8 +81,9 @@ inline void launch_pdl(void (*kernel)(KArgs...), int grid, int block, size_t sme
 
 // elementwise launchers (pq_elementwise.cu)
 cudaError_t launch_pack(const float* W, int N, int K, uint32_t* bits, int8_t* s8, float* scales, double* partial, cudaStream_t st);
+// st_quant: the stream of the quantisation kernel; it may differ from st only when E == 1 (no routing to wait for)
 cudaError_t launch_route_and_quant(const uint16_t* X, const uint16_t* Wr, int T, int K, int E, const SavedPtrs& sv, const FwdScratch& sc,
-                                   cudaStream_t st);
+                                   cudaStream_t st, cudaStream_t st_quant);
 cudaError_t launch_scatter_rows(const uint16_t* src, uint16_t* dst, const int* pos, int T, int row_elems, cudaStream_t st);
 cudaError_t launch_scaled_sign(const int8_t* s8, uint16_t* out, const float* beta, int beta_stride, int N, int K, cudaStream_t st);
 cudaError_t launch_scaled_b(const uint16_t* B, uint16_t* out, const float* alpha, int E, int N, int r, cudaStream_t st);
@@ -103,7 +104,9 @@ struct LayerArgs {
 };
 
 int gemm_debug(int mode, int M, int N, int K, const void* A, const void* B, void* D, int tile_n, cudaStream_t st);
-int gemm_forward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, const uint16_t* xs, uint16_t* Y, cudaStream_t st);
+// before_main: an event the fused forward GEMM waits for (work on another stream that feeds it), or nullptr
+int gemm_forward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, const uint16_t* xs, uint16_t* Y, cudaStream_t st,
+                 cudaEvent_t before_main);
 
 // decode path (pq_decode.cu)
 size_t decode_workspace_bytes(int M, int K, int N, int r, bool dump);
@@ -130,7 +133,8 @@ struct BwdBuffers {
   float* dbeta_partial;  // [2 * ceil(K/256), N]
   float* dalpha_partial; // [2 * E, N]
 };
+// before_dx: an event the input-gradient GEMM waits for (the scaled sign matrix made on another stream), or nullptr
 int gemm_backward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, const BwdBuffers& b, uint16_t* dX, float* dW, float* dA,
-                  float* dB, float* dWr, cudaStream_t st);
+                  float* dB, float* dWr, cudaStream_t st, cudaEvent_t before_dx);
 
 }  // namespace pq

@@ -83,3 +83,53 @@ def test_backward_is_deterministic():
     torch.cuda.synchronize()
     for a, b in zip(keep, (L.dX, L.dW, L.dA, L.dB, L.dWr, L.dalpha, L.dbeta)):
         assert torch.equal(a, b)
+
+
+def _all_outputs(L):
+    names = ("Y", "dX", "dW", "dA", "dB", "dWr", "dalpha", "dbeta")
+    return [getattr(L, n).clone() for n in names if getattr(L, n, None) is not None]
+
+
+@pytest.mark.parametrize("E", [1, 4])
+def test_helper_stream_changes_no_bit(E):
+    # the helper stream only reorders independent kernels: results are bit-identical with it on or off
+    c = I.make_linear_case(777, 512, 640, 64, E, seed=21)
+    L = run_fwd_bwd(c, False)
+    on = _all_outputs(L)
+    pqb.pq_set_option(pqb.PQ_OPT_SIDE_STREAM, 0)
+    try:
+        L.forward()
+        L.backward()
+        torch.cuda.synchronize()
+        off = _all_outputs(L)
+    finally:
+        pqb.pq_set_option(pqb.PQ_OPT_SIDE_STREAM, 1)
+    check_status()
+    for a, b in zip(on, off):
+        assert torch.equal(a, b)
+
+
+def test_helper_stream_under_graph_capture():
+    # a captured forward + backward holds the fork to the helper stream and the join as graph edges;
+    # replays match the eager call bit for bit
+    c = I.make_linear_case(640, 512, 512, 32, 1, seed=22)
+    L = run_fwd_bwd(c, False)      # eager run: creates the helper stream outside the capture
+    want = _all_outputs(L)
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(s):
+        L.forward()
+        L.backward()
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g, stream=s):
+            L.forward()
+            L.backward()
+    for t in (L.Y, L.dX, L.dW, L.dA, L.dB, L.dalpha, L.dbeta):
+        t.zero_()
+    for _ in range(3):
+        g.replay()
+    torch.cuda.synchronize()
+    check_status()
+    for a, b in zip(want, _all_outputs(L)):
+        assert torch.equal(a, b)
