@@ -33,7 +33,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel (the 2048 -> 5632
 # projection) from the committed ncu capture (profiles/gemm_kernels_up_projection_ncu.md); set to None
 # whenever the kernel changes until it is captured again.
-NCU_TRAFFIC_BYTES = {"bwd_dw": 359427328}
+NCU_TRAFFIC_BYTES = {"bwd_dw": None}
 
 
 def measured_peaks():
@@ -189,11 +189,14 @@ def run_ours(args):
     value = reps.whole_job_rate(tokens, ms_per_step)
 
     dw_ms = float(np.mean([a.elapsed_time(b) for row in ev for a, b in row]))
-    # algorithmic flops of the launch: dW = dY^T . (q/gamma) and, in the same launch, dB_e = dY^T . (g H)
-    dw_flops = float(np.mean([2.0 * L.T * L.N * L.K + 2.0 * L.T * L.N * L.r for L in layers]))
+    # algorithmic flops of the launch: dW = dY^T . (q/gamma).  (The HP tiles dB, dA and the router gradient are a
+    # launch of their own, profile id hp_db, and are not counted here.)  The launch shares the GPU with the chain
+    # scaled sign -> HP gradient GEMM -> dX on the library's helper stream, so its event time includes SMs it
+    # had to wait for.
+    dw_flops = float(np.mean([2.0 * L.T * L.N * L.K for L in layers]))
     achieved = dw_flops / (dw_ms * 1e-3) / 1e12
     peak = peaks["bf16_tflops_sustained"]
-    roofline = {"kernel": "k_gemm_bwd_dw (dW = dY^T . q/gamma and dB = dY^T . gH, bf16 tcgen05, fp32 accumulate)", "bound": "tensor",
+    roofline = {"kernel": "k_gemm_bwd_dw (dW = dY^T . q/gamma, bf16 tcgen05, fp32 accumulate)", "bound": "tensor",
                 "achieved": round(achieved, 1), "peak": peak, "unit": "TFLOP/s", "frac": round(achieved / peak, 4),
                 "peak_source": f"{peak_kind} bf16_tflops_sustained", "avg_launch_ms": round(dw_ms, 4),
                 "traffic": NCU_TRAFFIC_BYTES["bwd_dw"]}
@@ -234,7 +237,9 @@ def run_ours(args):
                   "value": round(reps.whole_job_rate(tokens, conc_ms), 1), "unit": "tokens/s",
                   "note": "each projection on its own stream; not the headline"}
 
-    # per-kernel breakdown: mean over a few extra (untimed) steps
+    # per-kernel breakdown: mean over a few extra (untimed) steps, every kernel on one stream (helper stream off) so
+    # that each pair of events brackets one kernel running alone; the weight gradient is then a single launch again
+    pqb.pq_set_option(pqb.PQ_OPT_SIDE_STREAM, 0)
     names = ["pack_sums", "binarize_pack", "router", "route_scan", "act_quant", "hp_up", "fwd", "scatter_rows", "scaled_sign",
              "hp_dh", "bwd_dx", "bwd_dw", "hp_db", "reduce_db", "hp_da", "reduce_da", "router_wgrad", "sum_partials", "sum_scalar"]
     bev = {n: (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for n in names}
@@ -252,6 +257,7 @@ def run_ours(args):
                 breakdown[n] += a.elapsed_time(b) * 1e3 / bsteps
     for n in names:
         pqb.pq_profile_events(pqb.KERNEL_IDS[n], None, None)
+    pqb.pq_set_option(pqb.PQ_OPT_SIDE_STREAM, 1)
     # an id that was not launched shows only the few microseconds between its two back-to-back records
     breakdown = {n: round(v, 1) for n, v in breakdown.items() if v > 8.0 * len(layers)}
 

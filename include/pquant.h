@@ -243,11 +243,14 @@ int pq_device_status(void* stream, int* code, int* where);
  *   PQ_OPT_DECODE_PDL (default 1): launch the decode kernels with programmatic stream
  *   serialisation, so that a kernel's prologue (barrier set-up, the copy of the sign bits)
  *   overlaps the tail of the kernel before it in the stream.  0 = plain stream order.
- *   PQ_OPT_SIDE_STREAM (default 1): pq_linear_forward and pq_linear_backward of a layer with
- *   an HP branch run kernels that do not depend on one another side by side, on a helper
- *   stream the library keeps per caller stream (created on first use); the helper's work is
- *   joined back inside the same call, so the caller's stream order is unchanged and a stream
- *   capture records one graph with a fork and a join.  0 = every kernel on the caller's stream. */
+ *   PQ_OPT_SIDE_STREAM (default 1): pq_linear_forward (dense layer with an HP branch) and
+ *   pq_linear_backward run kernels that do not depend on one another side by side, on a helper
+ *   stream the library keeps per caller stream (created on first use, never during a stream
+ *   capture); the helper's work is joined back inside the same call, so the caller's stream
+ *   order is unchanged and a stream capture records one graph with a fork and a join.  In the
+ *   backward pass the weight-gradient tiles that need only dY and q/gamma are one launch
+ *   (profile id bwd_dw) and the HP tiles (dB, dA, router) a second one (id hp_db).
+ *   0 = every kernel on the caller's stream, the weight gradient as one launch. */
 enum { PQ_OPT_DECODE_PDL = 1, PQ_OPT_SIDE_STREAM = 2 };
 int pq_set_option(int option, int value);
 

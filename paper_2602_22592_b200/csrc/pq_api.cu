@@ -118,19 +118,20 @@ static size_t carve_bwd_scratch(const pq_desc* d, void* base, BwdScratch* out) {
 static inline bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) != 0; }
 
 // ---------------------------------------------------------------------------
-// Helper stream: kernels of one call that do not depend on one another (the
-// activation quantisation and the HP up-projection of a dense layer; the scaled
-// sign matrix and the HP gradient GEMM) run side by side.  Every caller stream
-// gets one non-blocking helper stream and two events, created on first use and
-// kept; work forked to the helper is always joined back before the call's last
-// kernel, so the caller sees plain stream order.  Event record and wait are
-// legal under stream capture and become edges of the captured graph.
+// Helper stream: kernels of one call that do not depend on one another run side
+// by side (forward of a dense layer with an HP branch: the activation quantisation
+// next to the HP up-projection; backward: the weight-gradient GEMM next to the chain
+// scaled sign matrix -> HP gradient GEMM -> dX, each filling the other's last wave).
+// Every caller stream gets one non-blocking helper stream and three events, created
+// on first use and kept; work forked to the helper is always joined back before the
+// call's last kernel, so the caller sees plain stream order.  Event record and wait
+// are legal under stream capture and become edges of the captured graph.
 // ---------------------------------------------------------------------------
 static int g_side_streams = 1;
 
 struct SideCtx {
   cudaStream_t side = nullptr;
-  cudaEvent_t fork = nullptr, join = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr, mid = nullptr;
 };
 
 static SideCtx* side_for(cudaStream_t st) {
@@ -151,7 +152,8 @@ static SideCtx* side_for(cudaStream_t st) {
     SideCtx n;
     if (cudaStreamCreateWithFlags(&n.side, cudaStreamNonBlocking) != cudaSuccess ||
         cudaEventCreateWithFlags(&n.fork, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&n.join, cudaEventDisableTiming) != cudaSuccess) {
+        cudaEventCreateWithFlags(&n.join, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&n.mid, cudaEventDisableTiming) != cudaSuccess) {
       cudaGetLastError();
       return nullptr;   // the caller falls back to plain stream order
     }
@@ -428,13 +430,6 @@ int pq_linear_backward(const pq_desc* d, const uint16_t* dY, const uint16_t* X, 
   const int vec = (d->flags & PQ_SCALE_VECTOR) ? 1 : 0;
   LayerArgs a{d->T, d->K, d->N, d->r, E, vec, w_scales, alpha, beta, A, B, Wr};
 
-  // with an HP branch the scaled sign matrix is made on the helper stream while the HP gradient GEMM runs
-  SideCtx* side = hp ? side_for(st) : nullptr;
-  if (side) {
-    if (!side_fork(side, st)) return PQ_ERR_CUDA;
-    if (launch_scaled_sign(w_s8, sc.sb, beta, vec, d->N, d->K, side->side) != cudaSuccess) return PQ_ERR_CUDA;
-    if (cudaEventRecord(side->join, side->side) != cudaSuccess) return PQ_ERR_CUDA;
-  }
   BwdBuffers b{};
   if (routed(d)) {
     if (launch_scatter_rows(dY, sc.dys, sv.pos, d->T, d->N, st) != cudaSuccess) return PQ_ERR_CUDA;
@@ -444,17 +439,24 @@ int pq_linear_backward(const pq_desc* d, const uint16_t* dY, const uint16_t* X, 
     b.dys = dY;
     b.xs = X;
   }
-  if (!side && launch_scaled_sign(w_s8, sc.sb, beta, vec, d->N, d->K, st) != cudaSuccess) return PQ_ERR_CUDA;
+  // With the helper stream: what leads to dX (scaled sign matrix, scaled B, HP gradient GEMM, dX) runs there, the
+  // weight gradient on the caller's stream beside it; see BwdStreams.
+  SideCtx* side = side_for(st);
+  if (side && !side_fork(side, st)) return PQ_ERR_CUDA;
+  cudaStream_t sx = side ? side->side : st;
+  if (launch_scaled_sign(w_s8, sc.sb, beta, vec, d->N, d->K, sx) != cudaSuccess) return PQ_ERR_CUDA;
   b.sb = sc.sb;
   if (hp && vec) {
-    if (launch_scaled_b(B, sc.ba, alpha, E, d->N, d->r, st) != cudaSuccess) return PQ_ERR_CUDA;
+    if (launch_scaled_b(B, sc.ba, alpha, E, d->N, d->r, sx) != cudaSuccess) return PQ_ERR_CUDA;
     b.ba = sc.ba;
   } else {
     b.ba = B;
   }
   b.dhc = sc.dhc; b.gh = sc.gh; b.dl = sc.dl; b.dlc = sc.dlc;
   b.dbeta_partial = sc.dbeta_partial; b.dalpha_partial = sc.dalpha_partial;
-  rc = gemm_backward(a, w_s8, sv, b, dX, dW, dA, dB, dWr, st, side ? side->join : nullptr);
+  BwdStreams bs;
+  if (side) { bs.side = side->side; bs.dh_done = side->mid; bs.side_done = side->join; }
+  rc = gemm_backward(a, w_s8, sv, b, dX, dW, dA, dB, dWr, st, bs);
   if (rc) return rc;
 
   // dbeta_n = lam * sum over the column tiles of the partial sign-weighted row sums, dalpha_n = sum over experts

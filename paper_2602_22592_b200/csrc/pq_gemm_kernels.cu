@@ -814,13 +814,46 @@ struct BwdDwProblem {
 PQ_DEFINE_GEMM_KERNEL(k_gemm_bwd_dw, BwdDwProblem)
 
 int gemm_backward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, const BwdBuffers& b, uint16_t* dX, float* dW, float* dA,
-                  float* dB, float* dWr, cudaStream_t st, cudaEvent_t before_dx) {
+                  float* dB, float* dWr, cudaStream_t st, const BwdStreams& bs) {
   const int mtiles = (a.T + 127) / 128;
   const int ntk = (a.K + 255) / 256, ntn128 = (a.N + 127) / 128;
   const bool hp = a.r > 0;
   const int r64 = h_round_up(a.r, 64);
   const uint64_t item_rows = (uint64_t)sv.max_items * 128;  // rows of one plane; buffers hold two
+  cudaStream_t sx = bs.side ? bs.side : st;                 // stream of the HP gradient GEMM and dX
   int rc;
+
+  BwdDwProblem::Params w;
+  {
+    if (!map_mn(&w.tdyT, &w.dy_blk, b.dys, a.N, a.T, 2, 1, 2)) return PQ_ERR_CUDA;
+    if (!map_mn(&w.txt, &w.xt_blk, sv.xt, a.K, a.T, 2, 1, 4)) return PQ_ERR_CUDA;
+    w.tgh = w.txt; w.gh_blk = 0;
+    if (hp && !map_mn(&w.tgh, &w.gh_blk, b.gh, a.r, 2 * item_rows, 2, 1, r64 / 64)) return PQ_ERR_CUDA;
+    w.rt = sv.rt; w.s8 = w_s8; w.beta = a.beta; w.alpha = a.alpha; w.B = a.B; w.dW = dW; w.dB = dB;
+    w.dbeta_partial = b.dbeta_partial; w.dalpha_partial = b.dalpha_partial;
+    w.T = a.T; w.N = a.N; w.K = a.K; w.r = a.r; w.r64 = r64; w.E = a.E; w.sstride = a.scale_stride; w.item_rows = (int)item_rows;
+    w.ntn = ntn128; w.ntk = ntk; w.db_tiles = hp ? a.E * ntn128 : 0; w.da_tiles = hp ? a.E * ntk : 0;
+    w.tdlT = w.txt; w.txs = w.txt; w.tdhT = w.txt; w.xs_blk = 0; w.dh_blk = 0; w.wr_tiles = 0;
+    w.w_scales = a.w_scales; w.dWr = dWr; w.dA = dA;
+    if (hp) {
+      if (!map_mn(&w.txs, &w.xs_blk, b.xs, a.K, a.T, 2, 1, 4)) return PQ_ERR_CUDA;
+      if (!map_mn(&w.tdhT, &w.dh_blk, b.dhc, a.r, 2 * item_rows, 2, 1, 2)) return PQ_ERR_CUDA;
+    }
+    if (hp && a.E > 1) {
+      int unused = 0;
+      if (!map_mn(&w.tdlT, &unused, b.dlc, 16, a.T, 2, 1, 2)) return PQ_ERR_CUDA;
+      w.wr_tiles = ntk;
+    }
+    w.g = make_tile_grid(ntn128, ntk, 256);
+  }
+  if (bs.side) {
+    // the dW tiles proper need dY and q / gamma only: they start at once and take every SM; what follows on the
+    // other stream moves into their last wave
+    BwdDwProblem::Params m = w;
+    m.wr_tiles = 0; m.da_tiles = 0; m.db_tiles = 0;
+    rc = launch_gemm(KID_BWD_DW, k_gemm_bwd_dw, m, m.g.total, st);
+    if (rc) return rc;
+  }
   if (hp) {
     HpDhProblem::Params p;
     if (!map2d(&p.tdy, false, b.dys, a.N, a.T, 64, 128)) return PQ_ERR_CUDA;
@@ -828,8 +861,9 @@ int gemm_backward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, c
     p.rt = sv.rt; p.H = sv.h; p.gate = sv.gate; p.probs = sv.probs; p.w_scales = a.w_scales; p.alpha = a.alpha; p.beta = a.beta;
     p.dhc = b.dhc; p.gh = b.gh; p.dl = b.dl; p.dlc = b.dlc;
     p.T = a.T; p.N = a.N; p.r = a.r; p.E = a.E; p.bn = r64; p.sstride = a.scale_stride; p.item_rows = (int)item_rows;
-    rc = launch_gemm(KID_HP_DH, k_gemm_hp_dh, p, sv.max_items, st);
+    rc = launch_gemm(KID_HP_DH, k_gemm_hp_dh, p, sv.max_items, sx);
     if (rc) return rc;
+    if (bs.side && cudaEventRecord(bs.dh_done, sx) != cudaSuccess) return PQ_ERR_CUDA;
   }
   {
     BwdDxProblem::Params p;
@@ -847,34 +881,23 @@ int gemm_backward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, c
     p.rt = sv.rt; p.perm = (hp && a.E > 1) ? sv.perm : nullptr; p.w_scales = a.w_scales; p.beta = a.beta; p.dX = dX;
     p.T = a.T; p.N = a.N; p.K = a.K; p.r = a.r; p.E = hp ? a.E : 1; p.sstride = a.scale_stride; p.item_rows = (int)item_rows;
     p.g = make_tile_grid(mtiles, ntk, 256);
-    if (before_dx && cudaStreamWaitEvent(st, before_dx, 0) != cudaSuccess) return PQ_ERR_CUDA;
-    rc = launch_gemm(KID_BWD_DX, k_gemm_bwd_dx, p, p.g.total, st);
+    rc = launch_gemm(KID_BWD_DX, k_gemm_bwd_dx, p, p.g.total, sx);
     if (rc) return rc;
+    if (bs.side && cudaEventRecord(bs.side_done, sx) != cudaSuccess) return PQ_ERR_CUDA;
   }
-  {
-    BwdDwProblem::Params p;
-    if (!map_mn(&p.tdyT, &p.dy_blk, b.dys, a.N, a.T, 2, 1, 2)) return PQ_ERR_CUDA;
-    if (!map_mn(&p.txt, &p.xt_blk, sv.xt, a.K, a.T, 2, 1, 4)) return PQ_ERR_CUDA;
-    p.tgh = p.txt; p.gh_blk = 0;
-    if (hp && !map_mn(&p.tgh, &p.gh_blk, b.gh, a.r, 2 * item_rows, 2, 1, r64 / 64)) return PQ_ERR_CUDA;
-    p.rt = sv.rt; p.s8 = w_s8; p.beta = a.beta; p.alpha = a.alpha; p.B = a.B; p.dW = dW; p.dB = dB;
-    p.dbeta_partial = b.dbeta_partial; p.dalpha_partial = b.dalpha_partial;
-    p.T = a.T; p.N = a.N; p.K = a.K; p.r = a.r; p.r64 = r64; p.E = a.E; p.sstride = a.scale_stride; p.item_rows = (int)item_rows;
-    p.ntn = ntn128; p.ntk = ntk; p.db_tiles = hp ? a.E * ntn128 : 0; p.da_tiles = hp ? a.E * ntk : 0;
-    p.tdlT = p.txt; p.txs = p.txt; p.tdhT = p.txt; p.xs_blk = 0; p.dh_blk = 0; p.wr_tiles = 0;
-    p.w_scales = a.w_scales; p.dWr = dWr; p.dA = dA;
-    if (hp) {
-      if (!map_mn(&p.txs, &p.xs_blk, b.xs, a.K, a.T, 2, 1, 4)) return PQ_ERR_CUDA;
-      if (!map_mn(&p.tdhT, &p.dh_blk, b.dhc, a.r, 2 * item_rows, 2, 1, 2)) return PQ_ERR_CUDA;
-    }
-    if (hp && a.E > 1) {
-      int unused = 0;
-      if (!map_mn(&p.tdlT, &unused, b.dlc, 16, a.T, 2, 1, 2)) return PQ_ERR_CUDA;
-      p.wr_tiles = ntk;
-    }
-    p.g = make_tile_grid(ntn128, ntk, 256);
-    rc = launch_gemm(KID_BWD_DW, k_gemm_bwd_dw, p, p.wr_tiles + p.da_tiles + p.g.total + p.db_tiles, st);
+  if (!bs.side) {
+    rc = launch_gemm(KID_BWD_DW, k_gemm_bwd_dw, w, w.wr_tiles + w.da_tiles + w.g.total + w.db_tiles, st);
     if (rc) return rc;
+  } else {
+    if (hp) {
+      // dB, dA and the router gradient read what the HP gradient GEMM wrote
+      BwdDwProblem::Params x = w;
+      x.g.total = 0;
+      if (cudaStreamWaitEvent(st, bs.dh_done, 0) != cudaSuccess) return PQ_ERR_CUDA;
+      rc = launch_gemm(KID_HP_DB, k_gemm_bwd_dw, x, x.wr_tiles + x.da_tiles + x.db_tiles, st);
+      if (rc) return rc;
+    }
+    if (cudaStreamWaitEvent(st, bs.side_done, 0) != cudaSuccess) return PQ_ERR_CUDA;
   }
   return PQ_OK;
 }

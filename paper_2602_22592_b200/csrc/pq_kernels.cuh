@@ -133,8 +133,17 @@ struct BwdBuffers {
   float* dbeta_partial;  // [2 * ceil(K/256), N]
   float* dalpha_partial; // [2 * E, N]
 };
-// before_dx: an event the input-gradient GEMM waits for (the scaled sign matrix made on another stream), or nullptr
+// Where the backward GEMMs run.  side == nullptr: all on st, in the order HP gradient, dX, dW (one launch with the
+// HP tiles).  Otherwise the weight-gradient tiles that need nothing from the HP gradient GEMM are launched on st at
+// once, the HP gradient GEMM and dX follow one another on `side` (already ordered after the scaled sign matrix), and
+// the HP tiles of the weight gradient (dB, dA, router) go to st after `dh_done`; st then waits for `side_done`.
+// Kernels of the two streams fill one another's last waves.
+struct BwdStreams {
+  cudaStream_t side = nullptr;
+  cudaEvent_t dh_done = nullptr;     // recorded on side after the HP gradient GEMM
+  cudaEvent_t side_done = nullptr;   // recorded on side after dX
+};
 int gemm_backward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, const BwdBuffers& b, uint16_t* dX, float* dW, float* dA,
-                  float* dB, float* dWr, cudaStream_t st, cudaEvent_t before_dx);
+                  float* dB, float* dWr, cudaStream_t st, const BwdStreams& bs);
 
 }  // namespace pq
