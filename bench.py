@@ -33,7 +33,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel (the 2048 -> 5632
 # projection) from the committed ncu capture (profiles/gemm_kernels_up_projection_ncu.md); set to None
 # whenever the kernel changes until it is captured again.
-NCU_TRAFFIC_BYTES = {"bwd_dw": None}
+NCU_TRAFFIC_BYTES = {"bwd_dw": 218165248}
 
 
 def measured_peaks():
