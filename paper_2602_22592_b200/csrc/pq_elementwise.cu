@@ -125,16 +125,20 @@ __global__ void __launch_bounds__(256) k_binarize_pack(const float4* __restrict_
 }
 
 // ---------------------------------------------------------------------------
-// K4a: router (Sec. 3.3).  One warp per token.  Logits in fp32 with a fixed
+// K4a: router (Sec. 3.3).  One warp per token (or per two).  Logits in fp32 with a fixed
 // summation order -- lane j owns the 8-element chunks c with c mod 32 == j,
 // ascending k, fused multiply-add; lanes combined by the xor butterfly
 // 16, 8, 4, 2, 1 -- so that the top-1 index is reproducible bit for bit.
 // Softmax in fp32; ties go to the lowest index.  Also counts tokens per
 // expert for each block of kRouterTokensPerBlock consecutive tokens.
 // ---------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024) k_router(const uint4* __restrict__ X, const uint4* __restrict__ Wr, int T, int K, int E,
-                                                 int* __restrict__ expert, float* __restrict__ gate_tok,
-                                                 float* __restrict__ probs_tok, int* __restrict__ block_counts) {
+// EMAX: compile-time bound on E (the loops over experts are unrolled to it); TPW: tokens per warp -- the warp
+// walks the chunks once and applies each unpacked piece of Wr to TPW tokens.  Neither changes any token's
+// arithmetic: a lane's partial sum of (token, expert) is the same chain of fused multiply-adds.
+template <int EMAX, int TPW>
+__global__ void __launch_bounds__(32 * kRouterTokensPerBlock / TPW) k_router(const uint4* __restrict__ X, const uint4* __restrict__ Wr, int T, int K,
+                                                                             int E, int* __restrict__ expert, float* __restrict__ gate_tok,
+                                                                             float* __restrict__ probs_tok, int* __restrict__ block_counts) {
   pdl_launch_dependents();   // launched with programmatic stream serialisation: see launch_pdl
   pdl_wait();
   __shared__ int cnt[kMaxExperts];
@@ -142,68 +146,90 @@ __global__ void __launch_bounds__(1024) k_router(const uint4* __restrict__ X, co
   __syncthreads();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int chunks = K >> 3;
-  const int t = blockIdx.x * kRouterTokensPerBlock + warp;   // one warp per token
-  if (t < T) {
-    float acc[kMaxExperts];
+  const int t0 = blockIdx.x * kRouterTokensPerBlock + warp * TPW;   // this warp's first token
+  if (t0 < T) {
+    float acc[TPW][EMAX];
 #pragma unroll
-    for (int e = 0; e < kMaxExperts; ++e) acc[e] = 0.f;
-    const uint4* xrow = X + (long long)t * chunks;
-    auto fold = [&](const uint4& xv, int c) {
-      const float x0 = bf16lo(xv.x), x1 = bf16hi(xv.x), x2 = bf16lo(xv.y), x3 = bf16hi(xv.y);
-      const float x4 = bf16lo(xv.z), x5 = bf16hi(xv.z), x6 = bf16lo(xv.w), x7 = bf16hi(xv.w);
+    for (int u = 0; u < TPW; ++u)
 #pragma unroll
-      for (int e = 0; e < kMaxExperts; ++e) {
+      for (int e = 0; e < EMAX; ++e) acc[u][e] = 0.f;
+    const uint4* xrow[TPW];
+#pragma unroll
+    for (int u = 0; u < TPW; ++u) xrow[u] = X + (long long)min(t0 + u, T - 1) * chunks;   // a token past the end repeats the last one, unused
+    auto fold = [&](const uint4 (&xv)[TPW], int c) {
+      float x[TPW][8];
+#pragma unroll
+      for (int u = 0; u < TPW; ++u) {
+        x[u][0] = bf16lo(xv[u].x); x[u][1] = bf16hi(xv[u].x); x[u][2] = bf16lo(xv[u].y); x[u][3] = bf16hi(xv[u].y);
+        x[u][4] = bf16lo(xv[u].z); x[u][5] = bf16hi(xv[u].z); x[u][6] = bf16lo(xv[u].w); x[u][7] = bf16hi(xv[u].w);
+      }
+#pragma unroll
+      for (int e = 0; e < EMAX; ++e) {
         if (e < E) {
           const uint4 wv = __ldg(Wr + (long long)e * chunks + c);
-          float a = acc[e];
-          a = fmaf(x0, bf16lo(wv.x), a); a = fmaf(x1, bf16hi(wv.x), a);
-          a = fmaf(x2, bf16lo(wv.y), a); a = fmaf(x3, bf16hi(wv.y), a);
-          a = fmaf(x4, bf16lo(wv.z), a); a = fmaf(x5, bf16hi(wv.z), a);
-          a = fmaf(x6, bf16lo(wv.w), a); a = fmaf(x7, bf16hi(wv.w), a);
-          acc[e] = a;
+          const float w[8] = {bf16lo(wv.x), bf16hi(wv.x), bf16lo(wv.y), bf16hi(wv.y), bf16lo(wv.z), bf16hi(wv.z), bf16lo(wv.w), bf16hi(wv.w)};
+#pragma unroll
+          for (int u = 0; u < TPW; ++u) {
+            float a = acc[u][e];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) a = fmaf(x[u][i], w[i], a);
+            acc[u][e] = a;
+          }
         }
       }
     };
-    // the token's chunks in ascending order, two loads of X in flight (the 32 warps of the block hide the rest)
+    // the tokens' chunks in ascending order, two loads of each row in flight
     int c = lane;
     for (; c + 32 < chunks; c += 64) {
-      const uint4 xa = __ldg(xrow + c), xb = __ldg(xrow + c + 32);
+      uint4 xa[TPW], xb[TPW];
+#pragma unroll
+      for (int u = 0; u < TPW; ++u) { xa[u] = __ldg(xrow[u] + c); xb[u] = __ldg(xrow[u] + c + 32); }
       fold(xa, c);
       fold(xb, c + 32);
     }
-    if (c < chunks) fold(__ldg(xrow + c), c);
+    if (c < chunks) {
+      uint4 xa[TPW];
 #pragma unroll
-    for (int e = 0; e < kMaxExperts; ++e) {
-      if (e < E) {
-        float a = acc[e];
-        for (int d = 16; d > 0; d >>= 1) a = a + __shfl_xor_sync(0xffffffffu, a, d);
-        acc[e] = a;
+      for (int u = 0; u < TPW; ++u) xa[u] = __ldg(xrow[u] + c);
+      fold(xa, c);
+    }
+#pragma unroll
+    for (int u = 0; u < TPW; ++u) {
+      const int t = t0 + u;
+      if (t >= T) break;
+#pragma unroll
+      for (int e = 0; e < EMAX; ++e) {
+        if (e < E) {
+          float a = acc[u][e];
+          for (int d = 16; d > 0; d >>= 1) a = a + __shfl_xor_sync(0xffffffffu, a, d);
+          acc[u][e] = a;
+        }
       }
-    }
-    // every lane now holds all logits; lane 0 finishes the token
-    int best = 0;
-    float lmax = acc[0];
+      // every lane now holds all logits; lane 0 finishes the token
+      int best = 0;
+      float lmax = acc[u][0];
 #pragma unroll
-    for (int e = 1; e < kMaxExperts; ++e)
-      if (e < E && acc[e] > lmax) { lmax = acc[e]; best = e; }
-    float den = 0.f;
-    float pe[kMaxExperts];
+      for (int e = 1; e < EMAX; ++e)
+        if (e < E && acc[u][e] > lmax) { lmax = acc[u][e]; best = e; }
+      float den = 0.f;
+      float pe[EMAX];
 #pragma unroll
-    for (int e = 0; e < kMaxExperts; ++e) {
-      pe[e] = (e < E) ? expf(acc[e] - lmax) : 0.f;
-      den += pe[e];
-    }
-    const float inv = 1.0f / den;
-    if (lane == 0) {
-      expert[t] = best;
-      atomicAdd(&cnt[best], 1);
-    }
+      for (int e = 0; e < EMAX; ++e) {
+        pe[e] = (e < E) ? expf(acc[u][e] - lmax) : 0.f;
+        den += pe[e];
+      }
+      const float inv = 1.0f / den;
+      if (lane == 0) {
+        expert[t] = best;
+        atomicAdd(&cnt[best], 1);
+      }
 #pragma unroll
-    for (int e = 0; e < kMaxExperts; ++e) {
-      if (e < E) {
-        const float pr = pe[e] * inv;
-        if (lane == 0) probs_tok[(long long)t * E + e] = pr;
-        if (e == best && lane == 0) gate_tok[t] = pr;
+      for (int e = 0; e < EMAX; ++e) {
+        if (e < E) {
+          const float pr = pe[e] * inv;
+          if (lane == 0) probs_tok[(long long)t * E + e] = pr;
+          if (e == best && lane == 0) gate_tok[t] = pr;
+        }
       }
     }
   }
@@ -560,8 +586,13 @@ cudaError_t launch_route_and_quant(const uint16_t* X, const uint16_t* Wr, int T,
   const int nblocks = (T + kRouterTokensPerBlock - 1) / kRouterTokensPerBlock;
   if (E > 1) {
     LaunchScope ls(KID_ROUTER, st);
-    launch_pdl(k_router, nblocks, 32 * kRouterTokensPerBlock, 0, st, reinterpret_cast<const uint4*>(X), reinterpret_cast<const uint4*>(Wr), T, K, E, sv.expert, sc.gate_tok,
-                                      sc.probs_tok, sc.block_counts);
+    // up to 8 experts: two tokens per warp (half the loads and unpacking of Wr per token), 512 threads, two blocks per SM
+    if (E <= 4) launch_pdl(k_router<4, 2>, nblocks, 16 * kRouterTokensPerBlock, 0, st, reinterpret_cast<const uint4*>(X), reinterpret_cast<const uint4*>(Wr), T, K, E,
+                           sv.expert, sc.gate_tok, sc.probs_tok, sc.block_counts);
+    else if (E <= 8) launch_pdl(k_router<8, 2>, nblocks, 16 * kRouterTokensPerBlock, 0, st, reinterpret_cast<const uint4*>(X), reinterpret_cast<const uint4*>(Wr), T, K, E,
+                                sv.expert, sc.gate_tok, sc.probs_tok, sc.block_counts);
+    else launch_pdl(k_router<kMaxExperts, 1>, nblocks, 32 * kRouterTokensPerBlock, 0, st, reinterpret_cast<const uint4*>(X), reinterpret_cast<const uint4*>(Wr), T, K, E,
+                    sv.expert, sc.gate_tok, sc.probs_tok, sc.block_counts);
   }
   { LaunchScope ls(KID_ROUTE_SCAN, st);
   launch_pdl(k_route_scan, 1, 512, 0, st, T, E, nblocks, sc.block_counts, sc.block_base, sv.offsets, sv.rt); }
