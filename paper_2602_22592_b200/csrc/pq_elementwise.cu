@@ -136,7 +136,7 @@ __global__ void __launch_bounds__(256) k_binarize_pack(const float4* __restrict_
 // walks the chunks once and applies each unpacked piece of Wr to TPW tokens.  Neither changes any token's
 // arithmetic: a lane's partial sum of (token, expert) is the same chain of fused multiply-adds.
 template <int EMAX, int TPW>
-__global__ void __launch_bounds__(32 * kRouterTokensPerBlock / TPW) k_router(const uint4* __restrict__ X, const uint4* __restrict__ Wr, int T, int K,
+__global__ void __launch_bounds__(32 * kRouterTokensPerBlock / TPW, TPW >= 4 ? 2 : 1) k_router(const uint4* __restrict__ X, const uint4* __restrict__ Wr, int T, int K,
                                                                              int E, int* __restrict__ expert, float* __restrict__ gate_tok,
                                                                              float* __restrict__ probs_tok, int* __restrict__ block_counts) {
   pdl_launch_dependents();   // launched with programmatic stream serialisation: see launch_pdl
@@ -156,7 +156,7 @@ __global__ void __launch_bounds__(32 * kRouterTokensPerBlock / TPW) k_router(con
     const uint4* xrow[TPW];
 #pragma unroll
     for (int u = 0; u < TPW; ++u) xrow[u] = X + (long long)min(t0 + u, T - 1) * chunks;   // a token past the end repeats the last one, unused
-    auto fold = [&](const uint4 (&xv)[TPW], int c) {
+    auto fold = [&](const uint4 (&xv)[TPW], const uint4 (&wr)[EMAX]) {
       float x[TPW][8];
 #pragma unroll
       for (int u = 0; u < TPW; ++u) {
@@ -166,7 +166,7 @@ __global__ void __launch_bounds__(32 * kRouterTokensPerBlock / TPW) k_router(con
 #pragma unroll
       for (int e = 0; e < EMAX; ++e) {
         if (e < E) {
-          const uint4 wv = __ldg(Wr + (long long)e * chunks + c);
+          const uint4 wv = wr[e];
           const float w[8] = {bf16lo(wv.x), bf16hi(wv.x), bf16lo(wv.y), bf16hi(wv.y), bf16lo(wv.z), bf16hi(wv.z), bf16lo(wv.w), bf16hi(wv.w)};
 #pragma unroll
           for (int u = 0; u < TPW; ++u) {
@@ -178,20 +178,24 @@ __global__ void __launch_bounds__(32 * kRouterTokensPerBlock / TPW) k_router(con
         }
       }
     };
-    // the tokens' chunks in ascending order, two loads of each row in flight
+    // the tokens' chunks in ascending order; the next chunk of every row and this chunk's pieces of Wr are
+    // requested before the current chunk is folded in
     int c = lane;
-    for (; c + 32 < chunks; c += 64) {
-      uint4 xa[TPW], xb[TPW];
+    uint4 xc[TPW];
 #pragma unroll
-      for (int u = 0; u < TPW; ++u) { xa[u] = __ldg(xrow[u] + c); xb[u] = __ldg(xrow[u] + c + 32); }
-      fold(xa, c);
-      fold(xb, c + 32);
-    }
-    if (c < chunks) {
-      uint4 xa[TPW];
+    for (int u = 0; u < TPW; ++u) xc[u] = c < chunks ? __ldg(xrow[u] + c) : make_uint4(0u, 0u, 0u, 0u);
+    while (c < chunks) {
+      const int cn = c + 32;
+      uint4 xn[TPW];
 #pragma unroll
-      for (int u = 0; u < TPW; ++u) xa[u] = __ldg(xrow[u] + c);
-      fold(xa, c);
+      for (int u = 0; u < TPW; ++u) xn[u] = cn < chunks ? __ldg(xrow[u] + cn) : make_uint4(0u, 0u, 0u, 0u);
+      uint4 wr[EMAX];
+#pragma unroll
+      for (int e = 0; e < EMAX; ++e) wr[e] = e < E ? __ldg(Wr + (long long)e * chunks + c) : make_uint4(0u, 0u, 0u, 0u);
+      fold(xc, wr);
+#pragma unroll
+      for (int u = 0; u < TPW; ++u) xc[u] = xn[u];
+      c = cn;
     }
 #pragma unroll
     for (int u = 0; u < TPW; ++u) {
@@ -586,12 +590,12 @@ cudaError_t launch_route_and_quant(const uint16_t* X, const uint16_t* Wr, int T,
   const int nblocks = (T + kRouterTokensPerBlock - 1) / kRouterTokensPerBlock;
   if (E > 1) {
     LaunchScope ls(KID_ROUTER, st);
-    // up to 8 experts: two tokens per warp (half the loads and unpacking of Wr per token), 512 threads, two blocks per SM
-    if (E <= 4) launch_pdl(k_router<4, 2>, nblocks, 16 * kRouterTokensPerBlock, 0, st, reinterpret_cast<const uint4*>(X), reinterpret_cast<const uint4*>(Wr), T, K, E,
+    // two tokens per warp (half the loads and unpacking of Wr per token), 512 threads
+    if (E <= 4) launch_pdl(k_router<4, 4>, nblocks, 8 * kRouterTokensPerBlock, 0, st, reinterpret_cast<const uint4*>(X), reinterpret_cast<const uint4*>(Wr), T, K, E,
                            sv.expert, sc.gate_tok, sc.probs_tok, sc.block_counts);
-    else if (E <= 8) launch_pdl(k_router<8, 2>, nblocks, 16 * kRouterTokensPerBlock, 0, st, reinterpret_cast<const uint4*>(X), reinterpret_cast<const uint4*>(Wr), T, K, E,
+    else if (E <= 8) launch_pdl(k_router<8, 4>, nblocks, 8 * kRouterTokensPerBlock, 0, st, reinterpret_cast<const uint4*>(X), reinterpret_cast<const uint4*>(Wr), T, K, E,
                                 sv.expert, sc.gate_tok, sc.probs_tok, sc.block_counts);
-    else launch_pdl(k_router<kMaxExperts, 1>, nblocks, 32 * kRouterTokensPerBlock, 0, st, reinterpret_cast<const uint4*>(X), reinterpret_cast<const uint4*>(Wr), T, K, E,
+    else launch_pdl(k_router<kMaxExperts, 2>, nblocks, 16 * kRouterTokensPerBlock, 0, st, reinterpret_cast<const uint4*>(X), reinterpret_cast<const uint4*>(Wr), T, K, E,
                     sv.expert, sc.gate_tok, sc.probs_tok, sc.block_counts);
   }
   { LaunchScope ls(KID_ROUTE_SCAN, st);

@@ -175,6 +175,7 @@ CASES = {
     "dense_hp_ragged": dict(T=333, K=384, N=544, r=64, E=1),
     "routed8": dict(T=1000, K=512, N=768, r=128, E=8),
     "routed4_small_r": dict(T=520, K=256, N=256, r=16, E=4, scale_vector=True, alpha=1.5, beta=0.4),
+    "routed12": dict(T=300, K=320, N=256, r=16, E=12),   # more than 8 experts: the router's 16-wide instance
     # long rows: the activation quantiser keeps a row in registers of 1, 2 or 4 warps, or re-reads it
     "k2048": dict(T=70, K=2048, N=64, r=0, E=0),
     "k4096_routed": dict(T=200, K=4096, N=64, r=16, E=4),
