@@ -67,3 +67,15 @@ def test_null_arguments_rejected_before_any_launch(lib):
     L = lib.lib()
     assert L.pq_pack_weights(ctypes.byref(d), None, None, None, None, None, 0, None) == lib.PQ_ERR_NULL
     assert L.pq_debug_gemm(0, 128, 128, 128, None, None, None, None) == lib.PQ_ERR_NULL
+
+
+def test_launch_options_are_host_state(lib):
+    # options only set process-wide switches: no device is touched, unknown ids are refused
+    L = lib.lib()
+    for opt in (lib.PQ_OPT_DECODE_PDL, lib.PQ_OPT_SIDE_STREAM):
+        assert L.pq_set_option(opt, 0) == lib.PQ_OK
+        assert L.pq_set_option(opt, 1) == lib.PQ_OK
+    assert L.pq_set_option(99, 1) == lib.PQ_ERR_UNSUPPORTED
+    hdr = open(os.path.join(ROOT, "include", "pquant.h")).read()
+    assert re.search(r"PQ_OPT_DECODE_PDL\s*=\s*%d\b" % lib.PQ_OPT_DECODE_PDL, hdr)
+    assert re.search(r"PQ_OPT_SIDE_STREAM\s*=\s*%d\b" % lib.PQ_OPT_SIDE_STREAM, hdr)
