@@ -170,3 +170,31 @@ def test_full_size_projection_on_sampled_tokens(K, N, E):
         errs["dWr"] = rel_err(f32(L.dWr), g["dWr"])
     bad = {k: v for k, v in errs.items() if not v <= TOL_BF16}
     assert not bad, f"outside tolerance: {bad} (all: {errs})"
+
+
+def test_first_use_inside_a_capture_keeps_plain_stream_order():
+    # a stream whose first call is made while it is being captured gets no helper stream (nothing is created
+    # during a capture): the graph holds the kernels in plain order and replays to the same bits
+    c = I.make_linear_case(384, 256, 320, 32, 1, seed=23)
+    L = run_fwd_bwd(c, False)
+    want = _all_outputs(L)
+    s = torch.cuda.Stream()            # never used with the library before
+    s.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(s):
+        with torch.cuda.graph(g, stream=s):
+            L.forward()
+            L.backward()
+    for t in (L.Y, L.dX, L.dW, L.dA, L.dB, L.dalpha, L.dbeta):
+        t.zero_()
+    g.replay()
+    torch.cuda.synchronize()
+    check_status()
+    for a, b in zip(want, _all_outputs(L)):
+        assert torch.equal(a, b)
+    with torch.cuda.stream(s):         # after the capture the stream gets its helper as usual
+        L.forward()
+        L.backward()
+    torch.cuda.synchronize()
+    for a, b in zip(want, _all_outputs(L)):
+        assert torch.equal(a, b)
