@@ -198,3 +198,17 @@ def test_first_use_inside_a_capture_keeps_plain_stream_order():
     torch.cuda.synchronize()
     for a, b in zip(want, _all_outputs(L)):
         assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("T", [1, 3, 33, 130])
+def test_few_tokens_routed(T):
+    # fewer tokens than a router warp group, a block or a tile holds; most experts stay empty
+    c = I.make_linear_case(T, 256, 256, 32, 8, seed=40 + T, zipf=False)
+    f = O.linear_forward(c["X"], c["W"], c["A"], c["B"], c["Wr"], c["alpha"], c["beta"])
+    g = O.linear_backward(c["dY"], c["X"], f, c["A"], c["B"], c["Wr"], c["alpha"], c["beta"])
+    L = run_fwd_bwd(c, False)
+    sv = L.saved_view()
+    assert np.array_equal(sv["expert"].cpu().numpy(), f["idx"])
+    assert np.array_equal(sv["perm"].cpu().numpy(), f["perm"])
+    assert rel_err(f32(L.Y), f["Y"]) <= TOL_BF16
+    check_backward(c, L, f, g, False)
