@@ -15,9 +15,22 @@
  *
  * Conventions common to every entry point
  *   - every data pointer is a DEVICE pointer owned by the caller; the library
- *     never allocates, frees or keeps device memory between calls;
- *   - work is only enqueued on `stream` (a cudaStream_t passed as void*); no
- *     call synchronises the device;
+ *     never allocates or frees device memory and keeps no pointer into the
+ *     caller's memory between calls.  What it does keep, per process: a few
+ *     small file-scope device variables (a status word, the spin limit, the
+ *     64 KiB array of pq_pack_weights_static), and -- unless PQ_OPT_SIDE_STREAM
+ *     is 0 -- one helper stream and three events per (device, caller stream)
+ *     that has called pq_linear_forward / pq_linear_backward, created on first
+ *     use and kept until the process exits;
+ *   - work is only enqueued on `stream` (a cudaStream_t passed as void*) and on
+ *     that helper stream, which is joined back into `stream` inside the same
+ *     call; no call synchronises the device except pq_device_status and
+ *     pq_set_option(PQ_OPT_SPIN_CYCLES);
+ *   - threads: calls on different streams may come from different host threads;
+ *     the helper-stream table is locked.  pq_set_option, pq_profile_events and the
+ *     launch counter behind pq_kernel_launches are plain process-wide state without
+ *     locks: set options and register events while no other thread is inside the
+ *     library, and read the counter as an approximate figure under concurrency;
  *   - the return value is a status: PQ_OK (0) or a negative PQ_ERR_* code.
  *     Nothing is thrown.  After an error the outputs are undefined;
  *   - matrices are dense row-major: X[T,K] bf16, latent W[N,K] fp32,
@@ -179,8 +192,8 @@ int pq_decode_view_init(const pq_desc* d, void* ws, pq_decode_view* out);
  * gate and up projections of a block, the q/k/v projections, other sequences -- should
  * stream their weights back to back instead of paying a launch and a pipeline fill each).
  * Each item is what pq_linear_forward takes in its decode form; results are identical to n
- * separate calls.  `items` is a HOST array, read before the call returns.  Any n >= 1
- * (launched in groups of 16); every item needs its own ws. */
+ * separate calls.  `items` is a HOST array, read before the call returns.  1 <= n <= 4096
+ * (PQ_ERR_SHAPE otherwise; launched in groups of 16); every item needs its own ws. */
 typedef struct pq_decode_item {
   pq_desc desc;            /* T <= 16 */
   const uint16_t* X;       /* [T,K] bf16 */
@@ -218,6 +231,14 @@ int pq_linear_backward(const pq_desc* d, const uint16_t* dY, const uint16_t* X,
                        float* dW, float* dA, float* dB, float* dWr, float* dalpha, float* dbeta,
                        void* ws, size_t ws_bytes, void* stream);
 
+/* What pq_linear_backward leaves in its workspace, for tests and diagnostics.
+ *   dl [T,E] fp32: gradient of the router logits (Sec. 3.3, the router is trained end to end),
+ *   dl[p,j] = dg g (delta_{j,e} - p_j) for the token at SORTED position p; NULL when E <= 1. */
+typedef struct pq_bwd_view {
+  float* dl;
+} pq_bwd_view;
+int pq_bwd_view_init(const pq_desc* d, void* ws, pq_bwd_view* out);
+
 /* Test hook for the tensor-core engine: D[M,N] = A . B^T-style contraction with
  * raw accumulators written out (int32 for mode 0, fp32 otherwise), so that the
  * integer 1-bit product (Eq. 10) can be checked bit for bit.
@@ -250,8 +271,15 @@ int pq_device_status(void* stream, int* code, int* where);
  *   order is unchanged and a stream capture records one graph with a fork and a join.  In the
  *   backward pass the weight-gradient tiles that need only dY and q/gamma are one launch
  *   (profile id bwd_dw) and the HP tiles (dB, dA, router) a second one (id hp_db).
- *   0 = every kernel on the caller's stream, the weight gradient as one launch. */
-enum { PQ_OPT_DECODE_PDL = 1, PQ_OPT_SIDE_STREAM = 2 };
+ *   0 = every kernel on the caller's stream, the weight gradient as one launch.
+ *   PQ_OPT_SPIN_CYCLES: limit of every device-side spin-wait in SM clock cycles (value <= 0 restores
+ *   the default of 4e9, about two seconds).  A test hook: with a limit of a few cycles the first wait
+ *   that does not succeed at once runs out, the kernel stops issuing work, lets copies and MMAs in
+ *   flight finish, releases its TMEM and returns; pq_device_status then reports PQ_ERR_TIMEOUT and the
+ *   outputs of that call are undefined.  Applies to the current device; blocks until the device's
+ *   earlier work has finished.  Meant for pq_debug_gemm; do not shorten the limit around the decode
+ *   entry points, whose later stages read indices an abandoned stage has not delivered. */
+enum { PQ_OPT_DECODE_PDL = 1, PQ_OPT_SIDE_STREAM = 2, PQ_OPT_SPIN_CYCLES = 3 };
 int pq_set_option(int option, int value);
 
 /* Cumulative number of kernels this library has launched in this process. */

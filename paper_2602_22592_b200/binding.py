@@ -22,7 +22,7 @@ PQ_DECODE_DUMP_ACC = 2
 PQ_PHASE_PACK, PQ_PHASE_FWD, PQ_PHASE_BWD, PQ_PHASE_DECODE = 0, 1, 2, 3
 
 EXPORTS = ("pq_status_string", "pq_workspace_bytes", "pq_saved_bytes", "pq_saved_view_init",
-           "pq_decode_view_init", "pq_decode_batch", "pq_pack_weights", "pq_pack_weights_static", "pq_linear_forward", "pq_linear_backward", "pq_debug_gemm", "pq_debug_gemm_tile",
+           "pq_decode_view_init", "pq_bwd_view_init", "pq_decode_batch", "pq_pack_weights", "pq_pack_weights_static", "pq_linear_forward", "pq_linear_backward", "pq_debug_gemm", "pq_debug_gemm_tile",
            "pq_device_status", "pq_kernel_launches", "pq_profile_events", "pq_set_option")
 
 KERNEL_IDS = dict(pack_sums=0, binarize_pack=1, router=2, route_scan=3, act_quant=4, hp_up=5, fwd=6, scatter_rows=7,
@@ -58,6 +58,10 @@ class pq_decode_view(ctypes.Structure):
     _fields_ = [("tokens", ctypes.c_void_p), ("acc", ctypes.c_void_p)]
 
 
+class pq_bwd_view(ctypes.Structure):
+    _fields_ = [("dl", ctypes.c_void_p)]
+
+
 _lib = None
 
 
@@ -80,6 +84,8 @@ def lib() -> ctypes.CDLL:
         L.pq_saved_view_init.argtypes = [dp, vp, ctypes.POINTER(pq_saved_view)]
         L.pq_decode_view_init.restype = ci
         L.pq_decode_view_init.argtypes = [dp, vp, ctypes.POINTER(pq_decode_view)]
+        L.pq_bwd_view_init.restype = ci
+        L.pq_bwd_view_init.argtypes = [dp, vp, ctypes.POINTER(pq_bwd_view)]
         L.pq_decode_batch.restype = ci
         L.pq_decode_batch.argtypes = [ctypes.POINTER(pq_decode_item), ci, vp]
         L.pq_pack_weights.restype = ci
@@ -183,6 +189,17 @@ def pq_decode_view_init(d: pq_desc, ws: torch.Tensor) -> dict:
     return out
 
 
+def pq_bwd_view_init(d: pq_desc, ws: torch.Tensor) -> dict:
+    """Views into the backward workspace: dl [T,E], the router-logit gradient in sorted token order (None when E <= 1)."""
+    v = pq_bwd_view()
+    _check("pq_bwd_view_init", lib().pq_bwd_view_init(ctypes.byref(d), _ptr(ws), ctypes.byref(v)))
+    out = dict(dl=None)
+    if v.dl:
+        off = v.dl - ws.data_ptr()
+        out["dl"] = ws[off: off + 4 * d.T * d.E].view(torch.float32).view(d.T, d.E)
+    return out
+
+
 def pq_pack_weights(d, W, w_bits, w_s8, w_scales, ws, stream=None):
     _check("pq_pack_weights", lib().pq_pack_weights(ctypes.byref(d), _ptr(W), _ptr(w_bits), _ptr(w_s8), _ptr(w_scales),
                                                      _ptr(ws), _nbytes(ws), _stream(stream)))
@@ -248,6 +265,7 @@ def pq_device_status(stream=None) -> tuple[int, int]:
 
 PQ_OPT_DECODE_PDL = 1
 PQ_OPT_SIDE_STREAM = 2
+PQ_OPT_SPIN_CYCLES = 3
 
 
 def pq_set_option(option: int, value: int):

@@ -298,6 +298,16 @@ int pq_saved_view_init(const pq_desc* d, void* saved, pq_saved_view* out) {
   return PQ_OK;
 }
 
+int pq_bwd_view_init(const pq_desc* d, void* ws, pq_bwd_view* out) {
+  if (!d || !ws || !out) return PQ_ERR_NULL;
+  int rc = check_desc(d, true);
+  if (rc) return rc;
+  BwdScratch s;
+  carve_bwd_scratch(d, ws, &s);
+  out->dl = s.dl;
+  return PQ_OK;
+}
+
 int pq_decode_view_init(const pq_desc* d, void* ws, pq_decode_view* out) {
   if (!d || !ws || !out) return PQ_ERR_NULL;
   int rc = check_desc(d, false);
@@ -486,6 +496,12 @@ int pq_set_option(int option, int value) {
   switch (option) {
     case PQ_OPT_DECODE_PDL: decode_set_pdl(value); return PQ_OK;
     case PQ_OPT_SIDE_STREAM: g_side_streams = value ? 1 : 0; return PQ_OK;
+    case PQ_OPT_SPIN_CYCLES: {
+      // the limit lives in constant memory of the current device; the copy is ordered after everything
+      // already enqueued there (a blocking copy), so no running kernel sees it change
+      const long long cycles = value > 0 ? (long long)value : kDefaultSpinCycles;
+      return cudaMemcpyToSymbol(c_spin_cycles, &cycles, sizeof(cycles)) == cudaSuccess ? PQ_OK : PQ_ERR_CUDA;
+    }
     default: return PQ_ERR_UNSUPPORTED;
   }
 }

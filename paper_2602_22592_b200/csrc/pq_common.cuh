@@ -21,8 +21,12 @@ __device__ __forceinline__ void report_timeout(int where) {
   if (atomicCAS(&g_status[0], 0, PQ_ERR_TIMEOUT) == 0) g_status[1] = where;
 }
 
-// about two seconds at 2 GHz; every legitimate wait is micro- to milliseconds
-constexpr long long kSpinCycles = 4000000000LL;
+// Limit of every spin-wait, in SM clock cycles: about two seconds at 2 GHz, while every legitimate wait is
+// micro- to milliseconds.  It lives in constant memory so that a test can shorten it (pq_set_option,
+// PQ_OPT_SPIN_CYCLES) and watch a wait run out without anything being broken: the kernel then records
+// PQ_ERR_TIMEOUT, stops issuing work, lets what is in flight land and returns.
+constexpr long long kDefaultSpinCycles = 4000000000LL;
+__constant__ long long c_spin_cycles = kDefaultSpinCycles;
 
 // ---------------------------------------------------------------------------
 // bf16 helpers
@@ -66,12 +70,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait.  Returns false (after recording the failure) if the phase did
-// not complete within kSpinCycles; the caller must then stop issuing work.
+// not complete within c_spin_cycles; the caller must then stop issuing work.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int where) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   while (!mbar_try_wait(bar, parity)) {
-    if (clock64() - t0 > kSpinCycles) {
+    if (clock64() - t0 > c_spin_cycles) {
       report_timeout(where);
       return false;
     }

@@ -113,7 +113,7 @@ __device__ __forceinline__ void decode_wait(uint32_t bar, uint32_t parity, volat
   const long long t0 = clock64();
   while (!mbar_try_wait(bar, parity)) {
     if (*fail) return;
-    if (clock64() - t0 > kSpinCycles) {
+    if (clock64() - t0 > c_spin_cycles) {
       report_timeout(WHERE_OTHER);
       *fail = 1;
       return;

@@ -59,11 +59,15 @@ __global__ void __launch_bounds__(256) k_weight_partial_sums(const float4* __res
 
 // Every block re-reduces the (few hundred) partials in the same order, so all blocks agree on mu without
 // a grid-wide barrier: thread t sums partials t, t + 256, ... (ascending), then a fixed tree over the block.
+// The partials were written by the kernel before this one and the buffer is reused from call to call, so they are
+// read with L2 loads (ld.global.cg): a kernel launched with programmatic stream serialisation can be resident while
+// an older kernel still reads the previous call's values on the same SM, and the read-only data path gives no
+// guarantee against finding those in L1.
 __device__ __forceinline__ void reduce_partials(const double* partial, int nparts, double inv_count, float* mu, float* lam) {
   __shared__ double sh[2][8];
   __shared__ double fin[2];
   double s = 0.0, a = 0.0;
-  for (int i = threadIdx.x; i < nparts; i += 256) { s += partial[2 * i]; a += partial[2 * i + 1]; }
+  for (int i = threadIdx.x; i < nparts; i += 256) { s += __ldcg(partial + 2 * i); a += __ldcg(partial + 2 * i + 1); }
   for (int d = 16; d > 0; d >>= 1) {
     s += __shfl_xor_sync(0xffffffffu, s, d);
     a += __shfl_xor_sync(0xffffffffu, a, d);
@@ -85,7 +89,7 @@ __device__ __forceinline__ void reduce_partials(const double* partial, int npart
 // words (bit j of word i <-> k = 32 i + j, 1 <-> +1; App. A) and the +-1 int8
 // tile the tensor cores read.  Each thread owns 4 consecutive k.
 // ---------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) k_binarize_pack(const float4* __restrict__ W4, long long n4, const double* __restrict__ partial,
+__global__ void __launch_bounds__(256) k_binarize_pack(const float4* __restrict__ W4, long long n4, const double* partial,
                                                        int nparts, double inv_count, uint32_t* __restrict__ bits,
                                                        uint32_t* __restrict__ s8x4, float* __restrict__ scales) {
   pdl_launch_dependents();   // launched with programmatic stream serialisation: see launch_pdl

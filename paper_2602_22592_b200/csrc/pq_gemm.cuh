@@ -101,7 +101,7 @@ __device__ __forceinline__ bool pipe_wait(uint32_t bar, uint32_t parity, int whe
   const long long t0 = clock64();
   while (!mbar_try_wait(bar, parity)) {
     if (*abort_flag) return false;
-    if (clock64() - t0 > kSpinCycles) {
+    if (clock64() - t0 > c_spin_cycles) {
       report_timeout(where);
       *abort_flag = 1;
       return false;
@@ -312,7 +312,10 @@ __device__ __forceinline__ void gemm_body(const typename P::Params& p) {
       P::tile_init(p, tile, t);
       // per-row factors and addresses are fetched while the contraction is still running
       const typename P::Pre pre = P::prepare(p, t, quad, lane);
-      if (!pipe_wait(tfull_bar(ac.stage), ac.phase, WHERE_EPILOGUE, abort_flag)) { ok = false; break; }
+      // Every lane watches the barrier itself, but the warp takes ONE decision: what follows is full of
+      // warp-collective instructions (tcgen05.ld, shuffles), so a lane that gave up must take the others along.
+      ok = __all_sync(0xffffffffu, pipe_wait(tfull_bar(ac.stage), ac.phase, WHERE_EPILOGUE, abort_flag));
+      if (!ok) break;
       tc_fence_after();
       const uint32_t tlane = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
       P::epilogue(p, t, pre, tlane + Acc::col(ac.stage, 0), tlane + Acc::col(ac.stage, 1), quad, half, lane, epi_stage + (warp - 2) * kEpiWarpBytes);

@@ -20,48 +20,78 @@ def _f32(a, dev):
     return None if a is None else torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(dev).contiguous()
 
 
-class PQLinear:
-    """One decoupled linear layer of fixed shape on one CUDA device."""
+GUARD_BYTES = 4096      # canary band in front of and behind every guarded buffer
+GUARD_BYTE = 0xA5
 
-    def __init__(self, T, K, N, r=0, E=0, scale_vector=False, device="cuda:0", training=True, dump_acc=False):
+
+class PQLinear:
+    """One decoupled linear layer of fixed shape on one CUDA device.
+
+    guard=True puts a band of canary bytes in front of and behind every buffer the library writes
+    (outputs, packed weights, the saved buffer, the workspaces); `check_guards()` then tells whether
+    any kernel wrote outside the bytes it was given.  (torch's caching allocator rounds sizes up, so an
+    overrun of an exact-size tensor would otherwise land in slack nobody looks at.)"""
+
+    def __init__(self, T, K, N, r=0, E=0, scale_vector=False, device="cuda:0", training=True, dump_acc=False, guard=False):
         self.dev = torch.device(device)
         self.T, self.K, self.N, self.r, self.E = T, K, N, r, (E if r > 0 else 0)
         self.scale_vector = scale_vector
         self.desc = pqb.make_desc(T, K, N, r, self.E, 1, scale_vector)
-        dev = self.dev
-        u8 = dict(dtype=torch.uint8, device=dev)
-        self.w_bits = torch.empty((N, K // 32), dtype=torch.int32, device=dev)
-        self.w_s8 = torch.empty((N, K), dtype=torch.int8, device=dev)
-        self.w_scales = torch.empty(2, dtype=torch.float32, device=dev)
-        self.ws_pack = torch.empty(pqb.pq_workspace_bytes(self.desc, pqb.PQ_PHASE_PACK), **u8)
+        self.guard = guard
+        self._guards = []
+        self.w_bits = self._buf((N, K // 32), torch.int32)
+        self.w_s8 = self._buf((N, K), torch.int8)
+        self.w_scales = self._buf((2,), torch.float32)
+        self.ws_pack = self._buf((pqb.pq_workspace_bytes(self.desc, pqb.PQ_PHASE_PACK),), torch.uint8)
         self.training = training
         if training:
             nb = pqb.pq_saved_bytes(self.desc)
             if nb == 0:
                 raise pqb.PqError("pq_saved_bytes", pqb.PQ_ERR_SHAPE)
-            self.saved = torch.empty(nb, **u8)
-            self.ws_fwd = torch.empty(pqb.pq_workspace_bytes(self.desc, pqb.PQ_PHASE_FWD), **u8)
-            self.ws_bwd = torch.empty(max(16, pqb.pq_workspace_bytes(self.desc, pqb.PQ_PHASE_BWD)), **u8)
-            self.Y = torch.empty((T, N), dtype=torch.bfloat16, device=dev)
-            self.dX = torch.empty((T, K), dtype=torch.bfloat16, device=dev)
-            self.dW = torch.empty((N, K), dtype=torch.float32, device=dev)
+            self.saved = self._buf((nb,), torch.uint8)
+            self.ws_fwd = self._buf((pqb.pq_workspace_bytes(self.desc, pqb.PQ_PHASE_FWD),), torch.uint8)
+            self.ws_bwd = self._buf((max(16, pqb.pq_workspace_bytes(self.desc, pqb.PQ_PHASE_BWD)),), torch.uint8)
+            self.Y = self._buf((T, N), torch.bfloat16)
+            self.dX = self._buf((T, K), torch.bfloat16)
+            self.dW = self._buf((N, K), torch.float32)
             ns = N if scale_vector else 1
-            self.dalpha = torch.empty(ns, dtype=torch.float32, device=dev)
-            self.dbeta = torch.empty(ns, dtype=torch.float32, device=dev)
+            self.dalpha = self._buf((ns,), torch.float32)
+            self.dbeta = self._buf((ns,), torch.float32)
             if r > 0:
                 Ee = max(self.E, 1)
-                self.dA = torch.empty((Ee, r, K), dtype=torch.float32, device=dev)
-                self.dB = torch.empty((Ee, N, r), dtype=torch.float32, device=dev)
-                self.dWr = torch.empty((Ee, K), dtype=torch.float32, device=dev) if Ee > 1 else None
+                self.dA = self._buf((Ee, r, K), torch.float32)
+                self.dB = self._buf((Ee, N, r), torch.float32)
+                self.dWr = self._buf((Ee, K), torch.float32) if Ee > 1 else None
             else:
                 self.dA = self.dB = self.dWr = None
         else:
             # decode: T <= 16 tokens straight from the packed bits
             self.desc = pqb.make_desc(T, K, N, r, self.E, 1, scale_vector, dump_acc=dump_acc)
             nb = pqb.pq_workspace_bytes(self.desc, pqb.PQ_PHASE_DECODE)
-            self.ws_decode = torch.zeros(max(nb, 16), **u8) if T <= 16 else None
-            self.Y = torch.empty((T, N), dtype=torch.bfloat16, device=dev)
+            self.ws_decode = self._buf((max(nb, 16),), torch.uint8).zero_() if T <= 16 else None
+            self.Y = self._buf((T, N), torch.bfloat16)
         self.X = self.W = self.A = self.B = self.Wr = self.alpha = self.beta = self.dY = None
+
+    # -- buffers --------------------------------------------------------------
+    def _buf(self, shape, dtype):
+        """A device buffer the library writes into; with guard=True carved out of a larger allocation
+        whose first and last GUARD_BYTES hold the canary pattern."""
+        if not self.guard:
+            return torch.empty(shape, dtype=dtype, device=self.dev)
+        n = 1
+        for s in shape:
+            n *= s
+        nbytes = n * torch.empty(0, dtype=dtype).element_size()
+        raw = torch.full((nbytes + 2 * GUARD_BYTES,), GUARD_BYTE, dtype=torch.uint8, device=self.dev)
+        self._guards.append((raw, nbytes))
+        return raw[GUARD_BYTES:GUARD_BYTES + nbytes].view(dtype).view(*shape)
+
+    def check_guards(self) -> int:
+        """Number of canary bytes that no longer hold the pattern (0 = nothing was written out of bounds)."""
+        bad = 0
+        for raw, nbytes in self._guards:
+            bad += int((raw[:GUARD_BYTES] != GUARD_BYTE).sum()) + int((raw[GUARD_BYTES + nbytes:] != GUARD_BYTE).sum())
+        return bad
 
     # -- data ---------------------------------------------------------------
     def load_case(self, case: dict):
@@ -115,3 +145,6 @@ class PQLinear:
 
     def saved_view(self) -> dict:
         return pqb.pq_saved_view_init(self.desc, self.saved)
+
+    def bwd_view(self) -> dict:
+        return pqb.pq_bwd_view_init(self.desc, self.ws_bwd)

@@ -215,6 +215,56 @@ def test_single_expert_has_unit_gate_and_dense_form():
     assert "dWr" not in g
 
 
+def test_routed_forward_sum_written_out_term_by_term():
+    # Sec. 3.3 + Eq. 10-11 for a ROUTED layer, with python floats and plain loops only:
+    #   Y[t,n] = alpha_n * p[t,e*] * (B_e* (A_e* x_t))[n] + beta_n * (lam / gamma_t) * sum_k S[n,k] q[t,k]
+    # with e* the arg-max logit and p the softmax over all E logits.  Nothing of the oracle's forward is reused
+    # except its quantised operands (q, gamma, S, lam), which have pins of their own above.
+    T, K, N, r, E = 6, 32, 8, 4, 3
+    c = I.make_linear_case(T, K, N, r, E, seed=61, zipf=False, scale_vector=True)
+    c["Wr"] = I.bf16_values((c["Wr"] * 30).astype(np.float32))          # logits well apart: no near-tie, gates well below 1
+    c["alpha"] = np.linspace(1.1, 1.9, N).astype(np.float32)
+    c["beta"] = np.linspace(0.3, 0.7, N).astype(np.float32)
+    f = O.linear_forward(c["X"], c["W"], c["A"], c["B"], c["Wr"], c["alpha"], c["beta"])
+    X, A, B, Wr = ([[float(v) for v in row] for row in m] if m.ndim == 2 else [[[float(v) for v in row] for row in e] for e in m]
+                   for m in (c["X"], c["A"], c["B"], c["Wr"]))
+    lam = float(f["lam"])
+
+    def by_hand(use_gate=True, expert_shift=0, softmax_over_all=True):
+        Y = [[0.0] * N for _ in range(T)]
+        experts = []
+        for t in range(T):
+            logit = [sum(X[t][k] * Wr[e][k] for k in range(K)) for e in range(E)]
+            best = max(range(E), key=lambda e: (logit[e], -e))
+            m = max(logit)
+            den = sum(np.exp(l - m) for l in logit) if softmax_over_all else np.exp(logit[best] - m)
+            gate = np.exp(logit[best] - m) / den if use_gate else 1.0
+            e = (best + expert_shift) % E
+            experts.append(best)
+            h = [sum(A[e][j][k] * X[t][k] for k in range(K)) for j in range(r)]
+            for n in range(N):
+                z = sum(B[e][n][j] * h[j] for j in range(r))
+                acc = sum(int(f["S"][n, k]) * int(f["q"][t, k]) for k in range(K))
+                Y[t][n] = float(c["alpha"][n]) * gate * z + float(c["beta"][n]) * (lam / float(f["gamma"][t])) * acc
+        return np.array(Y), experts
+
+    want, experts = by_hand()
+    assert experts == f["idx"].tolist()
+    assert len(set(experts)) > 1                                          # more than one expert is really in use
+    assert 0.4 < float(f["gate"].min()) and float(f["gate"].max()) < 0.999   # the gate is not a disguised 1
+    # the HP term is a visible share of the output, so an error in it cannot hide in the tolerance
+    hp_share = np.abs(want - np.asarray(c["beta"], np.float64)[None, :] * f["y1"]).mean() / np.abs(want).mean()
+    assert hp_share > 0.05
+    tol = 1e-5 * np.abs(want).max()       # the oracle's gate comes from logits summed in fp32 order
+    assert np.max(np.abs(f["Y64"] - want)) <= tol
+    # planted mistakes: each one must break the same comparison
+    for wrong in (by_hand(use_gate=False)[0], by_hand(expert_shift=1)[0], by_hand(softmax_over_all=False)[0]):
+        assert np.max(np.abs(f["Y64"] - wrong)) > 100 * tol
+    assert np.max(np.abs(f["Y64"] - (want - 2 * np.asarray(c["beta"], np.float64)[None, :] * f["y1"]))) > 100 * tol   # sign of the 1-bit term
+    # and the stored output is that sum rounded once to bf16
+    assert np.array_equal(f["Y"], O.round_to_bf16(f["Y64"]))
+
+
 def test_bf16_rounding_helper():
     x = np.array([1.0, 1.00390625, 1.005859375, 1.01171875, -3.14159, 1e-3, 65504.0])
     r = O.round_to_bf16(x)

@@ -11,6 +11,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import pquant_oracle as O
 from paper_2602_22592_b200 import binding as pqb
 from paper_2602_22592_b200 import inputs as I
 
@@ -46,6 +47,37 @@ def test_static_pack_matches_regular_pack_twice_in_a_row():
         assert np.all(np.abs(sc_s - sc_r) <= 1e-5 * np.abs(sc_r[0]))      # lam, mu: fp32-accumulated-scale tolerance
         assert np.array_equal(bits_s, bits_r)
         assert np.array_equal(s8_s, s8_r)
+
+
+def test_static_pack_back_to_back_without_a_sync_matches_the_oracle():
+    # The documented way to share the one scratch array: several calls in stream order, nothing in between.  A large
+    # matrix, a small one with a shifted mean, a large one again: every call must see its own partial sums, not its
+    # neighbour's, and each result is checked against the CPU oracle (Eq. 3, 4, 6), bit for bit.
+    mats = [I.make_linear_case(1, 2048, 1536, 0, 0, seed=73, with_grad=False)["W"],
+            (I.make_linear_case(1, 256, 96, 0, 0, seed=74, with_grad=False)["W"] - np.float32(0.015)).astype(np.float32),
+            (I.make_linear_case(1, 1024, 2048, 0, 0, seed=75, with_grad=False)["W"] + np.float32(0.004)).astype(np.float32)]
+    dev = [torch.from_numpy(W).cuda() for W in mats]
+    outs = []
+    for W in mats:
+        N, K = W.shape
+        outs.append((torch.zeros((N, K // 32), dtype=torch.int32, device="cuda"), torch.zeros((N, K), dtype=torch.int8, device="cuda"),
+                     torch.zeros(2, dtype=torch.float32, device="cuda")))
+    # warm up the entry point (its first call on a device looks up the array's address), then measure free memory
+    pqb.pq_pack_weights_static(pqb.make_desc(128, mats[1].shape[1], mats[1].shape[0]), dev[1], *outs[1])
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    for W, Wd, (bits, s8, sc) in zip(mats, dev, outs):
+        pqb.pq_pack_weights_static(pqb.make_desc(128, W.shape[1], W.shape[0]), Wd, bits, s8, sc)     # no synchronisation in between
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before       # the calls took no device memory
+    for W, (bits, s8, sc) in zip(mats, outs):
+        mu, lam = O.weight_scales(W)
+        S = O.binarize(W, mu)
+        got = sc.cpu().numpy()
+        assert abs(got[0] - lam) <= 1e-5 * abs(lam) and abs(got[1] - mu) <= 1e-5 * abs(lam)
+        assert got[0] == lam and got[1] == mu
+        assert np.array_equal(s8.cpu().numpy(), S)
+        assert np.array_equal(bits.cpu().numpy().view(np.uint32), O.pack_bits(S))
 
 
 def test_static_pack_rejects_oversized_and_bad_arguments():
