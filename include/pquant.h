@@ -157,6 +157,16 @@ int pq_pack_weights(const pq_desc* d, const float* W, uint32_t* w_bits, int8_t* 
 int pq_pack_weights_static(const pq_desc* d, const float* W, uint32_t* w_bits, int8_t* w_s8,
                            float* w_scales, void* stream);
 
+/* INT8 high-precision branch (Sec. 3.2: the branch runs at 8-bit precision, its weights quantised the way the
+ * 8-bit activations are): Eq. 7-9 applied to each expert matrix as a whole,
+ *     gamma = 2^7 / max(max|w|, 1e-5),   code = clamp(rint(w * gamma), -128, 127)   (fp32, round half to even).
+ *   A [E,r,K], B [E,N,r] bf16 (in);  A8 [E,r,K], B8 [E,N,r] int8 (out);
+ *   hp_scales [E][2] float (out) = { gamma_A_e, gamma_B_e };
+ *   ws: workspace of pq_workspace_bytes(d, PQ_PHASE_PACK) bytes.
+ * r * K and N * r must be multiples of 8 (they are: r is a multiple of 8). */
+int pq_pack_experts(const pq_desc* d, const uint16_t* A, const uint16_t* B, int8_t* A8, int8_t* B8, float* hp_scales, void* ws,
+                    size_t ws_bytes, void* stream);
+
 /* Forward of the layer (Eq. 10-11, Sec. 3.3).
  *   training (w_s8 != NULL): tensor-core path; fills `saved` (may be NULL when
  *     no backward follows).  A, B may be NULL iff r == 0; Wr NULL iff E <= 1.

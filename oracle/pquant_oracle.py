@@ -241,6 +241,71 @@ def hp_branch_all_experts(X, A, B, weights):
 
 
 # --------------------------------------------------------------------------
+# high-precision branch in INT8 (Sec. 3.2: the branch runs at 8-bit precision,
+# its weights quantised the way the 8-bit activations are)
+# --------------------------------------------------------------------------
+def absmax_quant_matrix(Wm):
+    """Eq. 7-9 applied to a whole weight matrix: gamma_W = 2^7 / max|W| (one scale
+    per matrix, as the 1-bit branch has one lam per matrix), W8 = RoundClip(W * gamma_W)
+    in [-128, 127].  Same fp32 arithmetic as act_quant.  Returns W8 int8, gamma_W fp32."""
+    W32 = np.asarray(Wm, dtype=np.float32)
+    amax = np.maximum(np.float32(np.max(np.abs(W32))) if W32.size else np.float32(0), ACT_AMAX_FLOOR)
+    gamma = np.float32(ACT_QMAX / amax)
+    q = np.clip(np.rint((W32 * gamma).astype(np.float32)), -128.0, 127.0).astype(np.int8)
+    return q, gamma
+
+
+def quantize_experts(A, B):
+    """absmax_quant_matrix for every expert's two matrices: A8 [E,r,K], gA [E], B8 [E,N,r], gB [E]."""
+    E = A.shape[0]
+    A8, B8 = np.zeros(A.shape, np.int8), np.zeros(B.shape, np.int8)
+    gA, gB = np.zeros(E, np.float32), np.zeros(E, np.float32)
+    for e in range(E):
+        A8[e], gA[e] = absmax_quant_matrix(A[e])
+        B8[e], gB[e] = absmax_quant_matrix(B[e])
+    return A8, gA, B8, gB
+
+
+def requant_hidden(h_int):
+    """The hidden activation of the INT8 branch is an exact integer, h_int = A8 q; it enters the second 8-bit linear
+    quantised per token like any activation (Eq. 7-9).  Its real value is h_int / (gamma_A gamma_t), a positive
+    multiple of the integer, so the codes can be taken from the integers themselves:
+        gamma_h = fl32(128 / max(fl32(max_j |h_int|), 1e-5)),  qh = RoundClip(fl32(fl32(h_int) * gamma_h)),
+    every step one IEEE fp32 operation (the conversion of an integer above 2^24 rounds to nearest even).
+    Returns qh int8 [T,r], gamma_h fp32 [T] (the scale relative to h_int)."""
+    h32 = np.asarray(h_int, dtype=np.int64).astype(np.float32)
+    amax = np.max(np.abs(h32), axis=1) if h32.shape[1] else np.zeros(h32.shape[0], np.float32)
+    gamma_h = (ACT_QMAX / np.maximum(amax.astype(np.float32), ACT_AMAX_FLOOR)).astype(np.float32)
+    qh = np.clip(np.rint((h32 * gamma_h[:, None]).astype(np.float32)), -128.0, 127.0).astype(np.int8)
+    return qh, gamma_h
+
+
+def hp_branch_int8(q, gamma, A8, gA, B8, gB, idx):
+    """INT8 high-precision branch on the int8 activation codes q (the same codes the 1-bit branch multiplies):
+        h_int = A8_e q_t   (exact)        ->  qh, gamma_h = requant_hidden(h_int)
+        z_int = B8_e qh_t  (exact)        ->  z = z_int / (gamma_B gamma_h gamma_A gamma_t)   (fp64)
+    Returns dict(h_int, qh, gamma_h, z_int, z, scale) with scale[t] the fp64 factor z / z_int."""
+    q64 = np.asarray(q, dtype=np.int64)
+    T = q64.shape[0]
+    E, r, _ = A8.shape
+    N = B8.shape[1]
+    h_int = np.zeros((T, r), np.int64)
+    for e in range(E):
+        sel = np.nonzero(idx == e)[0]
+        if sel.size:
+            h_int[sel] = q64[sel] @ A8[e].astype(np.int64).T
+    assert np.all(np.abs(h_int) < 2 ** 31)
+    qh, gamma_h = requant_hidden(h_int)
+    z_int = np.zeros((T, N), np.int64)
+    for e in range(E):
+        sel = np.nonzero(idx == e)[0]
+        if sel.size:
+            z_int[sel] = qh[sel].astype(np.int64) @ B8[e].astype(np.int64).T
+    scale = 1.0 / (gB.astype(np.float64)[idx] * gamma_h.astype(np.float64) * gA.astype(np.float64)[idx] * np.asarray(gamma, np.float64))
+    return dict(h_int=h_int, qh=qh, gamma_h=gamma_h, z_int=z_int, z=z_int * scale[:, None], scale=scale)
+
+
+# --------------------------------------------------------------------------
 # the layer: forward (Eq. 10 + Eq. 11) and STE backward (App. B.1)
 # --------------------------------------------------------------------------
 def _scale_vec(s, N):
@@ -249,12 +314,14 @@ def _scale_vec(s, N):
     return np.broadcast_to(s, (N,)) if s.size == 1 else s
 
 
-def linear_forward(X, W, A=None, B=None, Wr=None, alpha=1.0, beta=1.0, S=None, lam=None):
+def linear_forward(X, W, A=None, B=None, Wr=None, alpha=1.0, beta=1.0, S=None, lam=None, hp_int8=None):
     """Forward of the decoupled linear layer.
 
     Y[t,n] = alpha_n * g_t * z_t[n] + beta_n * (lam/gamma_t) * acc[t,n]   (Eq. 10, 11)
     rounded once to bf16.  A/B None -> pure 1-bit layer (the MHA form).
     S/lam may be given instead of W (decode path from stored bits).
+    hp_int8: None -> bf16 HP branch on the un-quantised input; True -> the paper's INT8 branch, A and B
+    quantised here (quantize_experts); a tuple (A8, gA, B8, gB) -> the INT8 branch on stored int8 experts.
     Returns a dict with every intermediate.
     """
     out = {}
@@ -273,7 +340,13 @@ def linear_forward(X, W, A=None, B=None, Wr=None, alpha=1.0, beta=1.0, S=None, l
     if A is not None and A.shape[1] > 0:
         E = A.shape[0]
         rt = router(X, Wr if E > 1 else None)
-        h, z = hp_branch(X, A, B, rt["idx"])
+        if hp_int8 is None:
+            h, z = hp_branch(X, A, B, rt["idx"])
+        else:
+            A8, gA, B8, gB = quantize_experts(A, B) if hp_int8 is True else hp_int8
+            hp = hp_branch_int8(q, gamma, A8, gA, B8, gB, rt["idx"])
+            h, z = hp["h_int"] / (gA.astype(np.float64)[rt["idx"]] * gamma.astype(np.float64))[:, None], hp["z"]
+            out.update(A8=A8, gA=gA, B8=B8, gB=gB, h_int=hp["h_int"], qh=hp["qh"], gamma_h=hp["gamma_h"], z_int=hp["z_int"])
         perm, offsets = permutation(rt["idx"], E)
         out.update(h=h, z=z, perm=perm, offsets=offsets, **rt)
         y64 = al[None, :] * rt["gate"][:, None] * z + be[None, :] * y1
@@ -367,11 +440,11 @@ def rmsnorm(X, weight, eps):
     return round_to_bf16(y.astype(np.float64)).astype(np.float32)
 
 
-def decode_forward(X, bits, lam, A=None, B=None, Wr=None, alpha=1.0, beta=1.0, norm_weight=None, norm_eps=1e-6):
+def decode_forward(X, bits, lam, A=None, B=None, Wr=None, alpha=1.0, beta=1.0, norm_weight=None, norm_eps=1e-6, hp_int8=None):
     """Inference path (App. A): same forward, with S read back out of the
     packed 1-bit words instead of the latent weights; with `norm_weight` the
     input is the un-normalised activation and RMSNorm comes first."""
     if norm_weight is not None:
         X = rmsnorm(X, norm_weight, norm_eps)
     K = np.asarray(X).shape[1]
-    return linear_forward(X, None, A, B, Wr, alpha, beta, S=unpack_bits(bits, K), lam=lam)
+    return linear_forward(X, None, A, B, Wr, alpha, beta, S=unpack_bits(bits, K), lam=lam, hp_int8=hp_int8)

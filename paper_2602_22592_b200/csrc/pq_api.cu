@@ -329,6 +329,19 @@ int pq_pack_weights(const pq_desc* d, const float* W, uint32_t* w_bits, int8_t* 
   return e == cudaSuccess ? PQ_OK : PQ_ERR_CUDA;
 }
 
+int pq_pack_experts(const pq_desc* d, const uint16_t* A, const uint16_t* B, int8_t* A8, int8_t* B8, float* hp_scales, void* ws,
+                    size_t ws_bytes, void* stream) {
+  if (!d || !A || !B || !A8 || !B8 || !hp_scales || !ws) return PQ_ERR_NULL;
+  int rc = check_desc(d, false);
+  if (rc) return rc;
+  if (d->r <= 0) return PQ_ERR_SHAPE;
+  if (misaligned(A) || misaligned(B) || misaligned(A8) || misaligned(B8) || misaligned(ws)) return PQ_ERR_ALIGN;
+  if (ws_bytes < pq_workspace_bytes(d, PQ_PHASE_PACK)) return PQ_ERR_WORKSPACE;
+  cudaError_t e = launch_pack_experts(A, B, experts_of(d), d->r, d->K, d->N, A8, B8, hp_scales, static_cast<uint32_t*>(ws),
+                                      static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? PQ_OK : PQ_ERR_CUDA;
+}
+
 int pq_pack_weights_static(const pq_desc* d, const float* W, uint32_t* w_bits, int8_t* w_s8, float* w_scales, void* stream) {
   if (!d || !W || !w_bits || !w_scales) return PQ_ERR_NULL;
   if (d->size != sizeof(pq_desc) || d->N < 1 || d->K < 32 || d->K % 32) return PQ_ERR_SHAPE;

@@ -356,7 +356,7 @@ constexpr int kDecodeMetaBytes = 256;   // token info at the start of a slot
 // Experts used by the tokens [8 G, 8 G + 8) as a bit mask; producer and consumers walk it in ascending order.
 __device__ __forceinline__ unsigned decode_expert_mask(const DecodeTokInfo* tok, int M, int G) {
   unsigned mask = 0u;
-  for (int t = 8 * G; t < min(M, 8 * G + 8); ++t) mask |= 1u << tok[t].expert;
+  for (int t = 8 * G; t < min(M, 8 * G + 8); ++t) mask |= 1u << (tok[t].expert & 15);
   return mask;
 }
 
@@ -422,6 +422,7 @@ __global__ void __launch_bounds__(kDecodeMainThreads) k_decode_main(const __grid
     mbar_expect_tx(info_full, (uint32_t)bp.n * kDecodeMetaBytes);
     for (int l = 0; l < bp.n; ++l) bulk_load(smem_u32(smem + l * kDecodeMetaBytes), bp.lin[l].info, kDecodeMetaBytes, info_full);
     decode_wait(info_full, 0, fail);
+    if (*fail) return;                                       // nothing below may be issued from data that never arrived
     DecodeCursor cs, cq, cr;
     for (int l = 0; l < bp.n; ++l) {
       const DecodeLinear& L = bp.lin[l];
@@ -436,6 +437,7 @@ __global__ void __launch_bounds__(kDecodeMainThreads) k_decode_main(const __grid
           --early;                                          // bits already on their way
         } else {
           decode_wait(slot_empty(cs.idx), cs.phase ^ 1u, fail);
+          if (*fail) return;
           mbar_expect_tx(slot_full(cs.idx), bits_bytes + h_bytes);
           bulk_load(smem_u32(slot_ptr(cs.idx)), L.bits + (long long)n_lo * (L.K >> 5), bits_bytes, slot_full(cs.idx));
         }
@@ -448,6 +450,7 @@ __global__ void __launch_bounds__(kDecodeMainThreads) k_decode_main(const __grid
       for (int G = 0; G < ngroups; ++G) {
         const uint32_t q_bytes = (uint32_t)(npairs * min(8, L.M - 8 * G)) * 64u;
         decode_wait(q_empty(cq.idx), cq.phase ^ 1u, fail);
+        if (*fail) return;
         mbar_expect_tx(q_full(cq.idx), q_bytes);
         bulk_load(smem_u32(q_s) + cq.idx * bp.q_bytes, L.qfrag + (long long)G * npairs * 32, q_bytes, q_full(cq.idx));
         cq.next(bp.nq);
@@ -455,6 +458,7 @@ __global__ void __launch_bounds__(kDecodeMainThreads) k_decode_main(const __grid
         for (; emask; emask &= emask - 1) {
           const int e = __ffs(emask) - 1;
           decode_wait(ring_empty(cr.idx), cr.phase ^ 1u, fail);
+          if (*fail || e >= L.E) return;
           mbar_expect_tx(ring_full(cr.idx), (uint32_t)ncols * row_bytes);
           bulk_load(smem_u32(ring + cr.idx * bp.ring_stage_bytes), L.B + ((long long)e * L.N + n_lo) * L.r,
                     (uint32_t)ncols * row_bytes, ring_full(cr.idx));

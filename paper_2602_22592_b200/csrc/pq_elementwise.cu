@@ -560,6 +560,77 @@ __global__ void __launch_bounds__(1024) k_sum_scales(const float* __restrict__ v
   }
 }
 
+// ---------------------------------------------------------------------------
+// INT8 high-precision branch (Sec. 3.2): the expert matrices quantised the way the 8-bit activations are
+// (Eq. 7-9 with one scale per matrix): gamma = 128 / max(amax, 1e-5), code = clamp(rint(w * gamma), -128, 127).
+// Matrix id = 2 e + (0: A_e [r,K], 1: B_e [N,r]); grid (blocks, 2 E).
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) k_expert_amax(const uint4* __restrict__ A, const uint4* __restrict__ B, long long nA, long long nB,
+                                                     uint32_t* amax_bits) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int mat = blockIdx.y, e = mat >> 1;
+  const long long n = (mat & 1) ? nB : nA;                      // 16-byte pieces (8 values) of one matrix
+  const uint4* src = ((mat & 1) ? B : A) + (long long)e * n;
+  float amax = 0.f;
+  for (long long i = blockIdx.x * 256LL + threadIdx.x; i < n; i += gridDim.x * 256LL) {
+    const uint4 v = __ldg(src + i);
+    amax = fmaxf(amax, fmaxf(fmaxf(fabsf(bf16lo(v.x)), fabsf(bf16hi(v.x))), fmaxf(fabsf(bf16lo(v.y)), fabsf(bf16hi(v.y)))));
+    amax = fmaxf(amax, fmaxf(fmaxf(fabsf(bf16lo(v.z)), fabsf(bf16hi(v.z))), fmaxf(fabsf(bf16lo(v.w)), fabsf(bf16hi(v.w)))));
+  }
+  for (int d = 16; d > 0; d >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, d));
+  // non-negative floats order like their bit patterns; the maximum does not depend on the order of the updates
+  if ((threadIdx.x & 31) == 0) atomicMax(amax_bits + mat, __float_as_uint(amax));
+}
+
+__global__ void __launch_bounds__(256) k_expert_quant(const uint4* __restrict__ A, const uint4* __restrict__ B, long long nA, long long nB,
+                                                      const uint32_t* amax_bits, uint2* __restrict__ A8, uint2* __restrict__ B8,
+                                                      float* __restrict__ hp_scales) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int mat = blockIdx.y, e = mat >> 1;
+  const long long n = (mat & 1) ? nB : nA;
+  const uint4* src = ((mat & 1) ? B : A) + (long long)e * n;
+  uint2* dst = ((mat & 1) ? B8 : A8) + (long long)e * n;
+  const float gamma = __fdiv_rn(kActQmax, fmaxf(__uint_as_float(__ldcg(amax_bits + mat)), kActAmaxFloor));
+  if (blockIdx.x == 0 && threadIdx.x == 0) hp_scales[mat] = gamma;
+  for (long long i = blockIdx.x * 256LL + threadIdx.x; i < n; i += gridDim.x * 256LL) {
+    const uint4 v = __ldg(src + i);
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    int qi[8];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      qi[2 * j] = max(-128, min(127, __float2int_rn(__fmul_rn(bf16lo(w[j]), gamma))));
+      qi[2 * j + 1] = max(-128, min(127, __float2int_rn(__fmul_rn(bf16hi(w[j]), gamma))));
+    }
+    uint2 o;
+    o.x = (qi[0] & 0xFF) | ((qi[1] & 0xFF) << 8) | ((qi[2] & 0xFF) << 16) | ((qi[3] & 0xFF) << 24);
+    o.y = (qi[4] & 0xFF) | ((qi[5] & 0xFF) << 8) | ((qi[6] & 0xFF) << 16) | ((qi[7] & 0xFF) << 24);
+    dst[i] = o;
+  }
+}
+
+cudaError_t launch_pack_experts(const uint16_t* A, const uint16_t* B, int E, int r, int K, int N, int8_t* A8, int8_t* B8, float* hp_scales,
+                                uint32_t* amax_bits, cudaStream_t st) {
+  const long long nA = (long long)r * K / 8, nB = (long long)N * r / 8;
+  if (cudaMemsetAsync(amax_bits, 0, sizeof(uint32_t) * 2 * E, st) != cudaSuccess) return cudaGetLastError();
+  long long g = ((nA > nB ? nA : nB) + 1023) / 1024;
+  const int gx = (int)(g < 1 ? 1 : (g > 296 ? 296 : g));
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)gx, (unsigned)(2 * E), 1); cfg.blockDim = dim3(256, 1, 1); cfg.stream = st;
+  cfg.attrs = attr; cfg.numAttrs = 0;     // the first kernel follows a memset: plain stream order
+  { LaunchScope ls(KID_PACK_SUMS, st);
+    cudaLaunchKernelEx(&cfg, k_expert_amax, reinterpret_cast<const uint4*>(A), reinterpret_cast<const uint4*>(B), nA, nB, amax_bits); }
+  cfg.numAttrs = 1;
+  { LaunchScope ls(KID_BINARIZE_PACK, st);
+    cudaLaunchKernelEx(&cfg, k_expert_quant, reinterpret_cast<const uint4*>(A), reinterpret_cast<const uint4*>(B), nA, nB,
+                       static_cast<const uint32_t*>(amax_bits), reinterpret_cast<uint2*>(A8), reinterpret_cast<uint2*>(B8), hp_scales); }
+  return cudaGetLastError();
+}
+
 __global__ void k_fill_zero(uint4* p, long long n16) {
   pdl_launch_dependents();   // launched with programmatic stream serialisation: see launch_pdl
   pdl_wait();

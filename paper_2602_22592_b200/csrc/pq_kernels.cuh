@@ -90,6 +90,8 @@ cudaError_t launch_scaled_b(const uint16_t* B, uint16_t* out, const float* alpha
 cudaError_t launch_finalize_scales(const float* dbeta_partial, int nslots, const float* dalpha_partial, int E, int N, const float* w_scales,
                                    int vec, float* dbeta, float* dalpha, float* tmp_b, float* tmp_a, cudaStream_t st);
 cudaError_t launch_fill_zero(void* p, size_t bytes, cudaStream_t st);
+cudaError_t launch_pack_experts(const uint16_t* A, const uint16_t* B, int E, int r, int K, int N, int8_t* A8, int8_t* B8, float* hp_scales,
+                                uint32_t* amax_bits, cudaStream_t st);
 
 // tensor-core launchers (pq_gemm_kernels.cu).  All return a PQ_* status.
 struct LayerArgs {

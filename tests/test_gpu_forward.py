@@ -265,3 +265,22 @@ def test_argument_errors_are_reported():
     with pytest.raises(pqb.PqError) as ei:
         pqb.pq_linear_forward(L.desc, L.X, L.w_bits, L.w_s8, L.w_scales, L.A, L.B, None, L.alpha, L.beta, L.Y, L.saved, small)
     assert ei.value.status == pqb.PQ_ERR_WORKSPACE
+
+
+# ------------------------------------------------------------------ INT8 high-precision branch: expert quantisation (Sec. 3.2)
+@pytest.mark.parametrize("E,r,K,N", [(1, 32, 512, 512), (8, 128, 2048, 1024), (3, 40, 2080, 992), (8, 160, 3200, 8640)])
+def test_pack_experts_bit_exact(E, r, K, N):
+    c = I.make_linear_case(8, K, N, r, E, seed=17, exact_quota=False, with_grad=False)
+    d = pqb.make_desc(8, K, N, r, E)
+    A = torch.from_numpy(c["A"]).cuda().to(torch.bfloat16)
+    B = torch.from_numpy(c["B"]).cuda().to(torch.bfloat16)
+    A8 = torch.zeros((E, r, K), dtype=torch.int8, device="cuda")
+    B8 = torch.zeros((E, N, r), dtype=torch.int8, device="cuda")
+    sc = torch.zeros((E, 2), dtype=torch.float32, device="cuda")
+    ws = torch.empty(pqb.pq_workspace_bytes(d, pqb.PQ_PHASE_PACK), dtype=torch.uint8, device="cuda")
+    for _ in range(2):          # twice in a row: the scratch of the first call must not leak into the second
+        pqb.pq_pack_experts(d, A, B, A8, B8, sc, ws)
+    torch.cuda.synchronize()
+    wA8, gA, wB8, gB = O.quantize_experts(c["A"], c["B"])
+    assert np.array_equal(sc.cpu().numpy()[:, 0], gA) and np.array_equal(sc.cpu().numpy()[:, 1], gB)
+    assert np.array_equal(A8.cpu().numpy(), wA8) and np.array_equal(B8.cpu().numpy(), wB8)

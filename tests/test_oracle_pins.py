@@ -435,3 +435,93 @@ def test_decode_with_fused_norm_is_norm_then_decode():
     assert np.array_equal(a["Y"], b["Y"]) and np.array_equal(a["q"], b["q"])
     c = O.decode_forward(X, bits, lam)
     assert not np.array_equal(a["q"], c["q"])
+
+
+# ---------------------------------------------------------------- INT8 high-precision branch (Sec. 3.2)
+@pytest.mark.parametrize("row", _golden("weight_quant"))
+def test_weight_absmax_quant_worked(row):
+    W = _mat(row[0])
+    q, g = O.absmax_quant_matrix(W)
+    assert g == np.float32(float(row[1].split()[1]))
+    assert np.array_equal(q, _mat(row[2].split(None, 1)[1]).astype(np.int8))
+
+
+@pytest.mark.parametrize("row", _golden("requant"))
+def test_requant_hidden_worked(row):
+    h = _mat(row[0]).astype(np.int64)
+    qh, g = O.requant_hidden(h)
+    assert g[0] == np.float32(float(row[1].split()[1]))       # 0.5, 1.5 -> 0, 2 (ties to even) in the second row: 3/8, 5/8 round to 0, 1
+    assert np.array_equal(qh[0], np.array([int(v) for v in row[2].split()[1:]]))
+
+
+def test_int8_expert_weights_range_and_error_bound():
+    c = _case(3, zipf=False)
+    A8, gA, B8, gB = O.quantize_experts(c["A"], c["B"])
+    for W, W8, g in [(c["A"][e], A8[e], gA[e]) for e in range(3)] + [(c["B"][e], B8[e], gB[e]) for e in range(3)]:
+        assert W8.dtype == np.int8 and W8.min() >= -128 and W8.max() <= 127
+        assert np.abs(W8.astype(int)).max() >= 127                                  # the largest weight takes the top code
+        assert abs(float(g) * float(np.abs(W).max()) - 128.0) < 1e-3
+        err = np.abs(W.astype(np.float64) - W8 / np.float64(g))
+        clipped = np.rint(W * g) > 127
+        assert np.all(err[~clipped] <= 0.5 / g * (1 + 1e-5)) and np.all(err[clipped] <= 1.0 / g * (1 + 1e-5))
+
+
+def test_int8_branch_bruteforce_and_scale():
+    # every integer of the branch by python loops on a tiny routed case, and the real value it stands for
+    T, K, N, r, E = 5, 16, 6, 4, 2
+    c = I.make_linear_case(T, K, N, r, E, seed=71, zipf=False)
+    c["Wr"] = I.bf16_values((c["Wr"] * 30).astype(np.float32))
+    f = O.linear_forward(c["X"], c["W"], c["A"], c["B"], c["Wr"], c["alpha"], c["beta"], hp_int8=True)
+    A8, gA, B8, gB = f["A8"], f["gA"], f["B8"], f["gB"]
+    assert len(set(f["idx"].tolist())) == 2
+    for t in range(T):
+        e = int(f["idx"][t])
+        h = [sum(int(A8[e, j, k]) * int(f["q"][t, k]) for k in range(K)) for j in range(r)]
+        assert h == f["h_int"][t].tolist()
+        amax = max(abs(v) for v in h)
+        gh = np.float32(128.0) / np.float32(amax)
+        assert gh == f["gamma_h"][t]
+        qh = [int(np.clip(np.rint(np.float32(v) * gh), -128, 127)) for v in h]
+        assert qh == f["qh"][t].tolist()
+        for n in range(N):
+            zi = sum(int(B8[e, n, j]) * qh[j] for j in range(r))
+            assert zi == f["z_int"][t, n]
+            real = zi / (float(gB[e]) * float(gh) * float(gA[e]) * float(f["gamma"][t]))
+            assert abs(real - f["z"][t, n]) <= 1e-12 * max(1.0, abs(real))
+            want = float(c["alpha"][0]) * f["gate"][t] * real + float(c["beta"][0]) * f["y1"][t, n]
+            assert abs(want - f["Y64"][t, n]) <= 1e-12 * max(1.0, abs(want))
+
+
+def test_int8_branch_within_quantiser_bound_of_the_fp_branch():
+    # Sec. 4.6 (the FP16 ablation behaves like the INT8 branch): the INT8 result stays within the error bound the three
+    # quantisers (activations, weights, hidden codes) allow around the un-quantised product B_e A_e x.
+    c = _case(3, seed=23, T=48, K=128, N=40, r=16, zipf=False)
+    f8 = O.linear_forward(c["X"], c["W"], c["A"], c["B"], c["Wr"], c["alpha"], c["beta"], hp_int8=True)
+    ff = O.linear_forward(c["X"], c["W"], c["A"], c["B"], c["Wr"], c["alpha"], c["beta"])
+    assert np.array_equal(f8["idx"], ff["idx"])
+    X = c["X"].astype(np.float64)
+    idx = ff["idx"]
+    gt = f8["gamma"].astype(np.float64)
+    bound = np.zeros_like(ff["z"])
+    for t in range(48):
+        e = idx[t]
+        A, B = c["A"][e].astype(np.float64), c["B"][e].astype(np.float64)
+        dx, dA, dB = 1.0 / gt[t], 1.0 / float(f8["gA"][e]), 1.0 / float(f8["gB"][e])
+        h_err = np.abs(A).sum(axis=1) * dx + dA * (np.abs(X[t]) + dx).sum() + 1.0 / (float(f8["gamma_h"][t]) * float(f8["gA"][e]) * gt[t])
+        bound[t] = np.abs(B) @ h_err + dB * (np.abs(ff["h"][t]) + h_err).sum()
+    err = np.abs(f8["z"] - ff["z"])
+    assert np.all(err <= bound)
+    assert np.sqrt(np.mean(err ** 2)) < 0.05 * np.sqrt(np.mean(ff["z"] ** 2))      # and in practice a few percent
+    # planted mistakes break it: the hidden scale left out, the token's own scale left out
+    wrong1 = f8["z_int"] / (f8["gB"].astype(np.float64)[idx] * f8["gA"].astype(np.float64)[idx] * gt)[:, None]
+    wrong2 = f8["z_int"] / (f8["gB"].astype(np.float64)[idx] * f8["gA"].astype(np.float64)[idx] * f8["gamma_h"].astype(np.float64))[:, None]
+    for wrong in (wrong1, wrong2):
+        assert not np.all(np.abs(wrong - ff["z"]) <= bound)
+
+
+def test_int8_branch_decode_uses_stored_codes():
+    c = _case(2, seed=56, T=4, K=64, N=32, r=8, with_grad=False)
+    f = O.linear_forward(c["X"], c["W"], c["A"], c["B"], c["Wr"], c["alpha"], c["beta"], hp_int8=True)
+    stored = (f["A8"], f["gA"], f["B8"], f["gB"])
+    d = O.decode_forward(c["X"], O.pack_bits(f["S"]), f["lam"], c["A"] * 0, c["B"] * 0, c["Wr"], c["alpha"], c["beta"], hp_int8=stored)
+    assert np.array_equal(d["Y"], f["Y"]) and np.array_equal(d["z_int"], f["z_int"])
