@@ -183,6 +183,19 @@ int pq_linear_forward(const pq_desc* d, const uint16_t* X, const uint32_t* w_bit
                       const float* beta, uint16_t* Y, void* saved, size_t saved_bytes, void* ws,
                       size_t ws_bytes, void* stream);
 
+/* Forward with the paper's INT8 high-precision branch (Sec. 3.2), training-size path (tensor cores), forward only:
+ * the branch multiplies the SAME int8 activation codes q the 1-bit branch uses,
+ *     h_int = A8_e q_t (int32, exact);   qh, gamma_h = Eq. 7-9 on h_int (gamma_h = 2^7 / max_j |h_int|, from the integers);
+ *     z_int = B8_e qh_t (int32, exact);  z = z_int / (gamma_B gamma_h gamma_A gamma_t);
+ *     Y = alpha g z + beta (lam / gamma_t) acc                                    (Eq. 10-11)
+ * with A8, B8, hp_scales from pq_pack_experts.  Arguments as pq_linear_forward; r must be a multiple of 16
+ * (PQ_ERR_SHAPE otherwise), r <= 128.  With `saved` given, its h region holds the codes qh as int8
+ * [max_items*128, r] followed (256-byte aligned) by gamma_h as float [max_items*128], rows per item as for h.
+ * There is no INT8 backward: pq_linear_backward on a buffer saved by this call is not defined. */
+int pq_linear_forward_hp8(const pq_desc* d, const uint16_t* X, const int8_t* w_s8, const float* w_scales, const int8_t* A8,
+                          const int8_t* B8, const float* hp_scales, const uint16_t* Wr, const float* alpha, const float* beta,
+                          uint16_t* Y, void* saved, size_t saved_bytes, void* ws, size_t ws_bytes, void* stream);
+
 /* What the decode path leaves in its workspace, for tests and diagnostics.  One entry per
  * token: the routed expert, its gate g_t, gamma_t (Eq. 9) and the sum over k of the int8 codes. */
 typedef struct pq_decode_token {

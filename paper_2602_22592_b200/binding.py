@@ -22,7 +22,7 @@ PQ_DECODE_DUMP_ACC = 2
 PQ_PHASE_PACK, PQ_PHASE_FWD, PQ_PHASE_BWD, PQ_PHASE_DECODE = 0, 1, 2, 3
 
 EXPORTS = ("pq_status_string", "pq_workspace_bytes", "pq_saved_bytes", "pq_saved_view_init",
-           "pq_decode_view_init", "pq_bwd_view_init", "pq_decode_batch", "pq_pack_weights", "pq_pack_weights_static", "pq_pack_experts", "pq_linear_forward", "pq_linear_backward", "pq_debug_gemm", "pq_debug_gemm_tile",
+           "pq_decode_view_init", "pq_bwd_view_init", "pq_decode_batch", "pq_pack_weights", "pq_pack_weights_static", "pq_pack_experts", "pq_linear_forward", "pq_linear_forward_hp8", "pq_linear_backward", "pq_debug_gemm", "pq_debug_gemm_tile",
            "pq_device_status", "pq_kernel_launches", "pq_profile_events", "pq_set_option")
 
 KERNEL_IDS = dict(pack_sums=0, binarize_pack=1, router=2, route_scan=3, act_quant=4, hp_up=5, fwd=6, scatter_rows=7,
@@ -96,6 +96,8 @@ def lib() -> ctypes.CDLL:
         L.pq_pack_experts.argtypes = [dp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.pq_linear_forward.restype = ci
         L.pq_linear_forward.argtypes = [dp] + [vp] * 10 + [vp, sz, vp, sz, vp]
+        L.pq_linear_forward_hp8.restype = ci
+        L.pq_linear_forward_hp8.argtypes = [dp] + [vp] * 10 + [vp, sz, vp, sz, vp]
         L.pq_linear_backward.restype = ci
         L.pq_linear_backward.argtypes = [dp] + [vp] * 9 + [vp, sz] + [vp] * 7 + [vp, sz, vp]
         L.pq_debug_gemm.restype = ci
@@ -223,6 +225,13 @@ def pq_pack_experts(d, A, B, A8, B8, hp_scales, ws, stream=None):
 def pq_linear_forward(d, X, w_bits, w_s8, w_scales, A, B, Wr, alpha, beta, Y, saved, ws, stream=None):
     _check("pq_linear_forward", lib().pq_linear_forward(
         ctypes.byref(d), _ptr(X), _ptr(w_bits), _ptr(w_s8), _ptr(w_scales), _ptr(A), _ptr(B), _ptr(Wr), _ptr(alpha),
+        _ptr(beta), _ptr(Y), _ptr(saved), _nbytes(saved), _ptr(ws), _nbytes(ws), _stream(stream)))
+
+
+def pq_linear_forward_hp8(d, X, w_s8, w_scales, A8, B8, hp_scales, Wr, alpha, beta, Y, saved, ws, stream=None):
+    """Forward with the INT8 high-precision branch (Sec. 3.2); A8, B8, hp_scales come from pq_pack_experts."""
+    _check("pq_linear_forward_hp8", lib().pq_linear_forward_hp8(
+        ctypes.byref(d), _ptr(X), _ptr(w_s8), _ptr(w_scales), _ptr(A8), _ptr(B8), _ptr(hp_scales), _ptr(Wr), _ptr(alpha),
         _ptr(beta), _ptr(Y), _ptr(saved), _nbytes(saved), _ptr(ws), _nbytes(ws), _stream(stream)))
 
 

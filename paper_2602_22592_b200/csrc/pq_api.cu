@@ -363,11 +363,13 @@ static int check_decode_item(const pq_desc* d, const uint16_t* X, const uint32_t
   return PQ_OK;
 }
 
-int pq_linear_forward(const pq_desc* d, const uint16_t* X, const uint32_t* w_bits, const int8_t* w_s8, const float* w_scales,
-                      const uint16_t* A, const uint16_t* B, const uint16_t* Wr, const float* alpha, const float* beta, uint16_t* Y,
-                      void* saved, size_t saved_bytes, void* ws, size_t ws_bytes, void* stream) {
+// hp_scales != nullptr: INT8 HP branch, A and B are int8 codes (training path only)
+static int forward_impl(const pq_desc* d, const uint16_t* X, const uint32_t* w_bits, const int8_t* w_s8, const float* w_scales,
+                        const uint16_t* A, const uint16_t* B, const float* hp_scales, const uint16_t* Wr, const float* alpha, const float* beta,
+                        uint16_t* Y, void* saved, size_t saved_bytes, void* ws, size_t ws_bytes, void* stream) {
   if (!d || !X || !w_scales || !beta || !Y) return PQ_ERR_NULL;
   if (!w_s8) {
+    if (hp_scales) return PQ_ERR_UNSUPPORTED;
     // decode: a few tokens straight from the packed sign bits
     int rc = check_decode_item(d, X, w_bits, w_scales, A, B, Wr, alpha, beta, Y, ws, ws_bytes);
     if (rc) return rc;
@@ -397,13 +399,32 @@ int pq_linear_forward(const pq_desc* d, const uint16_t* X, const uint32_t* w_bit
   if (ws_bytes < used) return PQ_ERR_WORKSPACE;
   const int E = experts_of(d);
   LayerArgs a{d->T, d->K, d->N, d->r, E, (d->flags & PQ_SCALE_VECTOR) ? 1 : 0, w_scales, alpha, beta, A, B, Wr};
-  // dense layer with an HP branch: the quantisation runs on the helper stream next to scan -> up-projection
-  SideCtx* side = (d->r > 0 && !routed(d)) ? side_for(st) : nullptr;
+  if (hp_scales) {
+    if (d->r <= 0 || d->r % 16) return PQ_ERR_SHAPE;       // int8 rows of r bytes must be 16-byte multiples for TMA
+    a.hp_scales = hp_scales;
+  }
+  // dense layer with a bf16 HP branch: the quantisation runs on the helper stream next to scan -> up-projection
+  // (the INT8 branch multiplies the codes themselves, so its up-projection follows the quantisation)
+  SideCtx* side = (d->r > 0 && !routed(d) && !hp_scales) ? side_for(st) : nullptr;
   if (side && !side_fork(side, st)) return PQ_ERR_CUDA;
   if (launch_route_and_quant(X, Wr, d->T, d->K, routed(d) ? E : 1, sv, sc, st, side ? side->side : st) != cudaSuccess) return PQ_ERR_CUDA;
   if (side && cudaEventRecord(side->join, side->side) != cudaSuccess) return PQ_ERR_CUDA;
   const uint16_t* xs = routed(d) ? sv.xs : X;
   return gemm_forward(a, w_s8, sv, xs, Y, st, side ? side->join : nullptr);
+}
+
+int pq_linear_forward(const pq_desc* d, const uint16_t* X, const uint32_t* w_bits, const int8_t* w_s8, const float* w_scales,
+                      const uint16_t* A, const uint16_t* B, const uint16_t* Wr, const float* alpha, const float* beta, uint16_t* Y,
+                      void* saved, size_t saved_bytes, void* ws, size_t ws_bytes, void* stream) {
+  return forward_impl(d, X, w_bits, w_s8, w_scales, A, B, nullptr, Wr, alpha, beta, Y, saved, saved_bytes, ws, ws_bytes, stream);
+}
+
+int pq_linear_forward_hp8(const pq_desc* d, const uint16_t* X, const int8_t* w_s8, const float* w_scales, const int8_t* A8, const int8_t* B8,
+                          const float* hp_scales, const uint16_t* Wr, const float* alpha, const float* beta, uint16_t* Y, void* saved,
+                          size_t saved_bytes, void* ws, size_t ws_bytes, void* stream) {
+  if (!w_s8 || !A8 || !B8 || !hp_scales) return PQ_ERR_NULL;
+  return forward_impl(d, X, nullptr, w_s8, w_scales, reinterpret_cast<const uint16_t*>(A8), reinterpret_cast<const uint16_t*>(B8), hp_scales, Wr,
+                      alpha, beta, Y, saved, saved_bytes, ws, ws_bytes, stream);
 }
 
 int pq_decode_batch(const pq_decode_item* items, int n, void* stream) {

@@ -69,6 +69,15 @@ static bool map3d(CUtensorMap* m, const void* base, uint64_t inner, uint64_t mid
   return make_map(m, false, base, 3, dims, strides, box);
 }
 
+// int8 [outer][mid][inner] with the contraction index innermost: boxes of 128 bytes x box_mid rows of one batch entry;
+// `pitch` is the row stride in bytes (a multiple of 16, at least `inner`)
+static bool map3d_i8(CUtensorMap* m, const void* base, uint64_t inner, uint64_t pitch, uint64_t mid, uint64_t outer, uint32_t box_mid) {
+  const uint64_t dims[3] = {inner, mid, outer};
+  const uint64_t strides[2] = {pitch, pitch * mid};
+  const uint32_t box[3] = {128, box_mid, 1};
+  return make_map(m, true, base, 3, dims, strides, box);
+}
+
 // MN-major operand: matrix [batch][k_total][mn_total] with mn contiguous, read in 64 (mn) x 64 (k) boxes.
 // When mn_total is a multiple of 64 the map views the 64-wide column blocks as a dimension of their own,
 // (64, k_total, mn_total / 64[, batch]) -- base_rank 2 or 3 says whether the operand has the batch dimension --, so that ONE load delivers `nblk` boxes back to back; *blk = nblk.
@@ -260,6 +269,74 @@ struct HpUpProblem {
 PQ_DEFINE_GEMM_KERNEL(k_gemm_hp_up, HpUpProblem)
 
 // ---------------------------------------------------------------------------
+// F1 in INT8 (Sec. 3.2): h_int = q_sorted A8_e^T, exact in int32, one tile per item; the epilogue quantises each
+// row of h per token the way activations are (Eq. 7-9, taken from the integers: gamma_h = 128 / max |h_int|) and
+// writes the codes qh [items*128, rp] (row pitch rp = r rounded up to 16, padding zero) and gamma_h [items*128].
+// ---------------------------------------------------------------------------
+struct HpUp8Problem {
+  using Acc = AccDouble;
+  struct Params {
+    CUtensorMap tq, ta;  // q sorted [T,K] s8; A8 [E,r,K] s8
+    RoutingTables rt;
+    int8_t* qh;
+    float* gamma_h;
+    int K, r, rp, bn;
+  };
+  struct Tile { int item; int4 it; };
+  __device__ static int stage_cols(const Params& p) { return p.bn <= 128 ? 128 : 256; }
+  __device__ static int num_tiles(const Params& p) { return p.rt.n_items[0]; }
+  __device__ static void tile_init(const Params& p, int i, Tile& t) { t.item = i; t.it = p.rt.items[i]; }
+  __device__ static int num_segments(const Params&, const Tile&) { return 1; }
+  __device__ static void segment(const Params& p, const Tile& t, int, Segment& s) {
+    s.mode = MODE_I8_KK; s.acc = 0; s.bn = p.bn; s.ksteps = 4; s.nkb = (p.K + 127) / 128;
+    s.ta = &p.tq; s.a_rank = 2; s.a_x = 0; s.a_y = t.it.x * 128; s.a_z = 0;
+    s.tb = &p.ta; s.b_rank = 3; s.b_x = 0; s.b_y = 0; s.b_z = t.it.y;
+    s.b_box = p.bn; s.a_blk = 0; s.b_blk = 0;
+  }
+  using Pre = NoPre;
+  __device__ static Pre prepare(const Params&, const Tile&, int, int) { return Pre{}; }
+  __device__ static void epilogue(const Params& p, const Tile& t, const Pre& pre, uint32_t taddr, uint32_t, int quad, int half, int lane, uint8_t* stage) {
+    if (half) return;   // the maximum over a row's r columns stays in one thread
+    const int row = quad * 32 + lane;
+    const bool live = row >= t.it.z && row < t.it.w;
+    int amax = 0;
+    for (int c = 0; c * 32 < p.r; ++c) {
+      uint32_t v[32];
+      tmem_ld32(taddr + c * 32, v);
+      tmem_ld_wait();
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (c * 32 + j < p.r) amax = max(amax, abs((int)v[j]));
+    }
+    const float gamma_h = __fdiv_rn(kActQmax, fmaxf(__int2float_rn(amax), kActAmaxFloor));
+    const long long grow = (long long)t.item * 128 + row;
+    p.gamma_h[grow] = live ? gamma_h : 0.f;
+    uint4* out = reinterpret_cast<uint4*>(p.qh + grow * p.rp);
+    for (int c = 0; c * 32 < p.rp; ++c) {
+      uint32_t v[32];
+      tmem_ld32(taddr + c * 32, v);
+      tmem_ld_wait();
+      uint32_t w[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        uint32_t word = 0u;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+          const int col = c * 32 + 4 * j + b;
+          int code = 0;
+          if (live && col < p.r) code = max(-128, min(127, __float2int_rn(__fmul_rn(__int2float_rn((int)v[4 * j + b]), gamma_h))));
+          word |= (uint32_t)(code & 0xFF) << (8 * b);
+        }
+        w[j] = word;
+      }
+      if (c * 32 < p.rp) out[2 * c] = make_uint4(w[0], w[1], w[2], w[3]);
+      if (c * 32 + 16 < p.rp) out[2 * c + 1] = make_uint4(w[4], w[5], w[6], w[7]);
+    }
+  }
+};
+PQ_DEFINE_GEMM_KERNEL(k_gemm_hp_up8, HpUp8Problem)
+
+// ---------------------------------------------------------------------------
 // F2: fused output tile.  Accumulator 0 (int32): q S^T over K.  Accumulator 1
 // (fp32): H B_e^T over r, once per item of the tile (masked H rows are zero).
 // Epilogue: Y[token, n] = alpha_n g z + beta_n (lam / gamma) acc, rounded once.
@@ -279,6 +356,10 @@ struct FwdProblem {
     const float* alpha;
     const float* beta;
     uint16_t* Y;
+    // INT8 HP branch (Sec. 3.2): th / tb then map the int8 codes of h and of B_e, the second accumulator is int32, and
+    // its de-quantisation factor 1 / (gamma_B gamma_h gamma_A gamma_t) is folded into the row's HP factor
+    const float* gamma_h;    // [items*128], null for the bf16 branch
+    const float* hp_scales;  // [E][2] = {gamma_A, gamma_B}
     int T, N, K, r, sstride, item_rows;
   };
   struct Tile { TileCoord c; int bn, ib, ie; };
@@ -300,15 +381,16 @@ struct FwdProblem {
     } else {
       const int item = t.ib + (i - 1);
       const int e = p.rt.items[item].y;
-      s.mode = MODE_BF_KK; s.acc = 1; s.nkb = (p.r + 63) / 64;
-      s.ta = &p.th; s.a_rank = 2; s.a_x = 0; s.a_y = item * 128;
+      if (p.gamma_h) { s.mode = MODE_I8_KK; s.acc = 1; s.nkb = (p.r + 127) / 128; }
+      else { s.mode = MODE_BF_KK; s.acc = 1; s.nkb = (p.r + 63) / 64; }
+      s.ta = &p.th; s.a_rank = p.gamma_h ? 3 : 2; s.a_x = 0; s.a_y = item * 128;
       s.tb = &p.tb; s.b_rank = 3; s.b_x = 0; s.b_y = t.c.n0; s.b_z = e;
     }
   }
   // y = cb_n * acc + ca_n * z for 32 consecutive columns starting at n, packed to 16 bf16 pairs
   template <bool VEC>
   __device__ static __forceinline__ void combine32(const Params& p, int n, float cb, float ca, const uint32_t (&a)[32], const uint32_t (&z)[32],
-                                                  uint4* out) {
+                                                  uint4* out, bool z_is_int) {
     uint32_t w[16];
 #pragma unroll
     for (int q4 = 0; q4 < 8; ++q4) {
@@ -325,7 +407,7 @@ struct FwdProblem {
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         y[u] = b4[u] * (float)(int)a[4 * q4 + u];
-        if (HP) y[u] = fmaf(a4[u], __uint_as_float(z[4 * q4 + u]), y[u]);
+        if (HP) y[u] = fmaf(a4[u], z_is_int ? (float)(int)z[4 * q4 + u] : __uint_as_float(z[4 * q4 + u]), y[u]);
       }
       w[2 * q4] = pack_bf16x2(y[0], y[1]);
       w[2 * q4 + 1] = pack_bf16x2(y[2], y[3]);
@@ -343,6 +425,19 @@ struct FwdProblem {
       r.yrow = p.Y + (long long)token * p.N;
       r.cb = __fdiv_rn(p.w_scales[0], p.gamma[pos]);
       if (HP) r.ca = p.gate[pos];
+      if (HP && p.gamma_h) {
+        // the item of this row: its expert's weight scales and the row's own hidden scale
+        const int rel = quad * 32 + lane;
+        float deq = 0.f;
+        for (int it = t.ib; it < t.ie; ++it) {
+          const int4 d = p.rt.items[it];
+          if (rel >= d.z && rel < d.w) {
+            const float gh = p.gamma_h[(long long)it * 128 + rel];
+            deq = 1.0f / (p.hp_scales[2 * d.y + 1] * gh * p.hp_scales[2 * d.y] * p.gamma[pos]);
+          }
+        }
+        r.ca *= deq;
+      }
       if (!p.sstride) { r.cb *= p.beta[0]; if (HP) r.ca *= p.alpha[0]; }
     }
     return r;
@@ -361,8 +456,8 @@ struct FwdProblem {
           tmem_ld32(tacc + c * 64 + h * 32, a);
           if (HP) tmem_ld32(tz + c * 64 + h * 32, z);
           tmem_ld_wait();
-          if (vec) combine32<true>(p, nb, pre.cb, pre.ca, a, z, o + 4 * h);
-          else combine32<false>(p, nb, pre.cb, pre.ca, a, z, o + 4 * h);
+          if (vec) combine32<true>(p, nb, pre.cb, pre.ca, a, z, o + 4 * h, p.gamma_h != nullptr);
+          else combine32<false>(p, nb, pre.cb, pre.ca, a, z, o + 4 * h, p.gamma_h != nullptr);
         }
       }
       warp_store_rows(stage, o, pre.yrow ? pre.yrow + n0 : nullptr, min(64, min(t.bn - c * 64, p.N - n0)) * 2, lane);
@@ -372,6 +467,12 @@ struct FwdProblem {
 PQ_DEFINE_GEMM_KERNEL(k_gemm_fwd_hp, FwdProblem<true>)
 PQ_DEFINE_GEMM_KERNEL(k_gemm_fwd_1bit, FwdProblem<false>)
 
+// INT8 branch: the saved h region holds the codes qh [items*128, r] and, behind them, gamma_h [items*128]
+static inline float* hp8_gamma_h(const SavedPtrs& sv, int r) {
+  const size_t codes = ((size_t)sv.max_items * 128 * r + 255) / 256 * 256;
+  return reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(sv.h) + codes);
+}
+
 template <bool HP>
 static int fill_forward_params(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, uint16_t* Y, typename FwdProblem<HP>::Params& f) {
   using P = FwdProblem<HP>;
@@ -379,7 +480,14 @@ static int fill_forward_params(const LayerArgs& a, const int8_t* w_s8, const Sav
   if (!map2d(&f.tq, true, sv.q, a.K, a.T, 128, 128)) return PQ_ERR_CUDA;
   if (!map2d(&f.ts, true, w_s8, a.K, a.N, 128, 256)) return PQ_ERR_CUDA;
   f.th = f.tq; f.tb = f.tq;
-  if (HP) {
+  f.gamma_h = nullptr; f.hp_scales = a.hp_scales;
+  if (HP && a.hp_scales) {
+    // INT8 branch: codes of h [items*128, r] and of B_e [E, N, r], one byte per value
+    const uint64_t rows = (uint64_t)sv.max_items * 128;
+    if (!map3d_i8(&f.th, sv.h, a.r, a.r, rows, 1, 128)) return PQ_ERR_CUDA;
+    if (!map3d_i8(&f.tb, a.B, a.r, a.r, a.N, a.E, 256)) return PQ_ERR_CUDA;
+    f.gamma_h = hp8_gamma_h(sv, a.r);
+  } else if (HP) {
     if (!map2d(&f.th, false, sv.h, a.r, (uint64_t)sv.max_items * 256, 64, 128)) return PQ_ERR_CUDA;
     if (!map3d(&f.tb, a.B, a.r, a.N, a.E, 64, 256)) return PQ_ERR_CUDA;
   }
@@ -392,6 +500,20 @@ static int fill_forward_params(const LayerArgs& a, const int8_t* w_s8, const Sav
 
 int gemm_forward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, const uint16_t* xs, uint16_t* Y, cudaStream_t st,
                  cudaEvent_t before_main) {
+  if (a.r > 0 && a.hp_scales) {
+    HpUp8Problem::Params p;
+    p.rt = sv.rt; p.qh = reinterpret_cast<int8_t*>(sv.h); p.gamma_h = hp8_gamma_h(sv, a.r); p.K = a.K; p.r = a.r; p.rp = a.r;
+    p.bn = h_round_up(a.r, 16);
+    if (!map2d(&p.tq, true, sv.q, a.K, a.T, 128, 128)) return PQ_ERR_CUDA;
+    if (!map3d_i8(&p.ta, a.A, a.K, a.K, a.r, a.E, p.bn)) return PQ_ERR_CUDA;
+    int rc = launch_gemm(KID_HP_UP, k_gemm_hp_up8, p, sv.max_items, st);
+    if (rc) return rc;
+    FwdProblem<true>::Params f;
+    rc = fill_forward_params<true>(a, w_s8, sv, Y, f);
+    if (rc) return rc;
+    if (before_main && cudaStreamWaitEvent(st, before_main, 0) != cudaSuccess) return PQ_ERR_CUDA;
+    return launch_gemm(KID_FWD, k_gemm_fwd_hp, f, f.g.total, st);
+  }
   if (a.r > 0) {
     HpUpProblem::Params p;
     p.rt = sv.rt; p.H = sv.h; p.K = a.K; p.r = a.r; p.bn = h_round_up(a.r, 16); p.item_rows = sv.max_items * 128;

@@ -103,6 +103,7 @@ struct LayerArgs {
   const uint16_t* A;   // [E,r,K]
   const uint16_t* B;   // [E,N,r]
   const uint16_t* Wr;  // [E,K]
+  const float* hp_scales = nullptr;   // INT8 HP branch: [E][2] = {gamma_A, gamma_B}, and A, B then point to int8 codes
 };
 
 int gemm_debug(int mode, int M, int N, int K, const void* A, const void* B, void* D, int tile_n, cudaStream_t st);

@@ -138,6 +138,29 @@ class PQLinear:
                               self.Wr, self.alpha, self.beta, self.Y if Y is None else Y, self.saved, self.ws_fwd)
         return self.Y if Y is None else Y
 
+    def pack_experts(self):
+        """INT8 codes and scales of the expert matrices (Sec. 3.2), kept beside the bf16 originals."""
+        Ee = max(self.E, 1)
+        if getattr(self, "A8", None) is None:
+            self.A8 = self._buf((Ee, self.r, self.K), torch.int8)
+            self.B8 = self._buf((Ee, self.N, self.r), torch.int8)
+            self.hp_scales = self._buf((Ee, 2), torch.float32)
+        pqb.pq_pack_experts(self.desc, self.A, self.B, self.A8, self.B8, self.hp_scales, self.ws_pack)
+
+    def forward_hp8(self, X=None, Y=None):
+        """Forward with the INT8 high-precision branch (after pack() and pack_experts())."""
+        pqb.pq_linear_forward_hp8(self.desc, self.X if X is None else X, self.w_s8, self.w_scales, self.A8, self.B8, self.hp_scales,
+                                  self.Wr, self.alpha, self.beta, self.Y if Y is None else Y, self.saved, self.ws_fwd)
+        return self.Y if Y is None else Y
+
+    def hp8_view(self) -> dict:
+        """What forward_hp8 left in the saved h region: codes qh int8 [max_items*128, r] and gamma_h float [max_items*128]."""
+        sv = self.saved_view()
+        rows = sv["max_items"] * 128
+        raw = sv["h"].view(torch.uint8).reshape(-1)
+        codes = (rows * self.r + 255) // 256 * 256
+        return dict(qh=raw[:rows * self.r].view(torch.int8).view(rows, self.r), gamma_h=raw[codes:codes + 4 * rows].view(torch.float32))
+
     def backward(self, dY=None):
         pqb.pq_linear_backward(self.desc, self.dY if dY is None else dY, self.X, self.w_s8, self.w_scales, self.A, self.B,
                                self.Wr, self.alpha, self.beta, self.saved, self.dX, self.dW, self.dA, self.dB, self.dWr,

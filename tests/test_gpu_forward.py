@@ -284,3 +284,65 @@ def test_pack_experts_bit_exact(E, r, K, N):
     wA8, gA, wB8, gB = O.quantize_experts(c["A"], c["B"])
     assert np.array_equal(sc.cpu().numpy()[:, 0], gA) and np.array_equal(sc.cpu().numpy()[:, 1], gB)
     assert np.array_equal(A8.cpu().numpy(), wA8) and np.array_equal(B8.cpu().numpy(), wB8)
+
+
+HP8_CASES = {
+    "dense_r32": dict(T=333, K=384, N=544, r=32, E=1),
+    "routed8_r128": dict(T=1000, K=512, N=768, r=128, E=8),
+    "routed4_r16_vec": dict(T=520, K=256, N=256, r=16, E=4, scale_vector=True, alpha=1.5, beta=0.4),
+    "routed3_r48_long_rows": dict(T=200, K=4096, N=96, r=48, E=3),
+}
+
+
+@pytest.mark.parametrize("name", list(HP8_CASES))
+def test_forward_int8_hp_branch_matches_oracle(name):
+    # Sec. 3.2: the HP branch at 8-bit precision on the int8 activation codes.  Integers (codes of h and their scale,
+    # hence the exact int32 sums behind them) bit for bit; Y within the bf16 tolerance of the oracle's INT8 forward.
+    kw = dict(HP8_CASES[name])
+    sv = kw.pop("scale_vector", False)
+    c = I.make_linear_case(kw.pop("T"), kw.pop("K"), kw.pop("N"), kw.pop("r"), kw.pop("E"), seed=19, scale_vector=sv, **kw)
+    if sv:
+        c["alpha"] = (c["alpha"] * np.linspace(0.8, 1.2, c["N"])).astype(np.float32)
+        c["beta"] = (c["beta"] * np.linspace(1.2, 0.8, c["N"])).astype(np.float32)
+    f = O.linear_forward(c["X"], c["W"], c["A"], c["B"], c["Wr"], c["alpha"], c["beta"], hp_int8=True)
+    L = PQLinear(c["T"], c["K"], c["N"], c["r"], c["E"], scale_vector=sv, guard=True).load_case(c)
+    L.pack()
+    L.pack_experts()
+    L.forward_hp8()
+    torch.cuda.synchronize()
+    check_status()
+    assert L.check_guards() == 0
+    assert np.array_equal(L.A8.cpu().numpy(), f["A8"]) and np.array_equal(L.B8.cpu().numpy(), f["B8"])
+    svw = L.saved_view()
+    perm = svw["perm"].cpu().numpy()
+    assert np.array_equal(svw["q"].cpu().numpy(), f["q"][perm])
+    if c["E"] > 1:
+        assert np.array_equal(svw["expert"].cpu().numpy(), f["idx"])
+    h8 = L.hp8_view()
+    qh, gh = h8["qh"].cpu().numpy(), h8["gamma_h"].cpu().numpy()
+    items = svw["items"].cpu().numpy()[:int(svw["n_items"].cpu()[0])]
+    seen = 0
+    for i, (tile, e, lo, hi) in enumerate(items):
+        rows = np.arange(tile * 128 + lo, tile * 128 + hi)
+        tokens = perm[rows]
+        assert np.array_equal(qh[i * 128 + lo:i * 128 + hi], f["qh"][tokens])         # codes of h: exact int32 sums behind them
+        assert np.array_equal(gh[i * 128 + lo:i * 128 + hi], f["gamma_h"][tokens])
+        assert not np.any(qh[i * 128:i * 128 + lo]) and not np.any(qh[i * 128 + hi:(i + 1) * 128])
+        seen += len(rows)
+    assert seen == c["T"]
+    assert rel_err(f32(L.Y), f["Y"]) <= TOL_BF16
+    assert rms_err(f32(L.Y), f["Y"]) <= TOL_RMS
+    # and it is the INT8 branch, not the bf16 one
+    fb = O.linear_forward(c["X"], c["W"], c["A"], c["B"], c["Wr"], c["alpha"], c["beta"])
+    assert rms_err(f["Y"], fb["Y"]) > 2e-3
+
+
+def test_forward_int8_hp_rejects_odd_width():
+    L = PQLinear(128, 64, 64, 40, 1)
+    c = I.make_linear_case(128, 64, 64, 40, 1, seed=1)
+    L.load_case(c)
+    L.pack()
+    L.pack_experts()
+    with pytest.raises(pqb.PqError) as ei:
+        L.forward_hp8()
+    assert ei.value.status == pqb.PQ_ERR_SHAPE
