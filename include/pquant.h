@@ -314,7 +314,7 @@ long long pq_kernel_launches(void);
  * Ids: 0 weight sums, 1 binarize+pack, 2 router, 3 expert scan, 4 activation
  * quantise, 5 HP up-projection, 6 fused forward tile, 7 row scatter, 8 scaled
  * sign, 9 scaled B, 10 HP dH, 11 dX, 12 dW (with the dB, dA and router-weight
- * tiles), 16 per-feature scale gradients, 17 their sum over features, 18 debug
+ * tiles), 16 per-feature scale gradients (vector scales), 17 scalar scale gradients (one launch), 18 debug
  * GEMM, 19 decode token preparation, 20 decode main; 13-15, 21, 22 unused. */
 int pq_profile_events(int kernel_id, void* start_event, void* stop_event);
 

@@ -90,8 +90,8 @@ struct BwdScratch {
   uint16_t* dlc;
   float* dbeta_partial;
   float* dalpha_partial;
-  float* dalpha_vec;
-  float* dbeta_vec;
+  double* blk_sums;      // scalar feature scales: per-block fp64 sums of k_finalize_scales, [2 * ceil(N/128)]
+  unsigned* arrivals;    // ... and its arrival counter
 };
 
 static size_t carve_bwd_scratch(const pq_desc* d, void* base, BwdScratch* out) {
@@ -109,8 +109,8 @@ static size_t carve_bwd_scratch(const pq_desc* d, void* base, BwdScratch* out) {
   s.dlc = routed(d) ? c.take<uint16_t>(T * 16) : nullptr;
   s.dbeta_partial = c.take<float>(2 * ((K + 255) / 256) * N);   // two slots per 256-column tile of K
   s.dalpha_partial = r > 0 ? c.take<float>((size_t)2 * E * N) : nullptr;
-  s.dalpha_vec = c.take<float>(N);
-  s.dbeta_vec = c.take<float>(N);
+  s.blk_sums = c.take<double>(2 * ((N + 127) / 128));
+  s.arrivals = c.take<unsigned>(4);
   if (out) *out = s;
   return c.off;
 }
@@ -488,7 +488,7 @@ int pq_linear_backward(const pq_desc* d, const uint16_t* dY, const uint16_t* X, 
   SideCtx* side = side_for(st);
   if (side && !side_fork(side, st)) return PQ_ERR_CUDA;
   cudaStream_t sx = side ? side->side : st;
-  if (launch_scaled_sign(w_s8, sc.sb, beta, vec, d->N, d->K, sx) != cudaSuccess) return PQ_ERR_CUDA;
+  if (launch_scaled_sign(w_s8, sc.sb, beta, vec, d->N, d->K, sc.arrivals, sx) != cudaSuccess) return PQ_ERR_CUDA;
   b.sb = sc.sb;
   if (hp && vec) {
     if (launch_scaled_b(B, sc.ba, alpha, E, d->N, d->r, sx) != cudaSuccess) return PQ_ERR_CUDA;
@@ -507,7 +507,7 @@ int pq_linear_backward(const pq_desc* d, const uint16_t* dY, const uint16_t* X, 
   // of the dB-weighted row sums; the scalar form sums over n as well
   if (dalpha && !hp && cudaMemsetAsync(dalpha, 0, sizeof(float) * (vec ? d->N : 1), st) != cudaSuccess) return PQ_ERR_CUDA;
   if (launch_finalize_scales(sc.dbeta_partial, 2 * ((d->K + 255) / 256), hp ? sc.dalpha_partial : nullptr, 2 * E, d->N, w_scales, vec, dbeta,
-                             hp ? dalpha : nullptr, sc.dbeta_vec, sc.dalpha_vec, st) != cudaSuccess)
+                             hp ? dalpha : nullptr, sc.blk_sums, sc.arrivals, st) != cudaSuccess)
     return PQ_ERR_CUDA;
   return PQ_OK;
 }

@@ -469,9 +469,11 @@ __global__ void __launch_bounds__(256) k_scatter_rows(const uint4* __restrict__ 
 
 // Sb[n,k] = bf16(scale_n) * S[n,k]; scale_n = beta_n (vector form) or 1
 __global__ void __launch_bounds__(256) k_scaled_sign(const uint4* __restrict__ s8, uint4* __restrict__ out, const float* __restrict__ beta,
-                                                     int beta_stride, int N, int K) {
+                                                     int beta_stride, int N, int K, unsigned* __restrict__ arrivals) {
   pdl_launch_dependents();   // launched with programmatic stream serialisation: see launch_pdl
   pdl_wait();
+  // first kernel of every backward call: it also clears the arrival counter of the call's last kernel (k_finalize_scales)
+  if (arrivals && blockIdx.x == 0 && threadIdx.x == 0) *arrivals = 0u;
   const long long n16 = (long long)N * K / 16;
   const int per_row = K / 16;
   for (long long i = blockIdx.x * 256LL + threadIdx.x; i < n16; i += gridDim.x * 256LL) {
@@ -509,54 +511,60 @@ __global__ void __launch_bounds__(256) k_scaled_b(const uint32_t* __restrict__ B
 
 // Feature-scale gradients from their per-tile partials, one thread per output feature:
 //   dbeta_n = lam * sum_s dbeta_partial[s, n]      dalpha_n = sum_e dalpha_partial[e, n]   (slots / experts ascending)
+// Vector scales: written per feature.  Scalar scales (blk_sums != null): every block adds its features in fp64 (fixed
+// tree) into blk_sums[2 * block], the block that arrives last adds the blocks' sums in index order -- the result does
+// not depend on which block that is -- and writes the two scalars; `arrivals` was cleared by the call's first kernel.
 __global__ void __launch_bounds__(128) k_finalize_scales(const float* __restrict__ dbeta_partial, int nslots,
                                                          const float* __restrict__ dalpha_partial, int E, int N,
                                                          const float* __restrict__ w_scales, float* __restrict__ dbeta,
-                                                         float* __restrict__ dalpha) {
+                                                         float* __restrict__ dalpha, double* blk_sums, unsigned* arrivals) {
   pdl_launch_dependents();   // launched with programmatic stream serialisation: see launch_pdl
   pdl_wait();
   const int n = blockIdx.x * 128 + threadIdx.x;
-  if (n >= N) return;
-  float b = 0.f;
+  float b = 0.f, a = 0.f;
+  if (n < N) {
 #pragma unroll 8
-  for (int s = 0; s < nslots; ++s) b += dbeta_partial[(long long)s * N + n];
-  dbeta[n] = b * w_scales[0];
-  if (dalpha_partial) {
-    float a = 0.f;
+    for (int s = 0; s < nslots; ++s) b += dbeta_partial[(long long)s * N + n];
+    b *= w_scales[0];
+    if (dalpha_partial) {
 #pragma unroll 8
-    for (int e = 0; e < E; ++e) a += dalpha_partial[(long long)e * N + n];
-    dalpha[n] = a;
+      for (int e = 0; e < E; ++e) a += dalpha_partial[(long long)e * N + n];
+    }
   }
-}
-
-// Scalar feature scales: out_b[0] = sum_n vb[n], out_a[0] = sum_n va[n] (va may be null); one block, fp64, fixed tree.
-__global__ void __launch_bounds__(1024) k_sum_scales(const float* __restrict__ vb, const float* __restrict__ va, int N,
-                                                     float* __restrict__ out_b, float* __restrict__ out_a) {
-  pdl_launch_dependents();   // launched with programmatic stream serialisation: see launch_pdl
-  pdl_wait();
-  __shared__ double sh[2][32];
-  double sb = 0.0, sa = 0.0;
-  for (int n = threadIdx.x; n < N; n += 1024) {
-    sb += (double)vb[n];
-    if (va) sa += (double)va[n];
+  if (!blk_sums) {
+    if (n < N) {
+      dbeta[n] = b;
+      if (dalpha_partial) dalpha[n] = a;
+    }
+    return;
   }
+  __shared__ double sh[2][4];
+  __shared__ bool last;
+  double sb = (double)b, sa = (double)a;
   for (int d = 16; d > 0; d >>= 1) {
     sb += __shfl_xor_sync(0xffffffffu, sb, d);
     sa += __shfl_xor_sync(0xffffffffu, sa, d);
   }
   if ((threadIdx.x & 31) == 0) { sh[0][threadIdx.x >> 5] = sb; sh[1][threadIdx.x >> 5] = sa; }
   __syncthreads();
-  if (threadIdx.x < 32) {
-    sb = sh[0][threadIdx.x];
-    sa = sh[1][threadIdx.x];
-    for (int d = 16; d > 0; d >>= 1) {
-      sb += __shfl_xor_sync(0xffffffffu, sb, d);
-      sa += __shfl_xor_sync(0xffffffffu, sa, d);
-    }
-    if (threadIdx.x == 0) {
-      out_b[0] = (float)sb;
-      if (va) out_a[0] = (float)sa;
-    }
+  if (threadIdx.x == 0) {
+    blk_sums[2 * blockIdx.x] = (sh[0][0] + sh[0][1]) + (sh[0][2] + sh[0][3]);
+    blk_sums[2 * blockIdx.x + 1] = (sh[1][0] + sh[1][1]) + (sh[1][2] + sh[1][3]);
+    __threadfence();
+    last = atomicAdd(arrivals, 1u) == gridDim.x - 1;
+  }
+  __syncthreads();
+  if (!last || threadIdx.x >= 32) return;
+  __threadfence();
+  double tb = 0.0, ta = 0.0;
+  for (int i = threadIdx.x; i < (int)gridDim.x; i += 32) { tb += __ldcg(blk_sums + 2 * i); ta += __ldcg(blk_sums + 2 * i + 1); }
+  for (int d = 16; d > 0; d >>= 1) {
+    tb += __shfl_xor_sync(0xffffffffu, tb, d);
+    ta += __shfl_xor_sync(0xffffffffu, ta, d);
+  }
+  if (threadIdx.x == 0) {
+    dbeta[0] = (float)tb;
+    if (dalpha_partial) dalpha[0] = (float)ta;
   }
 }
 
@@ -696,11 +704,12 @@ cudaError_t launch_scatter_rows(const uint16_t* src, uint16_t* dst, const int* p
   return cudaGetLastError();
 }
 
-cudaError_t launch_scaled_sign(const int8_t* s8, uint16_t* out, const float* beta, int beta_stride, int N, int K, cudaStream_t st) {
+cudaError_t launch_scaled_sign(const int8_t* s8, uint16_t* out, const float* beta, int beta_stride, int N, int K, unsigned* arrivals,
+                               cudaStream_t st) {
   const long long n16 = (long long)N * K / 16;
   LaunchScope ls(KID_SCALED_SIGN, st);
   launch_pdl(k_scaled_sign, grid_for(n16, 256 * 2, 148 * 8), 256, 0, st, reinterpret_cast<const uint4*>(s8), reinterpret_cast<uint4*>(out), beta,
-                                                               beta_stride, N, K);
+                                                               beta_stride, N, K, arrivals);
   return cudaGetLastError();
 }
 
@@ -712,16 +721,10 @@ cudaError_t launch_scaled_b(const uint16_t* B, uint16_t* out, const float* alpha
 }
 
 cudaError_t launch_finalize_scales(const float* dbeta_partial, int nslots, const float* dalpha_partial, int E, int N, const float* w_scales,
-                                   int vec, float* dbeta, float* dalpha, float* tmp_b, float* tmp_a, cudaStream_t st) {
-  {
-    LaunchScope ls(KID_SUM_PARTIALS, st);
-    launch_pdl(k_finalize_scales, (N + 127) / 128, 128, 0, st, dbeta_partial, nslots, dalpha_partial, E, N, w_scales, vec ? dbeta : tmp_b,
-                                                       vec ? dalpha : tmp_a);
-  }
-  if (!vec) {
-    LaunchScope ls(KID_SUM_SCALAR, st);
-    launch_pdl(k_sum_scales, 1, 1024, 0, st, tmp_b, dalpha_partial ? tmp_a : nullptr, N, dbeta, dalpha);
-  }
+                                   int vec, float* dbeta, float* dalpha, double* blk_sums, unsigned* arrivals, cudaStream_t st) {
+  LaunchScope ls(vec ? KID_SUM_PARTIALS : KID_SUM_SCALAR, st);
+  launch_pdl(k_finalize_scales, (N + 127) / 128, 128, 0, st, dbeta_partial, nslots, dalpha_partial, E, N, w_scales, dbeta, dalpha,
+             vec ? nullptr : blk_sums, vec ? nullptr : arrivals);
   return cudaGetLastError();
 }
 

@@ -85,10 +85,12 @@ cudaError_t launch_pack(const float* W, int N, int K, uint32_t* bits, int8_t* s8
 cudaError_t launch_route_and_quant(const uint16_t* X, const uint16_t* Wr, int T, int K, int E, const SavedPtrs& sv, const FwdScratch& sc,
                                    cudaStream_t st, cudaStream_t st_quant);
 cudaError_t launch_scatter_rows(const uint16_t* src, uint16_t* dst, const int* pos, int T, int row_elems, cudaStream_t st);
-cudaError_t launch_scaled_sign(const int8_t* s8, uint16_t* out, const float* beta, int beta_stride, int N, int K, cudaStream_t st);
+// arrivals: counter of the call's k_finalize_scales launch, cleared here (null: nothing to clear)
+cudaError_t launch_scaled_sign(const int8_t* s8, uint16_t* out, const float* beta, int beta_stride, int N, int K, unsigned* arrivals,
+                               cudaStream_t st);
 cudaError_t launch_scaled_b(const uint16_t* B, uint16_t* out, const float* alpha, int E, int N, int r, cudaStream_t st);
 cudaError_t launch_finalize_scales(const float* dbeta_partial, int nslots, const float* dalpha_partial, int E, int N, const float* w_scales,
-                                   int vec, float* dbeta, float* dalpha, float* tmp_b, float* tmp_a, cudaStream_t st);
+                                   int vec, float* dbeta, float* dalpha, double* blk_sums, unsigned* arrivals, cudaStream_t st);
 cudaError_t launch_fill_zero(void* p, size_t bytes, cudaStream_t st);
 cudaError_t launch_pack_experts(const uint16_t* A, const uint16_t* B, int E, int r, int K, int N, int8_t* A8, int8_t* B8, float* hp_scales,
                                 uint32_t* amax_bits, cudaStream_t st);
