@@ -422,6 +422,62 @@ def linear_backward(dY, X, fwd, A=None, B=None, Wr=None, alpha=1.0, beta=1.0):
     return g
 
 
+# --------------------------------------------------------------------------
+# FFN-level decoupling (Eq. 11, Table 1): two parallel FFNs split along the hidden dimension
+# --------------------------------------------------------------------------
+def silu_fp32(g32):
+    """SiLU in the arithmetic both sides can reproduce: the logistic factor in fp64, rounded once to fp32, then one
+    fp32 multiply.  (An fp32 exponential differs from library to library in its last bit, and the result feeds a
+    quantiser.)"""
+    g32 = np.asarray(g32, dtype=np.float32)
+    s32 = (1.0 / (1.0 + np.exp(-g32.astype(np.float64)))).astype(np.float32)
+    return (g32 * s32).astype(np.float32)
+
+
+def ffn_int8(q, gamma, G8, gG, U8, gU, D8, gD):
+    """The INT8 FFN of hidden width r on the int8 activation codes q (Sec. 3.2, Eq. 11 first term; the LLaMA-style
+    gated form the paper's models use):
+        g = (G8 q) / (gamma_G gamma_t),  u = (U8 q) / (gamma_U gamma_t)       exact integers, de-quantised in fp32
+        m = silu(g) * u                                                       fp32
+        qm, gamma_m = Eq. 7-9 on m (per token)
+        z = (D8 qm) / (gamma_D gamma_m)
+    Every step up to the codes qm is pinned fp32 arithmetic: deq = fl(1 / fl(gamma_W gamma_t)), g = fl(fl(g_int) deq),
+    m = fl(silu_fp32(g) u).  Returns dict(g_int, u_int, m, qm, gamma_m, z_int, z)."""
+    q64 = np.asarray(q, dtype=np.int64)
+    g_int = q64 @ G8.astype(np.int64).T
+    u_int = q64 @ U8.astype(np.int64).T
+    assert np.all(np.abs(g_int) < 2 ** 31) and np.all(np.abs(u_int) < 2 ** 31)
+    gamma = np.asarray(gamma, dtype=np.float32)
+    deq_g = (np.float32(1.0) / (np.float32(gG) * gamma).astype(np.float32)).astype(np.float32)
+    deq_u = (np.float32(1.0) / (np.float32(gU) * gamma).astype(np.float32)).astype(np.float32)
+    g32 = (g_int.astype(np.float32) * deq_g[:, None]).astype(np.float32)
+    u32 = (u_int.astype(np.float32) * deq_u[:, None]).astype(np.float32)
+    m32 = (silu_fp32(g32) * u32).astype(np.float32)
+    qm, gamma_m = act_quant(m32)
+    z_int = qm.astype(np.int64) @ D8.astype(np.int64).T
+    z = z_int / (np.float64(gD) * gamma_m.astype(np.float64))[:, None]
+    return dict(g_int=g_int, u_int=u_int, m=m32, qm=qm, gamma_m=gamma_m, z_int=z_int, z=z)
+
+
+def ffn_decoupled_forward(X, Wg, Wu, Wd, G, U, D, alpha=2.0, beta=0.2):
+    """Eq. 11: Y = alpha FFN_INT8[:r](x) + beta FFN_INT1[r:](x), both FFNs gated (down(silu(gate x) * up x)).
+    Wg, Wu [F1, Dm], Wd [Dm, F1]: latent weights of the 1-bit FFN of hidden width F1 = D_ff - r, each a pure 1-bit
+    linear (Eq. 3-10) whose output is a bf16 tensor; G, U [r, Dm], D [Dm, r]: the INT8 FFN's matrices (bf16 values),
+    quantised per matrix.  The 1-bit FFN's hidden activation is bf16(silu(g1) * u1) with the product taken in fp64.
+    Returns dict with the pieces; Y rounded once to bf16."""
+    fg = linear_forward(X, Wg, beta=1.0)
+    fu = linear_forward(X, Wu, beta=1.0)
+    g1, u1 = fg["Y"], fu["Y"]
+    m1 = round_to_bf16(g1 / (1.0 + np.exp(-g1)) * u1)
+    fd = linear_forward(m1, Wd, beta=1.0)
+    G8, gG = absmax_quant_matrix(G)
+    U8, gU = absmax_quant_matrix(U)
+    D8, gD = absmax_quant_matrix(D)
+    hp = ffn_int8(fg["q"], fg["gamma"], G8, gG, U8, gU, D8, gD)
+    y64 = np.float64(alpha) * hp["z"] + np.float64(beta) * fd["y1"]
+    return dict(gate=fg, up=fu, down=fd, m1=m1, hp=hp, G8=G8, U8=U8, D8=D8, gG=gG, gU=gU, gD=gD, Y64=y64, Y=round_to_bf16(y64))
+
+
 def rmsnorm(X, weight, eps):
     """RMSNorm in front of the activation quantiser (App. A: at inference the norm is
     fused with the quantisation; the equations write it as LayerNorm(X)).

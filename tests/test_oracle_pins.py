@@ -525,3 +525,95 @@ def test_int8_branch_decode_uses_stored_codes():
     stored = (f["A8"], f["gA"], f["B8"], f["gB"])
     d = O.decode_forward(c["X"], O.pack_bits(f["S"]), f["lam"], c["A"] * 0, c["B"] * 0, c["Wr"], c["alpha"], c["beta"], hp_int8=stored)
     assert np.array_equal(d["Y"], f["Y"]) and np.array_equal(d["z_int"], f["z_int"])
+
+
+# ---------------------------------------------------------------- FFN-level decoupling (Eq. 11, Table 1)
+def _ffn_case(T=12, Dm=32, F1=64, r=16, seed=81):
+    rng = np.random.default_rng(seed)
+    X = I.bf16_values(rng.standard_normal((T, Dm)).astype(np.float32))
+    Wg, Wu = (rng.standard_normal((F1, Dm)) * 0.3).astype(np.float32), (rng.standard_normal((F1, Dm)) * 0.3).astype(np.float32)
+    Wd = (rng.standard_normal((Dm, F1)) * 0.3).astype(np.float32)
+    G = I.bf16_values((rng.standard_normal((r, Dm)) * 0.3).astype(np.float32))
+    U = I.bf16_values((rng.standard_normal((r, Dm)) * 0.3).astype(np.float32))
+    D = I.bf16_values((rng.standard_normal((Dm, r)) * 0.3).astype(np.float32))
+    return X, Wg, Wu, Wd, G, U, D
+
+
+def test_silu_reproducible_form_against_closed_values():
+    x = np.array([0.0, 1.0, -1.0, 20.0, -20.0, 0.5], np.float32)
+    want = [0.0, 1.0 / (1.0 + np.exp(-1.0)), -1.0 / (1.0 + np.exp(1.0)), 20.0, -20.0 * np.exp(-20.0) / (1 + np.exp(-20.0)), 0.5 / (1.0 + np.exp(-0.5))]
+    got = O.silu_fp32(x)
+    assert got.dtype == np.float32
+    assert np.allclose(got, want, rtol=2e-7, atol=1e-12)
+    assert got[1] + (-got[2]) == np.float32(1.0) or abs(float(got[1]) - float(got[2]) - 1.0) < 1e-6     # silu(x) - silu(-x) = x
+
+
+def test_ffn_decoupled_term_by_term():
+    # Eq. 11 on a tiny case with python floats: the 1-bit FFN as three hand-evaluated 1-bit linears, the INT8 FFN from
+    # its integers; planted mistakes (branch scales swapped, activation on the wrong operand, un-gated form) are caught
+    X, Wg, Wu, Wd, G, U, D = _ffn_case()
+    f = O.ffn_decoupled_forward(X, Wg, Wu, Wd, G, U, D, alpha=2.0, beta=0.2)
+    T, Dm = X.shape
+    F1, r = Wg.shape[0], G.shape[0]
+
+    def onebit(Xin, W):          # Eq. 3-10 by hand: fp32 scale decisions come from the pinned helpers, sums are python ints
+        mu, lam = O.weight_scales(W)
+        S = O.binarize(W, mu)
+        q, gam = O.act_quant(Xin)
+        out = [[float(lam) / float(gam[t]) * sum(int(S[n, k]) * int(q[t, k]) for k in range(Xin.shape[1])) for n in range(W.shape[0])]
+               for t in range(Xin.shape[0])]
+        return np.array(out), q, gam
+
+    g1, q, gam = onebit(X, Wg)
+    u1, _, _ = onebit(X, Wu)
+    g1b, u1b = O.round_to_bf16(g1), O.round_to_bf16(u1)
+    assert np.array_equal(g1b, f["gate"]["Y"]) and np.array_equal(u1b, f["up"]["Y"])
+    m1 = O.round_to_bf16(np.array([[g1b[t, j] / (1.0 + np.exp(-g1b[t, j])) * u1b[t, j] for j in range(F1)] for t in range(T)]))
+    y1, _, _ = onebit(m1.astype(np.float32), Wd)
+    G8, gG = O.absmax_quant_matrix(G); U8, gU = O.absmax_quant_matrix(U); D8, gD = O.absmax_quant_matrix(D)
+
+    def int8_ffn(act_on="gate", gated=True):
+        z = np.zeros((T, Dm))
+        for t in range(T):
+            gi = [sum(int(G8[j, k]) * int(q[t, k]) for k in range(Dm)) for j in range(r)]
+            ui = [sum(int(U8[j, k]) * int(q[t, k]) for k in range(Dm)) for j in range(r)]
+            assert gi == f["hp"]["g_int"][t].tolist() and ui == f["hp"]["u_int"][t].tolist()
+            g = [v / (float(gG) * float(gam[t])) for v in gi]
+            u = [v / (float(gU) * float(gam[t])) for v in ui]
+            a, b = (g, u) if act_on == "gate" else (u, g)
+            m = [a[j] / (1.0 + np.exp(-a[j])) * (b[j] if gated else 1.0) for j in range(r)]
+            amax = max(abs(v) for v in m)
+            codes = [int(np.clip(np.rint(v * 128.0 / amax), -128, 127)) for v in m]
+            for n in range(Dm):
+                z[t, n] = sum(int(D8[n, j]) * codes[j] for j in range(r)) / (float(gD) * 128.0 / amax)
+        return z
+
+    z = int8_ffn()
+    # codes decided in fp32 by the oracle may differ by one from the python-float decision at a rounding boundary: the
+    # real-valued z is compared within one code's worth
+    tol = np.abs(D8.astype(np.float64)).sum(axis=1)[None, :] * 1.01 / (float(gD) * f["hp"]["gamma_m"].astype(np.float64))[:, None]
+    assert np.all(np.abs(z - f["hp"]["z"]) <= tol)
+    want = 2.0 * z + 0.2 * y1
+    err = np.abs(f["Y64"] - want)
+    assert np.all(err <= 2.0 * tol + 1e-9)
+    scale = np.abs(want).mean()
+    assert err.mean() < 0.02 * scale
+    for wrong in (0.2 * z + 2.0 * y1, 2.0 * int8_ffn(act_on="up") + 0.2 * y1, 2.0 * int8_ffn(gated=False) + 0.2 * y1, 2.0 * z - 0.2 * y1):
+        assert np.abs(f["Y64"] - wrong).mean() > 0.1 * scale
+    assert np.array_equal(f["Y"], O.round_to_bf16(f["Y64"]))
+
+
+def test_ffn_decoupled_special_cases():
+    X, Wg, Wu, Wd, G, U, D = _ffn_case(seed=82)
+    f = O.ffn_decoupled_forward(X, Wg, Wu, Wd, G, U, D, alpha=0.0, beta=1.0)
+    # alpha = 0: the plain 1-bit FFN, i.e. three pure 1-bit linears around the gate
+    assert np.array_equal(f["Y"], O.round_to_bf16(f["down"]["y1"]))
+    # beta = 0: the INT8 FFN alone, within the quantisers' reach of the un-quantised gated FFN of width r
+    f8 = O.ffn_decoupled_forward(X, Wg, Wu, Wd, G, U, D, alpha=1.0, beta=0.0)
+    X64 = X.astype(np.float64)
+    g, u = X64 @ G.astype(np.float64).T, X64 @ U.astype(np.float64).T
+    ref = (g / (1.0 + np.exp(-g)) * u) @ D.astype(np.float64).T
+    rel = np.sqrt(np.mean((f8["Y64"] - ref) ** 2)) / np.sqrt(np.mean(ref ** 2))
+    assert rel < 0.05
+    # the codes of the hidden activation use the full range and the same quantiser as activations
+    assert np.all(np.abs(f8["hp"]["qm"].astype(int)).max(axis=1) >= 127)
