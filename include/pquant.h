@@ -196,6 +196,41 @@ int pq_linear_forward_hp8(const pq_desc* d, const uint16_t* X, const int8_t* w_s
                           const int8_t* B8, const float* hp_scales, const uint16_t* Wr, const float* alpha, const float* beta,
                           uint16_t* Y, void* saved, size_t saved_bytes, void* ws, size_t ws_bytes, void* stream);
 
+/* FFN-level decoupling, the form the paper trains (Eq. 11, Table 1): two parallel gated FFNs split along the hidden
+ * dimension,
+ *     Y = alpha * FFN_INT8[:r](x) + beta * FFN_INT1[r:](x),      FFN(x) = down( silu(gate x) * (up x) ),
+ * the 1-bit FFN of hidden width F1 = D_ff - r made of three pure 1-bit linears (Eq. 3-10, each output a bf16 tensor,
+ * inner feature scale 1), the INT8 FFN of hidden width r on the same int8 codes of x:
+ *     g = (G8 q) / (gamma_G gamma_t), u = (U8 q) / (gamma_U gamma_t)   (exact int32 sums, de-quantised in fp32)
+ *     m = silu(g) * u, with the logistic factor taken in fp64 and rounded once to fp32;  qm, gamma_m = Eq. 7-9 on m
+ *     FFN_INT8 = (D8 qm) / (gamma_D gamma_m).
+ * Forward only.  T >= 1; D, F1 multiples of 32; r a multiple of 16, 16 <= r <= 128 (PQ_ERR_SHAPE otherwise).
+ *   X [T,D] bf16;  g_s8, u_s8 [F1,D], d_s8 [D,F1] int8 sign matrices and their {lam, mu} from pq_pack_weights;
+ *   G8, U8 [r,D], D8 [D,r] int8 and hp_scales [3] = {gamma_G, gamma_U, gamma_D} (pq_pack_experts on (G, D) gives
+ *   {gamma_G, gamma_D}, on (U, D) gives gamma_U);  alpha, beta: one float each;  Y [T,D] bf16;
+ *   ws: pq_ffn_workspace_bytes(d) bytes.  The 1-bit FFN's hidden activation is bf16(silu(g1) * u1) in fp32. */
+typedef struct pq_ffn_desc {
+  uint32_t size, flags;   /* sizeof(pq_ffn_desc); flags must be 0 */
+  int32_t T, D, F1, r;
+} pq_ffn_desc;
+size_t pq_ffn_workspace_bytes(const pq_ffn_desc* d);
+int pq_ffn_forward(const pq_ffn_desc* d, const uint16_t* X, const int8_t* g_s8, const float* g_scales, const int8_t* u_s8,
+                   const float* u_scales, const int8_t* d_s8, const float* d_scales, const int8_t* G8, const int8_t* U8,
+                   const int8_t* D8, const float* hp_scales, const float* alpha, const float* beta, uint16_t* Y, void* ws,
+                   size_t ws_bytes, void* stream);
+/* What pq_ffn_forward leaves in its workspace, for tests: the bf16 outputs G1, U1 [T,F1] of the 1-bit gate and up
+ * projections and their gated product M1; the exact sums g_int, u_int [ceil(T/128)*128, r] of the INT8 FFN; the codes
+ * qm [.., r] and scales gamma_m of its hidden activation; the codes q_m1 [T,F1] and scales gamma_m1 of M1. */
+typedef struct pq_ffn_view {
+  uint16_t *G1, *U1, *M1;
+  int32_t *g_int, *u_int;
+  int8_t* qm;
+  float* gamma_m;
+  int8_t* q_m1;
+  float* gamma_m1;
+} pq_ffn_view;
+int pq_ffn_view_init(const pq_ffn_desc* d, void* ws, pq_ffn_view* out);
+
 /* What the decode path leaves in its workspace, for tests and diagnostics.  One entry per
  * token: the routed expert, its gate g_t, gamma_t (Eq. 9) and the sum over k of the int8 codes. */
 typedef struct pq_decode_token {

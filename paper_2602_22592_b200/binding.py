@@ -22,7 +22,7 @@ PQ_DECODE_DUMP_ACC = 2
 PQ_PHASE_PACK, PQ_PHASE_FWD, PQ_PHASE_BWD, PQ_PHASE_DECODE = 0, 1, 2, 3
 
 EXPORTS = ("pq_status_string", "pq_workspace_bytes", "pq_saved_bytes", "pq_saved_view_init",
-           "pq_decode_view_init", "pq_bwd_view_init", "pq_decode_batch", "pq_pack_weights", "pq_pack_weights_static", "pq_pack_experts", "pq_linear_forward", "pq_linear_forward_hp8", "pq_linear_backward", "pq_debug_gemm", "pq_debug_gemm_tile",
+           "pq_decode_view_init", "pq_bwd_view_init", "pq_decode_batch", "pq_pack_weights", "pq_pack_weights_static", "pq_pack_experts", "pq_linear_forward", "pq_linear_forward_hp8", "pq_ffn_workspace_bytes", "pq_ffn_forward", "pq_ffn_view_init", "pq_linear_backward", "pq_debug_gemm", "pq_debug_gemm_tile",
            "pq_device_status", "pq_kernel_launches", "pq_profile_events", "pq_set_option")
 
 KERNEL_IDS = dict(pack_sums=0, binarize_pack=1, router=2, route_scan=3, act_quant=4, hp_up=5, fwd=6, scatter_rows=7,
@@ -56,6 +56,15 @@ class pq_decode_item(ctypes.Structure):
 
 class pq_decode_view(ctypes.Structure):
     _fields_ = [("tokens", ctypes.c_void_p), ("acc", ctypes.c_void_p)]
+
+
+class pq_ffn_desc(ctypes.Structure):
+    _fields_ = [("size", ctypes.c_uint32), ("flags", ctypes.c_uint32), ("T", ctypes.c_int32), ("D", ctypes.c_int32),
+                ("F1", ctypes.c_int32), ("r", ctypes.c_int32)]
+
+
+class pq_ffn_view(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("G1", "U1", "M1", "g_int", "u_int", "qm", "gamma_m", "q_m1", "gamma_m1")]
 
 
 class pq_bwd_view(ctypes.Structure):
@@ -98,6 +107,13 @@ def lib() -> ctypes.CDLL:
         L.pq_linear_forward.argtypes = [dp] + [vp] * 10 + [vp, sz, vp, sz, vp]
         L.pq_linear_forward_hp8.restype = ci
         L.pq_linear_forward_hp8.argtypes = [dp] + [vp] * 10 + [vp, sz, vp, sz, vp]
+        fp = ctypes.POINTER(pq_ffn_desc)
+        L.pq_ffn_workspace_bytes.restype = sz
+        L.pq_ffn_workspace_bytes.argtypes = [fp]
+        L.pq_ffn_forward.restype = ci
+        L.pq_ffn_forward.argtypes = [fp] + [vp] * 15 + [sz, vp]
+        L.pq_ffn_view_init.restype = ci
+        L.pq_ffn_view_init.argtypes = [fp, vp, ctypes.POINTER(pq_ffn_view)]
         L.pq_linear_backward.restype = ci
         L.pq_linear_backward.argtypes = [dp] + [vp] * 9 + [vp, sz] + [vp] * 7 + [vp, sz, vp]
         L.pq_debug_gemm.restype = ci
@@ -230,9 +246,44 @@ def pq_linear_forward(d, X, w_bits, w_s8, w_scales, A, B, Wr, alpha, beta, Y, sa
 
 def pq_linear_forward_hp8(d, X, w_s8, w_scales, A8, B8, hp_scales, Wr, alpha, beta, Y, saved, ws, stream=None):
     """Forward with the INT8 high-precision branch (Sec. 3.2); A8, B8, hp_scales come from pq_pack_experts."""
-    _check("pq_linear_forward_hp8", lib().pq_linear_forward_hp8(
+    _check("pq_linear_forward_hp8", "pq_ffn_workspace_bytes", "pq_ffn_forward", "pq_ffn_view_init", lib().pq_linear_forward_hp8(
         ctypes.byref(d), _ptr(X), _ptr(w_s8), _ptr(w_scales), _ptr(A8), _ptr(B8), _ptr(hp_scales), _ptr(Wr), _ptr(alpha),
         _ptr(beta), _ptr(Y), _ptr(saved), _nbytes(saved), _ptr(ws), _nbytes(ws), _stream(stream)))
+
+
+def make_ffn_desc(T, D, F1, r) -> pq_ffn_desc:
+    return pq_ffn_desc(ctypes.sizeof(pq_ffn_desc), 0, T, D, F1, r)
+
+
+def pq_ffn_workspace_bytes(d: pq_ffn_desc) -> int:
+    return lib().pq_ffn_workspace_bytes(ctypes.byref(d))
+
+
+def pq_ffn_forward(d, X, g_s8, g_scales, u_s8, u_scales, d_s8, d_scales, G8, U8, D8, hp_scales, alpha, beta, Y, ws, stream=None):
+    """Eq. 11: Y = alpha FFN_INT8[:r](x) + beta FFN_INT1[r:](x) (forward)."""
+    _check("pq_ffn_forward", lib().pq_ffn_forward(
+        ctypes.byref(d), _ptr(X), _ptr(g_s8), _ptr(g_scales), _ptr(u_s8), _ptr(u_scales), _ptr(d_s8), _ptr(d_scales), _ptr(G8), _ptr(U8),
+        _ptr(D8), _ptr(hp_scales), _ptr(alpha), _ptr(beta), _ptr(Y), _ptr(ws), _nbytes(ws), _stream(stream)))
+
+
+def pq_ffn_view_init(d: pq_ffn_desc, ws: torch.Tensor) -> dict:
+    """Typed views of what pq_ffn_forward left in its workspace."""
+    v = pq_ffn_view()
+    _check("pq_ffn_view_init", lib().pq_ffn_view_init(ctypes.byref(d), _ptr(ws), ctypes.byref(v)))
+    base = ws.data_ptr()
+    rows = (d.T + 127) // 128 * 128
+
+    def view(ptr, dtype, *shape):
+        n = 1
+        for s in shape:
+            n *= s
+        nbytes = n * torch.empty(0, dtype=dtype).element_size()
+        return ws[ptr - base: ptr - base + nbytes].view(dtype).view(*shape)
+
+    return dict(G1=view(v.G1, torch.bfloat16, d.T, d.F1), U1=view(v.U1, torch.bfloat16, d.T, d.F1), M1=view(v.M1, torch.bfloat16, d.T, d.F1),
+                g_int=view(v.g_int, torch.int32, rows, d.r), u_int=view(v.u_int, torch.int32, rows, d.r),
+                qm=view(v.qm, torch.int8, rows, d.r), gamma_m=view(v.gamma_m, torch.float32, rows),
+                q_m1=view(v.q_m1, torch.int8, d.T, d.F1), gamma_m1=view(v.gamma_m1, torch.float32, d.T))
 
 
 def make_decode_items(entries):

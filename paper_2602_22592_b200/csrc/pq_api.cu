@@ -1,6 +1,7 @@
 // C ABI of the pQuant layer: argument checks, carving of the caller's saved /
 // workspace buffers, launch sequencing.  No device allocation, no device
 // synchronisation (except pq_device_status, which says so).
+#include <algorithm>
 #include <cstring>
 #include <map>
 #include <mutex>
@@ -366,7 +367,7 @@ static int check_decode_item(const pq_desc* d, const uint16_t* X, const uint32_t
 // hp_scales != nullptr: INT8 HP branch, A and B are int8 codes (training path only)
 static int forward_impl(const pq_desc* d, const uint16_t* X, const uint32_t* w_bits, const int8_t* w_s8, const float* w_scales,
                         const uint16_t* A, const uint16_t* B, const float* hp_scales, const uint16_t* Wr, const float* alpha, const float* beta,
-                        uint16_t* Y, void* saved, size_t saved_bytes, void* ws, size_t ws_bytes, void* stream) {
+                        uint16_t* Y, void* saved, size_t saved_bytes, void* ws, size_t ws_bytes, void* stream, bool hp_ext = false) {
   if (!d || !X || !w_scales || !beta || !Y) return PQ_ERR_NULL;
   if (!w_s8) {
     if (hp_scales) return PQ_ERR_UNSUPPORTED;
@@ -402,6 +403,7 @@ static int forward_impl(const pq_desc* d, const uint16_t* X, const uint32_t* w_b
   if (hp_scales) {
     if (d->r <= 0 || d->r % 16) return PQ_ERR_SHAPE;       // int8 rows of r bytes must be 16-byte multiples for TMA
     a.hp_scales = hp_scales;
+    a.hp_ext = hp_ext;
   }
   // dense layer with a bf16 HP branch: the quantisation runs on the helper stream next to scan -> up-projection
   // (the INT8 branch multiplies the codes themselves, so its up-projection follows the quantisation)
@@ -425,6 +427,132 @@ int pq_linear_forward_hp8(const pq_desc* d, const uint16_t* X, const int8_t* w_s
   if (!w_s8 || !A8 || !B8 || !hp_scales) return PQ_ERR_NULL;
   return forward_impl(d, X, nullptr, w_s8, w_scales, reinterpret_cast<const uint16_t*>(A8), reinterpret_cast<const uint16_t*>(B8), hp_scales, Wr,
                       alpha, beta, Y, saved, saved_bytes, ws, ws_bytes, stream);
+}
+
+// ---------------------------------------------------------------------------
+// FFN-level decoupling (Eq. 11): Y = alpha FFN_INT8[:r](x) + beta FFN_INT1[r:](x), composed of the entry points above.
+// ---------------------------------------------------------------------------
+static __device__ float g_unit_scale = 1.0f;   // beta of the 1-bit FFN's inner linears
+
+struct FfnCarve {
+  void* saved_x; size_t saved_x_bytes;
+  void* saved_d; size_t saved_d_bytes;
+  void* ws_fwd; size_t ws_fwd_bytes;
+  uint16_t *G1, *U1, *M1;
+  int *g_int, *u_int;
+  size_t total;
+};
+
+static pq_desc ffn_linear_desc(const pq_ffn_desc* d, int K, int N, int r) {
+  pq_desc x{};
+  x.size = sizeof(pq_desc); x.flags = 0; x.T = d->T; x.K = K; x.N = N; x.r = r; x.E = r > 0 ? 1 : 0; x.top_k = 1;
+  return x;
+}
+
+static int check_ffn_desc(const pq_ffn_desc* d) {
+  if (!d) return PQ_ERR_NULL;
+  if (d->size != sizeof(pq_ffn_desc)) return PQ_ERR_SHAPE;
+  if (d->T < 1 || d->D < 32 || d->D % 32 || d->F1 < 32 || d->F1 % 32) return PQ_ERR_SHAPE;
+  if (d->r < 16 || d->r % 16 || d->r > 128) return PQ_ERR_SHAPE;
+  return PQ_OK;
+}
+
+static void carve_ffn(const pq_ffn_desc* d, void* base, FfnCarve* o) {
+  Carver c(base);
+  const pq_desc dx = ffn_linear_desc(d, d->D, d->F1, 0), dd = ffn_linear_desc(d, d->F1, d->D, d->r);
+  o->saved_x_bytes = carve_saved(&dx, nullptr, nullptr);
+  o->saved_d_bytes = carve_saved(&dd, nullptr, nullptr);
+  o->ws_fwd_bytes = std::max(carve_fwd_scratch(&dx, nullptr, nullptr), carve_fwd_scratch(&dd, nullptr, nullptr));
+  o->saved_x = c.take<uint8_t>(o->saved_x_bytes);
+  o->saved_d = c.take<uint8_t>(o->saved_d_bytes);
+  o->ws_fwd = c.take<uint8_t>(o->ws_fwd_bytes);
+  const size_t tf = (size_t)d->T * d->F1, rows = (size_t)mtiles_of(&dx) * kTileRows;
+  o->G1 = c.take<uint16_t>(tf); o->U1 = c.take<uint16_t>(tf); o->M1 = c.take<uint16_t>(tf);
+  o->g_int = c.take<int>(rows * d->r); o->u_int = c.take<int>(rows * d->r);
+  o->total = c.off;
+}
+
+static int unit_scale_ptr(const float** out) {
+  constexpr int kMaxDevices = 64;
+  static const float* cache[kMaxDevices] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return PQ_ERR_CUDA;
+  if (!cache[dev]) {
+    float* ptr = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_unit_scale) != cudaSuccess || !ptr) return PQ_ERR_CUDA;
+    cache[dev] = ptr;
+  }
+  *out = cache[dev];
+  return PQ_OK;
+}
+
+size_t pq_ffn_workspace_bytes(const pq_ffn_desc* d) {
+  if (check_ffn_desc(d) != PQ_OK) return 0;
+  FfnCarve c;
+  carve_ffn(d, nullptr, &c);
+  return c.total;
+}
+
+int pq_ffn_view_init(const pq_ffn_desc* d, void* ws, pq_ffn_view* out) {
+  if (!d || !ws || !out) return PQ_ERR_NULL;
+  int rc = check_ffn_desc(d);
+  if (rc) return rc;
+  FfnCarve c;
+  carve_ffn(d, ws, &c);
+  const pq_desc dx = ffn_linear_desc(d, d->D, d->F1, 0), dd = ffn_linear_desc(d, d->F1, d->D, d->r);
+  SavedPtrs sx, sd;
+  carve_saved(&dx, c.saved_x, &sx);
+  carve_saved(&dd, c.saved_d, &sd);
+  out->G1 = c.G1; out->U1 = c.U1; out->M1 = c.M1; out->g_int = c.g_int; out->u_int = c.u_int;
+  out->qm = reinterpret_cast<int8_t*>(sd.h);
+  out->gamma_m = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(sd.h) + align_up((size_t)sd.max_items * kTileRows * d->r));
+  out->q_m1 = sd.q; out->gamma_m1 = sd.gamma;
+  return PQ_OK;
+}
+
+int pq_ffn_forward(const pq_ffn_desc* d, const uint16_t* X, const int8_t* g_s8, const float* g_scales, const int8_t* u_s8,
+                   const float* u_scales, const int8_t* d_s8, const float* d_scales, const int8_t* G8, const int8_t* U8, const int8_t* D8,
+                   const float* hp_scales, const float* alpha, const float* beta, uint16_t* Y, void* ws, size_t ws_bytes, void* stream) {
+  if (!X || !g_s8 || !g_scales || !u_s8 || !u_scales || !d_s8 || !d_scales || !G8 || !U8 || !D8 || !hp_scales || !alpha || !beta || !Y || !ws)
+    return PQ_ERR_NULL;
+  int rc = check_ffn_desc(d);
+  if (rc) return rc;
+  if (misaligned(X) || misaligned(g_s8) || misaligned(u_s8) || misaligned(d_s8) || misaligned(G8) || misaligned(U8) || misaligned(D8) ||
+      misaligned(Y) || misaligned(ws))
+    return PQ_ERR_ALIGN;
+  FfnCarve c;
+  carve_ffn(d, ws, &c);
+  if (ws_bytes < c.total) return PQ_ERR_WORKSPACE;
+  const float* one = nullptr;
+  rc = unit_scale_ptr(&one);
+  if (rc) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const pq_desc dx = ffn_linear_desc(d, d->D, d->F1, 0), dd = ffn_linear_desc(d, d->F1, d->D, d->r);
+  // 1-bit FFN, gate projection: also leaves the int8 codes of x and the tile table in saved_x
+  rc = forward_impl(&dx, X, nullptr, g_s8, g_scales, nullptr, nullptr, nullptr, nullptr, nullptr, one, c.G1, c.saved_x, c.saved_x_bytes,
+                    c.ws_fwd, c.ws_fwd_bytes, stream);
+  if (rc) return rc;
+  // INT8 FFN: exact sums of its gate and up projections on those codes, then its hidden activation as codes, written
+  // where the fused down projection expects the codes of h
+  SavedPtrs sx, sd;
+  carve_saved(&dx, c.saved_x, &sx);
+  carve_saved(&dd, c.saved_d, &sd);
+  LayerArgs a8{d->T, d->D, d->D, d->r, 1, 0, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+  rc = gemm_hp_up8(a8, sx, G8, c.g_int, st);
+  if (rc) return rc;
+  rc = gemm_hp_up8(a8, sx, U8, c.u_int, st);
+  if (rc) return rc;
+  int8_t* qm = reinterpret_cast<int8_t*>(sd.h);
+  float* gamma_m = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(sd.h) + align_up((size_t)sd.max_items * kTileRows * d->r));
+  if (launch_ffn8_act(c.g_int, c.u_int, sx.gamma, hp_scales, d->T, d->r, qm, gamma_m, st) != cudaSuccess) return PQ_ERR_CUDA;
+  // 1-bit FFN, up projection and gate
+  rc = forward_impl(&dx, X, nullptr, u_s8, u_scales, nullptr, nullptr, nullptr, nullptr, nullptr, one, c.U1, c.saved_x, c.saved_x_bytes,
+                    c.ws_fwd, c.ws_fwd_bytes, stream);
+  if (rc) return rc;
+  if (launch_swiglu(c.G1, c.U1, c.M1, (long long)d->T * d->F1, st) != cudaSuccess) return PQ_ERR_CUDA;
+  // down projections of both FFNs in one fused tile: beta (lam / gamma) (q(M1) . S_d) + alpha (D8 qm) / (gamma_D gamma_m)
+  return forward_impl(&dd, c.M1, nullptr, d_s8, d_scales, reinterpret_cast<const uint16_t*>(D8), reinterpret_cast<const uint16_t*>(D8),
+                      hp_scales + 1, nullptr, alpha, beta, Y, c.saved_d, c.saved_d_bytes, c.ws_fwd, c.ws_fwd_bytes, stream, true);
 }
 
 int pq_decode_batch(const pq_decode_item* items, int n, void* stream) {

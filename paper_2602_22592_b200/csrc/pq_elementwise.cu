@@ -639,6 +639,79 @@ cudaError_t launch_pack_experts(const uint16_t* A, const uint16_t* B, int E, int
   return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------------------
+// FFN-level decoupling (Eq. 11): the two small kernels between the projections.
+// ---------------------------------------------------------------------------
+// Hidden activation of the 1-bit FFN: M = bf16(silu(G) * U), element by element (fp32).
+__global__ void __launch_bounds__(256) k_swiglu(const uint4* __restrict__ G, const uint4* __restrict__ U, uint4* __restrict__ M, long long n8) {
+  pdl_launch_dependents();
+  pdl_wait();
+  for (long long i = blockIdx.x * 256LL + threadIdx.x; i < n8; i += gridDim.x * 256LL) {
+    const uint4 g = __ldg(G + i), u = __ldg(U + i);
+    const uint32_t gw[4] = {g.x, g.y, g.z, g.w}, uw[4] = {u.x, u.y, u.z, u.w};
+    uint32_t o[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float g0 = bf16lo(gw[j]), g1 = bf16hi(gw[j]);
+      o[j] = pack_bf16x2(g0 / (1.0f + __expf(-g0)) * bf16lo(uw[j]), g1 / (1.0f + __expf(-g1)) * bf16hi(uw[j]));
+    }
+    M[i] = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+}
+
+// Hidden activation of the INT8 FFN, one warp per token: from the exact sums g_int = G8 q, u_int = U8 q
+//   g = fl(fl(g_int) * fl(1 / fl(gamma_G gamma_t))), u likewise, m = fl(fl(g * s) * u) with the logistic factor s taken
+//   in fp64 and rounded once to fp32 (an fp32 exponential would not be reproducible, and m feeds a quantiser),
+// then Eq. 7-9 on the row of m: gamma_m = 128 / max(max|m|, 1e-5), codes clamp(rint(m gamma_m)).  r <= 128.
+__global__ void __launch_bounds__(256) k_ffn8_act(const int* __restrict__ g_int, const int* __restrict__ u_int, const float* __restrict__ gamma,
+                                                  const float* __restrict__ hp_scales, int T, int r, int8_t* __restrict__ qm,
+                                                  float* __restrict__ gamma_m) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int t = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (t >= T) return;
+  const float gt = gamma[t];
+  const float deq_g = __fdiv_rn(1.0f, __fmul_rn(hp_scales[0], gt)), deq_u = __fdiv_rn(1.0f, __fmul_rn(hp_scales[1], gt));
+  float m[4];
+  float amax = 0.f;
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int j = lane + 32 * k;
+    m[k] = 0.f;
+    if (j < r) {
+      const float g = __fmul_rn(__int2float_rn(g_int[(long long)t * r + j]), deq_g);
+      const float u = __fmul_rn(__int2float_rn(u_int[(long long)t * r + j]), deq_u);
+      const float s = (float)(1.0 / (1.0 + exp(-(double)g)));
+      m[k] = __fmul_rn(__fmul_rn(g, s), u);
+      amax = fmaxf(amax, fabsf(m[k]));
+    }
+  }
+  for (int d = 16; d > 0; d >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, d));
+  const float gm = __fdiv_rn(kActQmax, fmaxf(amax, kActAmaxFloor));
+  if (lane == 0) gamma_m[t] = gm;
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int j = lane + 32 * k;
+    if (j < r) qm[(long long)t * r + j] = (int8_t)max(-128, min(127, __float2int_rn(__fmul_rn(m[k], gm))));
+  }
+}
+
+cudaError_t launch_swiglu(const uint16_t* G, const uint16_t* U, uint16_t* M, long long n, cudaStream_t st) {
+  const long long n8 = n / 8;
+  long long g = (n8 + 1023) / 1024;
+  launch_pdl(k_swiglu, (int)(g < 1 ? 1 : (g > 148 * 8 ? 148 * 8 : g)), 256, 0, st, reinterpret_cast<const uint4*>(G), reinterpret_cast<const uint4*>(U),
+             reinterpret_cast<uint4*>(M), n8);
+  ++g_launches;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_ffn8_act(const int* g_int, const int* u_int, const float* gamma, const float* hp_scales, int T, int r, int8_t* qm,
+                            float* gamma_m, cudaStream_t st) {
+  launch_pdl(k_ffn8_act, (T + 7) / 8, 256, 0, st, g_int, u_int, gamma, hp_scales, T, r, qm, gamma_m);
+  ++g_launches;
+  return cudaGetLastError();
+}
+
 __global__ void k_fill_zero(uint4* p, long long n16) {
   pdl_launch_dependents();   // launched with programmatic stream serialisation: see launch_pdl
   pdl_wait();

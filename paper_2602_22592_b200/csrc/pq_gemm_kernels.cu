@@ -280,6 +280,7 @@ struct HpUp8Problem {
     RoutingTables rt;
     int8_t* qh;
     float* gamma_h;
+    int* raw;            // not null: write the exact sums h_int [items*128, r] instead of codes (the caller quantises later)
     int K, r, rp, bn;
   };
   struct Tile { int item; int4 it; };
@@ -296,6 +297,18 @@ struct HpUp8Problem {
   using Pre = NoPre;
   __device__ static Pre prepare(const Params&, const Tile&, int, int) { return Pre{}; }
   __device__ static void epilogue(const Params& p, const Tile& t, const Pre& pre, uint32_t taddr, uint32_t, int quad, int half, int lane, uint8_t* stage) {
+    if (p.raw) {
+      int* out = p.raw + ((long long)t.item * 128 + quad * 32 + lane) * p.r;
+      for (int c = half; c * 32 < p.r; c += 2) {
+        uint32_t v[32];
+        tmem_ld32(taddr + c * 32, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          if (c * 32 + 4 * j < p.r) reinterpret_cast<uint4*>(out + c * 32)[j] = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+      }
+      return;
+    }
     if (half) return;   // the maximum over a row's r columns stays in one thread
     const int row = quad * 32 + lane;
     const bool live = row >= t.it.z && row < t.it.w;
@@ -360,6 +373,7 @@ struct FwdProblem {
     // its de-quantisation factor 1 / (gamma_B gamma_h gamma_A gamma_t) is folded into the row's HP factor
     const float* gamma_h;    // [items*128], null for the bf16 branch
     const float* hp_scales;  // [E][2] = {gamma_A, gamma_B}
+    int hp_ext;              // the codes of h and gamma_h were written by the caller
     int T, N, K, r, sstride, item_rows;
   };
   struct Tile { TileCoord c; int bn, ib, ie; };
@@ -433,7 +447,9 @@ struct FwdProblem {
           const int4 d = p.rt.items[it];
           if (rel >= d.z && rel < d.w) {
             const float gh = p.gamma_h[(long long)it * 128 + rel];
-            deq = 1.0f / (p.hp_scales[2 * d.y + 1] * gh * p.hp_scales[2 * d.y] * p.gamma[pos]);
+            // hidden codes made by the library from h_int = A8 q carry gamma_A gamma_t; codes handed in from outside
+            // (the FFN-level form, whose hidden activation went through its non-linearity first) carry gamma_h alone
+            deq = p.hp_ext ? 1.0f / (p.hp_scales[2 * d.y + 1] * gh) : 1.0f / (p.hp_scales[2 * d.y + 1] * gh * p.hp_scales[2 * d.y] * p.gamma[pos]);
           }
         }
         r.ca *= deq;
@@ -480,7 +496,7 @@ static int fill_forward_params(const LayerArgs& a, const int8_t* w_s8, const Sav
   if (!map2d(&f.tq, true, sv.q, a.K, a.T, 128, 128)) return PQ_ERR_CUDA;
   if (!map2d(&f.ts, true, w_s8, a.K, a.N, 128, 256)) return PQ_ERR_CUDA;
   f.th = f.tq; f.tb = f.tq;
-  f.gamma_h = nullptr; f.hp_scales = a.hp_scales;
+  f.gamma_h = nullptr; f.hp_scales = a.hp_scales; f.hp_ext = a.hp_ext ? 1 : 0;
   if (HP && a.hp_scales) {
     // INT8 branch: codes of h [items*128, r] and of B_e [E, N, r], one byte per value
     const uint64_t rows = (uint64_t)sv.max_items * 128;
@@ -498,16 +514,25 @@ static int fill_forward_params(const LayerArgs& a, const int8_t* w_s8, const Sav
   return PQ_OK;
 }
 
+// h_int = q A8_e^T per item.  raw == nullptr: codes and scales of h into the saved h region; otherwise the exact sums
+// [items*128, r] into `raw` (A8 [E, r, K] int8).
+int gemm_hp_up8(const LayerArgs& a, const SavedPtrs& sv, const void* A8, int* raw, cudaStream_t st) {
+  HpUp8Problem::Params p;
+  p.rt = sv.rt; p.qh = reinterpret_cast<int8_t*>(sv.h); p.gamma_h = raw ? nullptr : hp8_gamma_h(sv, a.r); p.raw = raw;
+  p.K = a.K; p.r = a.r; p.rp = a.r; p.bn = h_round_up(a.r, 16);
+  if (!map2d(&p.tq, true, sv.q, a.K, a.T, 128, 128)) return PQ_ERR_CUDA;
+  if (!map3d_i8(&p.ta, A8, a.K, a.K, a.r, a.E, p.bn)) return PQ_ERR_CUDA;
+  return launch_gemm(KID_HP_UP, k_gemm_hp_up8, p, sv.max_items, st);
+}
+
 int gemm_forward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, const uint16_t* xs, uint16_t* Y, cudaStream_t st,
                  cudaEvent_t before_main) {
   if (a.r > 0 && a.hp_scales) {
-    HpUp8Problem::Params p;
-    p.rt = sv.rt; p.qh = reinterpret_cast<int8_t*>(sv.h); p.gamma_h = hp8_gamma_h(sv, a.r); p.K = a.K; p.r = a.r; p.rp = a.r;
-    p.bn = h_round_up(a.r, 16);
-    if (!map2d(&p.tq, true, sv.q, a.K, a.T, 128, 128)) return PQ_ERR_CUDA;
-    if (!map3d_i8(&p.ta, a.A, a.K, a.K, a.r, a.E, p.bn)) return PQ_ERR_CUDA;
-    int rc = launch_gemm(KID_HP_UP, k_gemm_hp_up8, p, sv.max_items, st);
-    if (rc) return rc;
+    int rc = PQ_OK;
+    if (!a.hp_ext) {
+      rc = gemm_hp_up8(a, sv, a.A, nullptr, st);
+      if (rc) return rc;
+    }
     FwdProblem<true>::Params f;
     rc = fill_forward_params<true>(a, w_s8, sv, Y, f);
     if (rc) return rc;

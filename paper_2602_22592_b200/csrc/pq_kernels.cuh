@@ -92,6 +92,9 @@ cudaError_t launch_scaled_b(const uint16_t* B, uint16_t* out, const float* alpha
 cudaError_t launch_finalize_scales(const float* dbeta_partial, int nslots, const float* dalpha_partial, int E, int N, const float* w_scales,
                                    int vec, float* dbeta, float* dalpha, double* blk_sums, unsigned* arrivals, cudaStream_t st);
 cudaError_t launch_fill_zero(void* p, size_t bytes, cudaStream_t st);
+cudaError_t launch_swiglu(const uint16_t* G, const uint16_t* U, uint16_t* M, long long n, cudaStream_t st);
+cudaError_t launch_ffn8_act(const int* g_int, const int* u_int, const float* gamma, const float* hp_scales, int T, int r, int8_t* qm,
+                            float* gamma_m, cudaStream_t st);
 cudaError_t launch_pack_experts(const uint16_t* A, const uint16_t* B, int E, int r, int K, int N, int8_t* A8, int8_t* B8, float* hp_scales,
                                 uint32_t* amax_bits, cudaStream_t st);
 
@@ -106,10 +109,12 @@ struct LayerArgs {
   const uint16_t* B;   // [E,N,r]
   const uint16_t* Wr;  // [E,K]
   const float* hp_scales = nullptr;   // INT8 HP branch: [E][2] = {gamma_A, gamma_B}, and A, B then point to int8 codes
+  bool hp_ext = false;                // INT8 HP branch whose hidden codes and gamma_h are already in the saved h region
 };
 
 int gemm_debug(int mode, int M, int N, int K, const void* A, const void* B, void* D, int tile_n, cudaStream_t st);
 // before_main: an event the fused forward GEMM waits for (work on another stream that feeds it), or nullptr
+int gemm_hp_up8(const LayerArgs& a, const SavedPtrs& sv, const void* A8, int* raw, cudaStream_t st);
 int gemm_forward(const LayerArgs& a, const int8_t* w_s8, const SavedPtrs& sv, const uint16_t* xs, uint16_t* Y, cudaStream_t st,
                  cudaEvent_t before_main);
 
