@@ -66,7 +66,8 @@ enum {
 
 enum {
   PQ_SCALE_VECTOR = 1u,    /* pq_desc.flags: alpha, beta have N entries instead of 1                      */
-  PQ_DECODE_DUMP_ACC = 2u  /* decode only, test hook: also write the exact int32 sums of the 1-bit product */
+  PQ_DECODE_DUMP_ACC = 2u, /* decode only, test hook: also write the exact int32 sums of the 1-bit product */
+  PQ_FUSED_RMSNORM = 8u    /* training path: the layer is called through pq_linear_forward_rms (sizes `saved`) */
 };
 
 enum { PQ_PHASE_PACK = 0, PQ_PHASE_FWD = 1, PQ_PHASE_BWD = 2, PQ_PHASE_DECODE = 3 };
@@ -182,6 +183,19 @@ int pq_linear_forward(const pq_desc* d, const uint16_t* X, const uint32_t* w_bit
                       const uint16_t* B, const uint16_t* Wr, const float* alpha,
                       const float* beta, uint16_t* Y, void* saved, size_t saved_bytes, void* ws,
                       size_t ws_bytes, void* stream);
+
+/* Training-size forward with RMSNorm fused in front of the activation quantiser (App. A: the norm merges with the
+ * quantisation, both being element-wise).  X is the UN-normalised activation; every use of a token -- quantiser, router,
+ * HP branch -- sees
+ *     bf16( fp32( fp32(x * s_t) * norm_weight_k ) ),   s_t = fp32( 1 / sqrt(mean_k x^2 + norm_eps) )   (mean, root in fp64),
+ * the values a separate bf16 norm layer would have handed over, which never exist in memory except as the sorted copy
+ * `xs` in `saved`.  d->flags must carry PQ_FUSED_RMSNORM (it sizes `saved` and the workspace: query them with the same
+ * desc); norm_weight [K] bf16, norm_eps > 0.  pq_linear_backward with the same desc then takes the layer's input from
+ * `saved` (its X argument is not read for the HP gradients) and returns dX with respect to the NORMALISED activation:
+ * the norm's own backward belongs to the caller. */
+int pq_linear_forward_rms(const pq_desc* d, const uint16_t* X, const uint16_t* norm_weight, float norm_eps, const int8_t* w_s8,
+                          const float* w_scales, const uint16_t* A, const uint16_t* B, const uint16_t* Wr, const float* alpha,
+                          const float* beta, uint16_t* Y, void* saved, size_t saved_bytes, void* ws, size_t ws_bytes, void* stream);
 
 /* Forward with the paper's INT8 high-precision branch (Sec. 3.2), training-size path (tensor cores), forward only:
  * the branch multiplies the SAME int8 activation codes q the 1-bit branch uses,

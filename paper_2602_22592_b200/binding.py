@@ -19,10 +19,11 @@ PQ_ERR_NULL, PQ_ERR_SHAPE, PQ_ERR_ALIGN, PQ_ERR_WORKSPACE = -1, -2, -3, -4
 PQ_ERR_UNSUPPORTED, PQ_ERR_CUDA, PQ_ERR_TIMEOUT, PQ_ERR_TOO_LARGE = -5, -6, -7, -8
 PQ_SCALE_VECTOR = 1
 PQ_DECODE_DUMP_ACC = 2
+PQ_FUSED_RMSNORM = 8
 PQ_PHASE_PACK, PQ_PHASE_FWD, PQ_PHASE_BWD, PQ_PHASE_DECODE = 0, 1, 2, 3
 
 EXPORTS = ("pq_status_string", "pq_workspace_bytes", "pq_saved_bytes", "pq_saved_view_init",
-           "pq_decode_view_init", "pq_bwd_view_init", "pq_decode_batch", "pq_pack_weights", "pq_pack_weights_static", "pq_pack_experts", "pq_linear_forward", "pq_linear_forward_hp8", "pq_ffn_workspace_bytes", "pq_ffn_forward", "pq_ffn_view_init", "pq_linear_backward", "pq_debug_gemm", "pq_debug_gemm_tile",
+           "pq_decode_view_init", "pq_bwd_view_init", "pq_decode_batch", "pq_pack_weights", "pq_pack_weights_static", "pq_pack_experts", "pq_linear_forward", "pq_linear_forward_hp8", "pq_linear_forward_rms", "pq_ffn_workspace_bytes", "pq_ffn_forward", "pq_ffn_view_init", "pq_linear_backward", "pq_debug_gemm", "pq_debug_gemm_tile",
            "pq_device_status", "pq_kernel_launches", "pq_profile_events", "pq_set_option")
 
 KERNEL_IDS = dict(pack_sums=0, binarize_pack=1, router=2, route_scan=3, act_quant=4, hp_up=5, fwd=6, scatter_rows=7,
@@ -105,6 +106,8 @@ def lib() -> ctypes.CDLL:
         L.pq_pack_experts.argtypes = [dp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.pq_linear_forward.restype = ci
         L.pq_linear_forward.argtypes = [dp] + [vp] * 10 + [vp, sz, vp, sz, vp]
+        L.pq_linear_forward_rms.restype = ci
+        L.pq_linear_forward_rms.argtypes = [dp, vp, vp, ctypes.c_float] + [vp] * 8 + [vp, sz, vp, sz, vp]
         L.pq_linear_forward_hp8.restype = ci
         L.pq_linear_forward_hp8.argtypes = [dp] + [vp] * 10 + [vp, sz, vp, sz, vp]
         fp = ctypes.POINTER(pq_ffn_desc)
@@ -150,8 +153,8 @@ def _check(fn, status):
         raise PqError(fn, status)
 
 
-def make_desc(T, K, N, r=0, E=0, top_k=1, scale_vector=False, dump_acc=False) -> pq_desc:
-    flags = (PQ_SCALE_VECTOR if scale_vector else 0) | (PQ_DECODE_DUMP_ACC if dump_acc else 0)
+def make_desc(T, K, N, r=0, E=0, top_k=1, scale_vector=False, dump_acc=False, fused_rmsnorm=False) -> pq_desc:
+    flags = (PQ_SCALE_VECTOR if scale_vector else 0) | (PQ_DECODE_DUMP_ACC if dump_acc else 0) | (PQ_FUSED_RMSNORM if fused_rmsnorm else 0)
     return pq_desc(ctypes.sizeof(pq_desc), flags, T, K, N, r, E, top_k)
 
 
@@ -244,9 +247,16 @@ def pq_linear_forward(d, X, w_bits, w_s8, w_scales, A, B, Wr, alpha, beta, Y, sa
         _ptr(beta), _ptr(Y), _ptr(saved), _nbytes(saved), _ptr(ws), _nbytes(ws), _stream(stream)))
 
 
+def pq_linear_forward_rms(d, X, norm_weight, norm_eps, w_s8, w_scales, A, B, Wr, alpha, beta, Y, saved, ws, stream=None):
+    """Training-size forward from un-normalised X with RMSNorm fused in front of the quantiser (d built with fused_rmsnorm=True)."""
+    _check("pq_linear_forward_rms", lib().pq_linear_forward_rms(
+        ctypes.byref(d), _ptr(X), _ptr(norm_weight), ctypes.c_float(norm_eps), _ptr(w_s8), _ptr(w_scales), _ptr(A), _ptr(B), _ptr(Wr),
+        _ptr(alpha), _ptr(beta), _ptr(Y), _ptr(saved), _nbytes(saved), _ptr(ws), _nbytes(ws), _stream(stream)))
+
+
 def pq_linear_forward_hp8(d, X, w_s8, w_scales, A8, B8, hp_scales, Wr, alpha, beta, Y, saved, ws, stream=None):
     """Forward with the INT8 high-precision branch (Sec. 3.2); A8, B8, hp_scales come from pq_pack_experts."""
-    _check("pq_linear_forward_hp8", "pq_ffn_workspace_bytes", "pq_ffn_forward", "pq_ffn_view_init", lib().pq_linear_forward_hp8(
+    _check("pq_linear_forward_hp8", lib().pq_linear_forward_hp8(
         ctypes.byref(d), _ptr(X), _ptr(w_s8), _ptr(w_scales), _ptr(A8), _ptr(B8), _ptr(hp_scales), _ptr(Wr), _ptr(alpha),
         _ptr(beta), _ptr(Y), _ptr(saved), _nbytes(saved), _ptr(ws), _nbytes(ws), _stream(stream)))
 

@@ -30,6 +30,7 @@ static inline int mtiles_of(const pq_desc* d) { return (d->T + kTileRows - 1) / 
 static inline int experts_of(const pq_desc* d) { return d->r > 0 ? (d->E < 1 ? 1 : d->E) : 1; }
 static inline int max_items_of(const pq_desc* d) { return mtiles_of(d) + experts_of(d) - 1; }
 static inline bool routed(const pq_desc* d) { return d->r > 0 && d->E > 1; }
+static inline bool normed(const pq_desc* d) { return (d->flags & PQ_FUSED_RMSNORM) != 0; }
 
 static int check_desc(const pq_desc* d, bool training) {
   if (!d) return PQ_ERR_NULL;
@@ -51,7 +52,7 @@ static size_t carve_saved(const pq_desc* d, void* base, SavedPtrs* out) {
   s.max_items = max_items_of(d);
   s.q = c.take<int8_t>(T * K);
   s.xt = c.take<uint16_t>(T * K);
-  s.xs = routed(d) ? c.take<uint16_t>(T * K) : nullptr;
+  s.xs = (routed(d) || normed(d)) ? c.take<uint16_t>(T * K) : nullptr;   // with a fused norm: the normalised activation
   s.gamma = c.take<float>(T);
   s.gate = c.take<float>(T);
   s.probs = routed(d) ? c.take<float>(T * E) : nullptr;
@@ -77,6 +78,7 @@ static size_t carve_fwd_scratch(const pq_desc* d, void* base, FwdScratch* out) {
   s.probs_tok = c.take<float>((size_t)d->T * E);
   s.block_counts = c.take<int>(nblocks * E);
   s.block_base = c.take<int>(nblocks * E);
+  s.rms = c.take<float>(d->T);
   if (out) *out = s;
   return c.off;
 }
@@ -367,7 +369,8 @@ static int check_decode_item(const pq_desc* d, const uint16_t* X, const uint32_t
 // hp_scales != nullptr: INT8 HP branch, A and B are int8 codes (training path only)
 static int forward_impl(const pq_desc* d, const uint16_t* X, const uint32_t* w_bits, const int8_t* w_s8, const float* w_scales,
                         const uint16_t* A, const uint16_t* B, const float* hp_scales, const uint16_t* Wr, const float* alpha, const float* beta,
-                        uint16_t* Y, void* saved, size_t saved_bytes, void* ws, size_t ws_bytes, void* stream, bool hp_ext = false) {
+                        uint16_t* Y, void* saved, size_t saved_bytes, void* ws, size_t ws_bytes, void* stream, bool hp_ext = false,
+                        const uint16_t* norm_weight = nullptr, float norm_eps = 0.f) {
   if (!d || !X || !w_scales || !beta || !Y) return PQ_ERR_NULL;
   if (!w_s8) {
     if (hp_scales) return PQ_ERR_UNSUPPORTED;
@@ -381,6 +384,8 @@ static int forward_impl(const pq_desc* d, const uint16_t* X, const uint32_t* w_b
   int rc = check_desc(d, true);
   if (rc) return rc;
   (void)w_bits;
+  if (normed(d) != (norm_weight != nullptr)) return PQ_ERR_NULL;           // the flag sizes the saved buffer
+  if (norm_weight && (!(norm_eps > 0.f) || misaligned(norm_weight))) return norm_eps > 0.f ? PQ_ERR_ALIGN : PQ_ERR_SHAPE;
   if (d->r > 0 && (!A || !B || !alpha)) return PQ_ERR_NULL;
   if (routed(d) && !Wr) return PQ_ERR_NULL;
   if (!ws) return PQ_ERR_NULL;
@@ -407,11 +412,13 @@ static int forward_impl(const pq_desc* d, const uint16_t* X, const uint32_t* w_b
   }
   // dense layer with a bf16 HP branch: the quantisation runs on the helper stream next to scan -> up-projection
   // (the INT8 branch multiplies the codes themselves, so its up-projection follows the quantisation)
-  SideCtx* side = (d->r > 0 && !routed(d) && !hp_scales) ? side_for(st) : nullptr;
+  // (with a fused norm the up-projection reads the normalised copy the quantiser writes, so it follows it)
+  SideCtx* side = (d->r > 0 && !routed(d) && !hp_scales && !norm_weight) ? side_for(st) : nullptr;
   if (side && !side_fork(side, st)) return PQ_ERR_CUDA;
-  if (launch_route_and_quant(X, Wr, d->T, d->K, routed(d) ? E : 1, sv, sc, st, side ? side->side : st) != cudaSuccess) return PQ_ERR_CUDA;
+  if (launch_route_and_quant(X, Wr, d->T, d->K, routed(d) ? E : 1, sv, sc, st, side ? side->side : st, norm_weight, norm_eps) != cudaSuccess)
+    return PQ_ERR_CUDA;
   if (side && cudaEventRecord(side->join, side->side) != cudaSuccess) return PQ_ERR_CUDA;
-  const uint16_t* xs = routed(d) ? sv.xs : X;
+  const uint16_t* xs = (routed(d) || norm_weight) ? sv.xs : X;
   return gemm_forward(a, w_s8, sv, xs, Y, st, side ? side->join : nullptr);
 }
 
@@ -419,6 +426,14 @@ int pq_linear_forward(const pq_desc* d, const uint16_t* X, const uint32_t* w_bit
                       const uint16_t* A, const uint16_t* B, const uint16_t* Wr, const float* alpha, const float* beta, uint16_t* Y,
                       void* saved, size_t saved_bytes, void* ws, size_t ws_bytes, void* stream) {
   return forward_impl(d, X, w_bits, w_s8, w_scales, A, B, nullptr, Wr, alpha, beta, Y, saved, saved_bytes, ws, ws_bytes, stream);
+}
+
+int pq_linear_forward_rms(const pq_desc* d, const uint16_t* X, const uint16_t* norm_weight, float norm_eps, const int8_t* w_s8,
+                          const float* w_scales, const uint16_t* A, const uint16_t* B, const uint16_t* Wr, const float* alpha, const float* beta,
+                          uint16_t* Y, void* saved, size_t saved_bytes, void* ws, size_t ws_bytes, void* stream) {
+  if (!w_s8 || !norm_weight) return PQ_ERR_NULL;
+  return forward_impl(d, X, nullptr, w_s8, w_scales, A, B, nullptr, Wr, alpha, beta, Y, saved, saved_bytes, ws, ws_bytes, stream, false,
+                      norm_weight, norm_eps);
 }
 
 int pq_linear_forward_hp8(const pq_desc* d, const uint16_t* X, const int8_t* w_s8, const float* w_scales, const int8_t* A8, const int8_t* B8,
@@ -609,7 +624,7 @@ int pq_linear_backward(const pq_desc* d, const uint16_t* dY, const uint16_t* X, 
     b.xs = sv.xs;
   } else {
     b.dys = dY;
-    b.xs = X;
+    b.xs = normed(d) ? sv.xs : X;      // the layer's input is the normalised activation the forward left in `saved`
   }
   // With the helper stream: what leads to dX (scaled sign matrix, scaled B, HP gradient GEMM, dX) runs there, the
   // weight gradient on the caller's stream beside it; see BwdStreams.

@@ -128,6 +128,37 @@ __global__ void __launch_bounds__(256) k_binarize_pack(const float4* __restrict_
   }
 }
 
+// RMSNorm fused in front of the quantiser (App. A): what every consumer of a token sees is
+//   bf16( fl32( fl32(x * s_t) * g_k ) ),   s_t = fl32( 1 / sqrt(mean_k x^2 + eps) )  (mean and root in fp64, k_row_rms),
+// the values a separate bf16 norm layer would have handed over.  One 16-byte piece (8 values) at a time.
+__device__ __forceinline__ uint4 rms_apply(const uint4& v, float s, const uint4& g) {
+  uint4 o;
+  o.x = pack_bf16x2(__fmul_rn(__fmul_rn(bf16lo(v.x), s), bf16lo(g.x)), __fmul_rn(__fmul_rn(bf16hi(v.x), s), bf16hi(g.x)));
+  o.y = pack_bf16x2(__fmul_rn(__fmul_rn(bf16lo(v.y), s), bf16lo(g.y)), __fmul_rn(__fmul_rn(bf16hi(v.y), s), bf16hi(g.y)));
+  o.z = pack_bf16x2(__fmul_rn(__fmul_rn(bf16lo(v.z), s), bf16lo(g.z)), __fmul_rn(__fmul_rn(bf16hi(v.z), s), bf16hi(g.z)));
+  o.w = pack_bf16x2(__fmul_rn(__fmul_rn(bf16lo(v.w), s), bf16lo(g.w)), __fmul_rn(__fmul_rn(bf16hi(v.w), s), bf16hi(g.w)));
+  return o;
+}
+
+// s_t for every token: one warp per row, squares summed in fp64 (lane-strided pieces ascending, then the butterfly).
+__global__ void __launch_bounds__(256) k_row_rms(const uint4* __restrict__ X, int T, int K, float eps, float* __restrict__ rms) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int t = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (t >= T) return;
+  const int chunks = K >> 3;
+  const uint4* row = X + (long long)t * chunks;
+  double ss = 0.0;
+  for (int c = lane; c < chunks; c += 32) {
+    const uint4 v = __ldg(row + c);
+    const double d0 = bf16lo(v.x), d1 = bf16hi(v.x), d2 = bf16lo(v.y), d3 = bf16hi(v.y);
+    const double d4 = bf16lo(v.z), d5 = bf16hi(v.z), d6 = bf16lo(v.w), d7 = bf16hi(v.w);
+    ss += ((d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3)) + ((d4 * d4 + d5 * d5) + (d6 * d6 + d7 * d7));
+  }
+  for (int d = 16; d > 0; d >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, d);
+  if (lane == 0) rms[t] = (float)(1.0 / sqrt(ss / (double)K + (double)eps));
+}
+
 // ---------------------------------------------------------------------------
 // K4a: router (Sec. 3.3).  One warp per token (or per two).  Logits in fp32 with a fixed
 // summation order -- lane j owns the 8-element chunks c with c mod 32 == j,
@@ -142,7 +173,8 @@ __global__ void __launch_bounds__(256) k_binarize_pack(const float4* __restrict_
 template <int EMAX, int TPW>
 __global__ void __launch_bounds__(32 * kRouterTokensPerBlock / TPW, TPW >= 4 ? 2 : 1) k_router(const uint4* __restrict__ X, const uint4* __restrict__ Wr, int T, int K,
                                                                              int E, int* __restrict__ expert, float* __restrict__ gate_tok,
-                                                                             float* __restrict__ probs_tok, int* __restrict__ block_counts) {
+                                                                             float* __restrict__ probs_tok, int* __restrict__ block_counts,
+                                                                             const uint4* __restrict__ norm_w, const float* __restrict__ rms) {
   pdl_launch_dependents();   // launched with programmatic stream serialisation: see launch_pdl
   pdl_wait();
   __shared__ int cnt[kMaxExperts];
@@ -184,15 +216,23 @@ __global__ void __launch_bounds__(32 * kRouterTokensPerBlock / TPW, TPW >= 4 ? 2
     };
     // the tokens' chunks in ascending order; the next chunk of every row and this chunk's pieces of Wr are
     // requested before the current chunk is folded in
+    float srow[TPW];
+#pragma unroll
+    for (int u = 0; u < TPW; ++u) srow[u] = norm_w ? rms[min(t0 + u, T - 1)] : 1.0f;
+    auto fetch_x = [&](int u, int cc) {
+      if (cc >= chunks) return make_uint4(0u, 0u, 0u, 0u);
+      const uint4 v = __ldg(xrow[u] + cc);
+      return norm_w ? rms_apply(v, srow[u], __ldg(norm_w + cc)) : v;      // the router sees the normalised token
+    };
     int c = lane;
     uint4 xc[TPW];
 #pragma unroll
-    for (int u = 0; u < TPW; ++u) xc[u] = c < chunks ? __ldg(xrow[u] + c) : make_uint4(0u, 0u, 0u, 0u);
+    for (int u = 0; u < TPW; ++u) xc[u] = fetch_x(u, c);
     while (c < chunks) {
       const int cn = c + 32;
       uint4 xn[TPW];
 #pragma unroll
-      for (int u = 0; u < TPW; ++u) xn[u] = cn < chunks ? __ldg(xrow[u] + cn) : make_uint4(0u, 0u, 0u, 0u);
+      for (int u = 0; u < TPW; ++u) xn[u] = fetch_x(u, cn);
       uint4 wr[EMAX];
 #pragma unroll
       for (int e = 0; e < EMAX; ++e) wr[e] = e < E ? __ldg(Wr + (long long)e * chunks + c) : make_uint4(0u, 0u, 0u, 0u);
@@ -362,7 +402,8 @@ __global__ void __launch_bounds__(256) k_act_quant(const uint4* __restrict__ X, 
                                                    const float* __restrict__ gate_tok, const float* __restrict__ probs_tok,
                                                    uint2* __restrict__ q, uint4* __restrict__ xt, uint4* __restrict__ xs,
                                                    float* __restrict__ gamma_s, float* __restrict__ gate_s, float* __restrict__ probs_s,
-                                                   int* __restrict__ perm, int* __restrict__ pos) {
+                                                   int* __restrict__ perm, int* __restrict__ pos, const uint4* __restrict__ norm_w,
+                                                   const float* __restrict__ rms) {
   pdl_launch_dependents();   // launched with programmatic stream serialisation: see launch_pdl
   pdl_wait();
   __shared__ float amax_sh[8];
@@ -374,6 +415,11 @@ __global__ void __launch_bounds__(256) k_act_quant(const uint4* __restrict__ X, 
   const int t = valid ? t_raw : T - 1;                  // idle warps of a shared row keep the barrier company
   const int chunks = K >> 3;
   const uint4* xrow = X + (long long)t * chunks;
+  const float srow = norm_w ? rms[t] : 1.0f;
+  auto fetch_x = [&](int c) {                      // with a fused RMSNorm every later step sees the normalised token
+    const uint4 v = __ldg(xrow + c);
+    return norm_w ? rms_apply(v, srow, __ldg(norm_w + c)) : v;
+  };
   uint4 held[CH > 0 ? CH : 1];
   float amax = 0.f;
   auto fold = [&](const uint4& v) {
@@ -384,12 +430,12 @@ __global__ void __launch_bounds__(256) k_act_quant(const uint4* __restrict__ X, 
 #pragma unroll
     for (int i = 0; i < CH; ++i) {
       const int c = slot + 32 * WPR * i;
-      held[i] = c < chunks ? __ldg(xrow + c) : make_uint4(0u, 0u, 0u, 0u);
+      held[i] = c < chunks ? fetch_x(c) : make_uint4(0u, 0u, 0u, 0u);
     }
 #pragma unroll
     for (int i = 0; i < CH; ++i) fold(held[i]);
   } else {
-    for (int c = slot; c < chunks; c += 32 * WPR) fold(__ldg(xrow + c));
+    for (int c = slot; c < chunks; c += 32 * WPR) fold(fetch_x(c));
   }
   int p = t;
   if (E > 1) {
@@ -451,7 +497,7 @@ __global__ void __launch_bounds__(256) k_act_quant(const uint4* __restrict__ X, 
       if (c < chunks) emit(c, held[i]);
     }
   } else {
-    for (int c = slot; c < chunks; c += 32 * WPR) emit(c, __ldg(xrow + c));
+    for (int c = slot; c < chunks; c += 32 * WPR) emit(c, fetch_x(c));
   }
 }
 
@@ -741,18 +787,24 @@ cudaError_t launch_pack(const float* W, int N, int K, uint32_t* bits, int8_t* s8
 }
 
 cudaError_t launch_route_and_quant(const uint16_t* X, const uint16_t* Wr, int T, int K, int E, const SavedPtrs& sv, const FwdScratch& sc,
-                                   cudaStream_t st, cudaStream_t st_quant) {
+                                   cudaStream_t st, cudaStream_t st_quant, const uint16_t* norm_weight, float norm_eps) {
   if (E > 1) st_quant = st;   // the sorted position of a token comes from the router and the scan
+  const uint4* nw = reinterpret_cast<const uint4*>(norm_weight);
+  if (nw) {
+    st_quant = st;
+    LaunchScope ls(KID_ROUTER, st);
+    launch_pdl(k_row_rms, (T + 7) / 8, 256, 0, st, reinterpret_cast<const uint4*>(X), T, K, norm_eps, sc.rms);
+  }
   const int nblocks = (T + kRouterTokensPerBlock - 1) / kRouterTokensPerBlock;
   if (E > 1) {
     LaunchScope ls(KID_ROUTER, st);
     // two tokens per warp (half the loads and unpacking of Wr per token), 512 threads
     if (E <= 4) launch_pdl(k_router<4, 4>, nblocks, 8 * kRouterTokensPerBlock, 0, st, reinterpret_cast<const uint4*>(X), reinterpret_cast<const uint4*>(Wr), T, K, E,
-                           sv.expert, sc.gate_tok, sc.probs_tok, sc.block_counts);
+                           sv.expert, sc.gate_tok, sc.probs_tok, sc.block_counts, nw, sc.rms);
     else if (E <= 8) launch_pdl(k_router<8, 4>, nblocks, 8 * kRouterTokensPerBlock, 0, st, reinterpret_cast<const uint4*>(X), reinterpret_cast<const uint4*>(Wr), T, K, E,
-                                sv.expert, sc.gate_tok, sc.probs_tok, sc.block_counts);
+                                sv.expert, sc.gate_tok, sc.probs_tok, sc.block_counts, nw, sc.rms);
     else launch_pdl(k_router<kMaxExperts, 2>, nblocks, 16 * kRouterTokensPerBlock, 0, st, reinterpret_cast<const uint4*>(X), reinterpret_cast<const uint4*>(Wr), T, K, E,
-                    sv.expert, sc.gate_tok, sc.probs_tok, sc.block_counts);
+                    sv.expert, sc.gate_tok, sc.probs_tok, sc.block_counts, nw, sc.rms);
   }
   { LaunchScope ls(KID_ROUTE_SCAN, st);
   launch_pdl(k_route_scan, 1, 512, 0, st, T, E, nblocks, sc.block_counts, sc.block_base, sv.offsets, sv.rt); }
@@ -767,7 +819,7 @@ cudaError_t launch_route_and_quant(const uint16_t* X, const uint16_t* Wr, int T,
   const int rows_per_block = 8 / wpr;
   launch_pdl(kern, (T + rows_per_block - 1) / rows_per_block, 256, 0, st_quant, reinterpret_cast<const uint4*>(X), T, K, E, sv.expert, sc.block_base, sv.offsets, sc.gate_tok,
                                     sc.probs_tok, reinterpret_cast<uint2*>(sv.q), reinterpret_cast<uint4*>(sv.xt),
-                                    reinterpret_cast<uint4*>(sv.xs), sv.gamma, sv.gate, sv.probs, sv.perm, sv.pos);
+                                    reinterpret_cast<uint4*>(sv.xs), sv.gamma, sv.gate, sv.probs, sv.perm, sv.pos, nw, sc.rms);
   return cudaGetLastError();
 }
 

@@ -62,6 +62,7 @@ struct FwdScratch {
   float* probs_tok;
   int* block_counts;
   int* block_base;
+  float* rms;          // [T] per-token factor of a fused RMSNorm
 };
 
 // Launch with programmatic stream serialisation: the kernel may be scheduled while its predecessor in the stream is
@@ -82,8 +83,10 @@ inline void launch_pdl(void (*kernel)(KArgs...), int grid, int block, size_t sme
 // elementwise launchers (pq_elementwise.cu)
 cudaError_t launch_pack(const float* W, int N, int K, uint32_t* bits, int8_t* s8, float* scales, double* partial, cudaStream_t st);
 // st_quant: the stream of the quantisation kernel; it may differ from st only when E == 1 (no routing to wait for)
+// norm_weight != nullptr: X is un-normalised and RMSNorm (gain [K] bf16, epsilon) is applied on the fly; the sorted copy
+// xs of the tokens is then written even without routing (it is the only place the normalised activation exists)
 cudaError_t launch_route_and_quant(const uint16_t* X, const uint16_t* Wr, int T, int K, int E, const SavedPtrs& sv, const FwdScratch& sc,
-                                   cudaStream_t st, cudaStream_t st_quant);
+                                   cudaStream_t st, cudaStream_t st_quant, const uint16_t* norm_weight = nullptr, float norm_eps = 0.f);
 cudaError_t launch_scatter_rows(const uint16_t* src, uint16_t* dst, const int* pos, int T, int row_elems, cudaStream_t st);
 // arrivals: counter of the call's k_finalize_scales launch, cleared here (null: nothing to clear)
 cudaError_t launch_scaled_sign(const int8_t* s8, uint16_t* out, const float* beta, int beta_stride, int N, int K, unsigned* arrivals,

@@ -32,11 +32,13 @@ class PQLinear:
     any kernel wrote outside the bytes it was given.  (torch's caching allocator rounds sizes up, so an
     overrun of an exact-size tensor would otherwise land in slack nobody looks at.)"""
 
-    def __init__(self, T, K, N, r=0, E=0, scale_vector=False, device="cuda:0", training=True, dump_acc=False, guard=False):
+    def __init__(self, T, K, N, r=0, E=0, scale_vector=False, device="cuda:0", training=True, dump_acc=False, guard=False,
+                 fused_rmsnorm=False):
         self.dev = torch.device(device)
         self.T, self.K, self.N, self.r, self.E = T, K, N, r, (E if r > 0 else 0)
         self.scale_vector = scale_vector
-        self.desc = pqb.make_desc(T, K, N, r, self.E, 1, scale_vector)
+        self.desc = pqb.make_desc(T, K, N, r, self.E, 1, scale_vector, fused_rmsnorm=fused_rmsnorm and training)
+        self.fused_rmsnorm = fused_rmsnorm and training
         self.guard = guard
         self._guards = []
         self.w_bits = self._buf((N, K // 32), torch.int32)
@@ -134,6 +136,10 @@ class PQLinear:
         return pqb.pq_decode_view_init(self.desc, self.ws_decode)
 
     def forward(self, X=None, Y=None):
+        if self.fused_rmsnorm:      # X is the un-normalised activation; norm_weight / norm_eps set by the caller
+            pqb.pq_linear_forward_rms(self.desc, self.X if X is None else X, self.norm_weight, self.norm_eps, self.w_s8, self.w_scales,
+                                      self.A, self.B, self.Wr, self.alpha, self.beta, self.Y if Y is None else Y, self.saved, self.ws_fwd)
+            return self.Y if Y is None else Y
         pqb.pq_linear_forward(self.desc, self.X if X is None else X, self.w_bits, self.w_s8, self.w_scales, self.A, self.B,
                               self.Wr, self.alpha, self.beta, self.Y if Y is None else Y, self.saved, self.ws_fwd)
         return self.Y if Y is None else Y

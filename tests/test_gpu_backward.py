@@ -278,3 +278,51 @@ def test_few_tokens_routed(T):
     assert np.array_equal(sv["perm"].cpu().numpy(), f["perm"])
     assert rel_err(f32(L.Y), f["Y"]) <= TOL_BF16
     check_backward(c, L, f, g, False)
+
+
+@pytest.mark.parametrize("shape", [dict(T=333, K=384, N=544, r=64, E=1), dict(T=1000, K=512, N=768, r=128, E=8),
+                                   dict(T=200, K=256, N=320, r=0, E=0), dict(T=200, K=4096, N=64, r=16, E=4),
+                                   dict(T=70, K=8704, N=64, r=0, E=0)])
+def test_training_path_with_fused_rmsnorm(shape):
+    # App. A: RMSNorm fused in front of the quantiser, training-size path.  X is un-normalised (rows stretched by very
+    # different factors); codes, scales and routing must equal the oracle's norm-then-layer exactly, the gradients are
+    # those with respect to the normalised activation.
+    c = I.make_linear_case(shape["T"], shape["K"], shape["N"], shape["r"], shape["E"], seed=27)
+    rng = np.random.default_rng(6)
+    c["X"] = I.bf16_values(c["X"] * rng.uniform(0.25, 6.0, size=(c["T"], 1)).astype(np.float32))
+    w = I.bf16_values(1.0 + 0.1 * rng.standard_normal(c["K"]).astype(np.float32))
+    eps = 1e-5
+    Xn = O.rmsnorm(c["X"], w, eps)
+    f = O.linear_forward(Xn, c["W"], c["A"], c["B"], c["Wr"], c["alpha"], c["beta"])
+    g = O.linear_backward(c["dY"], Xn, f, c["A"], c["B"], c["Wr"], c["alpha"], c["beta"])
+    L = PQLinear(c["T"], c["K"], c["N"], c["r"], c["E"], fused_rmsnorm=True, guard=True).load_case(c)
+    L.norm_weight = torch.from_numpy(w).to(L.X.device).to(torch.bfloat16)
+    L.norm_eps = eps
+    L.pack()
+    L.forward()
+    L.backward()
+    torch.cuda.synchronize()
+    check_status()
+    assert L.check_guards() == 0
+    sv = L.saved_view()
+    perm = sv["perm"].cpu().numpy()
+    assert np.array_equal(sv["q"].cpu().numpy(), f["q"][perm])
+    assert np.array_equal(f32(sv["gamma"]), f["gamma"][perm])
+    assert np.array_equal(f32(sv["xs"]), Xn[perm])                      # the normalised activation, bit for bit
+    if c["E"] > 1:
+        assert np.array_equal(sv["expert"].cpu().numpy(), f["idx"])
+    assert rel_err(f32(L.Y), f["Y"]) <= TOL_BF16 and rms_err(f32(L.Y), f["Y"]) <= TOL_RMS
+    check_backward(c, L, f, g, False)
+    # and it is not the layer applied to the un-normalised input
+    f_raw = O.linear_forward(c["X"], c["W"], c["A"], c["B"], c["Wr"], c["alpha"], c["beta"])
+    assert not np.array_equal(f_raw["q"], f["q"])
+
+
+def test_fused_rmsnorm_flag_and_arguments_must_agree():
+    c = I.make_linear_case(128, 64, 64, 32, 1, seed=1)
+    L = PQLinear(128, 64, 64, 32, 1).load_case(c)           # desc without the flag
+    L.pack()
+    w = torch.ones(64, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(pqb.PqError) as ei:
+        pqb.pq_linear_forward_rms(L.desc, L.X, w, 1e-5, L.w_s8, L.w_scales, L.A, L.B, None, L.alpha, L.beta, L.Y, L.saved, L.ws_fwd)
+    assert ei.value.status == pqb.PQ_ERR_NULL
