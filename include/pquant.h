@@ -288,8 +288,28 @@ typedef struct pq_decode_item {
    * an all-zero token would divide by zero). */
   const uint16_t* norm_weight;
   float norm_eps;
+  /* The weights in the layout of the streaming decode kernel (pq_pack_decode), or NULL.  When every item of a
+   * launch group carries them (w_bits_il, and B_il if r > 0), the group runs as ONE cooperative kernel that
+   * streams each weight byte once with coalesced loads; results: the same integers (codes, routing, sums over k),
+   * Y within the tolerance of the float epilogue (the expert product is summed in another order).  Otherwise, and
+   * for shapes that kernel does not take (r not a multiple of 8), the two-kernel path is used.  w_bits, A and B
+   * are needed in both cases (the rows of A_e are read in their natural layout). */
+  const uint32_t* w_bits_il;
+  const uint16_t* B_il;
 } pq_decode_item;
 int pq_decode_batch(const pq_decode_item* items, int n, void* stream);
+
+/* Weight layout of the streaming decode kernel (App. A: at batch size one the layer's cost is the bytes of its
+ * weights, so they are stored the way the kernel reads them; the paper's CPU kernels permute weights offline in the
+ * same spirit).  One-time, per linear:
+ *   w_bits_il: [ceil(N/128)][ceil(K/128)][4][32][4] uint32 -- for row group g and chunk c of 128 contraction values,
+ *     lane l's j-th feature 128 g + 32 j + l holds its four bit words 4 c .. 4 c + 3 (zero beyond N or K);
+ *   B_il: [E][4 ceil(N/128)][r/8][32][8] bf16 -- for a group of 32 features, lane l holds 8 consecutive hidden values
+ *     of row 32 group + l of B_e (zero beyond N).
+ * pq_decode_pack_bytes gives the two sizes in bytes (b_il_bytes = 0 when r = 0).  r must be a multiple of 8
+ * (PQ_ERR_SHAPE).  d->T is not used. */
+int pq_decode_pack_bytes(const pq_desc* d, size_t* bits_il_bytes, size_t* b_il_bytes);
+int pq_pack_decode(const pq_desc* d, const uint32_t* w_bits, const uint16_t* B, uint32_t* w_bits_il, uint16_t* B_il, void* stream);
 
 /* Straight-through backward (App. B.1): Sign, Round and Clip pass the gradient
  * unchanged; mu, lam, gamma are constants.  Every gradient is OVERWRITTEN.
@@ -350,8 +370,11 @@ int pq_device_status(void* stream, int* code, int* where);
  *   flight finish, releases its TMEM and returns; pq_device_status then reports PQ_ERR_TIMEOUT and the
  *   outputs of that call are undefined.  Applies to the current device; blocks until the device's
  *   earlier work has finished.  Meant for pq_debug_gemm; do not shorten the limit around the decode
- *   entry points, whose later stages read indices an abandoned stage has not delivered. */
-enum { PQ_OPT_DECODE_PDL = 1, PQ_OPT_SIDE_STREAM = 2, PQ_OPT_SPIN_CYCLES = 3 };
+ *   entry points, whose later stages read indices an abandoned stage has not delivered.
+ *   PQ_OPT_DECODE_STREAM (default 1): 0 = pq_decode_batch ignores w_bits_il / B_il and always uses the two-kernel path.
+ *   PQ_OPT_DECODE_PREFETCH (default 1): the streaming decode kernel asks for its sign bits to be brought into L2
+ *   while it prepares the tokens. */
+enum { PQ_OPT_DECODE_PDL = 1, PQ_OPT_SIDE_STREAM = 2, PQ_OPT_SPIN_CYCLES = 3, PQ_OPT_DECODE_STREAM = 4, PQ_OPT_DECODE_PREFETCH = 5 };
 int pq_set_option(int option, int value);
 
 /* Cumulative number of kernels this library has launched in this process. */

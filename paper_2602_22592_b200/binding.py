@@ -23,12 +23,12 @@ PQ_FUSED_RMSNORM = 8
 PQ_PHASE_PACK, PQ_PHASE_FWD, PQ_PHASE_BWD, PQ_PHASE_DECODE = 0, 1, 2, 3
 
 EXPORTS = ("pq_status_string", "pq_workspace_bytes", "pq_saved_bytes", "pq_saved_view_init",
-           "pq_decode_view_init", "pq_bwd_view_init", "pq_decode_batch", "pq_pack_weights", "pq_pack_weights_static", "pq_pack_experts", "pq_linear_forward", "pq_linear_forward_hp8", "pq_linear_forward_rms", "pq_ffn_workspace_bytes", "pq_ffn_forward", "pq_ffn_view_init", "pq_linear_backward", "pq_debug_gemm", "pq_debug_gemm_tile",
+           "pq_decode_view_init", "pq_bwd_view_init", "pq_decode_batch", "pq_decode_pack_bytes", "pq_pack_decode", "pq_pack_weights", "pq_pack_weights_static", "pq_pack_experts", "pq_linear_forward", "pq_linear_forward_hp8", "pq_linear_forward_rms", "pq_ffn_workspace_bytes", "pq_ffn_forward", "pq_ffn_view_init", "pq_linear_backward", "pq_debug_gemm", "pq_debug_gemm_tile",
            "pq_device_status", "pq_kernel_launches", "pq_profile_events", "pq_set_option")
 
 KERNEL_IDS = dict(pack_sums=0, binarize_pack=1, router=2, route_scan=3, act_quant=4, hp_up=5, fwd=6, scatter_rows=7,
                   scaled_sign=8, scaled_b=9, hp_dh=10, bwd_dx=11, bwd_dw=12, hp_db=13, hp_da=14, router_wgrad=15,
-                  sum_partials=16, sum_scalar=17, debug=18, decode_prep=19, decode_main=20, reduce_db=21, reduce_da=22)
+                  sum_partials=16, sum_scalar=17, debug=18, decode_prep=19, decode_main=20, reduce_db=21, reduce_da=22, decode_pack=23, decode_stream=24)
 
 
 class PqError(RuntimeError):
@@ -52,7 +52,8 @@ class pq_saved_view(ctypes.Structure):
 class pq_decode_item(ctypes.Structure):
     _fields_ = [("desc", pq_desc)] + [(n, ctypes.c_void_p) for n in
                                       ("X", "w_bits", "w_scales", "A", "B", "Wr", "alpha", "beta", "Y", "ws")] + [
-        ("ws_bytes", ctypes.c_size_t), ("norm_weight", ctypes.c_void_p), ("norm_eps", ctypes.c_float)]
+        ("ws_bytes", ctypes.c_size_t), ("norm_weight", ctypes.c_void_p), ("norm_eps", ctypes.c_float),
+        ("w_bits_il", ctypes.c_void_p), ("B_il", ctypes.c_void_p)]
 
 
 class pq_decode_view(ctypes.Structure):
@@ -104,6 +105,10 @@ def lib() -> ctypes.CDLL:
         L.pq_pack_weights_static.argtypes = [dp, vp, vp, vp, vp, vp]
         L.pq_pack_experts.restype = ci
         L.pq_pack_experts.argtypes = [dp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.pq_decode_pack_bytes.restype = ci
+        L.pq_decode_pack_bytes.argtypes = [dp, ctypes.POINTER(sz), ctypes.POINTER(sz)]
+        L.pq_pack_decode.restype = ci
+        L.pq_pack_decode.argtypes = [dp, vp, vp, vp, vp, vp]
         L.pq_linear_forward.restype = ci
         L.pq_linear_forward.argtypes = [dp] + [vp] * 10 + [vp, sz, vp, sz, vp]
         L.pq_linear_forward_rms.restype = ci
@@ -297,8 +302,9 @@ def pq_ffn_view_init(d: pq_ffn_desc, ws: torch.Tensor) -> dict:
 
 
 def make_decode_items(entries):
-    """ctypes array of pq_decode_item from (desc, X, w_bits, w_scales, A, B, Wr, alpha, beta, Y, ws[, norm_weight, norm_eps])
-    tuples of tensors (the last two: bf16 RMSNorm gain [K] and its epsilon, for un-normalised X).
+    """ctypes array of pq_decode_item from (desc, X, w_bits, w_scales, A, B, Wr, alpha, beta, Y, ws[, norm_weight, norm_eps
+    [, w_bits_il, B_il]]) tuples of tensors (norm_weight, norm_eps: bf16 RMSNorm gain [K] and its epsilon, for un-normalised X;
+    w_bits_il, B_il: the weights as laid out by pq_pack_decode).
     The array only holds pointers: keep the tensors alive while it is in use."""
     arr = (pq_decode_item * len(entries))()
     for i, entry in enumerate(entries):
@@ -306,12 +312,26 @@ def make_decode_items(entries):
         norm_weight, norm_eps = (entry[11], entry[12]) if len(entry) > 11 else (None, 0.0)
         arr[i].norm_weight = None if norm_weight is None else norm_weight.data_ptr()
         arr[i].norm_eps = float(norm_eps)
+        w_bits_il, B_il = (entry[13], entry[14]) if len(entry) > 13 else (None, None)
+        arr[i].w_bits_il = None if w_bits_il is None else w_bits_il.data_ptr()
+        arr[i].B_il = None if B_il is None else B_il.data_ptr()
         arr[i].desc = d
         for name, t in (("X", X), ("w_bits", w_bits), ("w_scales", w_scales), ("A", A), ("B", B), ("Wr", Wr), ("alpha", alpha),
                         ("beta", beta), ("Y", Y), ("ws", ws)):
             setattr(arr[i], name, None if t is None else t.data_ptr())
         arr[i].ws_bytes = _nbytes(ws)
     return arr
+
+
+def pq_decode_pack_bytes(d) -> tuple[int, int]:
+    a, b = ctypes.c_size_t(0), ctypes.c_size_t(0)
+    _check("pq_decode_pack_bytes", lib().pq_decode_pack_bytes(ctypes.byref(d), ctypes.byref(a), ctypes.byref(b)))
+    return a.value, b.value
+
+
+def pq_pack_decode(d, w_bits, B, w_bits_il, B_il, stream=None):
+    """Lay the sign bits and the rows of B_e out for the streaming decode kernel (one-time, per linear)."""
+    _check("pq_pack_decode", lib().pq_pack_decode(ctypes.byref(d), _ptr(w_bits), _ptr(B), _ptr(w_bits_il), _ptr(B_il), _stream(stream)))
 
 
 def pq_decode_batch(items, stream=None):
@@ -344,6 +364,8 @@ def pq_device_status(stream=None) -> tuple[int, int]:
 PQ_OPT_DECODE_PDL = 1
 PQ_OPT_SIDE_STREAM = 2
 PQ_OPT_SPIN_CYCLES = 3
+PQ_OPT_DECODE_STREAM = 4
+PQ_OPT_DECODE_PREFETCH = 5
 
 
 def pq_set_option(option: int, value: int):

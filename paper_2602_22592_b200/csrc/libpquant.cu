@@ -3,4 +3,5 @@
 #include "pq_elementwise.cu"
 #include "pq_gemm_kernels.cu"
 #include "pq_decode.cu"
+#include "pq_decode_stream.cu"
 #include "pq_api.cu"

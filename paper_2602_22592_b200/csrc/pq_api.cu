@@ -282,7 +282,8 @@ size_t pq_workspace_bytes(const pq_desc* d, int phase) {
       return carve_bwd_scratch(d, nullptr, nullptr);
     case PQ_PHASE_DECODE:
       if (check_desc(d, false) != PQ_OK || d->T > 16) return 0;
-      return decode_workspace_bytes(d->T, d->K, d->N, d->r, (d->flags & PQ_DECODE_DUMP_ACC) != 0);
+      return decode_workspace_bytes(d->T, d->K, d->N, d->r, (d->flags & PQ_DECODE_DUMP_ACC) != 0) +
+             decode_stream_extra_bytes(d->T, d->K, d->N, d->r);
     default: return 0;
   }
 }
@@ -570,6 +571,25 @@ int pq_ffn_forward(const pq_ffn_desc* d, const uint16_t* X, const int8_t* g_s8, 
                       hp_scales + 1, nullptr, alpha, beta, Y, c.saved_d, c.saved_d_bytes, c.ws_fwd, c.ws_fwd_bytes, stream, true);
 }
 
+int pq_decode_pack_bytes(const pq_desc* d, size_t* bits_il_bytes, size_t* b_il_bytes) {
+  if (!d || !bits_il_bytes || !b_il_bytes) return PQ_ERR_NULL;
+  int rc = check_desc(d, false);
+  if (rc) return rc;
+  if (d->r % 8) return PQ_ERR_SHAPE;
+  decode_pack_sizes(d->K, d->N, d->r, experts_of(d), bits_il_bytes, b_il_bytes);
+  return PQ_OK;
+}
+
+int pq_pack_decode(const pq_desc* d, const uint32_t* w_bits, const uint16_t* B, uint32_t* w_bits_il, uint16_t* B_il, void* stream) {
+  if (!d || !w_bits || !w_bits_il) return PQ_ERR_NULL;
+  int rc = check_desc(d, false);
+  if (rc) return rc;
+  if (d->r % 8) return PQ_ERR_SHAPE;
+  if (d->r > 0 && (!B || !B_il)) return PQ_ERR_NULL;
+  if (misaligned(w_bits) || misaligned(B) || misaligned(w_bits_il) || misaligned(B_il)) return PQ_ERR_ALIGN;
+  return decode_pack(d->K, d->N, d->r, experts_of(d), w_bits, B, w_bits_il, B_il, static_cast<cudaStream_t>(stream));
+}
+
 int pq_decode_batch(const pq_decode_item* items, int n, void* stream) {
   if (!items) return PQ_ERR_NULL;
   if (n < 1 || n > 4096) return PQ_ERR_SHAPE;
@@ -587,6 +607,12 @@ int pq_decode_batch(const pq_decode_item* items, int n, void* stream) {
     if (misaligned(it.norm_weight)) { rc = PQ_ERR_ALIGN; break; }
     if (it.norm_weight && !(it.norm_eps > 0.f)) { rc = PQ_ERR_SHAPE; break; }   // an all-zero token needs it
     args[i].norm_weight = it.norm_weight; args[i].norm_eps = it.norm_eps;
+    if (it.w_bits_il) {
+      if (misaligned(it.w_bits_il) || misaligned(it.B_il)) { rc = PQ_ERR_ALIGN; break; }
+      if (d->r > 0 && !it.B_il) { rc = PQ_ERR_NULL; break; }
+      if (it.ws_bytes < pq_workspace_bytes(d, PQ_PHASE_DECODE)) { rc = PQ_ERR_WORKSPACE; break; }
+      args[i].bits_il = it.w_bits_il; args[i].B_il = it.B_il;
+    }
   }
   if (rc == PQ_OK) rc = decode_batch(args, n, static_cast<cudaStream_t>(stream));
   delete[] args;
@@ -673,6 +699,8 @@ int pq_set_option(int option, int value) {
   switch (option) {
     case PQ_OPT_DECODE_PDL: decode_set_pdl(value); return PQ_OK;
     case PQ_OPT_SIDE_STREAM: g_side_streams = value ? 1 : 0; return PQ_OK;
+    case PQ_OPT_DECODE_STREAM: decode_stream_enable(value); return PQ_OK;
+    case PQ_OPT_DECODE_PREFETCH: decode_stream_prefetch(value); return PQ_OK;
     case PQ_OPT_SPIN_CYCLES: {
       // the limit lives in constant memory of the current device; the copy is ordered after everything
       // already enqueued there (a blocking copy), so no running kernel sees it change
@@ -703,6 +731,9 @@ int pq_device_status(void* stream, int* code, int* where) {
   if (host[0] != 0) {
     const int zero[2] = {0, 0};
     if (cudaMemcpyToSymbol(g_status, zero, sizeof(zero)) != cudaSuccess) return PQ_ERR_CUDA;
+    // a kernel that gave up may have left the decode kernel's grid barrier half counted
+    if (cudaDeviceSynchronize() != cudaSuccess) return PQ_ERR_CUDA;
+    decode_stream_reset();
   }
   return PQ_OK;
 }

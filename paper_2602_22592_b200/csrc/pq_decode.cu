@@ -797,7 +797,14 @@ static int decode_launch(const DecodeItemArgs* items, int n, cudaStream_t st) {
 int decode_batch(const DecodeItemArgs* items, int n, cudaStream_t st) {
   for (int i = 0; i < n; i += kDecodeMaxBatch) {
     const int m = n - i < kDecodeMaxBatch ? n - i : kDecodeMaxBatch;
-    const int rc = decode_launch(items + i, m, st);
+    // the streaming kernel takes a group whose items all carry its weight layout; otherwise the kernels above
+    int rc = PQ_ERR_UNSUPPORTED;
+    if (decode_stream_enabled()) {
+      bool all = true;
+      for (int k = 0; k < m; ++k) all = all && items[i + k].bits_il != nullptr;
+      if (all) rc = decode_stream_launch(items + i, m, st);
+    }
+    if (rc == PQ_ERR_UNSUPPORTED) rc = decode_launch(items + i, m, st);
     if (rc) return rc;
   }
   return PQ_OK;

@@ -17,7 +17,7 @@ constexpr float kActAmaxFloor = 1e-5f;     // all-zero row guard
 enum KernelId : int {
   KID_PACK_SUMS = 0, KID_BINARIZE_PACK, KID_ROUTER, KID_ROUTE_SCAN, KID_ACT_QUANT, KID_HP_UP, KID_FWD, KID_SCATTER_ROWS,
   KID_SCALED_SIGN, KID_SCALED_B, KID_HP_DH, KID_BWD_DX, KID_BWD_DW, KID_HP_DB, KID_HP_DA, KID_ROUTER_WGRAD, KID_SUM_PARTIALS,
-  KID_SUM_SCALAR, KID_DEBUG, KID_DECODE_PREP, KID_DECODE_MAIN, KID_REDUCE_DB, KID_REDUCE_DA, KID_COUNT
+  KID_SUM_SCALAR, KID_DEBUG, KID_DECODE_PREP, KID_DECODE_MAIN, KID_REDUCE_DB, KID_REDUCE_DA, KID_DECODE_PACK, KID_DECODE_STREAM, KID_COUNT
 };
 struct ProfileSlot { cudaEvent_t start, stop; };
 extern ProfileSlot g_profile[KID_COUNT];
@@ -129,7 +129,18 @@ struct DecodeItemArgs {
   LayerArgs a; const uint16_t* X; const uint32_t* bits; uint16_t* Y; void* ws; bool dump;
   const uint16_t* norm_weight = nullptr;   // RMSNorm gain [K] bf16, or null: X arrives normalised
   float norm_eps = 0.f;
+  const uint32_t* bits_il = nullptr;       // weights laid out by decode_pack (streaming kernel), or null
+  const uint16_t* B_il = nullptr;
 };
+// streaming decode kernel (pq_decode_stream.cu)
+void decode_pack_sizes(int K, int N, int r, int E, size_t* bits_bytes, size_t* b_bytes);
+int decode_pack(int K, int N, int r, int E, const uint32_t* bits, const uint16_t* B, uint32_t* bits_il, uint16_t* B_il, cudaStream_t st);
+size_t decode_stream_extra_bytes(int M, int K, int N, int r);
+int decode_stream_launch(const DecodeItemArgs* items, int n, cudaStream_t st);   // PQ_ERR_UNSUPPORTED: use the other kernels
+void decode_stream_enable(int on);
+void decode_stream_prefetch(int on);
+bool decode_stream_enabled();
+void decode_stream_reset();
 int decode_batch(const DecodeItemArgs* items, int n, cudaStream_t st);   // independent linears, launched together
 void decode_set_pdl(int on);
 DecodeViewPtrs decode_view(int M, int K, int N, int r, void* ws, bool dump);

@@ -73,6 +73,7 @@ class PQLinear:
             self.ws_decode = self._buf((max(nb, 16),), torch.uint8).zero_() if T <= 16 else None
             self.Y = self._buf((T, N), torch.bfloat16)
         self.X = self.W = self.A = self.B = self.Wr = self.alpha = self.beta = self.dY = None
+        self.w_bits_il = self.B_il = None
 
     # -- buffers --------------------------------------------------------------
     def _buf(self, shape, dtype):
@@ -110,13 +111,28 @@ class PQLinear:
         return self
 
     # -- calls --------------------------------------------------------------
+    stream_decode = True   # decode layers also get the streaming kernel's weight layout when they are packed
+
     def pack(self, bits_only=False):
         pqb.pq_pack_weights(self.desc, self.W, self.w_bits, None if bits_only else self.w_s8, self.w_scales, self.ws_pack)
+        if not self.training and PQLinear.stream_decode and self.T <= 16 and (self.r == 0 or self.B is not None):
+            self.pack_decode()
+
+    def pack_decode(self):
+        """Lay the packed bits and B out for the streaming decode kernel (after pack() and load_case()); decode() and
+        decode_entry() then hand both layouts to the library.  Returns False when the shape has no such layout."""
+        if self.r % 8:
+            return False
+        nb, nB = pqb.pq_decode_pack_bytes(self.desc)
+        self.w_bits_il = self._buf((nb,), torch.uint8)
+        self.B_il = self._buf((nB,), torch.uint8) if nB else None
+        pqb.pq_pack_decode(self.desc, self.w_bits, self.B, self.w_bits_il, self.B_il)
+        return True
 
     def decode(self, X=None, Y=None):
         """Inference forward from the packed sign bits (w_s8 is not used).  With `norm_weight` set, X is the
         un-normalised activation and RMSNorm is fused in front of the quantiser (a batch of one)."""
-        if getattr(self, "norm_weight", None) is not None:
+        if getattr(self, "norm_weight", None) is not None or self.w_bits_il is not None:
             entry = list(self.decode_entry())
             if X is not None: entry[1] = X
             if Y is not None: entry[9] = Y
@@ -130,7 +146,7 @@ class PQLinear:
     def decode_entry(self):
         """This layer's arguments as one entry for binding.make_decode_items."""
         return (self.desc, self.X, self.w_bits, self.w_scales, self.A, self.B, self.Wr, self.alpha, self.beta, self.Y, self.ws_decode,
-                getattr(self, "norm_weight", None), getattr(self, "norm_eps", 0.0))
+                getattr(self, "norm_weight", None), getattr(self, "norm_eps", 0.0), self.w_bits_il, self.B_il)
 
     def decode_view(self) -> dict:
         return pqb.pq_decode_view_init(self.desc, self.ws_decode)

@@ -13,6 +13,14 @@ from test_gpu_forward import TOL_BF16, check_status, f32, rel_err
 pytestmark = pytest.mark.gpu
 
 
+@pytest.fixture(autouse=True, params=["stream", "pair"])
+def decode_kernels(request):
+    """Every test runs twice: on the streaming kernel (weights in its own layout) and on the two-kernel path."""
+    PQLinear.stream_decode = request.param == "stream"
+    yield request.param
+    PQLinear.stream_decode = True
+
+
 def run_decode(c, scale_vector=False):
     L = PQLinear(c["T"], c["K"], c["N"], c["r"], c["E"], scale_vector=scale_vector, training=False, dump_acc=True).load_case(c)
     L.pack(bits_only=True)
