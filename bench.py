@@ -533,6 +533,10 @@ def build_decode_weights(ctx):
                              A=(torch.randn((E, r, K), generator=gen, device=device) * 0.02).to(torch.bfloat16),
                              B=(torch.randn((E, N, r), generator=gen, device=device) * 0.02).to(torch.bfloat16),
                              norm_weight=(1.0 + 0.1 * torch.randn((K,), generator=gen, device=device)).to(torch.bfloat16)))
+            # the same weights in the streaming decode kernel's layout (one-time, like the pack itself)
+            L.B = sets[-1]["B"]
+            L.pack_decode()
+            sets[-1]["w_bits_il"], sets[-1]["B_il"] = L.w_bits_il, L.B_il
             del L
     torch.cuda.synchronize()
     return sets
@@ -548,6 +552,8 @@ def make_decode_layers(ctx, M, weights, rmsnorm=False):
         act = I.decode_activations(M, w["K"], w["E"], seed=w["seed"])
         L.w_bits, L.w_scales, L.A, L.B = w["w_bits"], w["w_scales"], w["A"], w["B"]
         L.w_s8 = None
+        if ctx.decode_kernels == "stream":
+            L.w_bits_il, L.B_il = w["w_bits_il"], w["B_il"]
         L.X = torch.from_numpy(act["X"]).to(device).to(torch.bfloat16)
         L.Wr = torch.from_numpy(act["Wr"]).to(device).to(torch.bfloat16)
         L.alpha = torch.full((1,), 2.0, device=device)
@@ -860,6 +866,8 @@ def main():
     ap.add_argument("--decode-tokens", type=int, default=1, choices=range(1, 17), metavar="M")
     ap.add_argument("--decode-skip-serial", action="store_true", help="time only the batched graph (shorter runs under a profiler)")
     ap.add_argument("--decode-batch", type=int, default=16, help="independent decode linears per pq_decode_batch call")
+    ap.add_argument("--decode-kernels", default="stream", choices=["stream", "pair"],
+                    help="stream: the cooperative streaming kernel on weights in its own layout; pair: the two-kernel path on the plain layout")
     ap.add_argument("--decode-rmsnorm", action="store_true", help="decode from un-normalised activations, RMSNorm fused into the token preparation")
     ap.add_argument("--decoder-one-form", action="store_true", help="decoder workload: only the form with 8 experts on every projection")
     ap.add_argument("--cpu-tokens", type=int, default=8192, help="tokens per step of the CPU oracle (cpu_baseline and --impl reference)")
@@ -875,6 +883,7 @@ def main():
         run_reference(args)
         return
     ctx = Ctx()
+    ctx.decode_kernels = args.decode_kernels
     if args.workload == "decode":
         run_decode(args, ctx)
     elif args.workload == "decoder":

@@ -9,15 +9,20 @@
 // The kernel has two phases with one grid-wide barrier between them (hence the cooperative launch: every CTA
 // is resident, one per SM):
 //   phase 1  the CTAs whose share of the weight stream touches a linear split that linear's token work:
-//            RMSNorm (optional), absmax quantisation (Eq. 7-9), router (Sec. 3.3) and the rows of h = A_e x.
-//            The int8 codes go to global memory in the order the bit product reads them, h in fp32.
-//   phase 2  the chunks of all linears form one list that is cut into equal contiguous spans, one per CTA and
-//            then one per warp.  A warp multiplies its chunks (dp4a of 0/1 byte masks with the int8 codes:
-//            sum_k q S = 2 * sum_{bit set} q - sum q), adds its partial sums to an int32 accumulator in global
-//            memory and counts the chunks of the row group it has delivered; the warp that completes a row group
-//            reads the sums back, adds the expert product and writes Y (Eq. 10-11).
-// Nothing is staged through shared memory but the activations: the loads in flight live in registers, so the
-// stream needs no producer, no barriers between warps and no polling.
+//            RMSNorm (optional), absmax quantisation (Eq. 7-9), router (Sec. 3.3) and the rows of h = A_e x
+//            (every row cut into sixteen pieces, one per warp, so that a CTA with one row still has all its
+//            loads in flight at once).  The int8 codes go to global memory in the order the bit product
+//            reads them, h in fp32.
+//   phase 2  two lists of work items, each cut into equal contiguous shares, one per CTA and then one per warp:
+//            (a) the expert product z = B_e h for (token, group of 32 features): twenty coalesced loads in
+//                flight per lane, fp32 multiply-adds, z to global memory;
+//            (b) the chunks of sign bits: dp4a of 0/1 byte masks with the int8 codes
+//                (sum_k q S = 2 * sum_{bit set} q - sum q), partial sums added to an int32 accumulator in
+//                global memory.
+//            Every item reports to the counter of its row group (128 features x 8 tokens); the warp whose
+//            report completes the count reads the sums and z back and writes Y (Eq. 10-11).
+// Nothing is staged through shared memory but the activations and the router rows: the weight loads in flight
+// live in registers, so the stream needs no producer, no barriers between warps and no polling.
 #include <algorithm>
 #include <mutex>
 
@@ -49,23 +54,27 @@ struct StreamLinear {
   DecodeTokInfo* info;      // [16] expert, gate, gamma, code sum per token
   uint32_t* qg;             // [M][C * 32] words of int8 codes in bit-product order
   float* h;                 // [M][r]
+  float* z;                 // [M][G * 128] expert product
   int* acc;                 // [M][G * 128] partial sums over the set bits
-  unsigned* cnt;            // [token groups][G] chunks delivered
+  unsigned* cnt;            // [token groups][G] items reported
   int* acc_dump;            // [M, N] or null
   float norm_eps;
   int M, K, N, r, E, sstride;
   int G, C;                 // row groups; chunks per row group
-  int chunk0;               // position of this linear's first chunk in the launch-wide list
-  int cta_first, cta_count; // the CTAs whose span touches this linear
+  int chunk0;               // position of this linear's first chunk in the launch-wide list of chunks
+  int z0;                   // position of its first item in the launch-wide list of expert-product items (M * 4 G each)
+  int cta_first, cta_count; // the CTAs that share its token work
   int zero_words;           // int32 words from `acc` on that phase 1 clears (acc and cnt are adjacent)
 };
 struct StreamBatch {
   StreamLinear lin[kStreamMaxBatch];
   int n;
-  int total_chunks;
+  int total_chunks, total_z;
   int bar_slot;
   int prefetch;             // issue L2 prefetches for the span's sign bits before phase 1
-  int off_h, off_info;      // shared-memory carve-up: [x or q region][h][info]
+  int router_rows;          // router rows that fit in shared memory beside the token
+  int off_rows, off_part;   // phase 1 carve-up: [token][router rows][partial sums of h]
+  int off_h, off_info;      // phase 2 carve-up: [codes][h][token info]
 };
 
 // ---------------------------------------------------------------------------
@@ -163,6 +172,7 @@ __device__ __forceinline__ void stream_bar_depart(unsigned* bar) {
   }
 }
 
+
 // ---------------------------------------------------------------------------
 // phase 1: one token of one linear, rows [j_lo, j_hi) of h; `owner` also quantises and publishes the token
 // ---------------------------------------------------------------------------
@@ -174,15 +184,39 @@ struct StreamShared {
   int ok;
 };
 
-__device__ void stream_token(const StreamLinear& L, int t, int j_lo, int j_hi, bool owner, uint4* xs4, StreamShared& sh) {
+// copies `total` 16-byte pieces, eight loads in flight per thread: piece i goes from src(i) to dst(i)
+template <class Dst, class Src>
+__device__ __forceinline__ void stream_stage(int total, Dst dst, Src src) {
+  for (int base = threadIdx.x; base < total; base += kStreamThreads * 8) {
+    uint4 v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int i = base + u * kStreamThreads;
+      v[u] = i < total ? __ldg(src(i)) : make_uint4(0u, 0u, 0u, 0u);
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int i = base + u * kStreamThreads;
+      if (i < total) *dst(i) = v[u];
+    }
+  }
+}
+
+__device__ void stream_token(const StreamBatch& bp, const StreamLinear& L, int t, int j_lo, int j_hi, bool owner, uint8_t* smem, StreamShared& sh) {
   const int K = L.K, E = L.E, r = L.r;
   const int chunks = K >> 3;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  uint4* xs4 = reinterpret_cast<uint4*>(smem);
+  uint4* rows4 = reinterpret_cast<uint4*>(smem + bp.off_rows);
+  float* part = reinterpret_cast<float*>(smem + bp.off_part);
+  const uint4* x4 = reinterpret_cast<const uint4*>(L.X) + (long long)t * chunks;
+  const uint4* wr4 = reinterpret_cast<const uint4*>(L.Wr);
+  const int R = bp.router_rows;
   __syncthreads();   // the previous token's values are no longer read
-  {
-    const uint4* x4 = reinterpret_cast<const uint4*>(L.X) + (long long)t * chunks;
-    for (int c = threadIdx.x; c < chunks; c += kStreamThreads) xs4[c] = x4[c];
-  }
+  // the token and the first round of router rows travel together
+  const int first_rows = E > 1 ? min(R, E) : 0;
+  stream_stage(chunks * (1 + first_rows), [&](int i) { return i < chunks ? xs4 + i : rows4 + (i - chunks); },
+               [&](int i) { return i < chunks ? x4 + i : wr4 + (i - chunks); });
   __syncthreads();
   if (L.norm_w) {
     // RMSNorm in front of the quantiser (App. A): mean of squares and reciprocal root in fp64, the factor rounded
@@ -228,30 +262,30 @@ __device__ void stream_token(const StreamLinear& L, int t, int j_lo, int j_hi, b
   const float gamma = __fdiv_rn(kActQmax, fmaxf(amax, kActAmaxFloor));
 
   // router in the pinned fp32 order of the training path: lane j owns the chunks c = j mod 32, ascending, fused
-  // multiply-add; butterfly 16, 8, 4, 2, 1.  One warp per expert row, the row read straight from global memory.
+  // multiply-add; butterfly 16, 8, 4, 2, 1.  One warp per expert row of the round, out of shared memory.
   int best = 0;
   float gate = 1.0f;
   if (E > 1) {
-    for (int e = warp; e < E; e += kStreamWarps) {
-      const uint4* wrow = reinterpret_cast<const uint4*>(L.Wr) + (long long)e * chunks;
-      float acc = 0.f;
-      for (int c0 = lane; c0 < chunks; c0 += 128) {
-        uint4 wv[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) wv[u] = c0 + 32 * u < chunks ? __ldg(wrow + c0 + 32 * u) : make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          if (c0 + 32 * u < chunks) {
-            const uint4 xv = xs4[c0 + 32 * u];
-            acc = fmaf(bf16lo(xv.x), bf16lo(wv[u].x), acc); acc = fmaf(bf16hi(xv.x), bf16hi(wv[u].x), acc);
-            acc = fmaf(bf16lo(xv.y), bf16lo(wv[u].y), acc); acc = fmaf(bf16hi(xv.y), bf16hi(wv[u].y), acc);
-            acc = fmaf(bf16lo(xv.z), bf16lo(wv[u].z), acc); acc = fmaf(bf16hi(xv.z), bf16hi(wv[u].z), acc);
-            acc = fmaf(bf16lo(xv.w), bf16lo(wv[u].w), acc); acc = fmaf(bf16hi(xv.w), bf16hi(wv[u].w), acc);
-          }
-        }
+    for (int e0 = 0; e0 < E; e0 += R) {
+      const int n = min(R, E - e0);
+      if (e0 > 0) {
+        __syncthreads();   // the previous round's rows have been used
+        stream_stage(chunks * n, [&](int i) { return rows4 + i; }, [&](int i) { return wr4 + (long long)e0 * chunks + i; });
+        __syncthreads();
       }
-      for (int d = 16; d > 0; d >>= 1) acc = acc + __shfl_xor_sync(0xffffffffu, acc, d);
-      if (lane == 0) sh.logit[e] = acc;
+      for (int k = warp; k < n; k += kStreamWarps) {
+        const uint4* wrow = rows4 + (size_t)k * chunks;
+        float acc = 0.f;
+        for (int c = lane; c < chunks; c += 32) {
+          const uint4 xv = xs4[c], wv = wrow[c];
+          acc = fmaf(bf16lo(xv.x), bf16lo(wv.x), acc); acc = fmaf(bf16hi(xv.x), bf16hi(wv.x), acc);
+          acc = fmaf(bf16lo(xv.y), bf16lo(wv.y), acc); acc = fmaf(bf16hi(xv.y), bf16hi(wv.y), acc);
+          acc = fmaf(bf16lo(xv.z), bf16lo(wv.z), acc); acc = fmaf(bf16hi(xv.z), bf16hi(wv.z), acc);
+          acc = fmaf(bf16lo(xv.w), bf16lo(wv.w), acc); acc = fmaf(bf16hi(xv.w), bf16hi(wv.w), acc);
+        }
+        for (int d = 16; d > 0; d >>= 1) acc = acc + __shfl_xor_sync(0xffffffffu, acc, d);
+        if (lane == 0) sh.logit[e0 + k] = acc;
+      }
     }
     __syncthreads();
     float lmax = sh.logit[0];
@@ -264,6 +298,45 @@ __device__ void stream_token(const StreamLinear& L, int t, int j_lo, int j_hi, b
       if (e == best) pbest = pe;
     }
     gate = pbest * (1.0f / den);
+  }
+
+  // rows [j_lo, j_hi) of h = A_e x: warp w takes the w-th sixteenth of every row (whole 16-byte pieces), four rows
+  // at a time with every load issued before the first use; the sixteen partial sums of a row are added in warp
+  // order afterwards (fp32 accumulation over the bf16 operands)
+  const int nrows = r > 0 ? j_hi - j_lo : 0;
+  if (nrows > 0) {
+    const int s_lo = (int)((long long)chunks * warp / kStreamWarps), s_hi = (int)((long long)chunks * (warp + 1) / kStreamWarps);
+    const uint4* a4 = reinterpret_cast<const uint4*>(L.A) + ((long long)best * r + j_lo) * chunks;
+    for (int jb = 0; jb < nrows; jb += 4) {
+      float a0[4] = {0.f, 0.f, 0.f, 0.f}, a1[4] = {0.f, 0.f, 0.f, 0.f};
+      for (int c0 = s_lo + lane; c0 < s_hi; c0 += 128) {
+        uint4 wv[4][4];
+#pragma unroll
+        for (int rb = 0; rb < 4; ++rb)
+#pragma unroll
+          for (int u = 0; u < 4; ++u)
+            wv[rb][u] = (jb + rb < nrows && c0 + 32 * u < s_hi) ? __ldg(a4 + (long long)(jb + rb) * chunks + c0 + 32 * u) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          if (c0 + 32 * u < s_hi) {
+            const uint4 xv = xs4[c0 + 32 * u];
+#pragma unroll
+            for (int rb = 0; rb < 4; ++rb) {
+              a0[rb] = fmaf(bf16lo(xv.x), bf16lo(wv[rb][u].x), a0[rb]); a1[rb] = fmaf(bf16hi(xv.x), bf16hi(wv[rb][u].x), a1[rb]);
+              a0[rb] = fmaf(bf16lo(xv.y), bf16lo(wv[rb][u].y), a0[rb]); a1[rb] = fmaf(bf16hi(xv.y), bf16hi(wv[rb][u].y), a1[rb]);
+              a0[rb] = fmaf(bf16lo(xv.z), bf16lo(wv[rb][u].z), a0[rb]); a1[rb] = fmaf(bf16hi(xv.z), bf16hi(wv[rb][u].z), a1[rb]);
+              a0[rb] = fmaf(bf16lo(xv.w), bf16lo(wv[rb][u].w), a0[rb]); a1[rb] = fmaf(bf16hi(xv.w), bf16hi(wv[rb][u].w), a1[rb]);
+            }
+          }
+        }
+      }
+#pragma unroll
+      for (int rb = 0; rb < 4; ++rb) {
+        float a = a0[rb] + a1[rb];
+        for (int d = 16; d > 0; d >>= 1) a += __shfl_xor_sync(0xffffffffu, a, d);
+        if (lane == 0 && jb + rb < nrows) part[(jb + rb) * kStreamWarps + warp] = a;
+      }
+    }
   }
 
   if (owner) {
@@ -299,46 +372,25 @@ __device__ void stream_token(const StreamLinear& L, int t, int j_lo, int j_hi, b
     }
     for (int d = 16; d > 0; d >>= 1) rowsum += __shfl_xor_sync(0xffffffffu, rowsum, d);
     if (lane == 0) sh.red_i[warp] = rowsum;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      int tot = 0;
-      for (int w = 0; w < kStreamWarps; ++w) tot += sh.red_i[w];
-      L.info[t] = DecodeTokInfo{best, gate, gamma, tot};
-    }
   }
-
-  // rows [j_lo, j_hi) of h = A_e x (fp32 accumulation over the bf16 operands), one warp per row
-  if (r > 0) {
-    for (int j = j_lo + warp; j < j_hi; j += kStreamWarps) {
-      const uint4* arow = reinterpret_cast<const uint4*>(L.A) + ((long long)best * r + j) * chunks;
-      float a0 = 0.f, a1 = 0.f;
-      for (int c0 = lane; c0 < chunks; c0 += 256) {
-        uint4 wv[8];
+  __syncthreads();   // partial sums of h and of the codes are visible
+  if (owner && threadIdx.x == 0) {
+    int tot = 0;
+    for (int w = 0; w < kStreamWarps; ++w) tot += sh.red_i[w];
+    L.info[t] = DecodeTokInfo{best, gate, gamma, tot};
+  }
+  for (int i = threadIdx.x; i < nrows; i += kStreamThreads) {
+    float a = 0.f;
 #pragma unroll
-        for (int u = 0; u < 8; ++u) wv[u] = c0 + 32 * u < chunks ? __ldg(arow + c0 + 32 * u) : make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          if (c0 + 32 * u < chunks) {
-            const uint4 xv = xs4[c0 + 32 * u];
-            a0 = fmaf(bf16lo(xv.x), bf16lo(wv[u].x), a0); a1 = fmaf(bf16hi(xv.x), bf16hi(wv[u].x), a1);
-            a0 = fmaf(bf16lo(xv.y), bf16lo(wv[u].y), a0); a1 = fmaf(bf16hi(xv.y), bf16hi(wv[u].y), a1);
-            a0 = fmaf(bf16lo(xv.z), bf16lo(wv[u].z), a0); a1 = fmaf(bf16hi(xv.z), bf16hi(wv[u].z), a1);
-            a0 = fmaf(bf16lo(xv.w), bf16lo(wv[u].w), a0); a1 = fmaf(bf16hi(xv.w), bf16hi(wv[u].w), a1);
-          }
-        }
-      }
-      float a = a0 + a1;
-      for (int d = 16; d > 0; d >>= 1) a += __shfl_xor_sync(0xffffffffu, a, d);
-      if (lane == 0) L.h[(long long)t * r + j] = a;
-    }
+    for (int w = 0; w < kStreamWarps; ++w) a += part[i * kStreamWarps + w];
+    L.h[(long long)t * r + j_lo + i] = a;
   }
 }
 
 // ---------------------------------------------------------------------------
-// phase 2: the bit product of a warp's chunks [p_lo, p_hi) of one linear for the tokens of one group, and the
-// epilogue of every row group this warp completes.  MT = tokens of the group rounded up to a power of two;
-// with one token the masks need no shift (eight accumulators per feature, weighted 1 << b, exact in int32:
-// 127 * 128 * K < 2^31 for every K the library accepts).
+// phase 2.  Every work item reports to the counter of its row group (128 features x the tokens of one group of
+// eight); the report that completes the count (C chunks of sign bits, plus four expert-product items per token
+// when there is an HP branch) finishes the row group.
 // ---------------------------------------------------------------------------
 // four signed codes times four unsigned mask bytes (a mask byte can be 0x80)
 __device__ __forceinline__ int dp4a_s8u8(uint32_t q, uint32_t m, int c) {
@@ -347,53 +399,43 @@ __device__ __forceinline__ int dp4a_s8u8(uint32_t q, uint32_t m, int c) {
   return d;
 }
 
-template <int MT>
-__device__ __forceinline__ void stream_epilogue(const StreamLinear& L, int tg, int mg, int g, int (&vals)[4][MT], const float* hs,
-                                                const DecodeTokInfo* toks, int lane) {
+__device__ __forceinline__ unsigned stream_target(const StreamLinear& L, int tg) {
+  const int mg = min(kStreamTokenGroup, L.M - tg * kStreamTokenGroup);
+  return (unsigned)(L.C + (L.r > 0 ? 4 * mg : 0));
+}
+
+// Eq. 10-11 for row group g and the tokens of group tg: everything it needs is complete in global memory
+__device__ void stream_finish(const StreamLinear& L, int tg, int g, const DecodeTokInfo* toks, int lane) {
+  __threadfence();
   const float lam = __ldg(L.w_scales);
-  const int r = L.r, r8 = r >> 3;
-  const int G32 = L.G * 4;
+  const int Np = L.G * 128;
+  const int mg = min(kStreamTokenGroup, L.M - tg * kStreamTokenGroup);
+  float be[4], al[4];
 #pragma unroll
-  for (int t = 0; t < MT; ++t) {
-    if (t >= mg) break;
-    const DecodeTokInfo tk = toks[t];
+  for (int f = 0; f < 4; ++f) {
+    const int n = g * 128 + f * 32 + lane;
+    be[f] = n < L.N ? __ldg(L.beta + (long long)n * L.sstride) : 0.f;
+    al[f] = (n < L.N && L.r > 0) ? __ldg(L.alpha + (long long)n * L.sstride) : 0.f;
+  }
+  for (int t = 0; t < mg; ++t) {
     const int tok = tg * kStreamTokenGroup + t;
-    float z[4] = {0.f, 0.f, 0.f, 0.f};
-    if (r > 0) {
-      const uint4* bp = L.B_il + ((long long)tk.expert * G32 + g * 4) * r8 * 32 + lane;
-      const float* hv = hs + t * r;
-      for (int jc = 0; jc < r8; jc += 2) {
-        uint4 b[2][4];
-#pragma unroll
-        for (int u = 0; u < 2; ++u)
-#pragma unroll
-          for (int f = 0; f < 4; ++f) b[u][f] = jc + u < r8 ? __ldg(bp + ((long long)f * r8 + jc + u) * 32) : make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-          if (jc + u < r8) {
-            const float4 h0 = *reinterpret_cast<const float4*>(hv + (jc + u) * 8);
-            const float4 h1 = *reinterpret_cast<const float4*>(hv + (jc + u) * 8 + 4);
-#pragma unroll
-            for (int f = 0; f < 4; ++f) {
-              float a = z[f];
-              a = fmaf(bf16lo(b[u][f].x), h0.x, a); a = fmaf(bf16hi(b[u][f].x), h0.y, a);
-              a = fmaf(bf16lo(b[u][f].y), h0.z, a); a = fmaf(bf16hi(b[u][f].y), h0.w, a);
-              a = fmaf(bf16lo(b[u][f].z), h1.x, a); a = fmaf(bf16hi(b[u][f].z), h1.y, a);
-              a = fmaf(bf16lo(b[u][f].w), h1.z, a); a = fmaf(bf16hi(b[u][f].w), h1.w, a);
-              z[f] = a;
-            }
-          }
-        }
-      }
-    }
+    const DecodeTokInfo tk = toks[tok];
     const float deq = __fdiv_rn(lam, tk.gamma);
+    int m[4];
+    float z[4];
+#pragma unroll
+    for (int f = 0; f < 4; ++f) {
+      const long long at = (long long)tok * Np + g * 128 + f * 32 + lane;
+      m[f] = __ldcg(L.acc + at);
+      z[f] = L.r > 0 ? __ldcg(L.z + at) : 0.f;
+    }
 #pragma unroll
     for (int f = 0; f < 4; ++f) {
       const int n = g * 128 + f * 32 + lane;
       if (n < L.N) {
-        const int acc = 2 * vals[f][t] - tk.rowsum;
-        float y = __ldg(L.beta + (long long)n * L.sstride) * deq * (float)acc;
-        if (r > 0) y = fmaf(__ldg(L.alpha + (long long)n * L.sstride) * tk.gate, z[f], y);
+        const int acc = 2 * m[f] - tk.rowsum;
+        float y = be[f] * deq * (float)acc;
+        if (L.r > 0) y = fmaf(al[f] * tk.gate, z[f], y);
         L.Y[(long long)tok * L.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(y));
         if (L.acc_dump) L.acc_dump[(long long)tok * L.N + n] = acc;
       }
@@ -401,9 +443,55 @@ __device__ __forceinline__ void stream_epilogue(const StreamLinear& L, int tg, i
   }
 }
 
+// reports `units` finished items of row group (tg, g); true for the whole warp when that completes the count
+__device__ __forceinline__ bool stream_report(const StreamLinear& L, int tg, int g, unsigned units, int lane) {
+  __threadfence();
+  __syncwarp();
+  unsigned old = 0u;
+  if (lane == 0) old = atomicAdd(L.cnt + tg * L.G + g, units);
+  old = __shfl_sync(0xffffffffu, old, 0);
+  return old + units == stream_target(L, tg);
+}
+
+// (a) expert-product items [i_lo, i_hi) of one linear: item = token * 4G + group of 32 features; hs = h of all its tokens
+__device__ void stream_expert(const StreamLinear& L, int i_lo, int i_hi, const float* hs, const DecodeTokInfo* toks) {
+  const int lane = threadIdx.x & 31;
+  const int G32 = L.G * 4, r = L.r, r8 = r >> 3;
+  const int Np = L.G * 128;
+  for (int i = i_lo; i < i_hi; ++i) {
+    const int tok = i / G32, g32 = i - tok * G32;
+    if (g32 * 32 < L.N) {
+      const uint4* bp = L.B_il + ((long long)toks[tok].expert * G32 + g32) * r8 * 32 + lane;
+      const float* hv = hs + tok * r;
+      float z = 0.f;
+      for (int j0 = 0; j0 < r8; j0 += 20) {
+        uint4 b[20];
+#pragma unroll
+        for (int u = 0; u < 20; ++u) b[u] = j0 + u < r8 ? __ldg(bp + (long long)(j0 + u) * 32) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+        for (int u = 0; u < 20; ++u) {
+          if (j0 + u < r8) {
+            const float4 h0 = *reinterpret_cast<const float4*>(hv + (j0 + u) * 8);
+            const float4 h1 = *reinterpret_cast<const float4*>(hv + (j0 + u) * 8 + 4);
+            z = fmaf(bf16lo(b[u].x), h0.x, z); z = fmaf(bf16hi(b[u].x), h0.y, z);
+            z = fmaf(bf16lo(b[u].y), h0.z, z); z = fmaf(bf16hi(b[u].y), h0.w, z);
+            z = fmaf(bf16lo(b[u].z), h1.x, z); z = fmaf(bf16hi(b[u].z), h1.y, z);
+            z = fmaf(bf16lo(b[u].w), h1.z, z); z = fmaf(bf16hi(b[u].w), h1.w, z);
+          }
+        }
+      }
+      L.z[(long long)tok * Np + g32 * 32 + lane] = z;
+    }
+    const int tg = tok / kStreamTokenGroup, g = g32 >> 2;
+    if (stream_report(L, tg, g, 1u, lane)) stream_finish(L, tg, g, toks, lane);
+  }
+}
+
+// (b) chunks [p_lo, p_hi) of one linear for the tokens of group tg.  MT = tokens of the group rounded up to 1, 2, 4
+// or 8; with one token the masks need no shift (eight accumulators per feature, weighted 1 << b, exact in int32:
+// 127 * 128 * K < 2^31 for every K the library accepts).
 template <int MT>
-__device__ void stream_bits(const StreamLinear& L, int tg, int mg, int p_lo, int p_hi, const uint32_t* qs, int qwords, const float* hs,
-                            const DecodeTokInfo* toks) {
+__device__ void stream_bits(const StreamLinear& L, int tg, int mg, int p_lo, int p_hi, const uint32_t* qs, int qwords, const DecodeTokInfo* toks) {
   constexpr bool NS = MT == 1;
   constexpr int NA = NS ? 8 : 1;
   const int lane = threadIdx.x & 31;
@@ -457,46 +545,27 @@ __device__ void stream_bits(const StreamLinear& L, int tg, int mg, int p_lo, int
     src = nxt;
     ++p; ++c; ++delivered;
     if (c == C || p == p_hi) {
-      // hand the row group's partial sums over; the warp that delivers its last chunk finishes it
-      int vals[4][MT];
+      // hand the row group's partial sums over
 #pragma unroll
-      for (int f = 0; f < 4; ++f)
+      for (int t = 0; t < MT; ++t) {
+        if (t < mg) {
+          int* dst = L.acc + (long long)(tg * kStreamTokenGroup + t) * Np + g * 128 + lane;
 #pragma unroll
-        for (int t = 0; t < MT; ++t) {
-          int v = 0;
+          for (int f = 0; f < 4; ++f) {
+            int v = 0;
 #pragma unroll
-          for (int a = 0; a < NA; ++a) { v += NS ? (acc[f][t][a] >> a) : acc[f][t][a]; acc[f][t][a] = 0; }
-          vals[f][t] = v;
-        }
-      bool finish = delivered == C;
-      if (!finish) {
-#pragma unroll
-        for (int t = 0; t < MT; ++t) {
-          if (t < mg) {
-            int* dst = L.acc + (long long)(tg * kStreamTokenGroup + t) * Np + g * 128 + lane;
-#pragma unroll
-            for (int f = 0; f < 4; ++f) atomicAdd(dst + f * 32, vals[f][t]);
-          }
-        }
-        __threadfence();
-        __syncwarp();
-        unsigned old = 0u;
-        if (lane == 0) old = atomicAdd(L.cnt + tg * L.G + g, (unsigned)delivered);
-        old = __shfl_sync(0xffffffffu, old, 0);
-        finish = old + (unsigned)delivered == (unsigned)C;
-        if (finish) {
-          __threadfence();
-#pragma unroll
-          for (int t = 0; t < MT; ++t) {
-            if (t < mg) {
-              const int* from = L.acc + (long long)(tg * kStreamTokenGroup + t) * Np + g * 128 + lane;
-#pragma unroll
-              for (int f = 0; f < 4; ++f) vals[f][t] = __ldcg(from + f * 32);
-            }
+            for (int a = 0; a < NA; ++a) v += NS ? (acc[f][t][a] >> a) : acc[f][t][a];
+            atomicAdd(dst + f * 32, v);
           }
         }
       }
-      if (finish) stream_epilogue<MT>(L, tg, mg, g, vals, hs, toks, lane);
+#pragma unroll
+      for (int f = 0; f < 4; ++f)
+#pragma unroll
+        for (int t = 0; t < MT; ++t)
+#pragma unroll
+          for (int a = 0; a < NA; ++a) acc[f][t][a] = 0;
+      if (stream_report(L, tg, g, (unsigned)delivered, lane)) stream_finish(L, tg, g, toks, lane);
       if (c == C) { c = 0; ++g; }
       delivered = 0;
     }
@@ -512,8 +581,9 @@ __global__ void __launch_bounds__(kStreamThreads, 1) k_decode_stream(const __gri
   unsigned* bar = g_stream_bar[bp.bar_slot];
   const int nC = (int)gridDim.x, cta = (int)blockIdx.x;
   const int warp = threadIdx.x >> 5;
-  const long long T = bp.total_chunks;
+  const long long T = bp.total_chunks, Z = bp.total_z;
   const int span_lo = (int)(T * cta / nC), span_hi = (int)(T * (cta + 1) / nC);
+  const int zspan_lo = (int)(Z * cta / nC), zspan_hi = (int)(Z * (cta + 1) / nC);
 
   if (bp.prefetch) {
     // the sign bits of this CTA's span do not depend on phase 1: let them travel to L2 while it runs
@@ -534,7 +604,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) k_decode_stream(const __gri
     for (long long i = z_lo + threadIdx.x; i < z_hi; i += kStreamThreads) L.acc[i] = 0;
   }
 
-  // phase 1: token work of the linears this CTA's span touches
+  // phase 1: token work of the linears this CTA shares
   for (int l = 0; l < bp.n; ++l) {
     const StreamLinear& L = bp.lin[l];
     if (cta < L.cta_first || cta >= L.cta_first + L.cta_count) continue;
@@ -545,17 +615,31 @@ __global__ void __launch_bounds__(kStreamThreads, 1) k_decode_stream(const __gri
     if (u_lo >= u_hi) continue;
     for (int t = u_lo / rp; t <= (u_hi - 1) / rp; ++t) {
       const int j_lo = max(u_lo, t * rp) - t * rp, j_hi = min(u_hi, (t + 1) * rp) - t * rp;
-      stream_token(L, t, j_lo, j_hi, j_lo == 0, reinterpret_cast<uint4*>(stream_smem), sh);
+      stream_token(bp, L, t, j_lo, j_hi, j_lo == 0, stream_smem, sh);
     }
   }
   stream_bar_arrive(bar);
   const bool ok = stream_bar_wait(bar, &sh.ok);
 
-  // phase 2
   if (ok) {
     uint32_t* qs = reinterpret_cast<uint32_t*>(stream_smem);
     float* hs = reinterpret_cast<float*>(stream_smem + bp.off_h);
     DecodeTokInfo* toks = reinterpret_cast<DecodeTokInfo*>(stream_smem + bp.off_info);
+    // phase 2 (a): expert products.  What phase 1 wrote comes from other CTAs: read it through L2.
+    for (int l = 0; l < bp.n; ++l) {
+      const StreamLinear& L = bp.lin[l];
+      if (L.r == 0) continue;
+      const int zi = L.M * L.G * 4;
+      const int seg_lo = max(zspan_lo, L.z0) - L.z0, seg_hi = min(zspan_hi, L.z0 + zi) - L.z0;
+      if (seg_lo >= seg_hi) continue;
+      __syncthreads();
+      for (int i = threadIdx.x; i < L.M * L.r; i += kStreamThreads) hs[i] = __ldcg(L.h + i);
+      if (threadIdx.x < L.M) reinterpret_cast<int4*>(toks)[threadIdx.x] = __ldcg(reinterpret_cast<const int4*>(L.info) + threadIdx.x);
+      __syncthreads();
+      const int len = seg_hi - seg_lo;
+      stream_expert(L, seg_lo + (int)((long long)len * warp / kStreamWarps), seg_lo + (int)((long long)len * (warp + 1) / kStreamWarps), hs, toks);
+    }
+    // phase 2 (b): sign bits
     for (int l = 0; l < bp.n; ++l) {
       const StreamLinear& L = bp.lin[l];
       const int seg_lo = max(span_lo, L.chunk0) - L.chunk0, seg_hi = min(span_hi, L.chunk0 + L.G * L.C) - L.chunk0;
@@ -565,22 +649,18 @@ __global__ void __launch_bounds__(kStreamThreads, 1) k_decode_stream(const __gri
       const int p_lo = seg_lo + (int)((long long)len * warp / kStreamWarps), p_hi = seg_lo + (int)((long long)len * (warp + 1) / kStreamWarps);
       for (int tg = 0; tg * kStreamTokenGroup < L.M; ++tg) {
         const int mg = min(kStreamTokenGroup, L.M - tg * kStreamTokenGroup);
-        __syncthreads();   // the previous codes are no longer read
+        __syncthreads();   // the previous codes and token records are no longer read
         {
-          // written by other CTAs in phase 1: read through L2
           const uint4* from = reinterpret_cast<const uint4*>(L.qg + (long long)tg * kStreamTokenGroup * qwords);
           uint4* to = reinterpret_cast<uint4*>(qs);
           for (int i = threadIdx.x; i < mg * (qwords >> 2); i += kStreamThreads) to[i] = __ldcg(from + i);
-          const float* hfrom = L.h + (long long)tg * kStreamTokenGroup * L.r;
-          for (int i = threadIdx.x; i < mg * L.r; i += kStreamThreads) hs[i] = __ldcg(hfrom + i);
-          const int4* ifrom = reinterpret_cast<const int4*>(L.info + tg * kStreamTokenGroup);
-          if (threadIdx.x < mg) reinterpret_cast<int4*>(toks)[threadIdx.x] = __ldcg(ifrom + threadIdx.x);
+          if (threadIdx.x < L.M) reinterpret_cast<int4*>(toks)[threadIdx.x] = __ldcg(reinterpret_cast<const int4*>(L.info) + threadIdx.x);
         }
         __syncthreads();
-        if (mg == 1) stream_bits<1>(L, tg, mg, p_lo, p_hi, qs, qwords, hs, toks);
-        else if (mg == 2) stream_bits<2>(L, tg, mg, p_lo, p_hi, qs, qwords, hs, toks);
-        else if (mg <= 4) stream_bits<4>(L, tg, mg, p_lo, p_hi, qs, qwords, hs, toks);
-        else stream_bits<8>(L, tg, mg, p_lo, p_hi, qs, qwords, hs, toks);
+        if (mg == 1) stream_bits<1>(L, tg, mg, p_lo, p_hi, qs, qwords, toks);
+        else if (mg == 2) stream_bits<2>(L, tg, mg, p_lo, p_hi, qs, qwords, toks);
+        else if (mg <= 4) stream_bits<4>(L, tg, mg, p_lo, p_hi, qs, qwords, toks);
+        else stream_bits<8>(L, tg, mg, p_lo, p_hi, qs, qwords, toks);
       }
     }
   }
@@ -592,11 +672,13 @@ __global__ void __launch_bounds__(kStreamThreads, 1) k_decode_stream(const __gri
 // ---------------------------------------------------------------------------
 static inline size_t s_up256(size_t x) { return (x + 255) / 256 * 256; }
 
-// bytes this path needs in an item's workspace beyond what decode_workspace_bytes() counts
+// bytes this path needs in an item's workspace beyond what decode_workspace_bytes() counts:
+// codes | h | z | accumulators and counters
 size_t decode_stream_extra_bytes(int M, int K, int N, int r) {
   const size_t G = (N + 127) / 128, C = (K + 127) / 128;
   const size_t groups = (M + kStreamTokenGroup - 1) / kStreamTokenGroup;
-  return s_up256((size_t)M * C * 128) + s_up256((size_t)M * std::max(r, 1) * 4) + s_up256(((size_t)M * G * 128 + groups * G) * 4);
+  return s_up256((size_t)M * C * 128) + s_up256((size_t)M * std::max(r, 1) * 4) + s_up256((size_t)M * G * 128 * 4) +
+         s_up256(((size_t)M * G * 128 + groups * G) * 4);
 }
 
 static int g_decode_stream_on = 1;
@@ -634,8 +716,9 @@ int decode_stream_launch(const DecodeItemArgs* items, int n, cudaStream_t st) {
   if (n < 1 || n > kStreamMaxBatch) return PQ_ERR_UNSUPPORTED;
   StreamBatch bp{};
   bp.n = n;
-  long long total = 0;
-  size_t region0 = 0, hbytes = 0;
+  long long total = 0, total_z = 0;
+  size_t codes = 0, hbytes = 0, xbytes = 0, part = 0;
+  int max_e = 1;
   for (int i = 0; i < n; ++i) {
     const DecodeItemArgs& it = items[i];
     const int M = it.a.T, K = it.a.K, N = it.a.N, r = it.a.r;
@@ -653,36 +736,51 @@ int decode_stream_launch(const DecodeItemArgs* items, int n, cudaStream_t st) {
     w += decode_workspace_bytes(M, K, N, r, it.dump);
     L.qg = reinterpret_cast<uint32_t*>(w); w += s_up256((size_t)M * L.C * 128);
     L.h = reinterpret_cast<float*>(w); w += s_up256((size_t)M * std::max(r, 1) * 4);
+    L.z = reinterpret_cast<float*>(w); w += s_up256((size_t)M * L.G * 128 * 4);
     L.acc = reinterpret_cast<int*>(w);
     const int groups = (M + kStreamTokenGroup - 1) / kStreamTokenGroup;
     L.cnt = reinterpret_cast<unsigned*>(L.acc + (size_t)M * L.G * 128);
     L.zero_words = M * L.G * 128 + groups * L.G;
     L.chunk0 = (int)total;
     total += (long long)L.G * L.C;
-    if (total > (1ll << 30)) return PQ_ERR_UNSUPPORTED;
+    L.z0 = (int)total_z;
+    if (r > 0) total_z += (long long)M * L.G * 4;
+    if (total > (1ll << 30) || total_z > (1ll << 30)) return PQ_ERR_UNSUPPORTED;
     // the bit product is instantiated for 1, 2, 4 or 8 tokens and reads that many rows of codes (the surplus rows are
     // never used, but they must lie inside the allocation)
     const int mt = M >= 5 ? 8 : M >= 3 ? 4 : M;
-    region0 = std::max(region0, std::max((size_t)K * 2, (size_t)mt * L.C * 128));
-    hbytes = std::max(hbytes, (size_t)kStreamTokenGroup * std::max(r, 1) * 4);
+    codes = std::max(codes, (size_t)mt * L.C * 128);
+    hbytes = std::max(hbytes, (size_t)M * std::max(r, 1) * 4);
+    xbytes = std::max(xbytes, (size_t)K * 2);
+    part = std::max(part, (size_t)std::max(r, 1) * kStreamWarps * 4);
+    max_e = std::max(max_e, L.E);
   }
   bp.total_chunks = (int)total;
+  bp.total_z = (int)total_z;
+  // the token work of a linear is shared by the CTAs whose span of the chunk list touches it
   const int nC = sms;
   for (int i = 0; i < n; ++i) {
     StreamLinear& L = bp.lin[i];
     const long long lo = L.chunk0, hi = L.chunk0 + (long long)L.G * L.C;
-    int first = -1, count = 0;
-    for (int c = 0; c < nC; ++c) {
-      const long long s_lo = total * c / nC, s_hi = total * (c + 1) / nC;
-      if (std::max(s_lo, lo) < std::min(s_hi, hi)) { if (first < 0) first = c; ++count; }
-    }
-    if (first < 0) return PQ_ERR_UNSUPPORTED;
-    L.cta_first = first; L.cta_count = count;
+    int first = (int)(lo * nC / total);
+    while (first > 0 && total * first / nC > lo) --first;
+    while (total * (first + 1) / nC <= lo) ++first;
+    int last = first;
+    while (last + 1 < nC && total * (last + 1) / nC < hi) ++last;
+    L.cta_first = first; L.cta_count = last - first + 1;
   }
-  region0 = s_up256(region0);
-  bp.off_h = (int)region0;
-  bp.off_info = (int)(region0 + s_up256(hbytes));
-  const size_t smem = bp.off_info + 256;
+  // shared memory: phase 1 [token][router rows][partial sums], phase 2 [codes][h][token records]
+  xbytes = s_up256(xbytes);
+  const size_t avail = kStreamSmemLimit - xbytes - s_up256(part);
+  bp.router_rows = max_e > 1 ? (int)std::min<size_t>(max_e, avail / xbytes) : 0;
+  if (max_e > 1 && bp.router_rows < 1) return PQ_ERR_UNSUPPORTED;
+  bp.off_rows = (int)xbytes;
+  bp.off_part = (int)(xbytes + (size_t)bp.router_rows * xbytes);
+  const size_t smem1 = bp.off_part + s_up256(part);
+  bp.off_h = (int)s_up256(codes);
+  bp.off_info = (int)(bp.off_h + s_up256(hbytes));
+  const size_t smem2 = bp.off_info + 256;
+  const size_t smem = std::max(smem1, smem2);
   if (smem > kStreamSmemLimit) return PQ_ERR_UNSUPPORTED;
   bp.bar_slot = stream_bar_slot(st);
   if (bp.bar_slot < 0) return PQ_ERR_UNSUPPORTED;
