@@ -868,6 +868,7 @@ def main():
     ap.add_argument("--decode-batch", type=int, default=16, help="independent decode linears per pq_decode_batch call")
     ap.add_argument("--decode-kernels", default="stream", choices=["stream", "pair"],
                     help="stream: the cooperative streaming kernel on weights in its own layout; pair: the two-kernel path on the plain layout")
+    ap.add_argument("--decode-prefetch", type=int, default=1, choices=[0, 1], help="streaming decode kernel: L2 prefetch of the sign bits during the token work")
     ap.add_argument("--decode-rmsnorm", action="store_true", help="decode from un-normalised activations, RMSNorm fused into the token preparation")
     ap.add_argument("--decoder-one-form", action="store_true", help="decoder workload: only the form with 8 experts on every projection")
     ap.add_argument("--cpu-tokens", type=int, default=8192, help="tokens per step of the CPU oracle (cpu_baseline and --impl reference)")
@@ -884,6 +885,7 @@ def main():
         return
     ctx = Ctx()
     ctx.decode_kernels = args.decode_kernels
+    ctx.pqb.pq_set_option(ctx.pqb.PQ_OPT_DECODE_PREFETCH, args.decode_prefetch)
     if args.workload == "decode":
         run_decode(args, ctx)
     elif args.workload == "decoder":

@@ -66,15 +66,21 @@ struct StreamLinear {
   int cta_first, cta_count; // the CTAs that share its token work
   int zero_words;           // int32 words from `acc` on that phase 1 clears (acc and cnt are adjacent)
 };
+// The descriptor travels as kernel parameters (constant memory).  What every CTA needs to find its work sits in a few
+// compact tables in front, so that a CTA touches the records of its own one or two linears only: a first touch of a
+// cold parameter line costs a trip to memory, and a loop over sixteen records paid sixteen of them in a row.
 struct StreamBatch {
-  StreamLinear lin[kStreamMaxBatch];
   int n;
   int total_chunks, total_z;
   int bar_slot;
-  int prefetch;             // issue L2 prefetches for the span's sign bits before phase 1
+  int prefetch;             // chunks ahead of the bit product for which L2 prefetches are issued (0 = none)
   int router_rows;          // router rows that fit in shared memory beside the token
   int off_rows, off_part;   // phase 1 carve-up: [token][router rows][partial sums of h]
   int off_h, off_info;      // phase 2 carve-up: [codes][h][token info]
+  int chunk0[kStreamMaxBatch + 1];   // first chunk of every linear in the launch-wide list (and the total)
+  int z0[kStreamMaxBatch + 1];       // first expert-product item of every linear
+  unsigned char duty[160];           // linear whose token work CTA b shares (255: none)
+  StreamLinear lin[kStreamMaxBatch];
 };
 
 // ---------------------------------------------------------------------------
@@ -142,6 +148,17 @@ __device__ __forceinline__ void stream_bar_arrive(unsigned* bar) {
     atomicAdd(&bar[0], 1u);
   }
 }
+// Called by one thread right after the CTA's wait: once every CTA has got past the wait nobody reads the pair any more, and
+// the last one through leaves it clear for the next launch (nothing is left to do at the end of the kernel).
+__device__ __forceinline__ void stream_bar_depart(unsigned* bar) {
+  const unsigned old = atomicAdd(&bar[1], 1u);
+  if (old == gridDim.x - 1) {
+    bar[0] = 0u;
+    bar[1] = 0u;
+    __threadfence();
+  }
+}
+
 // returns false (for every thread of the CTA) when the wait ran out
 __device__ __forceinline__ bool stream_bar_wait(unsigned* bar, int* ok_sh) {
   if (threadIdx.x == 0) {
@@ -158,21 +175,9 @@ __device__ __forceinline__ bool stream_bar_wait(unsigned* bar, int* ok_sh) {
     *ok_sh = ok;
   }
   __syncthreads();
+  if (threadIdx.x == kStreamThreads - 32) stream_bar_depart(bar);   // its warp alone waits for the returned count
   return *ok_sh != 0;
 }
-__device__ __forceinline__ void stream_bar_depart(unsigned* bar) {
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    const unsigned old = atomicAdd(&bar[1], 1u);
-    if (old == gridDim.x - 1) {   // everybody has passed the wait: leave the pair clear for the next launch
-      bar[0] = 0u;
-      bar[1] = 0u;
-      __threadfence();
-    }
-  }
-}
-
-
 // ---------------------------------------------------------------------------
 // phase 1: one token of one linear, rows [j_lo, j_hi) of h; `owner` also quantises and publishes the token
 // ---------------------------------------------------------------------------
@@ -202,7 +207,49 @@ __device__ __forceinline__ void stream_stage(int total, Dst dst, Src src) {
   }
 }
 
-__device__ void stream_token(const StreamBatch& bp, const StreamLinear& L, int t, int j_lo, int j_hi, bool owner, uint8_t* smem, StreamShared& sh) {
+// Partial dot products of `nrows` rows (a4: first row, `chunks` 16-byte pieces each) with the token in shared memory
+// over this warp's pieces [s_lo, s_hi): 16 / UPL rows at a time, UPL loads per lane and row (more pieces: further rounds).
+template <int UPL>
+__device__ __forceinline__ void stream_h_rows(const uint4* a4, const uint4* xs4, float* part, int nrows, int chunks, int s_lo, int s_hi,
+                                              int warp, int lane) {
+  constexpr int RB = 16 / UPL;
+  for (int jb = 0; jb < nrows; jb += RB) {
+    float acc[RB];
+#pragma unroll
+    for (int rb = 0; rb < RB; ++rb) acc[rb] = 0.f;
+    for (int c0 = s_lo + lane; c0 < s_hi; c0 += 32 * UPL) {
+      uint4 wv[RB][UPL];
+#pragma unroll
+      for (int rb = 0; rb < RB; ++rb)
+#pragma unroll
+        for (int u = 0; u < UPL; ++u)
+          wv[rb][u] = (jb + rb < nrows && c0 + 32 * u < s_hi) ? __ldg(a4 + (long long)(jb + rb) * chunks + c0 + 32 * u) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+      for (int u = 0; u < UPL; ++u) {
+        if (c0 + 32 * u < s_hi) {
+          const uint4 xv = xs4[c0 + 32 * u];
+#pragma unroll
+          for (int rb = 0; rb < RB; ++rb) {
+            float a = acc[rb];
+            a = fmaf(bf16lo(xv.x), bf16lo(wv[rb][u].x), a); a = fmaf(bf16hi(xv.x), bf16hi(wv[rb][u].x), a);
+            a = fmaf(bf16lo(xv.y), bf16lo(wv[rb][u].y), a); a = fmaf(bf16hi(xv.y), bf16hi(wv[rb][u].y), a);
+            a = fmaf(bf16lo(xv.z), bf16lo(wv[rb][u].z), a); a = fmaf(bf16hi(xv.z), bf16hi(wv[rb][u].z), a);
+            a = fmaf(bf16lo(xv.w), bf16lo(wv[rb][u].w), a); a = fmaf(bf16hi(xv.w), bf16hi(wv[rb][u].w), a);
+            acc[rb] = a;
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int rb = 0; rb < RB; ++rb) {
+      float a = acc[rb];
+      for (int d = 16; d > 0; d >>= 1) a += __shfl_xor_sync(0xffffffffu, a, d);
+      if (lane == 0 && jb + rb < nrows) part[(jb + rb) * kStreamWarps + warp] = a;
+    }
+  }
+}
+
+__device__ void stream_token(const StreamBatch& bp, const StreamLinear& L, int t, int j_lo, int j_hi, bool owner, bool first, uint8_t* smem, StreamShared& sh) {
   const int K = L.K, E = L.E, r = L.r;
   const int chunks = K >> 3;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -213,8 +260,8 @@ __device__ void stream_token(const StreamBatch& bp, const StreamLinear& L, int t
   const uint4* wr4 = reinterpret_cast<const uint4*>(L.Wr);
   const int R = bp.router_rows;
   __syncthreads();   // the previous token's values are no longer read
-  // the token and the first round of router rows travel together
-  const int first_rows = E > 1 ? min(R, E) : 0;
+  // the token and the first round of router rows travel together; when all rows fit they stay for the CTA's later tokens
+  const int first_rows = (E > 1 && (first || R < E)) ? min(R, E) : 0;
   stream_stage(chunks * (1 + first_rows), [&](int i) { return i < chunks ? xs4 + i : rows4 + (i - chunks); },
                [&](int i) { return i < chunks ? x4 + i : wr4 + (i - chunks); });
   __syncthreads();
@@ -300,43 +347,16 @@ __device__ void stream_token(const StreamBatch& bp, const StreamLinear& L, int t
     gate = pbest * (1.0f / den);
   }
 
-  // rows [j_lo, j_hi) of h = A_e x: warp w takes the w-th sixteenth of every row (whole 16-byte pieces), four rows
-  // at a time with every load issued before the first use; the sixteen partial sums of a row are added in warp
-  // order afterwards (fp32 accumulation over the bf16 operands)
+  // rows [j_lo, j_hi) of h = A_e x: warp w takes the w-th sixteenth of every row (whole 16-byte pieces), sixteen
+  // loads per lane issued before the first use; the sixteen partial sums of a row are added in warp order afterwards
   const int nrows = r > 0 ? j_hi - j_lo : 0;
   if (nrows > 0) {
     const int s_lo = (int)((long long)chunks * warp / kStreamWarps), s_hi = (int)((long long)chunks * (warp + 1) / kStreamWarps);
     const uint4* a4 = reinterpret_cast<const uint4*>(L.A) + ((long long)best * r + j_lo) * chunks;
-    for (int jb = 0; jb < nrows; jb += 4) {
-      float a0[4] = {0.f, 0.f, 0.f, 0.f}, a1[4] = {0.f, 0.f, 0.f, 0.f};
-      for (int c0 = s_lo + lane; c0 < s_hi; c0 += 128) {
-        uint4 wv[4][4];
-#pragma unroll
-        for (int rb = 0; rb < 4; ++rb)
-#pragma unroll
-          for (int u = 0; u < 4; ++u)
-            wv[rb][u] = (jb + rb < nrows && c0 + 32 * u < s_hi) ? __ldg(a4 + (long long)(jb + rb) * chunks + c0 + 32 * u) : make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          if (c0 + 32 * u < s_hi) {
-            const uint4 xv = xs4[c0 + 32 * u];
-#pragma unroll
-            for (int rb = 0; rb < 4; ++rb) {
-              a0[rb] = fmaf(bf16lo(xv.x), bf16lo(wv[rb][u].x), a0[rb]); a1[rb] = fmaf(bf16hi(xv.x), bf16hi(wv[rb][u].x), a1[rb]);
-              a0[rb] = fmaf(bf16lo(xv.y), bf16lo(wv[rb][u].y), a0[rb]); a1[rb] = fmaf(bf16hi(xv.y), bf16hi(wv[rb][u].y), a1[rb]);
-              a0[rb] = fmaf(bf16lo(xv.z), bf16lo(wv[rb][u].z), a0[rb]); a1[rb] = fmaf(bf16hi(xv.z), bf16hi(wv[rb][u].z), a1[rb]);
-              a0[rb] = fmaf(bf16lo(xv.w), bf16lo(wv[rb][u].w), a0[rb]); a1[rb] = fmaf(bf16hi(xv.w), bf16hi(wv[rb][u].w), a1[rb]);
-            }
-          }
-        }
-      }
-#pragma unroll
-      for (int rb = 0; rb < 4; ++rb) {
-        float a = a0[rb] + a1[rb];
-        for (int d = 16; d > 0; d >>= 1) a += __shfl_xor_sync(0xffffffffu, a, d);
-        if (lane == 0 && jb + rb < nrows) part[(jb + rb) * kStreamWarps + warp] = a;
-      }
-    }
+    const int upl = ((chunks + kStreamWarps - 1) / kStreamWarps + 31) / 32;   // loads per lane and row
+    if (upl == 1) stream_h_rows<1>(a4, xs4, part, nrows, chunks, s_lo, s_hi, warp, lane);
+    else if (upl == 2) stream_h_rows<2>(a4, xs4, part, nrows, chunks, s_lo, s_hi, warp, lane);
+    else stream_h_rows<4>(a4, xs4, part, nrows, chunks, s_lo, s_hi, warp, lane);
   }
 
   if (owner) {
@@ -453,17 +473,19 @@ __device__ __forceinline__ bool stream_report(const StreamLinear& L, int tg, int
   return old + units == stream_target(L, tg);
 }
 
-// (a) expert-product items [i_lo, i_hi) of one linear: item = token * 4G + group of 32 features; hs = h of all its tokens
+// (a) expert-product items [i_lo, i_hi) of one linear: item = token * 4G + group of 32 features; hs = h of all its tokens.
+// Consecutive items of one row group are reported together.
 __device__ void stream_expert(const StreamLinear& L, int i_lo, int i_hi, const float* hs, const DecodeTokInfo* toks) {
   const int lane = threadIdx.x & 31;
   const int G32 = L.G * 4, r = L.r, r8 = r >> 3;
   const int Np = L.G * 128;
+  unsigned run = 0u;
   for (int i = i_lo; i < i_hi; ++i) {
     const int tok = i / G32, g32 = i - tok * G32;
     if (g32 * 32 < L.N) {
       const uint4* bp = L.B_il + ((long long)toks[tok].expert * G32 + g32) * r8 * 32 + lane;
       const float* hv = hs + tok * r;
-      float z = 0.f;
+      float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
       for (int j0 = 0; j0 < r8; j0 += 20) {
         uint4 b[20];
 #pragma unroll
@@ -473,17 +495,22 @@ __device__ void stream_expert(const StreamLinear& L, int i_lo, int i_hi, const f
           if (j0 + u < r8) {
             const float4 h0 = *reinterpret_cast<const float4*>(hv + (j0 + u) * 8);
             const float4 h1 = *reinterpret_cast<const float4*>(hv + (j0 + u) * 8 + 4);
-            z = fmaf(bf16lo(b[u].x), h0.x, z); z = fmaf(bf16hi(b[u].x), h0.y, z);
-            z = fmaf(bf16lo(b[u].y), h0.z, z); z = fmaf(bf16hi(b[u].y), h0.w, z);
-            z = fmaf(bf16lo(b[u].z), h1.x, z); z = fmaf(bf16hi(b[u].z), h1.y, z);
-            z = fmaf(bf16lo(b[u].w), h1.z, z); z = fmaf(bf16hi(b[u].w), h1.w, z);
+            z0 = fmaf(bf16lo(b[u].x), h0.x, z0); z1 = fmaf(bf16hi(b[u].x), h0.y, z1);
+            z2 = fmaf(bf16lo(b[u].y), h0.z, z2); z3 = fmaf(bf16hi(b[u].y), h0.w, z3);
+            z0 = fmaf(bf16lo(b[u].z), h1.x, z0); z1 = fmaf(bf16hi(b[u].z), h1.y, z1);
+            z2 = fmaf(bf16lo(b[u].w), h1.z, z2); z3 = fmaf(bf16hi(b[u].w), h1.w, z3);
           }
         }
       }
-      L.z[(long long)tok * Np + g32 * 32 + lane] = z;
+      L.z[(long long)tok * Np + g32 * 32 + lane] = (z0 + z1) + (z2 + z3);
     }
-    const int tg = tok / kStreamTokenGroup, g = g32 >> 2;
-    if (stream_report(L, tg, g, 1u, lane)) stream_finish(L, tg, g, toks, lane);
+    ++run;
+    const bool last_of_group = (g32 & 3) == 3 || i + 1 == i_hi;   // the next item belongs to another row group (or token)
+    if (last_of_group) {
+      const int tg = tok / kStreamTokenGroup, g = g32 >> 2;
+      if (stream_report(L, tg, g, run, lane)) stream_finish(L, tg, g, toks, lane);
+      run = 0u;
+    }
   }
 }
 
@@ -491,7 +518,8 @@ __device__ void stream_expert(const StreamLinear& L, int i_lo, int i_hi, const f
 // or 8; with one token the masks need no shift (eight accumulators per feature, weighted 1 << b, exact in int32:
 // 127 * 128 * K < 2^31 for every K the library accepts).
 template <int MT>
-__device__ void stream_bits(const StreamLinear& L, int tg, int mg, int p_lo, int p_hi, const uint32_t* qs, int qwords, const DecodeTokInfo* toks) {
+__device__ void stream_bits(const StreamLinear& L, int tg, int mg, int p_lo, int p_hi, const uint32_t* qs, int qwords, const DecodeTokInfo* toks,
+                            int ahead) {
   constexpr bool NS = MT == 1;
   constexpr int NA = NS ? 8 : 1;
   const int lane = threadIdx.x & 31;
@@ -512,7 +540,13 @@ __device__ void stream_bits(const StreamLinear& L, int tg, int mg, int p_lo, int
   uint4 w[4];
 #pragma unroll
   for (int f = 0; f < 4; ++f) w[f] = __ldg(src + f * 32);
+  // the first chunks of the range on their way to L2 (a chunk is sixteen 128-byte lines: lanes 0..15 ask for one each)
+  const char* line = reinterpret_cast<const char*>(L.bits_il + (long long)p * 128) + (lane & 15) * 128;
+  if (lane < 16)
+    for (int a = 2; a < ahead && p + a < p_hi; ++a) asm volatile("prefetch.global.L2 [%0];" ::"l"(line + (long long)a * 2048));
   while (p < p_hi) {
+    if (lane < 16 && ahead > 0 && p + ahead < p_hi) asm volatile("prefetch.global.L2 [%0];" ::"l"(line + (long long)ahead * 2048));
+    line += 2048;
     uint4 wn[4];
     const uint4* nxt = src + (p + 1 < p_hi ? 128 : 0);
 #pragma unroll
@@ -585,37 +619,38 @@ __global__ void __launch_bounds__(kStreamThreads, 1) k_decode_stream(const __gri
   const int span_lo = (int)(T * cta / nC), span_hi = (int)(T * (cta + 1) / nC);
   const int zspan_lo = (int)(Z * cta / nC), zspan_hi = (int)(Z * (cta + 1) / nC);
 
-  if (bp.prefetch) {
-    // the sign bits of this CTA's span do not depend on phase 1: let them travel to L2 while it runs
-    for (int l = 0; l < bp.n; ++l) {
-      const StreamLinear& L = bp.lin[l];
-      const int lo = max(span_lo, L.chunk0) - L.chunk0, hi = min(span_hi, L.chunk0 + L.G * L.C) - L.chunk0;
-      if (lo >= hi) continue;
-      const char* base = reinterpret_cast<const char*>(L.bits_il + (long long)lo * 128);
-      const long long lines = (long long)(hi - lo) * 16;   // 128-byte lines
-      for (long long i = threadIdx.x; i < lines; i += kStreamThreads) asm volatile("prefetch.global.L2 [%0];" ::"l"(base + i * 128));
-    }
+  // the linears whose chunks / expert-product items this CTA's spans touch
+  int l_lo = 0, l_hi = 0, zl_lo = 0, zl_hi = 0;
+  for (int l = 0; l < bp.n; ++l) {
+    if (bp.chunk0[l + 1] <= span_lo) l_lo = l + 1;
+    if (bp.chunk0[l] < span_hi) l_hi = l + 1;
+    if (bp.z0[l + 1] <= zspan_lo) zl_lo = l + 1;
+    if (bp.z0[l] < zspan_hi) zl_hi = l + 1;
   }
 
-  // phase 0: this CTA's share of every linear's accumulators and counters starts at zero
-  for (int l = 0; l < bp.n; ++l) {
+  // phase 0: accumulators and counters start at zero.  A linear's words are shared out in proportion to its chunks:
+  // the CTA that owns chunks [lo, hi) of its GC chunks clears words [ceil(lo W / GC), ceil(hi W / GC)).
+  for (int l = l_lo; l < l_hi; ++l) {
     const StreamLinear& L = bp.lin[l];
-    const long long z_lo = (long long)L.zero_words * cta / nC, z_hi = (long long)L.zero_words * (cta + 1) / nC;
-    for (long long i = z_lo + threadIdx.x; i < z_hi; i += kStreamThreads) L.acc[i] = 0;
+    const long long gc = (long long)L.G * L.C;
+    const int lo = max(span_lo, L.chunk0) - L.chunk0, hi = min(span_hi, L.chunk0 + (int)gc) - L.chunk0;
+    if (lo >= hi) continue;
+    const long long w_lo = ((long long)lo * L.zero_words + gc - 1) / gc, w_hi = ((long long)hi * L.zero_words + gc - 1) / gc;
+    for (long long i = w_lo + threadIdx.x; i < w_hi; i += kStreamThreads) L.acc[i] = 0;
   }
 
-  // phase 1: token work of the linears this CTA shares
-  for (int l = 0; l < bp.n; ++l) {
-    const StreamLinear& L = bp.lin[l];
-    if (cta < L.cta_first || cta >= L.cta_first + L.cta_count) continue;
+  // phase 1: this CTA's share of one linear's token work
+  if (bp.duty[cta] != 255) {
+    const StreamLinear& L = bp.lin[bp.duty[cta]];
     const int s = cta - L.cta_first;
     const int rp = max(L.r, 1);
     const long long U = (long long)L.M * rp;
     const int u_lo = (int)(U * s / L.cta_count), u_hi = (int)(U * (s + 1) / L.cta_count);
-    if (u_lo >= u_hi) continue;
-    for (int t = u_lo / rp; t <= (u_hi - 1) / rp; ++t) {
-      const int j_lo = max(u_lo, t * rp) - t * rp, j_hi = min(u_hi, (t + 1) * rp) - t * rp;
-      stream_token(bp, L, t, j_lo, j_hi, j_lo == 0, stream_smem, sh);
+    if (u_lo < u_hi) {
+      for (int t = u_lo / rp; t <= (u_hi - 1) / rp; ++t) {
+        const int j_lo = max(u_lo, t * rp) - t * rp, j_hi = min(u_hi, (t + 1) * rp) - t * rp;
+        stream_token(bp, L, t, j_lo, j_hi, j_lo == 0, t == u_lo / rp, stream_smem, sh);
+      }
     }
   }
   stream_bar_arrive(bar);
@@ -625,22 +660,8 @@ __global__ void __launch_bounds__(kStreamThreads, 1) k_decode_stream(const __gri
     uint32_t* qs = reinterpret_cast<uint32_t*>(stream_smem);
     float* hs = reinterpret_cast<float*>(stream_smem + bp.off_h);
     DecodeTokInfo* toks = reinterpret_cast<DecodeTokInfo*>(stream_smem + bp.off_info);
-    // phase 2 (a): expert products.  What phase 1 wrote comes from other CTAs: read it through L2.
-    for (int l = 0; l < bp.n; ++l) {
-      const StreamLinear& L = bp.lin[l];
-      if (L.r == 0) continue;
-      const int zi = L.M * L.G * 4;
-      const int seg_lo = max(zspan_lo, L.z0) - L.z0, seg_hi = min(zspan_hi, L.z0 + zi) - L.z0;
-      if (seg_lo >= seg_hi) continue;
-      __syncthreads();
-      for (int i = threadIdx.x; i < L.M * L.r; i += kStreamThreads) hs[i] = __ldcg(L.h + i);
-      if (threadIdx.x < L.M) reinterpret_cast<int4*>(toks)[threadIdx.x] = __ldcg(reinterpret_cast<const int4*>(L.info) + threadIdx.x);
-      __syncthreads();
-      const int len = seg_hi - seg_lo;
-      stream_expert(L, seg_lo + (int)((long long)len * warp / kStreamWarps), seg_lo + (int)((long long)len * (warp + 1) / kStreamWarps), hs, toks);
-    }
-    // phase 2 (b): sign bits
-    for (int l = 0; l < bp.n; ++l) {
+    // phase 2 (a): sign bits
+    for (int l = l_lo; l < l_hi; ++l) {
       const StreamLinear& L = bp.lin[l];
       const int seg_lo = max(span_lo, L.chunk0) - L.chunk0, seg_hi = min(span_hi, L.chunk0 + L.G * L.C) - L.chunk0;
       if (seg_lo >= seg_hi) continue;
@@ -657,14 +678,27 @@ __global__ void __launch_bounds__(kStreamThreads, 1) k_decode_stream(const __gri
           if (threadIdx.x < L.M) reinterpret_cast<int4*>(toks)[threadIdx.x] = __ldcg(reinterpret_cast<const int4*>(L.info) + threadIdx.x);
         }
         __syncthreads();
-        if (mg == 1) stream_bits<1>(L, tg, mg, p_lo, p_hi, qs, qwords, toks);
-        else if (mg == 2) stream_bits<2>(L, tg, mg, p_lo, p_hi, qs, qwords, toks);
-        else if (mg <= 4) stream_bits<4>(L, tg, mg, p_lo, p_hi, qs, qwords, toks);
-        else stream_bits<8>(L, tg, mg, p_lo, p_hi, qs, qwords, toks);
+        if (mg == 1) stream_bits<1>(L, tg, mg, p_lo, p_hi, qs, qwords, toks, bp.prefetch);
+        else if (mg == 2) stream_bits<2>(L, tg, mg, p_lo, p_hi, qs, qwords, toks, bp.prefetch);
+        else if (mg <= 4) stream_bits<4>(L, tg, mg, p_lo, p_hi, qs, qwords, toks, bp.prefetch);
+        else stream_bits<8>(L, tg, mg, p_lo, p_hi, qs, qwords, toks, bp.prefetch);
       }
     }
+    // phase 2 (b): expert products.  What phase 1 wrote comes from other CTAs: read it through L2.
+    for (int l = zl_lo; l < zl_hi; ++l) {
+      const StreamLinear& L = bp.lin[l];
+      if (L.r == 0) continue;
+      const int zi = L.M * L.G * 4;
+      const int seg_lo = max(zspan_lo, L.z0) - L.z0, seg_hi = min(zspan_hi, L.z0 + zi) - L.z0;
+      if (seg_lo >= seg_hi) continue;
+      __syncthreads();
+      for (int i = threadIdx.x; i < L.M * L.r; i += kStreamThreads) hs[i] = __ldcg(L.h + i);
+      if (threadIdx.x < L.M) reinterpret_cast<int4*>(toks)[threadIdx.x] = __ldcg(reinterpret_cast<const int4*>(L.info) + threadIdx.x);
+      __syncthreads();
+      const int len = seg_hi - seg_lo;
+      stream_expert(L, seg_lo + (int)((long long)len * warp / kStreamWarps), seg_lo + (int)((long long)len * (warp + 1) / kStreamWarps), hs, toks);
+    }
   }
-  stream_bar_depart(bar);
 }
 
 // ---------------------------------------------------------------------------
@@ -757,17 +791,34 @@ int decode_stream_launch(const DecodeItemArgs* items, int n, cudaStream_t st) {
   }
   bp.total_chunks = (int)total;
   bp.total_z = (int)total_z;
-  // the token work of a linear is shared by the CTAs whose span of the chunk list touches it
+  for (int i = 0; i <= kStreamMaxBatch; ++i) {
+    bp.chunk0[i] = i < n ? bp.lin[i].chunk0 : (int)total;
+    bp.z0[i] = i < n ? bp.lin[i].z0 : (int)total_z;
+  }
+  // the token work of a linear belongs to CTAs of its own, as many as its share of that work (at least one)
   const int nC = sms;
-  for (int i = 0; i < n; ++i) {
-    StreamLinear& L = bp.lin[i];
-    const long long lo = L.chunk0, hi = L.chunk0 + (long long)L.G * L.C;
-    int first = (int)(lo * nC / total);
-    while (first > 0 && total * first / nC > lo) --first;
-    while (total * (first + 1) / nC <= lo) ++first;
-    int last = first;
-    while (last + 1 < nC && total * (last + 1) / nC < hi) ++last;
-    L.cta_first = first; L.cta_count = last - first + 1;
+  if (n > nC) return PQ_ERR_UNSUPPORTED;
+  {
+    double cost[kStreamMaxBatch], sum = 0.0;
+    for (int i = 0; i < n; ++i) {
+      const StreamLinear& L = bp.lin[i];
+      cost[i] = (double)L.M * L.K * (L.r + (L.E > 1 ? L.E : 0) + 2);
+      sum += cost[i];
+    }
+    int next = 0;
+    double run = 0.0;
+    for (int i = 0; i < n; ++i) {
+      run += cost[i];
+      int end = i + 1 == n ? nC : (int)(run / sum * (nC - n) + 0.5) + (i + 1);   // one CTA each, the rest by cost
+      end = std::min(std::max(end, next + 1), nC - (n - 1 - i));
+      bp.lin[i].cta_first = next;
+      bp.lin[i].cta_count = end - next;
+      next = end;
+    }
+    if (nC > 160) return PQ_ERR_UNSUPPORTED;
+    for (int c = 0; c < 160; ++c) bp.duty[c] = 255;
+    for (int i = 0; i < n; ++i)
+      for (int c = bp.lin[i].cta_first; c < bp.lin[i].cta_first + bp.lin[i].cta_count; ++c) bp.duty[c] = (unsigned char)i;
   }
   // shared memory: phase 1 [token][router rows][partial sums], phase 2 [codes][h][token records]
   xbytes = s_up256(xbytes);
@@ -784,7 +835,7 @@ int decode_stream_launch(const DecodeItemArgs* items, int n, cudaStream_t st) {
   if (smem > kStreamSmemLimit) return PQ_ERR_UNSUPPORTED;
   bp.bar_slot = stream_bar_slot(st);
   if (bp.bar_slot < 0) return PQ_ERR_UNSUPPORTED;
-  bp.prefetch = g_decode_stream_prefetch;
+  bp.prefetch = g_decode_stream_prefetch ? 4 : 0;
   static const bool limit_set = cudaFuncSetAttribute(k_decode_stream, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStreamSmemLimit) == cudaSuccess;
   if (!limit_set) return PQ_ERR_CUDA;
   cudaLaunchAttribute attr[1];
