@@ -488,8 +488,10 @@ def subrecords(args, ctx, engine):
             weights = build_decode_weights(ctx)
             r = {"workload": decode_workload_text(None, False), "note": (
                 "fraction of the measured HBM rate = algorithmic bytes / time / hbm_gbs.  batched16: 16 independent linears per "
-                "launch pair (other sequences, parallel projections); pairs: what one sequence's model allows (gate + up of a block "
-                "together); serial: one call per linear, each after the previous one")}
+                "launch (other sequences, parallel projections), one cooperative streaming kernel on weights in its own layout; "
+                "pairs: what one sequence's model allows (gate + up of a block together); serial: one call per linear, each after "
+                "the previous one -- both on the two-kernel path, which the library picks for small groups"),
+                "kernels": ctx.decode_kernels}
             for M in (1, 4, 16):
                 d = measure_decode(ctx, M, max(5, min(args.steps, 20)), weights, full=True)
                 r[f"m{M}"] = {"batched16": d["batched"], "pairs": d["pairs"], "serial": d["serial"],
@@ -552,7 +554,7 @@ def make_decode_layers(ctx, M, weights, rmsnorm=False):
         act = I.decode_activations(M, w["K"], w["E"], seed=w["seed"])
         L.w_bits, L.w_scales, L.A, L.B = w["w_bits"], w["w_scales"], w["A"], w["B"]
         L.w_s8 = None
-        if ctx.decode_kernels == "stream":
+        if ctx.decode_kernels != "pair":
             L.w_bits_il, L.B_il = w["w_bits_il"], w["B_il"]
         L.X = torch.from_numpy(act["X"]).to(device).to(torch.bfloat16)
         L.Wr = torch.from_numpy(act["Wr"]).to(device).to(torch.bfloat16)
@@ -679,7 +681,8 @@ def run_decode(args, ctx):
             "dtype": "s8 x s8 -> s32 (1-bit branch), bf16 -> f32 (experts)", "data": "synthetic",
             "config": {"workload": decode_workload_text(M, args.decode_rmsnorm),
                        "linears_per_step": nlin, "l2": f"{d['algo'] / 1e6:.0f} MB of distinct weights per step, larger than L2",
-                       "launch": f"one CUDA graph per step, pq_decode_batch over groups of {args.decode_batch} independent linears", "replicas": ctx.world},
+                       "launch": f"one CUDA graph per step, pq_decode_batch over groups of {args.decode_batch} independent linears",
+                       "kernels": ctx.decode_kernels, "replicas": ctx.world},
             "roofline": {"kernel": "decode kernels (all launches of a step)", "bound": "hbm", "achieved": b["gbs"],
                          "peak": ctx.peaks["hbm_gbs"], "unit": "GB/s", "frac": b["hbm_frac"],
                          "peak_source": f"{ctx.peak_kind} hbm_gbs", "algorithmic_bytes_per_step": d["algo"],
@@ -866,8 +869,9 @@ def main():
     ap.add_argument("--decode-tokens", type=int, default=1, choices=range(1, 17), metavar="M")
     ap.add_argument("--decode-skip-serial", action="store_true", help="time only the batched graph (shorter runs under a profiler)")
     ap.add_argument("--decode-batch", type=int, default=16, help="independent decode linears per pq_decode_batch call")
-    ap.add_argument("--decode-kernels", default="stream", choices=["stream", "pair"],
-                    help="stream: the cooperative streaming kernel on weights in its own layout; pair: the two-kernel path on the plain layout")
+    ap.add_argument("--decode-kernels", default="auto", choices=["auto", "stream", "pair"],
+                    help="auto: the library picks per launch group; stream: the cooperative streaming kernel wherever the items allow; "
+                         "pair: the two-kernel path on the plain layout")
     ap.add_argument("--decode-prefetch", type=int, default=1, choices=[0, 1], help="streaming decode kernel: L2 prefetch of the sign bits during the token work")
     ap.add_argument("--decode-rmsnorm", action="store_true", help="decode from un-normalised activations, RMSNorm fused into the token preparation")
     ap.add_argument("--decoder-one-form", action="store_true", help="decoder workload: only the form with 8 experts on every projection")
@@ -885,6 +889,7 @@ def main():
         return
     ctx = Ctx()
     ctx.decode_kernels = args.decode_kernels
+    ctx.pqb.pq_set_option(ctx.pqb.PQ_OPT_DECODE_STREAM, {"auto": 1, "stream": 2, "pair": 0}[args.decode_kernels])
     ctx.pqb.pq_set_option(ctx.pqb.PQ_OPT_DECODE_PREFETCH, args.decode_prefetch)
     if args.workload == "decode":
         run_decode(args, ctx)

@@ -289,7 +289,8 @@ typedef struct pq_decode_item {
   const uint16_t* norm_weight;
   float norm_eps;
   /* The weights in the layout of the streaming decode kernel (pq_pack_decode), or NULL.  When every item of a
-   * launch group carries them (w_bits_il, and B_il if r > 0), the group runs as ONE cooperative kernel that
+   * launch group carries them (w_bits_il, and B_il if r > 0) and the group is large enough for it to pay
+   * (PQ_OPT_DECODE_STREAM), the group runs as ONE cooperative kernel that
    * streams each weight byte once with coalesced loads; results: the same integers (codes, routing, sums over k),
    * Y within the tolerance of the float epilogue (the expert product is summed in another order).  Otherwise, and
    * for shapes that kernel does not take (r not a multiple of 8), the two-kernel path is used.  w_bits, A and B
@@ -371,7 +372,9 @@ int pq_device_status(void* stream, int* code, int* where);
  *   outputs of that call are undefined.  Applies to the current device; blocks until the device's
  *   earlier work has finished.  Meant for pq_debug_gemm; do not shorten the limit around the decode
  *   entry points, whose later stages read indices an abandoned stage has not delivered.
- *   PQ_OPT_DECODE_STREAM (default 1): 0 = pq_decode_batch ignores w_bits_il / B_il and always uses the two-kernel path.
+ *   PQ_OPT_DECODE_STREAM (default 1): which launch groups of pq_decode_batch (up to 16 consecutive items) run on the
+ *   streaming kernel when their items carry w_bits_il / B_il.  1 = those for which it is the faster of the two paths
+ *   (12 or more linears; 6 or more when no item has more than two tokens); 2 = every group; 0 = none.
  *   PQ_OPT_DECODE_PREFETCH (default 1): the streaming decode kernel asks for its sign bits to be brought into L2
  *   while it prepares the tokens. */
 enum { PQ_OPT_DECODE_PDL = 1, PQ_OPT_SIDE_STREAM = 2, PQ_OPT_SPIN_CYCLES = 3, PQ_OPT_DECODE_STREAM = 4, PQ_OPT_DECODE_PREFETCH = 5 };

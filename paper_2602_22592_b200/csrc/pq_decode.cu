@@ -798,11 +798,19 @@ int decode_batch(const DecodeItemArgs* items, int n, cudaStream_t st) {
   for (int i = 0; i < n; i += kDecodeMaxBatch) {
     const int m = n - i < kDecodeMaxBatch ? n - i : kDecodeMaxBatch;
     // the streaming kernel takes a group whose items all carry its weight layout; otherwise the kernels above
+    // (measured on the 3B shapes: its grid barrier and its longer chain of dependent steps cost about as much as eight
+    // linears' worth of streaming, so small groups, and mid-sized groups of many tokens, stay on the two kernels above)
     int rc = PQ_ERR_UNSUPPORTED;
-    if (decode_stream_enabled()) {
+    const int mode = decode_stream_mode();
+    if (mode > 0) {
       bool all = true;
-      for (int k = 0; k < m; ++k) all = all && items[i + k].bits_il != nullptr;
-      if (all) rc = decode_stream_launch(items + i, m, st);
+      int max_m = 1;
+      for (int k = 0; k < m; ++k) {
+        all = all && items[i + k].bits_il != nullptr;
+        max_m = std::max(max_m, items[i + k].a.T);
+      }
+      const bool worth = mode > 1 || m >= 12 || (m >= 6 && max_m <= 2);
+      if (all && worth) rc = decode_stream_launch(items + i, m, st);
     }
     if (rc == PQ_ERR_UNSUPPORTED) rc = decode_launch(items + i, m, st);
     if (rc) return rc;

@@ -607,6 +607,56 @@ __device__ void stream_bits(const StreamLinear& L, int tg, int mg, int p_lo, int
 }
 
 // ---------------------------------------------------------------------------
+// half a CTA (eight warps, named barrier `bid`) walking a range of one of the two launch-wide work lists.
+// What phase 1 wrote comes from other CTAs: it is read through L2.
+// ---------------------------------------------------------------------------
+constexpr int kStreamHalfWarps = kStreamWarps / 2;
+constexpr int kStreamHalfThreads = kStreamThreads / 2;
+__device__ __forceinline__ void stream_half_sync(int bid) { asm volatile("bar.sync %0, %1;" ::"r"(bid), "n"(kStreamHalfThreads) : "memory"); }
+
+__device__ void stream_half_bits(const StreamBatch& bp, int lo, int hi, int bid, uint32_t* qs, DecodeTokInfo* toks) {
+  const int tid = threadIdx.x & (kStreamHalfThreads - 1), gw = tid >> 5;
+  for (int l = 0; l < bp.n; ++l) {
+    if (bp.chunk0[l + 1] <= lo || bp.chunk0[l] >= hi) continue;
+    const StreamLinear& L = bp.lin[l];
+    const int seg_lo = max(lo, L.chunk0) - L.chunk0, seg_hi = min(hi, bp.chunk0[l + 1]) - L.chunk0;
+    const int qwords = L.C * 32;
+    const int len = seg_hi - seg_lo;
+    const int p_lo = seg_lo + (int)((long long)len * gw / kStreamHalfWarps), p_hi = seg_lo + (int)((long long)len * (gw + 1) / kStreamHalfWarps);
+    for (int tg = 0; tg * kStreamTokenGroup < L.M; ++tg) {
+      const int mg = min(kStreamTokenGroup, L.M - tg * kStreamTokenGroup);
+      stream_half_sync(bid);   // the previous codes and token records are no longer read
+      {
+        const uint4* from = reinterpret_cast<const uint4*>(L.qg + (long long)tg * kStreamTokenGroup * qwords);
+        uint4* to = reinterpret_cast<uint4*>(qs);
+        for (int i = tid; i < mg * (qwords >> 2); i += kStreamHalfThreads) to[i] = __ldcg(from + i);
+        if (tid < L.M) reinterpret_cast<int4*>(toks)[tid] = __ldcg(reinterpret_cast<const int4*>(L.info) + tid);
+      }
+      stream_half_sync(bid);
+      if (mg == 1) stream_bits<1>(L, tg, mg, p_lo, p_hi, qs, qwords, toks, bp.prefetch);
+      else if (mg == 2) stream_bits<2>(L, tg, mg, p_lo, p_hi, qs, qwords, toks, bp.prefetch);
+      else if (mg <= 4) stream_bits<4>(L, tg, mg, p_lo, p_hi, qs, qwords, toks, bp.prefetch);
+      else stream_bits<8>(L, tg, mg, p_lo, p_hi, qs, qwords, toks, bp.prefetch);
+    }
+  }
+}
+
+__device__ void stream_half_expert(const StreamBatch& bp, int lo, int hi, int bid, float* hs, DecodeTokInfo* toks) {
+  const int tid = threadIdx.x & (kStreamHalfThreads - 1), gw = tid >> 5;
+  for (int l = 0; l < bp.n; ++l) {
+    if (bp.z0[l + 1] <= lo || bp.z0[l] >= hi || bp.z0[l + 1] == bp.z0[l]) continue;
+    const StreamLinear& L = bp.lin[l];
+    const int seg_lo = max(lo, L.z0) - L.z0, seg_hi = min(hi, bp.z0[l + 1]) - L.z0;
+    stream_half_sync(bid);
+    for (int i = tid; i < L.M * L.r; i += kStreamHalfThreads) hs[i] = __ldcg(L.h + i);
+    if (tid < L.M) reinterpret_cast<int4*>(toks)[tid] = __ldcg(reinterpret_cast<const int4*>(L.info) + tid);
+    stream_half_sync(bid);
+    const int len = seg_hi - seg_lo;
+    stream_expert(L, seg_lo + (int)((long long)len * gw / kStreamHalfWarps), seg_lo + (int)((long long)len * (gw + 1) / kStreamHalfWarps), hs, toks);
+  }
+}
+
+// ---------------------------------------------------------------------------
 // the kernel: grid = one CTA per SM (cooperative launch), 512 threads
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(kStreamThreads, 1) k_decode_stream(const __grid_constant__ StreamBatch bp) {
@@ -620,12 +670,10 @@ __global__ void __launch_bounds__(kStreamThreads, 1) k_decode_stream(const __gri
   const int zspan_lo = (int)(Z * cta / nC), zspan_hi = (int)(Z * (cta + 1) / nC);
 
   // the linears whose chunks / expert-product items this CTA's spans touch
-  int l_lo = 0, l_hi = 0, zl_lo = 0, zl_hi = 0;
+  int l_lo = 0, l_hi = 0;
   for (int l = 0; l < bp.n; ++l) {
     if (bp.chunk0[l + 1] <= span_lo) l_lo = l + 1;
     if (bp.chunk0[l] < span_hi) l_hi = l + 1;
-    if (bp.z0[l + 1] <= zspan_lo) zl_lo = l + 1;
-    if (bp.z0[l] < zspan_hi) zl_hi = l + 1;
   }
 
   // phase 0: accumulators and counters start at zero.  A linear's words are shared out in proportion to its chunks:
@@ -657,47 +705,19 @@ __global__ void __launch_bounds__(kStreamThreads, 1) k_decode_stream(const __gri
   const bool ok = stream_bar_wait(bar, &sh.ok);
 
   if (ok) {
+    // phase 2: the bit product is bound by instruction issue, the expert product by the latency of its loads, so
+    // the two halves of the CTA (eight warps each, a named barrier each) do one of each at a time: half 0 takes the
+    // first half of the CTA's chunks, then the second half of its expert-product items; half 1 the other way round.
     uint32_t* qs = reinterpret_cast<uint32_t*>(stream_smem);
     float* hs = reinterpret_cast<float*>(stream_smem + bp.off_h);
-    DecodeTokInfo* toks = reinterpret_cast<DecodeTokInfo*>(stream_smem + bp.off_info);
-    // phase 2 (a): sign bits
-    for (int l = l_lo; l < l_hi; ++l) {
-      const StreamLinear& L = bp.lin[l];
-      const int seg_lo = max(span_lo, L.chunk0) - L.chunk0, seg_hi = min(span_hi, L.chunk0 + L.G * L.C) - L.chunk0;
-      if (seg_lo >= seg_hi) continue;
-      const int qwords = L.C * 32;
-      const int len = seg_hi - seg_lo;
-      const int p_lo = seg_lo + (int)((long long)len * warp / kStreamWarps), p_hi = seg_lo + (int)((long long)len * (warp + 1) / kStreamWarps);
-      for (int tg = 0; tg * kStreamTokenGroup < L.M; ++tg) {
-        const int mg = min(kStreamTokenGroup, L.M - tg * kStreamTokenGroup);
-        __syncthreads();   // the previous codes and token records are no longer read
-        {
-          const uint4* from = reinterpret_cast<const uint4*>(L.qg + (long long)tg * kStreamTokenGroup * qwords);
-          uint4* to = reinterpret_cast<uint4*>(qs);
-          for (int i = threadIdx.x; i < mg * (qwords >> 2); i += kStreamThreads) to[i] = __ldcg(from + i);
-          if (threadIdx.x < L.M) reinterpret_cast<int4*>(toks)[threadIdx.x] = __ldcg(reinterpret_cast<const int4*>(L.info) + threadIdx.x);
-        }
-        __syncthreads();
-        if (mg == 1) stream_bits<1>(L, tg, mg, p_lo, p_hi, qs, qwords, toks, bp.prefetch);
-        else if (mg == 2) stream_bits<2>(L, tg, mg, p_lo, p_hi, qs, qwords, toks, bp.prefetch);
-        else if (mg <= 4) stream_bits<4>(L, tg, mg, p_lo, p_hi, qs, qwords, toks, bp.prefetch);
-        else stream_bits<8>(L, tg, mg, p_lo, p_hi, qs, qwords, toks, bp.prefetch);
-      }
-    }
-    // phase 2 (b): expert products.  What phase 1 wrote comes from other CTAs: read it through L2.
-    for (int l = zl_lo; l < zl_hi; ++l) {
-      const StreamLinear& L = bp.lin[l];
-      if (L.r == 0) continue;
-      const int zi = L.M * L.G * 4;
-      const int seg_lo = max(zspan_lo, L.z0) - L.z0, seg_hi = min(zspan_hi, L.z0 + zi) - L.z0;
-      if (seg_lo >= seg_hi) continue;
-      __syncthreads();
-      for (int i = threadIdx.x; i < L.M * L.r; i += kStreamThreads) hs[i] = __ldcg(L.h + i);
-      if (threadIdx.x < L.M) reinterpret_cast<int4*>(toks)[threadIdx.x] = __ldcg(reinterpret_cast<const int4*>(L.info) + threadIdx.x);
-      __syncthreads();
-      const int len = seg_hi - seg_lo;
-      stream_expert(L, seg_lo + (int)((long long)len * warp / kStreamWarps), seg_lo + (int)((long long)len * (warp + 1) / kStreamWarps), hs, toks);
-    }
+    const int half = warp / kStreamHalfWarps;
+    DecodeTokInfo* toks = reinterpret_cast<DecodeTokInfo*>(stream_smem + bp.off_info) + half * kDecodeMaxTokens;
+    const int span_mid = span_lo + (span_hi - span_lo) / 2, zspan_mid = zspan_lo + (zspan_hi - zspan_lo) / 2;
+    if (half == 0) stream_half_bits(bp, span_lo, span_mid, 1, qs, toks);
+    else stream_half_expert(bp, zspan_lo, zspan_mid, 2, hs, toks);
+    __syncthreads();   // the halves swap the code and h buffers
+    if (half == 0) stream_half_expert(bp, zspan_mid, zspan_hi, 1, hs, toks);
+    else stream_half_bits(bp, span_mid, span_hi, 2, qs, toks);
   }
 }
 
@@ -717,9 +737,9 @@ size_t decode_stream_extra_bytes(int M, int K, int N, int r) {
 
 static int g_decode_stream_on = 1;
 static int g_decode_stream_prefetch = 1;
-void decode_stream_enable(int on) { g_decode_stream_on = on ? 1 : 0; }
+void decode_stream_enable(int mode) { g_decode_stream_on = mode < 0 ? 0 : mode > 2 ? 2 : mode; }
 void decode_stream_prefetch(int on) { g_decode_stream_prefetch = on ? 1 : 0; }
-bool decode_stream_enabled() { return g_decode_stream_on != 0; }
+int decode_stream_mode() { return g_decode_stream_on; }
 
 void decode_stream_reset() {
   void* p = nullptr;
@@ -830,7 +850,7 @@ int decode_stream_launch(const DecodeItemArgs* items, int n, cudaStream_t st) {
   const size_t smem1 = bp.off_part + s_up256(part);
   bp.off_h = (int)s_up256(codes);
   bp.off_info = (int)(bp.off_h + s_up256(hbytes));
-  const size_t smem2 = bp.off_info + 256;
+  const size_t smem2 = bp.off_info + 2 * kDecodeMaxTokens * sizeof(DecodeTokInfo);
   const size_t smem = std::max(smem1, smem2);
   if (smem > kStreamSmemLimit) return PQ_ERR_UNSUPPORTED;
   bp.bar_slot = stream_bar_slot(st);

@@ -137,9 +137,9 @@ void decode_pack_sizes(int K, int N, int r, int E, size_t* bits_bytes, size_t* b
 int decode_pack(int K, int N, int r, int E, const uint32_t* bits, const uint16_t* B, uint32_t* bits_il, uint16_t* B_il, cudaStream_t st);
 size_t decode_stream_extra_bytes(int M, int K, int N, int r);
 int decode_stream_launch(const DecodeItemArgs* items, int n, cudaStream_t st);   // PQ_ERR_UNSUPPORTED: use the other kernels
-void decode_stream_enable(int on);
+void decode_stream_enable(int mode);   // 0 never, 1 where it pays (default), 2 wherever the items allow
 void decode_stream_prefetch(int on);
-bool decode_stream_enabled();
+int decode_stream_mode();
 void decode_stream_reset();
 int decode_batch(const DecodeItemArgs* items, int n, cudaStream_t st);   // independent linears, launched together
 void decode_set_pdl(int on);

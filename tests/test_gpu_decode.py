@@ -17,8 +17,10 @@ pytestmark = pytest.mark.gpu
 def decode_kernels(request):
     """Every test runs twice: on the streaming kernel (weights in its own layout) and on the two-kernel path."""
     PQLinear.stream_decode = request.param == "stream"
+    pqb.pq_set_option(pqb.PQ_OPT_DECODE_STREAM, 2 if request.param == "stream" else 0)   # 2: also for one small linear
     yield request.param
     PQLinear.stream_decode = True
+    pqb.pq_set_option(pqb.PQ_OPT_DECODE_STREAM, 1)
 
 
 def run_decode(c, scale_vector=False):
