@@ -872,6 +872,7 @@ def main():
     ap.add_argument("--decode-kernels", default="auto", choices=["auto", "stream", "pair"],
                     help="auto: the library picks per launch group; stream: the cooperative streaming kernel wherever the items allow; "
                          "pair: the two-kernel path on the plain layout")
+    ap.add_argument("--decode-mma-from", type=int, default=5, help="streaming decode kernel: token groups of at least this size use the tensor-core bit product")
     ap.add_argument("--decode-prefetch", type=int, default=1, choices=[0, 1], help="streaming decode kernel: L2 prefetch of the sign bits during the token work")
     ap.add_argument("--decode-rmsnorm", action="store_true", help="decode from un-normalised activations, RMSNorm fused into the token preparation")
     ap.add_argument("--decoder-one-form", action="store_true", help="decoder workload: only the form with 8 experts on every projection")
@@ -891,6 +892,7 @@ def main():
     ctx.decode_kernels = args.decode_kernels
     ctx.pqb.pq_set_option(ctx.pqb.PQ_OPT_DECODE_STREAM, {"auto": 1, "stream": 2, "pair": 0}[args.decode_kernels])
     ctx.pqb.pq_set_option(ctx.pqb.PQ_OPT_DECODE_PREFETCH, args.decode_prefetch)
+    ctx.pqb.pq_set_option(ctx.pqb.PQ_OPT_DECODE_MMA_FROM, args.decode_mma_from)
     if args.workload == "decode":
         run_decode(args, ctx)
     elif args.workload == "decoder":

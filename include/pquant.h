@@ -375,9 +375,12 @@ int pq_device_status(void* stream, int* code, int* where);
  *   PQ_OPT_DECODE_STREAM (default 1): which launch groups of pq_decode_batch (up to 16 consecutive items) run on the
  *   streaming kernel when their items carry w_bits_il / B_il.  1 = those for which it is the faster of the two paths
  *   (12 or more linears; 6 or more when no item has more than two tokens); 2 = every group; 0 = none.
- *   PQ_OPT_DECODE_PREFETCH (default 1): the streaming decode kernel asks for its sign bits to be brought into L2
- *   while it prepares the tokens. */
-enum { PQ_OPT_DECODE_PDL = 1, PQ_OPT_SIDE_STREAM = 2, PQ_OPT_SPIN_CYCLES = 3, PQ_OPT_DECODE_STREAM = 4, PQ_OPT_DECODE_PREFETCH = 5 };
+ *   PQ_OPT_DECODE_PREFETCH (default 1): the streaming decode kernel asks for the sign bits four chunks ahead of its
+ *   bit product to be brought into L2.
+ *   PQ_OPT_DECODE_MMA_FROM (default 5): the streaming decode kernel multiplies the sign bits of a group of at least this
+ *   many tokens on the tensor cores (mma.sync u8 x s8) and of fewer tokens with dp4a; both are exact.  17 = dp4a only. */
+enum { PQ_OPT_DECODE_PDL = 1, PQ_OPT_SIDE_STREAM = 2, PQ_OPT_SPIN_CYCLES = 3, PQ_OPT_DECODE_STREAM = 4, PQ_OPT_DECODE_PREFETCH = 5,
+       PQ_OPT_DECODE_MMA_FROM = 6 };
 int pq_set_option(int option, int value);
 
 /* Cumulative number of kernels this library has launched in this process. */

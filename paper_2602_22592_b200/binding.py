@@ -366,6 +366,7 @@ PQ_OPT_SIDE_STREAM = 2
 PQ_OPT_SPIN_CYCLES = 3
 PQ_OPT_DECODE_STREAM = 4
 PQ_OPT_DECODE_PREFETCH = 5
+PQ_OPT_DECODE_MMA_FROM = 6
 
 
 def pq_set_option(option: int, value: int):

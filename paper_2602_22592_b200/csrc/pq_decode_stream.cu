@@ -74,6 +74,7 @@ struct StreamBatch {
   int total_chunks, total_z;
   int bar_slot;
   int prefetch;             // chunks ahead of the bit product for which L2 prefetches are issued (0 = none)
+  int mma_from;             // token groups of at least this many tokens take the tensor-core bit product
   int router_rows;          // router rows that fit in shared memory beside the token
   int off_rows, off_part;   // phase 1 carve-up: [token][router rows][partial sums of h]
   int off_h, off_info;      // phase 2 carve-up: [codes][h][token info]
@@ -421,7 +422,7 @@ __device__ __forceinline__ int dp4a_s8u8(uint32_t q, uint32_t m, int c) {
 
 __device__ __forceinline__ unsigned stream_target(const StreamLinear& L, int tg) {
   const int mg = min(kStreamTokenGroup, L.M - tg * kStreamTokenGroup);
-  return (unsigned)(L.C + (L.r > 0 ? 4 * mg : 0));
+  return (unsigned)(2 * L.C + (L.r > 0 ? 4 * mg : 0));   // two units per chunk, one per expert-product item
 }
 
 // Eq. 10-11 for row group g and the tokens of group tg: everything it needs is complete in global memory
@@ -518,7 +519,7 @@ __device__ void stream_expert(const StreamLinear& L, int i_lo, int i_hi, const f
 // or 8; with one token the masks need no shift (eight accumulators per feature, weighted 1 << b, exact in int32:
 // 127 * 128 * K < 2^31 for every K the library accepts).
 template <int MT>
-__device__ void stream_bits(const StreamLinear& L, int tg, int mg, int p_lo, int p_hi, const uint32_t* qs, int qwords, const DecodeTokInfo* toks,
+__device__ void stream_bits(const StreamLinear& L, int tg, int mg, int p_lo, int p_hi, const uint32_t* qs, int qstride, const DecodeTokInfo* toks,
                             int ahead) {
   constexpr bool NS = MT == 1;
   constexpr int NA = NS ? 8 : 1;
@@ -558,7 +559,7 @@ __device__ void stream_bits(const StreamLinear& L, int tg, int mg, int p_lo, int
       for (int hh = 0; hh < 2; ++hh) {
         uint4 qq[MT];
 #pragma unroll
-        for (int t = 0; t < MT; ++t) qq[t] = *reinterpret_cast<const uint4*>(qc + t * qwords + i * 8 + hh * 4);
+        for (int t = 0; t < MT; ++t) qq[t] = *reinterpret_cast<const uint4*>(qc + t * qstride + i * 8 + hh * 4);
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
 #pragma unroll
@@ -599,60 +600,82 @@ __device__ void stream_bits(const StreamLinear& L, int tg, int mg, int p_lo, int
         for (int t = 0; t < MT; ++t)
 #pragma unroll
           for (int a = 0; a < NA; ++a) acc[f][t][a] = 0;
-      if (stream_report(L, tg, g, (unsigned)delivered, lane)) stream_finish(L, tg, g, toks, lane);
+      if (stream_report(L, tg, g, 2u * (unsigned)delivered, lane)) stream_finish(L, tg, g, toks, lane);
       if (c == C) { c = 0; ++g; }
       delivered = 0;
     }
   }
 }
 
-// ---------------------------------------------------------------------------
-// half a CTA (eight warps, named barrier `bid`) walking a range of one of the two launch-wide work lists.
-// What phase 1 wrote comes from other CTAs: it is read through L2.
-// ---------------------------------------------------------------------------
-constexpr int kStreamHalfWarps = kStreamWarps / 2;
-constexpr int kStreamHalfThreads = kStreamThreads / 2;
-__device__ __forceinline__ void stream_half_sync(int bid) { asm volatile("bar.sync %0, %1;" ::"r"(bid), "n"(kStreamHalfThreads) : "memory"); }
-
-__device__ void stream_half_bits(const StreamBatch& bp, int lo, int hi, int bid, uint32_t* qs, DecodeTokInfo* toks) {
-  const int tid = threadIdx.x & (kStreamHalfThreads - 1), gw = tid >> 5;
-  for (int l = 0; l < bp.n; ++l) {
-    if (bp.chunk0[l + 1] <= lo || bp.chunk0[l] >= hi) continue;
-    const StreamLinear& L = bp.lin[l];
-    const int seg_lo = max(lo, L.chunk0) - L.chunk0, seg_hi = min(hi, bp.chunk0[l + 1]) - L.chunk0;
-    const int qwords = L.C * 32;
-    const int len = seg_hi - seg_lo;
-    const int p_lo = seg_lo + (int)((long long)len * gw / kStreamHalfWarps), p_hi = seg_lo + (int)((long long)len * (gw + 1) / kStreamHalfWarps);
-    for (int tg = 0; tg * kStreamTokenGroup < L.M; ++tg) {
-      const int mg = min(kStreamTokenGroup, L.M - tg * kStreamTokenGroup);
-      stream_half_sync(bid);   // the previous codes and token records are no longer read
-      {
-        const uint4* from = reinterpret_cast<const uint4*>(L.qg + (long long)tg * kStreamTokenGroup * qwords);
-        uint4* to = reinterpret_cast<uint4*>(qs);
-        for (int i = tid; i < mg * (qwords >> 2); i += kStreamHalfThreads) to[i] = __ldcg(from + i);
-        if (tid < L.M) reinterpret_cast<int4*>(toks)[tid] = __ldcg(reinterpret_cast<const int4*>(L.info) + tid);
+// (b') the same chunks on the tensor cores (mma.sync m16n8k32, u8 masks x s8 codes, exact in int32), for five to eight
+// tokens: sixteen features x 32 contraction values x eight tokens per instruction, where dp4a pays once per token.
+// A block of a chunk is 128 rows of 16 bytes in feature order, so thread (g = lane / 4, c = lane % 4) finds the
+// four bit words of features 16 T + g and 16 T + g + 8 at rows of their own; like every thread of its quad it loads
+// them whole and takes the bits c + 8 j (mask 0x01010101 of w >> c) and c + 4 + 8 j (mask 0x10101010: the value 16,
+// summed in a second accumulator that stays an exact multiple of 16) -- the codes in shared memory are already in
+// that order (word b of a group of 32 holds k = b + 8 j).  A row group is walked in two halves of 64 features so
+// that the accumulators (4 tiles x 2 x 4) and a prefetched half block fit in registers.
+__device__ void stream_bits_mma(const StreamLinear& L, int tg, int mg, int p_lo, int p_hi, const uint32_t* qs, int qstride,
+                                const DecodeTokInfo* toks, int ahead) {
+  const int lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3;
+  const int C = L.C;
+  const int Np = L.G * 128;
+  const uint32_t* qtok = qs + min(g, mg - 1) * qstride + c;   // token g of the group (surplus lanes read the last one)
+  int p = p_lo;
+  while (p < p_hi) {
+    const int rg = p / C, c0 = p - rg * C, n = min(C - c0, p_hi - p);
+    for (int half = 0; half < 2; ++half) {
+      int a1[4][4], a16[4][4];
+#pragma unroll
+      for (int T = 0; T < 4; ++T)
+#pragma unroll
+        for (int u = 0; u < 4; ++u) { a1[T][u] = 0; a16[T][u] = 0; }
+      const uint4* blk = L.bits_il + (long long)p * 128 + half * 64 + g;
+      const char* line = reinterpret_cast<const char*>(L.bits_il + (long long)p * 128 + half * 64) + (lane & 7) * 128;
+      if (lane < 8)
+        for (int a = 1; a < ahead && a < n; ++a) asm volatile("prefetch.global.L2 [%0];" ::"l"(line + (long long)a * 2048));
+      uint4 w[4][2];
+#pragma unroll
+      for (int T = 0; T < 4; ++T) { w[T][0] = __ldg(blk + T * 16); w[T][1] = __ldg(blk + T * 16 + 8); }
+      for (int i = 0; i < n; ++i) {
+        if (lane < 8 && ahead > 0 && i + ahead < n) asm volatile("prefetch.global.L2 [%0];" ::"l"(line + (long long)(i + ahead) * 2048));
+        uint4 wn[4][2];
+        const uint4* nb = blk + (i + 1 < n ? 128 : 0);
+#pragma unroll
+        for (int T = 0; T < 4; ++T) { wn[T][0] = __ldg(nb + T * 16); wn[T][1] = __ldg(nb + T * 16 + 8); }
+        const uint32_t* qc = qtok + (c0 + i) * 32;
+#pragma unroll
+        for (int pr = 0; pr < 2; ++pr) {
+          const uint32_t q1a = qc[(2 * pr) * 8], q1b = qc[(2 * pr + 1) * 8], q16a = qc[(2 * pr) * 8 + 4], q16b = qc[(2 * pr + 1) * 8 + 4];
+#pragma unroll
+          for (int T = 0; T < 4; ++T) {
+            const uint32_t x00 = pr == 0 ? w[T][0].x : w[T][0].z, x01 = pr == 0 ? w[T][0].y : w[T][0].w;
+            const uint32_t x10 = pr == 0 ? w[T][1].x : w[T][1].z, x11 = pr == 0 ? w[T][1].y : w[T][1].w;
+            const uint32_t t00 = x00 >> c, t01 = x01 >> c, t10 = x10 >> c, t11 = x11 >> c;
+            const uint32_t m1[4] = {t00 & 0x01010101u, t10 & 0x01010101u, t01 & 0x01010101u, t11 & 0x01010101u};
+            const uint32_t m16[4] = {t00 & 0x10101010u, t10 & 0x10101010u, t01 & 0x10101010u, t11 & 0x10101010u};
+            mma_u8s8(a1[T], m1, q1a, q1b);
+            mma_u8s8(a16[T], m16, q16a, q16b);
+          }
+        }
+#pragma unroll
+        for (int T = 0; T < 4; ++T) { w[T][0] = wn[T][0]; w[T][1] = wn[T][1]; }
+        blk = nb;
       }
-      stream_half_sync(bid);
-      if (mg == 1) stream_bits<1>(L, tg, mg, p_lo, p_hi, qs, qwords, toks, bp.prefetch);
-      else if (mg == 2) stream_bits<2>(L, tg, mg, p_lo, p_hi, qs, qwords, toks, bp.prefetch);
-      else if (mg <= 4) stream_bits<4>(L, tg, mg, p_lo, p_hi, qs, qwords, toks, bp.prefetch);
-      else stream_bits<8>(L, tg, mg, p_lo, p_hi, qs, qwords, toks, bp.prefetch);
+      // accumulator u of tile T: feature 16 T + g (u < 2) or + 8, token 2 c + (u & 1)
+#pragma unroll
+      for (int T = 0; T < 4; ++T)
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int t = 2 * c + (u & 1);
+          if (t < mg) {
+            const int row = rg * 128 + half * 64 + T * 16 + g + (u >> 1) * 8;
+            atomicAdd(L.acc + (long long)(tg * kStreamTokenGroup + t) * Np + row, a1[T][u] + (a16[T][u] >> 4));
+          }
+        }
+      if (stream_report(L, tg, rg, (unsigned)n, lane)) stream_finish(L, tg, rg, toks, lane);
     }
-  }
-}
-
-__device__ void stream_half_expert(const StreamBatch& bp, int lo, int hi, int bid, float* hs, DecodeTokInfo* toks) {
-  const int tid = threadIdx.x & (kStreamHalfThreads - 1), gw = tid >> 5;
-  for (int l = 0; l < bp.n; ++l) {
-    if (bp.z0[l + 1] <= lo || bp.z0[l] >= hi || bp.z0[l + 1] == bp.z0[l]) continue;
-    const StreamLinear& L = bp.lin[l];
-    const int seg_lo = max(lo, L.z0) - L.z0, seg_hi = min(hi, bp.z0[l + 1]) - L.z0;
-    stream_half_sync(bid);
-    for (int i = tid; i < L.M * L.r; i += kStreamHalfThreads) hs[i] = __ldcg(L.h + i);
-    if (tid < L.M) reinterpret_cast<int4*>(toks)[tid] = __ldcg(reinterpret_cast<const int4*>(L.info) + tid);
-    stream_half_sync(bid);
-    const int len = seg_hi - seg_lo;
-    stream_expert(L, seg_lo + (int)((long long)len * gw / kStreamHalfWarps), seg_lo + (int)((long long)len * (gw + 1) / kStreamHalfWarps), hs, toks);
+    p += n;
   }
 }
 
@@ -670,10 +693,12 @@ __global__ void __launch_bounds__(kStreamThreads, 1) k_decode_stream(const __gri
   const int zspan_lo = (int)(Z * cta / nC), zspan_hi = (int)(Z * (cta + 1) / nC);
 
   // the linears whose chunks / expert-product items this CTA's spans touch
-  int l_lo = 0, l_hi = 0;
+  int l_lo = 0, l_hi = 0, zl_lo = 0, zl_hi = 0;
   for (int l = 0; l < bp.n; ++l) {
     if (bp.chunk0[l + 1] <= span_lo) l_lo = l + 1;
     if (bp.chunk0[l] < span_hi) l_hi = l + 1;
+    if (bp.z0[l + 1] <= zspan_lo) zl_lo = l + 1;
+    if (bp.z0[l] < zspan_hi) zl_hi = l + 1;
   }
 
   // phase 0: accumulators and counters start at zero.  A linear's words are shared out in proportion to its chunks:
@@ -705,19 +730,51 @@ __global__ void __launch_bounds__(kStreamThreads, 1) k_decode_stream(const __gri
   const bool ok = stream_bar_wait(bar, &sh.ok);
 
   if (ok) {
-    // phase 2: the bit product is bound by instruction issue, the expert product by the latency of its loads, so
-    // the two halves of the CTA (eight warps each, a named barrier each) do one of each at a time: half 0 takes the
-    // first half of the CTA's chunks, then the second half of its expert-product items; half 1 the other way round.
     uint32_t* qs = reinterpret_cast<uint32_t*>(stream_smem);
     float* hs = reinterpret_cast<float*>(stream_smem + bp.off_h);
-    const int half = warp / kStreamHalfWarps;
-    DecodeTokInfo* toks = reinterpret_cast<DecodeTokInfo*>(stream_smem + bp.off_info) + half * kDecodeMaxTokens;
-    const int span_mid = span_lo + (span_hi - span_lo) / 2, zspan_mid = zspan_lo + (zspan_hi - zspan_lo) / 2;
-    if (half == 0) stream_half_bits(bp, span_lo, span_mid, 1, qs, toks);
-    else stream_half_expert(bp, zspan_lo, zspan_mid, 2, hs, toks);
-    __syncthreads();   // the halves swap the code and h buffers
-    if (half == 0) stream_half_expert(bp, zspan_mid, zspan_hi, 1, hs, toks);
-    else stream_half_bits(bp, span_mid, span_hi, 2, qs, toks);
+    DecodeTokInfo* toks = reinterpret_cast<DecodeTokInfo*>(stream_smem + bp.off_info);
+    // phase 2 (a): sign bits
+    for (int l = l_lo; l < l_hi; ++l) {
+      const StreamLinear& L = bp.lin[l];
+      const int seg_lo = max(span_lo, L.chunk0) - L.chunk0, seg_hi = min(span_hi, L.chunk0 + L.G * L.C) - L.chunk0;
+      if (seg_lo >= seg_hi) continue;
+      const int qwords = L.C * 32, qstride = qwords + 4;   // the pad spreads the tokens' rows over the banks (mma variant)
+      const int len = seg_hi - seg_lo;
+      const int p_lo = seg_lo + (int)((long long)len * warp / kStreamWarps), p_hi = seg_lo + (int)((long long)len * (warp + 1) / kStreamWarps);
+      for (int tg = 0; tg * kStreamTokenGroup < L.M; ++tg) {
+        const int mg = min(kStreamTokenGroup, L.M - tg * kStreamTokenGroup);
+        __syncthreads();   // the previous codes and token records are no longer read
+        {
+          const int row4 = qwords >> 2;
+          const uint4* from = reinterpret_cast<const uint4*>(L.qg + (long long)tg * kStreamTokenGroup * qwords);
+          for (int i = threadIdx.x; i < mg * row4; i += kStreamThreads) {
+            const int t = i / row4, j = i - t * row4;
+            reinterpret_cast<uint4*>(qs + t * qstride)[j] = __ldcg(from + i);
+          }
+          if (threadIdx.x < L.M) reinterpret_cast<int4*>(toks)[threadIdx.x] = __ldcg(reinterpret_cast<const int4*>(L.info) + threadIdx.x);
+        }
+        __syncthreads();
+        if (mg >= bp.mma_from) stream_bits_mma(L, tg, mg, p_lo, p_hi, qs, qstride, toks, bp.prefetch);
+        else if (mg == 1) stream_bits<1>(L, tg, mg, p_lo, p_hi, qs, qstride, toks, bp.prefetch);
+        else if (mg == 2) stream_bits<2>(L, tg, mg, p_lo, p_hi, qs, qstride, toks, bp.prefetch);
+        else if (mg <= 4) stream_bits<4>(L, tg, mg, p_lo, p_hi, qs, qstride, toks, bp.prefetch);
+        else stream_bits<8>(L, tg, mg, p_lo, p_hi, qs, qstride, toks, bp.prefetch);
+      }
+    }
+    // phase 2 (b): expert products.  What phase 1 wrote comes from other CTAs: read it through L2.
+    for (int l = zl_lo; l < zl_hi; ++l) {
+      const StreamLinear& L = bp.lin[l];
+      if (L.r == 0) continue;
+      const int zi = L.M * L.G * 4;
+      const int seg_lo = max(zspan_lo, L.z0) - L.z0, seg_hi = min(zspan_hi, L.z0 + zi) - L.z0;
+      if (seg_lo >= seg_hi) continue;
+      __syncthreads();
+      for (int i = threadIdx.x; i < L.M * L.r; i += kStreamThreads) hs[i] = __ldcg(L.h + i);
+      if (threadIdx.x < L.M) reinterpret_cast<int4*>(toks)[threadIdx.x] = __ldcg(reinterpret_cast<const int4*>(L.info) + threadIdx.x);
+      __syncthreads();
+      const int len = seg_hi - seg_lo;
+      stream_expert(L, seg_lo + (int)((long long)len * warp / kStreamWarps), seg_lo + (int)((long long)len * (warp + 1) / kStreamWarps), hs, toks);
+    }
   }
 }
 
@@ -737,6 +794,8 @@ size_t decode_stream_extra_bytes(int M, int K, int N, int r) {
 
 static int g_decode_stream_on = 1;
 static int g_decode_stream_prefetch = 1;
+static int g_decode_stream_mma_from = 5;   // measured on the 3B shapes: dp4a is ahead up to four tokens, level at four
+void decode_stream_mma_from(int m) { g_decode_stream_mma_from = m < 1 ? 1 : m; }
 void decode_stream_enable(int mode) { g_decode_stream_on = mode < 0 ? 0 : mode > 2 ? 2 : mode; }
 void decode_stream_prefetch(int on) { g_decode_stream_prefetch = on ? 1 : 0; }
 int decode_stream_mode() { return g_decode_stream_on; }
@@ -803,7 +862,7 @@ int decode_stream_launch(const DecodeItemArgs* items, int n, cudaStream_t st) {
     // the bit product is instantiated for 1, 2, 4 or 8 tokens and reads that many rows of codes (the surplus rows are
     // never used, but they must lie inside the allocation)
     const int mt = M >= 5 ? 8 : M >= 3 ? 4 : M;
-    codes = std::max(codes, (size_t)mt * L.C * 128);
+    codes = std::max(codes, (size_t)mt * (L.C * 128 + 16));
     hbytes = std::max(hbytes, (size_t)M * std::max(r, 1) * 4);
     xbytes = std::max(xbytes, (size_t)K * 2);
     part = std::max(part, (size_t)std::max(r, 1) * kStreamWarps * 4);
@@ -850,12 +909,13 @@ int decode_stream_launch(const DecodeItemArgs* items, int n, cudaStream_t st) {
   const size_t smem1 = bp.off_part + s_up256(part);
   bp.off_h = (int)s_up256(codes);
   bp.off_info = (int)(bp.off_h + s_up256(hbytes));
-  const size_t smem2 = bp.off_info + 2 * kDecodeMaxTokens * sizeof(DecodeTokInfo);
+  const size_t smem2 = bp.off_info + 256;
   const size_t smem = std::max(smem1, smem2);
   if (smem > kStreamSmemLimit) return PQ_ERR_UNSUPPORTED;
   bp.bar_slot = stream_bar_slot(st);
   if (bp.bar_slot < 0) return PQ_ERR_UNSUPPORTED;
   bp.prefetch = g_decode_stream_prefetch ? 4 : 0;
+  bp.mma_from = g_decode_stream_mma_from;
   static const bool limit_set = cudaFuncSetAttribute(k_decode_stream, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStreamSmemLimit) == cudaSuccess;
   if (!limit_set) return PQ_ERR_CUDA;
   cudaLaunchAttribute attr[1];

@@ -139,6 +139,7 @@ size_t decode_stream_extra_bytes(int M, int K, int N, int r);
 int decode_stream_launch(const DecodeItemArgs* items, int n, cudaStream_t st);   // PQ_ERR_UNSUPPORTED: use the other kernels
 void decode_stream_enable(int mode);   // 0 never, 1 where it pays (default), 2 wherever the items allow
 void decode_stream_prefetch(int on);
+void decode_stream_mma_from(int m);
 int decode_stream_mode();
 void decode_stream_reset();
 int decode_batch(const DecodeItemArgs* items, int n, cudaStream_t st);   // independent linears, launched together

@@ -13,14 +13,18 @@ from test_gpu_forward import TOL_BF16, check_status, f32, rel_err
 pytestmark = pytest.mark.gpu
 
 
-@pytest.fixture(autouse=True, params=["stream", "pair"])
+@pytest.fixture(autouse=True, params=["stream", "stream_dp4a", "stream_mma", "pair"])
 def decode_kernels(request):
-    """Every test runs twice: on the streaming kernel (weights in its own layout) and on the two-kernel path."""
-    PQLinear.stream_decode = request.param == "stream"
-    pqb.pq_set_option(pqb.PQ_OPT_DECODE_STREAM, 2 if request.param == "stream" else 0)   # 2: also for one small linear
+    """Every test runs on the streaming kernel (weights in its own layout; bit product as the library picks it, on dp4a
+    only, on the tensor cores only) and on the two-kernel path."""
+    stream = request.param != "pair"
+    PQLinear.stream_decode = stream
+    pqb.pq_set_option(pqb.PQ_OPT_DECODE_STREAM, 2 if stream else 0)   # 2: also for one small linear
+    pqb.pq_set_option(pqb.PQ_OPT_DECODE_MMA_FROM, {"stream_dp4a": 17, "stream_mma": 1}.get(request.param, 5))
     yield request.param
     PQLinear.stream_decode = True
     pqb.pq_set_option(pqb.PQ_OPT_DECODE_STREAM, 1)
+    pqb.pq_set_option(pqb.PQ_OPT_DECODE_MMA_FROM, 5)
 
 
 def run_decode(c, scale_vector=False):
