@@ -67,6 +67,7 @@ enum {
 enum {
   PQ_SCALE_VECTOR = 1u,    /* pq_desc.flags: alpha, beta have N entries instead of 1                      */
   PQ_DECODE_DUMP_ACC = 2u, /* decode only, test hook: also write the exact int32 sums of the 1-bit product */
+  PQ_UNIT_GATES = 4u,      /* with top_k = E: every expert active with gate 1 (test mode, see pq_desc.top_k)     */
   PQ_FUSED_RMSNORM = 8u    /* training path: the layer is called through pq_linear_forward_rms (sizes `saved`) */
 };
 
@@ -75,8 +76,13 @@ enum { PQ_PHASE_PACK = 0, PQ_PHASE_FWD = 1, PQ_PHASE_BWD = 2, PQ_PHASE_DECODE = 
 /* Shape of one layer.  Constraints: T >= 1; K, N multiples of 32 (bit words,
  * 16-byte rows); r == 0 (pure 1-bit layer, the paper's attention projections,
  * E ignored) or r a multiple of 8 with 8 <= r <= 256 and 1 <= E <= 16;
- * top_k must be 1 (the paper's gating).  The training path additionally needs
- * r <= 128. */
+ * top_k = 1 (the paper's gating).  The training path additionally needs r <= 128.
+ * One more value of top_k is taken, as a test mode of the training-size forward (pq_linear_forward with w_s8,
+ * pq_saved_bytes, pq_workspace_bytes(PQ_PHASE_FWD)): top_k = E > 1 with PQ_UNIT_GATES in flags and E r <= 128 --
+ * every expert is active with weight one and the router is not read (Wr may be NULL), so the layer must equal the
+ * dense layer of width E r whose A is the experts' rows stacked and whose B is their columns side by side (the
+ * special case in which routing reduces to a dense branch, Sec. 3.3).  `saved` then has the dense layer's layout;
+ * pq_linear_backward, the decode path and the other forward variants return PQ_ERR_UNSUPPORTED for such a desc. */
 typedef struct pq_desc {
   uint32_t size;  /* sizeof(pq_desc), checked */
   uint32_t flags;

@@ -20,6 +20,7 @@ PQ_ERR_UNSUPPORTED, PQ_ERR_CUDA, PQ_ERR_TIMEOUT, PQ_ERR_TOO_LARGE = -5, -6, -7, 
 PQ_SCALE_VECTOR = 1
 PQ_DECODE_DUMP_ACC = 2
 PQ_FUSED_RMSNORM = 8
+PQ_UNIT_GATES = 4
 PQ_PHASE_PACK, PQ_PHASE_FWD, PQ_PHASE_BWD, PQ_PHASE_DECODE = 0, 1, 2, 3
 
 EXPORTS = ("pq_status_string", "pq_workspace_bytes", "pq_saved_bytes", "pq_saved_view_init",
@@ -158,8 +159,9 @@ def _check(fn, status):
         raise PqError(fn, status)
 
 
-def make_desc(T, K, N, r=0, E=0, top_k=1, scale_vector=False, dump_acc=False, fused_rmsnorm=False) -> pq_desc:
-    flags = (PQ_SCALE_VECTOR if scale_vector else 0) | (PQ_DECODE_DUMP_ACC if dump_acc else 0) | (PQ_FUSED_RMSNORM if fused_rmsnorm else 0)
+def make_desc(T, K, N, r=0, E=0, top_k=1, scale_vector=False, dump_acc=False, fused_rmsnorm=False, unit_gates=False) -> pq_desc:
+    flags = ((PQ_SCALE_VECTOR if scale_vector else 0) | (PQ_DECODE_DUMP_ACC if dump_acc else 0) | (PQ_FUSED_RMSNORM if fused_rmsnorm else 0)
+             | (PQ_UNIT_GATES if unit_gates else 0))
     return pq_desc(ctypes.sizeof(pq_desc), flags, T, K, N, r, E, top_k)
 
 

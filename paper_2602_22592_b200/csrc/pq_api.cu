@@ -32,13 +32,25 @@ static inline int max_items_of(const pq_desc* d) { return mtiles_of(d) + experts
 static inline bool routed(const pq_desc* d) { return d->r > 0 && d->E > 1; }
 static inline bool normed(const pq_desc* d) { return (d->flags & PQ_FUSED_RMSNORM) != 0; }
 
+// top_k = E with unit gates (a test mode of the training-size forward): every expert is active with weight one, which is
+// a dense branch of width E r whose A is the experts' rows stacked and whose B is their columns side by side
+static inline bool all_experts(const pq_desc* d) { return d->r > 0 && d->E > 1 && d->top_k == d->E; }
+static inline pq_desc dense_equivalent(const pq_desc* d) {
+  pq_desc e = *d;
+  e.r = d->r * d->E; e.E = 1; e.top_k = 1; e.flags = d->flags & ~(uint32_t)PQ_UNIT_GATES;
+  return e;
+}
+
 static int check_desc(const pq_desc* d, bool training) {
   if (!d) return PQ_ERR_NULL;
   if (d->size != sizeof(pq_desc)) return PQ_ERR_SHAPE;
   if (d->T < 1 || d->K < 32 || d->N < 32 || d->K % 32 || d->N % 32) return PQ_ERR_SHAPE;
   if (d->r < 0 || d->r % 8 || d->r > 256) return PQ_ERR_SHAPE;
   if (d->r > 0 && (d->E < 1 || d->E > kMaxExperts)) return PQ_ERR_SHAPE;
-  if (d->r > 0 && d->top_k != 1) return PQ_ERR_UNSUPPORTED;
+  if (d->r > 0 && d->top_k != 1) {
+    // only k = 1 (the paper's setting) and, forward only and on the training-size path, k = E with unit gates
+    if (!all_experts(d) || !(d->flags & PQ_UNIT_GATES) || !training || d->r * d->E > 128) return PQ_ERR_UNSUPPORTED;
+  }
   if (training && d->r > 128) return PQ_ERR_UNSUPPORTED;
   return PQ_OK;
 }
@@ -266,6 +278,11 @@ const char* pq_status_string(int s) {
 }
 
 size_t pq_saved_bytes(const pq_desc* d) {
+  if (d && d->size == sizeof(pq_desc) && all_experts(d)) {
+    if (check_desc(d, true) != PQ_OK) return 0;
+    const pq_desc e = dense_equivalent(d);
+    return carve_saved(&e, nullptr, nullptr);
+  }
   if (check_desc(d, false) != PQ_OK) return 0;
   return carve_saved(d, nullptr, nullptr);
 }
@@ -276,9 +293,13 @@ size_t pq_workspace_bytes(const pq_desc* d, int phase) {
     case PQ_PHASE_PACK: return align_up(sizeof(double) * 2 * kPackPartials);
     case PQ_PHASE_FWD:
       if (check_desc(d, true) != PQ_OK) return 0;
+      if (all_experts(d)) {   // the dense equivalent's needs, then the experts' B side by side
+        const pq_desc e = dense_equivalent(d);
+        return carve_fwd_scratch(&e, nullptr, nullptr) + carve_saved(&e, nullptr, nullptr) + align_up((size_t)d->N * e.r * 2);
+      }
       return carve_fwd_scratch(d, nullptr, nullptr) + carve_saved(d, nullptr, nullptr);
     case PQ_PHASE_BWD:
-      if (check_desc(d, true) != PQ_OK) return 0;
+      if (check_desc(d, true) != PQ_OK || all_experts(d)) return 0;
       return carve_bwd_scratch(d, nullptr, nullptr);
     case PQ_PHASE_DECODE:
       if (check_desc(d, false) != PQ_OK || d->T > 16) return 0;
@@ -385,6 +406,18 @@ static int forward_impl(const pq_desc* d, const uint16_t* X, const uint32_t* w_b
   int rc = check_desc(d, true);
   if (rc) return rc;
   (void)w_bits;
+  if (all_experts(d)) {
+    if (hp_scales || norm_weight || normed(d)) return PQ_ERR_UNSUPPORTED;
+    if (!A || !B || !alpha || !ws) return PQ_ERR_NULL;
+    if (misaligned(B) || misaligned(ws)) return PQ_ERR_ALIGN;
+    const pq_desc e = dense_equivalent(d);
+    const size_t side = align_up((size_t)d->N * e.r * 2);
+    if (ws_bytes < side) return PQ_ERR_WORKSPACE;
+    uint16_t* b_wide = reinterpret_cast<uint16_t*>(static_cast<uint8_t*>(ws) + (ws_bytes - side) / 256 * 256);
+    if (launch_concat_experts(B, d->E, d->N, d->r, b_wide, static_cast<cudaStream_t>(stream)) != cudaSuccess) return PQ_ERR_CUDA;
+    return forward_impl(&e, X, w_bits, w_s8, w_scales, A, b_wide, nullptr, nullptr, alpha, beta, Y, saved, saved_bytes, ws,
+                        (ws_bytes - side) / 256 * 256, stream);
+  }
   if (normed(d) != (norm_weight != nullptr)) return PQ_ERR_NULL;           // the flag sizes the saved buffer
   if (norm_weight && (!(norm_eps > 0.f) || misaligned(norm_weight))) return norm_eps > 0.f ? PQ_ERR_ALIGN : PQ_ERR_SHAPE;
   if (d->r > 0 && (!A || !B || !alpha)) return PQ_ERR_NULL;
@@ -624,6 +657,7 @@ int pq_linear_backward(const pq_desc* d, const uint16_t* dY, const uint16_t* X, 
                        const void* saved, size_t saved_bytes, uint16_t* dX, float* dW, float* dA, float* dB, float* dWr, float* dalpha,
                        float* dbeta, void* ws, size_t ws_bytes, void* stream) {
   if (!d || !dY || !X || !w_s8 || !w_scales || !beta || !saved || !dX || !dW || !dbeta || !ws) return PQ_ERR_NULL;
+  if (d->size == sizeof(pq_desc) && all_experts(d)) return PQ_ERR_UNSUPPORTED;   // the all-experts mode is forward only
   int rc = check_desc(d, true);
   if (rc) return rc;
   const bool hp = d->r > 0;

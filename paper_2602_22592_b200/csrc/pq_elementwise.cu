@@ -860,4 +860,23 @@ cudaError_t launch_fill_zero(void* p, size_t bytes, cudaStream_t st) {
   return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------------------
+// experts' down-projections side by side: out[n, e r + j] = B[e, n, j] (the all-experts test mode of the forward)
+// ---------------------------------------------------------------------------
+__global__ void k_concat_experts(const uint4* __restrict__ B, uint4* __restrict__ out, int E, int N, int r8) {
+  const long long o = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (o >= (long long)N * E * r8) return;
+  const int jc = (int)(o % r8);
+  const long long t = o / r8;
+  const int e = (int)(t % E);
+  const long long n = t / E;
+  out[o] = B[((long long)e * N + n) * r8 + jc];
+}
+cudaError_t launch_concat_experts(const uint16_t* B, int E, int N, int r, uint16_t* out, cudaStream_t st) {
+  const long long total = (long long)N * E * (r / 8);
+  LaunchScope ls(KID_SCATTER_ROWS, st);
+  k_concat_experts<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(reinterpret_cast<const uint4*>(B), reinterpret_cast<uint4*>(out), E, N, r / 8);
+  return cudaGetLastError();
+}
+
 }  // namespace pq

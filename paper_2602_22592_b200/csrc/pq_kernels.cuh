@@ -98,6 +98,7 @@ cudaError_t launch_fill_zero(void* p, size_t bytes, cudaStream_t st);
 cudaError_t launch_swiglu(const uint16_t* G, const uint16_t* U, uint16_t* M, long long n, cudaStream_t st);
 cudaError_t launch_ffn8_act(const int* g_int, const int* u_int, const float* gamma, const float* hp_scales, int T, int r, int8_t* qm,
                             float* gamma_m, cudaStream_t st);
+cudaError_t launch_concat_experts(const uint16_t* B, int E, int N, int r, uint16_t* out, cudaStream_t st);
 cudaError_t launch_pack_experts(const uint16_t* A, const uint16_t* B, int E, int r, int K, int N, int8_t* A8, int8_t* B8, float* hp_scales,
                                 uint32_t* amax_bits, cudaStream_t st);
 

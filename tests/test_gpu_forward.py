@@ -346,3 +346,51 @@ def test_forward_int8_hp_rejects_odd_width():
     with pytest.raises(pqb.PqError) as ei:
         L.forward_hp8()
     assert ei.value.status == pqb.PQ_ERR_SHAPE
+
+
+@pytest.mark.parametrize("T,K,N,r,E", [(300, 384, 544, 32, 4), (129, 256, 320, 16, 8), (64, 512, 96, 64, 2)])
+def test_all_experts_with_unit_gates_is_the_dense_layer_of_width_E_r(T, K, N, r, E):
+    # Sec. 3.3, the special case in which routing reduces to a dense branch: top_k = E with unit gates.  The oracle's
+    # sum over all experts (weights one) is the expected value; the same call on a dense layer built from the stacked A
+    # and the side-by-side B must give the same bits (it is the same arithmetic).
+    c = I.make_linear_case(T, K, N, r, E, seed=31)
+    L = PQLinear(T, K, N, r, E, guard=True).load_case(c)      # buffers and packed weights; its own desc is top-1
+    L.pack()
+    d = pqb.make_desc(T, K, N, r, E, top_k=E, unit_gates=True)
+    saved = torch.empty(pqb.pq_saved_bytes(d), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(pqb.pq_workspace_bytes(d, pqb.PQ_PHASE_FWD), dtype=torch.uint8, device="cuda")
+    assert saved.numel() > 0 and ws.numel() > 0
+    Y = torch.empty((T, N), dtype=torch.bfloat16, device="cuda")
+    pqb.pq_linear_forward(d, L.X, L.w_bits, L.w_s8, L.w_scales, L.A, L.B, None, L.alpha, L.beta, Y, saved, ws)
+    torch.cuda.synchronize()
+    check_status()
+    assert L.check_guards() == 0
+    f1 = O.linear_forward(c["X"], c["W"], alpha=c["alpha"], beta=c["beta"])                 # the 1-bit branch alone
+    z = O.hp_branch_all_experts(c["X"], c["A"], c["B"], np.ones((T, E)))
+    al = np.broadcast_to(np.asarray(c["alpha"], dtype=np.float64).reshape(-1), (N,))
+    want = O.round_to_bf16(al[None, :] * z + f1["Y64"])
+    assert rel_err(f32(Y), want) <= TOL_BF16 and rms_err(f32(Y), want) <= TOL_RMS
+    # the dense layer of width E r
+    Ld = PQLinear(T, K, N, r * E, 1).load_case(c)
+    Ld.A = L.A.reshape(1, E * r, K).contiguous()
+    Ld.B = L.B.permute(1, 0, 2).reshape(1, N, E * r).contiguous()
+    Ld.Wr = None
+    Ld.pack()
+    Ld.forward()
+    torch.cuda.synchronize()
+    assert torch.equal(Ld.Y, Y)
+    # not what top-1 routing gives
+    L.forward()
+    torch.cuda.synchronize()
+    assert not torch.equal(L.Y, Y)
+
+
+def test_all_experts_mode_limits():
+    d = pqb.make_desc(64, 256, 256, 32, 4, top_k=4)                       # without the unit-gate flag
+    assert pqb.pq_saved_bytes(d) == 0 and pqb.pq_workspace_bytes(d, pqb.PQ_PHASE_FWD) == 0
+    d = pqb.make_desc(64, 256, 256, 64, 4, top_k=4, unit_gates=True)      # E r > 128
+    assert pqb.pq_saved_bytes(d) == 0
+    d = pqb.make_desc(64, 256, 256, 32, 4, top_k=2, unit_gates=True)      # neither 1 nor E
+    assert pqb.pq_saved_bytes(d) == 0
+    d = pqb.make_desc(64, 256, 256, 32, 4, top_k=4, unit_gates=True)
+    assert pqb.pq_workspace_bytes(d, pqb.PQ_PHASE_BWD) == 0               # forward only
