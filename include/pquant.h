@@ -262,6 +262,9 @@ typedef struct pq_decode_token {
 typedef struct pq_decode_view {
   pq_decode_token* tokens; /* [T] (device)                                                        */
   int32_t* acc;            /* [T,N] sum_k S[n,k] q[t,k] when PQ_DECODE_DUMP_ACC is set, else NULL */
+  /* INT8 branch on the streaming kernel (pq_decode_item.A8): the exact integers it went through */
+  int32_t* hp_h_int;       /* [T,r] h_int = A8_e q                                                 */
+  int32_t* hp_z_int;       /* [T,N] z_int = B8_e qh when PQ_DECODE_DUMP_ACC is set, else NULL       */
 } pq_decode_view;
 int pq_decode_view_init(const pq_desc* d, void* ws, pq_decode_view* out);
 
@@ -303,6 +306,15 @@ typedef struct pq_decode_item {
    * are needed in both cases (the rows of A_e are read in their natural layout). */
   const uint32_t* w_bits_il;
   const uint16_t* B_il;
+  /* The paper's INT8 high-precision branch on the decode path (Sec. 3.2), or NULL for the bf16 branch: A8 [E,r,K] int8 and
+   * hp_scales [E][2] from pq_pack_experts, B8_il from pq_pack_decode_hp8.  The branch multiplies the token's int8 codes:
+   *   h_int = A8_e q (int32, exact);  qh, gamma_h = Eq. 7-9 on h_int;  z_int = B8_e qh (int32, exact);
+   *   z = z_int / (gamma_B gamma_h gamma_A gamma_t)
+   * -- the arithmetic of pq_linear_forward_hp8.  It runs on the streaming kernel only, whatever the group's size:
+   * w_bits_il is required (PQ_ERR_NULL), r a multiple of 16 (PQ_ERR_SHAPE); A, B and B_il are not read. */
+  const int8_t* A8;
+  const int8_t* B8_il;
+  const float* hp_scales;
 } pq_decode_item;
 int pq_decode_batch(const pq_decode_item* items, int n, void* stream);
 
@@ -317,6 +329,11 @@ int pq_decode_batch(const pq_decode_item* items, int n, void* stream);
  * (PQ_ERR_SHAPE).  d->T is not used. */
 int pq_decode_pack_bytes(const pq_desc* d, size_t* bits_il_bytes, size_t* b_il_bytes);
 int pq_pack_decode(const pq_desc* d, const uint32_t* w_bits, const uint16_t* B, uint32_t* w_bits_il, uint16_t* B_il, void* stream);
+/* The int8 codes B8 [E,N,r] of pq_pack_experts in the streaming decode kernel's order:
+ * B8_il [E][4 ceil(N/128)][r/16][32][16] int8 (lane l holds 16 consecutive hidden values of row 32 group + l, zero
+ * beyond N), pq_decode_pack_hp8_bytes(d) bytes (0 for a shape without this layout: r = 0 or not a multiple of 16). */
+size_t pq_decode_pack_hp8_bytes(const pq_desc* d);
+int pq_pack_decode_hp8(const pq_desc* d, const int8_t* B8, int8_t* B8_il, size_t b8_il_bytes, void* stream);
 
 /* Straight-through backward (App. B.1): Sign, Round and Clip pass the gradient
  * unchanged; mu, lam, gamma are constants.  Every gradient is OVERWRITTEN.

@@ -24,7 +24,7 @@ PQ_UNIT_GATES = 4
 PQ_PHASE_PACK, PQ_PHASE_FWD, PQ_PHASE_BWD, PQ_PHASE_DECODE = 0, 1, 2, 3
 
 EXPORTS = ("pq_status_string", "pq_workspace_bytes", "pq_saved_bytes", "pq_saved_view_init",
-           "pq_decode_view_init", "pq_bwd_view_init", "pq_decode_batch", "pq_decode_pack_bytes", "pq_pack_decode", "pq_pack_weights", "pq_pack_weights_static", "pq_pack_experts", "pq_linear_forward", "pq_linear_forward_hp8", "pq_linear_forward_rms", "pq_ffn_workspace_bytes", "pq_ffn_forward", "pq_ffn_view_init", "pq_linear_backward", "pq_debug_gemm", "pq_debug_gemm_tile",
+           "pq_decode_view_init", "pq_bwd_view_init", "pq_decode_batch", "pq_decode_pack_bytes", "pq_pack_decode", "pq_decode_pack_hp8_bytes", "pq_pack_decode_hp8", "pq_pack_weights", "pq_pack_weights_static", "pq_pack_experts", "pq_linear_forward", "pq_linear_forward_hp8", "pq_linear_forward_rms", "pq_ffn_workspace_bytes", "pq_ffn_forward", "pq_ffn_view_init", "pq_linear_backward", "pq_debug_gemm", "pq_debug_gemm_tile",
            "pq_device_status", "pq_kernel_launches", "pq_profile_events", "pq_set_option")
 
 KERNEL_IDS = dict(pack_sums=0, binarize_pack=1, router=2, route_scan=3, act_quant=4, hp_up=5, fwd=6, scatter_rows=7,
@@ -54,11 +54,12 @@ class pq_decode_item(ctypes.Structure):
     _fields_ = [("desc", pq_desc)] + [(n, ctypes.c_void_p) for n in
                                       ("X", "w_bits", "w_scales", "A", "B", "Wr", "alpha", "beta", "Y", "ws")] + [
         ("ws_bytes", ctypes.c_size_t), ("norm_weight", ctypes.c_void_p), ("norm_eps", ctypes.c_float),
-        ("w_bits_il", ctypes.c_void_p), ("B_il", ctypes.c_void_p)]
+        ("w_bits_il", ctypes.c_void_p), ("B_il", ctypes.c_void_p), ("A8", ctypes.c_void_p), ("B8_il", ctypes.c_void_p),
+        ("hp_scales", ctypes.c_void_p)]
 
 
 class pq_decode_view(ctypes.Structure):
-    _fields_ = [("tokens", ctypes.c_void_p), ("acc", ctypes.c_void_p)]
+    _fields_ = [("tokens", ctypes.c_void_p), ("acc", ctypes.c_void_p), ("hp_h_int", ctypes.c_void_p), ("hp_z_int", ctypes.c_void_p)]
 
 
 class pq_ffn_desc(ctypes.Structure):
@@ -110,6 +111,10 @@ def lib() -> ctypes.CDLL:
         L.pq_decode_pack_bytes.argtypes = [dp, ctypes.POINTER(sz), ctypes.POINTER(sz)]
         L.pq_pack_decode.restype = ci
         L.pq_pack_decode.argtypes = [dp, vp, vp, vp, vp, vp]
+        L.pq_decode_pack_hp8_bytes.restype = sz
+        L.pq_decode_pack_hp8_bytes.argtypes = [dp]
+        L.pq_pack_decode_hp8.restype = ci
+        L.pq_pack_decode_hp8.argtypes = [dp, vp, vp, sz, vp]
         L.pq_linear_forward.restype = ci
         L.pq_linear_forward.argtypes = [dp] + [vp] * 10 + [vp, sz, vp, sz, vp]
         L.pq_linear_forward_rms.restype = ci
@@ -216,6 +221,10 @@ def pq_decode_view_init(d: pq_desc, ws: torch.Tensor) -> dict:
                gamma=raw.view(torch.float32).view(d.T, 4)[:, 2], code_sum=raw.view(torch.int32).view(d.T, 4)[:, 3], acc=None)
     if v.acc:
         out["acc"] = ws[v.acc - base: v.acc - base + 4 * d.T * d.N].view(torch.int32).view(d.T, d.N)
+    if v.hp_h_int and d.r > 0:
+        out["hp_h_int"] = ws[v.hp_h_int - base: v.hp_h_int - base + 4 * d.T * d.r].view(torch.int32).view(d.T, d.r)
+    if v.hp_z_int:
+        out["hp_z_int"] = ws[v.hp_z_int - base: v.hp_z_int - base + 4 * d.T * d.N].view(torch.int32).view(d.T, d.N)
     return out
 
 
@@ -305,7 +314,7 @@ def pq_ffn_view_init(d: pq_ffn_desc, ws: torch.Tensor) -> dict:
 
 def make_decode_items(entries):
     """ctypes array of pq_decode_item from (desc, X, w_bits, w_scales, A, B, Wr, alpha, beta, Y, ws[, norm_weight, norm_eps
-    [, w_bits_il, B_il]]) tuples of tensors (norm_weight, norm_eps: bf16 RMSNorm gain [K] and its epsilon, for un-normalised X;
+    [, w_bits_il, B_il[, A8, B8_il, hp_scales]]]) tuples of tensors (norm_weight, norm_eps: bf16 RMSNorm gain [K] and its epsilon, for un-normalised X;
     w_bits_il, B_il: the weights as laid out by pq_pack_decode).
     The array only holds pointers: keep the tensors alive while it is in use."""
     arr = (pq_decode_item * len(entries))()
@@ -317,6 +326,10 @@ def make_decode_items(entries):
         w_bits_il, B_il = (entry[13], entry[14]) if len(entry) > 13 else (None, None)
         arr[i].w_bits_il = None if w_bits_il is None else w_bits_il.data_ptr()
         arr[i].B_il = None if B_il is None else B_il.data_ptr()
+        A8, B8_il, hp_scales = entry[15:18] if len(entry) > 15 else (None, None, None)   # INT8 high-precision branch
+        arr[i].A8 = None if A8 is None else A8.data_ptr()
+        arr[i].B8_il = None if B8_il is None else B8_il.data_ptr()
+        arr[i].hp_scales = None if hp_scales is None else hp_scales.data_ptr()
         arr[i].desc = d
         for name, t in (("X", X), ("w_bits", w_bits), ("w_scales", w_scales), ("A", A), ("B", B), ("Wr", Wr), ("alpha", alpha),
                         ("beta", beta), ("Y", Y), ("ws", ws)):
@@ -334,6 +347,15 @@ def pq_decode_pack_bytes(d) -> tuple[int, int]:
 def pq_pack_decode(d, w_bits, B, w_bits_il, B_il, stream=None):
     """Lay the sign bits and the rows of B_e out for the streaming decode kernel (one-time, per linear)."""
     _check("pq_pack_decode", lib().pq_pack_decode(ctypes.byref(d), _ptr(w_bits), _ptr(B), _ptr(w_bits_il), _ptr(B_il), _stream(stream)))
+
+
+def pq_decode_pack_hp8_bytes(d) -> int:
+    return lib().pq_decode_pack_hp8_bytes(ctypes.byref(d))
+
+
+def pq_pack_decode_hp8(d, B8, B8_il, stream=None):
+    """The int8 codes of B (pq_pack_experts) in the streaming decode kernel's order."""
+    _check("pq_pack_decode_hp8", lib().pq_pack_decode_hp8(ctypes.byref(d), _ptr(B8), _ptr(B8_il), _nbytes(B8_il), _stream(stream)))
 
 
 def pq_decode_batch(items, stream=None):

@@ -304,7 +304,7 @@ size_t pq_workspace_bytes(const pq_desc* d, int phase) {
     case PQ_PHASE_DECODE:
       if (check_desc(d, false) != PQ_OK || d->T > 16) return 0;
       return decode_workspace_bytes(d->T, d->K, d->N, d->r, (d->flags & PQ_DECODE_DUMP_ACC) != 0) +
-             decode_stream_extra_bytes(d->T, d->K, d->N, d->r);
+             decode_stream_extra_bytes(d->T, d->K, d->N, d->r, (d->flags & PQ_DECODE_DUMP_ACC) != 0);
     default: return 0;
   }
 }
@@ -341,6 +341,7 @@ int pq_decode_view_init(const pq_desc* d, void* ws, pq_decode_view* out) {
   const DecodeViewPtrs v = decode_view(d->T, d->K, d->N, d->r, ws, (d->flags & PQ_DECODE_DUMP_ACC) != 0);
   out->tokens = static_cast<pq_decode_token*>(v.tokens);
   out->acc = v.acc;
+  decode_stream_view(d->T, d->K, d->N, d->r, ws, (d->flags & PQ_DECODE_DUMP_ACC) != 0, &out->hp_h_int, &out->hp_z_int);
   return PQ_OK;
 }
 
@@ -623,6 +624,21 @@ int pq_pack_decode(const pq_desc* d, const uint32_t* w_bits, const uint16_t* B, 
   return decode_pack(d->K, d->N, d->r, experts_of(d), w_bits, B, w_bits_il, B_il, static_cast<cudaStream_t>(stream));
 }
 
+int pq_pack_decode_hp8(const pq_desc* d, const int8_t* B8, int8_t* B8_il, size_t b8_il_bytes, void* stream) {
+  if (!d || !B8 || !B8_il) return PQ_ERR_NULL;
+  int rc = check_desc(d, false);
+  if (rc) return rc;
+  if (d->r <= 0 || d->r % 16) return PQ_ERR_SHAPE;
+  if (misaligned(B8) || misaligned(B8_il)) return PQ_ERR_ALIGN;
+  if (b8_il_bytes < decode_pack_b8_bytes(d->N, d->r, experts_of(d))) return PQ_ERR_WORKSPACE;
+  return decode_pack_b8(d->N, d->r, experts_of(d), B8, B8_il, static_cast<cudaStream_t>(stream));
+}
+
+size_t pq_decode_pack_hp8_bytes(const pq_desc* d) {
+  if (check_desc(d, false) != PQ_OK || d->r <= 0 || d->r % 16) return 0;
+  return decode_pack_b8_bytes(d->N, d->r, experts_of(d));
+}
+
 int pq_decode_batch(const pq_decode_item* items, int n, void* stream) {
   if (!items) return PQ_ERR_NULL;
   if (n < 1 || n > 4096) return PQ_ERR_SHAPE;
@@ -631,8 +647,14 @@ int pq_decode_batch(const pq_decode_item* items, int n, void* stream) {
   int rc = PQ_OK;
   for (int i = 0; i < n && rc == PQ_OK; ++i) {
     const pq_decode_item& it = items[i];
-    rc = check_decode_item(&it.desc, it.X, it.w_bits, it.w_scales, it.A, it.B, it.Wr, it.alpha, it.beta, it.Y, it.ws, it.ws_bytes);
+    const bool hp8 = it.A8 != nullptr;
+    // the INT8 branch brings its own expert matrices: the bf16 ones are not read
+    rc = check_decode_item(&it.desc, it.X, it.w_bits, it.w_scales, hp8 ? reinterpret_cast<const uint16_t*>(it.A8) : it.A,
+                           hp8 ? reinterpret_cast<const uint16_t*>(it.B8_il) : it.B, it.Wr, it.alpha, it.beta, it.Y, it.ws, it.ws_bytes);
     if (rc) break;
+    if (hp8 && (!it.w_bits_il || !it.B8_il || !it.hp_scales)) { rc = PQ_ERR_NULL; break; }
+    if (hp8 && (it.desc.r <= 0 || it.desc.r % 16)) { rc = PQ_ERR_SHAPE; break; }
+    if (hp8 && (misaligned(it.A8) || misaligned(it.B8_il))) { rc = PQ_ERR_ALIGN; break; }
     const pq_desc* d = &it.desc;
     args[i].a = LayerArgs{d->T, d->K, d->N, d->r, experts_of(d), (d->flags & PQ_SCALE_VECTOR) ? 1 : 0, it.w_scales, it.alpha, it.beta, it.A, it.B, it.Wr};
     args[i].X = it.X; args[i].bits = it.w_bits; args[i].Y = it.Y; args[i].ws = it.ws;
@@ -642,9 +664,11 @@ int pq_decode_batch(const pq_decode_item* items, int n, void* stream) {
     args[i].norm_weight = it.norm_weight; args[i].norm_eps = it.norm_eps;
     if (it.w_bits_il) {
       if (misaligned(it.w_bits_il) || misaligned(it.B_il)) { rc = PQ_ERR_ALIGN; break; }
-      if (d->r > 0 && !it.B_il) { rc = PQ_ERR_NULL; break; }
+      if (d->r > 0 && !it.B_il && !hp8) { rc = PQ_ERR_NULL; break; }
       if (it.ws_bytes < pq_workspace_bytes(d, PQ_PHASE_DECODE)) { rc = PQ_ERR_WORKSPACE; break; }
-      args[i].bits_il = it.w_bits_il; args[i].B_il = it.B_il;
+      args[i].bits_il = it.w_bits_il;
+      args[i].B_il = hp8 ? reinterpret_cast<const uint16_t*>(it.B8_il) : it.B_il;
+      args[i].A8 = it.A8; args[i].hp_scales = it.hp_scales;
     }
   }
   if (rc == PQ_OK) rc = decode_batch(args, n, static_cast<cudaStream_t>(stream));

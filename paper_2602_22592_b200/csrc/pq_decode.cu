@@ -801,16 +801,20 @@ int decode_batch(const DecodeItemArgs* items, int n, cudaStream_t st) {
     // (measured on the 3B shapes: its grid barrier and its longer chain of dependent steps cost about as much as eight
     // linears' worth of streaming, so small groups, and mid-sized groups of many tokens, stay on the two kernels above)
     int rc = PQ_ERR_UNSUPPORTED;
-    const int mode = decode_stream_mode();
+    bool any_hp8 = false;
+    for (int k = 0; k < m; ++k) any_hp8 = any_hp8 || items[i + k].A8 != nullptr;
+    const int mode = any_hp8 ? 2 : decode_stream_mode();
     if (mode > 0) {
-      bool all = true;
+      bool all = true, hp8 = false;
       int max_m = 1;
       for (int k = 0; k < m; ++k) {
         all = all && items[i + k].bits_il != nullptr;
+        hp8 = hp8 || items[i + k].A8 != nullptr;
         max_m = std::max(max_m, items[i + k].a.T);
       }
-      const bool worth = mode > 1 || m >= 12 || (m >= 6 && max_m <= 2);
+      const bool worth = mode > 1 || hp8 || m >= 12 || (m >= 6 && max_m <= 2);
       if (all && worth) rc = decode_stream_launch(items + i, m, st);
+      if (hp8 && rc == PQ_ERR_UNSUPPORTED) return rc;       // the INT8 branch exists on the streaming kernel only
     }
     if (rc == PQ_ERR_UNSUPPORTED) rc = decode_launch(items + i, m, st);
     if (rc) return rc;

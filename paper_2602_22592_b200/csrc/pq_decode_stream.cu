@@ -44,7 +44,9 @@ struct StreamLinear {
   const uint16_t* X;        // [M, K] bf16
   const uint16_t* Wr;       // [E, K] bf16 or null
   const uint16_t* A;        // [E, r, K] bf16
-  const uint4* B_il;        // interleaved rows of B_e
+  const uint4* B_il;        // interleaved rows of B_e (bf16), or of the int8 codes B8_e when A8 is set
+  const int8_t* A8;         // [E, r, K] int8 codes of A_e: the INT8 high-precision branch (Sec. 3.2), or null
+  const float* hp_scales;   // [E][2] {gamma_A, gamma_B} of the INT8 branch
   const uint4* bits_il;     // interleaved sign bits
   const float* w_scales;
   const float* alpha;
@@ -53,11 +55,12 @@ struct StreamLinear {
   const uint16_t* norm_w;   // [K] bf16 or null
   DecodeTokInfo* info;      // [16] expert, gate, gamma, code sum per token
   uint32_t* qg;             // [M][C * 32] words of int8 codes in bit-product order
-  float* h;                 // [M][r]
+  float* h;                 // [M][r] (INT8 branch: the exact integers h_int = A8_e q, as int32)
   float* z;                 // [M][G * 128] expert product
   int* acc;                 // [M][G * 128] partial sums over the set bits
   unsigned* cnt;            // [token groups][G] items reported
   int* acc_dump;            // [M, N] or null
+  int* zint_dump;           // [M, N] exact sums of the INT8 branch's second product (test hook) or null
   float norm_eps;
   int M, K, N, r, E, sstride;
   int G, C;                 // row groups; chunks per row group
@@ -76,8 +79,10 @@ struct StreamBatch {
   int prefetch;             // chunks ahead of the bit product for which L2 prefetches are issued (0 = none)
   int mma_from;             // token groups of at least this many tokens take the tensor-core bit product
   int router_rows;          // router rows that fit in shared memory beside the token
-  int off_rows, off_part;   // phase 1 carve-up: [token][router rows][partial sums of h]
-  int off_h, off_info;      // phase 2 carve-up: [codes][h][token info]
+  int off_rows, off_part;   // phase 1 carve-up: [token][router rows][partial sums of h][the token's codes in natural order]
+  int off_qn;
+  int off_h, off_info;      // phase 2 carve-up: [codes][h][token info][INT8 branch: codes of h, their scales]
+  int off_qh;
   int chunk0[kStreamMaxBatch + 1];   // first chunk of every linear in the launch-wide list (and the total)
   int z0[kStreamMaxBatch + 1];       // first expert-product item of every linear
   unsigned char duty[160];           // linear whose token work CTA b shares (255: none)
@@ -113,6 +118,29 @@ __global__ void k_pack_decode_b(const uint4* __restrict__ B, uint4* __restrict__
   const int e = (int)(t / G32);
   const int n = g32 * 32 + lane;
   out[o] = n < N ? B[((long long)e * N + n) * r8 + jc] : make_uint4(0u, 0u, 0u, 0u);
+}
+
+// the same for the int8 codes B8 of the INT8 branch: lane l holds 16 consecutive hidden values of row 32 group + l
+__global__ void k_pack_decode_b8(const uint4* __restrict__ B8, uint4* __restrict__ out, int E, int N, int r16, int G32) {
+  const long long o = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (o >= (long long)E * G32 * r16 * 32) return;
+  const int lane = (int)(o & 31);
+  long long t = o >> 5;
+  const int jc = (int)(t % r16); t /= r16;
+  const int g32 = (int)(t % G32);
+  const int e = (int)(t / G32);
+  const int n = g32 * 32 + lane;
+  out[o] = n < N ? B8[((long long)e * N + n) * r16 + jc] : make_uint4(0u, 0u, 0u, 0u);
+}
+
+size_t decode_pack_b8_bytes(int N, int r, int E) { return (size_t)std::max(E, 1) * ((N + 127) / 128) * 4 * (size_t)(r / 16) * 512; }
+
+int decode_pack_b8(int N, int r, int E, const int8_t* B8, int8_t* B8_il, cudaStream_t st) {
+  const int G = (N + 127) / 128, Ee = std::max(E, 1);
+  const long long total = (long long)Ee * G * 4 * (r / 16) * 32;
+  LaunchScope ls(KID_DECODE_PACK, st);
+  k_pack_decode_b8<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(reinterpret_cast<const uint4*>(B8), reinterpret_cast<uint4*>(B8_il), Ee, N, r / 16, G * 4);
+  return cudaGetLastError() == cudaSuccess ? PQ_OK : PQ_ERR_CUDA;
 }
 
 void decode_pack_sizes(int K, int N, int r, int E, size_t* bits_bytes, size_t* b_bytes) {
@@ -250,6 +278,46 @@ __device__ __forceinline__ void stream_h_rows(const uint4* a4, const uint4* xs4,
   }
 }
 
+// The INT8 branch's first product (Sec. 3.2): rows of int8 codes A8_e against the token's int8 codes, exact in int32.
+// Same cutting as above with 16 codes per piece; the partial sums are integers, so their order does not matter.
+template <int UPL>
+__device__ __forceinline__ void stream_h_rows8(const uint4* a16, const uint4* q16, int* part, int nrows, int pieces, int s_lo, int s_hi,
+                                               int warp, int lane) {
+  constexpr int RB = 16 / UPL;
+  for (int jb = 0; jb < nrows; jb += RB) {
+    int acc[RB];
+#pragma unroll
+    for (int rb = 0; rb < RB; ++rb) acc[rb] = 0;
+    for (int c0 = s_lo + lane; c0 < s_hi; c0 += 32 * UPL) {
+      uint4 wv[RB][UPL];
+#pragma unroll
+      for (int rb = 0; rb < RB; ++rb)
+#pragma unroll
+        for (int u = 0; u < UPL; ++u)
+          wv[rb][u] = (jb + rb < nrows && c0 + 32 * u < s_hi) ? __ldg(a16 + (long long)(jb + rb) * pieces + c0 + 32 * u) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+      for (int u = 0; u < UPL; ++u) {
+        if (c0 + 32 * u < s_hi) {
+          const uint4 qv = q16[c0 + 32 * u];
+#pragma unroll
+          for (int rb = 0; rb < RB; ++rb) {
+            int a = acc[rb];
+            a = __dp4a((int)wv[rb][u].x, (int)qv.x, a); a = __dp4a((int)wv[rb][u].y, (int)qv.y, a);
+            a = __dp4a((int)wv[rb][u].z, (int)qv.z, a); a = __dp4a((int)wv[rb][u].w, (int)qv.w, a);
+            acc[rb] = a;
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int rb = 0; rb < RB; ++rb) {
+      int a = acc[rb];
+      for (int d = 16; d > 0; d >>= 1) a += __shfl_xor_sync(0xffffffffu, a, d);
+      if (lane == 0 && jb + rb < nrows) part[(jb + rb) * kStreamWarps + warp] = a;
+    }
+  }
+}
+
 __device__ void stream_token(const StreamBatch& bp, const StreamLinear& L, int t, int j_lo, int j_hi, bool owner, bool first, uint8_t* smem, StreamShared& sh) {
   const int K = L.K, E = L.E, r = L.r;
   const int chunks = K >> 3;
@@ -351,7 +419,32 @@ __device__ void stream_token(const StreamBatch& bp, const StreamLinear& L, int t
   // rows [j_lo, j_hi) of h = A_e x: warp w takes the w-th sixteenth of every row (whole 16-byte pieces), sixteen
   // loads per lane issued before the first use; the sixteen partial sums of a row are added in warp order afterwards
   const int nrows = r > 0 ? j_hi - j_lo : 0;
-  if (nrows > 0) {
+  if (nrows > 0 && L.A8) {
+    // INT8 branch: the token's codes in natural order (Eq. 7-9, the values the owner also writes out below)
+    uint2* qn = reinterpret_cast<uint2*>(smem + bp.off_qn);
+    for (int c = threadIdx.x; c < chunks; c += kStreamThreads) {
+      const uint4 v = xs4[c];
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+      uint32_t o[2] = {0u, 0u};
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int q0 = max(-128, min(127, __float2int_rn(__fmul_rn(bf16lo(w[u]), gamma))));
+        const int q1 = max(-128, min(127, __float2int_rn(__fmul_rn(bf16hi(w[u]), gamma))));
+        o[u >> 1] |= ((uint32_t)(q0 & 0xFF) | ((uint32_t)(q1 & 0xFF) << 8)) << (16 * (u & 1));
+      }
+      qn[c] = make_uint2(o[0], o[1]);
+    }
+    __syncthreads();
+    const int pieces = K >> 4;
+    const int s_lo = (int)((long long)pieces * warp / kStreamWarps), s_hi = (int)((long long)pieces * (warp + 1) / kStreamWarps);
+    const uint4* a16 = reinterpret_cast<const uint4*>(L.A8) + ((long long)best * r + j_lo) * pieces;
+    const int upl = ((pieces + kStreamWarps - 1) / kStreamWarps + 31) / 32;
+    int* parti = reinterpret_cast<int*>(part);
+    const uint4* q16 = reinterpret_cast<const uint4*>(qn);
+    if (upl == 1) stream_h_rows8<1>(a16, q16, parti, nrows, pieces, s_lo, s_hi, warp, lane);
+    else if (upl == 2) stream_h_rows8<2>(a16, q16, parti, nrows, pieces, s_lo, s_hi, warp, lane);
+    else stream_h_rows8<4>(a16, q16, parti, nrows, pieces, s_lo, s_hi, warp, lane);
+  } else if (nrows > 0) {
     const int s_lo = (int)((long long)chunks * warp / kStreamWarps), s_hi = (int)((long long)chunks * (warp + 1) / kStreamWarps);
     const uint4* a4 = reinterpret_cast<const uint4*>(L.A) + ((long long)best * r + j_lo) * chunks;
     const int upl = ((chunks + kStreamWarps - 1) / kStreamWarps + 31) / 32;   // loads per lane and row
@@ -401,10 +494,17 @@ __device__ void stream_token(const StreamBatch& bp, const StreamLinear& L, int t
     L.info[t] = DecodeTokInfo{best, gate, gamma, tot};
   }
   for (int i = threadIdx.x; i < nrows; i += kStreamThreads) {
-    float a = 0.f;
+    if (L.A8) {
+      int a = 0;
 #pragma unroll
-    for (int w = 0; w < kStreamWarps; ++w) a += part[i * kStreamWarps + w];
-    L.h[(long long)t * r + j_lo + i] = a;
+      for (int w = 0; w < kStreamWarps; ++w) a += reinterpret_cast<const int*>(part)[i * kStreamWarps + w];
+      reinterpret_cast<int*>(L.h)[(long long)t * r + j_lo + i] = a;
+    } else {
+      float a = 0.f;
+#pragma unroll
+      for (int w = 0; w < kStreamWarps; ++w) a += part[i * kStreamWarps + w];
+      L.h[(long long)t * r + j_lo + i] = a;
+    }
   }
 }
 
@@ -476,14 +576,36 @@ __device__ __forceinline__ bool stream_report(const StreamLinear& L, int tg, int
 
 // (a) expert-product items [i_lo, i_hi) of one linear: item = token * 4G + group of 32 features; hs = h of all its tokens.
 // Consecutive items of one row group are reported together.
-__device__ void stream_expert(const StreamLinear& L, int i_lo, int i_hi, const float* hs, const DecodeTokInfo* toks) {
+__device__ void stream_expert(const StreamLinear& L, int i_lo, int i_hi, const float* hs, const DecodeTokInfo* toks, const int8_t* qh8,
+                              const float* gh) {
   const int lane = threadIdx.x & 31;
   const int G32 = L.G * 4, r = L.r, r8 = r >> 3;
   const int Np = L.G * 128;
   unsigned run = 0u;
   for (int i = i_lo; i < i_hi; ++i) {
     const int tok = i / G32, g32 = i - tok * G32;
-    if (g32 * 32 < L.N) {
+    if (g32 * 32 < L.N && L.A8) {
+      // INT8 branch: z_int = B8_e qh (exact), z = z_int / (gamma_B gamma_h gamma_A gamma_t)
+      const int e = toks[tok].expert, r16 = r >> 4;
+      const uint4* bp = L.B_il + ((long long)e * G32 + g32) * r16 * 32 + lane;
+      const uint4* qv = reinterpret_cast<const uint4*>(qh8 + tok * r);
+      int zi = 0;
+      uint4 b[16];
+#pragma unroll
+      for (int u = 0; u < 16; ++u) b[u] = u < r16 ? __ldg(bp + (long long)u * 32) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+      for (int u = 0; u < 16; ++u) {
+        if (u < r16) {
+          const uint4 q = qv[u];
+          zi = __dp4a((int)b[u].x, (int)q.x, zi); zi = __dp4a((int)b[u].y, (int)q.y, zi);
+          zi = __dp4a((int)b[u].z, (int)q.z, zi); zi = __dp4a((int)b[u].w, (int)q.w, zi);
+        }
+      }
+      const float den = __fmul_rn(__fmul_rn(__fmul_rn(__ldg(L.hp_scales + 2 * e + 1), gh[tok]), __ldg(L.hp_scales + 2 * e)), toks[tok].gamma);
+      const int n = g32 * 32 + lane;
+      L.z[(long long)tok * Np + n] = __fdiv_rn((float)zi, den);
+      if (L.zint_dump && n < L.N) L.zint_dump[(long long)tok * L.N + n] = zi;
+    } else if (g32 * 32 < L.N) {
       const uint4* bp = L.B_il + ((long long)toks[tok].expert * G32 + g32) * r8 * 32 + lane;
       const float* hv = hs + tok * r;
       float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
@@ -772,8 +894,25 @@ __global__ void __launch_bounds__(kStreamThreads, 1) k_decode_stream(const __gri
       for (int i = threadIdx.x; i < L.M * L.r; i += kStreamThreads) hs[i] = __ldcg(L.h + i);
       if (threadIdx.x < L.M) reinterpret_cast<int4*>(toks)[threadIdx.x] = __ldcg(reinterpret_cast<const int4*>(L.info) + threadIdx.x);
       __syncthreads();
+      int8_t* qh8 = reinterpret_cast<int8_t*>(stream_smem + bp.off_qh);
+      float* gh = reinterpret_cast<float*>(stream_smem + bp.off_qh + kDecodeMaxTokens * 256);
+      if (L.A8) {
+        // the hidden activation enters the second 8-bit product quantised per token from its exact integers (Eq. 7-9):
+        // gamma_h = 128 / max(max_j |fl32(h_int)|, 1e-5), code = clamp(rint(fl32(h_int) * gamma_h)); warp t takes token t
+        for (int t = warp; t < L.M; t += kStreamWarps) {
+          const int* hi = reinterpret_cast<const int*>(hs) + t * L.r;
+          const int lane = threadIdx.x & 31;
+          float amax = 0.f;
+          for (int j = lane; j < L.r; j += 32) amax = fmaxf(amax, fabsf((float)hi[j]));
+          for (int d = 16; d > 0; d >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, d));
+          const float g = __fdiv_rn(kActQmax, fmaxf(amax, kActAmaxFloor));
+          for (int j = lane; j < L.r; j += 32) qh8[t * L.r + j] = (int8_t)max(-128, min(127, __float2int_rn(__fmul_rn((float)hi[j], g))));
+          if (lane == 0) gh[t] = g;
+        }
+        __syncthreads();
+      }
       const int len = seg_hi - seg_lo;
-      stream_expert(L, seg_lo + (int)((long long)len * warp / kStreamWarps), seg_lo + (int)((long long)len * (warp + 1) / kStreamWarps), hs, toks);
+      stream_expert(L, seg_lo + (int)((long long)len * warp / kStreamWarps), seg_lo + (int)((long long)len * (warp + 1) / kStreamWarps), hs, toks, qh8, gh);
     }
   }
 }
@@ -785,11 +924,20 @@ static inline size_t s_up256(size_t x) { return (x + 255) / 256 * 256; }
 
 // bytes this path needs in an item's workspace beyond what decode_workspace_bytes() counts:
 // codes | h | z | accumulators and counters
-size_t decode_stream_extra_bytes(int M, int K, int N, int r) {
+size_t decode_stream_extra_bytes(int M, int K, int N, int r, bool dump) {
   const size_t G = (N + 127) / 128, C = (K + 127) / 128;
   const size_t groups = (M + kStreamTokenGroup - 1) / kStreamTokenGroup;
   return s_up256((size_t)M * C * 128) + s_up256((size_t)M * std::max(r, 1) * 4) + s_up256((size_t)M * G * 128 * 4) +
-         s_up256(((size_t)M * G * 128 + groups * G) * 4);
+         s_up256(((size_t)M * G * 128 + groups * G) * 4) + (dump ? s_up256((size_t)M * N * 4) : 0);
+}
+// where the INT8 branch leaves its exact integers (h_int always, z_int with the dump flag), for the decode view
+void decode_stream_view(int M, int K, int N, int r, void* ws, bool dump, int** h_int, int** z_int) {
+  const size_t G = (N + 127) / 128, C = (K + 127) / 128;
+  const size_t groups = (M + kStreamTokenGroup - 1) / kStreamTokenGroup;
+  uint8_t* w = static_cast<uint8_t*>(ws) + decode_workspace_bytes(M, K, N, r, dump) + s_up256((size_t)M * C * 128);
+  *h_int = reinterpret_cast<int*>(w);
+  w += s_up256((size_t)M * std::max(r, 1) * 4) + s_up256((size_t)M * G * 128 * 4) + s_up256(((size_t)M * G * 128 + groups * G) * 4);
+  *z_int = dump ? reinterpret_cast<int*>(w) : nullptr;
 }
 
 static int g_decode_stream_on = 1;
@@ -836,11 +984,13 @@ int decode_stream_launch(const DecodeItemArgs* items, int n, cudaStream_t st) {
     const DecodeItemArgs& it = items[i];
     const int M = it.a.T, K = it.a.K, N = it.a.N, r = it.a.r;
     if (!it.bits_il || (r > 0 && !it.B_il) || (r & 7) || M > 16) return PQ_ERR_UNSUPPORTED;
+    if (it.A8 && (r <= 0 || (r & 15) || !it.hp_scales)) return PQ_ERR_UNSUPPORTED;
     StreamLinear& L = bp.lin[i];
     L.X = it.X; L.Wr = it.a.Wr; L.A = it.a.A; L.B_il = reinterpret_cast<const uint4*>(it.B_il);
     L.bits_il = reinterpret_cast<const uint4*>(it.bits_il);
     L.w_scales = it.a.w_scales; L.alpha = it.a.alpha; L.beta = it.a.beta; L.Y = it.Y;
     L.norm_w = it.norm_weight; L.norm_eps = it.norm_eps;
+    L.A8 = it.A8; L.hp_scales = it.hp_scales;
     L.M = M; L.K = K; L.N = N; L.r = r; L.E = (r > 0 && it.a.E > 1) ? it.a.E : 1; L.sstride = it.a.scale_stride;
     L.G = (N + 127) / 128; L.C = (K + 127) / 128;
     uint8_t* w = static_cast<uint8_t*>(it.ws);
@@ -854,6 +1004,8 @@ int decode_stream_launch(const DecodeItemArgs* items, int n, cudaStream_t st) {
     const int groups = (M + kStreamTokenGroup - 1) / kStreamTokenGroup;
     L.cnt = reinterpret_cast<unsigned*>(L.acc + (size_t)M * L.G * 128);
     L.zero_words = M * L.G * 128 + groups * L.G;
+    w += s_up256((size_t)L.zero_words * 4);
+    L.zint_dump = (it.dump && it.A8) ? reinterpret_cast<int*>(w) : nullptr;
     L.chunk0 = (int)total;
     total += (long long)L.G * L.C;
     L.z0 = (int)total_z;
@@ -901,15 +1053,17 @@ int decode_stream_launch(const DecodeItemArgs* items, int n, cudaStream_t st) {
   }
   // shared memory: phase 1 [token][router rows][partial sums], phase 2 [codes][h][token records]
   xbytes = s_up256(xbytes);
-  const size_t avail = kStreamSmemLimit - xbytes - s_up256(part);
+  const size_t avail = kStreamSmemLimit - xbytes - s_up256(part) - xbytes / 2;
   bp.router_rows = max_e > 1 ? (int)std::min<size_t>(max_e, avail / xbytes) : 0;
   if (max_e > 1 && bp.router_rows < 1) return PQ_ERR_UNSUPPORTED;
   bp.off_rows = (int)xbytes;
   bp.off_part = (int)(xbytes + (size_t)bp.router_rows * xbytes);
-  const size_t smem1 = bp.off_part + s_up256(part);
+  bp.off_qn = (int)(bp.off_part + s_up256(part));
+  const size_t smem1 = bp.off_qn + xbytes / 2;          // the token's int8 codes: half the bytes of its bf16 values
   bp.off_h = (int)s_up256(codes);
   bp.off_info = (int)(bp.off_h + s_up256(hbytes));
-  const size_t smem2 = bp.off_info + 256;
+  bp.off_qh = bp.off_info + 256;
+  const size_t smem2 = bp.off_qh + kDecodeMaxTokens * 256 + 256;
   const size_t smem = std::max(smem1, smem2);
   if (smem > kStreamSmemLimit) return PQ_ERR_UNSUPPORTED;
   bp.bar_slot = stream_bar_slot(st);

@@ -131,12 +131,17 @@ struct DecodeItemArgs {
   const uint16_t* norm_weight = nullptr;   // RMSNorm gain [K] bf16, or null: X arrives normalised
   float norm_eps = 0.f;
   const uint32_t* bits_il = nullptr;       // weights laid out by decode_pack (streaming kernel), or null
-  const uint16_t* B_il = nullptr;
+  const uint16_t* B_il = nullptr;          // bf16 rows of B_e, or the int8 codes B8_e when A8 is set
+  const int8_t* A8 = nullptr;              // INT8 high-precision branch: codes of A_e [E, r, K], or null
+  const float* hp_scales = nullptr;        // [E][2] {gamma_A, gamma_B}
 };
 // streaming decode kernel (pq_decode_stream.cu)
 void decode_pack_sizes(int K, int N, int r, int E, size_t* bits_bytes, size_t* b_bytes);
 int decode_pack(int K, int N, int r, int E, const uint32_t* bits, const uint16_t* B, uint32_t* bits_il, uint16_t* B_il, cudaStream_t st);
-size_t decode_stream_extra_bytes(int M, int K, int N, int r);
+size_t decode_stream_extra_bytes(int M, int K, int N, int r, bool dump);
+void decode_stream_view(int M, int K, int N, int r, void* ws, bool dump, int** h_int, int** z_int);
+size_t decode_pack_b8_bytes(int N, int r, int E);
+int decode_pack_b8(int N, int r, int E, const int8_t* B8, int8_t* B8_il, cudaStream_t st);
 int decode_stream_launch(const DecodeItemArgs* items, int n, cudaStream_t st);   // PQ_ERR_UNSUPPORTED: use the other kernels
 void decode_stream_enable(int mode);   // 0 never, 1 where it pays (default), 2 wherever the items allow
 void decode_stream_prefetch(int on);

@@ -74,6 +74,7 @@ class PQLinear:
             self.Y = self._buf((T, N), torch.bfloat16)
         self.X = self.W = self.A = self.B = self.Wr = self.alpha = self.beta = self.dY = None
         self.w_bits_il = self.B_il = None
+        self.B8_il = None   # set by pack_decode_hp8(): decode then runs the INT8 high-precision branch
 
     # -- buffers --------------------------------------------------------------
     def _buf(self, shape, dtype):
@@ -129,6 +130,13 @@ class PQLinear:
         pqb.pq_pack_decode(self.desc, self.w_bits, self.B, self.w_bits_il, self.B_il)
         return True
 
+    def pack_decode_hp8(self):
+        """INT8 high-precision branch for decode: quantise the experts (pack_experts) and lay B8 out for the streaming
+        kernel; decode() and decode_entry() then use it (needs pack_decode() too)."""
+        self.pack_experts()
+        self.B8_il = self._buf((pqb.pq_decode_pack_hp8_bytes(self.desc),), torch.uint8)
+        pqb.pq_pack_decode_hp8(self.desc, self.B8, self.B8_il)
+
     def decode(self, X=None, Y=None):
         """Inference forward from the packed sign bits (w_s8 is not used).  With `norm_weight` set, X is the
         un-normalised activation and RMSNorm is fused in front of the quantiser (a batch of one)."""
@@ -146,7 +154,8 @@ class PQLinear:
     def decode_entry(self):
         """This layer's arguments as one entry for binding.make_decode_items."""
         return (self.desc, self.X, self.w_bits, self.w_scales, self.A, self.B, self.Wr, self.alpha, self.beta, self.Y, self.ws_decode,
-                getattr(self, "norm_weight", None), getattr(self, "norm_eps", 0.0), self.w_bits_il, self.B_il)
+                getattr(self, "norm_weight", None), getattr(self, "norm_eps", 0.0), self.w_bits_il, self.B_il,
+                self.A8 if self.B8_il is not None else None, self.B8_il, self.hp_scales if self.B8_il is not None else None)
 
     def decode_view(self) -> dict:
         return pqb.pq_decode_view_init(self.desc, self.ws_decode)

@@ -241,3 +241,53 @@ def test_decode_rejects_too_many_tokens():
     with pytest.raises(pqb.PqError) as ei:
         pqb.pq_linear_forward(L.desc, L.X, L.w_bits, None, L.w_scales, L.A, L.B, L.Wr, L.alpha, L.beta, L.Y, None, ws)
     assert ei.value.status == pqb.PQ_ERR_SHAPE
+
+
+@pytest.mark.parametrize("shape", [dict(T=1, K=256, N=96, r=32, E=4), dict(T=16, K=512, N=2048, r=64, E=8), dict(T=9, K=384, N=320, r=160, E=1),
+                                   dict(T=5, K=2080, N=992, r=48, E=3), dict(T=1, K=3200, N=8640, r=160, E=8),
+                                   dict(T=4, K=8640, N=3200, r=160, E=8)])
+def test_decode_int8_hp_branch_matches_oracle(shape):
+    # Sec. 3.2 on the decode path: the branch multiplies the token's int8 codes by int8 expert matrices; every integer it
+    # goes through (h_int, and with it the codes of h; z_int) must equal the oracle's, Y within the float tolerance.
+    c = I.make_linear_case(shape["T"], shape["K"], shape["N"], shape["r"], shape["E"], seed=41)
+    L = PQLinear(c["T"], c["K"], c["N"], c["r"], c["E"], training=False, dump_acc=True, guard=True).load_case(c)
+    L.pack(bits_only=True)
+    if L.w_bits_il is None:
+        L.pack_decode()                  # the INT8 branch lives on the streaming kernel whatever the test's kernel choice
+    L.pack_decode_hp8()
+    L.decode()
+    torch.cuda.synchronize()
+    check_status()
+    assert L.check_guards() == 0
+    A8, gA, B8, gB = O.quantize_experts(c["A"], c["B"])
+    assert np.array_equal(L.A8.cpu().numpy(), A8) and np.array_equal(L.B8.cpu().numpy(), B8)
+    mu, lam = O.weight_scales(c["W"])
+    bits = O.pack_bits(O.binarize(c["W"], mu))
+    f = O.decode_forward(c["X"], bits, lam, c["A"], c["B"], c["Wr"], c["alpha"], c["beta"], hp_int8=(A8, gA, B8, gB))
+    v = L.decode_view()
+    assert np.array_equal(v["expert"].cpu().numpy(), f["idx"])
+    assert np.array_equal(f32(v["gamma"]), f["gamma"])
+    assert np.array_equal(v["acc"].cpu().numpy().astype(np.int64), f["acc"])
+    assert np.array_equal(v["hp_h_int"].cpu().numpy().astype(np.int64), f["h_int"])
+    assert np.array_equal(v["hp_z_int"].cpu().numpy().astype(np.int64), f["z_int"])
+    assert rel_err(f32(L.Y), f["Y"]) <= TOL_BF16
+    # and it is the INT8 branch, not the bf16 one
+    fb = O.decode_forward(c["X"], bits, lam, c["A"], c["B"], c["Wr"], c["alpha"], c["beta"])
+    assert not np.array_equal(fb["Y"], f["Y"])
+
+
+def test_decode_int8_hp_branch_argument_errors():
+    c = I.make_linear_case(2, 256, 128, 24, 2, seed=1)                   # r not a multiple of 16
+    L = PQLinear(2, 256, 128, 24, 2, training=False).load_case(c)
+    assert pqb.pq_decode_pack_hp8_bytes(L.desc) == 0
+    c = I.make_linear_case(2, 256, 128, 32, 2, seed=1)
+    L = PQLinear(2, 256, 128, 32, 2, training=False).load_case(c)
+    L.pack(bits_only=True)
+    if L.w_bits_il is None:
+        L.pack_decode()
+    L.pack_decode_hp8()
+    entry = list(L.decode_entry())
+    entry[13] = None                                                     # no streaming layout of the sign bits
+    with pytest.raises(pqb.PqError) as ei:
+        pqb.pq_decode_batch(pqb.make_decode_items([tuple(entry)]))
+    assert ei.value.status == pqb.PQ_ERR_NULL
