@@ -539,6 +539,11 @@ def build_decode_weights(ctx):
             L.B = sets[-1]["B"]
             L.pack_decode()
             sets[-1]["w_bits_il"], sets[-1]["B_il"] = L.w_bits_il, L.B_il
+            if ctx.decode_hp8:
+                # the INT8 high-precision branch: int8 codes of the experts, B8 in the streaming layout
+                L.A = sets[-1]["A"]
+                L.pack_decode_hp8()
+                sets[-1]["A8"], sets[-1]["B8_il"], sets[-1]["hp_scales"] = L.A8, L.B8_il, L.hp_scales
             del L
     torch.cuda.synchronize()
     return sets
@@ -556,6 +561,8 @@ def make_decode_layers(ctx, M, weights, rmsnorm=False):
         L.w_s8 = None
         if ctx.decode_kernels != "pair":
             L.w_bits_il, L.B_il = w["w_bits_il"], w["B_il"]
+        if ctx.decode_hp8:
+            L.A8, L.B8_il, L.hp_scales = w["A8"], w["B8_il"], w["hp_scales"]
         L.X = torch.from_numpy(act["X"]).to(device).to(torch.bfloat16)
         L.Wr = torch.from_numpy(act["Wr"]).to(device).to(torch.bfloat16)
         L.alpha = torch.full((1,), 2.0, device=device)
@@ -586,7 +593,7 @@ def measure_decode(ctx, M, steps, weights, full, batch=16, rmsnorm=False):
     algo = 0
     for L in layers:
         experts = L.decode_view()["expert"].cpu().numpy()
-        algo += L.N * L.K // 8 + 4 + len(set(experts.tolist())) * 2 * r * (L.K + L.N) + 2 * E * L.K + 2 * M * L.K + 2 * M * L.N
+        algo += L.N * L.K // 8 + 4 + len(set(experts.tolist())) * (1 if ctx.decode_hp8 else 2) * r * (L.K + L.N) + 2 * E * L.K + 2 * M * L.K + 2 * M * L.N
     keep = []
 
     def capture(b):
@@ -678,11 +685,12 @@ def run_decode(args, ctx):
             "metric": "pQuant decode linear (packed 1-bit weights) tokens/s", "value": round(reps.whole_job_rate(M * nlin, ms_per_step), 1),
             "unit": "token-linears/s", "n_gpus": ctx.world, "steps": args.steps, "warmup": 3,
             "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "s8 x s8 -> s32 (1-bit branch), bf16 -> f32 (experts)", "data": "synthetic",
+            "dtype": "s8 x s8 -> s32 (1-bit branch), " + ("s8 x s8 -> s32 (INT8 experts)" if ctx.decode_hp8 else "bf16 -> f32 (experts)"),
+            "data": "synthetic",
             "config": {"workload": decode_workload_text(M, args.decode_rmsnorm),
                        "linears_per_step": nlin, "l2": f"{d['algo'] / 1e6:.0f} MB of distinct weights per step, larger than L2",
                        "launch": f"one CUDA graph per step, pq_decode_batch over groups of {args.decode_batch} independent linears",
-                       "kernels": ctx.decode_kernels, "replicas": ctx.world},
+                       "kernels": ctx.decode_kernels, "hp_branch": "int8" if ctx.decode_hp8 else "bf16", "replicas": ctx.world},
             "roofline": {"kernel": "decode kernels (all launches of a step)", "bound": "hbm", "achieved": b["gbs"],
                          "peak": ctx.peaks["hbm_gbs"], "unit": "GB/s", "frac": b["hbm_frac"],
                          "peak_source": f"{ctx.peak_kind} hbm_gbs", "algorithmic_bytes_per_step": d["algo"],
@@ -872,6 +880,7 @@ def main():
     ap.add_argument("--decode-kernels", default="auto", choices=["auto", "stream", "pair"],
                     help="auto: the library picks per launch group; stream: the cooperative streaming kernel wherever the items allow; "
                          "pair: the two-kernel path on the plain layout")
+    ap.add_argument("--decode-hp8", action="store_true", help="decode with the INT8 high-precision branch (int8 experts: half the expert bytes)")
     ap.add_argument("--decode-mma-from", type=int, default=5, help="streaming decode kernel: token groups of at least this size use the tensor-core bit product")
     ap.add_argument("--decode-prefetch", type=int, default=1, choices=[0, 1], help="streaming decode kernel: L2 prefetch of the sign bits during the token work")
     ap.add_argument("--decode-rmsnorm", action="store_true", help="decode from un-normalised activations, RMSNorm fused into the token preparation")
@@ -890,6 +899,7 @@ def main():
         return
     ctx = Ctx()
     ctx.decode_kernels = args.decode_kernels
+    ctx.decode_hp8 = args.decode_hp8
     ctx.pqb.pq_set_option(ctx.pqb.PQ_OPT_DECODE_STREAM, {"auto": 1, "stream": 2, "pair": 0}[args.decode_kernels])
     ctx.pqb.pq_set_option(ctx.pqb.PQ_OPT_DECODE_PREFETCH, args.decode_prefetch)
     ctx.pqb.pq_set_option(ctx.pqb.PQ_OPT_DECODE_MMA_FROM, args.decode_mma_from)
