@@ -42,6 +42,40 @@ def test_bounded_wait_runs_out_and_the_next_call_is_correct():
     want = A[rows].cpu().numpy().astype(np.int64) @ B.cpu().numpy().astype(np.int64).T
     assert np.array_equal(D[rows].cpu().numpy().astype(np.int64), want)
 
+def test_grid_barrier_of_the_streaming_decode_kernel_runs_out_and_recovers():
+    # The streaming decode kernel's CTAs meet at one grid barrier with a bounded wait.  With a limit of one cycle the first
+    # poll that finds a CTA still missing gives up: that CTA records PQ_ERR_TIMEOUT and skips the rest of its work (nothing
+    # after the barrier reads what a missing CTA would have written), every CTA still leaves the barrier words balanced,
+    # and the next call with the normal limit is exact.  Only this kernel runs under the short limit.
+    c = I.make_linear_case(4, 512, 2048, 32, 4, seed=53)
+    L = PQLinear(4, 512, 2048, 32, 4, training=False, dump_acc=True).load_case(c)
+    pqb.pq_set_option(pqb.PQ_OPT_DECODE_STREAM, 2)
+    try:
+        L.pack(bits_only=True)
+        if L.w_bits_il is None:
+            L.pack_decode()
+        L.decode()
+        torch.cuda.synchronize()
+        check_status()
+        want = L.Y.clone()
+        acc = L.decode_view()["acc"].clone()
+        pqb.pq_set_option(pqb.PQ_OPT_SPIN_CYCLES, 1)
+        try:
+            L.decode()
+            code, where = pqb.pq_device_status()
+        finally:
+            pqb.pq_set_option(pqb.PQ_OPT_SPIN_CYCLES, 0)
+        assert code == pqb.PQ_ERR_TIMEOUT and where == 4
+        assert pqb.pq_device_status() == (0, 0)
+        for _ in range(2):
+            L.Y.zero_()
+            L.decode()
+            torch.cuda.synchronize()
+            check_status()
+            assert torch.equal(L.Y, want) and torch.equal(L.decode_view()["acc"], acc)
+    finally:
+        pqb.pq_set_option(pqb.PQ_OPT_DECODE_STREAM, 1)
+
 
 @pytest.mark.parametrize("shape", [dict(T=333, K=384, N=544, r=64, E=1), dict(T=1000, K=512, N=768, r=128, E=8),
                                    dict(T=200, K=256, N=320, r=0, E=0), dict(T=130, K=5632, N=96, r=16, E=4)])
