@@ -489,12 +489,14 @@ def subrecords(args, ctx, engine):
             r = {"workload": decode_workload_text(None, False), "note": (
                 "fraction of the measured HBM rate = algorithmic bytes / time / hbm_gbs.  batched16: 16 independent linears per "
                 "launch (other sequences, parallel projections), one cooperative streaming kernel on weights in its own layout; "
+                "batched_all: all 78 linears of the step handed to one pq_decode_batch call (one launch: the kernel's fixed costs -- "
+                "token work, grid barrier, launch gap -- are paid once); "
                 "pairs: what one sequence's model allows (gate + up of a block together); serial: one call per linear, each after "
                 "the previous one -- both on the two-kernel path, which the library picks for small groups"),
                 "kernels": ctx.decode_kernels}
             for M in (1, 4, 16):
                 d = measure_decode(ctx, M, max(5, min(args.steps, 20)), weights, full=True)
-                r[f"m{M}"] = {"batched16": d["batched"], "pairs": d["pairs"], "serial": d["serial"],
+                r[f"m{M}"] = {"batched16": d["batched"], "batched_all": d["batched_all"], "pairs": d["pairs"], "serial": d["serial"],
                               "algorithmic_bytes_per_step": d["algo"], "clocks": d["clocks"]}
             return r
         guarded("decode", dec)
@@ -637,6 +639,7 @@ def measure_decode(ctx, M, steps, weights, full, batch=16, rmsnorm=False):
     if full:
         out["serial"] = figures(time_graph(capture(1)))
         out["pairs"] = figures(time_graph(capture(2)))
+        out["batched_all"] = figures(time_graph(capture(nlin)))
     with ClockSampler(ctx.local) as clk:
         ms = time_graph(graph)
     out["batched"] = figures(ms)
@@ -695,7 +698,7 @@ def run_decode(args, ctx):
                          "peak": ctx.peaks["hbm_gbs"], "unit": "GB/s", "frac": b["hbm_frac"],
                          "peak_source": f"{ctx.peak_kind} hbm_gbs", "algorithmic_bytes_per_step": d["algo"],
                          "us_per_linear": b["us_per_linear"], "traffic": None},
-            "serial": d.get("serial"), "pairs": d.get("pairs"),
+            "serial": d.get("serial"), "pairs": d.get("pairs"), "batched_all": d.get("batched_all"),
             "cpu_baseline": cpu_baseline,
             "e2e": {"value": round(reps.whole_job_rate(M * nlin, ms_e2e), 1), "unit": "token-linears/s",
                     "h2d_bytes_per_step": sum(t.numel() * t.element_size() for t in hx),

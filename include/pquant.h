@@ -274,7 +274,8 @@ int pq_decode_view_init(const pq_desc* d, void* ws, pq_decode_view* out);
  * stream their weights back to back instead of paying a launch and a pipeline fill each).
  * Each item is what pq_linear_forward takes in its decode form; results are identical to n
  * separate calls.  `items` is a HOST array, read before the call returns.  1 <= n <= 4096
- * (PQ_ERR_SHAPE otherwise; launched in groups of 16); every item needs its own ws. */
+ * (PQ_ERR_SHAPE otherwise; launched in groups of up to 96 consecutive items on the streaming kernel, of 16 on the
+ * two-kernel path); every item needs its own ws. */
 typedef struct pq_decode_item {
   pq_desc desc;            /* T <= 16 */
   const uint16_t* X;       /* [T,K] bf16 */
@@ -395,7 +396,7 @@ int pq_device_status(void* stream, int* code, int* where);
  *   outputs of that call are undefined.  Applies to the current device; blocks until the device's
  *   earlier work has finished.  Meant for pq_debug_gemm; do not shorten the limit around the decode
  *   entry points, whose later stages read indices an abandoned stage has not delivered.
- *   PQ_OPT_DECODE_STREAM (default 1): which launch groups of pq_decode_batch (up to 16 consecutive items) run on the
+ *   PQ_OPT_DECODE_STREAM (default 1): which launch groups of pq_decode_batch (up to 96 consecutive items) run on the
  *   streaming kernel when their items carry w_bits_il / B_il.  1 = those for which it is the faster of the two paths
  *   (12 or more linears; 6 or more when no item has more than two tokens); 2 = every group; 0 = none.
  *   PQ_OPT_DECODE_PREFETCH (default 1): the streaming decode kernel asks for the sign bits four chunks ahead of its

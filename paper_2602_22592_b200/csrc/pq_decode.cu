@@ -794,30 +794,40 @@ static int decode_launch(const DecodeItemArgs* items, int n, cudaStream_t st) {
   return rc == PQ_ERR_UNSUPPORTED ? decode_launch_with(items, n, kDecodeMaxConsumerWarps, st) : rc;
 }
 
+// the launch groups of the streaming kernel are larger than those of the two-kernel path (defined in pq_decode_stream.cu)
+int decode_stream_max_batch();
+
 int decode_batch(const DecodeItemArgs* items, int n, cudaStream_t st) {
-  for (int i = 0; i < n; i += kDecodeMaxBatch) {
-    const int m = n - i < kDecodeMaxBatch ? n - i : kDecodeMaxBatch;
-    // the streaming kernel takes a group whose items all carry its weight layout; otherwise the kernels above
-    // (measured on the 3B shapes: its grid barrier and its longer chain of dependent steps cost about as much as eight
-    // linears' worth of streaming, so small groups, and mid-sized groups of many tokens, stay on the two kernels above)
-    int rc = PQ_ERR_UNSUPPORTED;
-    bool any_hp8 = false;
-    for (int k = 0; k < m; ++k) any_hp8 = any_hp8 || items[i + k].A8 != nullptr;
-    const int mode = any_hp8 ? 2 : decode_stream_mode();
-    if (mode > 0) {
-      bool all = true, hp8 = false;
-      int max_m = 1;
-      for (int k = 0; k < m; ++k) {
-        all = all && items[i + k].bits_il != nullptr;
-        hp8 = hp8 || items[i + k].A8 != nullptr;
-        max_m = std::max(max_m, items[i + k].a.T);
-      }
-      const bool worth = mode > 1 || hp8 || m >= 12 || (m >= 6 && max_m <= 2);
-      if (all && worth) rc = decode_stream_launch(items + i, m, st);
-      if (hp8 && rc == PQ_ERR_UNSUPPORTED) return rc;       // the INT8 branch exists on the streaming kernel only
+  int i = 0;
+  while (i < n) {
+    // The streaming kernel takes a group whose items all carry its weight layout, where it pays.  (Measured on the 3B
+    // shapes: its grid barrier and its longer chain of dependent steps cost about as much as eight linears' worth of
+    // streaming, so small groups, and mid-sized groups of many tokens, stay on the two kernels above.)
+    const int mode_opt = decode_stream_mode();
+    int m = std::min(n - i, decode_stream_max_batch());
+    bool all = true, hp8 = false;
+    int max_m = 1, run = 0;
+    for (int k = 0; k < m; ++k) {
+      if (!items[i + k].bits_il) { all = false; break; }
+      ++run;
+      hp8 = hp8 || items[i + k].A8 != nullptr;
+      max_m = std::max(max_m, items[i + k].a.T);
     }
-    if (rc == PQ_ERR_UNSUPPORTED) rc = decode_launch(items + i, m, st);
+    int rc = PQ_ERR_UNSUPPORTED;
+    if (!all) m = run;                                       // the items in front that carry the layout, if any
+    const int mode = hp8 ? 2 : mode_opt;
+    if (m > 0 && mode > 0 && (mode > 1 || hp8 || m >= 12 || (m >= 6 && max_m <= 2))) {
+      rc = decode_stream_launch(items + i, m, st);
+      if (hp8 && rc == PQ_ERR_UNSUPPORTED) return rc;        // the INT8 branch exists on the streaming kernel only
+    }
+    if (rc == PQ_ERR_UNSUPPORTED) {
+      m = std::min(n - i, kDecodeMaxBatch);
+      for (int k = 0; k < m; ++k)
+        if (items[i + k].A8) return PQ_ERR_UNSUPPORTED;
+      rc = decode_launch(items + i, m, st);
+    }
     if (rc) return rc;
+    i += m;
   }
   return PQ_OK;
 }

@@ -32,7 +32,7 @@ namespace pq {
 
 constexpr int kStreamThreads = 512;
 constexpr int kStreamWarps = kStreamThreads / 32;
-constexpr int kStreamMaxBatch = 16;
+constexpr int kStreamMaxBatch = 96;      // linears per launch: their records travel as kernel parameters (32 KB limit)
 constexpr int kStreamTokenGroup = 8;     // tokens whose codes sit in shared memory at once
 constexpr int kStreamBarSlots = 64;
 
@@ -66,7 +66,6 @@ struct StreamLinear {
   int G, C;                 // row groups; chunks per row group
   int chunk0;               // position of this linear's first chunk in the launch-wide list of chunks
   int z0;                   // position of its first item in the launch-wide list of expert-product items (M * 4 G each)
-  int cta_first, cta_count; // the CTAs that share its token work
   int zero_words;           // int32 words from `acc` on that phase 1 clears (acc and cnt are adjacent)
 };
 // The descriptor travels as kernel parameters (constant memory).  What every CTA needs to find its work sits in a few
@@ -85,7 +84,8 @@ struct StreamBatch {
   int off_qh;
   int chunk0[kStreamMaxBatch + 1];   // first chunk of every linear in the launch-wide list (and the total)
   int z0[kStreamMaxBatch + 1];       // first expert-product item of every linear
-  unsigned char duty[160];           // linear whose token work CTA b shares (255: none)
+  int cost0[kStreamMaxBatch + 1];    // token work before every linear, in units of K / 32 per (token, row of A_e)
+  int duty0[161];                    // where in that list the share of CTA b begins (and, one further, ends)
   StreamLinear lin[kStreamMaxBatch];
 };
 
@@ -318,6 +318,7 @@ __device__ __forceinline__ void stream_h_rows8(const uint4* a16, const uint4* q1
   }
 }
 
+template <bool HP8>
 __device__ void stream_token(const StreamBatch& bp, const StreamLinear& L, int t, int j_lo, int j_hi, bool owner, bool first, uint8_t* smem, StreamShared& sh) {
   const int K = L.K, E = L.E, r = L.r;
   const int chunks = K >> 3;
@@ -419,7 +420,7 @@ __device__ void stream_token(const StreamBatch& bp, const StreamLinear& L, int t
   // rows [j_lo, j_hi) of h = A_e x: warp w takes the w-th sixteenth of every row (whole 16-byte pieces), sixteen
   // loads per lane issued before the first use; the sixteen partial sums of a row are added in warp order afterwards
   const int nrows = r > 0 ? j_hi - j_lo : 0;
-  if (nrows > 0 && L.A8) {
+  if (HP8 && nrows > 0 && L.A8) {
     // INT8 branch: the token's codes in natural order (Eq. 7-9, the values the owner also writes out below)
     uint2* qn = reinterpret_cast<uint2*>(smem + bp.off_qn);
     for (int c = threadIdx.x; c < chunks; c += kStreamThreads) {
@@ -494,7 +495,7 @@ __device__ void stream_token(const StreamBatch& bp, const StreamLinear& L, int t
     L.info[t] = DecodeTokInfo{best, gate, gamma, tot};
   }
   for (int i = threadIdx.x; i < nrows; i += kStreamThreads) {
-    if (L.A8) {
+    if (HP8 && L.A8) {
       int a = 0;
 #pragma unroll
       for (int w = 0; w < kStreamWarps; ++w) a += reinterpret_cast<const int*>(part)[i * kStreamWarps + w];
@@ -576,6 +577,7 @@ __device__ __forceinline__ bool stream_report(const StreamLinear& L, int tg, int
 
 // (a) expert-product items [i_lo, i_hi) of one linear: item = token * 4G + group of 32 features; hs = h of all its tokens.
 // Consecutive items of one row group are reported together.
+template <bool HP8>
 __device__ void stream_expert(const StreamLinear& L, int i_lo, int i_hi, const float* hs, const DecodeTokInfo* toks, const int8_t* qh8,
                               const float* gh) {
   const int lane = threadIdx.x & 31;
@@ -584,7 +586,7 @@ __device__ void stream_expert(const StreamLinear& L, int i_lo, int i_hi, const f
   unsigned run = 0u;
   for (int i = i_lo; i < i_hi; ++i) {
     const int tok = i / G32, g32 = i - tok * G32;
-    if (g32 * 32 < L.N && L.A8) {
+    if (HP8 && g32 * 32 < L.N && L.A8) {
       // INT8 branch: z_int = B8_e qh (exact), z = z_int / (gamma_B gamma_h gamma_A gamma_t)
       const int e = toks[tok].expert, r16 = r >> 4;
       const uint4* bp = L.B_il + ((long long)e * G32 + g32) * r16 * 32 + lane;
@@ -804,6 +806,9 @@ __device__ void stream_bits_mma(const StreamLinear& L, int tg, int mg, int p_lo,
 // ---------------------------------------------------------------------------
 // the kernel: grid = one CTA per SM (cooperative launch), 512 threads
 // ---------------------------------------------------------------------------
+// HP8: some linear of the launch uses the INT8 high-precision branch; MMA: some token group is large enough for the
+// tensor-core bit product.  Separate instantiations, so that the common case carries neither's registers nor code.
+template <bool HP8, bool MMA>
 __global__ void __launch_bounds__(kStreamThreads, 1) k_decode_stream(const __grid_constant__ StreamBatch bp) {
   extern __shared__ __align__(128) uint8_t stream_smem[];
   __shared__ StreamShared sh;
@@ -834,17 +839,21 @@ __global__ void __launch_bounds__(kStreamThreads, 1) k_decode_stream(const __gri
     for (long long i = w_lo + threadIdx.x; i < w_hi; i += kStreamThreads) L.acc[i] = 0;
   }
 
-  // phase 1: this CTA's share of one linear's token work
-  if (bp.duty[cta] != 255) {
-    const StreamLinear& L = bp.lin[bp.duty[cta]];
-    const int s = cta - L.cta_first;
-    const int rp = max(L.r, 1);
-    const long long U = (long long)L.M * rp;
-    const int u_lo = (int)(U * s / L.cta_count), u_hi = (int)(U * (s + 1) / L.cta_count);
-    if (u_lo < u_hi) {
+  // phase 1: this CTA's share of the token work, a launch-wide list of (token, row of A_e) units weighted by the length
+  // of a row and cut into contiguous shares by the host; a unit belongs to the CTA in whose share it begins
+  {
+    const long long d_lo = bp.duty0[cta], d_hi = bp.duty0[cta + 1];
+    for (int l = 0; l < bp.n; ++l) {
+      if (bp.cost0[l + 1] <= d_lo || bp.cost0[l] >= d_hi) continue;
+      const StreamLinear& L = bp.lin[l];
+      const long long w = L.K >> 5, base = bp.cost0[l];
+      const int rp = max(L.r, 1);
+      const long long U = (long long)L.M * rp;
+      const int u_lo = (int)min(U, (max(d_lo - base, 0LL) + w - 1) / w), u_hi = (int)min(U, (max(d_hi - base, 0LL) + w - 1) / w);
+      if (u_lo >= u_hi) continue;
       for (int t = u_lo / rp; t <= (u_hi - 1) / rp; ++t) {
         const int j_lo = max(u_lo, t * rp) - t * rp, j_hi = min(u_hi, (t + 1) * rp) - t * rp;
-        stream_token(bp, L, t, j_lo, j_hi, j_lo == 0, t == u_lo / rp, stream_smem, sh);
+        stream_token<HP8>(bp, L, t, j_lo, j_hi, j_lo == 0, t == u_lo / rp, stream_smem, sh);
       }
     }
   }
@@ -876,7 +885,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) k_decode_stream(const __gri
           if (threadIdx.x < L.M) reinterpret_cast<int4*>(toks)[threadIdx.x] = __ldcg(reinterpret_cast<const int4*>(L.info) + threadIdx.x);
         }
         __syncthreads();
-        if (mg >= bp.mma_from) stream_bits_mma(L, tg, mg, p_lo, p_hi, qs, qstride, toks, bp.prefetch);
+        if (MMA && mg >= bp.mma_from) stream_bits_mma(L, tg, mg, p_lo, p_hi, qs, qstride, toks, bp.prefetch);
         else if (mg == 1) stream_bits<1>(L, tg, mg, p_lo, p_hi, qs, qstride, toks, bp.prefetch);
         else if (mg == 2) stream_bits<2>(L, tg, mg, p_lo, p_hi, qs, qstride, toks, bp.prefetch);
         else if (mg <= 4) stream_bits<4>(L, tg, mg, p_lo, p_hi, qs, qstride, toks, bp.prefetch);
@@ -896,7 +905,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) k_decode_stream(const __gri
       __syncthreads();
       int8_t* qh8 = reinterpret_cast<int8_t*>(stream_smem + bp.off_qh);
       float* gh = reinterpret_cast<float*>(stream_smem + bp.off_qh + kDecodeMaxTokens * 256);
-      if (L.A8) {
+      if (HP8 && L.A8) {
         // the hidden activation enters the second 8-bit product quantised per token from its exact integers (Eq. 7-9):
         // gamma_h = 128 / max(max_j |fl32(h_int)|, 1e-5), code = clamp(rint(fl32(h_int) * gamma_h)); warp t takes token t
         for (int t = warp; t < L.M; t += kStreamWarps) {
@@ -912,7 +921,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) k_decode_stream(const __gri
         __syncthreads();
       }
       const int len = seg_hi - seg_lo;
-      stream_expert(L, seg_lo + (int)((long long)len * warp / kStreamWarps), seg_lo + (int)((long long)len * (warp + 1) / kStreamWarps), hs, toks, qh8, gh);
+      stream_expert<HP8>(L, seg_lo + (int)((long long)len * warp / kStreamWarps), seg_lo + (int)((long long)len * (warp + 1) / kStreamWarps), hs, toks, qh8, gh);
     }
   }
 }
@@ -947,6 +956,7 @@ void decode_stream_mma_from(int m) { g_decode_stream_mma_from = m < 1 ? 1 : m; }
 void decode_stream_enable(int mode) { g_decode_stream_on = mode < 0 ? 0 : mode > 2 ? 2 : mode; }
 void decode_stream_prefetch(int on) { g_decode_stream_prefetch = on ? 1 : 0; }
 int decode_stream_mode() { return g_decode_stream_on; }
+int decode_stream_max_batch() { return kStreamMaxBatch; }
 
 void decode_stream_reset() {
   void* p = nullptr;
@@ -1026,30 +1036,32 @@ int decode_stream_launch(const DecodeItemArgs* items, int n, cudaStream_t st) {
     bp.chunk0[i] = i < n ? bp.lin[i].chunk0 : (int)total;
     bp.z0[i] = i < n ? bp.lin[i].z0 : (int)total_z;
   }
-  // the token work of a linear belongs to CTAs of its own, as many as its share of that work (at least one)
   const int nC = sms;
-  if (n > nC) return PQ_ERR_UNSUPPORTED;
   {
-    double cost[kStreamMaxBatch], sum = 0.0;
+    long long run = 0;
     for (int i = 0; i < n; ++i) {
-      const StreamLinear& L = bp.lin[i];
-      cost[i] = (double)L.M * L.K * (L.r + (L.E > 1 ? L.E : 0) + 2);
-      sum += cost[i];
+      bp.cost0[i] = (int)run;
+      run += (long long)bp.lin[i].M * std::max(bp.lin[i].r, 1) * (bp.lin[i].K >> 5);
+      if (run > (1ll << 30)) return PQ_ERR_UNSUPPORTED;
     }
-    int next = 0;
-    double run = 0.0;
-    for (int i = 0; i < n; ++i) {
-      run += cost[i];
-      int end = i + 1 == n ? nC : (int)(run / sum * (nC - n) + 0.5) + (i + 1);   // one CTA each, the rest by cost
-      end = std::min(std::max(end, next + 1), nC - (n - 1 - i));
-      bp.lin[i].cta_first = next;
-      bp.lin[i].cta_count = end - next;
-      next = end;
-    }
+    for (int i = n; i <= kStreamMaxBatch; ++i) bp.cost0[i] = (int)run;
     if (nC > 160) return PQ_ERR_UNSUPPORTED;
-    for (int c = 0; c < 160; ++c) bp.duty[c] = 255;
-    for (int i = 0; i < n; ++i)
-      for (int c = bp.lin[i].cta_first; c < bp.lin[i].cta_first + bp.lin[i].cta_count; ++c) bp.duty[c] = (unsigned char)i;
+    if (4 * n <= nC) {
+      // few linears: every linear gets CTAs of its own, as many as its share of the work (at least one), so that no CTA
+      // prepares tokens of two linears (the token, the router rows and the routing are a fixed cost per CTA and linear)
+      int next = 0;
+      for (int i = 0; i < n; ++i) {
+        int end = i + 1 == n ? nC : (int)((double)bp.cost0[i + 1] / (double)run * (nC - n) + 0.5) + (i + 1);
+        end = std::min(std::max(end, next + 1), nC - (n - 1 - i));
+        const long long c0 = bp.cost0[i], c1 = bp.cost0[i + 1];
+        for (int c = next; c < end; ++c) bp.duty0[c] = (int)(c0 + (c1 - c0) * (c - next) / (end - next));
+        next = end;
+      }
+      bp.duty0[nC] = (int)run;
+    } else {
+      // many linears: equal shares of the list, whatever linears they fall on
+      for (int c = 0; c <= nC; ++c) bp.duty0[c] = (int)(run * c / nC);
+    }
   }
   // shared memory: phase 1 [token][router rows][partial sums], phase 2 [codes][h][token records]
   xbytes = s_up256(xbytes);
@@ -1070,7 +1082,20 @@ int decode_stream_launch(const DecodeItemArgs* items, int n, cudaStream_t st) {
   if (bp.bar_slot < 0) return PQ_ERR_UNSUPPORTED;
   bp.prefetch = g_decode_stream_prefetch ? 4 : 0;
   bp.mma_from = g_decode_stream_mma_from;
-  static const bool limit_set = cudaFuncSetAttribute(k_decode_stream, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStreamSmemLimit) == cudaSuccess;
+  bool hp8 = false, mma = false;
+  for (int i = 0; i < n; ++i) {
+    hp8 = hp8 || bp.lin[i].A8 != nullptr;
+    const int M = bp.lin[i].M;
+    mma = mma || std::min(M, kStreamTokenGroup) >= bp.mma_from || (M > kStreamTokenGroup && M - kStreamTokenGroup >= bp.mma_from);
+  }
+  using Kern = void (*)(StreamBatch);
+  const Kern kern = hp8 ? (mma ? (Kern)k_decode_stream<true, true> : (Kern)k_decode_stream<true, false>)
+                        : (mma ? (Kern)k_decode_stream<false, true> : (Kern)k_decode_stream<false, false>);
+  static const bool limit_set =
+      cudaFuncSetAttribute(k_decode_stream<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStreamSmemLimit) == cudaSuccess &&
+      cudaFuncSetAttribute(k_decode_stream<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStreamSmemLimit) == cudaSuccess &&
+      cudaFuncSetAttribute(k_decode_stream<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStreamSmemLimit) == cudaSuccess &&
+      cudaFuncSetAttribute(k_decode_stream<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStreamSmemLimit) == cudaSuccess;
   if (!limit_set) return PQ_ERR_CUDA;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeCooperative;
@@ -1079,7 +1104,7 @@ int decode_stream_launch(const DecodeItemArgs* items, int n, cudaStream_t st) {
   cfg.stream = st; cfg.attrs = attr; cfg.numAttrs = 1;
   cfg.gridDim = dim3(nC, 1, 1); cfg.blockDim = dim3(kStreamThreads, 1, 1); cfg.dynamicSmemBytes = smem;
   LaunchScope ls(KID_DECODE_STREAM, st);
-  if (cudaLaunchKernelEx(&cfg, k_decode_stream, bp) != cudaSuccess) return PQ_ERR_CUDA;
+  if (cudaLaunchKernelEx(&cfg, kern, bp) != cudaSuccess) return PQ_ERR_CUDA;
   return PQ_OK;
 }
 
