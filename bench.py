@@ -883,6 +883,7 @@ def main():
     ap.add_argument("--decode-kernels", default="auto", choices=["auto", "stream", "pair"],
                     help="auto: the library picks per launch group; stream: the cooperative streaming kernel wherever the items allow; "
                          "pair: the two-kernel path on the plain layout")
+    ap.add_argument("--decode-interleave", type=int, default=1, choices=[0, 1, 2], help="streaming decode kernel: side-by-side walk of its two work lists (0 never, 1 auto, 2 always)")
     ap.add_argument("--decode-hp8", action="store_true", help="decode with the INT8 high-precision branch (int8 experts: half the expert bytes)")
     ap.add_argument("--decode-mma-from", type=int, default=5, help="streaming decode kernel: token groups of at least this size use the tensor-core bit product")
     ap.add_argument("--decode-prefetch", type=int, default=1, choices=[0, 1], help="streaming decode kernel: L2 prefetch of the sign bits during the token work")
@@ -903,6 +904,7 @@ def main():
     ctx = Ctx()
     ctx.decode_kernels = args.decode_kernels
     ctx.decode_hp8 = args.decode_hp8
+    ctx.pqb.pq_set_option(ctx.pqb.PQ_OPT_DECODE_INTERLEAVE, args.decode_interleave)
     ctx.pqb.pq_set_option(ctx.pqb.PQ_OPT_DECODE_STREAM, {"auto": 1, "stream": 2, "pair": 0}[args.decode_kernels])
     ctx.pqb.pq_set_option(ctx.pqb.PQ_OPT_DECODE_PREFETCH, args.decode_prefetch)
     ctx.pqb.pq_set_option(ctx.pqb.PQ_OPT_DECODE_MMA_FROM, args.decode_mma_from)

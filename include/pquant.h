@@ -402,9 +402,11 @@ int pq_device_status(void* stream, int* code, int* where);
  *   PQ_OPT_DECODE_PREFETCH (default 1): the streaming decode kernel asks for the sign bits four chunks ahead of its
  *   bit product to be brought into L2.
  *   PQ_OPT_DECODE_MMA_FROM (default 5): the streaming decode kernel multiplies the sign bits of a group of at least this
- *   many tokens on the tensor cores (mma.sync u8 x s8) and of fewer tokens with dp4a; both are exact.  17 = dp4a only. */
+ *   many tokens on the tensor cores (mma.sync u8 x s8) and of fewer tokens with dp4a; both are exact.  17 = dp4a only.
+ *   PQ_OPT_DECODE_INTERLEAVE (default 1): the streaming decode kernel lets the two halves of a CTA walk the sign bits and
+ *   the expert products side by side.  1 = where it measured faster (no linear of the launch has more than eight tokens); 2 = always; 0 = never. */
 enum { PQ_OPT_DECODE_PDL = 1, PQ_OPT_SIDE_STREAM = 2, PQ_OPT_SPIN_CYCLES = 3, PQ_OPT_DECODE_STREAM = 4, PQ_OPT_DECODE_PREFETCH = 5,
-       PQ_OPT_DECODE_MMA_FROM = 6 };
+       PQ_OPT_DECODE_MMA_FROM = 6, PQ_OPT_DECODE_INTERLEAVE = 7 };
 int pq_set_option(int option, int value);
 
 /* Cumulative number of kernels this library has launched in this process. */

@@ -391,6 +391,7 @@ PQ_OPT_SPIN_CYCLES = 3
 PQ_OPT_DECODE_STREAM = 4
 PQ_OPT_DECODE_PREFETCH = 5
 PQ_OPT_DECODE_MMA_FROM = 6
+PQ_OPT_DECODE_INTERLEAVE = 7
 
 
 def pq_set_option(option: int, value: int):

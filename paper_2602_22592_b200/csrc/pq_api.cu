@@ -760,6 +760,7 @@ int pq_set_option(int option, int value) {
     case PQ_OPT_DECODE_STREAM: decode_stream_enable(value); return PQ_OK;
     case PQ_OPT_DECODE_PREFETCH: decode_stream_prefetch(value); return PQ_OK;
     case PQ_OPT_DECODE_MMA_FROM: decode_stream_mma_from(value); return PQ_OK;
+    case PQ_OPT_DECODE_INTERLEAVE: decode_stream_interleave(value); return PQ_OK;
     case PQ_OPT_SPIN_CYCLES: {
       // the limit lives in constant memory of the current device; the copy is ordered after everything
       // already enqueued there (a blocking copy), so no running kernel sees it change

@@ -77,6 +77,7 @@ struct StreamBatch {
   int bar_slot;
   int prefetch;             // chunks ahead of the bit product for which L2 prefetches are issued (0 = none)
   int mma_from;             // token groups of at least this many tokens take the tensor-core bit product
+  int interleave;           // the two halves of a CTA walk the two work lists of phase 2 side by side
   int router_rows;          // router rows that fit in shared memory beside the token
   int off_rows, off_part;   // phase 1 carve-up: [token][router rows][partial sums of h][the token's codes in natural order]
   int off_qn;
@@ -806,6 +807,9 @@ __device__ void stream_bits_mma(const StreamLinear& L, int tg, int mg, int p_lo,
 // ---------------------------------------------------------------------------
 // the kernel: grid = one CTA per SM (cooperative launch), 512 threads
 // ---------------------------------------------------------------------------
+// barrier of one group of warps of the CTA (ids 1 and 2; 0 is __syncthreads)
+__device__ __forceinline__ void stream_group_sync(int bid, int nthreads) { asm volatile("bar.sync %0, %1;" ::"r"(bid), "r"(nthreads) : "memory"); }
+
 // HP8: some linear of the launch uses the INT8 high-precision branch; MMA: some token group is large enough for the
 // tensor-core bit product.  Separate instantiations, so that the common case carries neither's registers nor code.
 template <bool HP8, bool MMA>
@@ -861,67 +865,82 @@ __global__ void __launch_bounds__(kStreamThreads, 1) k_decode_stream(const __gri
   const bool ok = stream_bar_wait(bar, &sh.ok);
 
   if (ok) {
+    // phase 2: two steps.  Alone, the whole CTA walks its chunks of sign bits, then its expert-product items.  With
+    // `interleave` the two halves of the CTA (eight warps and a named barrier each) do one of each at a time -- half 0
+    // the first half of the chunks, then the second half of the items, half 1 the other way round -- so that a list
+    // bound by instruction issue and a list bound by memory run side by side; the host turns it on where it measured faster (up to eight tokens per linear).
     uint32_t* qs = reinterpret_cast<uint32_t*>(stream_smem);
     float* hs = reinterpret_cast<float*>(stream_smem + bp.off_h);
-    DecodeTokInfo* toks = reinterpret_cast<DecodeTokInfo*>(stream_smem + bp.off_info);
-    // phase 2 (a): sign bits
-    for (int l = l_lo; l < l_hi; ++l) {
-      const StreamLinear& L = bp.lin[l];
-      const int seg_lo = max(span_lo, L.chunk0) - L.chunk0, seg_hi = min(span_hi, L.chunk0 + L.G * L.C) - L.chunk0;
-      if (seg_lo >= seg_hi) continue;
-      const int qwords = L.C * 32, qstride = qwords + 4;   // the pad spreads the tokens' rows over the banks (mma variant)
-      const int len = seg_hi - seg_lo;
-      const int p_lo = seg_lo + (int)((long long)len * warp / kStreamWarps), p_hi = seg_lo + (int)((long long)len * (warp + 1) / kStreamWarps);
-      for (int tg = 0; tg * kStreamTokenGroup < L.M; ++tg) {
-        const int mg = min(kStreamTokenGroup, L.M - tg * kStreamTokenGroup);
-        __syncthreads();   // the previous codes and token records are no longer read
-        {
-          const int row4 = qwords >> 2;
-          const uint4* from = reinterpret_cast<const uint4*>(L.qg + (long long)tg * kStreamTokenGroup * qwords);
-          for (int i = threadIdx.x; i < mg * row4; i += kStreamThreads) {
-            const int t = i / row4, j = i - t * row4;
-            reinterpret_cast<uint4*>(qs + t * qstride)[j] = __ldcg(from + i);
+    const int ngroups = bp.interleave ? 2 : 1;
+    const int gthreads = kStreamThreads / ngroups, gwarps = gthreads / 32;
+    const int grp = threadIdx.x / gthreads, gtid = threadIdx.x - grp * gthreads, gw = gtid >> 5;
+    const int bid = 1 + grp;
+    DecodeTokInfo* toks = reinterpret_cast<DecodeTokInfo*>(stream_smem + bp.off_info) + grp * kDecodeMaxTokens;
+    const int span_mid = span_lo + (span_hi - span_lo) / 2, zspan_mid = zspan_lo + (zspan_hi - zspan_lo) / 2;
+    for (int step = 0; step < 2; ++step) {
+      const bool bits_now = ngroups == 1 ? step == 0 : (grp ^ step) == 0;
+      if (bits_now) {
+        const int lo = ngroups == 1 ? span_lo : (grp == 0 ? span_lo : span_mid), hi = ngroups == 1 ? span_hi : (grp == 0 ? span_mid : span_hi);
+        for (int l = 0; l < bp.n; ++l) {
+          if (bp.chunk0[l + 1] <= lo || bp.chunk0[l] >= hi) continue;
+          const StreamLinear& L = bp.lin[l];
+          const int seg_lo = max(lo, L.chunk0) - L.chunk0, seg_hi = min(hi, bp.chunk0[l + 1]) - L.chunk0;
+          const int qwords = L.C * 32, qstride = qwords + 4;   // the pad spreads the tokens' rows over the banks (mma variant)
+          const int len = seg_hi - seg_lo;
+          const int p_lo = seg_lo + (int)((long long)len * gw / gwarps), p_hi = seg_lo + (int)((long long)len * (gw + 1) / gwarps);
+          for (int tg = 0; tg * kStreamTokenGroup < L.M; ++tg) {
+            const int mg = min(kStreamTokenGroup, L.M - tg * kStreamTokenGroup);
+            stream_group_sync(bid, gthreads);   // the previous codes and token records are no longer read
+            {
+              // written by other CTAs in phase 1: read through L2
+              const int row4 = qwords >> 2;
+              const uint4* from = reinterpret_cast<const uint4*>(L.qg + (long long)tg * kStreamTokenGroup * qwords);
+              for (int i = gtid; i < mg * row4; i += gthreads) {
+                const int t = i / row4, j = i - t * row4;
+                reinterpret_cast<uint4*>(qs + t * qstride)[j] = __ldcg(from + i);
+              }
+              if (gtid < L.M) reinterpret_cast<int4*>(toks)[gtid] = __ldcg(reinterpret_cast<const int4*>(L.info) + gtid);
+            }
+            stream_group_sync(bid, gthreads);
+            if (MMA && mg >= bp.mma_from) stream_bits_mma(L, tg, mg, p_lo, p_hi, qs, qstride, toks, bp.prefetch);
+            else if (mg == 1) stream_bits<1>(L, tg, mg, p_lo, p_hi, qs, qstride, toks, bp.prefetch);
+            else if (mg == 2) stream_bits<2>(L, tg, mg, p_lo, p_hi, qs, qstride, toks, bp.prefetch);
+            else if (mg <= 4) stream_bits<4>(L, tg, mg, p_lo, p_hi, qs, qstride, toks, bp.prefetch);
+            else stream_bits<8>(L, tg, mg, p_lo, p_hi, qs, qstride, toks, bp.prefetch);
           }
-          if (threadIdx.x < L.M) reinterpret_cast<int4*>(toks)[threadIdx.x] = __ldcg(reinterpret_cast<const int4*>(L.info) + threadIdx.x);
         }
-        __syncthreads();
-        if (MMA && mg >= bp.mma_from) stream_bits_mma(L, tg, mg, p_lo, p_hi, qs, qstride, toks, bp.prefetch);
-        else if (mg == 1) stream_bits<1>(L, tg, mg, p_lo, p_hi, qs, qstride, toks, bp.prefetch);
-        else if (mg == 2) stream_bits<2>(L, tg, mg, p_lo, p_hi, qs, qstride, toks, bp.prefetch);
-        else if (mg <= 4) stream_bits<4>(L, tg, mg, p_lo, p_hi, qs, qstride, toks, bp.prefetch);
-        else stream_bits<8>(L, tg, mg, p_lo, p_hi, qs, qstride, toks, bp.prefetch);
-      }
-    }
-    // phase 2 (b): expert products.  What phase 1 wrote comes from other CTAs: read it through L2.
-    for (int l = zl_lo; l < zl_hi; ++l) {
-      const StreamLinear& L = bp.lin[l];
-      if (L.r == 0) continue;
-      const int zi = L.M * L.G * 4;
-      const int seg_lo = max(zspan_lo, L.z0) - L.z0, seg_hi = min(zspan_hi, L.z0 + zi) - L.z0;
-      if (seg_lo >= seg_hi) continue;
-      __syncthreads();
-      for (int i = threadIdx.x; i < L.M * L.r; i += kStreamThreads) hs[i] = __ldcg(L.h + i);
-      if (threadIdx.x < L.M) reinterpret_cast<int4*>(toks)[threadIdx.x] = __ldcg(reinterpret_cast<const int4*>(L.info) + threadIdx.x);
-      __syncthreads();
-      int8_t* qh8 = reinterpret_cast<int8_t*>(stream_smem + bp.off_qh);
-      float* gh = reinterpret_cast<float*>(stream_smem + bp.off_qh + kDecodeMaxTokens * 256);
-      if (HP8 && L.A8) {
-        // the hidden activation enters the second 8-bit product quantised per token from its exact integers (Eq. 7-9):
-        // gamma_h = 128 / max(max_j |fl32(h_int)|, 1e-5), code = clamp(rint(fl32(h_int) * gamma_h)); warp t takes token t
-        for (int t = warp; t < L.M; t += kStreamWarps) {
-          const int* hi = reinterpret_cast<const int*>(hs) + t * L.r;
-          const int lane = threadIdx.x & 31;
-          float amax = 0.f;
-          for (int j = lane; j < L.r; j += 32) amax = fmaxf(amax, fabsf((float)hi[j]));
-          for (int d = 16; d > 0; d >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, d));
-          const float g = __fdiv_rn(kActQmax, fmaxf(amax, kActAmaxFloor));
-          for (int j = lane; j < L.r; j += 32) qh8[t * L.r + j] = (int8_t)max(-128, min(127, __float2int_rn(__fmul_rn((float)hi[j], g))));
-          if (lane == 0) gh[t] = g;
+      } else {
+        const int lo = ngroups == 1 ? zspan_lo : (grp == 1 ? zspan_lo : zspan_mid), hi = ngroups == 1 ? zspan_hi : (grp == 1 ? zspan_mid : zspan_hi);
+        for (int l = 0; l < bp.n; ++l) {
+          if (bp.z0[l + 1] <= lo || bp.z0[l] >= hi || bp.z0[l + 1] == bp.z0[l]) continue;
+          const StreamLinear& L = bp.lin[l];
+          const int seg_lo = max(lo, L.z0) - L.z0, seg_hi = min(hi, bp.z0[l + 1]) - L.z0;
+          stream_group_sync(bid, gthreads);
+          for (int i = gtid; i < L.M * L.r; i += gthreads) hs[i] = __ldcg(L.h + i);
+          if (gtid < L.M) reinterpret_cast<int4*>(toks)[gtid] = __ldcg(reinterpret_cast<const int4*>(L.info) + gtid);
+          stream_group_sync(bid, gthreads);
+          int8_t* qh8 = reinterpret_cast<int8_t*>(stream_smem + bp.off_qh);
+          float* gh = reinterpret_cast<float*>(stream_smem + bp.off_qh + kDecodeMaxTokens * 256);
+          if (HP8 && L.A8) {
+            // the hidden activation enters the second 8-bit product quantised per token from its exact integers (Eq. 7-9):
+            // gamma_h = 128 / max(max_j |fl32(h_int)|, 1e-5), code = clamp(rint(fl32(h_int) * gamma_h)); a warp per token
+            for (int t = gw; t < L.M; t += gwarps) {
+              const int* hi32 = reinterpret_cast<const int*>(hs) + t * L.r;
+              const int lane = threadIdx.x & 31;
+              float amax = 0.f;
+              for (int j = lane; j < L.r; j += 32) amax = fmaxf(amax, fabsf((float)hi32[j]));
+              for (int d = 16; d > 0; d >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, d));
+              const float g = __fdiv_rn(kActQmax, fmaxf(amax, kActAmaxFloor));
+              for (int j = lane; j < L.r; j += 32) qh8[t * L.r + j] = (int8_t)max(-128, min(127, __float2int_rn(__fmul_rn((float)hi32[j], g))));
+              if (lane == 0) gh[t] = g;
+            }
+            stream_group_sync(bid, gthreads);
+          }
+          const int len = seg_hi - seg_lo;
+          stream_expert<HP8>(L, seg_lo + (int)((long long)len * gw / gwarps), seg_lo + (int)((long long)len * (gw + 1) / gwarps), hs, toks, qh8, gh);
         }
-        __syncthreads();
       }
-      const int len = seg_hi - seg_lo;
-      stream_expert<HP8>(L, seg_lo + (int)((long long)len * warp / kStreamWarps), seg_lo + (int)((long long)len * (warp + 1) / kStreamWarps), hs, toks, qh8, gh);
+      __syncthreads();   // the halves swap the code and h buffers (alone: the bit product's buffers are free)
     }
   }
 }
@@ -951,6 +970,8 @@ void decode_stream_view(int M, int K, int N, int r, void* ws, bool dump, int** h
 
 static int g_decode_stream_on = 1;
 static int g_decode_stream_prefetch = 1;
+static int g_decode_stream_interleave = 1;
+void decode_stream_interleave(int mode) { g_decode_stream_interleave = mode < 0 ? 0 : mode > 2 ? 2 : mode; }
 static int g_decode_stream_mma_from = 5;   // measured on the 3B shapes: dp4a is ahead up to four tokens, level at four
 void decode_stream_mma_from(int m) { g_decode_stream_mma_from = m < 1 ? 1 : m; }
 void decode_stream_enable(int mode) { g_decode_stream_on = mode < 0 ? 0 : mode > 2 ? 2 : mode; }
@@ -1074,7 +1095,7 @@ int decode_stream_launch(const DecodeItemArgs* items, int n, cudaStream_t st) {
   const size_t smem1 = bp.off_qn + xbytes / 2;          // the token's int8 codes: half the bytes of its bf16 values
   bp.off_h = (int)s_up256(codes);
   bp.off_info = (int)(bp.off_h + s_up256(hbytes));
-  bp.off_qh = bp.off_info + 256;
+  bp.off_qh = bp.off_info + 2 * kDecodeMaxTokens * (int)sizeof(DecodeTokInfo);   // one set of token records per half
   const size_t smem2 = bp.off_qh + kDecodeMaxTokens * 256 + 256;
   const size_t smem = std::max(smem1, smem2);
   if (smem > kStreamSmemLimit) return PQ_ERR_UNSUPPORTED;
@@ -1082,6 +1103,13 @@ int decode_stream_launch(const DecodeItemArgs* items, int n, cudaStream_t st) {
   if (bp.bar_slot < 0) return PQ_ERR_UNSUPPORTED;
   bp.prefetch = g_decode_stream_prefetch ? 4 : 0;
   bp.mma_from = g_decode_stream_mma_from;
+  {
+    // measured on the 3B shapes: ahead by 1-4 % at one token, 6-16 % at four, behind by 2-4 % at sixteen (two token groups
+    // walk the chunks twice, and half a CTA restages the codes for each)
+    int max_m = 1;
+    for (int i = 0; i < n; ++i) max_m = std::max(max_m, bp.lin[i].M);
+    bp.interleave = g_decode_stream_interleave > 1 || (g_decode_stream_interleave == 1 && max_m <= kStreamTokenGroup);
+  }
   bool hp8 = false, mma = false;
   for (int i = 0; i < n; ++i) {
     hp8 = hp8 || bp.lin[i].A8 != nullptr;

@@ -146,6 +146,7 @@ int decode_stream_launch(const DecodeItemArgs* items, int n, cudaStream_t st);  
 void decode_stream_enable(int mode);   // 0 never, 1 where it pays (default), 2 wherever the items allow
 void decode_stream_prefetch(int on);
 void decode_stream_mma_from(int m);
+void decode_stream_interleave(int mode);
 int decode_stream_mode();
 void decode_stream_reset();
 int decode_batch(const DecodeItemArgs* items, int n, cudaStream_t st);   // independent linears, launched together

@@ -21,7 +21,10 @@ def decode_kernels(request):
     PQLinear.stream_decode = stream
     pqb.pq_set_option(pqb.PQ_OPT_DECODE_STREAM, 2 if stream else 0)   # 2: also for one small linear
     pqb.pq_set_option(pqb.PQ_OPT_DECODE_MMA_FROM, {"stream_dp4a": 17, "stream_mma": 1}.get(request.param, 5))
+    # the forced variants also walk the two work lists side by side (two halves of a CTA), the plain one in turn
+    pqb.pq_set_option(pqb.PQ_OPT_DECODE_INTERLEAVE, 2 if request.param in ("stream_dp4a", "stream_mma") else 0)
     yield request.param
+    pqb.pq_set_option(pqb.PQ_OPT_DECODE_INTERLEAVE, 1)
     PQLinear.stream_decode = True
     pqb.pq_set_option(pqb.PQ_OPT_DECODE_STREAM, 1)
     pqb.pq_set_option(pqb.PQ_OPT_DECODE_MMA_FROM, 5)
