@@ -294,3 +294,29 @@ def test_decode_int8_hp_branch_argument_errors():
     with pytest.raises(pqb.PqError) as ei:
         pqb.pq_decode_batch(pqb.make_decode_items([tuple(entry)]))
     assert ei.value.status == pqb.PQ_ERR_NULL
+
+
+def test_decode_on_two_streams_at_once():
+    # calls on different streams may overlap on the device: each stream's launches of the streaming kernel keep grid-barrier
+    # words of their own, and every layer has its own workspace
+    layers = []
+    for i, kw in enumerate([dict(T=3, K=1024, N=2560, r=64, E=4), dict(T=1, K=2048, N=1024, r=32, E=8)]):
+        c = I.make_linear_case(kw["T"], kw["K"], kw["N"], kw["r"], kw["E"], seed=90 + i, exact_quota=False, with_grad=False)
+        L = PQLinear(c["T"], c["K"], c["N"], c["r"], c["E"], training=False, dump_acc=True).load_case(c)
+        L.pack(bits_only=True)
+        L.decode()
+        layers.append(L)
+    torch.cuda.synchronize()
+    want = [L.Y.clone() for L in layers]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    for L in layers:
+        L.Y.zero_()
+    torch.cuda.synchronize()
+    for _ in range(6):
+        for L, s in zip(layers, streams):
+            with torch.cuda.stream(s):
+                L.decode()
+    torch.cuda.synchronize()
+    check_status()
+    for L, y in zip(layers, want):
+        assert torch.equal(L.Y, y)
