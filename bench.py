@@ -34,24 +34,25 @@ import numpy as np
 METRIC = "pQuant linear fwd+bwd tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel (the dW tiles of the 2048 -> 5632
-# projection) from an ncu capture, stamped with the hash of the kernel sources it was taken from: once any source
-# changes the stamp no longer matches and the bench line reports null until the kernel is captured again.
-NCU_TRAFFIC = {"bwd_dw": {"bytes": 218562048, "sources_sha16": "d973cace158e0285"}}
+# projection) from an ncu capture, stamped with the hash of the files that kernel is compiled from (the tensor-core engine,
+# the GEMM kernels, the shared device helpers): once one of them changes the stamp no longer matches and the bench line
+# reports null until the kernel is captured again.
+NCU_TRAFFIC = {"bwd_dw": {"bytes": 218562048, "sources_sha16": "e1887889fce22bf8", "files": ("pq_gemm.cuh", "pq_gemm_kernels.cu", "pq_common.cuh")}}
 
 
-def sources_sha16() -> str:
-    """Hash of every file the library is built from."""
+def sources_sha16(files) -> str:
+    """Hash of the named files of the library's source directory."""
     from paper_2602_22592_b200 import build as pqbuild
     h = hashlib.sha256()
-    for path in pqbuild.sources():
-        with open(path, "rb") as f:
+    for name in files:
+        with open(os.path.join(pqbuild.CSRC, name), "rb") as f:
             h.update(f.read())
     return h.hexdigest()[:16]
 
 
 def ncu_traffic(kernel: str):
     rec = NCU_TRAFFIC.get(kernel)
-    return rec["bytes"] if rec and rec["sources_sha16"] == sources_sha16() else None
+    return rec["bytes"] if rec and rec["sources_sha16"] == sources_sha16(rec["files"]) else None
 
 
 def measured_peaks():

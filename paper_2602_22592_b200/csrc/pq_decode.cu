@@ -821,7 +821,10 @@ int decode_batch(const DecodeItemArgs* items, int n, cudaStream_t st) {
       if (hp8 && rc == PQ_ERR_UNSUPPORTED) return rc;        // the INT8 branch exists on the streaming kernel only
     }
     if (rc == PQ_ERR_UNSUPPORTED) {
-      m = std::min(n - i, kDecodeMaxBatch);
+      // the two-kernel path: the same run of items that carry the layout, or the run in front that does not
+      if (m == 0)
+        while (i + m < n && m < kDecodeMaxBatch && !items[i + m].bits_il) ++m;
+      m = std::min(m, kDecodeMaxBatch);
       for (int k = 0; k < m; ++k)
         if (items[i + k].A8) return PQ_ERR_UNSUPPORTED;
       rc = decode_launch(items + i, m, st);

@@ -320,3 +320,35 @@ def test_decode_on_two_streams_at_once():
     check_status()
     for L, y in zip(layers, want):
         assert torch.equal(L.Y, y)
+
+
+def test_decode_batch_mixing_items_with_and_without_the_streaming_layout(decode_kernels):
+    # a batch whose items only partly carry the streaming kernel's weight layout is cut into runs: the runs that carry it
+    # go to the streaming kernel, the others to the two-kernel path; every item gets what a call of its own gives
+    if decode_kernels == "pair":
+        pytest.skip("needs the streaming layout")
+    shapes = [dict(T=2, K=512, N=640, r=32, E=4), dict(T=1, K=1024, N=256, r=64, E=2), dict(T=7, K=256, N=1152, r=16, E=8)]
+    layers = []
+    for i in range(9):
+        kw = shapes[i % 3]
+        c = I.make_linear_case(kw["T"], kw["K"], kw["N"], kw["r"], kw["E"], seed=120 + i, exact_quota=False, with_grad=False)
+        L = PQLinear(c["T"], c["K"], c["N"], c["r"], c["E"], training=False, dump_acc=True).load_case(c)
+        L.pack(bits_only=True)
+        L.decode()
+        layers.append(L)
+    torch.cuda.synchronize()
+    want = [L.Y.clone() for L in layers]
+    entries = []
+    for i, L in enumerate(layers):
+        e = list(L.decode_entry())
+        if i in (2, 3, 7):          # these go without the layout
+            e[13] = e[14] = None
+        entries.append(tuple(e))
+        L.Y.zero_()
+    pqb.pq_decode_batch(pqb.make_decode_items(entries))
+    torch.cuda.synchronize()
+    check_status()
+    for L, y in zip(layers, want):
+        assert rel_err(f32(L.Y), f32(y)) <= 1e-2      # the two paths sum the expert product in different orders
+    for i in (0, 1, 4, 5, 6, 8):
+        assert torch.equal(layers[i].Y, want[i])
