@@ -303,7 +303,8 @@ typedef struct pq_decode_item {
    * (PQ_OPT_DECODE_STREAM), the group runs as ONE cooperative kernel that
    * streams each weight byte once with coalesced loads; results: the same integers (codes, routing, sums over k),
    * Y within the tolerance of the float epilogue (the expert product is summed in another order).  Otherwise, and
-   * for shapes that kernel does not take (r not a multiple of 8), the two-kernel path is used.  w_bits, A and B
+   * for shapes that kernel does not take (r not a multiple of 8), the two-kernel path is used.  Items of one launch
+   * group that read the same X (same pointer, T, K and norm) are quantised once.  w_bits, A and B
    * are needed in both cases (the rows of A_e are read in their natural layout). */
   const uint32_t* w_bits_il;
   const uint16_t* B_il;

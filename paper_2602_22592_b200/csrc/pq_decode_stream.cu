@@ -54,6 +54,8 @@ struct StreamLinear {
   uint16_t* Y;              // [M, N]
   const uint16_t* norm_w;   // [K] bf16 or null
   DecodeTokInfo* info;      // [16] expert, gate, gamma, code sum per token
+  const DecodeTokInfo* info_q;  // where gamma and the code sum come from: `info`, or the record of an earlier linear of the
+                            // launch that reads the same activations (then `qg` is that linear's too and nothing is quantised here)
   uint32_t* qg;             // [M][C * 32] words of int8 codes in bit-product order
   float* h;                 // [M][r] (INT8 branch: the exact integers h_int = A8_e q, as int32)
   float* z;                 // [M][G * 128] expert product
@@ -66,6 +68,7 @@ struct StreamLinear {
   int G, C;                 // row groups; chunks per row group
   int chunk0;               // position of this linear's first chunk in the launch-wide list of chunks
   int z0;                   // position of its first item in the launch-wide list of expert-product items (M * 4 G each)
+  int share;                // 1: codes, gamma and code sum are another linear's (see info_q)
   int zero_words;           // int32 words from `acc` on that phase 1 clears (acc and cnt are adjacent)
 };
 // The descriptor travels as kernel parameters (constant memory).  What every CTA needs to find its work sits in a few
@@ -455,7 +458,7 @@ __device__ void stream_token(const StreamBatch& bp, const StreamLinear& L, int t
     else stream_h_rows<4>(a4, xs4, part, nrows, chunks, s_lo, s_hi, warp, lane);
   }
 
-  if (owner) {
+  if (owner && !L.share) {
     // Eq. 7-9; a thread turns 32 values of k into the 8 words the bit product reads: word b holds the codes of
     // k = b, b + 8, b + 16, b + 24 (the bytes that the mask 0x01010101 << b selects from a weight word)
     const int ngroups = L.C * 4;
@@ -492,8 +495,9 @@ __device__ void stream_token(const StreamBatch& bp, const StreamLinear& L, int t
   __syncthreads();   // partial sums of h and of the codes are visible
   if (owner && threadIdx.x == 0) {
     int tot = 0;
-    for (int w = 0; w < kStreamWarps; ++w) tot += sh.red_i[w];
-    L.info[t] = DecodeTokInfo{best, gate, gamma, tot};
+    if (!L.share)
+      for (int w = 0; w < kStreamWarps; ++w) tot += sh.red_i[w];
+    L.info[t] = DecodeTokInfo{best, gate, gamma, tot};   // (shared codes: the code sum is filled in from info_q in phase 2)
   }
   for (int i = threadIdx.x; i < nrows; i += kStreamThreads) {
     if (HP8 && L.A8) {
@@ -807,6 +811,19 @@ __device__ void stream_bits_mma(const StreamLinear& L, int tg, int mg, int p_lo,
 // ---------------------------------------------------------------------------
 // the kernel: grid = one CTA per SM (cooperative launch), 512 threads
 // ---------------------------------------------------------------------------
+// A token's record as phase 2 uses it: routing from the linear's own record, gamma and code sum from the linear whose
+// codes it multiplies (itself unless it shares another's activations).  Written by other CTAs: read through L2.
+__device__ __forceinline__ DecodeTokInfo stream_record(const StreamLinear& L, int t) {
+  const int4 a = __ldcg(reinterpret_cast<const int4*>(L.info) + t);
+  DecodeTokInfo r{a.x, __int_as_float(a.y), __int_as_float(a.z), a.w};
+  if (L.share) {
+    const int4 b = __ldcg(reinterpret_cast<const int4*>(L.info_q) + t);
+    r.gamma = __int_as_float(b.z);
+    r.rowsum = b.w;
+  }
+  return r;
+}
+
 // barrier of one group of warps of the CTA (ids 1 and 2; 0 is __syncthreads)
 __device__ __forceinline__ void stream_group_sync(int bid, int nthreads) { asm volatile("bar.sync %0, %1;" ::"r"(bid), "r"(nthreads) : "memory"); }
 
@@ -899,7 +916,10 @@ __global__ void __launch_bounds__(kStreamThreads, 1) k_decode_stream(const __gri
                 const int t = i / row4, j = i - t * row4;
                 reinterpret_cast<uint4*>(qs + t * qstride)[j] = __ldcg(from + i);
               }
-              if (gtid < L.M) reinterpret_cast<int4*>(toks)[gtid] = __ldcg(reinterpret_cast<const int4*>(L.info) + gtid);
+              if (gtid < L.M) {
+                toks[gtid] = stream_record(L, gtid);
+                if (L.share && seg_lo == 0 && tg == 0) L.info[gtid] = toks[gtid];   // complete the record for the decode view
+              }
             }
             stream_group_sync(bid, gthreads);
             if (MMA && mg >= bp.mma_from) stream_bits_mma(L, tg, mg, p_lo, p_hi, qs, qstride, toks, bp.prefetch);
@@ -917,7 +937,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) k_decode_stream(const __gri
           const int seg_lo = max(lo, L.z0) - L.z0, seg_hi = min(hi, bp.z0[l + 1]) - L.z0;
           stream_group_sync(bid, gthreads);
           for (int i = gtid; i < L.M * L.r; i += gthreads) hs[i] = __ldcg(L.h + i);
-          if (gtid < L.M) reinterpret_cast<int4*>(toks)[gtid] = __ldcg(reinterpret_cast<const int4*>(L.info) + gtid);
+          if (gtid < L.M) toks[gtid] = stream_record(L, gtid);
           stream_group_sync(bid, gthreads);
           int8_t* qh8 = reinterpret_cast<int8_t*>(stream_smem + bp.off_qh);
           float* gh = reinterpret_cast<float*>(stream_smem + bp.off_qh + kDecodeMaxTokens * 256);
@@ -1037,6 +1057,16 @@ int decode_stream_launch(const DecodeItemArgs* items, int n, cudaStream_t st) {
     L.zero_words = M * L.G * 128 + groups * L.G;
     w += s_up256((size_t)L.zero_words * 4);
     L.zint_dump = (it.dump && it.A8) ? reinterpret_cast<int*>(w) : nullptr;
+    // N1 (App. A, "without redundant data reads"): a linear that reads the same activations as an earlier one of the
+    // launch (gate and up of a block, q / k / v) multiplies that linear's codes instead of quantising again
+    L.info_q = L.info; L.share = 0;
+    for (int j = 0; j < i; ++j) {
+      const DecodeItemArgs& o = items[j];
+      if (o.X == it.X && o.a.T == M && o.a.K == K && o.norm_weight == it.norm_weight && o.norm_eps == it.norm_eps && !bp.lin[j].share) {
+        L.qg = bp.lin[j].qg; L.info_q = bp.lin[j].info; L.share = 1;
+        break;
+      }
+    }
     L.chunk0 = (int)total;
     total += (long long)L.G * L.C;
     L.z0 = (int)total_z;

@@ -352,3 +352,32 @@ def test_decode_batch_mixing_items_with_and_without_the_streaming_layout(decode_
         assert rel_err(f32(L.Y), f32(y)) <= 1e-2      # the two paths sum the expert product in different orders
     for i in (0, 1, 4, 5, 6, 8):
         assert torch.equal(layers[i].Y, want[i])
+
+
+def test_decode_batch_items_that_share_their_activations(decode_kernels):
+    # gate and up of a block (or q / k / v) read the same X: in one batch the streaming kernel quantises it once and the
+    # later items multiply the first one's codes (App. A, no redundant reads).  Every item still gets exactly what a call
+    # of its own gives, and its record (gamma, code sum) in its own workspace.
+    shapes = [dict(T=3, K=1024, N=2560, r=64, E=4), dict(T=3, K=1024, N=640, r=32, E=8), dict(T=3, K=1024, N=1152, r=0, E=0)]
+    layers, cases = [], []
+    for i, kw in enumerate(shapes):
+        c = I.make_linear_case(kw["T"], kw["K"], kw["N"], kw["r"], kw["E"], seed=140 + i, exact_quota=False, with_grad=False)
+        L = PQLinear(c["T"], c["K"], c["N"], c["r"], c["E"], training=False, dump_acc=True).load_case(c)
+        if i > 0:
+            L.X = layers[0].X                     # the same tensor, not a copy
+            c["X"] = cases[0]["X"]
+        L.pack(bits_only=True)
+        L.decode()
+        layers.append(L)
+        cases.append(c)
+    torch.cuda.synchronize()
+    want = [L.Y.clone() for L in layers]
+    for L in layers:
+        L.Y.zero_()
+        L.ws_decode.zero_()
+    pqb.pq_decode_batch(pqb.make_decode_items([L.decode_entry() for L in layers]))
+    torch.cuda.synchronize()
+    check_status()
+    for L, y, c in zip(layers, want, cases):
+        assert torch.equal(L.Y, y)
+        check_decode(c, L)
