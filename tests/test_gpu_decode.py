@@ -62,6 +62,7 @@ DECODE_CASES = {
     "m9_dense_hp": dict(T=9, K=384, N=320, r=160, E=1),
     "m3_pure_1bit": dict(T=3, K=1024, N=64, r=0, E=0),
     "m12_vector_scales": dict(T=12, K=320, N=4736, r=16, E=2, scale_vector=True, alpha=1.5, beta=0.4),
+    "m2_widest_hp": dict(T=2, K=512, N=288, r=256, E=2),           # the widest branch the decode path takes
 }
 
 
@@ -247,7 +248,7 @@ def test_decode_rejects_too_many_tokens():
 
 
 @pytest.mark.parametrize("shape", [dict(T=1, K=256, N=96, r=32, E=4), dict(T=16, K=512, N=2048, r=64, E=8), dict(T=9, K=384, N=320, r=160, E=1),
-                                   dict(T=5, K=2080, N=992, r=48, E=3), dict(T=1, K=3200, N=8640, r=160, E=8),
+                                   dict(T=5, K=2080, N=992, r=48, E=3), dict(T=2, K=512, N=288, r=256, E=2), dict(T=1, K=3200, N=8640, r=160, E=8),
                                    dict(T=4, K=8640, N=3200, r=160, E=8)])
 def test_decode_int8_hp_branch_matches_oracle(shape):
     # Sec. 3.2 on the decode path: the branch multiplies the token's int8 codes by int8 expert matrices; every integer it
