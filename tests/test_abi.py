@@ -39,6 +39,37 @@ def test_struct_layout_matches_header(lib):
     assert d.size == 32 and d.flags == lib.PQ_SCALE_VECTOR
 
 
+def test_every_struct_of_the_header_has_the_same_layout_in_the_binding(lib, tmp_path):
+    # the header compiled as plain C (it has to be: the boundary is a C ABI) prints size and field offsets of each struct;
+    # the ctypes mirrors must agree field by field
+    structs = {"pq_desc": lib.pq_desc, "pq_decode_item": lib.pq_decode_item, "pq_decode_view": lib.pq_decode_view,
+               "pq_ffn_desc": lib.pq_ffn_desc, "pq_ffn_view": lib.pq_ffn_view, "pq_bwd_view": lib.pq_bwd_view}
+    lines = ["#include <stdio.h>", "#include <stddef.h>", '#include "pquant.h"', "int main(void) {"]
+    for name, cls in structs.items():
+        lines.append(f'  printf("{name} sizeof %zu\\n", sizeof({name}));')
+        for field, _ in cls._fields_:
+            lines.append(f'  printf("{name} {field} %zu\\n", offsetof({name}, {field}));')
+    lines += ["  return 0;", "}"]
+    src = tmp_path / "layout.c"
+    src.write_text("\n".join(lines))
+    exe = tmp_path / "layout"
+    import subprocess
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)], check=True)
+    out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split("\n")
+    seen = 0
+    for line in out:
+        if not line:
+            continue
+        name, field, value = line.split()
+        cls = structs[name]
+        if field == "sizeof":
+            assert ctypes.sizeof(cls) == int(value), name
+        else:
+            assert getattr(cls, field).offset == int(value), f"{name}.{field}"
+        seen += 1
+    assert seen == sum(1 + len(c._fields_) for c in structs.values())
+
+
 def test_status_strings(lib):
     assert lib.pq_status_string(0) == "ok"
     for s in range(-7, 0):
